@@ -1,0 +1,390 @@
+/*
+ * CPU oracle for the CASK compression event -- TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, double-precision restatement of what one compression event
+ * computes for one unit (one sequence x layer x KV head).  It is used by the
+ * tests, the smoke check and the benchmark's cpu_baseline leg to judge the
+ * CUDA library; it shares no code with that library and the library never
+ * calls it.  No blocking, fusion or reordering: every function walks the
+ * definition it cites so it can be checked against the paper by eye.
+ *
+ * Where the paper states a formula the function cites it.  Where the paper is
+ * silent the reading taken here is listed beside the function ("reading:");
+ * those choices (score form, gamma, tau, eps, reserve, seed rule) are fixed by
+ * this project's written definition, not by the paper: for them parity with
+ * the paper itself is "parity unpinned".
+ *
+ * Inputs are the cache values as float (bf16 or fp32 values, promoted exactly
+ * to double).  Row kinds: 0 dropped, 1 kept prefix, 2 recent, 3 core, 4 seed
+ * (representative anchor), 5 merged into a seed's group.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+enum {
+    ORC_NOOP_UNDER_BUDGET = 1,
+    ORC_PREFIX_EVICTED = 2,
+    ORC_DECODE_CONSOLIDATED = 4,
+    ORC_PREFIX_BUDGET_EXHAUSTED = 8,
+    ORC_MERGE_INACTIVE = 16
+};
+
+enum { PL_BP = 0, PL_PKEEP, PL_BD, PL_R, PL_C, PL_M, PL_FLAGS, PL_NOUT };
+
+/* ---- total order used by every selection: score descending, row ascending ---- */
+typedef struct { double s; int i; } orc_item;
+
+static int orc_cmp(const void* a, const void* b) {
+    const orc_item* x = (const orc_item*)a;
+    const orc_item* y = (const orc_item*)b;
+    if (x->s > y->s) return -1;
+    if (x->s < y->s) return 1;
+    return (x->i > y->i) - (x->i < y->i);
+}
+
+/*
+ * Score (Sec. 1 "assign scalar importance to each token"; the deployed scorer
+ * has no formula in the paper -- reading: windowed attention mass).
+ * For query head h < g and window position j < W, with the window query j
+ * sitting at cache row T-W+j:
+ *     x_hji = <q_hj, k_i> / sqrt(d)
+ *     key i is visible to query j  iff  i <= T-W+j      (causal != 0; else all)
+ *     lse_hj = log sum_{visible i} exp(x_hji)
+ *     p_hji  = exp(x_hji - lse_hj) on visible keys, 0 elsewhere
+ *     s_i    = (1/(g W)) sum_{h,j} p_hji
+ * lse_in (nullable, [g*W]) replaces the computed normaliser.
+ */
+void cask_oracle_score(const float* K, const float* Q, int T, int d, int g, int W, int causal,
+                       const double* lse_in, double* s, double* lse_out) {
+    double* x = (double*)malloc(sizeof(double) * (size_t)(T > 0 ? T : 1));
+    const double inv_sqrt_d = 1.0 / sqrt((double)d);
+    for (int i = 0; i < T; ++i) s[i] = 0.0;
+    for (int h = 0; h < g; ++h) {
+        for (int j = 0; j < W; ++j) {
+            const float* q = Q + ((size_t)h * W + j) * d;
+            int nvis = causal ? (T - W + j + 1) : T;
+            if (nvis > T) nvis = T;
+            if (nvis < 0) nvis = 0;
+            double mx = -INFINITY;
+            for (int i = 0; i < nvis; ++i) {
+                const float* k = K + (size_t)i * d;
+                double acc = 0.0;
+                for (int c = 0; c < d; ++c) acc += (double)q[c] * (double)k[c];
+                x[i] = acc * inv_sqrt_d;
+                if (x[i] > mx) mx = x[i];
+            }
+            double lse;
+            if (lse_in) {
+                lse = lse_in[h * W + j];
+            } else {
+                double z = 0.0;
+                for (int i = 0; i < nvis; ++i) z += exp(x[i] - mx);
+                lse = (nvis > 0) ? mx + log(z) : 0.0;
+            }
+            if (lse_out) lse_out[h * W + j] = lse;
+            for (int i = 0; i < nvis; ++i) s[i] += exp(x[i] - lse);
+        }
+    }
+    const double inv_rows = 1.0 / ((double)g * (double)W);
+    for (int i = 0; i < T; ++i) s[i] *= inv_rows;
+    free(x);
+}
+
+/*
+ * Budget split (Sec. 2.2: Stage 1 evicts the prefix "to secure slack for the
+ * decode stage"; Sec. 2.3: |R| <= B, C subset of R, scratch uses only the
+ * remaining budget; Sec. 5.2: when the prefix encroaches on the budget the
+ * available slots collapse).  Reading (the paper gives no numbers):
+ *   B_p = B - reserve;  P_keep = min(P, B_p);  B_d = B - P_keep;  N_d = T - P
+ *   T <= B            -> NOOP_UNDER_BUDGET: every row kept
+ *   r = min(W, N_d)      recent rows, always protected
+ *   N_d <= B_d        -> every decode row kept as a singleton, no merge
+ *   B_d < r + 2       -> PREFIX_BUDGET_EXHAUSTED: no room for the recent window
+ *                        plus one core slot plus one representative; keep the
+ *                        last min(r,B_d) rows and the best of the rest, no merge
+ *   else c = min(ceil(gamma (B_d - r)), B_d - r - 1),  m = B_d - r - c  (>= 1)
+ */
+void cask_oracle_plan(int T, int P, int B, int reserve, int W, double gamma, int* plan) {
+    int Nd = T - P;
+    int Bp = B - reserve;
+    int Pkeep = P < Bp ? P : Bp;
+    int Bd = B - Pkeep;
+    int r = W < Nd ? W : Nd;
+    int c = 0, m = 0, flags = 0, nout;
+    if (T <= B) {
+        flags = ORC_NOOP_UNDER_BUDGET;
+        Pkeep = P;
+        Bd = B - P;
+        c = Nd - r;
+        nout = T;
+    } else {
+        if (P > Bp) flags |= ORC_PREFIX_EVICTED;
+        if (Nd <= Bd) {
+            c = Nd - r;
+            nout = Pkeep + Nd;
+        } else if (Bd < r + 2) {
+            flags |= ORC_PREFIX_BUDGET_EXHAUSTED;
+            r = r < Bd ? r : Bd;
+            c = Bd - r;
+            nout = Pkeep + Bd;
+        } else {
+            flags |= ORC_DECODE_CONSOLIDATED;
+            int room = Bd - r;
+            c = (int)ceil(gamma * (double)room);
+            if (c > room - 1) c = room - 1;
+            if (c < 0) c = 0;
+            m = room - c;
+            nout = Pkeep + Bd;
+        }
+    }
+    plan[PL_BP] = Bp; plan[PL_PKEEP] = Pkeep; plan[PL_BD] = Bd; plan[PL_R] = r;
+    plan[PL_C] = c; plan[PL_M] = m; plan[PL_FLAGS] = flags; plan[PL_NOUT] = nout;
+}
+
+/* mark the `k` greatest rows of [lo,hi) whose kind is 0 with `mark` */
+static void orc_mark_top(const double* s, int lo, int hi, int k, uint8_t* kind, uint8_t mark) {
+    int n = 0;
+    orc_item* it = (orc_item*)malloc(sizeof(orc_item) * (size_t)(hi > lo ? hi - lo : 1));
+    for (int i = lo; i < hi; ++i)
+        if (kind[i] == 0) { it[n].s = s[i]; it[n].i = i; ++n; }
+    qsort(it, (size_t)n, sizeof(orc_item), orc_cmp);
+    if (k > n) k = n;
+    for (int t = 0; t < k; ++t) kind[it[t].i] = mark;
+    free(it);
+}
+
+/*
+ * Stage 1, prefix eviction (Sec. 2.2).  If the prefix exceeds its share keep
+ * its P_keep greatest rows under the total order; otherwise keep all of it.
+ * Writes kind[0:P] (1 kept, 0 evicted).
+ */
+void cask_oracle_prefix_evict(const double* s, int P, const int* plan, uint8_t* kind) {
+    for (int i = 0; i < P; ++i) kind[i] = 0;
+    if (P <= plan[PL_PKEEP]) {
+        for (int i = 0; i < P; ++i) kind[i] = 1;
+    } else {
+        orc_mark_top(s, 0, P, plan[PL_PKEEP], kind, 1);
+    }
+}
+
+/*
+ * Protected core (Sec. 2.1: answer formation / state anchoring -> highest
+ * score; "recent reasoning pivots" -> recency).  recent = rows [T-r, T);
+ * core = the c greatest rows of [P, T-r).  Writes kind[P:T] (2, 3, else 0).
+ */
+void cask_oracle_select_core(const double* s, int T, int P, const int* plan, uint8_t* kind) {
+    int r = plan[PL_R], c = plan[PL_C];
+    for (int i = P; i < T; ++i) kind[i] = 0;
+    for (int i = T - r; i < T; ++i) kind[i] = 2;
+    orc_mark_top(s, P, T - r, c, kind, 3);
+}
+
+/*
+ * Scratch consolidation (Sec. 2.1 "representative construction only on this
+ * part"; Sec. 2.4 m-folding; Sec. 2.5 cosine as the base merge geometry).
+ * Scratch S = rows of [P, T-r) with kind 0.  Reading: the m greatest rows of S
+ * become seeds; every other j in S goes to the seed with the largest cosine
+ * similarity of keys (ties: smallest seed row; a zero-norm row has similarity
+ * 0) if that similarity is >= tau, else it is dropped and its a_j counts as
+ * lost mass (the |Delta m_G| term of Sec. 2.6).  Merge weights (Sec. 2.4):
+ *     a_i = s_i + eps,  m_G = sum_{i in G} a_i,  w_i = a_i / m_G.
+ * Outputs: kind (adds 4 seed, 5 merged), seed_of (row of the group's seed, -1),
+ * weight (w_i for group members, untouched elsewhere), sim / sim2 (best and
+ * second-best similarity of each non-seed scratch row; -2 where undefined).
+ * Returns flags to OR into the unit's status (MERGE_INACTIVE if nobody joins).
+ */
+int cask_oracle_consolidate(const float* K, const double* s, int T, int P, int d, const int* plan,
+                            double tau, double eps, uint8_t* kind, int* seed_of, double* weight,
+                            double* sim, double* sim2, double* lost_mass) {
+    int r = plan[PL_R], m = plan[PL_M];
+    for (int i = 0; i < T; ++i) { seed_of[i] = -1; if (sim) sim[i] = -2.0; if (sim2) sim2[i] = -2.0; }
+    *lost_mass = 0.0;
+    if (m <= 0) return 0;
+    orc_mark_top(s, P, T - r, m, kind, 4);
+    int* seeds = (int*)malloc(sizeof(int) * (size_t)m);
+    double* snorm = (double*)malloc(sizeof(double) * (size_t)m);
+    int ns = 0;
+    for (int i = P; i < T - r; ++i)
+        if (kind[i] == 4) {
+            seeds[ns] = i;
+            double n2 = 0.0;
+            for (int c = 0; c < d; ++c) n2 += (double)K[(size_t)i * d + c] * (double)K[(size_t)i * d + c];
+            snorm[ns] = sqrt(n2);
+            seed_of[i] = i;
+            ++ns;
+        }
+    int joined = 0;
+    for (int j = P; j < T - r; ++j) {
+        if (kind[j] != 0) continue;
+        const float* kj = K + (size_t)j * d;
+        double n2 = 0.0;
+        for (int c = 0; c < d; ++c) n2 += (double)kj[c] * (double)kj[c];
+        double nj = sqrt(n2);
+        double best = -INFINITY, second = -INFINITY;
+        int best_u = -1;
+        for (int u = 0; u < ns; ++u) {           /* seeds[] ascends, so '>' keeps the smallest row on ties */
+            const float* ku = K + (size_t)seeds[u] * d;
+            double dot = 0.0;
+            for (int c = 0; c < d; ++c) dot += (double)kj[c] * (double)ku[c];
+            double sm = (nj > 0.0 && snorm[u] > 0.0) ? dot / (nj * snorm[u]) : 0.0;
+            if (sm > best) { second = best; best = sm; best_u = u; }
+            else if (sm > second) second = sm;
+        }
+        if (sim) sim[j] = best;
+        if (sim2) sim2[j] = (ns > 1) ? second : -2.0;
+        if (best_u >= 0 && best >= tau) {
+            kind[j] = 5;
+            seed_of[j] = seeds[best_u];
+            ++joined;
+        } else {
+            *lost_mass += s[j] + eps;
+        }
+    }
+    for (int u = 0; u < ns; ++u) {
+        double mG = 0.0;
+        for (int i = P; i < T - r; ++i)
+            if (seed_of[i] == seeds[u]) mG += s[i] + eps;
+        for (int i = P; i < T - r; ++i)
+            if (seed_of[i] == seeds[u]) weight[i] = (s[i] + eps) / mG;
+    }
+    free(seeds);
+    free(snorm);
+    return joined == 0 ? ORC_MERGE_INACTIVE : 0;
+}
+
+/*
+ * Compaction (Sec. 2.3: |R| <= B).  Output slots are the rows of kind 1..4 in
+ * ascending row order; a representative sits at its seed's row.  A slot of
+ * kind 4 holds k~ = sum_i w_i k_i, v~ = sum_i w_i v_i over its group (Sec. 2.4);
+ * every other slot is a copy of its row.  slot_mass = sum of a_i over the
+ * slot's members.  assign[i] = slot of row i's anchor or -1; weight of kept
+ * singletons is set to 1 and of dropped rows to 0.
+ */
+void cask_oracle_compact(const float* K, const float* V, int T, int d, const uint8_t* kind,
+                         const int* seed_of, double* weight, const double* s, double eps,
+                         double* k_out, double* v_out, int* n_out, int* slot_src, uint8_t* slot_kind,
+                         double* slot_mass, int* assign) {
+    int n = 0;
+    for (int i = 0; i < T; ++i) {
+        assign[i] = -1;
+        if (kind[i] >= 1 && kind[i] <= 4) {
+            slot_src[n] = i;
+            slot_kind[n] = kind[i];
+            assign[i] = n;
+            ++n;
+        }
+    }
+    *n_out = n;
+    for (int i = 0; i < T; ++i) {
+        if (kind[i] == 5) assign[i] = assign[seed_of[i]];
+        if (kind[i] >= 1 && kind[i] <= 3) weight[i] = 1.0;
+        if (kind[i] == 0) weight[i] = 0.0;
+    }
+    for (int t = 0; t < n; ++t) {
+        int src = slot_src[t];
+        double* ko = k_out + (size_t)t * d;
+        double* vo = v_out + (size_t)t * d;
+        if (slot_kind[t] != 4) {
+            for (int c = 0; c < d; ++c) { ko[c] = K[(size_t)src * d + c]; vo[c] = V[(size_t)src * d + c]; }
+            slot_mass[t] = s[src] + eps;
+        } else {
+            double mass = 0.0;
+            for (int c = 0; c < d; ++c) { ko[c] = 0.0; vo[c] = 0.0; }
+            for (int i = 0; i < T; ++i) {
+                if (seed_of[i] != src || (kind[i] != 4 && kind[i] != 5)) continue;
+                mass += s[i] + eps;
+                for (int c = 0; c < d; ++c) {
+                    ko[c] += weight[i] * (double)K[(size_t)i * d + c];
+                    vo[c] += weight[i] * (double)V[(size_t)i * d + c];
+                }
+            }
+            slot_mass[t] = mass;
+        }
+    }
+}
+
+/* The whole event for one unit, the steps above in order.  plan[8] is written. */
+void cask_oracle_event(const float* K, const float* V, const float* Q, int T, int P, int B, int reserve,
+                       int d, int g, int W, int causal, double gamma, double tau, double eps,
+                       const double* lse_in, double* s, int* plan, uint8_t* kind, int* seed_of,
+                       double* weight, double* sim, double* sim2, double* k_out, double* v_out,
+                       int* n_out, int* slot_src, uint8_t* slot_kind, double* slot_mass, int* assign,
+                       int* status, double* lost_mass) {
+    cask_oracle_score(K, Q, T, d, g, W, causal, lse_in, s, NULL);
+    cask_oracle_plan(T, P, B, reserve, W, gamma, plan);
+    for (int i = 0; i < T; ++i) weight[i] = 0.0;
+    cask_oracle_prefix_evict(s, P, plan, kind);
+    cask_oracle_select_core(s, T, P, plan, kind);
+    int fl = cask_oracle_consolidate(K, s, T, P, d, plan, tau, eps, kind, seed_of, weight, sim, sim2,
+                                     lost_mass);
+    if (!(plan[PL_FLAGS] & ORC_DECODE_CONSOLIDATED)) fl = 0;
+    cask_oracle_compact(K, V, T, d, kind, seed_of, weight, s, eps, k_out, v_out, n_out, slot_src,
+                        slot_kind, slot_mass, assign);
+    *status = plan[PL_FLAGS] | fl;
+}
+
+/*
+ * Many independent units (Sec. 2.3 constrains one cache at a time; nothing
+ * couples units), rows contiguous: unit u owns rows [tok_off[u], tok_off[u+1])
+ * of K, V and of every per-row output, slots [u*Bmax, (u+1)*Bmax) of the slot
+ * outputs, and Q[u].  OpenMP runs units in parallel when compiled with it.
+ */
+void cask_oracle_event_batch(int n_units, const float* K, const float* V, const float* Q,
+                             const int64_t* tok_off, const int* P, const int* B, const int* reserve,
+                             int d, int g, int W, int causal, double gamma, double tau, double eps,
+                             int Bmax, double* s, int* plan, uint8_t* kind, int* seed_of, double* weight,
+                             double* sim, double* sim2, double* k_out, double* v_out, int* n_out,
+                             int* slot_src, uint8_t* slot_kind, double* slot_mass, int* assign,
+                             int* status, double* lost_mass) {
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1)
+#endif
+    for (int u = 0; u < n_units; ++u) {
+        size_t a = (size_t)tok_off[u];
+        int T = (int)(tok_off[u + 1] - tok_off[u]);
+        size_t so = (size_t)u * (size_t)Bmax;
+        cask_oracle_event(K + a * d, V + a * d, Q + (size_t)u * g * W * d, T, P[u], B[u], reserve[u], d, g,
+                          W, causal, gamma, tau, eps, NULL, s + a, plan + (size_t)u * 8, kind + a,
+                          seed_of + a, weight + a, sim ? sim + a : NULL, sim2 ? sim2 + a : NULL,
+                          k_out + so * d, v_out + so * d, n_out + u, slot_src + so, slot_kind + so,
+                          slot_mass + so, assign + a, status + u, lost_mass + u);
+    }
+}
+
+/* Scores only, many units (used where only the dominant step is timed or compared). */
+void cask_oracle_score_batch(int n_units, const float* K, const float* Q, const int64_t* tok_off, int d,
+                             int g, int W, int causal, double* s, double* lse_out) {
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1)
+#endif
+    for (int u = 0; u < n_units; ++u) {
+        size_t a = (size_t)tok_off[u];
+        int T = (int)(tok_off[u + 1] - tok_off[u]);
+        cask_oracle_score(K + a * d, Q + (size_t)u * g * W * d, T, d, g, W, causal, NULL, s + a,
+                          lse_out ? lse_out + (size_t)u * g * W : NULL);
+    }
+}
+
+/* Round doubles to the nearest bfloat16 value (ties to even), returned as float. */
+void cask_oracle_round_bf16(const double* x, size_t n, float* out) {
+    for (size_t i = 0; i < n; ++i) {
+        double v = x[i];
+        if (v == 0.0 || !isfinite(v)) { out[i] = (float)v; continue; }
+        int e;
+        frexp(v, &e);                 /* |v| in [2^(e-1), 2^e) */
+        int q = e - 8;                /* 8 significant bits */
+        if (q < -133) q = -133;       /* bf16 subnormal quantum */
+        out[i] = (float)ldexp(nearbyint(ldexp(v, -q)), q);
+    }
+}
+
+int cask_oracle_threads(void) {
+#ifdef _OPENMP
+    extern int omp_get_max_threads(void);
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

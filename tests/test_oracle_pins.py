@@ -1,0 +1,372 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, independent of the oracle's own code.
+
+Each test names the passage it leans on.  None of them needs a GPU.
+"""
+import itertools
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import cask_oracle as orc
+from paper_2604_10900_b200 import workloads as wl
+
+import bruteforce_event as bf
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rand_unit(rng, T, d, g, W):
+    K = rng.standard_normal((T, d)).astype(np.float32)
+    V = rng.standard_normal((T, d)).astype(np.float32)
+    Q = rng.standard_normal((g, W, d)).astype(np.float32)
+    return K, V, Q
+
+
+# ---- score -----------------------------------------------------------------
+
+def test_score_is_a_distribution():
+    """Mean of softmax rows: s_i >= 0 and sum_i s_i = 1 (softmax, by construction)."""
+    rng = np.random.default_rng(1)
+    for T, d, g, W in [(40, 8, 2, 5), (257, 64, 4, 16), (33, 16, 1, 33)]:
+        K, _, Q = _rand_unit(rng, T, d, g, W)
+        for causal in (0, 1):
+            s, _ = orc.score(K, Q, causal=causal)
+            assert (s >= 0).all()
+            assert abs(s.sum() - 1.0) < 1e-12
+
+
+def test_score_reduces_to_library_softmax():
+    """W = 1, g = 1, non-causal: s = softmax(q K^T / sqrt(d)), checked against torch's CPU softmax."""
+    import torch
+    rng = np.random.default_rng(2)
+    K, _, Q = _rand_unit(rng, 300, 32, 1, 1)
+    s, lse = orc.score(K, Q, causal=0)
+    x = torch.from_numpy(K.astype(np.float64)) @ torch.from_numpy(Q[0, 0].astype(np.float64)) / math.sqrt(32)
+    ref = torch.softmax(x, dim=0).numpy()
+    assert np.allclose(s, ref, rtol=1e-12, atol=1e-15)
+    assert abs(lse[0, 0] - torch.logsumexp(x, 0).item()) < 1e-12
+
+
+def test_score_multi_row_against_library_softmax_with_mask():
+    """g, W > 1 causal: the same thing written with a masked library softmax (mask: key i <= T-W+j)."""
+    import torch
+    rng = np.random.default_rng(3)
+    T, d, g, W = 90, 16, 3, 7
+    K, _, Q = _rand_unit(rng, T, d, g, W)
+    s, _ = orc.score(K, Q, causal=1)
+    x = torch.einsum("hjc,ic->hji", torch.from_numpy(Q).double(), torch.from_numpy(K).double()) / math.sqrt(d)
+    i = torch.arange(T)[None, None, :]
+    j = torch.arange(W)[None, :, None]
+    x = x.masked_fill(i > T - W + j, float("-inf"))
+    ref = torch.softmax(x, dim=-1).mean(dim=(0, 1)).numpy()
+    assert np.allclose(s, ref, rtol=1e-12, atol=1e-15)
+
+
+def test_score_identical_keys_closed_form_golden():
+    """All keys equal: every visible key gets 1/(number visible); hand-worked fixture."""
+    g_ = json.load(open(os.path.join(GOLD, "identical_keys_score.json")))
+    T, W, g = g_["T"], g_["W"], g_["g"]
+    K = np.tile(np.array([[0.5, -1.25, 2.0]], np.float32), (T, 1))
+    Q = np.random.default_rng(4).standard_normal((g, W, 3)).astype(np.float32)
+    s, _ = orc.score(K, Q, causal=1)
+    ref = np.array(g_["s_num"], np.float64) / g_["s_den"]
+    assert np.allclose(s, ref, rtol=1e-13)
+
+
+def test_score_identical_keys_closed_form_general():
+    T, W, g, d = 57, 9, 2, 4
+    K = np.tile(np.array([[1.0, 2.0, -3.0, 0.25]], np.float32), (T, 1))
+    Q = np.random.default_rng(5).standard_normal((g, W, d)).astype(np.float32)
+    s, _ = orc.score(K, Q, causal=1)
+    ref = np.array([sum(1.0 / (T - W + j + 1) for j in range(W) if i <= T - W + j) / W for i in range(T)])
+    assert np.allclose(s, ref, rtol=1e-12)
+
+
+def test_score_supplied_lse_matches_computed():
+    rng = np.random.default_rng(6)
+    K, _, Q = _rand_unit(rng, 120, 16, 2, 8)
+    s0, lse = orc.score(K, Q, causal=1)
+    s1, _ = orc.score(K, Q, causal=1, lse_in=lse)
+    assert np.allclose(s0, s1, rtol=1e-13)
+
+
+# ---- budget split ----------------------------------------------------------
+
+def test_budget_split_golden_table():
+    """Hand-worked rows for every benchmark shape and both sides of the exhausted boundary (Sec. 2.2, 2.3, 5.2)."""
+    tab = json.load(open(os.path.join(GOLD, "budget_split_table.json")))
+    for T, P, B, res, W, Bp, Pk, Bd, r, c, m, exh, nout in tab["rows"]:
+        pl = orc.plan(T, P, B, res, W, 0.5)
+        assert list(pl[:6]) == [Bp, Pk, Bd, r, c, m], (T, P, B, res)
+        assert bool(pl[6] & orc.PREFIX_BUDGET_EXHAUSTED) == bool(exh)
+        assert pl[7] == nout
+
+
+def test_budget_respected_exactly_everywhere():
+    """n_out = min(P,B_p) + min(N_d, B - min(P,B_p)); equals B when T > B and N_d >= B_d; identity when T <= B."""
+    for T in range(1, 15):
+        for P in range(0, T + 1):
+            for B in range(1, 16):
+                for res in range(0, B + 1):
+                    for W in (1, 2, 3, 5):
+                        if W > T:
+                            continue
+                        pl = orc.plan(T, P, B, res, W, 0.5)
+                        Nd = T - P
+                        if T <= B:
+                            assert pl[6] & orc.NOOP_UNDER_BUDGET and pl[7] == T
+                            continue
+                        Pk = min(P, B - res)
+                        want = Pk + min(Nd, B - Pk)
+                        assert pl[7] == want <= B
+                        if Nd >= B - Pk:
+                            assert pl[7] == B
+                        # slots add up: kept prefix + recent + core + reps = n_out
+                        assert pl[1] + pl[3] + pl[4] + pl[5] == pl[7]
+                        if pl[6] & orc.DECODE_CONSOLIDATED:
+                            assert pl[5] >= 1 and pl[2] >= pl[3] + 2
+                        if pl[6] & orc.PREFIX_BUDGET_EXHAUSTED:
+                            assert pl[5] == 0 and pl[2] < min(W, Nd) + 2 and Nd > pl[2]
+                        assert bool(pl[6] & orc.PREFIX_EVICTED) == (P > B - res)
+
+
+# ---- selections ------------------------------------------------------------
+
+def test_prefix_eviction_is_brute_force_top_k():
+    """Stage 1 (Sec. 2.2): evicted rows are exactly the P - B_p smallest under (score desc, row asc); untouched if P <= B_p."""
+    rng = np.random.default_rng(7)
+    for P, Bp in [(50, 20), (50, 50), (50, 70), (7, 0)]:
+        s = rng.random(P + 30)
+        s[3] = s[11] = s[12]          # exact ties resolve by row index
+        pl = np.array([Bp, min(P, Bp), 0, 0, 0, 0, 0, 0], np.int32)
+        kind = np.zeros(P + 30, np.uint8)
+        orc.prefix_evict(s, P, pl, kind)
+        order = sorted(range(P), key=lambda i: (-s[i], i))
+        want = set(order[:min(P, Bp)])
+        assert set(np.nonzero(kind[:P] == 1)[0].tolist()) == want
+        assert (kind[P:] == 0).all()
+
+
+def test_tau_above_one_is_plain_top_k_eviction():
+    """tau > 1: nothing can join, so the decode keep-set is recent + top-(c+m) of the rest (textbook top-k)."""
+    rng = np.random.default_rng(8)
+    T, P, B, res, d, g, W = 200, 40, 64, 32, 16, 2, 8
+    K, V, Q = _rand_unit(rng, T, d, g, W)
+    o = orc.event(K, V, Q, P, B, res, tau=1.5)
+    pl = o["plan"]
+    r, c, m = pl[3], pl[4], pl[5]
+    s = o["s"]
+    rest = sorted(range(P, T - r), key=lambda i: (-s[i], i))[:c + m]
+    kept_decode = set(np.nonzero(o["kind"][P:] >= 2)[0] + P)
+    assert kept_decode == set(rest) | set(range(T - r, T))
+    assert not (o["kind"] == 5).any()
+    assert o["status"] & orc.MERGE_INACTIVE
+    assert o["n_out"] == B
+
+
+# ---- core / merge invariants -------------------------------------------------
+
+def _event_tiny(head=0, **kw):
+    w = wl.WORKLOADS["tiny"]
+    k, v, q = wl.make_unit(w, 0, 0, head)
+    return (k, v, q, w), orc.event(k, v, q, w.prefix, w.budget, w.reserve, **kw)
+
+
+def test_core_is_never_merged_and_copied_bit_identically():
+    """C subset R (Sec. 2.3); the core is not a merge target (Sec. 2.1)."""
+    (k, v, q, w), o = _event_tiny()
+    for t in range(o["n_out"]):
+        src, kd = o["slot_src"][t], o["slot_kind"][t]
+        members = np.nonzero(o["assign"] == t)[0]
+        if kd in (1, 2, 3):
+            assert members.tolist() == [src]
+            assert o["weight"][src] == 1.0
+            assert np.array_equal(o["k_out"][t], k[src].astype(np.float64))
+            assert np.array_equal(o["v_out"][t], v[src].astype(np.float64))
+    # all recent rows and exactly c core rows present
+    pl = o["plan"]
+    assert (o["kind"][-pl[3]:] == 2).all()
+    assert np.count_nonzero(o["kind"] == 3) == pl[4]
+    assert np.count_nonzero(o["kind"] == 4) == pl[5]
+
+
+def test_merge_weights_and_mass():
+    """Sec. 2.4: weights of a group sum to 1, slot mass is the sum of a_i; tau = -1 loses no mass."""
+    (k, v, q, w), o = _event_tiny(tau=-1.0)
+    eps = 1e-9
+    a = o["s"] + eps
+    for t in range(o["n_out"]):
+        members = np.nonzero(o["assign"] == t)[0]
+        assert abs(o["weight"][members].sum() - 1.0) < 1e-12
+        assert abs(o["slot_mass"][t] - a[members].sum()) < 1e-15
+    scratch = (o["kind"] == 4) | (o["kind"] == 5) | ((o["kind"] == 0) & (np.arange(len(a)) >= w.prefix))
+    reps = o["slot_kind"] == 4
+    assert abs(o["slot_mass"][reps].sum() - a[scratch].sum()) < 1e-12
+    assert o["lost_mass"] == 0.0
+    assert not (o["kind"][w.prefix:] == 0).any()
+
+
+def test_lost_mass_is_dropped_scratch_mass():
+    (k, v, q, w), o = _event_tiny()
+    a = o["s"] + 1e-9
+    dropped = (o["kind"] == 0) & (np.arange(len(a)) >= w.prefix)
+    assert abs(o["lost_mass"] - a[dropped].sum()) < 1e-12
+
+
+def test_merge_rule_worked_example_golden():
+    """Sec. 2.4 equations on numbers worked by hand."""
+    g_ = json.load(open(os.path.join(GOLD, "merge_rule_worked.json")))
+    K = np.array(g_["k"], np.float32)
+    V = np.array(g_["v"], np.float32)
+    kind = np.array([4, 5], np.uint8)
+    seed_of = np.array([0, 0], np.int32)
+    o = orc.compact(K, V, kind, seed_of, np.array(g_["w"]), np.array(g_["a"]), eps=0.0)
+    assert o["n_out"] == 1
+    assert np.allclose(o["k_out"][0], g_["k_tilde"], rtol=1e-15)
+    assert np.allclose(o["v_out"][0], g_["v_tilde"], rtol=1e-15)
+    assert o["slot_mass"][0] == g_["m_G"]
+    # and the weights consolidate() derives from scores are a_i / m_G
+    K2 = np.array([[1, 0], [1, 0], [0, 1]], np.float32)         # rows 0,1 identical; row 2 is the recent row
+    s = np.array([1.0, 3.0, 0.5])
+    pl = np.array([0, 0, 2, 1, 0, 1, orc.DECODE_CONSOLIDATED, 2], np.int32)
+    kind2 = np.zeros(3, np.uint8)
+    orc.select_core(s, 3, 0, pl, kind2)
+    c = orc.consolidate(K2, s, 0, pl, kind2, tau=0.9, eps=0.0)
+    assert kind2.tolist() == [5, 4, 2]
+    assert c["seed_of"].tolist() == [1, 1, -1]
+    assert np.allclose(c["weight"][:2], [0.25, 0.75], rtol=1e-15)
+
+
+def test_representative_is_the_exact_linear_surrogate():
+    """Exact form of the diagnostic of Sec. 2.6: sum_i w_i <q,k_i> = <q,k~>; each coordinate inside the members' range."""
+    (k, v, q, w), o = _event_tiny()
+    rng = np.random.default_rng(9)
+    probe = rng.standard_normal(w.head_dim)
+    checked = 0
+    for t in np.nonzero(o["slot_kind"] == 4)[0]:
+        mem = np.nonzero(o["assign"] == t)[0]
+        if len(mem) < 2:
+            continue
+        checked += 1
+        lhs = (o["weight"][mem] * (k[mem].astype(np.float64) @ probe)).sum()
+        assert abs(lhs - o["k_out"][t] @ probe) < 1e-10
+        for src, out in ((k, o["k_out"]), (v, o["v_out"])):
+            lo, hi = src[mem].min(0) - 1e-12, src[mem].max(0) + 1e-12
+            assert ((out[t] >= lo) & (out[t] <= hi)).all()
+    assert checked > 0
+
+
+def test_exact_duplicates_merge_to_their_centre():
+    """sigma = 0: members of a group are identical, so any convex combination equals the centre (to rounding of the weights); equal scores resolve by row."""
+    w = wl.WORKLOADS["tiny"].with_(noise=0.0)
+    k, v, q = wl.make_unit(w, 0, 0, 0)
+    o = orc.event(k, v, q, w.prefix, w.budget, w.reserve)
+    n_groups = 0
+    for t in np.nonzero(o["slot_kind"] == 4)[0]:
+        mem = np.nonzero(o["assign"] == t)[0]
+        src = o["slot_src"][t]
+        assert (k[mem] == k[src]).all()
+        assert np.allclose(o["k_out"][t], k[src].astype(np.float64), rtol=1e-14, atol=0)
+        assert np.allclose(o["v_out"][t], v[src].astype(np.float64), rtol=1e-14, atol=0)
+        n_groups += len(mem) > 1
+    assert n_groups > 0
+    # duplicates below the window have identical scores: the earlier row must win the seed slot
+    s = o["s"]
+    for t in np.nonzero(o["slot_kind"] == 4)[0]:
+        mem = np.nonzero(o["assign"] == t)[0]
+        src = o["slot_src"][t]
+        tied = [i for i in mem if s[i] == s[src]]
+        assert src == min(tied)
+
+
+def test_planted_clusters_are_recovered_with_full_purity():
+    """Tiny config: 24 planted centres, noise 0.05: in-cluster cosine ~0.9975 vs cross-cluster far below tau."""
+    w = wl.WORKLOADS["tiny"]
+    for head in (0, 1):
+        k, v, q = wl.make_unit(w, 0, 0, head)
+        o = orc.event(k, v, q, w.prefix, w.budget, w.reserve)
+        kn = k / np.linalg.norm(k, axis=1, keepdims=True)
+        joiners = np.nonzero(o["kind"] == 5)[0]
+        assert len(joiners) > 0
+        for j in joiners:
+            assert kn[j] @ kn[o["seed_of"][j]] > 0.99          # same planted cluster
+        # a dropped scratch row has no seed in its own cluster
+        seeds = np.nonzero(o["kind"] == 4)[0]
+        dropped = np.nonzero((o["kind"] == 0) & (np.arange(len(k)) >= w.prefix))[0]
+        assert (kn[dropped] @ kn[seeds].T).max() < 0.9
+
+
+# ---- whole event vs the separately written brute force -----------------------
+
+def _cmp_with_bruteforce(K, V, Q, P, B, res, tau):
+    o = orc.event(K, V, Q, P, B, res, tau=tau)
+    b = bf.event(K.tolist(), V.tolist(), Q.tolist(), P, B, res, tau=tau)
+    assert np.allclose(o["s"], b["s"], rtol=1e-12, atol=1e-300)
+    assert o["kind"].tolist() == b["kind"]
+    assert o["slot_src"].tolist() == b["slots"]
+    assert o["assign"].tolist() == b["assign"]
+    assert o["n_out"] == b["n_out"]
+    assert o["status"] == b["flags"], (o["status"], b["flags"], P, B, res)
+    assert np.allclose(o["weight"], b["weight"], rtol=1e-12, atol=0)
+    assert np.allclose(o["slot_mass"], b["mass"], rtol=1e-12)
+    assert abs(o["lost_mass"] - b["lost"]) < 1e-12
+    if o["n_out"]:
+        assert np.allclose(o["k_out"], np.array(b["k_out"]), rtol=1e-12, atol=1e-14)
+        assert np.allclose(o["v_out"], np.array(b["v_out"]), rtol=1e-12, atol=1e-14)
+
+
+def test_whole_event_against_bruteforce_all_small_shapes():
+    """Every (T, P, B, reserve, W) with T <= 12 on clustered rows, including both sides of B_d = r + 2."""
+    rng = np.random.default_rng(10)
+    n = 0
+    for T in (5, 9, 12):
+        centres = rng.standard_normal((3, 4))
+        K = (centres[rng.integers(0, 3, T)] + 0.05 * rng.standard_normal((T, 4))).astype(np.float32)
+        V = rng.standard_normal((T, 4)).astype(np.float32)
+        for W in (1, 2, 4):
+            Q = rng.standard_normal((2, W, 4)).astype(np.float32)
+            for P, B in itertools.product(range(0, T + 1), range(1, T + 2)):
+                for res in range(0, B + 1):
+                    _cmp_with_bruteforce(K, V, Q, P, B, res, tau=0.9 if (P + B) % 2 else -1.0)
+                    n += 1
+    assert n > 1500
+
+
+def test_whole_event_against_bruteforce_exhausted_boundary():
+    rng = np.random.default_rng(11)
+    T, P, W, d = 16, 10, 3, 4
+    K, V, Q = _rand_unit(rng, T, d, 2, W)
+    B = 9
+    seen = set()
+    for res in range(0, B + 1):
+        o = orc.event(K, V, Q, P, B, res)
+        seen.add(bool(o["status"] & orc.PREFIX_BUDGET_EXHAUSTED))
+        _cmp_with_bruteforce(K, V, Q, P, B, res, tau=0.5)
+        Bd = B - min(P, B - res)
+        assert bool(o["status"] & orc.PREFIX_BUDGET_EXHAUSTED) == (T - P > Bd and Bd < W + 2)
+    assert seen == {True, False}
+
+
+def test_units_are_independent():
+    """A unit's result does not depend on its neighbours in the batch or on their order."""
+    w = wl.WORKLOADS["tiny"]
+    b = wl.make_batch(w)
+    full = orc.event_batch(wl.as_float32(b.k, w.dtype), b.v, b.q, b.tok_off, b.P, b.B, b.reserve)
+    for u in range(b.n_units):
+        k, v, q = b.unit(u)
+        one = orc.event(k, v, q, w.prefix, w.budget, w.reserve)
+        a, e = int(b.tok_off[u]), int(b.tok_off[u + 1])
+        assert np.array_equal(full["s"][a:e], one["s"])
+        assert np.array_equal(full["kind"][a:e], one["kind"])
+        assert np.array_equal(full["k_out"][u][:one["n_out"]], one["k_out"])
+
+
+def test_bf16_rounding_helper():
+    x = np.array([1.0, 1.0 + 2 ** -8, 1.0 + 3 * 2 ** -8, -3.14159, 1e-40, 0.0, 300.5])
+    got = orc.round_bf16(x)
+    ref = wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(x.astype(np.float32)))
+    assert got[0] == 1.0 and got[1] == 1.0 and got[2] == np.float32(1.0 + 2 ** -6)   # ties to even
+    assert np.array_equal(got[3:], ref[3:])
