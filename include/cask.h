@@ -1,0 +1,246 @@
+/*
+ * cask.h -- C-ABI boundary of the B200 compression-event library (libcask.so).
+ *
+ * One "unit" is one (sequence, layer, KV head): a cache of T rows of head_dim
+ * elements for keys and for values, rows [0,P) the prompt prefix and rows
+ * [P,T) the decode trace, plus the last W ("window") queries of the g query
+ * heads that share the KV head.  A compression event reduces every unit to at
+ * most B rows.  Units are independent; a batch is a ragged list of units.
+ *
+ * Conventions that hold for every call unless a parameter says otherwise:
+ *   - DEVICE pointers: k, v, q, lse_in, every output array, the workspace.
+ *     They are owned by the caller; the library allocates no device memory.
+ *   - HOST pointers: the cask_batch struct itself and its per-unit integer
+ *     arrays (T, P, B, reserve, k_off, v_off, tok_off); they are read during
+ *     the call and may be freed when it returns.
+ *   - Calls are asynchronous on the context's stream.  The int returned is 0
+ *     or a negative CASK_ERR_* found on the host BEFORE any launch; nothing
+ *     on the device traps.  Per-unit outcomes are CASK_ST_* bits.
+ *   - Inputs are never modified; outputs must not alias inputs.
+ *   - Per-row arrays ("[sumT]") are indexed by tok_off[u] + i.
+ *   - Per-slot arrays are [n_units, Bmax]; Bmax >= max_u B[u].
+ */
+#ifndef CASK_H
+#define CASK_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- return codes ------------------------------------------------------- */
+#define CASK_OK                 0
+#define CASK_ERR_NULL          -1   /* a required pointer is NULL                     */
+#define CASK_ERR_SHAPE         -2   /* head_dim/group/window/T/P/B/reserve out of range */
+#define CASK_ERR_ALIGN         -3   /* a base pointer, offset or row stride breaks the 16-byte rule */
+#define CASK_ERR_WORKSPACE     -4   /* workspace NULL or smaller than cask_workspace_bytes */
+#define CASK_ERR_UNSUPPORTED   -5   /* a documented but unbuilt mode (paged cache)    */
+#define CASK_ERR_CUDA          -6   /* a CUDA runtime call failed (see cask_last_cuda_error) */
+#define CASK_ERR_PARAM         -7   /* gamma/tau/eps/causal out of range              */
+
+/* ---- per-unit status bits (plan[6], unit_status[u]) --------------------- */
+#define CASK_ST_NOOP_UNDER_BUDGET        1   /* T <= B: every row kept                        */
+#define CASK_ST_PREFIX_EVICTED           2   /* stage 1 removed prefix rows                   */
+#define CASK_ST_DECODE_CONSOLIDATED      4   /* stage 2 ran core protection + consolidation   */
+#define CASK_ST_PREFIX_BUDGET_EXHAUSTED  8   /* decode share cannot hold window + core + rep  */
+#define CASK_ST_MERGE_INACTIVE          16   /* stage 2 ran but no row joined any seed        */
+#define CASK_ST_TIMEOUT                 32   /* a bounded device wait gave up                 */
+#define CASK_ST_BOUNDS                  64   /* a device-side index check failed              */
+
+/* ---- row kinds (kind[i], slot_kind[t]) ---------------------------------- */
+#define CASK_KIND_DROPPED  0
+#define CASK_KIND_PREFIX   1   /* kept prefix row                          */
+#define CASK_KIND_RECENT   2   /* one of the last r decode rows            */
+#define CASK_KIND_CORE     3   /* protected core chosen by score           */
+#define CASK_KIND_SEED     4   /* anchor of a representative               */
+#define CASK_KIND_MERGED   5   /* scratch row folded into a representative */
+
+/* ---- plan[u][0..7] ------------------------------------------------------ */
+#define CASK_PLAN_BP     0   /* prefix share B_p = B - reserve            */
+#define CASK_PLAN_PKEEP  1   /* prefix rows kept = min(P, B_p)            */
+#define CASK_PLAN_BD     2   /* decode share B_d = B - P_keep             */
+#define CASK_PLAN_R      3   /* recent rows r                             */
+#define CASK_PLAN_C      4   /* core rows chosen by score c               */
+#define CASK_PLAN_M      5   /* representatives m                         */
+#define CASK_PLAN_FLAGS  6   /* structural CASK_ST_* bits                 */
+#define CASK_PLAN_NOUT   7   /* rows after the event                      */
+
+#define CASK_DTYPE_BF16 0
+#define CASK_DTYPE_FP32 1
+
+typedef struct cask_ctx cask_ctx;
+
+/*
+ * A ragged batch of independent units (Sec. 2.3 of the paper constrains one
+ * cache at a time: |R| <= B, C subset of R; nothing couples units).
+ * Layout: contiguous rows.  Row i of unit u starts at element
+ *   k + k_off[u] + i*row_stride            (same for v with v_off)
+ * row_stride >= head_dim; base pointers, offsets*elem and row_stride*elem must
+ * be multiples of 16 bytes.  q is [n_units, group, window, head_dim], dense;
+ * window query j of a unit belongs to cache row T-window+j.
+ */
+typedef struct {
+    int32_t n_units;
+    int32_t head_dim;        /* d: multiple of 8, 8..256                        */
+    int32_t group;           /* g: query heads per KV head, >= 1                */
+    int32_t window;          /* W: 1 <= W <= T[u] for every unit               */
+    int32_t dtype;           /* CASK_DTYPE_BF16 | CASK_DTYPE_FP32 (k, v, q, outputs) */
+    int32_t page_size;       /* 0 = contiguous rows; > 0 (paged) -> CASK_ERR_UNSUPPORTED */
+    const void* k;           /* DEVICE */
+    const void* v;           /* DEVICE */
+    const int64_t* k_off;    /* HOST [n_units], elements                        */
+    const int64_t* v_off;    /* HOST [n_units], elements                        */
+    int64_t row_stride;      /* elements                                        */
+    const void* q;           /* DEVICE [n_units, g, W, d]                       */
+    const float* lse_in;     /* DEVICE [n_units, g, W] natural-log normalisers of the
+                                window queries, or NULL to have them computed   */
+    const int32_t* T;        /* HOST [n_units] rows in the cache                */
+    const int32_t* P;        /* HOST [n_units] prefix rows, 0 <= P <= T         */
+    const int32_t* B;        /* HOST [n_units] budget, >= 1                     */
+    const int32_t* reserve;  /* HOST [n_units] slots held back for decode, 0..B */
+    const int64_t* tok_off;  /* HOST [n_units+1] offsets into per-row arrays; tok_off[u+1]-tok_off[u] >= T[u] */
+} cask_batch;
+
+/*
+ * Policy parameters.  The paper gives no values for them (it names a "reserve
+ * schedule" and leaves a_i open, Sec. 2.4 / 7.2); defaults in parentheses.
+ */
+typedef struct {
+    float gamma;        /* (0.5) share of the non-recent decode slots given to the core, 0..1 */
+    float tau;          /* (0.9) minimum cosine similarity for a scratch row to join a seed   */
+    float eps;          /* (1e-9) a_i = s_i + eps keeps every group mass positive, > 0        */
+    int32_t causal;     /* (1) window query j sees rows i <= T-W+j; 0: every query sees all rows */
+    int32_t score_path; /* (0) 0: tensor-core scoring when the shape allows; 1: always the SIMT kernels */
+} cask_params;
+
+/* Outputs of a whole event.  DEVICE pointers; "optional" ones may be NULL. */
+typedef struct {
+    void* k_out;           /* [n_units, Bmax, d] cache dtype; rows >= n_out[u] are not written */
+    void* v_out;           /* [n_units, Bmax, d]                                             */
+    int32_t Bmax;
+    int32_t* n_out;        /* [n_units] rows kept (== plan[7])                                */
+    int32_t* slot_src;     /* [n_units, Bmax] cache row each slot is anchored at, -1 beyond n_out */
+    uint8_t* slot_kind;    /* [n_units, Bmax] CASK_KIND_*, 0 beyond n_out                     */
+    float* slot_mass;      /* [n_units, Bmax] m_G = sum of a_i over the slot's members        */
+    int32_t* assign;       /* [sumT] slot a row went to, -1 if dropped                        */
+    float* weight;         /* [sumT] 1 kept singleton, w_i = a_i/m_G group member, 0 dropped  */
+    uint8_t* kind;         /* [sumT] CASK_KIND_*                                              */
+    int32_t* seed_of;      /* [sumT] cache row of the group's seed (seeds point at themselves), else -1 */
+    int32_t* plan;         /* [n_units, 8] CASK_PLAN_*                                        */
+    int32_t* unit_status;  /* [n_units] CASK_ST_* bits                                        */
+    float* lost_mass;      /* [n_units] sum of a_j over scratch rows that joined nobody       */
+    float* s;              /* optional [sumT] scores                                          */
+    float* lse;            /* optional [n_units, g, W] natural-log normalisers used           */
+    float* sim;            /* optional [sumT] best cosine similarity of non-seed scratch rows, -2 elsewhere */
+} cask_outputs;
+
+/* ---- context ------------------------------------------------------------ */
+
+/* Creates a context bound to `device` and `cuda_stream` (a cudaStream_t, NULL =
+ * default stream).  Owns a small pinned staging buffer for per-unit descriptors. */
+int cask_create(cask_ctx** out, int device, void* cuda_stream);
+int cask_destroy(cask_ctx* ctx);
+int cask_set_stream(cask_ctx* ctx, void* cuda_stream);
+const char* cask_strerror(int code);
+/* Name of the last CUDA error seen by this context ("" if none). */
+const char* cask_last_cuda_error(const cask_ctx* ctx);
+/* Kernels launched by this context since creation (every call adds its own). */
+int64_t cask_launch_count(const cask_ctx* ctx);
+/* 1 if the last cask_score / cask_compress_event used the tensor-core kernels. */
+int cask_last_score_path_tensor(const cask_ctx* ctx);
+
+/* Bytes of workspace that any call below needs for this batch (host-only arithmetic). */
+size_t cask_workspace_bytes(const cask_batch* batch, const cask_params* params);
+
+/*
+ * Budget split on the host (Sec. 2.2 slack for the decode stage, Sec. 2.3 |R| <= B
+ * with C subset of R, Sec. 5.2 collapse of the available slots).  The paper
+ * gives no numbers; the rule used is
+ *   B_p = B - reserve;  P_keep = min(P, B_p);  B_d = B - P_keep;  N_d = T - P;
+ *   T <= B       -> NOOP_UNDER_BUDGET, all rows kept;
+ *   r = min(W, N_d);
+ *   N_d <= B_d   -> every decode row kept (c = N_d - r, m = 0);
+ *   B_d < r + 2  -> PREFIX_BUDGET_EXHAUSTED: r = min(r, B_d), c = B_d - r, m = 0;
+ *   else DECODE_CONSOLIDATED: c = min(ceil(gamma (B_d - r)), B_d - r - 1), m = B_d - r - c.
+ * Fills plan[n_units*8] (HOST).  The device calls use the same rule.
+ */
+int cask_plan_host(const cask_batch* batch, const cask_params* params, int32_t* plan_host);
+
+/* ---- the staged hot path -------------------------------------------------- */
+
+/*
+ * Score (Sec. 1: scalar importance per token; the deployed scorer has no
+ * formula in the paper, this library uses windowed attention mass):
+ *   x_hji = <q_hj, k_i>/sqrt(d);  p = softmax over visible i;  s_i = mean_{h,j} p_hji.
+ * s [sumT] fp32 out; lse_out optional [n_units, g, W].
+ */
+int cask_score(cask_ctx* ctx, const cask_batch* batch, const cask_params* params,
+               float* s, float* lse_out, void* ws, size_t ws_bytes);
+
+/*
+ * Stage 1, prefix eviction (Sec. 2.2): writes plan[n_units,8] and kind for the
+ * prefix rows [0,P): the P_keep rows greatest under (score descending, row
+ * ascending) get CASK_KIND_PREFIX, the others 0; all P rows if P <= B_p.
+ * Decode rows of `kind` are set to 0.
+ */
+int cask_prefix_evict(cask_ctx* ctx, const cask_batch* batch, const cask_params* params,
+                      const float* s, uint8_t* kind, int32_t* plan, void* ws, size_t ws_bytes);
+
+/*
+ * Protected core (Sec. 2.1, 2.3): last r decode rows -> CASK_KIND_RECENT, the c
+ * greatest of rows [P, T-r) -> CASK_KIND_CORE; other decode rows stay 0.
+ * `plan` is the array cask_prefix_evict wrote.
+ */
+int cask_select_core(cask_ctx* ctx, const cask_batch* batch, const cask_params* params,
+                     const float* s, const int32_t* plan, uint8_t* kind, void* ws, size_t ws_bytes);
+
+/*
+ * Scratch consolidation (Sec. 2.1, 2.4, 2.5): among decode rows of kind 0 the m
+ * greatest become seeds (4); every other one joins the seed of highest cosine
+ * similarity if that is >= tau (5) or is dropped (0).  Writes seed_of, weight
+ * (w_i = a_i/m_G for group members, 0 for dropped scratch), optional sim,
+ * unit_status (plan flags | MERGE_INACTIVE) and lost_mass.
+ */
+int cask_consolidate_scratch(cask_ctx* ctx, const cask_batch* batch, const cask_params* params,
+                             const float* s, const int32_t* plan, uint8_t* kind, int32_t* seed_of,
+                             float* weight, float* sim, int32_t* unit_status, float* lost_mass,
+                             void* ws, size_t ws_bytes);
+
+/*
+ * Compaction (Sec. 2.3 |R| <= B; Sec. 2.4 merge rule): slots are the rows of
+ * kind 1..4 in ascending row order; a slot of kind 4 holds sum_i w_i k_i and
+ * sum_i w_i v_i over its group (members in ascending row order, fp32
+ * accumulation, rounded once to the cache dtype; a group of one is a byte
+ * copy); every other slot is a byte copy of its row.  `weight` is read for
+ * kinds 4/5 and finalised (1 for kinds 1..3, 0 for kind 0).  Uses out->k_out,
+ * v_out, Bmax, n_out, slot_src, slot_kind, slot_mass, assign; other fields of
+ * `out` are ignored.
+ */
+int cask_compact(cask_ctx* ctx, const cask_batch* batch, const cask_params* params,
+                 const float* s, const uint8_t* kind, const int32_t* seed_of, float* weight,
+                 const cask_outputs* out, void* ws, size_t ws_bytes);
+
+/* The five steps above in order on one stream; results are bit-identical to
+ * calling them one by one. */
+int cask_compress_event(cask_ctx* ctx, const cask_batch* batch, const cask_params* params,
+                        const cask_outputs* out, void* ws, size_t ws_bytes);
+
+/*
+ * The same event for callers whose cache lives in HOST memory (ideally
+ * page-locked): batch->k, v, q, lse_in and every pointer in `out` are HOST
+ * pointers here.  dev_buf is a DEVICE buffer of at least
+ * cask_host_event_device_bytes() that holds the staged inputs, outputs and the
+ * workspace.  Copies in, runs cask_compress_event, copies out and synchronises
+ * the stream before returning.  Rows of a unit must be dense (row_stride ==
+ * head_dim) and units laid out at k_off[u] == v_off[u] == tok_off[u]*head_dim.
+ */
+size_t cask_host_event_device_bytes(const cask_batch* batch, const cask_params* params, int32_t Bmax);
+int cask_compress_event_host(cask_ctx* ctx, const cask_batch* host_batch, const cask_params* params,
+                             const cask_outputs* host_out, void* dev_buf, size_t dev_bytes);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CASK_H */

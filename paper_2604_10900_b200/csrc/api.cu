@@ -1,0 +1,519 @@
+// C-ABI layer of libcask: argument checks, budget split, workspace carving, call sequencing.
+// Every error is found here, on the host, before anything is launched.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "cask_internal.cuh"
+
+using namespace cask;
+
+struct cask_ctx {
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    UnitDesc* pinned = nullptr;      // staging for the per-unit descriptors
+    size_t pinned_units = 0;
+    cudaEvent_t staged = nullptr;    // recorded after the last descriptor upload
+    bool staged_pending = false;
+    int64_t launches = 0;
+    cudaError_t last_err = cudaSuccess;
+    int last_tc = 0;
+    void* tmap_encode = nullptr;     // cuTensorMapEncodeTiled, resolved at creation
+};
+
+namespace {
+
+inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+inline size_t elem_size(int dtype) { return dtype == CASK_DTYPE_BF16 ? 2 : 4; }
+
+// The budget split (Sec. 2.2, 2.3, 5.2); the rule is stated beside cask_plan_host in cask.h.
+void plan_unit(int T, int P, int B, int reserve, int W, float gamma, int32_t* pl) {
+    const int Nd = T - P;
+    const int Bp = B - reserve;
+    int Pkeep = std::min(P, Bp), Bd, r = std::min(W, Nd), c = 0, m = 0, flags = 0, nout;
+    if (T <= B) {
+        flags = CASK_ST_NOOP_UNDER_BUDGET;
+        Pkeep = P;
+        Bd = B - P;
+        c = Nd - r;
+        nout = T;
+    } else {
+        Bd = B - Pkeep;
+        if (P > Bp) flags |= CASK_ST_PREFIX_EVICTED;
+        if (Nd <= Bd) {
+            c = Nd - r;
+            nout = Pkeep + Nd;
+        } else if (Bd < r + 2) {
+            flags |= CASK_ST_PREFIX_BUDGET_EXHAUSTED;
+            r = std::min(r, Bd);
+            c = Bd - r;
+            nout = Pkeep + Bd;
+        } else {
+            flags |= CASK_ST_DECODE_CONSOLIDATED;
+            const int room = Bd - r;
+            c = (int)std::ceil((double)gamma * (double)room);
+            c = std::max(0, std::min(c, room - 1));
+            m = room - c;
+            nout = Pkeep + Bd;
+        }
+    }
+    pl[CASK_PLAN_BP] = Bp; pl[CASK_PLAN_PKEEP] = Pkeep; pl[CASK_PLAN_BD] = Bd; pl[CASK_PLAN_R] = r;
+    pl[CASK_PLAN_C] = c; pl[CASK_PLAN_M] = m; pl[CASK_PLAN_FLAGS] = flags; pl[CASK_PLAN_NOUT] = nout;
+}
+
+int check_batch(const cask_batch* b, const cask_params* p) {
+    if (!b || !p) return CASK_ERR_NULL;
+    if (b->n_units < 0) return CASK_ERR_SHAPE;
+    if (b->page_size != 0) return CASK_ERR_UNSUPPORTED;
+    if (b->dtype != CASK_DTYPE_BF16 && b->dtype != CASK_DTYPE_FP32) return CASK_ERR_SHAPE;
+    if (b->head_dim < 8 || b->head_dim > 256 || b->head_dim % 8) return CASK_ERR_SHAPE;
+    if (b->group < 1 || b->window < 1 || (int64_t)b->group * b->window > 65536) return CASK_ERR_SHAPE;
+    if (!(p->gamma >= 0.f && p->gamma <= 1.f) || !(p->eps > 0.f) || std::isnan(p->tau) ||
+        (p->causal != 0 && p->causal != 1) || (p->score_path != 0 && p->score_path != 1))
+        return CASK_ERR_PARAM;
+    if (b->n_units == 0) return CASK_OK;
+    if (!b->k || !b->v || !b->q || !b->k_off || !b->v_off || !b->T || !b->P || !b->B || !b->reserve ||
+        !b->tok_off)
+        return CASK_ERR_NULL;
+    const size_t e = elem_size(b->dtype);
+    if (b->row_stride < b->head_dim) return CASK_ERR_SHAPE;
+    if (((uintptr_t)b->k | (uintptr_t)b->v | (uintptr_t)b->q) % 16 || (b->row_stride * e) % 16)
+        return CASK_ERR_ALIGN;
+    if (b->lse_in && (uintptr_t)b->lse_in % 4) return CASK_ERR_ALIGN;
+    for (int u = 0; u < b->n_units; ++u) {
+        const int T = b->T[u], P = b->P[u], B = b->B[u], R = b->reserve[u];
+        if (T < 1 || b->window > T || P < 0 || P > T || B < 1 || R < 0 || R > B) return CASK_ERR_SHAPE;
+        if (b->k_off[u] < 0 || b->v_off[u] < 0) return CASK_ERR_SHAPE;
+        if ((b->k_off[u] * e) % 16 || (b->v_off[u] * e) % 16) return CASK_ERR_ALIGN;
+        if (b->tok_off[u] < 0 || b->tok_off[u + 1] - b->tok_off[u] < T) return CASK_ERR_SHAPE;
+    }
+    return CASK_OK;
+}
+
+struct Sizes {
+    int64_t sum_T = 0, sum_m = 0;
+    int total_chunks = 0, max_chunks = 0, max_m = 0, max_T = 0, max_P = 0, max_B = 0;
+};
+
+Sizes batch_sizes(const cask_batch* b, const cask_params* p) {
+    Sizes z;
+    z.sum_T = b->n_units ? b->tok_off[b->n_units] : 0;
+    for (int u = 0; u < b->n_units; ++u) {
+        int32_t pl[8];
+        plan_unit(b->T[u], b->P[u], b->B[u], b->reserve[u], b->window, p->gamma, pl);
+        const int nch = (b->T[u] + kChunkKeys - 1) / kChunkKeys;
+        z.total_chunks += nch;
+        z.max_chunks = std::max(z.max_chunks, nch);
+        z.sum_m += pl[CASK_PLAN_M];
+        z.max_m = std::max(z.max_m, pl[CASK_PLAN_M]);
+        z.max_T = std::max(z.max_T, b->T[u]);
+        z.max_P = std::max(z.max_P, b->P[u]);
+        z.max_B = std::max(z.max_B, b->B[u]);
+    }
+    return z;
+}
+
+// Lays the workspace out; with base == nullptr only the size is computed.
+Workspace carve(char* base, const cask_batch* b, const Sizes& z) {
+    Workspace w{};
+    size_t off = 0;
+    auto take = [&](size_t bytes) -> char* {
+        char* p = base ? base + off : nullptr;
+        off += align_up(std::max<size_t>(bytes, 16));
+        return p;
+    };
+    const size_t n = (size_t)b->n_units, rows = (size_t)b->group * b->window, sumT = (size_t)z.sum_T;
+    w.desc = (UnitDesc*)take(n * sizeof(UnitDesc));
+    w.s = (float*)take(sumT * 4);
+    w.rowm = (float*)take(n * rows * 4);
+    w.roww = (float*)take(n * rows * 4);
+    w.part_m = (float*)take((size_t)z.total_chunks * rows * 4);
+    w.part_l = (float*)take((size_t)z.total_chunks * rows * 4);
+    w.seed_rows = (int32_t*)take((size_t)z.sum_m * 4);
+    w.seed_norm = (float*)take((size_t)z.sum_m * 4);
+    w.seed_k = take(((size_t)z.sum_m + 256) * b->head_dim * elem_size(b->dtype));
+    w.grp = (int32_t*)take(sumT * 4);
+    w.mass_fx = (unsigned long long*)take(n * ((size_t)z.max_m + 1) * 8);
+    w.njoin = (int32_t*)take(n * 4);
+    w.mem_row = (int32_t*)take(sumT * 4);
+    w.mem_slot = (int32_t*)take(sumT * 4);
+    w.n_mem = (int32_t*)take(n * 4);
+    w.err = (int32_t*)take(16);
+    w.bytes = off;
+    return w;
+}
+
+int fail_cuda(cask_ctx* ctx, cudaError_t e) {
+    ctx->last_err = e;
+    return CASK_ERR_CUDA;
+}
+
+// Validates, builds and uploads the per-unit descriptors, resolves the launch record.
+int prepare(cask_ctx* ctx, const cask_batch* b, const cask_params* p, void* ws, size_t ws_bytes, Launch& L,
+            Workspace& W) {
+    if (!ctx) return CASK_ERR_NULL;
+    int rc = check_batch(b, p);
+    if (rc != CASK_OK) return rc;
+    if (b->n_units == 0) return CASK_OK;
+    const Sizes z = batch_sizes(b, p);
+    W = carve(nullptr, b, z);
+    if (!ws || ws_bytes < W.bytes || (uintptr_t)ws % 256) return CASK_ERR_WORKSPACE;
+    W = carve((char*)ws, b, z);
+
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    if (ctx->staged_pending) {
+        e = cudaEventSynchronize(ctx->staged);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+        ctx->staged_pending = false;
+    }
+    if (ctx->pinned_units < (size_t)b->n_units) {
+        if (ctx->pinned) cudaFreeHost(ctx->pinned);
+        ctx->pinned = nullptr;
+        ctx->pinned_units = 0;
+        e = cudaMallocHost((void**)&ctx->pinned, sizeof(UnitDesc) * (size_t)b->n_units);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+        ctx->pinned_units = (size_t)b->n_units;
+    }
+    int chunk0 = 0, seed_base = 0;
+    const int64_t q_unit = (int64_t)b->group * b->window * b->head_dim;
+    for (int u = 0; u < b->n_units; ++u) {
+        UnitDesc& d = ctx->pinned[u];
+        d.k_off = b->k_off[u];
+        d.v_off = b->v_off[u];
+        d.q_off = q_unit * u;
+        d.tok_off = b->tok_off[u];
+        d.T = b->T[u]; d.P = b->P[u]; d.B = b->B[u]; d.reserve = b->reserve[u];
+        plan_unit(d.T, d.P, d.B, d.reserve, b->window, p->gamma, d.plan);
+        d.chunk0 = chunk0;
+        d.n_chunks = (d.T + kChunkKeys - 1) / kChunkKeys;
+        d.seed_base = seed_base;
+        d.pad = 0;
+        chunk0 += d.n_chunks;
+        seed_base += d.plan[CASK_PLAN_M];
+    }
+    e = cudaMemcpyAsync(W.desc, ctx->pinned, sizeof(UnitDesc) * (size_t)b->n_units, cudaMemcpyHostToDevice,
+                        ctx->stream);
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    e = cudaEventRecord(ctx->staged, ctx->stream);
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    ctx->staged_pending = true;
+
+    L.stream = ctx->stream;
+    L.sh.n_units = b->n_units; L.sh.d = b->head_dim; L.sh.g = b->group; L.sh.W = b->window;
+    L.sh.rows = b->group * b->window; L.sh.dtype = b->dtype; L.sh.row_stride = b->row_stride;
+    L.sh.causal = p->causal;
+    L.desc = W.desc; L.hdesc = ctx->pinned;
+    L.k = b->k; L.v = b->v; L.q = b->q;
+    L.max_T = z.max_T; L.max_m = z.max_m; L.max_chunks = z.max_chunks; L.total_chunks = z.total_chunks;
+    L.max_P = z.max_P; L.max_B = z.max_B; L.sum_T = z.sum_T;
+    L.launches = &ctx->launches;
+    return CASK_OK;
+}
+
+int run_score(cask_ctx* ctx, const Launch& L, const cask_batch* b, const cask_params* p, float* s,
+              float* lse_out, Workspace& W) {
+    cudaError_t e;
+    if (p->score_path == 0 && ctx->tmap_encode && score_tc_supported(L)) {
+        ctx->last_tc = 1;
+        e = launch_score_tc(L, b->lse_in, s, lse_out, W, ctx->tmap_encode);
+    } else {
+        ctx->last_tc = 0;
+        e = launch_score_simt(L, b->lse_in, s, lse_out, W);
+    }
+    return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
+}
+
+}  // namespace
+
+extern "C" {
+
+int cask_create(cask_ctx** out, int device, void* cuda_stream) {
+    if (!out) return CASK_ERR_NULL;
+    *out = nullptr;
+    cudaError_t e = cudaSetDevice(device);
+    if (e != cudaSuccess) return CASK_ERR_CUDA;
+    cask_ctx* c = new (std::nothrow) cask_ctx();
+    if (!c) return CASK_ERR_CUDA;
+    c->device = device;
+    c->stream = (cudaStream_t)cuda_stream;
+    e = cudaEventCreateWithFlags(&c->staged, cudaEventDisableTiming);
+    if (e != cudaSuccess) { delete c; return CASK_ERR_CUDA; }
+    cudaDriverEntryPointQueryResult qres;
+    void* fn = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+        c->tmap_encode = fn;
+    else
+        cudaGetLastError();
+    *out = c;
+    return CASK_OK;
+}
+
+int cask_destroy(cask_ctx* ctx) {
+    if (!ctx) return CASK_ERR_NULL;
+    cudaSetDevice(ctx->device);
+    if (ctx->staged_pending) cudaEventSynchronize(ctx->staged);
+    if (ctx->pinned) cudaFreeHost(ctx->pinned);
+    if (ctx->staged) cudaEventDestroy(ctx->staged);
+    delete ctx;
+    return CASK_OK;
+}
+
+int cask_set_stream(cask_ctx* ctx, void* cuda_stream) {
+    if (!ctx) return CASK_ERR_NULL;
+    ctx->stream = (cudaStream_t)cuda_stream;
+    return CASK_OK;
+}
+
+const char* cask_strerror(int code) {
+    switch (code) {
+        case CASK_OK: return "ok";
+        case CASK_ERR_NULL: return "a required pointer is NULL";
+        case CASK_ERR_SHAPE: return "shape out of range (head_dim, group, window, T, P, B, reserve, offsets)";
+        case CASK_ERR_ALIGN: return "pointer, offset or row stride is not a multiple of 16 bytes";
+        case CASK_ERR_WORKSPACE: return "workspace missing, misaligned (256 B) or too small";
+        case CASK_ERR_UNSUPPORTED: return "mode not built (paged cache)";
+        case CASK_ERR_CUDA: return "CUDA runtime error";
+        case CASK_ERR_PARAM: return "policy parameter out of range";
+        default: return "unknown error";
+    }
+}
+
+const char* cask_last_cuda_error(const cask_ctx* ctx) {
+    if (!ctx || ctx->last_err == cudaSuccess) return "";
+    return cudaGetErrorName(ctx->last_err);
+}
+
+int64_t cask_launch_count(const cask_ctx* ctx) { return ctx ? ctx->launches : 0; }
+int cask_last_score_path_tensor(const cask_ctx* ctx) { return ctx ? ctx->last_tc : 0; }
+
+size_t cask_workspace_bytes(const cask_batch* batch, const cask_params* params) {
+    if (check_batch(batch, params) != CASK_OK || batch->n_units == 0) return 0;
+    return carve(nullptr, batch, batch_sizes(batch, params)).bytes;
+}
+
+int cask_plan_host(const cask_batch* b, const cask_params* p, int32_t* plan_host) {
+    if (!b || !p || !plan_host) return CASK_ERR_NULL;
+    if (b->n_units > 0 && (!b->T || !b->P || !b->B || !b->reserve)) return CASK_ERR_NULL;
+    if (!(p->gamma >= 0.f && p->gamma <= 1.f)) return CASK_ERR_PARAM;
+    for (int u = 0; u < b->n_units; ++u) {
+        const int T = b->T[u], P = b->P[u], B = b->B[u], R = b->reserve[u];
+        if (T < 1 || b->window < 1 || b->window > T || P < 0 || P > T || B < 1 || R < 0 || R > B)
+            return CASK_ERR_SHAPE;
+        plan_unit(T, P, B, R, b->window, p->gamma, plan_host + (size_t)u * 8);
+    }
+    return CASK_OK;
+}
+
+int cask_score(cask_ctx* ctx, const cask_batch* b, const cask_params* p, float* s, float* lse_out, void* ws,
+               size_t ws_bytes) {
+    if (!s) return CASK_ERR_NULL;
+    Launch L{};
+    Workspace W{};
+    int rc = prepare(ctx, b, p, ws, ws_bytes, L, W);
+    if (rc != CASK_OK || b->n_units == 0) return rc;
+    return run_score(ctx, L, b, p, s, lse_out, W);
+}
+
+int cask_prefix_evict(cask_ctx* ctx, const cask_batch* b, const cask_params* p, const float* s, uint8_t* kind,
+                      int32_t* plan, void* ws, size_t ws_bytes) {
+    if (!s || !kind || !plan) return CASK_ERR_NULL;
+    Launch L{};
+    Workspace W{};
+    int rc = prepare(ctx, b, p, ws, ws_bytes, L, W);
+    if (rc != CASK_OK || b->n_units == 0) return rc;
+    cudaError_t e = launch_prefix_evict(L, s, kind, plan);
+    return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
+}
+
+int cask_select_core(cask_ctx* ctx, const cask_batch* b, const cask_params* p, const float* s,
+                     const int32_t* plan, uint8_t* kind, void* ws, size_t ws_bytes) {
+    if (!s || !kind || !plan) return CASK_ERR_NULL;
+    Launch L{};
+    Workspace W{};
+    int rc = prepare(ctx, b, p, ws, ws_bytes, L, W);
+    if (rc != CASK_OK || b->n_units == 0) return rc;
+    cudaError_t e = launch_select_core(L, s, plan, kind);
+    return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
+}
+
+int cask_consolidate_scratch(cask_ctx* ctx, const cask_batch* b, const cask_params* p, const float* s,
+                             const int32_t* plan, uint8_t* kind, int32_t* seed_of, float* weight, float* sim,
+                             int32_t* unit_status, float* lost_mass, void* ws, size_t ws_bytes) {
+    if (!s || !kind || !plan || !seed_of || !weight || !unit_status || !lost_mass) return CASK_ERR_NULL;
+    Launch L{};
+    Workspace W{};
+    int rc = prepare(ctx, b, p, ws, ws_bytes, L, W);
+    if (rc != CASK_OK || b->n_units == 0) return rc;
+    cudaError_t e = launch_consolidate(L, *p, s, plan, kind, seed_of, weight, sim, unit_status, lost_mass, W);
+    return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
+}
+
+static int max_budget(const cask_batch* b) {
+    int mb = 0;
+    if (b && b->B)
+        for (int u = 0; u < b->n_units; ++u) mb = std::max(mb, b->B[u]);
+    return mb;
+}
+
+static int check_compact_out(const cask_outputs* o, int max_B) {
+    if (!o) return CASK_ERR_NULL;
+    if (!o->k_out || !o->v_out || !o->n_out || !o->slot_src || !o->slot_kind || !o->slot_mass || !o->assign)
+        return CASK_ERR_NULL;
+    if (o->Bmax < max_B) return CASK_ERR_SHAPE;
+    if (((uintptr_t)o->k_out | (uintptr_t)o->v_out) % 16) return CASK_ERR_ALIGN;
+    return CASK_OK;
+}
+
+int cask_compact(cask_ctx* ctx, const cask_batch* b, const cask_params* p, const float* s, const uint8_t* kind,
+                 const int32_t* seed_of, float* weight, const cask_outputs* out, void* ws, size_t ws_bytes) {
+    if (!s || !kind || !seed_of || !weight) return CASK_ERR_NULL;
+    int rc = check_compact_out(out, max_budget(b));
+    if (rc != CASK_OK) return rc;
+    Launch L{};
+    Workspace W{};
+    rc = prepare(ctx, b, p, ws, ws_bytes, L, W);
+    if (rc != CASK_OK || b->n_units == 0) return rc;
+    cudaError_t e = launch_compact(L, *p, s, kind, seed_of, weight, *out, W);
+    return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
+}
+
+int cask_compress_event(cask_ctx* ctx, const cask_batch* b, const cask_params* p, const cask_outputs* out,
+                        void* ws, size_t ws_bytes) {
+    int rc = check_compact_out(out, max_budget(b));
+    if (rc != CASK_OK) return rc;
+    if (!out->weight || !out->kind || !out->seed_of || !out->plan || !out->unit_status || !out->lost_mass)
+        return CASK_ERR_NULL;
+    Launch L{};
+    Workspace W{};
+    rc = prepare(ctx, b, p, ws, ws_bytes, L, W);
+    if (rc != CASK_OK || b->n_units == 0) return rc;
+    float* s = out->s ? out->s : W.s;
+    rc = run_score(ctx, L, b, p, s, out->lse, W);
+    if (rc != CASK_OK) return rc;
+    cudaError_t e = launch_prefix_evict(L, s, out->kind, out->plan);
+    if (e == cudaSuccess) e = launch_select_core(L, s, out->plan, out->kind);
+    if (e == cudaSuccess)
+        e = launch_consolidate(L, *p, s, out->plan, out->kind, out->seed_of, out->weight, out->sim,
+                               out->unit_status, out->lost_mass, W);
+    if (e == cudaSuccess) e = launch_compact(L, *p, s, out->kind, out->seed_of, out->weight, *out, W);
+    return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
+}
+
+// ---- host-resident caches ------------------------------------------------------------------
+
+namespace {
+struct HostStage {
+    char *k, *v, *q, *lse_in;
+    cask_outputs o;
+    char* ws;
+    size_t ws_bytes, bytes;
+    size_t kv_bytes, q_bytes, lse_bytes;
+};
+
+HostStage stage_layout(char* base, const cask_batch* b, const cask_params* p, int32_t Bmax) {
+    HostStage h{};
+    size_t off = 0;
+    auto take = [&](size_t bytes) -> char* {
+        char* ptr = base ? base + off : nullptr;
+        off += align_up(std::max<size_t>(bytes, 16));
+        return ptr;
+    };
+    const size_t e = elem_size(b->dtype), n = (size_t)b->n_units, d = (size_t)b->head_dim;
+    const size_t sumT = (size_t)b->tok_off[b->n_units], rows = (size_t)b->group * b->window;
+    h.kv_bytes = sumT * d * e;
+    h.q_bytes = n * rows * d * e;
+    h.lse_bytes = n * rows * 4;
+    h.k = take(h.kv_bytes);
+    h.v = take(h.kv_bytes);
+    h.q = take(h.q_bytes);
+    h.lse_in = take(h.lse_bytes);
+    h.o.Bmax = Bmax;
+    h.o.k_out = take(n * Bmax * d * e);
+    h.o.v_out = take(n * Bmax * d * e);
+    h.o.n_out = (int32_t*)take(n * 4);
+    h.o.slot_src = (int32_t*)take(n * Bmax * 4);
+    h.o.slot_kind = (uint8_t*)take(n * Bmax);
+    h.o.slot_mass = (float*)take(n * Bmax * 4);
+    h.o.assign = (int32_t*)take(sumT * 4);
+    h.o.weight = (float*)take(sumT * 4);
+    h.o.kind = (uint8_t*)take(sumT);
+    h.o.seed_of = (int32_t*)take(sumT * 4);
+    h.o.plan = (int32_t*)take(n * 32);
+    h.o.unit_status = (int32_t*)take(n * 4);
+    h.o.lost_mass = (float*)take(n * 4);
+    h.o.s = (float*)take(sumT * 4);
+    h.o.lse = (float*)take(n * rows * 4);
+    h.o.sim = (float*)take(sumT * 4);
+    h.ws_bytes = carve(nullptr, b, batch_sizes(b, p)).bytes;
+    h.ws = take(h.ws_bytes);
+    h.bytes = off;
+    return h;
+}
+
+int check_host_layout(const cask_batch* b) {
+    if (b->row_stride != b->head_dim) return CASK_ERR_SHAPE;
+    for (int u = 0; u < b->n_units; ++u)
+        if (b->k_off[u] != b->tok_off[u] * b->head_dim || b->v_off[u] != b->k_off[u]) return CASK_ERR_SHAPE;
+    return CASK_OK;
+}
+}  // namespace
+
+size_t cask_host_event_device_bytes(const cask_batch* b, const cask_params* p, int32_t Bmax) {
+    if (check_batch(b, p) != CASK_OK || b->n_units == 0 || Bmax < 1) return 0;
+    return stage_layout(nullptr, b, p, Bmax).bytes;
+}
+
+int cask_compress_event_host(cask_ctx* ctx, const cask_batch* hb, const cask_params* p,
+                             const cask_outputs* ho, void* dev_buf, size_t dev_bytes) {
+    if (!ctx || !ho) return CASK_ERR_NULL;
+    int rc = check_batch(hb, p);
+    if (rc != CASK_OK) return rc;
+    if (hb->n_units == 0) return CASK_OK;
+    rc = check_host_layout(hb);
+    if (rc != CASK_OK) return rc;
+    if (ho->Bmax < 1) return CASK_ERR_SHAPE;
+    HostStage h = stage_layout(nullptr, hb, p, ho->Bmax);
+    if (!dev_buf || dev_bytes < h.bytes || (uintptr_t)dev_buf % 256) return CASK_ERR_WORKSPACE;
+    h = stage_layout((char*)dev_buf, hb, p, ho->Bmax);
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    cudaStream_t st = ctx->stream;
+    e = cudaMemcpyAsync(h.k, hb->k, h.kv_bytes, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h.v, hb->v, h.kv_bytes, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h.q, hb->q, h.q_bytes, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && hb->lse_in)
+        e = cudaMemcpyAsync(h.lse_in, hb->lse_in, h.lse_bytes, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    cask_batch db = *hb;
+    db.k = h.k; db.v = h.v; db.q = h.q;
+    db.lse_in = hb->lse_in ? (const float*)h.lse_in : nullptr;
+    rc = cask_compress_event(ctx, &db, p, &h.o, h.ws, h.ws_bytes);
+    if (rc != CASK_OK) return rc;
+    const size_t es = elem_size(hb->dtype), n = (size_t)hb->n_units, d = (size_t)hb->head_dim;
+    const size_t sumT = (size_t)hb->tok_off[hb->n_units], rows = (size_t)hb->group * hb->window;
+    const size_t Bm = (size_t)ho->Bmax;
+    struct Cp { void* dst; const void* src; size_t bytes; };
+    const Cp cps[] = {
+        {ho->k_out, h.o.k_out, n * Bm * d * es}, {ho->v_out, h.o.v_out, n * Bm * d * es},
+        {ho->n_out, h.o.n_out, n * 4}, {ho->slot_src, h.o.slot_src, n * Bm * 4},
+        {ho->slot_kind, h.o.slot_kind, n * Bm}, {ho->slot_mass, h.o.slot_mass, n * Bm * 4},
+        {ho->assign, h.o.assign, sumT * 4}, {ho->weight, h.o.weight, sumT * 4},
+        {ho->kind, h.o.kind, sumT}, {ho->seed_of, h.o.seed_of, sumT * 4},
+        {ho->plan, h.o.plan, n * 32}, {ho->unit_status, h.o.unit_status, n * 4},
+        {ho->lost_mass, h.o.lost_mass, n * 4}, {ho->s, h.o.s, sumT * 4},
+        {ho->lse, h.o.lse, n * rows * 4}, {ho->sim, h.o.sim, sumT * 4},
+    };
+    for (const Cp& c : cps) {
+        if (!c.dst) continue;
+        e = cudaMemcpyAsync(c.dst, c.src, c.bytes, cudaMemcpyDeviceToHost, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+    }
+    e = cudaStreamSynchronize(st);
+    return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
+}
+
+}  // extern "C"

@@ -1,0 +1,144 @@
+// Internal declarations shared by the kernels and the C-ABI layer of libcask.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/cask.h"
+
+namespace cask {
+
+// Per-unit descriptor, built on the host for every call and uploaded to the
+// head of the workspace.  Offsets are in elements of the cache dtype.
+struct UnitDesc {
+    int64_t k_off;
+    int64_t v_off;
+    int64_t q_off;
+    int64_t tok_off;
+    int32_t T, P, B, reserve;
+    int32_t plan[8];
+    int32_t chunk0;     // first score-partial chunk of this unit
+    int32_t n_chunks;   // key chunks of this unit in the normaliser pass
+    int32_t seed_base;  // first entry of this unit in the seed tables
+    int32_t pad;
+};
+
+struct Shape {
+    int n_units, d, g, W, rows;   // rows = g*W
+    int dtype;
+    int64_t row_stride;
+    int causal;
+};
+
+// Kernel ids for the optional per-kernel event timing.
+enum KernelId {
+    KID_SCORE_NORM = 0, KID_ROW_COMBINE, KID_SCORE_MASS, KID_PREFIX_EVICT, KID_SELECT_CORE, KID_SEEDS,
+    KID_SEED_GATHER, KID_ASSIGN, KID_WEIGHTS, KID_SLOT_SCAN, KID_GATHER_MERGE, KID_COUNT
+};
+
+// Records a CUDA event pair around every launch while switched on (defined in api.cu).
+struct Profiler {
+    bool on = false;
+    void begin(int id, cudaStream_t st);
+    void end(cudaStream_t st);
+    void* impl = nullptr;
+};
+
+// Everything a launch needs, resolved by the API layer.
+struct Launch {
+    cudaStream_t stream;
+    Shape sh;
+    const UnitDesc* desc;     // device
+    const UnitDesc* hdesc;    // host copy (for grid sizing)
+    const void* k;
+    const void* v;
+    const void* q;
+    int max_T, max_m, max_chunks, total_chunks, max_P, max_B;
+    int64_t sum_T;
+    int64_t* launches;        // counter to bump
+    Profiler* prof;
+};
+
+// Scope guard around one kernel launch: counts it and, in profiling mode, times it.
+struct Timed {
+    const Launch& L;
+    Timed(const Launch& l, int id) : L(l) {
+        ++*L.launches;
+        if (L.prof && L.prof->on) L.prof->begin(id, L.stream);
+    }
+    ~Timed() {
+        if (L.prof && L.prof->on) L.prof->end(L.stream);
+    }
+};
+
+constexpr int kChunkKeys = 2048;    // keys per normaliser-pass chunk
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kNegBig = -1.0e30f;   // finite stand-in for -inf in running maxima
+
+// ---- workspace carving ------------------------------------------------------
+struct Workspace {
+    UnitDesc* desc;
+    float* s;            // [sumT]   scores when the caller keeps none
+    float* rowm;         // [units*rows] row offset in log2 units
+    float* roww;         // [units*rows] row weight 1/(rows * sum)
+    float* part_m;       // [total_chunks*rows]
+    float* part_l;       // [total_chunks*rows]
+    int32_t* seed_rows;  // [sum m]     seed cache rows, ascending per unit
+    float* seed_norm;    // [sum m]
+    void* seed_k;        // [sum m_pad, d] gathered seed keys (cache dtype)
+    int32_t* grp;        // [sumT] seed slot (0..m) of a joined row, -1
+    unsigned long long* mass_fx;  // [units*(max_m+1)] fixed-point group masses (+ lost mass)
+    int32_t* njoin;      // [units]
+    int32_t* mem_row;    // [sumT] rows of kind 4/5 in ascending order
+    int32_t* mem_slot;   // [sumT] slot each of them feeds
+    int32_t* n_mem;      // [units]
+    int32_t* err;        // [1]
+    size_t bytes;
+};
+
+// ---- kernels (defined in the .cu files) --------------------------------------
+cudaError_t launch_score_simt(const Launch& L, const float* lse_in, float* s, float* lse_out,
+                              Workspace& ws);
+cudaError_t launch_row_combine(const Launch& L, const float* lse_in, float* lse_out, Workspace& ws);
+cudaError_t launch_prefix_evict(const Launch& L, const float* s, uint8_t* kind, int32_t* plan);
+cudaError_t launch_select_core(const Launch& L, const float* s, const int32_t* plan, uint8_t* kind);
+cudaError_t launch_consolidate(const Launch& L, const cask_params& prm, const float* s,
+                               const int32_t* plan, uint8_t* kind, int32_t* seed_of, float* weight,
+                               float* sim, int32_t* unit_status, float* lost_mass, Workspace& ws);
+cudaError_t launch_compact(const Launch& L, const cask_params& prm, const float* s, const uint8_t* kind,
+                           const int32_t* seed_of, float* weight, const cask_outputs& out, Workspace& ws);
+
+// Tensor-core scoring (tcgen05 + TMA); returns cudaErrorNotSupported when the shape does not fit.
+bool score_tc_supported(const Launch& L);
+cudaError_t launch_score_tc(const Launch& L, const float* lse_in, float* s, float* lse_out,
+                            Workspace& ws, void* tmap_encode_fn);
+
+// ---- small device helpers ------------------------------------------------------
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+    static __device__ __forceinline__ float ld(const float* p) { return *p; }
+    static __device__ __forceinline__ void st(float* p, float x) { *p = x; }
+};
+template <> struct Elem<__nv_bfloat16> {
+    static __device__ __forceinline__ float ld(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+    static __device__ __forceinline__ void st(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
+};
+
+// order-preserving map float -> uint32 (greater float <=> greater key)
+__device__ __forceinline__ uint32_t order_key(float x) {
+    uint32_t b = __float_as_uint(x);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+// fixed-point image of a mass a in [0, 2^20): 2^43 steps per unit
+constexpr double kMassScale = 8796093022208.0;   // 2^43
+__device__ __forceinline__ unsigned long long mass_to_fx(float a) {
+    return (unsigned long long)__double2ll_rn((double)a * kMassScale);
+}
+__device__ __forceinline__ float fx_to_mass(unsigned long long f) {
+    return (float)((double)f / kMassScale);
+}
+
+}  // namespace cask

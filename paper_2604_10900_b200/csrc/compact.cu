@@ -1,0 +1,194 @@
+// Compaction to the budget (Sec. 2.3: |R| <= B) with the weighted K/V merge of Sec. 2.4:
+//   slot order = ascending anchor row; kinds 1..3 and lone seeds are byte copies;
+//   a seed with joiners holds sum_i w_i k_i, sum_i w_i v_i (members in ascending row order).
+#include "cask_internal.cuh"
+
+namespace cask {
+
+namespace {
+
+constexpr int kScanThreads = 1024;
+
+// ---- 1. per-unit ordered scan: slots, index map, member list -------------------------------
+__global__ void __launch_bounds__(kScanThreads) slot_scan_kernel(
+    const UnitDesc* __restrict__ desc, const uint8_t* __restrict__ kind, const int32_t* __restrict__ seed_of,
+    float* __restrict__ weight, int Bmax, int32_t* __restrict__ n_out, int32_t* __restrict__ slot_src,
+    uint8_t* __restrict__ slot_kind, float* __restrict__ slot_mass, int32_t* __restrict__ assign,
+    int32_t* __restrict__ mem_row, int32_t* __restrict__ mem_slot, int32_t* __restrict__ n_mem) {
+    __shared__ unsigned wk[kScanThreads / 32], wm[kScanThreads / 32];
+    const int u = blockIdx.x;
+    const UnitDesc& ud = desc[u];
+    const int T = ud.T;
+    const int64_t o = ud.tok_off;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    unsigned base_k = 0, base_m = 0;
+    for (int i0 = 0; i0 < T; i0 += blockDim.x) {
+        const int i = i0 + threadIdx.x;
+        const uint8_t kd = (i < T) ? kind[o + i] : (uint8_t)0;
+        const bool keep = kd >= CASK_KIND_PREFIX && kd <= CASK_KIND_SEED;
+        const bool mem = kd == CASK_KIND_SEED || kd == CASK_KIND_MERGED;
+        const unsigned bk = __ballot_sync(0xffffffffu, keep), bm = __ballot_sync(0xffffffffu, mem);
+        __syncthreads();
+        if (lane == 0) { wk[w] = __popc(bk); wm[w] = __popc(bm); }
+        __syncthreads();
+        unsigned pk = 0, pm = 0, ak = 0, am = 0;
+        for (int x = 0; x < nw; ++x) {
+            if (x < w) { pk += wk[x]; pm += wm[x]; }
+            ak += wk[x];
+            am += wm[x];
+        }
+        const unsigned below = (1u << lane) - 1u;
+        if (i < T) {
+            int slot = -1;
+            if (keep) {
+                slot = (int)(base_k + pk + __popc(bk & below));
+                if (slot < Bmax) {
+                    slot_src[(size_t)u * Bmax + slot] = i;
+                    slot_kind[(size_t)u * Bmax + slot] = kd;
+                } else {
+                    slot = -1;        // more kept rows than slots: cannot happen for a valid plan
+                }
+            }
+            assign[o + i] = slot;
+            if (mem) mem_row[o + base_m + pm + __popc(bm & below)] = i;
+            if (kd >= CASK_KIND_PREFIX && kd <= CASK_KIND_CORE) weight[o + i] = 1.f;
+            if (kd == CASK_KIND_DROPPED) weight[o + i] = 0.f;
+        }
+        base_k += ak;
+        base_m += am;
+    }
+    const int nk = min((int)base_k, Bmax), nm = (int)base_m;
+    if (threadIdx.x == 0) { n_out[u] = nk; n_mem[u] = nm; }
+    for (int t = nk + threadIdx.x; t < Bmax; t += blockDim.x) {
+        slot_src[(size_t)u * Bmax + t] = -1;
+        slot_kind[(size_t)u * Bmax + t] = 0;
+        slot_mass[(size_t)u * Bmax + t] = 0.f;
+    }
+    __syncthreads();
+    // members point at their seed's slot
+    for (int e = threadIdx.x; e < nm; e += blockDim.x) {
+        const int i = mem_row[o + e];
+        int slot = -1;
+        if (kind[o + i] == CASK_KIND_SEED) {
+            slot = assign[o + i];
+        } else {
+            const int sd = seed_of[o + i];
+            if (sd >= 0 && sd < T && kind[o + sd] == CASK_KIND_SEED) slot = assign[o + sd];
+            assign[o + i] = slot;
+        }
+        mem_slot[o + e] = slot;
+    }
+}
+
+// ---- 2. one warp per slot: byte copy, or ordered weighted merge ----------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) gather_merge_kernel(
+    const UnitDesc* __restrict__ desc, Shape sh, const T* __restrict__ K, const T* __restrict__ V,
+    const float* __restrict__ s, const float* __restrict__ weight, float eps, int Bmax,
+    const int32_t* __restrict__ n_out, const int32_t* __restrict__ slot_src,
+    const uint8_t* __restrict__ slot_kind, const int32_t* __restrict__ mem_row,
+    const int32_t* __restrict__ mem_slot, const int32_t* __restrict__ n_mem, T* __restrict__ k_out,
+    T* __restrict__ v_out, float* __restrict__ slot_mass) {
+    const int u = blockIdx.y;
+    const UnitDesc& ud = desc[u];
+    const int lane = threadIdx.x & 31;
+    const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (t >= n_out[u]) return;
+    const int d = sh.d;
+    const int64_t o = ud.tok_off;
+    const int src = slot_src[(size_t)u * Bmax + t];
+    const uint8_t kd = slot_kind[(size_t)u * Bmax + t];
+    T* ko = k_out + ((size_t)u * Bmax + t) * d;
+    T* vo = v_out + ((size_t)u * Bmax + t) * d;
+    const T* ksrc = K + ud.k_off + (int64_t)src * sh.row_stride;
+    const T* vsrc = V + ud.v_off + (int64_t)src * sh.row_stride;
+    const int nvec = d * (int)sizeof(T) / 16;
+
+    bool copy = true;
+    float mass = s[o + src] + eps;
+    if (kd == CASK_KIND_SEED) {
+        constexpr int kMaxPerLane = 8;      // d <= 256
+        float ak[kMaxPerLane], av[kMaxPerLane];
+#pragma unroll
+        for (int x = 0; x < kMaxPerLane; ++x) { ak[x] = 0.f; av[x] = 0.f; }
+        int count = 0;
+        float msum = 0.f;
+        const int nm = n_mem[u];
+        for (int e0 = 0; e0 < nm; e0 += 32) {
+            const int e = e0 + lane;
+            const int row = (e < nm) ? mem_row[o + e] : -1;
+            const bool hit = (e < nm) && mem_slot[o + e] == t;
+            unsigned bal = __ballot_sync(0xffffffffu, hit);
+            while (bal) {
+                const int l = __ffs(bal) - 1;
+                bal &= bal - 1;
+                const int i = __shfl_sync(0xffffffffu, row, l);
+                const float wi = weight[o + i];
+                msum += s[o + i] + eps;
+                ++count;
+                const T* kr = K + ud.k_off + (int64_t)i * sh.row_stride;
+                const T* vr = V + ud.v_off + (int64_t)i * sh.row_stride;
+#pragma unroll
+                for (int x = 0; x < kMaxPerLane; ++x) {
+                    const int c = lane + 32 * x;
+                    if (c < d) {
+                        ak[x] = fmaf(wi, Elem<T>::ld(kr + c), ak[x]);
+                        av[x] = fmaf(wi, Elem<T>::ld(vr + c), av[x]);
+                    }
+                }
+            }
+        }
+        if (count > 1) {
+            copy = false;
+            mass = msum;
+#pragma unroll
+            for (int x = 0; x < kMaxPerLane; ++x) {
+                const int c = lane + 32 * x;
+                if (c < d) {
+                    Elem<T>::st(ko + c, ak[x]);
+                    Elem<T>::st(vo + c, av[x]);
+                }
+            }
+        }
+    }
+    if (copy) {
+        for (int x = lane; x < 2 * nvec; x += 32) {
+            const bool isv = x >= nvec;
+            const int c = isv ? x - nvec : x;
+            const uint4 val = reinterpret_cast<const uint4*>(isv ? vsrc : ksrc)[c];
+            reinterpret_cast<uint4*>(isv ? vo : ko)[c] = val;
+        }
+    }
+    if (lane == 0) slot_mass[(size_t)u * Bmax + t] = mass;
+}
+
+template <typename T>
+cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const uint8_t* kind,
+                const int32_t* seed_of, float* weight, const cask_outputs& out, Workspace& ws) {
+    const Shape& sh = L.sh;
+    {
+        Timed t(L, KID_SLOT_SCAN);
+        slot_scan_kernel<<<sh.n_units, kScanThreads, 0, L.stream>>>(L.desc, kind, seed_of, weight, out.Bmax,
+                                                                    out.n_out, out.slot_src, out.slot_kind,
+                                                                    out.slot_mass, out.assign, ws.mem_row,
+                                                                    ws.mem_slot, ws.n_mem);
+    }
+    const int slots = min(out.Bmax, max(L.max_B, 1));
+    {
+        Timed t(L, KID_GATHER_MERGE);
+        gather_merge_kernel<T><<<dim3((slots + 7) / 8, sh.n_units), 256, 0, L.stream>>>(
+            L.desc, sh, (const T*)L.k, (const T*)L.v, s, weight, prm.eps, out.Bmax, out.n_out, out.slot_src,
+            out.slot_kind, ws.mem_row, ws.mem_slot, ws.n_mem, (T*)out.k_out, (T*)out.v_out, out.slot_mass);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_compact(const Launch& L, const cask_params& prm, const float* s, const uint8_t* kind,
+                           const int32_t* seed_of, float* weight, const cask_outputs& out, Workspace& ws) {
+    if (L.sh.dtype == CASK_DTYPE_BF16) return run<__nv_bfloat16>(L, prm, s, kind, seed_of, weight, out, ws);
+    return run<float>(L, prm, s, kind, seed_of, weight, out, ws);
+}
+
+}  // namespace cask

@@ -1,0 +1,290 @@
+// Scratch consolidation (Sec. 2.1, 2.4, 2.5): seed selection, cosine assignment of the
+// remaining scratch rows to seeds, group masses and merge weights.
+#include "select.cuh"
+
+namespace cask {
+
+namespace {
+
+constexpr int kTile = 64;
+constexpr int kThreads = 256;
+
+// ---- 1. seeds: the m greatest scratch rows; ordered list of their rows -------------------
+__global__ void __launch_bounds__(kSelThreads) seeds_kernel(const UnitDesc* __restrict__ desc,
+                                                            const float* __restrict__ s,
+                                                            const int32_t* __restrict__ plan,
+                                                            uint8_t* __restrict__ kind,
+                                                            int32_t* __restrict__ seed_of,
+                                                            float* __restrict__ weight,
+                                                            float* __restrict__ sim, int32_t* __restrict__ grp,
+                                                            int32_t* __restrict__ seed_rows,
+                                                            unsigned long long* __restrict__ mass_fx,
+                                                            int32_t* __restrict__ njoin, int max_m) {
+    __shared__ SelectSmem sm;
+    const int u = blockIdx.x;
+    const UnitDesc& ud = desc[u];
+    const int T = ud.T, P = ud.P;
+    const int64_t o = ud.tok_off;
+    int r = max(0, min(plan[u * 8 + CASK_PLAN_R], T - P));
+    int m = max(0, min(plan[u * 8 + CASK_PLAN_M], ud.plan[CASK_PLAN_M]));
+    // a row left as MERGED/SEED by an earlier call on the same arrays is scratch again
+    for (int i = threadIdx.x; i < T; i += blockDim.x) {
+        uint8_t kd = kind[o + i];
+        if (kd == CASK_KIND_SEED || kd == CASK_KIND_MERGED) kind[o + i] = CASK_KIND_DROPPED;
+        seed_of[o + i] = -1;
+        weight[o + i] = 0.f;
+        grp[o + i] = -1;
+        if (sim) sim[o + i] = -2.f;
+    }
+    for (int j = threadIdx.x; j <= max_m; j += blockDim.x) mass_fx[(size_t)u * (max_m + 1) + j] = 0ull;
+    if (threadIdx.x == 0) njoin[u] = 0;
+    __syncthreads();
+    if (m <= 0) return;
+    block_topk_mark(s + o, kind + o, P, T - r, m, CASK_KIND_SEED, sm);
+    // ordered compaction of the seed rows
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    unsigned base = 0;
+    for (int i0 = P; i0 < T - r; i0 += blockDim.x) {
+        int i = i0 + threadIdx.x;
+        bool is = (i < T - r) && kind[o + i] == CASK_KIND_SEED;
+        unsigned bal = __ballot_sync(0xffffffffu, is);
+        __syncthreads();
+        if (lane == 0) sm.warp_cnt[w] = __popc(bal);
+        __syncthreads();
+        unsigned before = 0, all = 0;
+        for (int x = 0; x < nw; ++x) {
+            unsigned c = sm.warp_cnt[x];
+            if (x < w) before += c;
+            all += c;
+        }
+        if (is) {
+            unsigned idx = base + before + __popc(bal & ((1u << lane) - 1u));
+            if (idx < (unsigned)m) {
+                seed_rows[ud.seed_base + idx] = i;
+                seed_of[o + i] = i;
+                grp[o + i] = (int)idx;
+            }
+        }
+        base += all;
+    }
+}
+
+// ---- 2. gather seed keys, their norms and their own mass ---------------------------------
+template <typename T>
+__global__ void seed_gather_kernel(const UnitDesc* __restrict__ desc, Shape sh, const T* __restrict__ K,
+                                   const float* __restrict__ s, const int32_t* __restrict__ plan,
+                                   const int32_t* __restrict__ seed_rows, T* __restrict__ seed_k,
+                                   float* __restrict__ seed_norm, unsigned long long* __restrict__ mass_fx,
+                                   int max_m, float eps) {
+    const int u = blockIdx.y, j = blockIdx.x;
+    const UnitDesc& ud = desc[u];
+    const int m = max(0, min(plan[u * 8 + CASK_PLAN_M], ud.plan[CASK_PLAN_M]));
+    if (j >= m) return;
+    const int row = seed_rows[ud.seed_base + j];
+    const T* src = K + ud.k_off + (int64_t)row * sh.row_stride;
+    T* dst = seed_k + (size_t)(ud.seed_base + j) * sh.d;
+    float n2 = 0.f;
+    for (int c = threadIdx.x; c < sh.d; c += 32) {
+        T x = src[c];
+        dst[c] = x;
+        float f = Elem<T>::ld(&x);
+        n2 = fmaf(f, f, n2);
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, off);
+    if (threadIdx.x == 0) {
+        seed_norm[ud.seed_base + j] = sqrtf(n2);
+        atomicAdd(&mass_fx[(size_t)u * (max_m + 1) + j], mass_to_fx(s[ud.tok_off + row] + eps));
+    }
+}
+
+// ---- 3. assignment: cosine of every scratch row against every seed, argmax, threshold -----
+template <typename T>
+__global__ void __launch_bounds__(kThreads) assign_simt_kernel(
+    const UnitDesc* __restrict__ desc, Shape sh, const T* __restrict__ K, const float* __restrict__ s,
+    const int32_t* __restrict__ plan, const int32_t* __restrict__ seed_rows, const T* __restrict__ seed_k,
+    const float* __restrict__ seed_norm, uint8_t* __restrict__ kind, int32_t* __restrict__ seed_of,
+    float* __restrict__ sim, int32_t* __restrict__ grp, unsigned long long* __restrict__ mass_fx,
+    int32_t* __restrict__ njoin, int max_m, float tau, float eps) {
+    extern __shared__ float smem[];
+    const int u = blockIdx.y;
+    const UnitDesc& ud = desc[u];
+    const int T_ = ud.T, P = ud.P;
+    const int r = max(0, min(plan[u * 8 + CASK_PLAN_R], T_ - P));
+    const int m = max(0, min(plan[u * 8 + CASK_PLAN_M], ud.plan[CASK_PLAN_M]));
+    const int lo = P + blockIdx.x * kTile, hi = T_ - r;
+    if (m <= 0 || lo >= hi) return;
+    const int d = sh.d, pitch = d + 1;
+    float* St = smem;
+    float* Rt = smem + kTile * pitch;
+    float* rnorm = Rt + kTile * pitch;     // [64] norms of the stationary rows
+    const int ty = threadIdx.x / 16, tx = threadIdx.x % 16;
+    const int nrows = min(kTile, hi - lo);
+
+    // stationary tile: 64 candidate rows
+    {
+        const int vec_per_row = d / 8;
+        for (int idx = threadIdx.x; idx < kTile * vec_per_row; idx += kThreads) {
+            int rr = idx / vec_per_row, c8 = (idx % vec_per_row) * 8;
+#pragma unroll
+            for (int t = 0; t < 8; ++t)
+                St[rr * pitch + c8 + t] =
+                    (rr < nrows) ? Elem<T>::ld(K + ud.k_off + (int64_t)(lo + rr) * sh.row_stride + c8 + t) : 0.f;
+        }
+    }
+    __syncthreads();
+    {
+        // 4 threads per row, fixed combination order
+        int rr = threadIdx.x / 4, part = threadIdx.x % 4;
+        float n2 = 0.f;
+        for (int c = part; c < d; c += 4) n2 = fmaf(St[rr * pitch + c], St[rr * pitch + c], n2);
+        n2 += __shfl_xor_sync(0xffffffffu, n2, 1);
+        n2 += __shfl_xor_sync(0xffffffffu, n2, 2);
+        if (part == 0) rnorm[rr] = sqrtf(n2);
+    }
+    float best[4];
+    int best_u[4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a) { best[a] = -INFINITY; best_u[a] = -1; }
+
+    for (int u0 = 0; u0 < m; u0 += kTile) {
+        __syncthreads();
+        const int vec_per_row = d / 8;
+        const int nseed = min(kTile, m - u0);
+        for (int idx = threadIdx.x; idx < kTile * vec_per_row; idx += kThreads) {
+            int rr = idx / vec_per_row, c8 = (idx % vec_per_row) * 8;
+#pragma unroll
+            for (int t = 0; t < 8; ++t)
+                Rt[rr * pitch + c8 + t] =
+                    (rr < nseed) ? Elem<T>::ld(seed_k + (size_t)(ud.seed_base + u0 + rr) * d + c8 + t) : 0.f;
+        }
+        __syncthreads();
+        float acc[4][4];
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+#pragma unroll 4
+        for (int c = 0; c < d; ++c) {
+            float sa[4], rb[4];
+#pragma unroll
+            for (int a = 0; a < 4; ++a) sa[a] = St[(ty + 16 * a) * pitch + c];
+#pragma unroll
+            for (int b = 0; b < 4; ++b) rb[b] = Rt[(tx + 16 * b) * pitch + c];
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(sa[a], rb[b], acc[a][b]);
+        }
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            int su = u0 + tx + 16 * b;
+            if (su >= m) continue;
+            float nu = seed_norm[ud.seed_base + su];
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+                float nj = rnorm[ty + 16 * a];
+                float sm_ = (nj > 0.f && nu > 0.f) ? acc[a][b] / (nj * nu) : 0.f;
+                if (sm_ > best[a]) { best[a] = sm_; best_u[a] = su; }
+            }
+        }
+    }
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+#pragma unroll
+        for (int off = 8; off >= 1; off >>= 1) {
+            float ob = __shfl_xor_sync(0xffffffffu, best[a], off);
+            int ou = __shfl_xor_sync(0xffffffffu, best_u[a], off);
+            if (ou >= 0 && (ob > best[a] || (ob == best[a] && ou < best_u[a]) || best_u[a] < 0)) {
+                best[a] = ob;
+                best_u[a] = ou;
+            }
+        }
+        int rr = ty + 16 * a;
+        int i = lo + rr;
+        if (tx == 0 && rr < nrows && kind[ud.tok_off + i] == CASK_KIND_DROPPED) {
+            if (sim) sim[ud.tok_off + i] = best[a];
+            unsigned long long fx = mass_to_fx(s[ud.tok_off + i] + eps);
+            if (best_u[a] >= 0 && best[a] >= tau) {
+                kind[ud.tok_off + i] = CASK_KIND_MERGED;
+                seed_of[ud.tok_off + i] = seed_rows[ud.seed_base + best_u[a]];
+                grp[ud.tok_off + i] = best_u[a];
+                atomicAdd(&mass_fx[(size_t)u * (max_m + 1) + best_u[a]], fx);
+                atomicAdd(&njoin[u], 1);
+            } else {
+                atomicAdd(&mass_fx[(size_t)u * (max_m + 1) + max_m], fx);
+            }
+        }
+    }
+}
+
+// ---- 4. merge weights w_i = a_i / m_G, lost mass, status ---------------------------------
+__global__ void weights_kernel(const UnitDesc* __restrict__ desc, const float* __restrict__ s,
+                               const int32_t* __restrict__ plan, const int32_t* __restrict__ grp,
+                               const unsigned long long* __restrict__ mass_fx,
+                               const int32_t* __restrict__ njoin, float* __restrict__ weight,
+                               int32_t* __restrict__ unit_status, float* __restrict__ lost_mass, int max_m,
+                               float eps) {
+    const int u = blockIdx.y;
+    const UnitDesc& ud = desc[u];
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    const unsigned long long* mf = mass_fx + (size_t)u * (max_m + 1);
+    if (i < ud.T) {
+        int gidx = grp[ud.tok_off + i];
+        if (gidx >= 0 && gidx < max_m) weight[ud.tok_off + i] = (s[ud.tok_off + i] + eps) / fx_to_mass(mf[gidx]);
+    }
+    if (i == 0) {
+        int fl = plan[u * 8 + CASK_PLAN_FLAGS];
+        if ((fl & CASK_ST_DECODE_CONSOLIDATED) && njoin[u] == 0) fl |= CASK_ST_MERGE_INACTIVE;
+        unit_status[u] = fl;
+        lost_mass[u] = fx_to_mass(mf[max_m]);
+    }
+}
+
+template <typename T>
+cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const int32_t* plan, uint8_t* kind,
+                int32_t* seed_of, float* weight, float* sim, int32_t* unit_status, float* lost_mass,
+                Workspace& ws) {
+    const Shape& sh = L.sh;
+    const int max_m = L.max_m;
+    {
+        Timed t(L, KID_SEEDS);
+        seeds_kernel<<<sh.n_units, kSelThreads, 0, L.stream>>>(L.desc, s, plan, kind, seed_of, weight, sim,
+                                                               ws.grp, ws.seed_rows, ws.mass_fx, ws.njoin, max_m);
+    }
+    if (max_m > 0) {
+        {
+            Timed t(L, KID_SEED_GATHER);
+            seed_gather_kernel<T><<<dim3(max_m, sh.n_units), 32, 0, L.stream>>>(
+                L.desc, sh, (const T*)L.k, s, plan, ws.seed_rows, (T*)ws.seed_k, ws.seed_norm, ws.mass_fx, max_m,
+                prm.eps);
+        }
+        const size_t smem = ((size_t)2 * kTile * (sh.d + 1) + kTile) * sizeof(float);
+        cudaError_t e = cudaFuncSetAttribute(assign_simt_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)smem);
+        if (e != cudaSuccess) return e;
+        const int max_nd = L.max_T;   // upper bound on decode rows of any unit
+        Timed t(L, KID_ASSIGN);
+        assign_simt_kernel<T><<<dim3((max_nd + kTile - 1) / kTile, sh.n_units), kThreads, smem, L.stream>>>(
+            L.desc, sh, (const T*)L.k, s, plan, ws.seed_rows, (const T*)ws.seed_k, ws.seed_norm, kind, seed_of,
+            sim, ws.grp, ws.mass_fx, ws.njoin, max_m, prm.tau, prm.eps);
+    }
+    {
+        Timed t(L, KID_WEIGHTS);
+        weights_kernel<<<dim3((L.max_T + 255) / 256, sh.n_units), 256, 0, L.stream>>>(
+            L.desc, s, plan, ws.grp, ws.mass_fx, ws.njoin, weight, unit_status, lost_mass, max_m, prm.eps);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_consolidate(const Launch& L, const cask_params& prm, const float* s, const int32_t* plan,
+                               uint8_t* kind, int32_t* seed_of, float* weight, float* sim,
+                               int32_t* unit_status, float* lost_mass, Workspace& ws) {
+    if (L.sh.dtype == CASK_DTYPE_BF16)
+        return run<__nv_bfloat16>(L, prm, s, plan, kind, seed_of, weight, sim, unit_status, lost_mass, ws);
+    return run<float>(L, prm, s, plan, kind, seed_of, weight, sim, unit_status, lost_mass, ws);
+}
+
+}  // namespace cask

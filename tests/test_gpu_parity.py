@@ -1,0 +1,313 @@
+"""GPU parity: the CUDA library against the CPU oracle, element by element, through the C-ABI."""
+import numpy as np
+import pytest
+
+from paper_2604_10900_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def _small(name, **kw):
+    """A benchmark-shaped workload cut down so the oracle finishes in seconds."""
+    return wl.WORKLOADS[name].with_(**kw)
+
+
+def _run(w, units=None, tau=0.9, **prm):
+    import gpu_harness as gh
+    hb = wl.make_batch(w, units)
+    run = gh.GpuRun(hb, tau=tau, **prm)
+    g = run.event()
+    o = gh.run_oracle(hb, tau=tau, causal=prm.get("causal", 1), gamma=prm.get("gamma", 0.5))
+    st = gh.compare_event(hb, g, o, tau=tau)
+    return hb, run, g, o, st
+
+
+def test_tiny_config_whole_event():
+    """Config 1: fp32 cache, d=64, 1024 rows, budget 128 (both heads)."""
+    hb, run, g, o, st = _run(wl.WORKLOADS["tiny"])
+    assert st["cascaded"] == 0 and st["merged_elems"] > 0
+    assert (g["n_out"] == 128).all()
+    assert not run.ctx.used_tensor_path
+
+
+@pytest.mark.parametrize("score_path", [0, 1])
+def test_reasoning_shape_bf16(score_path):
+    """Config-2 shape (d=128, g=7, W=64, bf16, outlier channels, geometric clusters), 2 layers, ragged tail."""
+    w = _small("reasoning8k_b384", layers=2, decode=2048 + 37)
+    hb, run, g, o, st = _run(w, score_path=score_path)
+    assert st["cascaded"] <= 1
+    assert st["merged_elems"] > 0
+    assert st["max_score_rel"] < 1e-5
+
+
+@pytest.mark.parametrize("score_path", [0, 1])
+def test_long_reasoning_shape_bf16(score_path):
+    """Config-3 shape (g=4, W=128 -> 512 query rows), several key tiles and a ragged last tile."""
+    w = _small("reasoning32k_b512", layers=1, kv_heads=3, decode=4096 + 77)
+    hb, run, g, o, st = _run(w, score_path=score_path)
+    assert st["cascaded"] <= 1
+    assert (g["n_out"] == 512).all()
+
+
+def test_prompt_heavy_two_stage():
+    """Config-4 shape: prefix eviction fires before decode consolidation."""
+    w = _small("prompt_heavy", layers=1, kv_heads=2, prefix=3072, decode=1024, budget=1024, reserve=256)
+    hb, run, g, o, st = _run(w)
+    from oracle import cask_oracle as orc
+    assert (g["unit_status"] & orc.PREFIX_EVICTED).all() and (g["unit_status"] & orc.DECODE_CONSOLIDATED).all()
+    assert (g["n_out"] == 1024).all()
+
+
+@pytest.mark.parametrize("reserve,exhausted", [(66, False), (65, True), (64, True)])
+def test_prefix_budget_exhausted_boundary(reserve, exhausted):
+    """Config-4 variant around B_d = r + 2 (Sec. 5.2: the available slots collapse)."""
+    w = _small("prompt_heavy_boundary", layers=1, kv_heads=1, prefix=2048, decode=512, budget=512, reserve=reserve)
+    hb, run, g, o, st = _run(w)
+    from oracle import cask_oracle as orc
+    assert bool(g["unit_status"][0] & orc.PREFIX_BUDGET_EXHAUSTED) == exhausted
+    assert g["n_out"][0] == 512
+    if exhausted:
+        assert not np.isin(g["kind"], (4, 5)).any()
+
+
+def test_ragged_batch_mixed_outcomes():
+    """Units of different length and budget in one call: under budget, prefix-only, decode-active."""
+    base = wl.WORKLOADS["tiny"].with_(dtype=wl.DTYPE_BF16, head_dim=128, group=2, window=8)
+    import gpu_harness as gh
+    parts = []
+    specs = [(128, 896, 128, 64), (16, 40, 64, 32), (300, 0, 128, 64), (64, 131, 96, 90), (10, 500, 700, 100)]
+    ks, vs, qs, T, P, B, R = [], [], [], [], [], [], []
+    for i, (p, nd, b, r) in enumerate(specs):
+        w = base.with_(prefix=p, decode=nd, budget=b, reserve=r)
+        k, v, q = wl.make_unit(w, i, 0, 0)
+        ks.append(k); vs.append(v); qs.append(q[None])
+        T.append(p + nd); P.append(p); B.append(b); R.append(r)
+    tok = np.concatenate([[0], np.cumsum(T)]).astype(np.int64)
+    hb = wl.Batch(wl=base, k=np.concatenate(ks), v=np.concatenate(vs), q=np.concatenate(qs),
+                  T=np.array(T, np.int32), P=np.array(P, np.int32), B=np.array(B, np.int32),
+                  reserve=np.array(R, np.int32), tok_off=tok, unit_ids=[(i, 0, 0) for i in range(len(T))])
+    run = gh.GpuRun(hb)
+    g = run.event()
+    o = gh.run_oracle(hb)
+    st = gh.compare_event(hb, g, o)
+    from oracle import cask_oracle as orc
+    assert g["unit_status"][1] & orc.NOOP_UNDER_BUDGET and g["n_out"][1] == 56
+    assert g["unit_status"][4] & orc.NOOP_UNDER_BUDGET
+    assert g["n_out"][2] == 64          # prefix-only event leaves the reserve free
+    # unit independence: each unit alone gives the same bytes as inside the batch
+    for u in (0, 3):
+        one = wl.Batch(wl=base, k=ks[u], v=vs[u], q=qs[u], T=hb.T[u:u + 1], P=hb.P[u:u + 1], B=hb.B[u:u + 1],
+                       reserve=hb.reserve[u:u + 1], tok_off=np.array([0, T[u]], np.int64), unit_ids=[(u, 0, 0)])
+        g1 = gh.GpuRun(one).event()
+        a = int(tok[u])
+        assert np.array_equal(g1["s"], g["s"][a:a + T[u]])
+        assert np.array_equal(g1["kind"], g["kind"][a:a + T[u]])
+        n = int(g1["n_out"][0])
+        assert np.array_equal(g1["k_out"][0][:n], g["k_out"][u][:n])
+        assert np.array_equal(g1["v_out"][0][:n], g["v_out"][u][:n])
+
+
+@pytest.mark.parametrize("tau", [-1.0, 1.5])
+def test_tau_extremes(tau):
+    """tau = -1 merges every scratch row (no lost mass); tau > 1 is plain top-k eviction."""
+    hb, run, g, o, st = _run(wl.WORKLOADS["tiny"], tau=tau)
+    if tau < 0:
+        assert (g["lost_mass"] == 0).all()
+        assert not ((g["kind"] == 0) & (np.arange(len(g["kind"])) % 1024 >= 128)).any()
+    else:
+        from oracle import cask_oracle as orc
+        assert (g["unit_status"] & orc.MERGE_INACTIVE).all() and not (g["kind"] == 5).any()
+
+
+def test_non_causal_and_other_gamma():
+    _run(wl.WORKLOADS["tiny"], causal=0)
+    _run(wl.WORKLOADS["tiny"], gamma=0.25)
+
+
+def test_strided_rows_and_fp32_d128():
+    import gpu_harness as gh
+    w = wl.WORKLOADS["tiny"].with_(head_dim=128)
+    hb = wl.make_batch(w)
+    g = gh.GpuRun(hb, row_stride=160).event()
+    o = gh.run_oracle(hb)
+    gh.compare_event(hb, g, o)
+    wb = wl.WORKLOADS["tiny"].with_(dtype=wl.DTYPE_BF16)       # bf16 with d = 64: SIMT path
+    hb = wl.make_batch(wb)
+    run = gh.GpuRun(hb, row_stride=72)
+    g = run.event()
+    gh.compare_event(hb, g, gh.run_oracle(hb))
+
+
+def test_supplied_normalisers():
+    """lse_in from the oracle: the normaliser pass is skipped and scores still match."""
+    import gpu_harness as gh
+    w = wl.WORKLOADS["tiny"]
+    hb = wl.make_batch(w)
+    o = gh.run_oracle(hb)
+    from oracle import cask_oracle as orc
+    _, lse = orc.score_batch(hb.k, hb.q, hb.tok_off)
+    run = gh.GpuRun(hb, lse_in=lse.reshape(hb.n_units, -1))
+    n0 = run.ctx.launches
+    g = run.event()
+    gh.compare_event(hb, g, o)
+    run2 = gh.GpuRun(hb)
+    run2.event()
+    assert run.ctx.launches - n0 < run2.ctx.launches       # one pass fewer
+
+
+def test_deterministic_and_staged_equals_fused():
+    """Same inputs twice -> same bytes; the five staged calls give the event's bytes."""
+    import gpu_harness as gh
+    import torch
+    w = _small("reasoning8k_b384", layers=1, kv_heads=2, decode=1500)
+    hb = wl.make_batch(w)
+    run = gh.GpuRun(hb)
+    g1 = run.event()
+    g2 = run.event()
+    for k in g1:
+        assert np.array_equal(g1[k], g2[k]), k
+    cb = run.cb
+    st = gh.GpuRun(hb)
+    o = st.out
+    cb.cask_score(st.ctx, st.batch, st.prm, o["s"], o["lse"], st.ws, st.ws_bytes)
+    cb.cask_prefix_evict(st.ctx, st.batch, st.prm, o["s"], o["kind"], o["plan"], st.ws, st.ws_bytes)
+    cb.cask_select_core(st.ctx, st.batch, st.prm, o["s"], o["plan"], o["kind"], st.ws, st.ws_bytes)
+    cb.cask_consolidate_scratch(st.ctx, st.batch, st.prm, o["s"], o["plan"], o["kind"], o["seed_of"], o["weight"],
+                                o["sim"], o["unit_status"], o["lost_mass"], st.ws, st.ws_bytes)
+    cb.cask_compact(st.ctx, st.batch, st.prm, o["s"], o["kind"], o["seed_of"], o["weight"], st.out_struct, st.ws,
+                    st.ws_bytes)
+    torch.cuda.synchronize()
+    g3 = st.numpy_outputs()
+    for k in g1:
+        assert np.array_equal(g1[k], g3[k]), k
+
+
+def test_stages_with_oracle_intermediates_injected():
+    """Each stage fed the oracle's upstream results (as fp32): selections must match with no exemption."""
+    import gpu_harness as gh
+    import torch
+    from oracle import cask_oracle as orc
+    w = _small("reasoning8k_b512", layers=1, kv_heads=2, decode=3000)
+    hb = wl.make_batch(w)
+    run = gh.GpuRun(hb)
+    cb, o = run.cb, run.out
+    kf, vf, qf = (wl.as_float32(x, w.dtype) for x in (hb.k, hb.v, hb.q))
+    s64, _ = orc.score_batch(kf, qf, hb.tok_off)
+    s32 = s64.astype(np.float32)
+    sd = s32.astype(np.float64)              # the oracle works on exactly the values the GPU gets
+    s_dev = run.dev_f32(s32)
+    cb.cask_prefix_evict(run.ctx, run.batch, run.prm, s_dev, o["kind"], o["plan"], run.ws, run.ws_bytes)
+    cb.cask_select_core(run.ctx, run.batch, run.prm, s_dev, o["plan"], o["kind"], run.ws, run.ws_bytes)
+    torch.cuda.synchronize()
+    kind_g = o["kind"].cpu().numpy()
+    plan_g = o["plan"].cpu().numpy()
+    for u in range(hb.n_units):
+        a, T, P = int(hb.tok_off[u]), int(hb.T[u]), int(hb.P[u])
+        pl = orc.plan(T, P, int(hb.B[u]), int(hb.reserve[u]), w.window, 0.5)
+        assert np.array_equal(plan_g[u], pl)
+        kind = np.zeros(T, np.uint8)
+        orc.prefix_evict(sd[a:a + T], P, pl, kind)
+        orc.select_core(sd[a:a + T], T, P, pl, kind)
+        assert np.array_equal(kind_g[a:a + T], kind), f"unit {u}"
+    # consolidation on the oracle's kinds
+    cb.cask_consolidate_scratch(run.ctx, run.batch, run.prm, s_dev, o["plan"], o["kind"], o["seed_of"], o["weight"],
+                                o["sim"], o["unit_status"], o["lost_mass"], run.ws, run.ws_bytes)
+    torch.cuda.synchronize()
+    kind_g2, seed_g, sim_g, w_g = (o[x].cpu().numpy() for x in ("kind", "seed_of", "sim", "weight"))
+    inj_kind, inj_seed, inj_w = kind_g2.copy(), seed_g.copy(), w_g.astype(np.float64)
+    for u in range(hb.n_units):
+        a, T, P = int(hb.tok_off[u]), int(hb.T[u]), int(hb.P[u])
+        kind = kind_g[a:a + T].copy()
+        c = orc.consolidate(kf[a:a + T], sd[a:a + T], P, plan_g[u], kind, tau=0.9, eps=float(np.float32(1e-9)))
+        assert np.array_equal(kind == 4, kind_g2[a:a + T] == 4), "seed sets (same scores) must match exactly"
+        near = (np.abs(c["sim"] - 0.9) <= gh.SIM_BAND) | ((c["sim2"] > -1.5) & (c["sim"] - c["sim2"] <= gh.SIM_BAND))
+        bad = (kind != kind_g2[a:a + T]) | (c["seed_of"] != seed_g[a:a + T])
+        assert not (bad & ~near).any(), f"unit {u}: non-exempt assignment differences"
+        has = c["sim"] > -1.5
+        assert np.abs(sim_g[a:a + T][has] - c["sim"][has]).max() < 2e-6
+        same = ~bad
+        assert np.allclose(w_g[a:a + T][same], c["weight"][same], rtol=2e-5, atol=1e-9)
+        inj_kind[a:a + T], inj_seed[a:a + T], inj_w[a:a + T] = kind, c["seed_of"], c["weight"]
+    # compaction on the oracle's kinds / seeds / weights
+    kd, so, wt = run.dev_arr(inj_kind, np.uint8), run.dev_arr(inj_seed, np.int32), run.dev_f32(inj_w)
+    cb.cask_compact(run.ctx, run.batch, run.prm, s_dev, kd, so, wt, run.out_struct, run.ws, run.ws_bytes)
+    torch.cuda.synchronize()
+    g = run.numpy_outputs()
+    for u in range(hb.n_units):
+        a, T = int(hb.tok_off[u]), int(hb.T[u])
+        oc = orc.compact(kf[a:a + T], vf[a:a + T], inj_kind[a:a + T], inj_seed[a:a + T],
+                         inj_w[a:a + T].astype(np.float32).astype(np.float64), sd[a:a + T],
+                         eps=float(np.float32(1e-9)))
+        n = oc["n_out"]
+        assert g["n_out"][u] == n
+        assert np.array_equal(g["slot_src"][u][:n], oc["slot_src"])
+        assert np.array_equal(g["slot_kind"][u][:n], oc["slot_kind"])
+        assert np.array_equal(g["assign"][a:a + T], oc["assign"])
+        assert np.allclose(g["slot_mass"][u][:n], oc["slot_mass"], rtol=2e-5)
+        err = np.abs(g["k_out"][u][:n].astype(np.float64) - oc["k_out"])
+        assert (err <= np.maximum(2e-2, 2.0 ** -7 * np.abs(oc["k_out"]))).all()
+        errv = np.abs(g["v_out"][u][:n].astype(np.float64) - oc["v_out"])
+        assert (errv <= np.maximum(2e-2, 2.0 ** -7 * np.abs(oc["v_out"]))).all()
+
+
+def test_bad_arguments_are_refused_on_the_host_before_any_launch():
+    import gpu_harness as gh
+    hb = wl.make_batch(wl.WORKLOADS["tiny"])
+    run = gh.GpuRun(hb)
+    cb = run.cb
+    n0 = run.ctx.launches
+
+    def rc(**chg):
+        b, keep = cb.make_batch(run.dev["k"], run.dev["v"], run.dev["q"],
+                                chg.get("T", hb.T), chg.get("P", hb.P), chg.get("B", hb.B),
+                                chg.get("reserve", hb.reserve), hb.tok_off, chg.get("d", 64), 4,
+                                chg.get("W", 16), chg.get("dtype", 1), row_stride=chg.get("row_stride"),
+                                page_size=chg.get("page_size", 0))
+        if chg.get("null_k"):
+            b.k = None
+        return cb.cask_compress_event(run.ctx, b, chg.get("prm", run.prm), run.out_struct,
+                                      chg.get("ws", run.ws), chg.get("ws_bytes", run.ws_bytes), check=False)
+
+    assert rc() == cb.OK
+    n1 = run.ctx.launches
+    assert rc(null_k=True) == cb.ERR_NULL
+    assert rc(B=np.array([0, 128], np.int32)) == cb.ERR_SHAPE
+    assert rc(P=np.array([2000, 128], np.int32)) == cb.ERR_SHAPE
+    assert rc(W=2000) == cb.ERR_SHAPE
+    assert rc(reserve=np.array([129, 0], np.int32)) == cb.ERR_SHAPE
+    assert rc(d=60) == cb.ERR_SHAPE
+    assert rc(row_stride=66) == cb.ERR_ALIGN
+    assert rc(page_size=16) == cb.ERR_UNSUPPORTED
+    assert rc(ws_bytes=1024) == cb.ERR_WORKSPACE
+    assert rc(prm=cb.params(gamma=1.5)) == cb.ERR_PARAM
+    assert rc(prm=cb.params(eps=0.0)) == cb.ERR_PARAM
+    small = cb.make_outputs(run.out, 64)
+    b, keep = cb.make_batch(run.dev["k"], run.dev["v"], run.dev["q"], hb.T, hb.P, hb.B, hb.reserve, hb.tok_off,
+                            64, 4, 16, 1)
+    assert cb.cask_compress_event(run.ctx, b, run.prm, small, run.ws, run.ws_bytes, check=False) == cb.ERR_SHAPE
+    import torch
+    torch.cuda.synchronize()
+    assert run.ctx.launches == n1 > n0       # the refused calls launched nothing; the context is still usable
+    run.event()
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    """cask_compress_event_host (host K/V/Q and host outputs) gives the bytes of the device call."""
+    import gpu_harness as gh
+    import torch
+    w = _small("reasoning8k_b384", layers=1, kv_heads=2, decode=1000)
+    hb = wl.make_batch(w)
+    run = gh.GpuRun(hb)
+    g = run.event()
+    cb = run.cb
+    hbatch, keep = cb.make_batch(hb.k, hb.v, hb.q, hb.T, hb.P, hb.B, hb.reserve, hb.tok_off, w.head_dim, w.group,
+                                 w.window, w.dtype)
+    nbytes = cb.cask_host_event_device_bytes(hbatch, run.prm, run.Bmax)
+    assert nbytes > 0
+    dev = torch.empty(nbytes, dtype=torch.uint8, device="cuda:0")
+    ho = {k: (np.zeros(tuple(t.shape), np.uint16) if t.dtype == torch.bfloat16 else np.zeros(tuple(t.shape), t.cpu().numpy().dtype))
+          for k, t in run.out.items()}
+    cb.cask_compress_event_host(run.ctx, hbatch, run.prm, cb.make_outputs(ho, run.Bmax), dev, nbytes)
+    for k in g:
+        got = wl.bf16_bits_to_f32(ho[k]) if ho[k].dtype == np.uint16 else ho[k]
+        assert np.array_equal(got, g[k]), k
