@@ -148,6 +148,16 @@ const char* cask_strerror(int code);
 const char* cask_last_cuda_error(const cask_ctx* ctx);
 /* Kernels launched by this context since creation (every call adds its own). */
 int64_t cask_launch_count(const cask_ctx* ctx);
+/*
+ * Optional per-kernel timing.  While enabled, every kernel launch of this context is
+ * bracketed by a CUDA event pair on the context's stream.  cask_profile_read waits for
+ * the recorded events, adds up the elapsed milliseconds and launch counts per kernel id
+ * (arrays of cask_kernel_count() entries, HOST) and forgets them.
+ */
+int cask_profile_enable(cask_ctx* ctx, int on);
+int cask_profile_read(cask_ctx* ctx, float* ms, int64_t* launches);
+int cask_kernel_count(void);
+const char* cask_kernel_name(int id);
 /* 1 if the last cask_score / cask_compress_event used the tensor-core kernels. */
 int cask_last_score_path_tensor(const cask_ctx* ctx);
 

@@ -26,7 +26,8 @@ DTYPE_BF16, DTYPE_FP32 = 0, 1
 
 EXPORTS = (
     "cask_create", "cask_destroy", "cask_set_stream", "cask_strerror", "cask_last_cuda_error",
-    "cask_launch_count", "cask_last_score_path_tensor", "cask_workspace_bytes", "cask_plan_host",
+    "cask_launch_count", "cask_last_score_path_tensor", "cask_profile_enable", "cask_profile_read",
+    "cask_kernel_count", "cask_kernel_name", "cask_workspace_bytes", "cask_plan_host",
     "cask_score", "cask_prefix_evict", "cask_select_core", "cask_consolidate_scratch", "cask_compact",
     "cask_compress_event", "cask_host_event_device_bytes", "cask_compress_event_host",
 )
@@ -83,6 +84,10 @@ def lib():
         L.cask_launch_count.argtypes = [vp]
         L.cask_launch_count.restype = C.c_int64
         L.cask_last_score_path_tensor.argtypes = [vp]
+        L.cask_profile_enable.argtypes = [vp, i32]
+        L.cask_profile_read.argtypes = [vp, vp, vp]
+        L.cask_kernel_name.argtypes = [i32]
+        L.cask_kernel_name.restype = C.c_char_p
         L.cask_workspace_bytes.argtypes = [PB, PP]
         L.cask_workspace_bytes.restype = sz
         L.cask_plan_host.argtypes = [PB, PP, vp]
@@ -194,6 +199,20 @@ class Context:
     @property
     def launches(self) -> int:
         return int(lib().cask_launch_count(self.handle))
+
+    def profile_enable(self, on: bool = True):
+        lib().cask_profile_enable(self.handle, int(on))
+
+    def profile_read(self) -> Dict[str, Dict]:
+        """{kernel name: {"ms": total, "launches": n}} since the last read."""
+        n = lib().cask_kernel_count()
+        ms = np.zeros(n, np.float32)
+        cnt = np.zeros(n, np.int64)
+        rc = lib().cask_profile_read(self.handle, ms.ctypes.data, cnt.ctypes.data)
+        if rc != OK:
+            raise CaskError(rc, self.handle)
+        return {lib().cask_kernel_name(i).decode(): dict(ms=float(ms[i]), launches=int(cnt[i]))
+                for i in range(n) if cnt[i]}
 
     @property
     def used_tensor_path(self) -> bool:

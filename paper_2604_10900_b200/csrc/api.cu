@@ -10,6 +10,31 @@
 
 using namespace cask;
 
+namespace {
+struct ProfRecord { int id; cudaEvent_t a, b; };
+struct ProfImpl {
+    std::vector<ProfRecord> live;     // recorded, not yet read
+    std::vector<cudaEvent_t> pool;    // events ready for reuse
+    cudaEvent_t get() {
+        if (!pool.empty()) { cudaEvent_t e = pool.back(); pool.pop_back(); return e; }
+        cudaEvent_t e = nullptr;
+        cudaEventCreate(&e);
+        return e;
+    }
+};
+}  // namespace
+
+void cask::Profiler::begin(int id, cudaStream_t st) {
+    ProfImpl* pi = (ProfImpl*)impl;
+    ProfRecord r{id, pi->get(), pi->get()};
+    cudaEventRecord(r.a, st);
+    pi->live.push_back(r);
+}
+void cask::Profiler::end(cudaStream_t st) {
+    ProfImpl* pi = (ProfImpl*)impl;
+    cudaEventRecord(pi->live.back().b, st);
+}
+
 struct cask_ctx {
     int device = 0;
     cudaStream_t stream = nullptr;
@@ -21,6 +46,8 @@ struct cask_ctx {
     cudaError_t last_err = cudaSuccess;
     int last_tc = 0;
     void* tmap_encode = nullptr;     // cuTensorMapEncodeTiled, resolved at creation
+    Profiler prof;
+    ProfImpl prof_impl;
 };
 
 namespace {
@@ -210,6 +237,7 @@ int prepare(cask_ctx* ctx, const cask_batch* b, const cask_params* p, void* ws, 
     L.max_T = z.max_T; L.max_m = z.max_m; L.max_chunks = z.max_chunks; L.total_chunks = z.total_chunks;
     L.max_P = z.max_P; L.max_B = z.max_B; L.sum_T = z.sum_T;
     L.launches = &ctx->launches;
+    L.prof = &ctx->prof;
     return CASK_OK;
 }
 
@@ -239,6 +267,7 @@ int cask_create(cask_ctx** out, int device, void* cuda_stream) {
     if (!c) return CASK_ERR_CUDA;
     c->device = device;
     c->stream = (cudaStream_t)cuda_stream;
+    c->prof.impl = &c->prof_impl;
     e = cudaEventCreateWithFlags(&c->staged, cudaEventDisableTiming);
     if (e != cudaSuccess) { delete c; return CASK_ERR_CUDA; }
     cudaDriverEntryPointQueryResult qres;
@@ -258,6 +287,8 @@ int cask_destroy(cask_ctx* ctx) {
     if (ctx->staged_pending) cudaEventSynchronize(ctx->staged);
     if (ctx->pinned) cudaFreeHost(ctx->pinned);
     if (ctx->staged) cudaEventDestroy(ctx->staged);
+    for (ProfRecord& r : ctx->prof_impl.live) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+    for (cudaEvent_t e : ctx->prof_impl.pool) cudaEventDestroy(e);
     delete ctx;
     return CASK_OK;
 }
@@ -288,6 +319,41 @@ const char* cask_last_cuda_error(const cask_ctx* ctx) {
 }
 
 int64_t cask_launch_count(const cask_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int cask_profile_enable(cask_ctx* ctx, int on) {
+    if (!ctx) return CASK_ERR_NULL;
+    ctx->prof.on = on != 0;
+    return CASK_OK;
+}
+
+int cask_kernel_count(void) { return KID_COUNT; }
+
+const char* cask_kernel_name(int id) {
+    static const char* names[KID_COUNT] = {"score_norm", "row_combine", "score_mass", "prefix_evict",
+                                           "select_core", "seeds", "seed_gather", "assign", "weights",
+                                           "slot_scan", "gather_merge"};
+    return (id >= 0 && id < KID_COUNT) ? names[id] : "";
+}
+
+int cask_profile_read(cask_ctx* ctx, float* ms, int64_t* launches) {
+    if (!ctx || !ms || !launches) return CASK_ERR_NULL;
+    for (int i = 0; i < KID_COUNT; ++i) { ms[i] = 0.f; launches[i] = 0; }
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    for (ProfRecord& r : ctx->prof_impl.live) {
+        e = cudaEventSynchronize(r.b);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+        float t = 0.f;
+        e = cudaEventElapsedTime(&t, r.a, r.b);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+        ms[r.id] += t;
+        launches[r.id] += 1;
+        ctx->prof_impl.pool.push_back(r.a);
+        ctx->prof_impl.pool.push_back(r.b);
+    }
+    ctx->prof_impl.live.clear();
+    return CASK_OK;
+}
 int cask_last_score_path_tensor(const cask_ctx* ctx) { return ctx ? ctx->last_tc : 0; }
 
 size_t cask_workspace_bytes(const cask_batch* batch, const cask_params* params) {
