@@ -38,6 +38,7 @@ def test_reasoning_shape_bf16(score_path):
     assert st["cascaded"] <= 1
     assert st["merged_elems"] > 0
     assert st["max_score_rel"] < 1e-5
+    assert run.ctx.used_tensor_path == (score_path == 0)
 
 
 @pytest.mark.parametrize("score_path", [0, 1])
@@ -47,6 +48,8 @@ def test_long_reasoning_shape_bf16(score_path):
     hb, run, g, o, st = _run(w, score_path=score_path)
     assert st["cascaded"] <= 1
     assert (g["n_out"] == 512).all()
+    assert run.ctx.used_tensor_path == (score_path == 0)
+    print("score path", score_path, "max rel err", st["max_score_rel"], "exempt rows", st["exempt_rows"], "flipped", st["flipped_rows"])
 
 
 def test_prompt_heavy_two_stage():
