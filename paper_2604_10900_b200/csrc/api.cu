@@ -204,7 +204,7 @@ int prepare(cask_ctx* ctx, const cask_batch* b, const cask_params* p, void* ws, 
         if (e != cudaSuccess) return fail_cuda(ctx, e);
         ctx->pinned_units = (size_t)b->n_units;
     }
-    int chunk0 = 0, seed_base = 0;
+    int chunk0 = 0, seed_base = 0, atile0 = 0;
     const int64_t q_unit = (int64_t)b->group * b->window * b->head_dim;
     for (int u = 0; u < b->n_units; ++u) {
         UnitDesc& d = ctx->pinned[u];
@@ -217,9 +217,12 @@ int prepare(cask_ctx* ctx, const cask_batch* b, const cask_params* p, void* ws, 
         d.chunk0 = chunk0;
         d.n_chunks = (d.T + kChunkKeys - 1) / kChunkKeys;
         d.seed_base = seed_base;
+        d.atile0 = atile0;
+        d.n_atiles = d.plan[CASK_PLAN_M] > 0 ? (d.T - d.plan[CASK_PLAN_R] - d.P + 127) / 128 : 0;
         d.pad = 0;
         chunk0 += d.n_chunks;
         seed_base += d.plan[CASK_PLAN_M];
+        atile0 += d.n_atiles;
     }
     e = cudaMemcpyAsync(W.desc, ctx->pinned, sizeof(UnitDesc) * (size_t)b->n_units, cudaMemcpyHostToDevice,
                         ctx->stream);
@@ -236,6 +239,9 @@ int prepare(cask_ctx* ctx, const cask_batch* b, const cask_params* p, void* ws, 
     L.k = b->k; L.v = b->v; L.q = b->q;
     L.max_T = z.max_T; L.max_m = z.max_m; L.max_chunks = z.max_chunks; L.total_chunks = z.total_chunks;
     L.max_P = z.max_P; L.max_B = z.max_B; L.sum_T = z.sum_T;
+    L.total_atiles = atile0;
+    L.tmap_encode = ctx->tmap_encode;
+    L.force_simt = p->score_path;
     L.launches = &ctx->launches;
     L.prof = &ctx->prof;
     return CASK_OK;

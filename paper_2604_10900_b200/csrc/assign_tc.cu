@@ -1,0 +1,325 @@
+// Assignment of scratch rows to seeds on the tensor cores (Sec. 2.5: cosine as the base merge
+// geometry): D[row, seed] = <k_row, k_seed> for 128-row tiles of the decode region against the
+// unit's m <= 256 gathered seed keys, then per row the argmax of the cosine and the threshold tau.
+//
+// The contraction is small (2*128*m*128 flop per tile) next to the 32 KB of K it consumes, so the
+// kernel is bound by the K stream: a 4-stage TMA ring feeds one persistent CTA per SM.
+//   warp 0     TMA producer: seed matrix once per unit, K tiles through the ring
+//   warp 1     TMEM allocation, tcgen05.mma issue
+//   warps 4-7  epilogue: squared row norms from the staged tile, argmax over the TMEM columns
+// The accumulator (m columns) is double-buffered in TMEM columns [0,256) and [256,512).
+#include "tc_common.cuh"
+
+namespace cask {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kTileRows = 128;
+constexpr int kStages = 4;
+constexpr int kThreadsA = 256;
+constexpr int kEpiWarp0 = 4;
+constexpr int kEpiThreads = 128;
+constexpr uint32_t kSeedRegionBytes = 256 * 128;       // 256 seeds x 64 bf16
+constexpr uint32_t kSeedBytes = 2 * kSeedRegionBytes;
+constexpr uint32_t kKRegionBytes = 128 * 128;
+constexpr uint32_t kKStageBytes = 2 * kKRegionBytes;
+
+struct __align__(8) ABarriers {
+    uint64_t b_full, b_empty;
+    uint64_t k_full[kStages], k_empty[kStages];
+    uint64_t d_full[2], d_empty[2];
+    uint64_t nu_ready;
+};
+
+struct ASmemTail {
+    ABarriers bar;
+    uint32_t tmem_base;
+    int abort;
+    float inv_nu[2][256];     // 1/|k_seed| (0 for a zero seed), double-buffered by unit
+};
+
+constexpr size_t kSmemBytesA = 1024 + kSeedBytes + kStages * kKStageBytes + sizeof(ASmemTail);
+
+// Walks this CTA's contiguous range of scratch tiles, unit by unit.
+struct TileWalk {
+    const UnitDesc* desc;
+    int g, g_end, u, n_units;
+    __device__ void init(const UnitDesc* d, int n_units_, int total) {
+        desc = d;
+        n_units = n_units_;
+        g = (int)(((long long)total * blockIdx.x) / gridDim.x);
+        g_end = (int)(((long long)total * (blockIdx.x + 1)) / gridDim.x);
+        int lo = 0, hi = n_units - 1;
+        while (lo < hi) {                       // last unit with atile0 <= g
+            int mid = (lo + hi + 1) >> 1;
+            if (d[mid].atile0 <= g) lo = mid; else hi = mid - 1;
+        }
+        u = lo;
+        skip_empty();
+    }
+    __device__ void skip_empty() {
+        while (u < n_units - 1 && g >= desc[u].atile0 + desc[u].n_atiles) ++u;
+    }
+    __device__ bool valid() const { return g < g_end; }
+    __device__ int tile_in_unit() const { return g - desc[u].atile0; }
+    // tiles of the current unit that belong to this CTA from g on
+    __device__ int run() const { return min(g_end, desc[u].atile0 + desc[u].n_atiles) - g; }
+    __device__ void advance(int n) {
+        g += n;
+        if (g < g_end) { ++u; skip_empty(); }
+    }
+};
+
+__global__ void __launch_bounds__(kThreadsA, 1)
+assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmSeed,
+                 const UnitDesc* __restrict__ desc, Shape sh, int total_tiles, const float* __restrict__ s,
+                 const int32_t* __restrict__ plan, const int32_t* __restrict__ seed_rows,
+                 const float* __restrict__ seed_norm, uint8_t* __restrict__ kind, int32_t* __restrict__ seed_of,
+                 float* __restrict__ sim, int32_t* __restrict__ grp, unsigned long long* __restrict__ mass_fx,
+                 int32_t* __restrict__ njoin, int max_m, float tau, float eps, int32_t* __restrict__ err) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* b_smem = smem;
+    uint8_t* k_smem = smem + kSeedBytes;
+    ASmemTail* tail = reinterpret_cast<ASmemTail*>(k_smem + kStages * kKStageBytes);
+    ABarriers& bar = tail->bar;
+    volatile int* abort_flag = &tail->abort;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        mbar_init(&bar.b_full, 1);
+        mbar_init(&bar.b_empty, 1);
+        for (int i = 0; i < kStages; ++i) { mbar_init(&bar.k_full[i], 1); mbar_init(&bar.k_empty[i], 1 + 4); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&bar.d_full[i], 1); mbar_init(&bar.d_empty[i], 4); }
+        mbar_init(&bar.nu_ready, kEpiThreads);
+        tail->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tail->tmem_base)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tail->tmem_base;
+
+    TileWalk wk;
+    wk.init(desc, sh.n_units, total_tiles);
+
+    if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            uint32_t kit = 0, ucount = 0;
+            bool ok = true;
+            while (wk.valid() && ok) {
+                const UnitDesc& ud = desc[wk.u];
+                ok = mbar_wait(&bar.b_empty, (ucount & 1u) ^ 1u, abort_flag);
+                if (!ok) break;
+                mbar_expect_tx(&bar.b_full, kSeedBytes);
+                tma_load_2d(b_smem, &tmSeed, &bar.b_full, 0, ud.seed_base);
+                tma_load_2d(b_smem + kSeedRegionBytes, &tmSeed, &bar.b_full, 64, ud.seed_base);
+                ++ucount;
+                const int row0 = (int)(ud.k_off / sh.row_stride) + ud.P + wk.tile_in_unit() * kTileRows;
+                const int nt = wk.run();
+                for (int t = 0; t < nt && ok; ++t, ++kit) {
+                    const int st = kit % kStages;
+                    ok = mbar_wait(&bar.k_empty[st], ((kit / kStages) & 1u) ^ 1u, abort_flag);
+                    if (!ok) break;
+                    mbar_expect_tx(&bar.k_full[st], kKStageBytes);
+                    uint8_t* dst = k_smem + st * kKStageBytes;
+                    tma_load_2d(dst, &tmK, &bar.k_full[st], 0, row0 + t * kTileRows);
+                    tma_load_2d(dst + kKRegionBytes, &tmK, &bar.k_full[st], 64, row0 + t * kTileRows);
+                }
+                wk.advance(nt);
+            }
+            if (!ok) {
+                for (uint32_t j = (kit >= (uint32_t)kStages ? kit - kStages : 0); j < kit; ++j)
+                    for (uint32_t it = 0; it < 4096 && !mbar_try(&bar.k_full[j % kStages], (j / kStages) & 1u); ++it) {}
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            uint32_t kit = 0, ucount = 0;
+            bool ok = true;
+            const uint32_t b_addr = smem_u32(b_smem), k_addr = smem_u32(k_smem);
+            while (wk.valid() && ok) {
+                const UnitDesc& ud = desc[wk.u];
+                const int m = max(0, min(plan[wk.u * 8 + CASK_PLAN_M], ud.plan[CASK_PLAN_M]));
+                const uint32_t idesc = umma_idesc(max(16, (m + 15) & ~15));
+                ok = mbar_wait(&bar.b_full, ucount & 1u, abort_flag);
+                if (!ok) break;
+                ++ucount;
+                const int nt = wk.run();
+                for (int t = 0; t < nt && ok; ++t, ++kit) {
+                    const int st = kit % kStages, buf = kit & 1;
+                    ok = mbar_wait(&bar.k_full[st], (kit / kStages) & 1u, abort_flag);
+                    if (!ok) break;
+                    ok = mbar_wait(&bar.d_empty[buf], ((kit >> 1) & 1u) ^ 1u, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t kst = k_addr + st * kKStageBytes;
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {
+                        const int kb = kk >> 2, ks = kk & 3;
+                        uint64_t a = umma_desc(kst + kb * kKRegionBytes + ks * 32);
+                        uint64_t b = umma_desc(b_addr + kb * kSeedRegionBytes + ks * 32);
+                        tc_mma(tmem_base + 256 * buf, a, b, idesc, kk != 0);
+                    }
+                    tc_commit(&bar.d_full[buf]);
+                    tc_commit(&bar.k_empty[st]);
+                }
+                wk.advance(nt);
+                tc_commit(&bar.b_empty);
+            }
+        }
+    } else if (warp >= kEpiWarp0) {
+        // ================= epilogue =================
+        const int qd = warp & 3;
+        const int etid = threadIdx.x - kEpiWarp0 * 32;
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * qd) << 16);
+        const int my_row = 32 * qd + lane;                   // row of the tile this thread owns
+        uint32_t kit = 0, ucount = 0;
+        bool ok = true;
+        while (wk.valid() && ok) {
+            const UnitDesc& ud = desc[wk.u];
+            const int u = wk.u;
+            const int T = ud.T, P = ud.P;
+            const int r = max(0, min(plan[u * 8 + CASK_PLAN_R], T - P));
+            const int m = max(0, min(plan[u * 8 + CASK_PLAN_M], ud.plan[CASK_PLAN_M]));
+            const int hi = T - r;
+            float* inv = tail->inv_nu[ucount & 1u];
+            for (int c = etid; c < 256; c += kEpiThreads) {
+                float nu = (c < m) ? seed_norm[ud.seed_base + c] : 0.f;
+                inv[c] = nu > 0.f ? 1.f / nu : 0.f;
+            }
+            mbar_arrive(&bar.nu_ready);
+            ok = mbar_wait(&bar.nu_ready, ucount & 1u, abort_flag);
+            if (!ok) break;
+            ++ucount;
+            const int tile0 = wk.tile_in_unit();
+            const int nt = wk.run();
+            for (int t = 0; t < nt && ok; ++t, ++kit) {
+                const int st = kit % kStages, buf = kit & 1;
+                // squared norm of this thread's row, read from the staged tile (any order of the
+                // sixteen 16-byte pieces of the row gives the same set of elements)
+                ok = mbar_wait(&bar.k_full[st], (kit / kStages) & 1u, abort_flag);
+                if (!ok) break;
+                float n2 = 0.f;
+                {
+                    const uint8_t* base = k_smem + st * kKStageBytes + my_row * 128;
+#pragma unroll
+                    for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            const uint4 raw = *reinterpret_cast<const uint4*>(base + kb * kKRegionBytes + (((c + lane) & 7) << 4));
+                            const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+                            for (int x = 0; x < 4; ++x) {
+                                const float2 f = __bfloat1622float2(h2[x]);
+                                n2 = fmaf(f.x, f.x, n2);
+                                n2 = fmaf(f.y, f.y, n2);
+                            }
+                        }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bar.k_empty[st]);
+                ok = mbar_wait(&bar.d_full[buf], (kit >> 1) & 1u, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                float best = -INFINITY, best_dot = 0.f;
+                int best_u = -1;
+                for (int cc = 0; cc < m; cc += 32) {
+                    float v[32];
+                    tc_ld32(lane_addr + 256 * buf + cc, v);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int x = 0; x < 32; ++x) {
+                        const float val = v[x] * inv[cc + x];
+                        if (cc + x < m && val > best) { best = val; best_dot = v[x]; best_u = cc + x; }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bar.d_empty[buf]);
+                const int i = P + (tile0 + t) * kTileRows + my_row;
+                if (i < hi && best_u >= 0 && kind[ud.tok_off + i] == CASK_KIND_DROPPED) {
+                    const float nj = sqrtf(n2);
+                    const float nu = seed_norm[ud.seed_base + best_u];
+                    const float sm_ = (nj > 0.f && nu > 0.f) ? best_dot / (nj * nu) : 0.f;
+                    if (sim) sim[ud.tok_off + i] = sm_;
+                    const unsigned long long fx = mass_to_fx(s[ud.tok_off + i] + eps);
+                    if (sm_ >= tau) {
+                        kind[ud.tok_off + i] = CASK_KIND_MERGED;
+                        seed_of[ud.tok_off + i] = seed_rows[ud.seed_base + best_u];
+                        grp[ud.tok_off + i] = best_u;
+                        atomicAdd(&mass_fx[(size_t)u * (max_m + 1) + best_u], fx);
+                        atomicAdd(&njoin[u], 1);
+                    } else {
+                        atomicAdd(&mass_fx[(size_t)u * (max_m + 1) + max_m], fx);
+                    }
+                }
+            }
+            wk.advance(nt);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && tail->abort) atomicOr(err, CASK_ST_TIMEOUT);
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+}  // namespace
+
+bool assign_tc_supported(const Launch& L) {
+    const Shape& sh = L.sh;
+    if (sh.dtype != CASK_DTYPE_BF16 || sh.d != 128 || L.max_m > 256 || L.max_m < 1 || L.total_atiles < 1)
+        return false;
+    int64_t max_row = 0;
+    for (int u = 0; u < sh.n_units; ++u) {
+        const UnitDesc& d = L.hdesc[u];
+        if (d.k_off % sh.row_stride != 0) return false;
+        max_row = std::max<int64_t>(max_row, d.k_off / sh.row_stride + d.T);
+    }
+    return max_row < (int64_t)1 << 31;
+}
+
+cudaError_t launch_assign_tc(const Launch& L, const cask_params& prm, const float* s, const int32_t* plan,
+                             uint8_t* kind, int32_t* seed_of, float* sim, Workspace& ws, void* tmap_encode_fn) {
+    const Shape& sh = L.sh;
+    int64_t k_rows = 0, sum_m = 0;
+    for (int u = 0; u < sh.n_units; ++u) {
+        k_rows = std::max<int64_t>(k_rows, L.hdesc[u].k_off / sh.row_stride + L.hdesc[u].T);
+        sum_m += L.hdesc[u].plan[CASK_PLAN_M];
+    }
+    CUtensorMap tmK, tmSeed;
+    if (!encode_rows_bf16(tmap_encode_fn, &tmK, L.k, (uint64_t)k_rows, (uint64_t)sh.row_stride * 2, kTileRows))
+        return cudaErrorInvalidValue;
+    // the seed table has 256 spare rows behind the last seed, so a full box never leaves the allocation
+    if (!encode_rows_bf16(tmap_encode_fn, &tmSeed, ws.seed_k, (uint64_t)sum_m + 256, 256, 256))
+        return cudaErrorInvalidValue;
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    const int grid = std::max(1, std::min(sms, L.total_atiles));
+    e = cudaFuncSetAttribute(assign_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytesA);
+    if (e != cudaSuccess) return e;
+    {
+        Timed t(L, KID_ASSIGN);
+        assign_tc_kernel<<<grid, kThreadsA, kSmemBytesA, L.stream>>>(
+            tmK, tmSeed, L.desc, sh, L.total_atiles, s, plan, ws.seed_rows, ws.seed_norm, kind, seed_of, sim, ws.grp,
+            ws.mass_fx, ws.njoin, L.max_m, prm.tau, prm.eps, ws.err);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace cask

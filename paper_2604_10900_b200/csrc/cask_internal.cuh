@@ -21,6 +21,8 @@ struct UnitDesc {
     int32_t chunk0;     // first score-partial chunk of this unit
     int32_t n_chunks;   // key chunks of this unit in the normaliser pass
     int32_t seed_base;  // first entry of this unit in the seed tables
+    int32_t atile0;     // first 128-row scratch tile of this unit in the assignment pass
+    int32_t n_atiles;   // scratch tiles of this unit: ceil((T - r - P)/128) when m > 0, else 0
     int32_t pad;
 };
 
@@ -54,10 +56,12 @@ struct Launch {
     const void* k;
     const void* v;
     const void* q;
-    int max_T, max_m, max_chunks, total_chunks, max_P, max_B;
+    int max_T, max_m, max_chunks, total_chunks, total_atiles, max_P, max_B;
     int64_t sum_T;
     int64_t* launches;        // counter to bump
     Profiler* prof;
+    void* tmap_encode;        // cuTensorMapEncodeTiled or nullptr
+    int force_simt;
 };
 
 // Scope guard around one kernel launch: counts it and, in profiling mode, times it.
@@ -109,6 +113,11 @@ cudaError_t launch_consolidate(const Launch& L, const cask_params& prm, const fl
                                float* sim, int32_t* unit_status, float* lost_mass, Workspace& ws);
 cudaError_t launch_compact(const Launch& L, const cask_params& prm, const float* s, const uint8_t* kind,
                            const int32_t* seed_of, float* weight, const cask_outputs& out, Workspace& ws);
+
+// Tensor-core assignment of scratch rows to seeds (cosine Gram + argmax), same outputs as the SIMT kernel.
+bool assign_tc_supported(const Launch& L);
+cudaError_t launch_assign_tc(const Launch& L, const cask_params& prm, const float* s, const int32_t* plan,
+                             uint8_t* kind, int32_t* seed_of, float* sim, Workspace& ws, void* tmap_encode_fn);
 
 // Tensor-core scoring (tcgen05 + TMA); returns cudaErrorNotSupported when the shape does not fit.
 bool score_tc_supported(const Launch& L);

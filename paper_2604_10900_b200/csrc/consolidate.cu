@@ -259,6 +259,10 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const i
                 L.desc, sh, (const T*)L.k, s, plan, ws.seed_rows, (T*)ws.seed_k, ws.seed_norm, ws.mass_fx, max_m,
                 prm.eps);
         }
+        if (!L.force_simt && L.tmap_encode && assign_tc_supported(L)) {
+            cudaError_t e = launch_assign_tc(L, prm, s, plan, kind, seed_of, sim, ws, L.tmap_encode);
+            if (e != cudaSuccess) return e;
+        } else {
         const size_t smem = ((size_t)2 * kTile * (sh.d + 1) + kTile) * sizeof(float);
         cudaError_t e = cudaFuncSetAttribute(assign_simt_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)smem);
@@ -268,6 +272,7 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const i
         assign_simt_kernel<T><<<dim3((max_nd + kTile - 1) / kTile, sh.n_units), kThreads, smem, L.stream>>>(
             L.desc, sh, (const T*)L.k, s, plan, ws.seed_rows, (const T*)ws.seed_k, ws.seed_norm, kind, seed_of,
             sim, ws.grp, ws.mass_fx, ws.njoin, max_m, prm.tau, prm.eps);
+        }
     }
     {
         Timed t(L, KID_WEIGHTS);
