@@ -39,6 +39,7 @@ extern "C" {
 #define CASK_ERR_UNSUPPORTED   -5   /* a documented but unbuilt mode (paged cache)    */
 #define CASK_ERR_CUDA          -6   /* a CUDA runtime call failed (see cask_last_cuda_error) */
 #define CASK_ERR_PARAM         -7   /* gamma/tau/eps/causal out of range              */
+#define CASK_ERR_TOO_LARGE     -8   /* batch exceeds a fixed capacity (cask_score_noalloc) */
 
 /* ---- per-unit status bits (plan[6], unit_status[u]) --------------------- */
 #define CASK_ST_NOOP_UNDER_BUDGET        1   /* T <= B: every row kept                        */
@@ -249,6 +250,36 @@ int cask_compress_event(cask_ctx* ctx, const cask_batch* batch, const cask_param
 size_t cask_host_event_device_bytes(const cask_batch* batch, const cask_params* params, int32_t Bmax);
 int cask_compress_event_host(cask_ctx* ctx, const cask_batch* host_batch, const cask_params* params,
                              const cask_outputs* host_out, void* dev_buf, size_t dev_bytes);
+
+/*
+ * cask_score for callers that cannot allocate device memory (no counterpart in the paper: it
+ * describes no memory management at all).
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a serving engine that has
+ * given the whole device to its own memory pool, in a plugin loaded after the memory budget was
+ * fixed, or anywhere a workspace cannot be obtained -- and that therefore cannot provide the
+ * workspace cask_score asks for.  Here the scratch (unit descriptors, normaliser partials, row
+ * tables) sits in one fixed array of CASK_NOALLOC_SCRATCH_BYTES inside the library image; every GPU
+ * that loads the library holds that much memory until the process exits.  The call takes no
+ * context and makes no cudaMalloc / cudaFree / cudaMallocHost or other allocating call.
+ *
+ * Same inputs and outputs as cask_score (s [sumT] DEVICE out, lse_out optional DEVICE out), on
+ * `device` and `cuda_stream`; it always uses the SIMT scoring kernels, so the scores equal those of
+ * cask_score with score_path = 1 and agree with the tensor-core path to rounding.
+ * Limits: n_units <= CASK_NOALLOC_MAX_UNITS and
+ *   256-byte-rounded sizes of 2 * n_units*g*W*4 + 2 * (sum_u ceil(T[u]/2048))*g*W*4 bytes
+ *   + the descriptor table  <=  CASK_NOALLOC_SCRATCH_BYTES;
+ * beyond either, CASK_ERR_TOO_LARGE is returned before anything is launched.
+ * The first call on a device looks the array's device address up (cudaGetSymbolAddress, once per
+ * device); make that first call before any stream capture begins.  All calls on a device share
+ * the one array: two calls whose kernels may overlap on the GPU (different streams, or different
+ * host threads without ordering) race on it and must be serialised by the caller.  Nothing in the
+ * array needs clearing between calls: each call writes every word it later reads.
+ */
+#define CASK_NOALLOC_SCRATCH_BYTES (4 * 1024 * 1024)
+#define CASK_NOALLOC_MAX_UNITS 64
+int cask_score_noalloc(int device, void* cuda_stream, const cask_batch* batch, const cask_params* params,
+                       float* s, float* lse_out);
 
 #ifdef __cplusplus
 }

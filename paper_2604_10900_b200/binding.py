@@ -19,6 +19,8 @@ LIB_PATH = os.path.join(_HERE, "libcask.so")
 # mirrors of the header's constants
 OK = 0
 ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_UNSUPPORTED, ERR_CUDA, ERR_PARAM = -1, -2, -3, -4, -5, -6, -7
+ERR_TOO_LARGE = -8
+NOALLOC_SCRATCH_BYTES, NOALLOC_MAX_UNITS = 4 * 1024 * 1024, 64
 ST_NOOP_UNDER_BUDGET, ST_PREFIX_EVICTED, ST_DECODE_CONSOLIDATED = 1, 2, 4
 ST_PREFIX_BUDGET_EXHAUSTED, ST_MERGE_INACTIVE, ST_TIMEOUT, ST_BOUNDS = 8, 16, 32, 64
 KIND_DROPPED, KIND_PREFIX, KIND_RECENT, KIND_CORE, KIND_SEED, KIND_MERGED = 0, 1, 2, 3, 4, 5
@@ -29,7 +31,7 @@ EXPORTS = (
     "cask_launch_count", "cask_last_score_path_tensor", "cask_profile_enable", "cask_profile_read",
     "cask_kernel_count", "cask_kernel_name", "cask_workspace_bytes", "cask_plan_host",
     "cask_score", "cask_prefix_evict", "cask_select_core", "cask_consolidate_scratch", "cask_compact",
-    "cask_compress_event", "cask_host_event_device_bytes", "cask_compress_event_host",
+    "cask_compress_event", "cask_host_event_device_bytes", "cask_compress_event_host", "cask_score_noalloc",
 )
 
 
@@ -100,6 +102,7 @@ def lib():
         L.cask_host_event_device_bytes.argtypes = [PB, PP, C.c_int32]
         L.cask_host_event_device_bytes.restype = sz
         L.cask_compress_event_host.argtypes = [vp, PB, PP, PO, vp, sz]
+        L.cask_score_noalloc.argtypes = [i32, vp, PB, PP, vp, vp]
         _lib = L
     return _lib
 
@@ -293,6 +296,15 @@ def cask_compress_event_host(ctx, host_batch, prm, host_out: CaskOutputs, dev_bu
                                         _ptr(dev_buf), dev_bytes)
     if check:
         _check(rc, ctx)
+    return rc
+
+
+def cask_score_noalloc(device: int, stream, batch, prm, s, lse_out=None, check: bool = True) -> int:
+    """Scoring for callers that cannot allocate: the scratch is a fixed array inside the library
+    (no context, no workspace).  See ``cask_score_noalloc`` in ``include/cask.h`` for the limits."""
+    rc = lib().cask_score_noalloc(device, stream, C.byref(batch), C.byref(prm), _ptr(s), _ptr(lse_out))
+    if check:
+        _check(rc)
     return rc
 
 

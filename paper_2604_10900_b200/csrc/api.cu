@@ -262,6 +262,11 @@ int run_score(cask_ctx* ctx, const Launch& L, const cask_batch* b, const cask_pa
 
 }  // namespace
 
+namespace cask {
+// The host-side argument check, for entry points that live in other files.
+int check_batch_host(const cask_batch* b, const cask_params* p) { return check_batch(b, p); }
+}  // namespace cask
+
 extern "C" {
 
 int cask_create(cask_ctx** out, int device, void* cuda_stream) {
@@ -315,6 +320,7 @@ const char* cask_strerror(int code) {
         case CASK_ERR_UNSUPPORTED: return "mode not built (paged cache)";
         case CASK_ERR_CUDA: return "CUDA runtime error";
         case CASK_ERR_PARAM: return "policy parameter out of range";
+        case CASK_ERR_TOO_LARGE: return "batch exceeds the fixed capacity of the no-allocation entry point";
         default: return "unknown error";
     }
 }
