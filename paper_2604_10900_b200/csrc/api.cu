@@ -156,8 +156,9 @@ Workspace carve(char* base, const cask_batch* b, const Sizes& z) {
     w.s = (float*)take(sumT * 4);
     w.rowm = (float*)take(n * rows * 4);
     w.roww = (float*)take(n * rows * 4);
-    w.part_m = (float*)take((size_t)z.total_chunks * rows * 4);
-    w.part_l = (float*)take((size_t)z.total_chunks * rows * 4);
+    const size_t parts = std::max((size_t)z.total_chunks, score_tc_partial_slots(b->n_units));
+    w.part_m = (float*)take(parts * rows * 4);
+    w.part_l = (float*)take(parts * rows * 4);
     w.seed_rows = (int32_t*)take((size_t)z.sum_m * 4);
     w.seed_norm = (float*)take((size_t)z.sum_m * 4);
     w.seed_k = take(((size_t)z.sum_m + 256) * b->head_dim * elem_size(b->dtype));
@@ -204,7 +205,7 @@ int prepare(cask_ctx* ctx, const cask_batch* b, const cask_params* p, void* ws, 
         if (e != cudaSuccess) return fail_cuda(ctx, e);
         ctx->pinned_units = (size_t)b->n_units;
     }
-    int chunk0 = 0, seed_base = 0, atile0 = 0;
+    int chunk0 = 0, seed_base = 0, atile0 = 0, tile0 = 0;
     const int64_t q_unit = (int64_t)b->group * b->window * b->head_dim;
     for (int u = 0; u < b->n_units; ++u) {
         UnitDesc& d = ctx->pinned[u];
@@ -219,7 +220,8 @@ int prepare(cask_ctx* ctx, const cask_batch* b, const cask_params* p, void* ws, 
         d.seed_base = seed_base;
         d.atile0 = atile0;
         d.n_atiles = d.plan[CASK_PLAN_M] > 0 ? (d.T - d.plan[CASK_PLAN_R] - d.P + 127) / 128 : 0;
-        d.pad = 0;
+        d.tile0 = tile0;
+        tile0 += (d.T + 127) / 128;
         chunk0 += d.n_chunks;
         seed_base += d.plan[CASK_PLAN_M];
         atile0 += d.n_atiles;
@@ -240,6 +242,7 @@ int prepare(cask_ctx* ctx, const cask_batch* b, const cask_params* p, void* ws, 
     L.max_T = z.max_T; L.max_m = z.max_m; L.max_chunks = z.max_chunks; L.total_chunks = z.total_chunks;
     L.max_P = z.max_P; L.max_B = z.max_B; L.sum_T = z.sum_T;
     L.total_atiles = atile0;
+    L.total_tiles = tile0;
     L.tmap_encode = ctx->tmap_encode;
     L.force_simt = p->score_path;
     L.launches = &ctx->launches;

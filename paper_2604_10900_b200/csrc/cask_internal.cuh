@@ -23,7 +23,7 @@ struct UnitDesc {
     int32_t seed_base;  // first entry of this unit in the seed tables
     int32_t atile0;     // first 128-row scratch tile of this unit in the assignment pass
     int32_t n_atiles;   // scratch tiles of this unit: ceil((T - r - P)/128) when m > 0, else 0
-    int32_t pad;
+    int32_t tile0;      // first 128-key tile of this unit in the unit-major tile sequence of the scoring passes
 };
 
 struct Shape {
@@ -56,7 +56,7 @@ struct Launch {
     const void* k;
     const void* v;
     const void* q;
-    int max_T, max_m, max_chunks, total_chunks, total_atiles, max_P, max_B;
+    int max_T, max_m, max_chunks, total_chunks, total_atiles, max_P, max_B, total_tiles;
     int64_t sum_T;
     int64_t* launches;        // counter to bump
     Profiler* prof;
@@ -121,6 +121,7 @@ cudaError_t launch_assign_tc(const Launch& L, const cask_params& prm, const floa
 
 // Tensor-core scoring (tcgen05 + TMA); returns cudaErrorNotSupported when the shape does not fit.
 bool score_tc_supported(const Launch& L);
+size_t score_tc_partial_slots(int n_units);   // entries per normaliser-partial table
 cudaError_t launch_score_tc(const Launch& L, const float* lse_in, float* s, float* lse_out,
                             Workspace& ws, void* tmap_encode_fn);
 

@@ -1,20 +1,33 @@
 // Windowed attention-mass scoring on the 5th-generation tensor cores (bf16 cache, head_dim 128).
 //
 // Both passes contract the unit's window queries Q_w [rows<=512, 128] with 128-key tiles of K:
-//   pass N (normaliser): D[query, key]  -> per query row running max / sum of 2^(y - max)
+//   pass N (normaliser): D[query, key]  -> per query row a reference r and sum of 2^(y - r)
 //   pass S (score mass): D[key, query]  -> per key  sum_r roww_r * 2^(y_kr - rowm_r)
-// so that the reduction always runs along the TMEM columns a single thread owns (no
-// cross-thread reduction).  The two passes use the same shared-memory operand tiles
-// (K-major, 128-byte swizzle, written by TMA); only the role of the operands (A <-> B) and
-// the instruction shape differ.
+// so that the reduction always runs along the TMEM columns a single thread owns.  The two
+// passes use the same shared-memory operand tiles (K-major, 128-byte swizzle, written by
+// TMA); only the role of the operands (A <-> B) differs.
 //
-// One persistent CTA per SM, 12 warps:
-//   warp 0      TMA producer (one lane): Q once per unit, K tiles through a 2-stage ring
-//   warp 1      TMEM allocation; one lane issues tcgen05.mma and the commits
-//   warps 4-11  epilogue: tcgen05.ld of the fp32 accumulators + exp2 arithmetic
-// The 512 TMEM columns hold one 128x512 accumulator split in two 256-column halves that
-// ping-pong between the tensor pipe and the epilogue.  Every mbarrier wait is bounded; when
-// one gives up the CTA raises an error flag, drains and frees its TMEM.
+// One persistent CTA per SM, 20 warps:
+//   warp 0      TMA producer (one lane): Q once per segment, K tiles through a 2-stage ring
+//   warps 1-2   one lane each issues tcgen05.mma and the commits: warp 1 for the even accumulator
+//               slots, warp 2 for the odd ones, so that one keeps the tensor pipe fed while the other
+//               waits for a slot to be released (warp 1 also owns the TMEM allocation)
+//   warps 4-19  epilogue: tcgen05.ld of the fp32 accumulators + the exponentials
+// The 512 TMEM columns are four accumulator slots of 128 columns (one 128-row block of
+// queries each).  The epilogue warps form two groups of eight (two per TMEM lane quadrant, 64
+// columns each); group g drains slots g and g+2 in turn, so while it works on one of its
+// slots the tensor pipe refills the other and neither side waits for the other.
+//
+// The exponentials are the bottleneck (16 ex2 per clock per SM against 65,536 per tile), so a
+// fixed share of the columns is evaluated on the FMA pipe instead: round-to-nearest split
+// 2^t = 2^n * 2^f, |f| <= 1/2, degree-5 minimax polynomial for 2^f (relative error 2.4e-7,
+// the same order as ex2.approx).
+//
+// Work is split by tiles, not by units: CTA b owns the contiguous tile range
+// [total*b/grid, total*(b+1)/grid) of the unit-major tile sequence and walks it segment by
+// segment (a segment = its tiles inside one unit).  Pass N leaves one partial per segment
+// row and column half at index 2*(unit + CTA) + half; score_tc_combine folds them.  Every mbarrier wait is
+// bounded; when one gives up the CTA raises an error flag, drains and frees its TMEM.
 #include "tc_common.cuh"
 
 namespace cask {
@@ -26,67 +39,164 @@ using namespace tc;
 constexpr int kTileKeys = 128;
 constexpr int kD = 128;
 constexpr int kStages = 2;
-constexpr int kThreadsTc = 384;
+constexpr int kSlots = 4;                 // accumulator slots of 128 TMEM columns
 constexpr int kEpiWarp0 = 4;
-constexpr int kEpiThreads = 256;
+constexpr int kEpiWarps = 4 * kSlots;
+constexpr int kThreadsTc = (kEpiWarp0 + kEpiWarps) * 32;
 constexpr uint32_t kQRegionBytes = 256 * 128;          // 256 rows x 64 bf16
 constexpr uint32_t kQBytes = 4 * kQRegionBytes;        // 2 row halves x 2 K blocks
 constexpr uint32_t kKRegionBytes = 128 * 128;          // 128 keys x 64 bf16
 constexpr uint32_t kKStageBytes = 2 * kKRegionBytes;
-constexpr int kTilesPerChunk = kChunkKeys / kTileKeys;
+constexpr int kMaxSms = 1024;                          // upper bound used when sizing the partial tables
+
+// Columns (of every 32) whose exponential runs on the FMA pipe.
+constexpr uint32_t kPolyMaskN = 0x80808080u;
+constexpr uint32_t kPolyMaskS = 0x80808080u;
 
 struct __align__(8) Barriers {
     uint64_t q_full, q_empty;
     uint64_t k_full[kStages], k_empty[kStages];
-    uint64_t d_full[2], d_empty[2];
-    uint64_t rw_ready;      // pass S: all epilogue threads have written the row table of the unit
+    uint64_t d_full[kSlots], d_empty[kSlots];
+    uint64_t rw_ready;      // pass S: the row table of the segment is written
+    uint64_t red_full[8];   // pass S: every warp's partial key sums of a tile are in shared memory
 };
 
 struct TcSmemTail {
     Barriers bar;
     uint32_t tmem_base;
     int abort;
-    float2 rw[2][512];     // pass S: {rowm, roww} per query row, double-buffered by unit
+    alignas(16) float rc[2][512];  // pass S: rowm - log2(roww) per query row, double-buffered by segment
+    float red[8][4][128];         // pass S: partial key sums per (group, column half), eight tiles deep
 };
 
 constexpr size_t kSmemBytes = 1024 + kQBytes + kStages * kKStageBytes + sizeof(TcSmemTail);
+static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
-// Walks this CTA's contiguous range of key chunks, unit by unit.
-struct ChunkWalk {
+// 2^t for t in [-125, 125] on the FMA pipe.
+__device__ __forceinline__ float ex2_poly(float t) {
+    const float fl = t + 12582912.f;              // 1.5 * 2^23: the integer nearest to t lands in the low mantissa bits
+    const float f = t - (fl - 12582912.f);        // |f| <= 1/2
+    float p = 1.327644451521337e-3f;
+    p = fmaf(p, f, 9.67553723603487e-3f);
+    p = fmaf(p, f, 5.550713464617729e-2f);
+    p = fmaf(p, f, 2.4022120237350464e-1f);
+    p = fmaf(p, f, 6.931469440460205e-1f);
+    p = fmaf(p, f, 1.0000001192092896f);
+    return __int_as_float(__float_as_int(p) + (__float_as_int(fl) << 23));
+}
+
+// Pass S, one block of 32 query columns (rows r0..r0+31 of the window) for the key this thread owns:
+// adds sum_r 2^(y_r*scale2 - rc[r]) over the visible rows to the four partial sums.
+__device__ __forceinline__ void mass_block(const float (&v)[32], const float* rc, int r0, bool fast, int causal, int W,
+                                           int jmin, float scale2, float& a0, float& a1, float& a2, float& a3) {
+    if (fast) {
+        const float4* rc4 = reinterpret_cast<const float4*>(&rc[r0]);
+#pragma unroll
+        for (int x = 0; x < 8; ++x) {
+            const float4 c4 = rc4[x];
+            const float t0 = fmaf(v[4 * x], scale2, -c4.x), t1 = fmaf(v[4 * x + 1], scale2, -c4.y);
+            const float t2 = fmaf(v[4 * x + 2], scale2, -c4.z), t3 = fmaf(v[4 * x + 3], scale2, -c4.w);
+            a0 += ((kPolyMaskS >> (4 * x)) & 1u) ? ex2_poly(fmaxf(t0, -125.f)) : ex2(t0);
+            a1 += ((kPolyMaskS >> (4 * x + 1)) & 1u) ? ex2_poly(fmaxf(t1, -125.f)) : ex2(t1);
+            a2 += ((kPolyMaskS >> (4 * x + 2)) & 1u) ? ex2_poly(fmaxf(t2, -125.f)) : ex2(t2);
+            a3 += ((kPolyMaskS >> (4 * x + 3)) & 1u) ? ex2_poly(fmaxf(t3, -125.f)) : ex2(t3);
+        }
+    } else {
+#pragma unroll
+        for (int x = 0; x < 32; ++x) {
+            const int r = r0 + x;
+            const bool vis = !causal || (r % W) >= jmin;
+            if (vis) a0 += ex2(fmaf(v[x], scale2, -rc[r]));
+        }
+    }
+}
+
+// Pass N, one block of 32 key columns for the query row this thread owns: folds them into the
+// running (reference, sum of 2^(y*scale2 - reference)).  nvis = visible columns (slow path only).
+__device__ __forceinline__ void norm_block(const float (&v)[32], bool fast, int nvis, float scale2, float& mref,
+                                           float& lr) {
+    if (fast) {
+        float b0 = 0.f, b1 = 0.f, b2 = 0.f, b3 = 0.f;
+#pragma unroll
+        for (int x = 0; x < 32; x += 4) {
+            const float t0 = fmaf(v[x], scale2, -mref), t1 = fmaf(v[x + 1], scale2, -mref);
+            const float t2 = fmaf(v[x + 2], scale2, -mref), t3 = fmaf(v[x + 3], scale2, -mref);
+            b0 += ((kPolyMaskN >> x) & 1u) ? ex2_poly(fminf(fmaxf(t0, -125.f), 125.f)) : ex2(t0);
+            b1 += ((kPolyMaskN >> (x + 1)) & 1u) ? ex2_poly(fminf(fmaxf(t1, -125.f), 125.f)) : ex2(t1);
+            b2 += ((kPolyMaskN >> (x + 2)) & 1u) ? ex2_poly(fminf(fmaxf(t2, -125.f), 125.f)) : ex2(t2);
+            b3 += ((kPolyMaskN >> (x + 3)) & 1u) ? ex2_poly(fminf(fmaxf(t3, -125.f), 125.f)) : ex2(t3);
+        }
+        float lb = (b0 + b1) + (b2 + b3);
+        if (!(lb <= 65536.f)) {
+            // A column exceeds the reference by more than 16 (or the reference is still unset): move the
+            // reference to the block maximum and redo the block.
+            float cm = v[0];
+#pragma unroll
+            for (int x = 1; x < 32; ++x) cm = fmaxf(cm, v[x]);
+            cm *= scale2;
+            if (cm > mref) {
+                lr *= ex2(mref - cm);
+                mref = cm;
+            }
+            b0 = 0.f; b1 = 0.f;
+#pragma unroll
+            for (int x = 0; x < 32; x += 2) {
+                b0 += ex2(fmaf(v[x], scale2, -mref));
+                b1 += ex2(fmaf(v[x + 1], scale2, -mref));
+            }
+            lb = b0 + b1;
+        }
+        lr += lb;
+    } else {
+        float cm = kNegBig;
+#pragma unroll
+        for (int x = 0; x < 32; ++x)
+            if (x < nvis) cm = fmaxf(cm, v[x] * scale2);
+        if (cm > mref) {
+            lr *= ex2(mref - cm);
+            mref = cm;
+        }
+#pragma unroll
+        for (int x = 0; x < 32; ++x)
+            if (x < nvis) lr += ex2(fmaf(v[x], scale2, -mref));
+    }
+}
+
+// Walks this CTA's contiguous range of key tiles, segment by segment.
+struct TileWalk {
     const UnitDesc* desc;
-    int c, c_end, u;
-    int chunk0, n_chunks, T;
-    __device__ void init(const UnitDesc* d, int n_units, int total_chunks) {
+    int t, t_end, u;
+    int tile0, n_tiles, T;
+    __device__ void init(const UnitDesc* d, int n_units, int total_tiles) {
         desc = d;
-        c = (int)(((long long)total_chunks * blockIdx.x) / gridDim.x);
-        c_end = (int)(((long long)total_chunks * (blockIdx.x + 1)) / gridDim.x);
+        t = (int)(((long long)total_tiles * blockIdx.x) / gridDim.x);
+        t_end = (int)(((long long)total_tiles * (blockIdx.x + 1)) / gridDim.x);
         int lo = 0, hi = n_units - 1;
-        while (lo < hi) {                       // last unit with chunk0 <= c
+        while (lo < hi) {                       // last unit with tile0 <= t
             int mid = (lo + hi + 1) >> 1;
-            if (d[mid].chunk0 <= c) lo = mid; else hi = mid - 1;
+            if (d[mid].tile0 <= t) lo = mid; else hi = mid - 1;
         }
         u = lo;
         load();
     }
-    __device__ void load() { chunk0 = desc[u].chunk0; n_chunks = desc[u].n_chunks; T = desc[u].T; }
-    __device__ bool valid() const { return c < c_end; }
-    __device__ int key_begin() const { return (c - chunk0) * kChunkKeys; }
-    __device__ int n_tiles() const {
-        int rem = T - key_begin();
-        return min(kTilesPerChunk, (rem + kTileKeys - 1) / kTileKeys);
+    __device__ void load() {
+        tile0 = desc[u].tile0;
+        T = desc[u].T;
+        n_tiles = (T + kTileKeys - 1) / kTileKeys;
     }
-    // returns true when the next chunk belongs to another unit
-    __device__ bool advance() {
-        ++c;
-        if (c >= chunk0 + n_chunks && c < c_end) { ++u; load(); return true; }
-        return c >= c_end;
+    __device__ bool valid() const { return t < t_end; }
+    __device__ int key_begin() const { return (t - tile0) * kTileKeys; }
+    __device__ int seg_tiles() const { return min(t_end, tile0 + n_tiles) - t; }
+    __device__ void next_segment() {
+        t += seg_tiles();
+        if (t < t_end) { ++u; load(); }
     }
 };
 
 template <int PASS>   // 0: normaliser, 1: score mass
 __global__ void __launch_bounds__(kThreadsTc, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
-                const UnitDesc* __restrict__ desc, Shape sh, int total_chunks,
+                const UnitDesc* __restrict__ desc, Shape sh, int total_tiles,
                 float* __restrict__ part_m, float* __restrict__ part_l, const float* __restrict__ rowm,
                 const float* __restrict__ roww, float* __restrict__ s, int32_t* __restrict__ err) {
     extern __shared__ uint8_t smem_raw[];
@@ -99,15 +209,18 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rows = sh.rows;
-    const int n_blocks = (rows + 127) >> 7;          // 128-row query blocks (pass N)
-    const int n_halves = (rows + 255) >> 8;          // 256-column accumulator halves in use
+    const int n_slots = (rows + 127) >> 7;           // 128-row query blocks in use
+    const int n_halves = (rows + 255) >> 8;          // 256-row Q regions in use
+    const int n_issuers = min(2, n_slots);
+    const int n_groups = n_issuers;                  // epilogue groups of eight warps
 
     if (threadIdx.x == 0) {
         mbar_init(&bar.q_full, 1);
-        mbar_init(&bar.q_empty, 1);
-        for (int i = 0; i < kStages; ++i) { mbar_init(&bar.k_full[i], 1); mbar_init(&bar.k_empty[i], 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&bar.d_full[i], 1); mbar_init(&bar.d_empty[i], 8); }
-        mbar_init(&bar.rw_ready, kEpiThreads);
+        mbar_init(&bar.q_empty, n_issuers);
+        for (int i = 0; i < kStages; ++i) { mbar_init(&bar.k_full[i], 1); mbar_init(&bar.k_empty[i], n_issuers); }
+        for (int i = 0; i < kSlots; ++i) { mbar_init(&bar.d_full[i], 1); mbar_init(&bar.d_empty[i], 8); }
+        mbar_init(&bar.rw_ready, 256 * n_groups);
+        for (int i = 0; i < 8; ++i) mbar_init(&bar.red_full[i], 8 * n_groups);
         tail->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -120,27 +233,24 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     tc_fence_after();
     const uint32_t tmem_base = tail->tmem_base;
 
-    ChunkWalk wk;
-    wk.init(desc, sh.n_units, total_chunks);
+    TileWalk wk;
+    wk.init(desc, sh.n_units, total_tiles);
 
     if (warp == 0) {
         // ================= TMA producer =================
         if (lane == 0) {
-            uint32_t kit = 0, qcount = 0;
-            bool new_unit = true, ok = true;
-            while (wk.valid() && ok) {
+            uint32_t kit = 0, seg = 0;
+            bool ok = true;
+            for (; wk.valid() && ok; wk.next_segment(), ++seg) {
                 const UnitDesc& ud = desc[wk.u];
-                if (new_unit) {
-                    ok = mbar_wait(&bar.q_empty, (qcount & 1u) ^ 1u, abort_flag);
-                    if (!ok) break;
-                    mbar_expect_tx(&bar.q_full, n_halves * 2 * kQRegionBytes);
-                    for (int nh = 0; nh < n_halves; ++nh)
-                        for (int kb = 0; kb < 2; ++kb)
-                            tma_load_3d(q_smem + (nh * 2 + kb) * kQRegionBytes, &tmQ, &bar.q_full, kb * 64, nh * 256, wk.u);
-                    ++qcount;
-                }
+                ok = mbar_wait(&bar.q_empty, (seg & 1u) ^ 1u, abort_flag);
+                if (!ok) break;
+                mbar_expect_tx(&bar.q_full, n_halves * 2 * kQRegionBytes);
+                for (int nh = 0; nh < n_halves; ++nh)
+                    for (int kb = 0; kb < 2; ++kb)
+                        tma_load_3d(q_smem + (nh * 2 + kb) * kQRegionBytes, &tmQ, &bar.q_full, kb * 64, nh * 256, wk.u);
                 const int krow0 = (int)(ud.k_off / sh.row_stride) + wk.key_begin();
-                const int nt = wk.n_tiles();
+                const int nt = wk.seg_tiles();
                 for (int t = 0; t < nt && ok; ++t, ++kit) {
                     const int st = kit % kStages;
                     ok = mbar_wait(&bar.k_empty[st], ((kit / kStages) & 1u) ^ 1u, abort_flag);
@@ -150,7 +260,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     tma_load_2d(dst, &tmK, &bar.k_full[st], 0, krow0 + t * kTileKeys);
                     tma_load_2d(dst + kKRegionBytes, &tmK, &bar.k_full[st], 64, krow0 + t * kTileKeys);
                 }
-                new_unit = wk.advance();
             }
             if (!ok) {
                 // copies already issued may still be landing: give each armed stage a bounded wait
@@ -158,193 +267,161 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     for (uint32_t it = 0; it < 4096 && !mbar_try(&bar.k_full[j % kStages], (j / kStages) & 1u); ++it) {}
             }
         }
-    } else if (warp == 1) {
-        // ================= MMA issuer =================
+    } else if (warp <= n_issuers) {
+        // ================= MMA issuers =================
         if (lane == 0) {
-            uint32_t kit = 0, qcount = 0, dcount = 0;
-            bool new_unit = true, ok = true;
-            const uint32_t q_addr = smem_u32(q_smem), k_addr = smem_u32(k_smem);
-            while (wk.valid() && ok) {
-                if (new_unit) {
-                    ok = mbar_wait(&bar.q_full, qcount & 1u, abort_flag);
-                    if (!ok) break;
-                    ++qcount;
-                }
-                const int nt = wk.n_tiles();
-                for (int t = 0; t < nt && ok; ++t, ++kit, ++dcount) {
+            const int j0 = warp - 1;               // this issuer's slots: j0, j0 + 2
+            uint32_t kit = 0, seg = 0;
+            bool ok = true;
+            // Low descriptor words of the two operand bases; every tile of both operands is reached by
+            // adding a compile-time constant (the address field counts 16-byte units and cannot carry).
+            const uint32_t q_lo = umma_desc_lo(smem_u32(q_smem)), k_lo = umma_desc_lo(smem_u32(k_smem));
+            for (; wk.valid() && ok; wk.next_segment(), ++seg) {
+                ok = mbar_wait(&bar.q_full, seg & 1u, abort_flag);
+                if (!ok) break;
+                const int nt = wk.seg_tiles();
+                for (int t = 0; t < nt && ok; ++t, ++kit) {
                     const int st = kit % kStages;
                     ok = mbar_wait(&bar.k_full[st], (kit / kStages) & 1u, abort_flag);
                     if (!ok) break;
-                    const uint32_t kst = k_addr + st * kKStageBytes;
-                    for (int h = 0; h < n_halves && ok; ++h) {
-                        ok = mbar_wait(&bar.d_empty[h], (dcount & 1u) ^ 1u, abort_flag);
+                    const uint32_t kst_lo = k_lo + st * (kKStageBytes >> 4);
+#pragma unroll
+                    for (int jj = 0; jj < kSlots; jj += 2) {
+                        const int j = jj + j0;
+                        if (j >= n_slots || !ok) break;
+                        ok = mbar_wait(&bar.d_empty[j], (kit & 1u) ^ 1u, abort_flag);
                         if (!ok) break;
                         tc_fence_after();
-                        if (PASS == 1) {
-                            const int ncols = min(256, rows - 256 * h);
-                            const uint32_t idesc = umma_idesc(ncols);
+                        const uint32_t qblk_lo = q_lo + (((j >> 1) * 2 * kQRegionBytes + (j & 1) * (128 * 128)) >> 4);
+                        const uint32_t idesc = umma_idesc(PASS == 1 ? min(128, rows - 128 * j) : 128);
+                        if (PASS == 1) tc_mma_lo<false>(tmem_base + 128 * j, kst_lo, qblk_lo, idesc);
+                        else tc_mma_lo<false>(tmem_base + 128 * j, qblk_lo, kst_lo, idesc);
 #pragma unroll
-                            for (int kk = 0; kk < 8; ++kk) {
-                                const int kb = kk >> 2, ks = kk & 3;
-                                uint64_t a = umma_desc(kst + kb * kKRegionBytes + ks * 32);
-                                uint64_t b = umma_desc(q_addr + (h * 2 + kb) * kQRegionBytes + ks * 32);
-                                tc_mma(tmem_base + 256 * h, a, b, idesc, kk != 0);
-                            }
-                        } else {
-                            const uint32_t idesc = umma_idesc(128);
-                            for (int cs = 0; cs < 2; ++cs) {
-                                const int mb = 2 * h + cs;
-                                if (mb >= n_blocks) break;
-#pragma unroll
-                                for (int kk = 0; kk < 8; ++kk) {
-                                    const int kb = kk >> 2, ks = kk & 3;
-                                    uint64_t a = umma_desc(q_addr + (h * 2 + kb) * kQRegionBytes + cs * (128 * 128) + ks * 32);
-                                    uint64_t b = umma_desc(kst + kb * kKRegionBytes + ks * 32);
-                                    tc_mma(tmem_base + 128 * mb, a, b, idesc, kk != 0);
-                                }
-                            }
+                        for (int kk = 1; kk < 8; ++kk) {
+                            const int kb = kk >> 2, ks = kk & 3;
+                            const uint32_t dq = qblk_lo + ((kb * kQRegionBytes + ks * 32) >> 4);
+                            const uint32_t dk = kst_lo + ((kb * kKRegionBytes + ks * 32) >> 4);
+                            if (PASS == 1) tc_mma_lo<true>(tmem_base + 128 * j, dk, dq, idesc);
+                            else tc_mma_lo<true>(tmem_base + 128 * j, dq, dk, idesc);
                         }
-                        tc_commit(&bar.d_full[h]);
+                        tc_commit(&bar.d_full[j]);
                     }
                     tc_commit(&bar.k_empty[st]);
                 }
-                new_unit = wk.advance();
-                if (new_unit) tc_commit(&bar.q_empty);
+                if (ok) tc_commit(&bar.q_empty);
             }
         }
-    } else if (warp >= kEpiWarp0) {
+    } else if (warp >= kEpiWarp0 && ((warp - kEpiWarp0) >> 3) < n_groups) {
         // ================= epilogue =================
         const int ew = warp - kEpiWarp0;
-        const int qd = warp & 3;                 // TMEM lane quadrant this warp may read
-        const int cs = ew >> 2;                  // which 128-column slice of each half
-        const int etid = threadIdx.x - kEpiWarp0 * 32;
+        const int qd = ew & 3;                   // TMEM lane quadrant (== warp % 4)
+        const int ch = (ew >> 2) & 1;            // which 64 columns of a slot
+        const int g = ew >> 3;                   // group: drains slots g and g + 2 in turn
+        const int etid = ew * 32 + lane;
         const float scale2 = kLog2e * rsqrtf((float)kD);
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * qd) << 16);
-        uint32_t dcount = 0, ucount = 0;
-        bool new_unit = true, ok = true;
-        const float2* rw = tail->rw[0];
-        while (wk.valid() && ok) {
-            const UnitDesc& ud = desc[wk.u];
-            const int T = ud.T;
+        const uint32_t taddr = tmem_base + ((uint32_t)(32 * qd) << 16) + 64 * ch;
+        uint32_t kit = 0, seg = 0;
+        bool ok = true;
+        // pass S: key offsets of the last two tiles, folded two tiles late by the warps ew < 4
+        int64_t pend_off[2] = {-1, -1};
+        // pass N: running reference / sum of the two query rows this thread works on
+        float mm[2] = {kNegBig, kNegBig}, l_run[2] = {0.f, 0.f};
+
+        for (; wk.valid() && ok; wk.next_segment(), ++seg) {
+            const int T = wk.T;
+            const int64_t tok_off = desc[wk.u].tok_off;
             const int last_all = sh.causal ? T - sh.W : T - 1;     // last key every query sees
-            if (PASS == 1 && new_unit) {
-                // A thread can be at most one unit ahead of the slowest one (it has passed the previous
-                // rw_ready phase), so writing the other buffer never races with a reader.
-                float2* dst = tail->rw[ucount & 1u];
-                for (int r = etid; r < 512; r += kEpiThreads)
-                    dst[r] = (r < rows) ? make_float2(rowm[(size_t)wk.u * rows + r], roww[(size_t)wk.u * rows + r])
-                                        : make_float2(0.f, 0.f);
+            const float* rc = tail->rc[seg & 1u];
+            if (PASS == 1) {
+                // Every thread has passed the rw_ready phase of the previous segment, so nobody still
+                // reads the buffer used two segments ago.  roww * 2^(y - rowm) = 2^(y - (rowm - log2 roww)).
+                float* dst = tail->rc[seg & 1u];
+                dst[etid] = (etid < rows) ? rowm[(size_t)wk.u * rows + etid] - log2f(roww[(size_t)wk.u * rows + etid])
+                                          : 1.0e30f;
                 mbar_arrive(&bar.rw_ready);
-                ok = mbar_wait(&bar.rw_ready, ucount & 1u, abort_flag);
+                ok = mbar_wait(&bar.rw_ready, seg & 1u, abort_flag);
                 if (!ok) break;
-                rw = dst;
-                ++ucount;
-            }
-            // pass N state: the two query rows this thread owns (one per half)
-            float m_run[2] = {kNegBig, kNegBig}, l_run[2] = {0.f, 0.f};
-            int lastvis[2];
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int r = 128 * (2 * h + cs) + 32 * qd + lane;
-                lastvis[h] = (r < rows) ? (sh.causal ? T - sh.W + (r % sh.W) : T - 1) : -1;
+            } else {
+                mm[0] = mm[1] = kNegBig;
+                l_run[0] = l_run[1] = 0.f;
             }
             const int key_begin = wk.key_begin();
-            const int nt = wk.n_tiles();
-            for (int t = 0; t < nt && ok; ++t, ++dcount) {
+            const int nt = wk.seg_tiles();
+            // The columns of its two slots this warp reads (64 of each, fewer in a ragged last slot).
+            const int j0 = g, j1 = g + 2;
+            const int cend0 = PASS == 1 ? min(64 * ch + 64, rows - 128 * j0) - 64 * ch : 64;
+            const int cend1 = PASS == 1 ? min(64 * ch + 64, rows - 128 * j1) - 64 * ch : 64;
+            const int row0 = 128 * j0 + 32 * qd + lane, row1 = 128 * j1 + 32 * qd + lane;      // pass N
+            const int lastvis0 = (row0 < rows) ? (sh.causal ? T - sh.W + (row0 % sh.W) : T - 1) : -1;
+            const int lastvis1 = (row1 < rows) ? (sh.causal ? T - sh.W + (row1 % sh.W) : T - 1) : -1;
+            for (int t = 0; t < nt && ok; ++t, ++kit) {
                 const int key0 = key_begin + t * kTileKeys;
                 const bool fast = key0 + kTileKeys - 1 <= last_all;
-                float acc = 0.f;
                 const int my_key = key0 + 32 * qd + lane;           // pass S: the key this thread owns
-                const int jmin = my_key - (T - sh.W);                // pass S: first window position that sees it
-                for (int h = 0; h < n_halves && ok; ++h) {
-                    ok = mbar_wait(&bar.d_full[h], dcount & 1u, abort_flag);
+                const int jmin = my_key - (T - sh.W);               // pass S: first window position that sees it
+                const int kcol = key0 + 64 * ch;                    // pass N: first key column of this warp
+                float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+                for (int p = 0; p < 2; ++p) {
+                    const int j = p ? j1 : j0;
+                    if (j >= n_slots || !ok) break;
+                    ok = mbar_wait(&bar.d_full[j], kit & 1u, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    if (PASS == 1) {
-                        const int ncols = min(256, rows - 256 * h);
-                        for (int cc = 128 * cs; cc < min(128 * cs + 128, ncols); cc += 32) {
-                            float v[32];
-                            tc_ld32(lane_addr + 256 * h + cc, v);
-                            tc_wait_ld();
-                            const float4* rw4 = reinterpret_cast<const float4*>(&rw[256 * h + cc]);
-                            if (fast) {
-#pragma unroll
-                                for (int x = 0; x < 16; ++x) {
-                                    const float4 p = rw4[x];
-                                    acc = fmaf(ex2(fmaf(v[2 * x], scale2, -p.x)), p.y, acc);
-                                    acc = fmaf(ex2(fmaf(v[2 * x + 1], scale2, -p.z)), p.w, acc);
-                                }
-                            } else {
-#pragma unroll
-                                for (int x = 0; x < 32; ++x) {
-                                    const int r = 256 * h + cc + x;
-                                    const float2 p = rw[r];
-                                    const bool vis = r < rows && (!sh.causal || (r % sh.W) >= jmin);
-                                    if (vis) acc = fmaf(ex2(fmaf(v[x], scale2, -p.x)), p.y, acc);
-                                }
-                            }
-                        }
-                    } else {
-                        const int mb = 2 * h + cs;
-                        if (mb < n_blocks) {
-                            for (int cc = 0; cc < 128; cc += 32) {
-                                float v[32];
-                                tc_ld32(lane_addr + 128 * mb + cc, v);
-                                tc_wait_ld();
-                                if (fast) {
-                                    float cm = v[0];
-#pragma unroll
-                                    for (int x = 1; x < 32; ++x) cm = fmaxf(cm, v[x]);
-                                    cm *= scale2;
-                                    if (cm > m_run[h]) {
-                                        l_run[h] *= ex2(m_run[h] - cm);
-                                        m_run[h] = cm;
-                                    }
-                                    const float mm = m_run[h];
-                                    float l0 = 0.f, l1 = 0.f;
-#pragma unroll
-                                    for (int x = 0; x < 32; x += 2) {
-                                        l0 += ex2(fmaf(v[x], scale2, -mm));
-                                        l1 += ex2(fmaf(v[x + 1], scale2, -mm));
-                                    }
-                                    l_run[h] += l0 + l1;
-                                } else {
-                                    const int nvis = lastvis[h] - (key0 + cc) + 1;      // visible columns of this chunk
-                                    float cm = kNegBig;
-#pragma unroll
-                                    for (int x = 0; x < 32; ++x)
-                                        if (x < nvis) cm = fmaxf(cm, v[x] * scale2);
-                                    if (cm > m_run[h]) {
-                                        l_run[h] *= ex2(m_run[h] - cm);
-                                        m_run[h] = cm;
-                                    }
-                                    const float mm = m_run[h];
-#pragma unroll
-                                    for (int x = 0; x < 32; ++x)
-                                        if (x < nvis) l_run[h] += ex2(fmaf(v[x], scale2, -mm));
-                                }
-                            }
-                        }
+                    const int cend = p ? cend1 : cend0;
+                    for (int cc = 0; cc < cend; cc += 32) {
+                        float v[32];
+                        tc_ld32(taddr + 128 * j + cc, v);
+                        tc_wait_ld_regs(v);
+                        if (PASS == 1) mass_block(v, rc, 128 * j + 64 * ch + cc, fast, sh.causal, sh.W, jmin, scale2, a0, a1, a2, a3);
+                        else norm_block(v, fast, (p ? lastvis1 : lastvis0) - (kcol + cc) + 1, scale2, mm[p], l_run[p]);
                     }
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&bar.d_empty[h]);
+                    if (lane == 0) mbar_arrive(&bar.d_empty[j]);
                 }
-                // the two column slices of a key meet in the zero-initialised score array; with two
-                // addends the sum does not depend on the order of arrival
-                if (PASS == 1 && ok && my_key < T) atomicAdd(&s[ud.tok_off + my_key], acc);
-            }
-            if (PASS == 0 && ok) {
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const int r = 128 * (2 * h + cs) + 32 * qd + lane;
-                    if (r < rows) {
-                        part_m[(size_t)wk.c * rows + r] = m_run[h];
-                        part_l[(size_t)wk.c * rows + r] = l_run[h];
+                if (PASS == 1 && ok) {
+                    tail->red[kit & 7u][ew >> 2][32 * qd + lane] = (a0 + a1) + (a2 + a3);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bar.red_full[kit & 7u]);
+                    if (ew < 4) {
+                        // Fold the tile before the previous one: every warp finished it long ago.  The
+                        // two-stage key ring keeps every warp within two tiles of every other, so with
+                        // eight buffers the one read here cannot be the one being rewritten.
+                        const int64_t off = pend_off[kit & 1u];
+                        if (kit >= 2) {
+                            const uint32_t pk = kit - 2;
+                            ok = mbar_wait(&bar.red_full[pk & 7u], (pk >> 3) & 1u, abort_flag);
+                            if (!ok) break;
+                            float acc = tail->red[pk & 7u][0][32 * qd + lane];
+                            for (int k = 1; k < 2 * n_groups; ++k) acc += tail->red[pk & 7u][k][32 * qd + lane];
+                            if (off >= 0) s[off] = acc;
+                        }
+                        pend_off[kit & 1u] = (my_key < T) ? tok_off + my_key : -1;
                     }
                 }
             }
-            new_unit = wk.advance();
+            if (PASS == 0 && ok) {
+#pragma unroll
+                for (int p = 0; p < 2; ++p) {
+                    const int my_row = 128 * (g + 2 * p) + 32 * qd + lane;
+                    if (my_row < rows) {
+                        const size_t o = ((size_t)(wk.u + blockIdx.x) * 2 + ch) * rows + my_row;
+                        part_m[o] = mm[p];
+                        part_l[o] = l_run[p];
+                    }
+                }
+            }
+        }
+        if (PASS == 1 && ew < 4 && ok) {
+            // the last two tiles of this CTA
+            for (uint32_t pk = (kit >= 2 ? kit - 2 : 0); pk < kit; ++pk) {
+                if (!mbar_wait(&bar.red_full[pk & 7u], (pk >> 3) & 1u, abort_flag)) break;
+                float acc = tail->red[pk & 7u][0][32 * qd + lane];
+                for (int k = 1; k < 2 * n_groups; ++k) acc += tail->red[pk & 7u][k][32 * qd + lane];
+                const int64_t off = pend_off[pk & 1u];
+                if (off >= 0) s[off] = acc;
+            }
         }
     }
 
@@ -357,7 +434,53 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     }
 }
 
+// CTA that owns tile x when `total` tiles are split over `grid` CTAs as in TileWalk::init.
+__device__ __forceinline__ int owner_cta(long long x, long long total, long long grid) {
+    long long b = (x * grid) / total;
+    while (b + 1 < grid && (total * (b + 1)) / grid <= x) ++b;
+    while (b > 0 && (total * b) / grid > x) --b;
+    return (int)b;
+}
+
+// Folds the per-segment (reference, sum) pairs of every query row into the row offset and weight
+// used by the score pass: rowm = max reference, roww = 1/(rows * sum 2^(y - rowm)).  With
+// caller-supplied natural-log normalisers: rowm = lse*log2(e), roww = 1/rows.
+__global__ void score_tc_combine(const UnitDesc* __restrict__ desc, int rows, int total_tiles, int grid,
+                                 const float* __restrict__ part_m, const float* __restrict__ part_l,
+                                 const float* __restrict__ lse_in, float* __restrict__ rowm,
+                                 float* __restrict__ roww, float* __restrict__ lse_out) {
+    const int u = blockIdx.x;
+    const UnitDesc& ud = desc[u];
+    const float inv_rows = 1.f / (float)rows;
+    const int n_tiles = (ud.T + kTileKeys - 1) / kTileKeys;
+    const int b0 = owner_cta(ud.tile0, total_tiles, grid);
+    const int b1 = owner_cta((long long)ud.tile0 + n_tiles - 1, total_tiles, grid);
+    for (int r = threadIdx.x; r < rows; r += blockDim.x) {
+        const size_t o = (size_t)u * rows + r;
+        if (lse_in) {
+            const float lse = lse_in[o];
+            rowm[o] = lse * kLog2e;
+            roww[o] = inv_rows;
+            if (lse_out) lse_out[o] = lse;
+            continue;
+        }
+        float m = kNegBig;
+        for (int b = 2 * b0; b <= 2 * b1 + 1; ++b) m = fmaxf(m, part_m[((size_t)2 * u + b) * rows + r]);
+        float l = 0.f;
+        for (int b = 2 * b0; b <= 2 * b1 + 1; ++b) {
+            const size_t p = ((size_t)2 * u + b) * rows + r;
+            l += part_l[p] * exp2f(part_m[p] - m);
+        }
+        rowm[o] = m;
+        roww[o] = inv_rows / l;
+        if (lse_out) lse_out[o] = (m + log2f(l)) * kLn2;
+    }
+}
+
 }  // namespace
+
+// Entries of each normaliser-partial table the tensor-core path needs (one per unit + CTA).
+size_t score_tc_partial_slots(int n_units) { return 2 * ((size_t)n_units + kMaxSms); }
 
 bool score_tc_supported(const Launch& L) {
     const Shape& sh = L.sh;
@@ -405,23 +528,24 @@ cudaError_t launch_score_tc(const Launch& L, const float* lse_in, float* s, floa
     if (e != cudaSuccess) return e;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    const int grid = std::max(1, std::min(sms, L.total_chunks));
+    const int grid = std::max(1, std::min(std::min(sms, kMaxSms), L.total_tiles));
     e = cudaFuncSetAttribute(score_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(score_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess) return e;
     if (!lse_in) {
         Timed t(L, KID_SCORE_NORM);
-        score_tc_kernel<0><<<grid, kThreadsTc, kSmemBytes, L.stream>>>(tmK, tmQ, L.desc, sh, L.total_chunks, ws.part_m,
+        score_tc_kernel<0><<<grid, kThreadsTc, kSmemBytes, L.stream>>>(tmK, tmQ, L.desc, sh, L.total_tiles, ws.part_m,
                                                                        ws.part_l, nullptr, nullptr, nullptr, ws.err);
     }
-    e = launch_row_combine(L, lse_in, lse_out, ws);
-    if (e != cudaSuccess) return e;
-    e = cudaMemsetAsync(s, 0, sizeof(float) * (size_t)L.sum_T, L.stream);
-    if (e != cudaSuccess) return e;
+    {
+        Timed t(L, KID_ROW_COMBINE);
+        score_tc_combine<<<sh.n_units, 128, 0, L.stream>>>(L.desc, sh.rows, L.total_tiles, grid, ws.part_m, ws.part_l,
+                                                           lse_in, ws.rowm, ws.roww, lse_out);
+    }
     {
         Timed t(L, KID_SCORE_MASS);
-        score_tc_kernel<1><<<grid, kThreadsTc, kSmemBytes, L.stream>>>(tmK, tmQ, L.desc, sh, L.total_chunks, nullptr,
+        score_tc_kernel<1><<<grid, kThreadsTc, kSmemBytes, L.stream>>>(tmK, tmQ, L.desc, sh, L.total_tiles, nullptr,
                                                                        nullptr, ws.rowm, ws.roww, s, ws.err);
     }
     return cudaGetLastError();
