@@ -4,10 +4,13 @@
 //
 // The contraction is small (2*128*m*128 flop per tile) next to the 32 KB of K it consumes, so the
 // kernel is bound by the K stream: a 4-stage TMA ring feeds one persistent CTA per SM.
-//   warp 0     TMA producer: seed matrix once per unit, K tiles through the ring
-//   warp 1     TMEM allocation, tcgen05.mma issue
-//   warps 4-7  epilogue: squared row norms from the staged tile, argmax over the TMEM columns
-// The accumulator (m columns) is double-buffered in TMEM columns [0,256) and [256,512).
+//   warp 0      TMA producer: seed matrix once per unit, K tiles through the ring
+//   warp 1      TMEM allocation, tcgen05.mma issue
+//   warps 4-19  epilogue in groups of four warps (one per TMEM lane quadrant); group e takes the
+//               tiles e, e+G, e+2G, ... of the CTA and owns one accumulator buffer, so up to G
+//               tiles are in flight and the global-memory round trips of a tile (row kind, score,
+//               the fixed-point mass atomics) overlap with the next tiles
+// G = 4 buffers of 128 TMEM columns when every unit has m <= 128 seeds, else 2 buffers of 256.
 #include "tc_common.cuh"
 
 namespace cask {
@@ -18,9 +21,9 @@ using namespace tc;
 
 constexpr int kTileRows = 128;
 constexpr int kStages = 4;
-constexpr int kThreadsA = 256;
 constexpr int kEpiWarp0 = 4;
-constexpr int kEpiThreads = 128;
+constexpr int kMaxGroups = 4;
+constexpr int kThreadsA = (kEpiWarp0 + 4 * kMaxGroups) * 32;
 constexpr uint32_t kSeedRegionBytes = 256 * 128;       // 256 seeds x 64 bf16
 constexpr uint32_t kSeedBytes = 2 * kSeedRegionBytes;
 constexpr uint32_t kKRegionBytes = 128 * 128;
@@ -29,7 +32,7 @@ constexpr uint32_t kKStageBytes = 2 * kKRegionBytes;
 struct __align__(8) ABarriers {
     uint64_t b_full, b_empty;
     uint64_t k_full[kStages], k_empty[kStages];
-    uint64_t d_full[2], d_empty[2];
+    uint64_t d_full[kMaxGroups], d_empty[kMaxGroups];
     uint64_t nu_ready;
 };
 
@@ -74,10 +77,11 @@ struct TileWalk {
 
 __global__ void __launch_bounds__(kThreadsA, 1)
 assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmSeed,
-                 const UnitDesc* __restrict__ desc, Shape sh, int total_tiles, const float* __restrict__ s,
-                 const int32_t* __restrict__ plan, const int32_t* __restrict__ seed_rows,
-                 const float* __restrict__ seed_norm, uint8_t* __restrict__ kind, int32_t* __restrict__ seed_of,
-                 float* __restrict__ sim, int32_t* __restrict__ grp, unsigned long long* __restrict__ mass_fx,
+                 const UnitDesc* __restrict__ desc, Shape sh, int total_tiles, int n_groups,
+                 const float* __restrict__ s, const int32_t* __restrict__ plan,
+                 const int32_t* __restrict__ seed_rows, const float* __restrict__ seed_norm,
+                 uint8_t* __restrict__ kind, int32_t* __restrict__ seed_of, float* __restrict__ sim,
+                 int32_t* __restrict__ grp, unsigned long long* __restrict__ mass_fx,
                  int32_t* __restrict__ njoin, int max_m, float tau, float eps, int32_t* __restrict__ err) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -87,13 +91,14 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     ABarriers& bar = tail->bar;
     volatile int* abort_flag = &tail->abort;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int buf_cols = 512 / n_groups;                 // TMEM columns per accumulator buffer
 
     if (threadIdx.x == 0) {
         mbar_init(&bar.b_full, 1);
         mbar_init(&bar.b_empty, 1);
         for (int i = 0; i < kStages; ++i) { mbar_init(&bar.k_full[i], 1); mbar_init(&bar.k_empty[i], 1 + 4); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&bar.d_full[i], 1); mbar_init(&bar.d_empty[i], 4); }
-        mbar_init(&bar.nu_ready, kEpiThreads);
+        for (int i = 0; i < kMaxGroups; ++i) { mbar_init(&bar.d_full[i], 1); mbar_init(&bar.d_empty[i], 4); }
+        mbar_init(&bar.nu_ready, 128 * n_groups);
         tail->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -145,7 +150,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         if (lane == 0) {
             uint32_t kit = 0, ucount = 0;
             bool ok = true;
-            const uint32_t b_addr = smem_u32(b_smem), k_addr = smem_u32(k_smem);
+            const uint32_t b_lo = umma_desc_lo(smem_u32(b_smem)), k_lo = umma_desc_lo(smem_u32(k_smem));
             while (wk.valid() && ok) {
                 const UnitDesc& ud = desc[wk.u];
                 const int m = max(0, min(plan[wk.u * 8 + CASK_PLAN_M], ud.plan[CASK_PLAN_M]));
@@ -155,32 +160,36 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 ++ucount;
                 const int nt = wk.run();
                 for (int t = 0; t < nt && ok; ++t, ++kit) {
-                    const int st = kit % kStages, buf = kit & 1;
+                    const int st = kit % kStages;
+                    const uint32_t buf = kit % (uint32_t)n_groups, use = kit / (uint32_t)n_groups;
                     ok = mbar_wait(&bar.k_full[st], (kit / kStages) & 1u, abort_flag);
                     if (!ok) break;
-                    ok = mbar_wait(&bar.d_empty[buf], ((kit >> 1) & 1u) ^ 1u, abort_flag);
+                    ok = mbar_wait(&bar.d_empty[buf], (use & 1u) ^ 1u, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t kst = k_addr + st * kKStageBytes;
+                    const uint32_t kst_lo = k_lo + st * (kKStageBytes >> 4);
+                    const uint32_t d_addr = tmem_base + buf * buf_cols;
+                    tc_mma_lo<false>(d_addr, kst_lo, b_lo, idesc);
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {
+                    for (int kk = 1; kk < 8; ++kk) {
                         const int kb = kk >> 2, ks = kk & 3;
-                        uint64_t a = umma_desc(kst + kb * kKRegionBytes + ks * 32);
-                        uint64_t b = umma_desc(b_addr + kb * kSeedRegionBytes + ks * 32);
-                        tc_mma(tmem_base + 256 * buf, a, b, idesc, kk != 0);
+                        tc_mma_lo<true>(d_addr, kst_lo + ((kb * kKRegionBytes + ks * 32) >> 4),
+                                        b_lo + ((kb * kSeedRegionBytes + ks * 32) >> 4), idesc);
                     }
                     tc_commit(&bar.d_full[buf]);
                     tc_commit(&bar.k_empty[st]);
                 }
                 wk.advance(nt);
-                tc_commit(&bar.b_empty);
+                if (ok) tc_commit(&bar.b_empty);
             }
         }
-    } else if (warp >= kEpiWarp0) {
+    } else if (warp >= kEpiWarp0 && ((warp - kEpiWarp0) >> 2) < n_groups) {
         // ================= epilogue =================
-        const int qd = warp & 3;
-        const int etid = threadIdx.x - kEpiWarp0 * 32;
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * qd) << 16);
+        const int ew = warp - kEpiWarp0;
+        const int qd = ew & 3;                               // TMEM lane quadrant (== warp % 4)
+        const uint32_t eg = (uint32_t)(ew >> 2);             // group: tiles eg, eg + G, ... and buffer eg
+        const int etid = ew * 32 + lane;
+        const uint32_t taddr = tmem_base + ((uint32_t)(32 * qd) << 16) + eg * buf_cols;
         const int my_row = 32 * qd + lane;                   // row of the tile this thread owns
         uint32_t kit = 0, ucount = 0;
         bool ok = true;
@@ -188,13 +197,16 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const UnitDesc& ud = desc[wk.u];
             const int u = wk.u;
             const int T = ud.T, P = ud.P;
+            const int64_t tok_off = ud.tok_off;
+            const int seed_base = ud.seed_base;
             const int r = max(0, min(plan[u * 8 + CASK_PLAN_R], T - P));
             const int m = max(0, min(plan[u * 8 + CASK_PLAN_M], ud.plan[CASK_PLAN_M]));
             const int hi = T - r;
+            unsigned long long* mass_u = mass_fx + (size_t)u * (max_m + 1);
             float* inv = tail->inv_nu[ucount & 1u];
-            for (int c = etid; c < 256; c += kEpiThreads) {
-                float nu = (c < m) ? seed_norm[ud.seed_base + c] : 0.f;
-                inv[c] = nu > 0.f ? 1.f / nu : 0.f;
+            if (etid < 256) {
+                const float nu = (etid < m) ? seed_norm[seed_base + etid] : 0.f;
+                inv[etid] = nu > 0.f ? 1.f / nu : 0.f;
             }
             mbar_arrive(&bar.nu_ready);
             ok = mbar_wait(&bar.nu_ready, ucount & 1u, abort_flag);
@@ -203,7 +215,14 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const int tile0 = wk.tile_in_unit();
             const int nt = wk.run();
             for (int t = 0; t < nt && ok; ++t, ++kit) {
-                const int st = kit % kStages, buf = kit & 1;
+                if (kit % (uint32_t)n_groups != eg) continue;
+                const int st = kit % kStages;
+                const uint32_t use = kit / (uint32_t)n_groups;
+                // the row's kind and score are fetched now and used after the contraction
+                const int i = P + (tile0 + t) * kTileRows + my_row;
+                const bool in_range = i < hi;
+                const uint8_t kd = in_range ? kind[tok_off + i] : (uint8_t)CASK_KIND_RECENT;
+                const float sc = in_range ? s[tok_off + i] : 0.f;
                 // squared norm of this thread's row, read from the staged tile (any order of the
                 // sixteen 16-byte pieces of the row gives the same set of elements)
                 ok = mbar_wait(&bar.k_full[st], (kit / kStages) & 1u, abort_flag);
@@ -227,15 +246,15 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bar.k_empty[st]);
-                ok = mbar_wait(&bar.d_full[buf], (kit >> 1) & 1u, abort_flag);
+                ok = mbar_wait(&bar.d_full[eg], use & 1u, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
                 float best = -INFINITY, best_dot = 0.f;
                 int best_u = -1;
                 for (int cc = 0; cc < m; cc += 32) {
                     float v[32];
-                    tc_ld32(lane_addr + 256 * buf + cc, v);
-                    tc_wait_ld();
+                    tc_ld32(taddr + cc, v);
+                    tc_wait_ld_regs(v);
 #pragma unroll
                     for (int x = 0; x < 32; ++x) {
                         const float val = v[x] * inv[cc + x];
@@ -244,23 +263,33 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&bar.d_empty[buf]);
-                const int i = P + (tile0 + t) * kTileRows + my_row;
-                if (i < hi && best_u >= 0 && kind[ud.tok_off + i] == CASK_KIND_DROPPED) {
+                if (lane == 0) mbar_arrive(&bar.d_empty[eg]);
+
+                const bool cand = in_range && best_u >= 0 && kd == CASK_KIND_DROPPED;
+                float sm_ = 0.f;
+                if (cand) {
                     const float nj = sqrtf(n2);
-                    const float nu = seed_norm[ud.seed_base + best_u];
-                    const float sm_ = (nj > 0.f && nu > 0.f) ? best_dot / (nj * nu) : 0.f;
-                    if (sim) sim[ud.tok_off + i] = sm_;
-                    const unsigned long long fx = mass_to_fx(s[ud.tok_off + i] + eps);
-                    if (sm_ >= tau) {
-                        kind[ud.tok_off + i] = CASK_KIND_MERGED;
-                        seed_of[ud.tok_off + i] = seed_rows[ud.seed_base + best_u];
-                        grp[ud.tok_off + i] = best_u;
-                        atomicAdd(&mass_fx[(size_t)u * (max_m + 1) + best_u], fx);
-                        atomicAdd(&njoin[u], 1);
-                    } else {
-                        atomicAdd(&mass_fx[(size_t)u * (max_m + 1) + max_m], fx);
-                    }
+                    const float nu = seed_norm[seed_base + best_u];
+                    sm_ = (nj > 0.f && nu > 0.f) ? best_dot / (nj * nu) : 0.f;
+                    if (sim) sim[tok_off + i] = sm_;
+                }
+                const bool joined = cand && sm_ >= tau;
+                const unsigned long long fx = cand ? mass_to_fx(sc + eps) : 0ull;
+                if (joined) {
+                    kind[tok_off + i] = CASK_KIND_MERGED;
+                    seed_of[tok_off + i] = seed_rows[seed_base + best_u];
+                    grp[tok_off + i] = best_u;
+                    atomicAdd(&mass_u[best_u], fx);
+                }
+                // Joiner count and lost mass go out once per warp: the fixed-point sums are exact, so
+                // the grouping of the additions does not show in the result.
+                const unsigned jb = __ballot_sync(0xffffffffu, joined);
+                unsigned long long lost = joined ? 0ull : fx;
+#pragma unroll
+                for (int off = 16; off >= 1; off >>= 1) lost += __shfl_xor_sync(0xffffffffu, lost, off);
+                if (lane == 0) {
+                    if (jb) atomicAdd(&njoin[u], __popc(jb));
+                    if (lost) atomicAdd(&mass_u[max_m], lost);
                 }
             }
             wk.advance(nt);
@@ -316,7 +345,7 @@ cudaError_t launch_assign_tc(const Launch& L, const cask_params& prm, const floa
     {
         Timed t(L, KID_ASSIGN);
         assign_tc_kernel<<<grid, kThreadsA, kSmemBytesA, L.stream>>>(
-            tmK, tmSeed, L.desc, sh, L.total_atiles, s, plan, ws.seed_rows, ws.seed_norm, kind, seed_of, sim, ws.grp,
+            tmK, tmSeed, L.desc, sh, L.total_atiles, L.max_m <= 128 ? 4 : 2, s, plan, ws.seed_rows, ws.seed_norm, kind, seed_of, sim, ws.grp,
             ws.mass_fx, ws.njoin, L.max_m, prm.tau, prm.eps, ws.err);
     }
     return cudaGetLastError();

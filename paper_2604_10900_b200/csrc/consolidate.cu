@@ -41,32 +41,14 @@ __global__ void __launch_bounds__(kSelThreads) seeds_kernel(const UnitDesc* __re
     __syncthreads();
     if (m <= 0) return;
     block_topk_mark(s + o, kind + o, P, T - r, m, CASK_KIND_SEED, sm);
-    // ordered compaction of the seed rows
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
-    unsigned base = 0;
-    for (int i0 = P; i0 < T - r; i0 += blockDim.x) {
-        int i = i0 + threadIdx.x;
-        bool is = (i < T - r) && kind[o + i] == CASK_KIND_SEED;
-        unsigned bal = __ballot_sync(0xffffffffu, is);
-        __syncthreads();
-        if (lane == 0) sm.warp_cnt[w] = __popc(bal);
-        __syncthreads();
-        unsigned before = 0, all = 0;
-        for (int x = 0; x < nw; ++x) {
-            unsigned c = sm.warp_cnt[x];
-            if (x < w) before += c;
-            all += c;
+    // ordered list of the seed rows
+    block_ordered_rows(kind + o, P, T - r, CASK_KIND_SEED, sm, [&](unsigned idx, int i) {
+        if (idx < (unsigned)m) {
+            seed_rows[ud.seed_base + idx] = i;
+            seed_of[o + i] = i;
+            grp[o + i] = (int)idx;
         }
-        if (is) {
-            unsigned idx = base + before + __popc(bal & ((1u << lane) - 1u));
-            if (idx < (unsigned)m) {
-                seed_rows[ud.seed_base + idx] = i;
-                seed_of[o + i] = i;
-                grp[o + i] = (int)idx;
-            }
-        }
-        base += all;
-    }
+    });
 }
 
 // ---- 2. gather seed keys, their norms and their own mass ---------------------------------

@@ -1,17 +1,22 @@
 // Block-wide exact top-k by radix select on order-preserving uint32 score keys.
 // Total order: score descending, then row index ascending (the k-th score may be
 // tied; ties are taken in index order).
+//
+// Three histogram sweeps narrow the key of the k-th greatest row digit by digit (12 + 12 + 8
+// bits), a last sweep marks everything above it and the rows equal to it.  The sweeps read the
+// unit's scores from global memory; after the first one they are L1/L2 hits.
 #pragma once
 #include "cask_internal.cuh"
 
 namespace cask {
 
 constexpr int kSelThreads = 1024;
+constexpr int kSelBins = 4096;
 
 struct SelectSmem {
-    unsigned hist[256];
+    unsigned hist[kSelBins];
     unsigned warp_cnt[kSelThreads / 32];
-    unsigned prefix, krem, total, run;
+    unsigned digit, krem, neq;
 };
 
 // Sum of `v` over the block, returned to every thread.
@@ -28,14 +33,86 @@ __device__ __forceinline__ unsigned block_sum(unsigned v, SelectSmem& sm) {
     return t;
 }
 
+// Exclusive prefix of `v` over the block in thread order (total returned through `total`).
+__device__ __forceinline__ unsigned block_excl_scan(unsigned v, SelectSmem& sm, unsigned& total) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    unsigned incl = v;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        unsigned o = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += o;
+    }
+    __syncthreads();
+    if (lane == 31) sm.warp_cnt[w] = incl;
+    __syncthreads();
+    unsigned wv = (lane < nw) ? sm.warp_cnt[lane] : 0u;
+    unsigned wincl = wv;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        unsigned o = __shfl_up_sync(0xffffffffu, wincl, off);
+        if (lane >= off) wincl += o;
+    }
+    total = __shfl_sync(0xffffffffu, wincl, 31);
+    const unsigned wbefore = __shfl_sync(0xffffffffu, wincl - wv, w);
+    return wbefore + incl - v;
+}
+
+// With sm.hist[0..nbins) filled: the digit d such that fewer than krem keys lie in the bins above d
+// and at least krem in the bins >= d.  Leaves d in sm.digit, the rank inside bin d in sm.krem and
+// the population of bin d in sm.neq.  nbins <= 4 * blockDim.x.
+__device__ __forceinline__ void find_digit(SelectSmem& sm, int nbins, unsigned krem) {
+    const int tid = threadIdx.x;
+    // thread t owns the four bins nbins-1-4t .. nbins-4-4t, in descending order
+    unsigned c[4], tot = 0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const int b = nbins - 1 - 4 * tid - q;
+        c[q] = (b >= 0) ? sm.hist[b] : 0u;
+        tot += c[q];
+    }
+    unsigned total;
+    const unsigned before = block_excl_scan(tot, sm, total);
+    if (before < krem && krem <= before + tot) {
+        unsigned run = before;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            if (run < krem && krem <= run + c[q]) {
+                sm.digit = (unsigned)(nbins - 1 - 4 * tid - q);
+                sm.krem = krem - run;
+                sm.neq = c[q];
+            }
+            run += c[q];
+        }
+    }
+    __syncthreads();
+}
+
 // Among rows [lo,hi) with kind == 0, give `mark` to the k greatest.  All threads of the
 // block must call it with the same arguments.  s and kind are per-unit pointers.
 __device__ inline void block_topk_mark(const float* __restrict__ s, uint8_t* kind, int lo, int hi, int k,
-                                uint8_t mark, SelectSmem& sm) {
+                                       uint8_t mark, SelectSmem& sm) {
     if (k <= 0 || hi <= lo) return;
     const int tid = threadIdx.x, lane = tid & 31, nthr = blockDim.x;
+    const int span = hi - lo;
+    const int iters = (span + nthr - 1) / nthr;
+
+    // ---- sweep 1: top 12 bits ----
+    for (int b = tid; b < kSelBins; b += nthr) sm.hist[b] = 0;
+    __syncthreads();
     unsigned mine = 0;
-    for (int i = lo + tid; i < hi; i += nthr) mine += (kind[i] == 0);
+    for (int it = 0; it < iters; it += 4) {
+        unsigned key[4];
+        bool el[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int i = lo + (it + q) * nthr + tid;
+            el[q] = (i < hi) && kind[i] == 0;
+            key[q] = el[q] ? order_key(s[i]) : 0u;
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            if (el[q]) { atomicAdd(&sm.hist[key[q] >> 20], 1u); ++mine; }
+    }
     const unsigned n_elig = block_sum(mine, sm);
     if ((unsigned)k >= n_elig) {
         for (int i = lo + tid; i < hi; i += nthr)
@@ -43,77 +120,97 @@ __device__ inline void block_topk_mark(const float* __restrict__ s, uint8_t* kin
         __syncthreads();
         return;
     }
-    unsigned prefix = 0, mask = 0, krem = (unsigned)k;
-    const int span = hi - lo;
-    const int iters = (span + nthr - 1) / nthr;
-    for (int pass = 0; pass < 4; ++pass) {
-        const int shift = 24 - 8 * pass;
-        if (tid < 256) sm.hist[tid] = 0;
-        __syncthreads();
-        for (int it = 0; it < iters; ++it) {
-            int i = lo + it * nthr + tid;
-            unsigned bucket = 256u + lane;          // unique per lane: matches nobody
-            if (i < hi && kind[i] == 0) {
-                unsigned key = order_key(s[i]);
-                if ((key & mask) == prefix) bucket = (key >> shift) & 255u;
-            }
-            unsigned peers = __match_any_sync(0xffffffffu, bucket);
-            if (bucket < 256u && lane == __ffs(peers) - 1) atomicAdd(&sm.hist[bucket], __popc(peers));
+    find_digit(sm, kSelBins, (unsigned)k);
+    const unsigned d1 = sm.digit;
+    unsigned krem = sm.krem;
+    __syncthreads();
+
+    // ---- sweep 2: next 12 bits among the keys whose top digit is d1 ----
+    for (int b = tid; b < kSelBins; b += nthr) sm.hist[b] = 0;
+    __syncthreads();
+    for (int it = 0; it < iters; it += 4) {
+        unsigned key[4];
+        bool el[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int i = lo + (it + q) * nthr + tid;
+            el[q] = (i < hi) && kind[i] == 0;
+            key[q] = el[q] ? order_key(s[i]) : 0u;
         }
-        __syncthreads();
-        if (tid < 32) {
-            // lane L owns buckets 255-8L .. 248-8L (descending); find where the running count reaches krem
-            unsigned c[8], tot = 0;
 #pragma unroll
-            for (int t = 0; t < 8; ++t) { c[t] = sm.hist[255 - 8 * lane - t]; tot += c[t]; }
-            unsigned incl = tot;
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                unsigned o = __shfl_up_sync(0xffffffffu, incl, off);
-                if (lane >= off) incl += o;
-            }
-            unsigned before = incl - tot;           // count in buckets greater than this lane's
-            if (before < krem && krem <= incl) {
-                unsigned run = before;
-#pragma unroll
-                for (int t = 0; t < 8; ++t) {
-                    if (run < krem && krem <= run + c[t]) {
-                        sm.prefix = prefix | ((unsigned)(255 - 8 * lane - t) << shift);
-                        sm.krem = krem - run;
-                    }
-                    run += c[t];
-                }
-            }
-        }
-        __syncthreads();
-        prefix = sm.prefix;
-        krem = sm.krem;
-        mask |= 0xFFu << shift;
-        __syncthreads();
+        for (int q = 0; q < 4; ++q)
+            if (el[q] && (key[q] >> 20) == d1) atomicAdd(&sm.hist[(key[q] >> 8) & 0xFFFu], 1u);
     }
-    // prefix is now the key of the k-th greatest; krem of the rows equal to it are taken, lowest index first
+    __syncthreads();
+    find_digit(sm, kSelBins, krem);
+    const unsigned d12 = (d1 << 12) | sm.digit;
+    krem = sm.krem;
+    __syncthreads();
+
+    // ---- sweep 3: last 8 bits ----
+    for (int b = tid; b < 256; b += nthr) sm.hist[b] = 0;
+    __syncthreads();
+    for (int it = 0; it < iters; it += 4) {
+        unsigned key[4];
+        bool el[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int i = lo + (it + q) * nthr + tid;
+            el[q] = (i < hi) && kind[i] == 0;
+            key[q] = el[q] ? order_key(s[i]) : 0u;
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            if (el[q] && (key[q] >> 8) == d12) atomicAdd(&sm.hist[key[q] & 0xFFu], 1u);
+    }
+    __syncthreads();
+    find_digit(sm, 256, krem);
+    const unsigned thr = (d12 << 8) | sm.digit;     // key of the k-th greatest row
+    krem = sm.krem;                                  // how many of the rows equal to it are taken
+    const unsigned neq = sm.neq;
+    __syncthreads();
+
+    // ---- marking ----
+    if (krem == neq) {
+        for (int i = lo + tid; i < hi; i += nthr)
+            if (kind[i] == 0 && order_key(s[i]) >= thr) kind[i] = mark;
+        __syncthreads();
+        return;
+    }
+    // ties at the threshold: the lowest-index krem of them, found by an ordered scan
     unsigned eq_before = 0;
     for (int it = 0; it < iters; ++it) {
-        int i = lo + it * nthr + tid;
-        bool elig = (i < hi) && kind[i] == 0;
-        unsigned key = elig ? order_key(s[i]) : 0u;
-        bool gt = elig && key > prefix;
-        bool eq = elig && key == prefix;
-        unsigned bal = __ballot_sync(0xffffffffu, eq);
-        unsigned in_warp = __popc(bal & ((1u << lane) - 1u));
-        __syncthreads();
-        if (lane == 0) sm.warp_cnt[tid >> 5] = __popc(bal);
-        __syncthreads();
-        unsigned before = 0, all = 0;
-        for (int w = 0; w < (nthr >> 5); ++w) {
-            unsigned c = sm.warp_cnt[w];
-            if (w < (tid >> 5)) before += c;
-            all += c;
-        }
-        if (gt || (eq && eq_before + before + in_warp < krem)) kind[i] = mark;
+        const int i = lo + it * nthr + tid;
+        const bool elig = (i < hi) && kind[i] == 0;
+        const unsigned key = elig ? order_key(s[i]) : 0u;
+        const bool gt = elig && key > thr;
+        const bool eq = elig && key == thr;
+        const unsigned bal = __ballot_sync(0xffffffffu, eq);
+        const unsigned in_warp = __popc(bal & ((1u << lane) - 1u));
+        unsigned all;
+        const unsigned before = block_excl_scan(lane == 0 ? __popc(bal) : 0u, sm, all);
+        const unsigned wbefore = __shfl_sync(0xffffffffu, before, 0);
+        if (gt || (eq && eq_before + wbefore + in_warp < krem)) kind[i] = mark;
         eq_before += all;
     }
     __syncthreads();
+}
+
+// Rows of [lo,hi) with kind == want, in ascending order: calls emit(rank, row) for each.  Every
+// thread walks one contiguous chunk, so one block scan orders the whole range.
+template <typename Emit>
+__device__ inline void block_ordered_rows(const uint8_t* kind, int lo, int hi, uint8_t want, SelectSmem& sm,
+                                          Emit emit) {
+    const int span = hi - lo;
+    if (span <= 0) return;
+    const int chunk = (span + (int)blockDim.x - 1) / (int)blockDim.x;
+    const int b = lo + (int)threadIdx.x * chunk, e = min(hi, b + chunk);
+    unsigned cnt = 0;
+    for (int i = b; i < e; ++i) cnt += (kind[i] == want);
+    unsigned total;
+    unsigned rank = block_excl_scan(cnt, sm, total);
+    for (int i = b; i < e; ++i)
+        if (kind[i] == want) emit(rank++, i);
 }
 
 }  // namespace cask
