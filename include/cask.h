@@ -36,7 +36,8 @@ extern "C" {
 #define CASK_ERR_SHAPE         -2   /* head_dim/group/window/T/P/B/reserve out of range */
 #define CASK_ERR_ALIGN         -3   /* a base pointer, offset or row stride breaks the 16-byte rule */
 #define CASK_ERR_WORKSPACE     -4   /* workspace NULL or smaller than cask_workspace_bytes */
-#define CASK_ERR_UNSUPPORTED   -5   /* a documented but unbuilt mode (paged cache)    */
+#define CASK_ERR_UNSUPPORTED   -5   /* a documented but unbuilt combination (paged cache through
+                                       the host-buffer or the no-allocation entry point) */
 #define CASK_ERR_CUDA          -6   /* a CUDA runtime call failed (see cask_last_cuda_error) */
 #define CASK_ERR_PARAM         -7   /* gamma/tau/eps/causal out of range              */
 #define CASK_ERR_TOO_LARGE     -8   /* batch exceeds a fixed capacity (cask_score_noalloc) */
@@ -76,8 +77,17 @@ typedef struct cask_ctx cask_ctx;
 /*
  * A ragged batch of independent units (Sec. 2.3 of the paper constrains one
  * cache at a time: |R| <= B, C subset of R; nothing couples units).
- * Layout: contiguous rows.  Row i of unit u starts at element
+ * Layout, contiguous (page_size == 0): row i of unit u starts at element
  *   k + k_off[u] + i*row_stride            (same for v with v_off)
+ * Layout, paged (page_size > 0): k and v are page pools of n_pages pages of
+ * page_size rows; row i of unit u starts at element
+ *   k + (block_table[bt_off[u] + i/page_size]*page_size + i%page_size)*row_stride
+ * (same page ids for v); k_off and v_off are ignored.  The block table is read
+ * on the device; a page id outside [0, n_pages) raises CASK_ST_BOUNDS for the
+ * call and is treated as page 0, so nothing is read out of bounds.  The
+ * tensor-core kernels serve page sizes 8, 16, 32, 64 and multiples of 128;
+ * other page sizes run on the SIMT kernels.  The compacted cache is always
+ * written dense ([n_units, Bmax, d]).
  * row_stride >= head_dim; base pointers, offsets*elem and row_stride*elem must
  * be multiples of 16 bytes.  q is [n_units, group, window, head_dim], dense;
  * window query j of a unit belongs to cache row T-window+j.
@@ -88,7 +98,7 @@ typedef struct {
     int32_t group;           /* g: query heads per KV head, >= 1                */
     int32_t window;          /* W: 1 <= W <= T[u] for every unit               */
     int32_t dtype;           /* CASK_DTYPE_BF16 | CASK_DTYPE_FP32 (k, v, q, outputs) */
-    int32_t page_size;       /* 0 = contiguous rows; > 0 (paged) -> CASK_ERR_UNSUPPORTED */
+    int32_t page_size;       /* 0 = contiguous rows; > 0 = rows per page of a paged cache */
     const void* k;           /* DEVICE */
     const void* v;           /* DEVICE */
     const int64_t* k_off;    /* HOST [n_units], elements                        */
@@ -102,6 +112,10 @@ typedef struct {
     const int32_t* B;        /* HOST [n_units] budget, >= 1                     */
     const int32_t* reserve;  /* HOST [n_units] slots held back for decode, 0..B */
     const int64_t* tok_off;  /* HOST [n_units+1] offsets into per-row arrays; tok_off[u+1]-tok_off[u] >= T[u] */
+    /* paged cache only (page_size > 0) */
+    const int32_t* block_table; /* DEVICE physical page id of every logical page, unit after unit */
+    const int64_t* bt_off;   /* HOST [n_units+1] first entry of each unit; bt_off[u+1]-bt_off[u] >= ceil(T[u]/page_size) */
+    int64_t n_pages;         /* pages in the k and v pools                      */
 } cask_batch;
 
 /*
@@ -161,6 +175,10 @@ int cask_kernel_count(void);
 const char* cask_kernel_name(int id);
 /* 1 if the last cask_score / cask_compress_event used the tensor-core kernels. */
 int cask_last_score_path_tensor(const cask_ctx* ctx);
+/* Device-side flags (CASK_ST_TIMEOUT, CASK_ST_BOUNDS) raised by the kernels of the last call of this
+ * context; waits for the context's stream.  cask_consolidate_scratch and cask_compress_event also OR
+ * them into unit_status. */
+int cask_last_device_flags(cask_ctx* ctx, int32_t* flags_host);
 
 /* Bytes of workspace that any call below needs for this batch (host-only arithmetic). */
 size_t cask_workspace_bytes(const cask_batch* batch, const cask_params* params);
@@ -245,7 +263,8 @@ int cask_compress_event(cask_ctx* ctx, const cask_batch* batch, const cask_param
  * cask_host_event_device_bytes() that holds the staged inputs, outputs and the
  * workspace.  Copies in, runs cask_compress_event, copies out and synchronises
  * the stream before returning.  Rows of a unit must be dense (row_stride ==
- * head_dim) and units laid out at k_off[u] == v_off[u] == tok_off[u]*head_dim.
+ * head_dim) and units laid out at k_off[u] == v_off[u] == tok_off[u]*head_dim;
+ * a paged batch is refused with CASK_ERR_UNSUPPORTED.
  */
 size_t cask_host_event_device_bytes(const cask_batch* batch, const cask_params* params, int32_t Bmax);
 int cask_compress_event_host(cask_ctx* ctx, const cask_batch* host_batch, const cask_params* params,

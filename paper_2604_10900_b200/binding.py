@@ -28,7 +28,7 @@ DTYPE_BF16, DTYPE_FP32 = 0, 1
 
 EXPORTS = (
     "cask_create", "cask_destroy", "cask_set_stream", "cask_strerror", "cask_last_cuda_error",
-    "cask_launch_count", "cask_last_score_path_tensor", "cask_profile_enable", "cask_profile_read",
+    "cask_launch_count", "cask_last_score_path_tensor", "cask_last_device_flags", "cask_profile_enable", "cask_profile_read",
     "cask_kernel_count", "cask_kernel_name", "cask_workspace_bytes", "cask_plan_host",
     "cask_score", "cask_prefix_evict", "cask_select_core", "cask_consolidate_scratch", "cask_compact",
     "cask_compress_event", "cask_host_event_device_bytes", "cask_compress_event_host", "cask_score_noalloc",
@@ -44,6 +44,7 @@ class CaskBatch(C.Structure):
         ("q", C.c_void_p), ("lse_in", C.c_void_p),
         ("T", C.c_void_p), ("P", C.c_void_p), ("B", C.c_void_p), ("reserve", C.c_void_p),
         ("tok_off", C.c_void_p),
+        ("block_table", C.c_void_p), ("bt_off", C.c_void_p), ("n_pages", C.c_int64),
     ]
 
 
@@ -86,6 +87,7 @@ def lib():
         L.cask_launch_count.argtypes = [vp]
         L.cask_launch_count.restype = C.c_int64
         L.cask_last_score_path_tensor.argtypes = [vp]
+        L.cask_last_device_flags.argtypes = [vp, vp]
         L.cask_profile_enable.argtypes = [vp, i32]
         L.cask_profile_read.argtypes = [vp, vp, vp]
         L.cask_kernel_name.argtypes = [i32]
@@ -146,9 +148,12 @@ class HostArrays:
 
 
 def make_batch(k, v, q, T, P, B, reserve, tok_off, head_dim: int, group: int, window: int, dtype: int,
-               k_off=None, v_off=None, row_stride: Optional[int] = None, lse_in=None, page_size: int = 0):
+               k_off=None, v_off=None, row_stride: Optional[int] = None, lse_in=None, page_size: int = 0,
+               block_table=None, bt_off=None, n_pages: int = 0):
     """Fills a cask_batch.  k, v, q, lse_in: tensors/arrays/addresses (device for the device calls,
-    host for cask_compress_event_host).  Returns (struct, keepalive)."""
+    host for cask_compress_event_host).  Paged cache: page_size > 0, k and v the page pools,
+    block_table a device int32 tensor, bt_off the host offsets of the units in it.
+    Returns (struct, keepalive)."""
     tok_off = np.ascontiguousarray(tok_off, np.int64)
     if k_off is None:
         k_off = tok_off[:-1] * head_dim
@@ -163,7 +168,11 @@ def make_batch(k, v, q, T, P, B, reserve, tok_off, head_dim: int, group: int, wi
     b.row_stride = head_dim if row_stride is None else row_stride
     b.T, b.P, b.B, b.reserve = h.T.ctypes.data, h.P.ctypes.data, h.B.ctypes.data, h.reserve.ctypes.data
     b.tok_off = h.tok_off.ctypes.data
-    return b, (h, k, v, q, lse_in)
+    bt_host = None if bt_off is None else np.ascontiguousarray(bt_off, np.int64)
+    b.block_table = _ptr(block_table)
+    b.bt_off = None if bt_host is None else bt_host.ctypes.data
+    b.n_pages = n_pages
+    return b, (h, k, v, q, lse_in, block_table, bt_host)
 
 
 def make_outputs(d: Dict, Bmax: int) -> CaskOutputs:
@@ -220,6 +229,14 @@ class Context:
     @property
     def used_tensor_path(self) -> bool:
         return bool(lib().cask_last_score_path_tensor(self.handle))
+
+    def device_flags(self) -> int:
+        """CASK_ST_* bits raised on the device by the last call (waits for the stream)."""
+        f = C.c_int32(0)
+        rc = lib().cask_last_device_flags(self.handle, C.byref(f))
+        if rc != OK:
+            raise CaskError(rc, self.handle)
+        return int(f.value)
 
 
 def _check(rc: int, ctx: Optional[Context] = None):

@@ -1,5 +1,6 @@
 // C-ABI layer of libcask: argument checks, budget split, workspace carving, call sequencing.
 // Every error is found here, on the host, before anything is launched.
+#include <climits>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -45,6 +46,7 @@ struct cask_ctx {
     int64_t launches = 0;
     cudaError_t last_err = cudaSuccess;
     int last_tc = 0;
+    const int32_t* flags_dev = nullptr;   // flag word of the last call's workspace
     void* tmap_encode = nullptr;     // cuTensorMapEncodeTiled, resolved at creation
     Profiler prof;
     ProfImpl prof_impl;
@@ -93,7 +95,7 @@ void plan_unit(int T, int P, int B, int reserve, int W, float gamma, int32_t* pl
 int check_batch(const cask_batch* b, const cask_params* p) {
     if (!b || !p) return CASK_ERR_NULL;
     if (b->n_units < 0) return CASK_ERR_SHAPE;
-    if (b->page_size != 0) return CASK_ERR_UNSUPPORTED;
+    if (b->page_size < 0) return CASK_ERR_SHAPE;
     if (b->dtype != CASK_DTYPE_BF16 && b->dtype != CASK_DTYPE_FP32) return CASK_ERR_SHAPE;
     if (b->head_dim < 8 || b->head_dim > 256 || b->head_dim % 8) return CASK_ERR_SHAPE;
     if (b->group < 1 || b->window < 1 || (int64_t)b->group * b->window > 65536) return CASK_ERR_SHAPE;
@@ -101,9 +103,11 @@ int check_batch(const cask_batch* b, const cask_params* p) {
         (p->causal != 0 && p->causal != 1) || (p->score_path != 0 && p->score_path != 1))
         return CASK_ERR_PARAM;
     if (b->n_units == 0) return CASK_OK;
-    if (!b->k || !b->v || !b->q || !b->k_off || !b->v_off || !b->T || !b->P || !b->B || !b->reserve ||
-        !b->tok_off)
-        return CASK_ERR_NULL;
+    const bool paged = b->page_size > 0;
+    if (!b->k || !b->v || !b->q || !b->T || !b->P || !b->B || !b->reserve || !b->tok_off) return CASK_ERR_NULL;
+    if (!paged && (!b->k_off || !b->v_off)) return CASK_ERR_NULL;
+    if (paged && (!b->block_table || !b->bt_off)) return CASK_ERR_NULL;
+    if (paged && (b->n_pages < 1 || (uintptr_t)b->block_table % 4)) return CASK_ERR_SHAPE;
     const size_t e = elem_size(b->dtype);
     if (b->row_stride < b->head_dim) return CASK_ERR_SHAPE;
     if (((uintptr_t)b->k | (uintptr_t)b->v | (uintptr_t)b->q) % 16 || (b->row_stride * e) % 16)
@@ -112,8 +116,14 @@ int check_batch(const cask_batch* b, const cask_params* p) {
     for (int u = 0; u < b->n_units; ++u) {
         const int T = b->T[u], P = b->P[u], B = b->B[u], R = b->reserve[u];
         if (T < 1 || b->window > T || P < 0 || P > T || B < 1 || R < 0 || R > B) return CASK_ERR_SHAPE;
-        if (b->k_off[u] < 0 || b->v_off[u] < 0) return CASK_ERR_SHAPE;
-        if ((b->k_off[u] * e) % 16 || (b->v_off[u] * e) % 16) return CASK_ERR_ALIGN;
+        if (paged) {
+            const int64_t need = ((int64_t)T + b->page_size - 1) / b->page_size;
+            if (b->bt_off[u] < 0 || b->bt_off[u + 1] - b->bt_off[u] < need || b->bt_off[u + 1] > INT32_MAX)
+                return CASK_ERR_SHAPE;
+        } else {
+            if (b->k_off[u] < 0 || b->v_off[u] < 0) return CASK_ERR_SHAPE;
+            if ((b->k_off[u] * e) % 16 || (b->v_off[u] * e) % 16) return CASK_ERR_ALIGN;
+        }
         if (b->tok_off[u] < 0 || b->tok_off[u + 1] - b->tok_off[u] < T) return CASK_ERR_SHAPE;
     }
     return CASK_OK;
@@ -205,12 +215,17 @@ int prepare(cask_ctx* ctx, const cask_batch* b, const cask_params* p, void* ws, 
         if (e != cudaSuccess) return fail_cuda(ctx, e);
         ctx->pinned_units = (size_t)b->n_units;
     }
+    Shape shp{};
+    shp.page_size = b->page_size;
+    const int a_sub = b->page_size ? assign_tc_box_rows(shp) : 0;    // page piece the assignment tiles start on
     int chunk0 = 0, seed_base = 0, atile0 = 0, tile0 = 0;
     const int64_t q_unit = (int64_t)b->group * b->window * b->head_dim;
     for (int u = 0; u < b->n_units; ++u) {
         UnitDesc& d = ctx->pinned[u];
-        d.k_off = b->k_off[u];
-        d.v_off = b->v_off[u];
+        d.k_off = b->page_size ? 0 : b->k_off[u];
+        d.v_off = b->page_size ? 0 : b->v_off[u];
+        d.bt0 = b->page_size ? (int32_t)b->bt_off[u] : 0;
+        d.pad = 0;
         d.q_off = q_unit * u;
         d.tok_off = b->tok_off[u];
         d.T = b->T[u]; d.P = b->P[u]; d.B = b->B[u]; d.reserve = b->reserve[u];
@@ -219,7 +234,8 @@ int prepare(cask_ctx* ctx, const cask_batch* b, const cask_params* p, void* ws, 
         d.n_chunks = (d.T + kChunkKeys - 1) / kChunkKeys;
         d.seed_base = seed_base;
         d.atile0 = atile0;
-        d.n_atiles = d.plan[CASK_PLAN_M] > 0 ? (d.T - d.plan[CASK_PLAN_R] - d.P + 127) / 128 : 0;
+        const int a0 = d.P - (a_sub > 0 ? d.P % a_sub : 0);
+        d.n_atiles = d.plan[CASK_PLAN_M] > 0 ? (d.T - d.plan[CASK_PLAN_R] - a0 + 127) / 128 : 0;
         d.tile0 = tile0;
         tile0 += (d.T + 127) / 128;
         chunk0 += d.n_chunks;
@@ -232,11 +248,15 @@ int prepare(cask_ctx* ctx, const cask_batch* b, const cask_params* p, void* ws, 
     e = cudaEventRecord(ctx->staged, ctx->stream);
     if (e != cudaSuccess) return fail_cuda(ctx, e);
     ctx->staged_pending = true;
+    e = cudaMemsetAsync(W.err, 0, 16, ctx->stream);      // device-side flags of this call
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    ctx->flags_dev = W.err;
 
     L.stream = ctx->stream;
     L.sh.n_units = b->n_units; L.sh.d = b->head_dim; L.sh.g = b->group; L.sh.W = b->window;
     L.sh.rows = b->group * b->window; L.sh.dtype = b->dtype; L.sh.row_stride = b->row_stride;
     L.sh.causal = p->causal;
+    L.sh.page_size = b->page_size; L.sh.n_pages = b->n_pages; L.sh.bt = b->block_table; L.sh.err = W.err;
     L.desc = W.desc; L.hdesc = ctx->pinned;
     L.k = b->k; L.v = b->v; L.q = b->q;
     L.max_T = z.max_T; L.max_m = z.max_m; L.max_chunks = z.max_chunks; L.total_chunks = z.total_chunks;
@@ -320,7 +340,7 @@ const char* cask_strerror(int code) {
         case CASK_ERR_SHAPE: return "shape out of range (head_dim, group, window, T, P, B, reserve, offsets)";
         case CASK_ERR_ALIGN: return "pointer, offset or row stride is not a multiple of 16 bytes";
         case CASK_ERR_WORKSPACE: return "workspace missing, misaligned (256 B) or too small";
-        case CASK_ERR_UNSUPPORTED: return "mode not built (paged cache)";
+        case CASK_ERR_UNSUPPORTED: return "mode not built (paged cache through the host-buffer entry point)";
         case CASK_ERR_CUDA: return "CUDA runtime error";
         case CASK_ERR_PARAM: return "policy parameter out of range";
         case CASK_ERR_TOO_LARGE: return "batch exceeds the fixed capacity of the no-allocation entry point";
@@ -370,6 +390,17 @@ int cask_profile_read(cask_ctx* ctx, float* ms, int64_t* launches) {
     return CASK_OK;
 }
 int cask_last_score_path_tensor(const cask_ctx* ctx) { return ctx ? ctx->last_tc : 0; }
+
+int cask_last_device_flags(cask_ctx* ctx, int32_t* flags_host) {
+    if (!ctx || !flags_host) return CASK_ERR_NULL;
+    *flags_host = 0;
+    if (!ctx->flags_dev) return CASK_OK;
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(flags_host, ctx->flags_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, ctx->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+    return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
+}
 
 size_t cask_workspace_bytes(const cask_batch* batch, const cask_params* params) {
     if (check_batch(batch, params) != CASK_OK || batch->n_units == 0) return 0;
@@ -553,6 +584,7 @@ int cask_compress_event_host(cask_ctx* ctx, const cask_batch* hb, const cask_par
     if (!ctx || !ho) return CASK_ERR_NULL;
     int rc = check_batch(hb, p);
     if (rc != CASK_OK) return rc;
+    if (hb->page_size != 0) return CASK_ERR_UNSUPPORTED;
     if (hb->n_units == 0) return CASK_OK;
     rc = check_host_layout(hb);
     if (rc != CASK_OK) return rc;

@@ -77,7 +77,7 @@ struct TileWalk {
 
 __global__ void __launch_bounds__(kThreadsA, 1)
 assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmSeed,
-                 const UnitDesc* __restrict__ desc, Shape sh, int total_tiles, int n_groups,
+                 const UnitDesc* __restrict__ desc, Shape sh, int total_tiles, int n_groups, int sub_rows,
                  const float* __restrict__ s, const int32_t* __restrict__ plan,
                  const int32_t* __restrict__ seed_rows, const float* __restrict__ seed_norm,
                  uint8_t* __restrict__ kind, int32_t* __restrict__ seed_of, float* __restrict__ sim,
@@ -127,16 +127,30 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 tma_load_2d(b_smem, &tmSeed, &bar.b_full, 0, ud.seed_base);
                 tma_load_2d(b_smem + kSeedRegionBytes, &tmSeed, &bar.b_full, 64, ud.seed_base);
                 ++ucount;
-                const int row0 = (int)(ud.k_off / sh.row_stride) + ud.P + wk.tile_in_unit() * kTileRows;
+                // first cache row of the unit's tile sequence (a page-piece boundary in a paged cache)
+                const int a0 = ud.P - (sh.page_size ? ud.P % sub_rows : 0);
+                const int lrow0 = a0 + wk.tile_in_unit() * kTileRows;
+                const int krow0 = sh.page_size ? 0 : (int)(ud.k_off / sh.row_stride);
                 const int nt = wk.run();
                 for (int t = 0; t < nt && ok; ++t, ++kit) {
                     const int st = kit % kStages;
                     ok = mbar_wait(&bar.k_empty[st], ((kit / kStages) & 1u) ^ 1u, abort_flag);
                     if (!ok) break;
-                    mbar_expect_tx(&bar.k_full[st], kKStageBytes);
                     uint8_t* dst = k_smem + st * kKStageBytes;
-                    tma_load_2d(dst, &tmK, &bar.k_full[st], 0, row0 + t * kTileRows);
-                    tma_load_2d(dst + kKRegionBytes, &tmK, &bar.k_full[st], 64, row0 + t * kTileRows);
+                    const int lrow = lrow0 + t * kTileRows;
+                    if (sh.page_size == 0) {
+                        mbar_expect_tx(&bar.k_full[st], kKStageBytes);
+                        tma_load_2d(dst, &tmK, &bar.k_full[st], 0, krow0 + lrow);
+                        tma_load_2d(dst + kKRegionBytes, &tmK, &bar.k_full[st], 64, krow0 + lrow);
+                    } else {
+                        const int n_sub = min(kTileRows / sub_rows, (ud.T - lrow + sub_rows - 1) / sub_rows);
+                        mbar_expect_tx(&bar.k_full[st], (uint32_t)n_sub * sub_rows * 256u);
+                        for (int sb = 0; sb < n_sub; ++sb) {
+                            const int prow = (int)paged_row(sh, ud, lrow + sb * sub_rows);
+                            tma_load_2d(dst + sb * sub_rows * 128, &tmK, &bar.k_full[st], 0, prow);
+                            tma_load_2d(dst + kKRegionBytes + sb * sub_rows * 128, &tmK, &bar.k_full[st], 64, prow);
+                        }
+                    }
                 }
                 wk.advance(nt);
             }
@@ -202,6 +216,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const int r = max(0, min(plan[u * 8 + CASK_PLAN_R], T - P));
             const int m = max(0, min(plan[u * 8 + CASK_PLAN_M], ud.plan[CASK_PLAN_M]));
             const int hi = T - r;
+            const int a0 = P - (sh.page_size ? P % sub_rows : 0);
             unsigned long long* mass_u = mass_fx + (size_t)u * (max_m + 1);
             float* inv = tail->inv_nu[ucount & 1u];
             if (etid < 256) {
@@ -219,8 +234,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 const int st = kit % kStages;
                 const uint32_t use = kit / (uint32_t)n_groups;
                 // the row's kind and score are fetched now and used after the contraction
-                const int i = P + (tile0 + t) * kTileRows + my_row;
-                const bool in_range = i < hi;
+                const int i = a0 + (tile0 + t) * kTileRows + my_row;
+                const bool in_range = i >= P && i < hi;
                 const uint8_t kd = in_range ? kind[tok_off + i] : (uint8_t)CASK_KIND_RECENT;
                 const float sc = in_range ? s[tok_off + i] : 0.f;
                 // squared norm of this thread's row, read from the staged tile (any order of the
@@ -307,10 +322,19 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
 }  // namespace
 
+// Rows per TMA box of the key stream (see the scoring kernel): 128, one page piece, or 0 if unsupported.
+int assign_tc_box_rows(const Shape& sh) {
+    if (sh.page_size == 0) return kTileRows;
+    if (sh.page_size % kTileRows == 0) return kTileRows;
+    if (sh.page_size >= 8 && kTileRows % sh.page_size == 0) return sh.page_size;
+    return 0;
+}
+
 bool assign_tc_supported(const Launch& L) {
     const Shape& sh = L.sh;
     if (sh.dtype != CASK_DTYPE_BF16 || sh.d != 128 || L.max_m > 256 || L.max_m < 1 || L.total_atiles < 1)
         return false;
+    if (sh.page_size) return assign_tc_box_rows(sh) != 0 && sh.n_pages * sh.page_size < ((int64_t)1 << 31);
     int64_t max_row = 0;
     for (int u = 0; u < sh.n_units; ++u) {
         const UnitDesc& d = L.hdesc[u];
@@ -323,13 +347,14 @@ bool assign_tc_supported(const Launch& L) {
 cudaError_t launch_assign_tc(const Launch& L, const cask_params& prm, const float* s, const int32_t* plan,
                              uint8_t* kind, int32_t* seed_of, float* sim, Workspace& ws, void* tmap_encode_fn) {
     const Shape& sh = L.sh;
-    int64_t k_rows = 0, sum_m = 0;
+    int64_t k_rows = sh.page_size ? sh.n_pages * sh.page_size : 0, sum_m = 0;
     for (int u = 0; u < sh.n_units; ++u) {
-        k_rows = std::max<int64_t>(k_rows, L.hdesc[u].k_off / sh.row_stride + L.hdesc[u].T);
+        if (!sh.page_size) k_rows = std::max<int64_t>(k_rows, L.hdesc[u].k_off / sh.row_stride + L.hdesc[u].T);
         sum_m += L.hdesc[u].plan[CASK_PLAN_M];
     }
+    const int sub_rows = assign_tc_box_rows(sh);
     CUtensorMap tmK, tmSeed;
-    if (!encode_rows_bf16(tmap_encode_fn, &tmK, L.k, (uint64_t)k_rows, (uint64_t)sh.row_stride * 2, kTileRows))
+    if (!encode_rows_bf16(tmap_encode_fn, &tmK, L.k, (uint64_t)k_rows, (uint64_t)sh.row_stride * 2, sub_rows))
         return cudaErrorInvalidValue;
     // the seed table has 256 spare rows behind the last seed, so a full box never leaves the allocation
     if (!encode_rows_bf16(tmap_encode_fn, &tmSeed, ws.seed_k, (uint64_t)sum_m + 256, 256, 256))
@@ -345,7 +370,7 @@ cudaError_t launch_assign_tc(const Launch& L, const cask_params& prm, const floa
     {
         Timed t(L, KID_ASSIGN);
         assign_tc_kernel<<<grid, kThreadsA, kSmemBytesA, L.stream>>>(
-            tmK, tmSeed, L.desc, sh, L.total_atiles, L.max_m <= 128 ? 4 : 2, s, plan, ws.seed_rows, ws.seed_norm, kind, seed_of, sim, ws.grp,
+            tmK, tmSeed, L.desc, sh, L.total_atiles, L.max_m <= 128 ? 4 : 2, sub_rows, s, plan, ws.seed_rows, ws.seed_norm, kind, seed_of, sim, ws.grp,
             ws.mass_fx, ws.njoin, L.max_m, prm.tau, prm.eps, ws.err);
     }
     return cudaGetLastError();

@@ -24,6 +24,8 @@ struct UnitDesc {
     int32_t atile0;     // first 128-row scratch tile of this unit in the assignment pass
     int32_t n_atiles;   // scratch tiles of this unit: ceil((T - r - P)/128) when m > 0, else 0
     int32_t tile0;      // first 128-key tile of this unit in the unit-major tile sequence of the scoring passes
+    int32_t bt0;        // paged cache: first entry of this unit in the block table
+    int32_t pad;
 };
 
 struct Shape {
@@ -31,6 +33,11 @@ struct Shape {
     int dtype;
     int64_t row_stride;
     int causal;
+    // paged cache (page_size > 0): row i of a unit lives in physical page bt[bt0 + i / page_size]
+    int page_size;
+    int64_t n_pages;
+    const int32_t* bt;   // device
+    int32_t* err;        // device flag word (CASK_ST_TIMEOUT, CASK_ST_BOUNDS)
 };
 
 // Kernel ids for the optional per-kernel event timing.
@@ -116,6 +123,7 @@ cudaError_t launch_compact(const Launch& L, const cask_params& prm, const float*
 
 // Tensor-core assignment of scratch rows to seeds (cosine Gram + argmax), same outputs as the SIMT kernel.
 bool assign_tc_supported(const Launch& L);
+int assign_tc_box_rows(const Shape& sh);   // rows per TMA box of the key stream, 0 if the page size does not fit
 cudaError_t launch_assign_tc(const Launch& L, const cask_params& prm, const float* s, const int32_t* plan,
                              uint8_t* kind, int32_t* seed_of, float* sim, Workspace& ws, void* tmap_encode_fn);
 
@@ -126,6 +134,23 @@ cudaError_t launch_score_tc(const Launch& L, const float* lse_in, float* s, floa
                             Workspace& ws, void* tmap_encode_fn);
 
 // ---- small device helpers ------------------------------------------------------
+// Physical row (in units of rows of the K/V arrays) of logical row i of a unit in a paged cache.  A
+// page id outside the pool raises CASK_ST_BOUNDS and is replaced by page 0, so nothing is read out
+// of bounds.
+__device__ __forceinline__ int64_t paged_row(const Shape& sh, const UnitDesc& ud, int i) {
+    int32_t pg = sh.bt[ud.bt0 + i / sh.page_size];
+    if ((uint64_t)(int64_t)pg >= (uint64_t)sh.n_pages) {
+        atomicOr(sh.err, CASK_ST_BOUNDS);
+        pg = 0;
+    }
+    return (int64_t)pg * sh.page_size + i % sh.page_size;
+}
+// Element offset of logical row i of a unit in the K (unit_off = k_off) or V (v_off) array.
+__device__ __forceinline__ int64_t row_elem_off(const Shape& sh, const UnitDesc& ud, int64_t unit_off, int i) {
+    if (sh.page_size == 0) return unit_off + (int64_t)i * sh.row_stride;
+    return paged_row(sh, ud, i) * sh.row_stride;
+}
+
 template <typename T> struct Elem;
 template <> struct Elem<float> {
     static __device__ __forceinline__ float ld(const float* p) { return *p; }

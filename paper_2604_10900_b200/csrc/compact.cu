@@ -100,8 +100,8 @@ __global__ void __launch_bounds__(256) gather_merge_kernel(
     const uint8_t kd = slot_kind[(size_t)u * Bmax + t];
     T* ko = k_out + ((size_t)u * Bmax + t) * d;
     T* vo = v_out + ((size_t)u * Bmax + t) * d;
-    const T* ksrc = K + ud.k_off + (int64_t)src * sh.row_stride;
-    const T* vsrc = V + ud.v_off + (int64_t)src * sh.row_stride;
+    const T* ksrc = K + row_elem_off(sh, ud, ud.k_off, src);
+    const T* vsrc = V + row_elem_off(sh, ud, ud.v_off, src);
     const int nvec = d * (int)sizeof(T) / 16;
 
     bool copy = true;
@@ -126,8 +126,8 @@ __global__ void __launch_bounds__(256) gather_merge_kernel(
                 const float wi = weight[o + i];
                 msum += s[o + i] + eps;
                 ++count;
-                const T* kr = K + ud.k_off + (int64_t)i * sh.row_stride;
-                const T* vr = V + ud.v_off + (int64_t)i * sh.row_stride;
+                const T* kr = K + row_elem_off(sh, ud, ud.k_off, i);
+                const T* vr = V + row_elem_off(sh, ud, ud.v_off, i);
 #pragma unroll
                 for (int x = 0; x < kMaxPerLane; ++x) {
                     const int c = lane + 32 * x;

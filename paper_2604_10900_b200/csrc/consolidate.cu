@@ -63,7 +63,7 @@ __global__ void seed_gather_kernel(const UnitDesc* __restrict__ desc, Shape sh, 
     const int m = max(0, min(plan[u * 8 + CASK_PLAN_M], ud.plan[CASK_PLAN_M]));
     if (j >= m) return;
     const int row = seed_rows[ud.seed_base + j];
-    const T* src = K + ud.k_off + (int64_t)row * sh.row_stride;
+    const T* src = K + row_elem_off(sh, ud, ud.k_off, row);
     T* dst = seed_k + (size_t)(ud.seed_base + j) * sh.d;
     float n2 = 0.f;
     for (int c = threadIdx.x; c < sh.d; c += 32) {
@@ -111,7 +111,7 @@ __global__ void __launch_bounds__(kThreads) assign_simt_kernel(
 #pragma unroll
             for (int t = 0; t < 8; ++t)
                 St[rr * pitch + c8 + t] =
-                    (rr < nrows) ? Elem<T>::ld(K + ud.k_off + (int64_t)(lo + rr) * sh.row_stride + c8 + t) : 0.f;
+                    (rr < nrows) ? Elem<T>::ld(K + row_elem_off(sh, ud, ud.k_off, lo + rr) + c8 + t) : 0.f;
         }
     }
     __syncthreads();
@@ -206,7 +206,7 @@ __global__ void weights_kernel(const UnitDesc* __restrict__ desc, const float* _
                                const unsigned long long* __restrict__ mass_fx,
                                const int32_t* __restrict__ njoin, float* __restrict__ weight,
                                int32_t* __restrict__ unit_status, float* __restrict__ lost_mass, int max_m,
-                               float eps) {
+                               float eps, const int32_t* __restrict__ err) {
     const int u = blockIdx.y;
     const UnitDesc& ud = desc[u];
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -218,7 +218,7 @@ __global__ void weights_kernel(const UnitDesc* __restrict__ desc, const float* _
     if (i == 0) {
         int fl = plan[u * 8 + CASK_PLAN_FLAGS];
         if ((fl & CASK_ST_DECODE_CONSOLIDATED) && njoin[u] == 0) fl |= CASK_ST_MERGE_INACTIVE;
-        unit_status[u] = fl;
+        unit_status[u] = fl | *err;     // device-side flags of this call (bounded wait gave up, bad page id)
         lost_mass[u] = fx_to_mass(mf[max_m]);
     }
 }
@@ -259,7 +259,7 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const i
     {
         Timed t(L, KID_WEIGHTS);
         weights_kernel<<<dim3((L.max_T + 255) / 256, sh.n_units), 256, 0, L.stream>>>(
-            L.desc, s, plan, ws.grp, ws.mass_fx, ws.njoin, weight, unit_status, lost_mass, max_m, prm.eps);
+            L.desc, s, plan, ws.grp, ws.mass_fx, ws.njoin, weight, unit_status, lost_mass, max_m, prm.eps, ws.err);
     }
     return cudaGetLastError();
 }

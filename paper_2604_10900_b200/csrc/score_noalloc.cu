@@ -41,6 +41,7 @@ extern "C" int cask_score_noalloc(int device, void* cuda_stream, const cask_batc
     if (!s) return CASK_ERR_NULL;
     int rc = check_batch_host(b, p);
     if (rc != CASK_OK) return rc;
+    if (b->page_size != 0) return CASK_ERR_UNSUPPORTED;     // contiguous caches only
     if (b->n_units == 0) return CASK_OK;
     if (device < 0 || device >= kMaxDevices) return CASK_ERR_SHAPE;
     if (b->n_units > CASK_NOALLOC_MAX_UNITS) return CASK_ERR_TOO_LARGE;

@@ -15,6 +15,29 @@ namespace {
 constexpr int kTile = 64;
 constexpr int kThreads = 256;
 
+// Tile of 64 rows starting at row0 of `src` with a fixed row pitch (the dense query block).
+template <typename T>
+__device__ __forceinline__ void load_tile(float* dst, int pitch, const T* src, int64_t row_stride,
+                                          int row0, int n_valid_rows, int d);
+
+// Tile of 64 cache rows of a unit (contiguous or paged keys).
+template <typename T>
+__device__ __forceinline__ void load_key_tile(float* dst, int pitch, const T* K, const Shape& sh, const UnitDesc& ud,
+                                              int row0, int n_valid_rows, int d) {
+    if (sh.page_size == 0) {
+        load_tile<T>(dst, pitch, K + ud.k_off, sh.row_stride, row0, n_valid_rows, d);
+        return;
+    }
+    const int vec_per_row = d / 8;
+    for (int idx = threadIdx.x; idx < kTile * vec_per_row; idx += kThreads) {
+        int r = idx / vec_per_row, c8 = (idx % vec_per_row) * 8;
+#pragma unroll
+        for (int t = 0; t < 8; ++t)
+            dst[r * pitch + c8 + t] =
+                (r < n_valid_rows) ? Elem<T>::ld(K + row_elem_off(sh, ud, ud.k_off, row0 + r) + c8 + t) : 0.f;
+    }
+}
+
 template <typename T>
 __device__ __forceinline__ void load_tile(float* dst, int pitch, const T* src, int64_t row_stride,
                                           int row0, int n_valid_rows, int d) {
@@ -101,7 +124,7 @@ __global__ void __launch_bounds__(kThreads) score_norm_simt(const UnitDesc* __re
     const int key_end = min(Tn, (kc + 1) * kChunkKeys);
     for (int key0 = kc * kChunkKeys; key0 < key_end; key0 += kTile) {
         __syncthreads();
-        load_tile<T>(Rt, pitch, K + ud.k_off, sh.row_stride, key0, min(kTile, Tn - key0), d);
+        load_key_tile<T>(Rt, pitch, K, sh, ud, key0, min(kTile, Tn - key0), d);
         __syncthreads();
         float acc[4][4];
         tile_product(St, Rt, pitch, d, ty, tx, acc);
@@ -165,7 +188,7 @@ __global__ void __launch_bounds__(kThreads) score_mass_simt(const UnitDesc* __re
     const float* rm = rowm + (size_t)blockIdx.y * rows;
     const float* rw = roww + (size_t)blockIdx.y * rows;
 
-    load_tile<T>(St, pitch, K + ud.k_off, sh.row_stride, key0, min(kTile, Tn - key0), d);
+    load_key_tile<T>(St, pitch, K, sh, ud, key0, min(kTile, Tn - key0), d);
     float accs[4] = {0.f, 0.f, 0.f, 0.f};
     for (int row0 = 0; row0 < rows; row0 += kTile) {
         __syncthreads();

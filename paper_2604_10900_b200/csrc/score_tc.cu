@@ -196,7 +196,7 @@ struct TileWalk {
 template <int PASS>   // 0: normaliser, 1: score mass
 __global__ void __launch_bounds__(kThreadsTc, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
-                const UnitDesc* __restrict__ desc, Shape sh, int total_tiles,
+                const UnitDesc* __restrict__ desc, Shape sh, int total_tiles, int sub_rows,
                 float* __restrict__ part_m, float* __restrict__ part_l, const float* __restrict__ rowm,
                 const float* __restrict__ roww, float* __restrict__ s, int32_t* __restrict__ err) {
     extern __shared__ uint8_t smem_raw[];
@@ -249,16 +249,30 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 for (int nh = 0; nh < n_halves; ++nh)
                     for (int kb = 0; kb < 2; ++kb)
                         tma_load_3d(q_smem + (nh * 2 + kb) * kQRegionBytes, &tmQ, &bar.q_full, kb * 64, nh * 256, wk.u);
-                const int krow0 = (int)(ud.k_off / sh.row_stride) + wk.key_begin();
+                const int krow0 = sh.page_size ? 0 : (int)(ud.k_off / sh.row_stride);
+                const int key_begin = wk.key_begin();
                 const int nt = wk.seg_tiles();
                 for (int t = 0; t < nt && ok; ++t, ++kit) {
                     const int st = kit % kStages;
                     ok = mbar_wait(&bar.k_empty[st], ((kit / kStages) & 1u) ^ 1u, abort_flag);
                     if (!ok) break;
-                    mbar_expect_tx(&bar.k_full[st], kKStageBytes);
                     uint8_t* dst = k_smem + st * kKStageBytes;
-                    tma_load_2d(dst, &tmK, &bar.k_full[st], 0, krow0 + t * kTileKeys);
-                    tma_load_2d(dst + kKRegionBytes, &tmK, &bar.k_full[st], 64, krow0 + t * kTileKeys);
+                    const int key0 = key_begin + t * kTileKeys;
+                    if (sh.page_size == 0) {
+                        mbar_expect_tx(&bar.k_full[st], kKStageBytes);
+                        tma_load_2d(dst, &tmK, &bar.k_full[st], 0, krow0 + key0);
+                        tma_load_2d(dst + kKRegionBytes, &tmK, &bar.k_full[st], 64, krow0 + key0);
+                    } else {
+                        // one box of sub_rows rows per page piece; pieces past the end of the unit are not read
+                        // (their accumulator rows / columns are masked by the epilogue)
+                        const int n_sub = min(kTileKeys / sub_rows, (wk.T - key0 + sub_rows - 1) / sub_rows);
+                        mbar_expect_tx(&bar.k_full[st], (uint32_t)n_sub * sub_rows * 256u);
+                        for (int sb = 0; sb < n_sub; ++sb) {
+                            const int prow = (int)paged_row(sh, ud, key0 + sb * sub_rows);
+                            tma_load_2d(dst + sb * sub_rows * 128, &tmK, &bar.k_full[st], 0, prow);
+                            tma_load_2d(dst + kKRegionBytes + sb * sub_rows * 128, &tmK, &bar.k_full[st], 64, prow);
+                        }
+                    }
                 }
             }
             if (!ok) {
@@ -482,10 +496,20 @@ __global__ void score_tc_combine(const UnitDesc* __restrict__ desc, int rows, in
 // Entries of each normaliser-partial table the tensor-core path needs (one per unit + CTA).
 size_t score_tc_partial_slots(int n_units) { return 2 * ((size_t)n_units + kMaxSms); }
 
+// Rows per TMA box of the key stream: a whole 128-key tile for a contiguous cache, one page piece for
+// a paged one (0: the page size does not tile 128 rows).
+static int key_box_rows(const Shape& sh) {
+    if (sh.page_size == 0) return kTileKeys;
+    if (sh.page_size % kTileKeys == 0) return kTileKeys;
+    if (sh.page_size >= 8 && kTileKeys % sh.page_size == 0) return sh.page_size;
+    return 0;
+}
+
 bool score_tc_supported(const Launch& L) {
     const Shape& sh = L.sh;
     if (sh.dtype != CASK_DTYPE_BF16 || sh.d != kD) return false;
     if (sh.rows % 32 != 0 || sh.rows < 32 || sh.rows > 512) return false;
+    if (sh.page_size) return key_box_rows(sh) != 0 && sh.n_pages * sh.page_size < ((int64_t)1 << 31);
     int64_t max_row = 0;
     for (int u = 0; u < sh.n_units; ++u) {
         const UnitDesc& d = L.hdesc[u];
@@ -499,14 +523,15 @@ cudaError_t launch_score_tc(const Launch& L, const float* lse_in, float* s, floa
                             void* tmap_encode_fn) {
     const Shape& sh = L.sh;
     EncodeTiledFn encode = (EncodeTiledFn)tmap_encode_fn;
-    int64_t k_rows = 0;
-    for (int u = 0; u < sh.n_units; ++u)
+    int64_t k_rows = sh.page_size ? sh.n_pages * sh.page_size : 0;
+    for (int u = 0; u < sh.n_units && !sh.page_size; ++u)
         k_rows = std::max<int64_t>(k_rows, L.hdesc[u].k_off / sh.row_stride + L.hdesc[u].T);
+    const int sub_rows = key_box_rows(sh);
     CUtensorMap tmK, tmQ;
     {
         cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)k_rows};
         cuuint64_t strides[1] = {(cuuint64_t)sh.row_stride * 2};
-        cuuint32_t box[2] = {64, kTileKeys};
+        cuuint32_t box[2] = {64, (cuuint32_t)sub_rows};
         cuuint32_t estr[2] = {1, 1};
         if (encode(&tmK, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(L.k), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -535,7 +560,7 @@ cudaError_t launch_score_tc(const Launch& L, const float* lse_in, float* s, floa
     if (e != cudaSuccess) return e;
     if (!lse_in) {
         Timed t(L, KID_SCORE_NORM);
-        score_tc_kernel<0><<<grid, kThreadsTc, kSmemBytes, L.stream>>>(tmK, tmQ, L.desc, sh, L.total_tiles, ws.part_m,
+        score_tc_kernel<0><<<grid, kThreadsTc, kSmemBytes, L.stream>>>(tmK, tmQ, L.desc, sh, L.total_tiles, sub_rows, ws.part_m,
                                                                        ws.part_l, nullptr, nullptr, nullptr, ws.err);
     }
     {
@@ -545,7 +570,7 @@ cudaError_t launch_score_tc(const Launch& L, const float* lse_in, float* s, floa
     }
     {
         Timed t(L, KID_SCORE_MASS);
-        score_tc_kernel<1><<<grid, kThreadsTc, kSmemBytes, L.stream>>>(tmK, tmQ, L.desc, sh, L.total_tiles, nullptr,
+        score_tc_kernel<1><<<grid, kThreadsTc, kSmemBytes, L.stream>>>(tmK, tmQ, L.desc, sh, L.total_tiles, sub_rows, nullptr,
                                                                        nullptr, ws.rowm, ws.roww, s, ws.err);
     }
     return cudaGetLastError();

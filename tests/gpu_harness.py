@@ -34,7 +34,8 @@ def run_oracle(hb: wl.Batch, **kw) -> Dict:
 class GpuRun:
     """Device copies of a host batch plus everything needed to call the library on it."""
 
-    def __init__(self, hb: wl.Batch, device="cuda:0", row_stride=None, lse_in=None, **prm_kw):
+    def __init__(self, hb: wl.Batch, device="cuda:0", row_stride=None, lse_in=None, page_size=0, bad_page=None,
+                 **prm_kw):
         import torch
         from paper_2604_10900_b200 import binding as cb
         self.cb, self.torch, self.hb = cb, torch, hb
@@ -51,10 +52,34 @@ class GpuRun:
                 return p
             self.dev["k"], self.dev["v"] = pad(self.dev["k"]), pad(self.dev["v"])
             k_off = hb.tok_off[:-1] * row_stride
+        paged = {}
+        if page_size:
+            # Scatter the rows into a pool of shuffled pages (plus a few unused ones); the unused tail of a
+            # unit's last page and the spare pages hold a finite junk value that must never show up.
+            ps = int(page_size)
+            n_lp = [(int(t) + ps - 1) // ps for t in hb.T]
+            bt_off = np.concatenate([[0], np.cumsum(n_lp)]).astype(np.int64)
+            n_pages = int(bt_off[-1]) + 3
+            perm = np.random.default_rng(1234).permutation(n_pages).astype(np.int32)
+            table = perm[:int(bt_off[-1])].copy()
+            stride = d if row_stride is None else row_stride
+            src = np.concatenate([np.arange(int(hb.tok_off[u]), int(hb.tok_off[u]) + int(hb.T[u])) for u in range(hb.n_units)])
+            dst = np.concatenate([table[bt_off[u] + np.arange(int(hb.T[u])) // ps].astype(np.int64) * ps
+                                  + np.arange(int(hb.T[u])) % ps for u in range(hb.n_units)])
+            src_t, dst_t = torch.from_numpy(src).to(device), torch.from_numpy(dst).to(device)
+            for name in ("k", "v"):
+                pool = torch.full((n_pages * ps, stride), 768.0, dtype=torch.float32, device=device).to(self.dev[name].dtype)
+                pool[dst_t, :d] = self.dev[name][src_t, :d]
+                self.dev[name] = pool
+            if bad_page is not None:
+                table[bad_page] = n_pages + 5
+            self.block_table = torch.from_numpy(table).to(device)
+            paged = dict(page_size=ps, block_table=self.block_table, bt_off=bt_off, n_pages=n_pages)
+            k_off = None
         self.lse_in = None if lse_in is None else torch.from_numpy(np.ascontiguousarray(lse_in, np.float32)).to(device)
         self.batch, self._keep = cb.make_batch(
             self.dev["k"], self.dev["v"], self.dev["q"], hb.T, hb.P, hb.B, hb.reserve, hb.tok_off, d, w.group,
-            w.window, w.dtype, k_off=k_off, row_stride=row_stride, lse_in=self.lse_in)
+            w.window, w.dtype, k_off=k_off, row_stride=row_stride, lse_in=self.lse_in, **paged)
         self.prm = cb.params(**prm_kw)
         self.ctx = cb.Context(torch.device(device).index or 0, torch.cuda.current_stream(device).cuda_stream)
         self.ws, self.ws_bytes = cb.alloc_workspace(self.batch, self.prm, device)

@@ -280,7 +280,7 @@ def test_bad_arguments_are_refused_on_the_host_before_any_launch():
     assert rc(reserve=np.array([129, 0], np.int32)) == cb.ERR_SHAPE
     assert rc(d=60) == cb.ERR_SHAPE
     assert rc(row_stride=66) == cb.ERR_ALIGN
-    assert rc(page_size=16) == cb.ERR_UNSUPPORTED
+    assert rc(page_size=16) == cb.ERR_NULL            # a paged batch without its block table
     assert rc(ws_bytes=1024) == cb.ERR_WORKSPACE
     assert rc(prm=cb.params(gamma=1.5)) == cb.ERR_PARAM
     assert rc(prm=cb.params(eps=0.0)) == cb.ERR_PARAM
