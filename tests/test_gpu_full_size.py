@@ -1,0 +1,117 @@
+"""GPU parity at the benchmark's full sizes, in the launch configuration bench.py times.
+
+The whole workload runs in one call (all layers x KV heads of one sequence).  Every unit is checked
+against properties that hold at any size (budget met exactly, protected rows copied bit for bit,
+weights of every slot summing to one, selection counts equal to the plan, scores a distribution);
+a few units, chosen by a fixed rule, are compared element by element with the oracle.
+"""
+import numpy as np
+import pytest
+
+from paper_2604_10900_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+KIND_PREFIX, KIND_RECENT, KIND_CORE, KIND_SEED, KIND_MERGED = 1, 2, 3, 4, 5
+
+
+def _properties(hb, g):
+    w = hb.wl
+    kf = hb.k.view(np.uint16) if w.dtype == wl.DTYPE_BF16 else hb.k
+    vf = hb.v.view(np.uint16) if w.dtype == wl.DTYPE_BF16 else hb.v
+    from paper_2604_10900_b200 import workloads as W
+    for u in range(hb.n_units):
+        a, T, P, B = int(hb.tok_off[u]), int(hb.T[u]), int(hb.P[u]), int(hb.B[u])
+        sl = slice(a, a + T)
+        pl = g["plan"][u]
+        pkeep, bd, r, c, m, nout = int(pl[1]), int(pl[2]), int(pl[3]), int(pl[4]), int(pl[5]), int(pl[7])
+        n_out = int(g["n_out"][u])
+        assert n_out == nout == min(P, B - int(hb.reserve[u])) + min(T - P, B - min(P, B - int(hb.reserve[u])))
+        if T > B and T - P >= bd:
+            assert n_out == B                                    # the budget is met exactly
+        kind = g["kind"][sl]
+        assert (kind[:P] == KIND_PREFIX).sum() == pkeep and np.isin(kind[:P], (0, KIND_PREFIX)).all()
+        assert (kind[T - r:] == KIND_RECENT).all() and (kind == KIND_RECENT).sum() == r
+        assert (kind == KIND_CORE).sum() == c and (kind == KIND_SEED).sum() == m
+        s = g["s"][sl].astype(np.float64)
+        assert (s >= 0).all() and abs(s.sum() - 1.0) < 1e-4
+        # selections are by score: every core row outranks every seed, every seed every other scratch row
+        dec = np.arange(P, T - r)
+        if c and m:
+            assert s[dec][kind[dec] == KIND_CORE].min() >= s[dec][kind[dec] == KIND_SEED].max()
+        rest = np.isin(kind[dec], (0, KIND_MERGED))
+        if m and rest.any():
+            assert s[dec][kind[dec] == KIND_SEED].min() >= s[dec][rest].max()
+        asg, wgt = g["assign"][sl], g["weight"][sl].astype(np.float64)
+        kept = asg >= 0
+        assert (asg[kind == 0] == -1).all() and (wgt[kind == 0] == 0).all()
+        sums = np.bincount(asg[kept], weights=wgt[kept], minlength=n_out)
+        assert np.allclose(sums, 1.0, atol=1e-5)                 # convex combination per slot (Sec. 2.4)
+        counts = np.bincount(asg[kept], minlength=n_out)
+        src = g["slot_src"][u][:n_out]
+        assert (np.diff(src) > 0).all()                          # ascending anchor rows
+        assert np.array_equal(g["slot_kind"][u][:n_out], kind[src])
+        single = counts == 1
+        assert single[np.isin(kind[src], (KIND_PREFIX, KIND_RECENT, KIND_CORE))].all()   # core never merged
+        ko = g["k_out_bits"][u][:n_out]
+        vo = g["v_out_bits"][u][:n_out]
+        assert np.array_equal(ko[single], kf[a + src[single]]) and np.array_equal(vo[single], vf[a + src[single]])
+        merged = kind == KIND_MERGED
+        assert (g["seed_of"][sl][merged] >= P).all() and (kind[g["seed_of"][sl][merged]] == KIND_SEED).all()
+
+
+def _slice_units(g, hb, idx, hb_s):
+    """The GPU outputs of units `idx` of batch hb, laid out as the outputs of sub-batch hb_s."""
+    out = {}
+    rows = np.concatenate([np.arange(int(hb.tok_off[u]), int(hb.tok_off[u]) + int(hb.T[u])) for u in idx])
+    for k, v in g.items():
+        if k.endswith("_bits"):
+            continue
+        if v.ndim >= 1 and v.shape[0] == int(hb.tok_off[-1]):
+            out[k] = v[rows]
+        elif v.ndim >= 1 and v.shape[0] == hb.n_units:
+            out[k] = v[idx]
+        else:
+            out[k] = v
+    assert len(rows) == int(hb_s.tok_off[-1])
+    return out
+
+
+def _full(name, sample):
+    import torch
+    import gpu_harness as gh
+    w = wl.WORKLOADS[name]
+    hb = wl.make_batch(w, threads=16)
+    run = gh.GpuRun(hb)
+    g = run.event()
+    assert run.ctx.used_tensor_path and run.ctx.device_flags() == 0
+    for nm in ("k_out", "v_out"):
+        t = run.out[nm]
+        g[nm + "_bits"] = t.view(torch.uint16).cpu().numpy() if t.dtype == torch.bfloat16 else t.cpu().numpy()
+    _properties(hb, g)
+    units = [hb.unit_ids[u] for u in sample]
+    hb_s = wl.make_batch(w, units)
+    for j, u in enumerate(sample):                      # the generator is per unit: same bytes
+        a, b = int(hb.tok_off[u]), int(hb.tok_off[u + 1])
+        assert np.array_equal(hb_s.unit(j)[0], hb.k[a:b])
+    o = gh.run_oracle(hb_s)
+    st = gh.compare_event(hb_s, _slice_units(g, hb, sample, hb_s), o)
+    print(name, "sampled units", sample, st)
+    return st
+
+
+def test_reasoning32k_b512_full_size():
+    """36 layers x 8 KV heads, 33,280 rows per unit: the benchmark's default workload."""
+    st = _full("reasoning32k_b512", [0, 143, 287])
+    assert st["max_score_rel"] < 1e-5
+
+
+def test_reasoning8k_b384_full_size():
+    st = _full("reasoning8k_b384", [0, 55, 111])
+    assert st["max_score_rel"] < 1e-5
+
+
+def test_prompt_heavy_full_size():
+    """Prefix eviction to 1536 rows before decode consolidation, budget 2048, m = 224 seeds."""
+    st = _full("prompt_heavy", [3, 60, 108])
+    assert st["max_score_rel"] < 1e-5
