@@ -34,6 +34,16 @@ from paper_2604_10900_b200 import workloads as wl  # noqa: E402
 METRIC = "kv_tokens_compressed_per_s"
 UNIT = "tokens/s"
 
+# DRAM bytes per cache row (dram__bytes_read.sum + dram__bytes_write.sum of one launch / rows streamed) from the
+# ncu captures summarised under profiles/; traffic grows in proportion to the rows a launch streams.
+NCU_TRAFFIC = {
+    "score_norm": (268.2, "profiles/score_tc_reasoning32k_16units.txt"),
+    "score_mass": (271.1, "profiles/score_tc_reasoning32k_16units.txt"),
+    "assign": (264.3, "profiles/assign_tc_reasoning32k_16units.txt"),
+}
+# ex2 units: 16 results per clock per SM (special-function pipe), 148 SMs, 1.965 GHz maximum SM clock.
+EX2_PEAK_T_PER_S = 148 * 16 * 1.965e9 / 1e12
+
 
 def _peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -135,8 +145,11 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device(device))
     w = wl.WORKLOADS[args.workload]
+    # A batch of many sequences does not fit one GPU with all its layers (64 sequences x 36 layers x 8 heads of
+    # the serving sweep hold 179 GB of K/V): it runs on a slice of the layers, every sequence present.
+    n_layers = w.layers if w.n_seqs == 1 else min(w.layers, args.layer_slice or 6)
     units = wl.unit_list(w, seqs=range(rank, rank + 1)) if w.n_seqs == 1 else \
-        wl.shard_units(wl.unit_list(w), rank, world)
+        wl.shard_units(wl.unit_list(w, layers=range(n_layers)), rank, world)
     if args.max_units:
         units = units[:args.max_units]
 
@@ -257,30 +270,34 @@ def run_ours(args):
         return
 
     # ---- roofline of the dominant kernel -------------------------------------------------------
+    ctx_tensor_path = ctx.used_tensor_path
     peaks = _peaks()
     per_kernel = {k: dict(ms_per_launch=v["ms"] / v["launches"], launches_per_step=v["launches"] / args.steps,
                           share=v["ms"] / max(sum(x["ms"] for x in prof.values()), 1e-9)) for k, v in prof.items()}
     top = max(prof, key=lambda k: prof[k]["ms"])
     top_ms = prof[top]["ms"] / prof[top]["launches"]
     flops_pass = 2.0 * rows * float(sum_T) * d        # one Q_w K^T contraction over every unit
-    if top in ("score_norm", "score_mass", "score_norm_tc", "score_mass_tc"):
-        achieved = flops_pass / (top_ms * 1e-3) / 1e12
-        roof = dict(kernel=top, bound="tensor", achieved=achieved, peak=peaks["bf16_tflops_sustained"],
-                    unit="TFLOP/s", frac=achieved / peaks["bf16_tflops_sustained"], traffic=None,
-                    peak_source=peaks["source"] + " (sustained cuBLAS bf16)", ms_per_launch=top_ms,
-                    flops_per_launch=flops_pass)
+    tensor_roof = None
+    if top in ("score_norm", "score_mass"):
+        # One exponential per (query row, key): the pass is bound by the ex2 pipe, not by the contraction that
+        # feeds it (profiles/score_tc_*: ex2 pipe 65-72 % busy, tensor pipe 37-40 %, DRAM 17 %).
+        exps = float(rows) * float(sum_T)
+        achieved = exps / (top_ms * 1e-3) / 1e12
+        roof = dict(kernel=top, bound="alu", achieved=achieved, peak=EX2_PEAK_T_PER_S, unit="Texp/s",
+                    frac=achieved / EX2_PEAK_T_PER_S, traffic=None,
+                    peak_source="148 SMs x 16 ex2/clk x 1.965 GHz", ms_per_launch=top_ms, exps_per_launch=exps)
+        t_ach = flops_pass / (top_ms * 1e-3) / 1e12
+        tensor_roof = dict(kernel=top, bound="tensor", achieved=t_ach, peak=peaks["bf16_tflops_sustained"],
+                           unit="TFLOP/s", frac=t_ach / peaks["bf16_tflops_sustained"],
+                           peak_source=peaks["source"] + " (sustained cuBLAS bf16)", flops_per_launch=flops_pass)
     else:
         byts = algorithmic_bytes(hb, n_out, kind)
         achieved = byts / (top_ms * 1e-3) / 1e9
         roof = dict(kernel=top, bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
                     frac=achieved / peaks["hbm_gbs"], traffic=None, peak_source=peaks["source"], ms_per_launch=top_ms)
-    traffic_file = os.path.join(ROOT, "profiles", "dram_traffic.json")
-    if os.path.exists(traffic_file):
-        tr = json.load(open(traffic_file))
-        ent = tr.get(top)
-        if ent:
-            roof["traffic"] = ent["bytes_per_unit_token"] * float(sum_T)
-            roof["traffic_source"] = ent.get("source")
+    if top in NCU_TRAFFIC and ctx_tensor_path:
+        roof["traffic"] = NCU_TRAFFIC[top][0] * float(sum_T)
+        roof["traffic_source"] = NCU_TRAFFIC[top][1] + " (bytes per cache row x rows of this launch)"
     ev_bytes = algorithmic_bytes(hb, n_out, kind)
     t_hbm = ev_bytes / (peaks["hbm_gbs"] * 1e9)
     n_pass = 2          # normaliser pass + score pass (no caller-supplied normalisers here)
@@ -305,8 +322,12 @@ def run_ours(args):
                    "l2": "inputs larger than L2: %.2f GB of K/V read per step" % ((hb.k.nbytes + hb.v.nbytes) / 1e9),
                    "score_path": "tcgen05" if ctx.used_tensor_path else "simt", "gen_seconds": round(t_gen, 1),
                    "reduced": bool(args.max_units),
+                   **({"sequences": w.n_seqs, "layers_per_pass": n_layers, "layers": w.layers,
+                       "events_per_s": w.n_seqs * n_layers / w.layers / (ms_step * 1e-3),
+                       "events_per_s_note": "one event = all layers of one sequence; this pass held layers_per_pass of them"}
+                      if w.n_seqs > 1 else {}),
                    "status_bits_seen": int(np.bitwise_or.reduce(status))},
-        "roofline": roof, "event_roofline": event, "kernels": per_kernel,
+        "roofline": roof, "tensor_roofline": tensor_roof, "event_roofline": event, "kernels": per_kernel,
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                 "ms_per_step": e2e_ms, "steps": e2e_steps},
@@ -381,6 +402,8 @@ def main():
     ap.add_argument("--cpu-units", type=int, default=32, help="units in the oracle's bounded sample")
     ap.add_argument("--max-units", type=int, default=0, help="debug: cut the workload to this many units")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layer-slice", type=int, default=0,
+                    help="layers per pass for multi-sequence workloads (default 6)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
