@@ -51,7 +51,11 @@ constexpr int kMaxSms = 1024;                          // upper bound used when 
 
 // Columns (of every 32) whose exponential runs on the FMA pipe.
 constexpr uint32_t kPolyMaskN = 0x80808080u;
-constexpr uint32_t kPolyMaskS = 0x80808080u;
+constexpr uint32_t kPolyPairsS = 0x8080u;      // pairs of columns (of the 16 in a block of 32) on the FMA pipe
+#ifndef CASK_POLY_PAIRS16
+#define CASK_POLY_PAIRS16 0x80u
+#endif
+constexpr uint32_t kPolyPairs16 = CASK_POLY_PAIRS16;   // the same for the 8 pairs of a 16-column chunk
 
 struct __align__(8) Barriers {
     uint64_t q_full, q_empty;
@@ -65,7 +69,7 @@ struct TcSmemTail {
     Barriers bar;
     uint32_t tmem_base;
     int abort;
-    alignas(16) float rc[2][512];  // pass S: rowm - log2(roww) per query row, double-buffered by segment
+    alignas(16) float rc[2][512];  // pass S: log2(roww) - rowm per query row, double-buffered by segment
     float red[8][4][128];         // pass S: partial key sums per (group, column half), eight tiles deep
 };
 
@@ -85,29 +89,54 @@ __device__ __forceinline__ float ex2_poly(float t) {
     return __int_as_float(__float_as_int(p) + (__float_as_int(fl) << 23));
 }
 
+// 2^t for a pair of t in [-125, 125] on the FMA pipe (packed arithmetic).
+__device__ __forceinline__ uint64_t ex2_poly2(uint64_t t2) {
+    const uint64_t magic = pack2(12582912.f, 12582912.f);
+    const uint64_t fl = add2(t2, magic);
+    const uint64_t f = sub2(t2, sub2(fl, magic));
+    uint64_t p = pack2(1.327644451521337e-3f, 1.327644451521337e-3f);
+    p = fma2(p, f, pack2(9.67553723603487e-3f, 9.67553723603487e-3f));
+    p = fma2(p, f, pack2(5.550713464617729e-2f, 5.550713464617729e-2f));
+    p = fma2(p, f, pack2(2.4022120237350464e-1f, 2.4022120237350464e-1f));
+    p = fma2(p, f, pack2(6.931469440460205e-1f, 6.931469440460205e-1f));
+    p = fma2(p, f, pack2(1.0000001192092896f, 1.0000001192092896f));
+    float p0, p1, n0, n1;
+    unpack2(p, p0, p1);
+    unpack2(fl, n0, n1);
+    return pack2(__int_as_float(__float_as_int(p0) + (__float_as_int(n0) << 23)),
+                 __int_as_float(__float_as_int(p1) + (__float_as_int(n1) << 23)));
+}
+
 // Pass S, one block of 32 query columns (rows r0..r0+31 of the window) for the key this thread owns:
-// adds sum_r 2^(y_r*scale2 - rc[r]) over the visible rows to the four partial sums.
-__device__ __forceinline__ void mass_block(const float (&v)[32], const float* rc, int r0, bool fast, int causal, int W,
-                                           int jmin, float scale2, float& a0, float& a1, float& a2, float& a3) {
+// adds sum_r 2^(y_r*scale2 + nc[r]) over the visible rows to the two packed pairs of partial sums.
+// Pairs of columns go through packed fp32 instructions; the pairs named by kPolyPairsS take the polynomial.
+__device__ __forceinline__ void mass_block(const float (&v)[32], const float* nc, int r0, bool fast, int causal, int W,
+                                           int jmin, float scale2, uint64_t& a01, uint64_t& a23) {
     if (fast) {
-        const float4* rc4 = reinterpret_cast<const float4*>(&rc[r0]);
+        const float4* nc4 = reinterpret_cast<const float4*>(&nc[r0]);
+        const uint64_t s2 = pack2(scale2, scale2);
 #pragma unroll
         for (int x = 0; x < 8; ++x) {
-            const float4 c4 = rc4[x];
-            const float t0 = fmaf(v[4 * x], scale2, -c4.x), t1 = fmaf(v[4 * x + 1], scale2, -c4.y);
-            const float t2 = fmaf(v[4 * x + 2], scale2, -c4.z), t3 = fmaf(v[4 * x + 3], scale2, -c4.w);
-            a0 += ((kPolyMaskS >> (4 * x)) & 1u) ? ex2_poly(fmaxf(t0, -125.f)) : ex2(t0);
-            a1 += ((kPolyMaskS >> (4 * x + 1)) & 1u) ? ex2_poly(fmaxf(t1, -125.f)) : ex2(t1);
-            a2 += ((kPolyMaskS >> (4 * x + 2)) & 1u) ? ex2_poly(fmaxf(t2, -125.f)) : ex2(t2);
-            a3 += ((kPolyMaskS >> (4 * x + 3)) & 1u) ? ex2_poly(fmaxf(t3, -125.f)) : ex2(t3);
+            const float4 c4 = nc4[x];
+            const uint64_t tA = fma2(pack2(v[4 * x], v[4 * x + 1]), s2, pack2(c4.x, c4.y));
+            const uint64_t tB = fma2(pack2(v[4 * x + 2], v[4 * x + 3]), s2, pack2(c4.z, c4.w));
+            float t0, t1, t2, t3;
+            unpack2(tA, t0, t1);
+            unpack2(tB, t2, t3);
+            if ((kPolyPairsS >> (2 * x)) & 1u) a01 = add2(a01, ex2_poly2(pack2(fmaxf(t0, -125.f), fmaxf(t1, -125.f))));
+            else a01 = add2(a01, pack2(ex2(t0), ex2(t1)));
+            if ((kPolyPairsS >> (2 * x + 1)) & 1u) a23 = add2(a23, ex2_poly2(pack2(fmaxf(t2, -125.f), fmaxf(t3, -125.f))));
+            else a23 = add2(a23, pack2(ex2(t2), ex2(t3)));
         }
     } else {
+        float a = 0.f;
 #pragma unroll
         for (int x = 0; x < 32; ++x) {
             const int r = r0 + x;
             const bool vis = !causal || (r % W) >= jmin;
-            if (vis) a0 += ex2(fmaf(v[x], scale2, -rc[r]));
+            if (vis) a += ex2(fmaf(v[x], scale2, nc[r]));
         }
+        a01 = add2(a01, pack2(a, 0.f));
     }
 }
 
@@ -348,10 +377,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             const float* rc = tail->rc[seg & 1u];
             if (PASS == 1) {
                 // Every thread has passed the rw_ready phase of the previous segment, so nobody still
-                // reads the buffer used two segments ago.  roww * 2^(y - rowm) = 2^(y - (rowm - log2 roww)).
+                // reads the buffer used two segments ago.  roww * 2^(y - rowm) = 2^(y + (log2 roww - rowm)).
                 float* dst = tail->rc[seg & 1u];
-                dst[etid] = (etid < rows) ? rowm[(size_t)wk.u * rows + etid] - log2f(roww[(size_t)wk.u * rows + etid])
-                                          : 1.0e30f;
+                dst[etid] = (etid < rows) ? log2f(roww[(size_t)wk.u * rows + etid]) - rowm[(size_t)wk.u * rows + etid]
+                                          : -1.0e30f;
                 mbar_arrive(&bar.rw_ready);
                 ok = mbar_wait(&bar.rw_ready, seg & 1u, abort_flag);
                 if (!ok) break;
@@ -365,6 +394,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             const int j0 = g, j1 = g + 2;
             const int cend0 = PASS == 1 ? min(64 * ch + 64, rows - 128 * j0) - 64 * ch : 64;
             const int cend1 = PASS == 1 ? min(64 * ch + 64, rows - 128 * j1) - 64 * ch : 64;
+            const bool full_cols = j1 < n_slots && cend0 == 64 && cend1 == 64;
             const int row0 = 128 * j0 + 32 * qd + lane, row1 = 128 * j1 + 32 * qd + lane;      // pass N
             const int lastvis0 = (row0 < rows) ? (sh.causal ? T - sh.W + (row0 % sh.W) : T - 1) : -1;
             const int lastvis1 = (row1 < rows) ? (sh.causal ? T - sh.W + (row1 % sh.W) : T - 1) : -1;
@@ -374,27 +404,130 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 const int my_key = key0 + 32 * qd + lane;           // pass S: the key this thread owns
                 const int jmin = my_key - (T - sh.W);               // pass S: first window position that sees it
                 const int kcol = key0 + 64 * ch;                    // pass N: first key column of this warp
-                float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll
-                for (int p = 0; p < 2; ++p) {
-                    const int j = p ? j1 : j0;
-                    if (j >= n_slots || !ok) break;
-                    ok = mbar_wait(&bar.d_full[j], kit & 1u, abort_flag);
+                uint64_t a01 = 0ull, a23 = 0ull;      // pass S: two packed pairs of partial key sums
+                if (fast && full_cols) {
+                    // Streamed form of the common tile: eight chunks of 16 columns.  The arguments of a chunk's
+                    // exponentials are formed first; that frees the accumulator registers, so the next chunk's
+                    // TMEM load (or the slot's release) is issued before the exponentials and its latency hides
+                    // behind them.
+                    const uint64_t s2 = pack2(scale2, scale2);
+                    float v[16];
+                    ok = mbar_wait(&bar.d_full[j0], kit & 1u, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    const int cend = p ? cend1 : cend0;
-                    for (int cc = 0; cc < cend; cc += 32) {
-                        float v[32];
-                        tc_ld32(taddr + 128 * j + cc, v);
-                        tc_wait_ld_regs(v);
-                        if (PASS == 1) mass_block(v, rc, 128 * j + 64 * ch + cc, fast, sh.causal, sh.W, jmin, scale2, a0, a1, a2, a3);
-                        else norm_block(v, fast, (p ? lastvis1 : lastvis0) - (kcol + cc) + 1, scale2, mm[p], l_run[p]);
+                    tc_ld16(taddr + 128 * j0, v);
+                    tc_wait_ld_regs(v);
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const int p = c >> 2, j = p ? j1 : j0, col = 16 * (c & 3);
+                        uint64_t t2[8];
+                        if (PASS == 1) {
+                            const float4* nc4 = reinterpret_cast<const float4*>(&rc[128 * j + 64 * ch + col]);
+#pragma unroll
+                            for (int x = 0; x < 4; ++x) {
+                                const float4 c4 = nc4[x];
+                                t2[2 * x] = fma2(pack2(v[4 * x], v[4 * x + 1]), s2, pack2(c4.x, c4.y));
+                                t2[2 * x + 1] = fma2(pack2(v[4 * x + 2], v[4 * x + 3]), s2, pack2(c4.z, c4.w));
+                            }
+                        } else {
+                            const uint64_t nm2 = pack2(-mm[p], -mm[p]);
+#pragma unroll
+                            for (int x = 0; x < 8; ++x) t2[x] = fma2(pack2(v[2 * x], v[2 * x + 1]), s2, nm2);
+                        }
+                        if (PASS == 1 && (c == 3 || c == 7)) {           // the slot's last columns are in registers
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&bar.d_empty[j]);
+                        }
+                        if (c == 3) {
+                            ok = mbar_wait(&bar.d_full[j1], kit & 1u, abort_flag);
+                            if (!ok) break;
+                            tc_fence_after();
+                        }
+                        if (c < 7) tc_ld16(taddr + 128 * (((c + 1) >> 2) ? j1 : j0) + 16 * ((c + 1) & 3), v);
+                        if (PASS == 1) {
+#pragma unroll
+                            for (int x = 0; x < 8; ++x) {
+                                float t0, t1;
+                                unpack2(t2[x], t0, t1);
+                                const uint64_t e2 = ((kPolyPairs16 >> x) & 1u)
+                                                        ? ex2_poly2(pack2(fmaxf(t0, -125.f), fmaxf(t1, -125.f)))
+                                                        : pack2(ex2(t0), ex2(t1));
+                                if (x & 1) a23 = add2(a23, e2); else a01 = add2(a01, e2);
+                            }
+                        } else {
+                            uint64_t b01 = 0ull, b23 = 0ull;
+#pragma unroll
+                            for (int x = 0; x < 8; ++x) {
+                                float t0, t1;
+                                unpack2(t2[x], t0, t1);
+                                const uint64_t e2 = ((kPolyPairs16 >> x) & 1u)
+                                                        ? ex2_poly2(pack2(fminf(fmaxf(t0, -125.f), 125.f), fminf(fmaxf(t1, -125.f), 125.f)))
+                                                        : pack2(ex2(t0), ex2(t1));
+                                if (x & 1) b23 = add2(b23, e2); else b01 = add2(b01, e2);
+                            }
+                            float b0, b1;
+                            unpack2(add2(b01, b23), b0, b1);
+                            float lb = b0 + b1;
+                            const bool redo = !(lb <= 65536.f);
+                            if (__any_sync(0xffffffffu, redo)) {
+                                // Some row of the warp has a column that exceeds its reference by more than 16
+                                // (or its reference is still unset).  The whole warp reads the chunk again (the
+                                // load is warp-wide; the slot is still held); the rows concerned move their
+                                // reference to the chunk maximum and redo the chunk.
+                                float w[16];
+                                tc_ld16(taddr + 128 * j + col, w);
+                                tc_wait_ld_regs(w);
+                                if (redo) {
+                                    float cm = w[0];
+#pragma unroll
+                                    for (int x = 1; x < 16; ++x) cm = fmaxf(cm, w[x]);
+                                    cm *= scale2;
+                                    if (cm > mm[p]) {
+                                        l_run[p] *= ex2(mm[p] - cm);
+                                        mm[p] = cm;
+                                    }
+                                    lb = 0.f;
+#pragma unroll
+                                    for (int x = 0; x < 16; ++x) lb += ex2(fmaf(w[x], scale2, -mm[p]));
+                                }
+                                __syncwarp();
+                            }
+                            l_run[p] += lb;
+                            if (c == 3 || c == 7) {           // the slot is no longer needed
+                                tc_fence_before();
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(&bar.d_empty[j]);
+                            }
+                        }
+                        if (c < 7) tc_wait_ld_regs(v);
                     }
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&bar.d_empty[j]);
+                    if (!ok) break;
+                } else {
+#pragma unroll
+                    for (int p = 0; p < 2; ++p) {
+                        const int j = p ? j1 : j0;
+                        if (j >= n_slots || !ok) break;
+                        ok = mbar_wait(&bar.d_full[j], kit & 1u, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const int cend = p ? cend1 : cend0;
+                        for (int cc = 0; cc < cend; cc += 32) {
+                            float v[32];
+                            tc_ld32(taddr + 128 * j + cc, v);
+                            tc_wait_ld_regs(v);
+                            if (PASS == 1) mass_block(v, rc, 128 * j + 64 * ch + cc, fast, sh.causal, sh.W, jmin, scale2, a01, a23);
+                            else norm_block(v, fast, (p ? lastvis1 : lastvis0) - (kcol + cc) + 1, scale2, mm[p], l_run[p]);
+                        }
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&bar.d_empty[j]);
+                    }
                 }
                 if (PASS == 1 && ok) {
+                    float a0, a1, a2, a3;
+                    unpack2(a01, a0, a1);
+                    unpack2(a23, a2, a3);
                     tail->red[kit & 7u][ew >> 2][32 * qd + lane] = (a0 + a1) + (a2 + a3);
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bar.red_full[kit & 7u]);
