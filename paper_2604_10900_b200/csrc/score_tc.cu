@@ -52,10 +52,9 @@ constexpr int kMaxSms = 1024;                          // upper bound used when 
 // Columns (of every 32) whose exponential runs on the FMA pipe.
 constexpr uint32_t kPolyMaskN = 0x80808080u;
 constexpr uint32_t kPolyPairsS = 0x8080u;      // pairs of columns (of the 16 in a block of 32) on the FMA pipe
-#ifndef CASK_POLY_PAIRS16
-#define CASK_POLY_PAIRS16 0x80u
-#endif
-constexpr uint32_t kPolyPairs16 = CASK_POLY_PAIRS16;   // the same for the 8 pairs of a 16-column chunk
+// the same for the 8 pairs of a 16-column chunk of the streamed path (normaliser pass / score pass)
+constexpr uint32_t kPolyPairs16N = 0x88u;
+constexpr uint32_t kPolyPairs16S = 0x80u;
 
 struct __align__(8) Barriers {
     uint64_t q_full, q_empty;
@@ -450,7 +449,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                             for (int x = 0; x < 8; ++x) {
                                 float t0, t1;
                                 unpack2(t2[x], t0, t1);
-                                const uint64_t e2 = ((kPolyPairs16 >> x) & 1u)
+                                const uint64_t e2 = ((kPolyPairs16S >> x) & 1u)
                                                         ? ex2_poly2(pack2(fmaxf(t0, -125.f), fmaxf(t1, -125.f)))
                                                         : pack2(ex2(t0), ex2(t1));
                                 if (x & 1) a23 = add2(a23, e2); else a01 = add2(a01, e2);
@@ -461,7 +460,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                             for (int x = 0; x < 8; ++x) {
                                 float t0, t1;
                                 unpack2(t2[x], t0, t1);
-                                const uint64_t e2 = ((kPolyPairs16 >> x) & 1u)
+                                const uint64_t e2 = ((kPolyPairs16N >> x) & 1u)
                                                         ? ex2_poly2(pack2(fminf(fmaxf(t0, -125.f), 125.f), fminf(fmaxf(t1, -125.f), 125.f)))
                                                         : pack2(ex2(t0), ex2(t1));
                                 if (x & 1) b23 = add2(b23, e2); else b01 = add2(b01, e2);
