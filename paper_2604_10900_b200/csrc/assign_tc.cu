@@ -10,7 +10,9 @@
 //               tiles e, e+G, e+2G, ... of the CTA and owns one accumulator buffer, so up to G
 //               tiles are in flight and the global-memory round trips of a tile (row kind, score,
 //               the fixed-point mass atomics) overlap with the next tiles
-// G = 4 buffers of 128 TMEM columns when every unit has m <= 128 seeds, else 2 buffers of 256.
+// With m <= 128 seeds in every unit the TMEM holds four buffers of 128 columns, one per group.  With more
+// seeds it holds two buffers of 256 columns and two groups share each: one takes the seed columns
+// the first columns and finishes the row, the other takes the rest and hands its best seed over through shared memory.
 #include "tc_common.cuh"
 
 namespace cask {
@@ -34,6 +36,7 @@ struct __align__(8) ABarriers {
     uint64_t k_full[kStages], k_empty[kStages];
     uint64_t d_full[kMaxGroups], d_empty[kMaxGroups];
     uint64_t nu_ready;
+    uint64_t x_full[2];      // shared buffers: the second group's best seed of a tile is in shared memory
 };
 
 struct ASmemTail {
@@ -41,6 +44,8 @@ struct ASmemTail {
     uint32_t tmem_base;
     int abort;
     float inv_nu[2][256];     // 1/|k_seed| (0 for a zero seed), double-buffered by unit
+    float x_val[2][2][128];   // shared buffers: best dot product / seed norm and its seed,
+    int x_idx[2][2][128];     //   per buffer, per use parity, per tile row
 };
 
 constexpr size_t kSmemBytesA = 1024 + kSeedBytes + kStages * kKStageBytes + sizeof(ASmemTail);
@@ -75,9 +80,42 @@ struct TileWalk {
     }
 };
 
+// Best seed among the accumulator columns [c_lo, c_hi) of this thread's row: the greatest dot * 1/|k_seed|, the
+// first column among equals.  A block of 32 columns costs a multiply and a maximum per column; the position of
+// the maximum is looked for only in a block that beats everything before it.
+__device__ __forceinline__ void best_seed(uint32_t taddr, const float* inv, int c_lo, int c_hi, float& best, int& best_u) {
+    for (int cc = c_lo; cc < c_hi; cc += 32) {
+        float v[32];
+        tc_ld32(taddr + cc, v);
+        tc_wait_ld_regs(v);
+        float bm = -INFINITY;
+        if (cc + 32 <= c_hi) {
+#pragma unroll
+            for (int x = 0; x < 32; ++x) {
+                v[x] *= inv[cc + x];
+                bm = fmaxf(bm, v[x]);
+            }
+        } else {
+#pragma unroll
+            for (int x = 0; x < 32; ++x) {
+                v[x] = (cc + x < c_hi) ? v[x] * inv[cc + x] : -INFINITY;
+                bm = fmaxf(bm, v[x]);
+            }
+        }
+        if (bm > best) {
+            best = bm;
+            int at = 31;
+#pragma unroll
+            for (int x = 30; x >= 0; --x)
+                if (v[x] == bm) at = x;
+            best_u = cc + at;
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kThreadsA, 1)
 assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmSeed,
-                 const UnitDesc* __restrict__ desc, Shape sh, int total_tiles, int n_groups, int sub_rows,
+                 const UnitDesc* __restrict__ desc, Shape sh, int total_tiles, int n_bufs, int sub_rows,
                  const float* __restrict__ s, const int32_t* __restrict__ plan,
                  const int32_t* __restrict__ seed_rows, const float* __restrict__ seed_norm,
                  uint8_t* __restrict__ kind, int32_t* __restrict__ seed_of, float* __restrict__ sim,
@@ -91,14 +129,17 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     ABarriers& bar = tail->bar;
     volatile int* abort_flag = &tail->abort;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int buf_cols = 512 / n_groups;                 // TMEM columns per accumulator buffer
+    const int buf_cols = 512 / n_bufs;                   // TMEM columns per accumulator buffer
+    const int split = kMaxGroups / n_bufs;               // groups sharing one buffer (1 or 2)
 
     if (threadIdx.x == 0) {
         mbar_init(&bar.b_full, 1);
         mbar_init(&bar.b_empty, 1);
         for (int i = 0; i < kStages; ++i) { mbar_init(&bar.k_full[i], 1); mbar_init(&bar.k_empty[i], 1 + 4); }
-        for (int i = 0; i < kMaxGroups; ++i) { mbar_init(&bar.d_full[i], 1); mbar_init(&bar.d_empty[i], 4); }
-        mbar_init(&bar.nu_ready, 128 * n_groups);
+        for (int i = 0; i < kMaxGroups; ++i) { mbar_init(&bar.d_full[i], 1); mbar_init(&bar.d_empty[i], 4 * split); }
+        mbar_init(&bar.nu_ready, 128 * kMaxGroups);
+        mbar_init(&bar.x_full[0], 4);
+        mbar_init(&bar.x_full[1], 4);
         tail->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -175,7 +216,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 const int nt = wk.run();
                 for (int t = 0; t < nt && ok; ++t, ++kit) {
                     const int st = kit % kStages;
-                    const uint32_t buf = kit % (uint32_t)n_groups, use = kit / (uint32_t)n_groups;
+                    const uint32_t buf = kit % (uint32_t)n_bufs, use = kit / (uint32_t)n_bufs;
                     ok = mbar_wait(&bar.k_full[st], (kit / kStages) & 1u, abort_flag);
                     if (!ok) break;
                     ok = mbar_wait(&bar.d_empty[buf], (use & 1u) ^ 1u, abort_flag);
@@ -197,11 +238,12 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 if (ok) tc_commit(&bar.b_empty);
             }
         }
-    } else if (warp >= kEpiWarp0 && ((warp - kEpiWarp0) >> 2) < n_groups) {
+    } else if (warp >= kEpiWarp0) {
         // ================= epilogue =================
         const int ew = warp - kEpiWarp0;
         const int qd = ew & 3;                               // TMEM lane quadrant (== warp % 4)
-        const uint32_t eg = (uint32_t)(ew >> 2);             // group: tiles eg, eg + G, ... and buffer eg
+        const uint32_t eg = (uint32_t)(ew >> 2) % (uint32_t)n_bufs;   // buffer: tiles eg, eg + n_bufs, ...
+        const int half = (ew >> 2) / n_bufs;                 // 0: finishes the row; 1: the later seed columns only
         const int etid = ew * 32 + lane;
         const uint32_t taddr = tmem_base + ((uint32_t)(32 * qd) << 16) + eg * buf_cols;
         const int my_row = 32 * qd + lane;                   // row of the tile this thread owns
@@ -217,6 +259,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const int m = max(0, min(plan[u * 8 + CASK_PLAN_M], ud.plan[CASK_PLAN_M]));
             const int hi = T - r;
             const int a0 = P - (sh.page_size ? P % sub_rows : 0);
+            // shared buffers: the finishing group also computes the row norm, so it takes fewer seed columns
+            const int c_split = split == 2 ? min(m, 32 * max(1, (((m + 31) >> 5) - 2) / 2)) : m;
             unsigned long long* mass_u = mass_fx + (size_t)u * (max_m + 1);
             float* inv = tail->inv_nu[ucount & 1u];
             if (etid < 256) {
@@ -230,9 +274,27 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const int tile0 = wk.tile_in_unit();
             const int nt = wk.run();
             for (int t = 0; t < nt && ok; ++t, ++kit) {
-                if (kit % (uint32_t)n_groups != eg) continue;
+                if (kit % (uint32_t)n_bufs != eg) continue;
                 const int st = kit % kStages;
-                const uint32_t use = kit / (uint32_t)n_groups;
+                const uint32_t use = kit / (uint32_t)n_bufs;
+                if (half == 1) {
+                    // second group of a shared buffer: best seed among the columns [c_split, m)
+                    ok = mbar_wait(&bar.d_full[eg], use & 1u, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    float best = -INFINITY;
+                    int best_u = -1;
+                    best_seed(taddr, inv, c_split, m, best, best_u);
+                    tc_fence_before();
+                    tail->x_val[eg][use & 1u][my_row] = best;
+                    tail->x_idx[eg][use & 1u][my_row] = best_u;
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive(&bar.d_empty[eg]);
+                        mbar_arrive(&bar.x_full[eg]);
+                    }
+                    continue;
+                }
                 // the row's kind and score are fetched now and used after the contraction
                 const int i = a0 + (tile0 + t) * kTileRows + my_row;
                 const bool in_range = i >= P && i < hi;
@@ -242,7 +304,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 // sixteen 16-byte pieces of the row gives the same set of elements)
                 ok = mbar_wait(&bar.k_full[st], (kit / kStages) & 1u, abort_flag);
                 if (!ok) break;
-                float n2 = 0.f;
+                uint64_t n2p = 0ull;
                 {
                     const uint8_t* base = k_smem + st * kKStageBytes + my_row * 128;
 #pragma unroll
@@ -250,42 +312,48 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll
                         for (int c = 0; c < 8; ++c) {
                             const uint4 raw = *reinterpret_cast<const uint4*>(base + kb * kKRegionBytes + (((c + lane) & 7) << 4));
-                            const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+                            // a bf16 is the upper half of an fp32: two integer operations unpack a pair
+                            const uint32_t wv[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
                             for (int x = 0; x < 4; ++x) {
-                                const float2 f = __bfloat1622float2(h2[x]);
-                                n2 = fmaf(f.x, f.x, n2);
-                                n2 = fmaf(f.y, f.y, n2);
+                                const uint64_t f2 = pack2(__uint_as_float(wv[x] << 16), __uint_as_float(wv[x] & 0xFFFF0000u));
+                                n2p = fma2(f2, f2, n2p);
                             }
                         }
                 }
+                float n2, n2b;
+                unpack2(n2p, n2, n2b);
+                n2 += n2b;
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bar.k_empty[st]);
                 ok = mbar_wait(&bar.d_full[eg], use & 1u, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                float best = -INFINITY, best_dot = 0.f;
+                float best = -INFINITY;
                 int best_u = -1;
-                for (int cc = 0; cc < m; cc += 32) {
-                    float v[32];
-                    tc_ld32(taddr + cc, v);
-                    tc_wait_ld_regs(v);
-#pragma unroll
-                    for (int x = 0; x < 32; ++x) {
-                        const float val = v[x] * inv[cc + x];
-                        if (cc + x < m && val > best) { best = val; best_dot = v[x]; best_u = cc + x; }
+                best_seed(taddr, inv, 0, c_split, best, best_u);
+                tc_fence_before();
+                if (split == 2) {
+                    // The other group's candidate has the larger seed indices, so it wins only when strictly
+                    // better: the same outcome as one scan over all columns.  The buffer is released after this
+                    // read, so the other group cannot start the buffer's next use (and overwrite its hand-over
+                    // slot or run a barrier phase ahead) before it.
+                    ok = mbar_wait(&bar.x_full[eg], use & 1u, abort_flag);
+                    if (!ok) break;
+                    const float ov = tail->x_val[eg][use & 1u][my_row];
+                    if (ov > best) {
+                        best = ov;
+                        best_u = tail->x_idx[eg][use & 1u][my_row];
                     }
                 }
-                tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bar.d_empty[eg]);
 
                 const bool cand = in_range && best_u >= 0 && kd == CASK_KIND_DROPPED;
                 float sm_ = 0.f;
                 if (cand) {
-                    const float nj = sqrtf(n2);
-                    const float nu = seed_norm[seed_base + best_u];
-                    sm_ = (nj > 0.f && nu > 0.f) ? best_dot / (nj * nu) : 0.f;
+                    const float nj = sqrtf(n2);              // best = <k_row, k_seed> / |k_seed| (0 for a zero seed)
+                    sm_ = nj > 0.f ? best / nj : 0.f;
                     if (sim) sim[tok_off + i] = sm_;
                 }
                 const bool joined = cand && sm_ >= tau;

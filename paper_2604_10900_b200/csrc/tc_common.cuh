@@ -10,6 +10,7 @@ namespace tc {
 
 constexpr uint32_t kSpinLimit = 1u << 26;
 constexpr uint64_t kWaitLimitNs = 1000000000ull;     // one second
+constexpr uint32_t kSuspendHintNs = 2000u;
 
 // ---- PTX wrappers ------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -23,13 +24,15 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* b, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* b) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(b)) : "memory");
 }
+// One probe of a barrier phase.  The suspend-time hint lets the hardware park the thread until the phase
+// completes (or the hint runs out) instead of returning at once, so a waiting warp costs almost no issue slots.
 __device__ __forceinline__ bool mbar_try(uint64_t* b, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(b)), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(smem_u32(b)), "r"(parity), "r"(kSuspendHintNs) : "memory");
     return ok != 0;
 }
 __device__ __forceinline__ uint64_t global_ns() {

@@ -52,6 +52,14 @@ def test_long_reasoning_shape_bf16(score_path):
     print("score path", score_path, "max rel err", st["max_score_rel"], "exempt rows", st["exempt_rows"], "flipped", st["flipped_rows"])
 
 
+def test_many_seeds_share_accumulator_buffers():
+    """Budget 1024 on the config-3 shape: m = 192 seeds, so two epilogue groups split the seed columns."""
+    w = _small("reasoning32k_b1024", layers=1, kv_heads=2, decode=4096 + 77)
+    hb, run, g, o, st = _run(w)
+    assert (g["plan"][:, 5] == 192).all() and (g["n_out"] == 1024).all()
+    assert st["cascaded"] <= 1 and st["merged_elems"] > 0
+
+
 def test_prompt_heavy_two_stage():
     """Config-4 shape: prefix eviction fires before decode consolidation."""
     w = _small("prompt_heavy", layers=1, kv_heads=2, prefix=3072, decode=1024, budget=1024, reserve=256)
