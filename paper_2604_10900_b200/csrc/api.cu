@@ -178,6 +178,9 @@ Workspace carve(char* base, const cask_batch* b, const Sizes& z) {
     w.mem_row = (int32_t*)take(sumT * 4);
     w.mem_slot = (int32_t*)take(sumT * 4);
     w.n_mem = (int32_t*)take(n * 4);
+    w.seed_slot = (int32_t*)take(n * (size_t)std::max(z.max_B, 1) * 4);
+    w.n_seed = (int32_t*)take(n * 4);
+    w.max_B = std::max(z.max_B, 1);
     w.err = (int32_t*)take(16);
     w.bytes = off;
     return w;

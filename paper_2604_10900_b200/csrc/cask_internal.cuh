@@ -105,6 +105,9 @@ struct Workspace {
     int32_t* mem_row;    // [sumT] rows of kind 4/5 in ascending order
     int32_t* mem_slot;   // [sumT] slot each of them feeds
     int32_t* n_mem;      // [units]
+    int32_t* seed_slot;  // [units*max_B] slots of kind SEED, any order
+    int32_t* n_seed;     // [units]
+    int32_t max_B;
     int32_t* err;        // [1]
     size_t bytes;
 };

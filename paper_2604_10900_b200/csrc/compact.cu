@@ -14,8 +14,11 @@ __global__ void __launch_bounds__(kScanThreads) slot_scan_kernel(
     const UnitDesc* __restrict__ desc, const uint8_t* __restrict__ kind, const int32_t* __restrict__ seed_of,
     float* __restrict__ weight, int Bmax, int32_t* __restrict__ n_out, int32_t* __restrict__ slot_src,
     uint8_t* __restrict__ slot_kind, float* __restrict__ slot_mass, int32_t* __restrict__ assign,
-    int32_t* __restrict__ mem_row, int32_t* __restrict__ mem_slot, int32_t* __restrict__ n_mem) {
+    int32_t* __restrict__ mem_row, int32_t* __restrict__ mem_slot, int32_t* __restrict__ n_mem,
+    int32_t* __restrict__ seed_slot, int32_t* __restrict__ n_seed, int max_B) {
     __shared__ unsigned wk[kScanThreads / 32], wm[kScanThreads / 32];
+    __shared__ int seeds_listed;
+    if (threadIdx.x == 0) seeds_listed = 0;
     const int u = blockIdx.x;
     const UnitDesc& ud = desc[u];
     const int T = ud.T;
@@ -65,6 +68,14 @@ __global__ void __launch_bounds__(kScanThreads) slot_scan_kernel(
         slot_mass[(size_t)u * Bmax + t] = 0.f;
     }
     __syncthreads();
+    // the slots that hold a representative, for the merge kernel (any order)
+    for (int t = threadIdx.x; t < nk; t += blockDim.x)
+        if (slot_kind[(size_t)u * Bmax + t] == CASK_KIND_SEED) {
+            const int at = atomicAdd(&seeds_listed, 1);
+            if (at < max_B) seed_slot[(size_t)u * max_B + at] = t;
+        }
+    __syncthreads();
+    if (threadIdx.x == 0) n_seed[u] = min(seeds_listed, max_B);
     // members point at their seed's slot
     for (int e = threadIdx.x; e < nm; e += blockDim.x) {
         const int i = mem_row[o + e];
@@ -80,86 +91,95 @@ __global__ void __launch_bounds__(kScanThreads) slot_scan_kernel(
     }
 }
 
-// ---- 2. one warp per slot: byte copy, or ordered weighted merge ----------------------------
+// ---- 2. one warp per slot: byte copy of the slot's anchor row ------------------------------
 template <typename T>
-__global__ void __launch_bounds__(256) gather_merge_kernel(
+__global__ void __launch_bounds__(256) slot_copy_kernel(
     const UnitDesc* __restrict__ desc, Shape sh, const T* __restrict__ K, const T* __restrict__ V,
-    const float* __restrict__ s, const float* __restrict__ weight, float eps, int Bmax,
-    const int32_t* __restrict__ n_out, const int32_t* __restrict__ slot_src,
-    const uint8_t* __restrict__ slot_kind, const int32_t* __restrict__ mem_row,
-    const int32_t* __restrict__ mem_slot, const int32_t* __restrict__ n_mem, T* __restrict__ k_out,
-    T* __restrict__ v_out, float* __restrict__ slot_mass) {
+    const float* __restrict__ s, float eps, int Bmax, const int32_t* __restrict__ n_out,
+    const int32_t* __restrict__ slot_src, T* __restrict__ k_out, T* __restrict__ v_out,
+    float* __restrict__ slot_mass) {
     const int u = blockIdx.y;
     const UnitDesc& ud = desc[u];
     const int lane = threadIdx.x & 31;
     const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (t >= n_out[u]) return;
     const int d = sh.d;
-    const int64_t o = ud.tok_off;
     const int src = slot_src[(size_t)u * Bmax + t];
-    const uint8_t kd = slot_kind[(size_t)u * Bmax + t];
     T* ko = k_out + ((size_t)u * Bmax + t) * d;
     T* vo = v_out + ((size_t)u * Bmax + t) * d;
     const T* ksrc = K + row_elem_off(sh, ud, ud.k_off, src);
     const T* vsrc = V + row_elem_off(sh, ud, ud.v_off, src);
     const int nvec = d * (int)sizeof(T) / 16;
+    for (int x = lane; x < 2 * nvec; x += 32) {
+        const bool isv = x >= nvec;
+        const int c = isv ? x - nvec : x;
+        const uint4 val = reinterpret_cast<const uint4*>(isv ? vsrc : ksrc)[c];
+        reinterpret_cast<uint4*>(isv ? vo : ko)[c] = val;
+    }
+    if (lane == 0) slot_mass[(size_t)u * Bmax + t] = s[ud.tok_off + src] + eps;
+}
 
-    bool copy = true;
-    float mass = s[o + src] + eps;
-    if (kd == CASK_KIND_SEED) {
-        constexpr int kMaxPerLane = 8;      // d <= 256
-        float ak[kMaxPerLane], av[kMaxPerLane];
+// ---- 3. one warp per representative with joiners: ordered weighted merge over its copy -----
+template <typename T>
+__global__ void __launch_bounds__(256) slot_merge_kernel(
+    const UnitDesc* __restrict__ desc, Shape sh, const T* __restrict__ K, const T* __restrict__ V,
+    const float* __restrict__ s, const float* __restrict__ weight, float eps, int Bmax,
+    const int32_t* __restrict__ seed_slot, const int32_t* __restrict__ n_seed, int max_B,
+    const int32_t* __restrict__ mem_row, const int32_t* __restrict__ mem_slot,
+    const int32_t* __restrict__ n_mem, T* __restrict__ k_out, T* __restrict__ v_out,
+    float* __restrict__ slot_mass) {
+    const int u = blockIdx.y;
+    const UnitDesc& ud = desc[u];
+    const int lane = threadIdx.x & 31;
+    const int j = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (j >= n_seed[u]) return;
+    const int t = seed_slot[(size_t)u * max_B + j];
+    const int d = sh.d;
+    const int64_t o = ud.tok_off;
+    constexpr int kMaxPerLane = 8;      // d <= 256
+    float ak[kMaxPerLane], av[kMaxPerLane];
 #pragma unroll
-        for (int x = 0; x < kMaxPerLane; ++x) { ak[x] = 0.f; av[x] = 0.f; }
-        int count = 0;
-        float msum = 0.f;
-        const int nm = n_mem[u];
-        for (int e0 = 0; e0 < nm; e0 += 32) {
-            const int e = e0 + lane;
-            const int row = (e < nm) ? mem_row[o + e] : -1;
-            const bool hit = (e < nm) && mem_slot[o + e] == t;
-            unsigned bal = __ballot_sync(0xffffffffu, hit);
-            while (bal) {
-                const int l = __ffs(bal) - 1;
-                bal &= bal - 1;
-                const int i = __shfl_sync(0xffffffffu, row, l);
-                const float wi = weight[o + i];
-                msum += s[o + i] + eps;
-                ++count;
-                const T* kr = K + row_elem_off(sh, ud, ud.k_off, i);
-                const T* vr = V + row_elem_off(sh, ud, ud.v_off, i);
-#pragma unroll
-                for (int x = 0; x < kMaxPerLane; ++x) {
-                    const int c = lane + 32 * x;
-                    if (c < d) {
-                        ak[x] = fmaf(wi, Elem<T>::ld(kr + c), ak[x]);
-                        av[x] = fmaf(wi, Elem<T>::ld(vr + c), av[x]);
-                    }
-                }
-            }
-        }
-        if (count > 1) {
-            copy = false;
-            mass = msum;
+    for (int x = 0; x < kMaxPerLane; ++x) { ak[x] = 0.f; av[x] = 0.f; }
+    int count = 0;
+    float msum = 0.f;
+    const int nm = n_mem[u];
+    for (int e0 = 0; e0 < nm; e0 += 32) {
+        const int e = e0 + lane;
+        const int row = (e < nm) ? mem_row[o + e] : -1;
+        const bool hit = (e < nm) && mem_slot[o + e] == t;
+        unsigned bal = __ballot_sync(0xffffffffu, hit);
+        while (bal) {
+            const int l = __ffs(bal) - 1;
+            bal &= bal - 1;
+            const int i = __shfl_sync(0xffffffffu, row, l);
+            const float wi = weight[o + i];
+            msum += s[o + i] + eps;
+            ++count;
+            const T* kr = K + row_elem_off(sh, ud, ud.k_off, i);
+            const T* vr = V + row_elem_off(sh, ud, ud.v_off, i);
 #pragma unroll
             for (int x = 0; x < kMaxPerLane; ++x) {
                 const int c = lane + 32 * x;
                 if (c < d) {
-                    Elem<T>::st(ko + c, ak[x]);
-                    Elem<T>::st(vo + c, av[x]);
+                    ak[x] = fmaf(wi, Elem<T>::ld(kr + c), ak[x]);
+                    av[x] = fmaf(wi, Elem<T>::ld(vr + c), av[x]);
                 }
             }
         }
     }
-    if (copy) {
-        for (int x = lane; x < 2 * nvec; x += 32) {
-            const bool isv = x >= nvec;
-            const int c = isv ? x - nvec : x;
-            const uint4 val = reinterpret_cast<const uint4*>(isv ? vsrc : ksrc)[c];
-            reinterpret_cast<uint4*>(isv ? vo : ko)[c] = val;
+    if (count > 1) {       // a lone seed keeps its byte copy
+        T* ko = k_out + ((size_t)u * Bmax + t) * d;
+        T* vo = v_out + ((size_t)u * Bmax + t) * d;
+#pragma unroll
+        for (int x = 0; x < kMaxPerLane; ++x) {
+            const int c = lane + 32 * x;
+            if (c < d) {
+                Elem<T>::st(ko + c, ak[x]);
+                Elem<T>::st(vo + c, av[x]);
+            }
         }
+        if (lane == 0) slot_mass[(size_t)u * Bmax + t] = msum;
     }
-    if (lane == 0) slot_mass[(size_t)u * Bmax + t] = mass;
 }
 
 template <typename T>
@@ -171,14 +191,20 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const u
         slot_scan_kernel<<<sh.n_units, kScanThreads, 0, L.stream>>>(L.desc, kind, seed_of, weight, out.Bmax,
                                                                     out.n_out, out.slot_src, out.slot_kind,
                                                                     out.slot_mass, out.assign, ws.mem_row,
-                                                                    ws.mem_slot, ws.n_mem);
+                                                                    ws.mem_slot, ws.n_mem, ws.seed_slot, ws.n_seed,
+                                                                    ws.max_B);
     }
     const int slots = min(out.Bmax, max(L.max_B, 1));
     {
+        // the merge kernel overwrites slots the copy kernel wrote: same stream, in order
         Timed t(L, KID_GATHER_MERGE);
-        gather_merge_kernel<T><<<dim3((slots + 7) / 8, sh.n_units), 256, 0, L.stream>>>(
-            L.desc, sh, (const T*)L.k, (const T*)L.v, s, weight, prm.eps, out.Bmax, out.n_out, out.slot_src,
-            out.slot_kind, ws.mem_row, ws.mem_slot, ws.n_mem, (T*)out.k_out, (T*)out.v_out, out.slot_mass);
+        slot_copy_kernel<T><<<dim3((slots + 7) / 8, sh.n_units), 256, 0, L.stream>>>(
+            L.desc, sh, (const T*)L.k, (const T*)L.v, s, prm.eps, out.Bmax, out.n_out, out.slot_src, (T*)out.k_out,
+            (T*)out.v_out, out.slot_mass);
+        slot_merge_kernel<T><<<dim3((std::min(slots, ws.max_B) + 7) / 8, sh.n_units), 256, 0, L.stream>>>(
+            L.desc, sh, (const T*)L.k, (const T*)L.v, s, weight, prm.eps, out.Bmax, ws.seed_slot, ws.n_seed, ws.max_B,
+            ws.mem_row, ws.mem_slot, ws.n_mem, (T*)out.k_out, (T*)out.v_out, out.slot_mass);
+        ++*L.launches;
     }
     return cudaGetLastError();
 }
