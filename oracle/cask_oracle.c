@@ -33,6 +33,16 @@ enum {
 
 enum { PL_BP = 0, PL_PKEEP, PL_BD, PL_R, PL_C, PL_M, PL_FLAGS, PL_NOUT };
 
+/*
+ * Merge weight of a row (Sec. 2.4 leaves a_i open: "local score mass, similarity weight, or
+ * position-aware importance").  Reading: a_i = s_i + eps, plus the group mass the row already
+ * carries when it is itself a representative of an earlier event (mass_in, nullable), so that
+ * folding "preserves group mass" across events.
+ */
+static double orc_a(const double* s, const double* mass_in, double eps, int i) {
+    return s[i] + eps + (mass_in ? mass_in[i] : 0.0);
+}
+
 /* ---- total order used by every selection: score descending, row ascending ---- */
 typedef struct { double s; int i; } orc_item;
 
@@ -189,15 +199,15 @@ void cask_oracle_select_core(const double* s, int T, int P, const int* plan, uin
  * similarity of keys (ties: smallest seed row; a zero-norm row has similarity
  * 0) if that similarity is >= tau, else it is dropped and its a_j counts as
  * lost mass (the |Delta m_G| term of Sec. 2.6).  Merge weights (Sec. 2.4):
- *     a_i = s_i + eps,  m_G = sum_{i in G} a_i,  w_i = a_i / m_G.
+ *     a_i = s_i + eps (+ carried mass, see orc_a),  m_G = sum_{i in G} a_i,  w_i = a_i / m_G.
  * Outputs: kind (adds 4 seed, 5 merged), seed_of (row of the group's seed, -1),
  * weight (w_i for group members, untouched elsewhere), sim / sim2 (best and
  * second-best similarity of each non-seed scratch row; -2 where undefined).
  * Returns flags to OR into the unit's status (MERGE_INACTIVE if nobody joins).
  */
 int cask_oracle_consolidate(const float* K, const double* s, int T, int P, int d, const int* plan,
-                            double tau, double eps, uint8_t* kind, int* seed_of, double* weight,
-                            double* sim, double* sim2, double* lost_mass) {
+                            double tau, double eps, const double* mass_in, uint8_t* kind, int* seed_of,
+                            double* weight, double* sim, double* sim2, double* lost_mass) {
     int r = plan[PL_R], m = plan[PL_M];
     for (int i = 0; i < T; ++i) { seed_of[i] = -1; if (sim) sim[i] = -2.0; if (sim2) sim2[i] = -2.0; }
     *lost_mass = 0.0;
@@ -239,15 +249,15 @@ int cask_oracle_consolidate(const float* K, const double* s, int T, int P, int d
             seed_of[j] = seeds[best_u];
             ++joined;
         } else {
-            *lost_mass += s[j] + eps;
+            *lost_mass += orc_a(s, mass_in, eps, j);
         }
     }
     for (int u = 0; u < ns; ++u) {
         double mG = 0.0;
         for (int i = P; i < T - r; ++i)
-            if (seed_of[i] == seeds[u]) mG += s[i] + eps;
+            if (seed_of[i] == seeds[u]) mG += orc_a(s, mass_in, eps, i);
         for (int i = P; i < T - r; ++i)
-            if (seed_of[i] == seeds[u]) weight[i] = (s[i] + eps) / mG;
+            if (seed_of[i] == seeds[u]) weight[i] = orc_a(s, mass_in, eps, i) / mG;
     }
     free(seeds);
     free(snorm);
@@ -264,7 +274,7 @@ int cask_oracle_consolidate(const float* K, const double* s, int T, int P, int d
  */
 void cask_oracle_compact(const float* K, const float* V, int T, int d, const uint8_t* kind,
                          const int* seed_of, double* weight, const double* s, double eps,
-                         double* k_out, double* v_out, int* n_out, int* slot_src, uint8_t* slot_kind,
+                         const double* mass_in, double* k_out, double* v_out, int* n_out, int* slot_src, uint8_t* slot_kind,
                          double* slot_mass, int* assign) {
     int n = 0;
     for (int i = 0; i < T; ++i) {
@@ -288,13 +298,13 @@ void cask_oracle_compact(const float* K, const float* V, int T, int d, const uin
         double* vo = v_out + (size_t)t * d;
         if (slot_kind[t] != 4) {
             for (int c = 0; c < d; ++c) { ko[c] = K[(size_t)src * d + c]; vo[c] = V[(size_t)src * d + c]; }
-            slot_mass[t] = s[src] + eps;
+            slot_mass[t] = orc_a(s, mass_in, eps, src);
         } else {
             double mass = 0.0;
             for (int c = 0; c < d; ++c) { ko[c] = 0.0; vo[c] = 0.0; }
             for (int i = 0; i < T; ++i) {
                 if (seed_of[i] != src || (kind[i] != 4 && kind[i] != 5)) continue;
-                mass += s[i] + eps;
+                mass += orc_a(s, mass_in, eps, i);
                 for (int c = 0; c < d; ++c) {
                     ko[c] += weight[i] * (double)K[(size_t)i * d + c];
                     vo[c] += weight[i] * (double)V[(size_t)i * d + c];
@@ -305,24 +315,47 @@ void cask_oracle_compact(const float* K, const float* V, int T, int d, const uin
     }
 }
 
+/*
+ * Representative-set mass diagnostics (Sec. 2.6):
+ *     rho_core = sum_{k in C} s_k / sum_{k in TopK} s_k,   rho_rep = sum_{k in R} s_k / sum_{k in TopK} s_k.
+ * Reading: s is the score of this event; TopK is the B greatest rows of the whole cache (the best any
+ * B-row cache could hold); C = recent + core rows; the mass of R is the mass its slots carry
+ * (slot_mass: a kept row its a_i, a representative its group mass m_G).
+ */
+void cask_oracle_diagnostics(const double* s, int T, int B, const uint8_t* kind, const double* slot_mass,
+                             int n_out, double* rho_core, double* rho_rep) {
+    orc_item* it = (orc_item*)malloc(sizeof(orc_item) * (size_t)(T > 0 ? T : 1));
+    for (int i = 0; i < T; ++i) { it[i].s = s[i]; it[i].i = i; }
+    qsort(it, (size_t)T, sizeof(orc_item), orc_cmp);
+    double top = 0.0, core = 0.0, rep = 0.0;
+    for (int t = 0; t < T && t < B; ++t) top += it[t].s;
+    for (int i = 0; i < T; ++i)
+        if (kind[i] == 2 || kind[i] == 3) core += s[i];
+    for (int t = 0; t < n_out; ++t) rep += slot_mass[t];
+    *rho_core = top > 0.0 ? core / top : 0.0;
+    *rho_rep = top > 0.0 ? rep / top : 0.0;
+    free(it);
+}
+
 /* The whole event for one unit, the steps above in order.  plan[8] is written. */
 void cask_oracle_event(const float* K, const float* V, const float* Q, int T, int P, int B, int reserve,
                        int d, int g, int W, int causal, double gamma, double tau, double eps,
-                       const double* lse_in, double* s, int* plan, uint8_t* kind, int* seed_of,
-                       double* weight, double* sim, double* sim2, double* k_out, double* v_out,
+                       const double* lse_in, const double* mass_in, double* s, int* plan, uint8_t* kind,
+                       int* seed_of, double* weight, double* sim, double* sim2, double* k_out, double* v_out,
                        int* n_out, int* slot_src, uint8_t* slot_kind, double* slot_mass, int* assign,
-                       int* status, double* lost_mass) {
+                       int* status, double* lost_mass, double* rho /* nullable [2]: core, rep */) {
     cask_oracle_score(K, Q, T, d, g, W, causal, lse_in, s, NULL);
     cask_oracle_plan(T, P, B, reserve, W, gamma, plan);
     for (int i = 0; i < T; ++i) weight[i] = 0.0;
     cask_oracle_prefix_evict(s, P, plan, kind);
     cask_oracle_select_core(s, T, P, plan, kind);
-    int fl = cask_oracle_consolidate(K, s, T, P, d, plan, tau, eps, kind, seed_of, weight, sim, sim2,
+    int fl = cask_oracle_consolidate(K, s, T, P, d, plan, tau, eps, mass_in, kind, seed_of, weight, sim, sim2,
                                      lost_mass);
     if (!(plan[PL_FLAGS] & ORC_DECODE_CONSOLIDATED)) fl = 0;
-    cask_oracle_compact(K, V, T, d, kind, seed_of, weight, s, eps, k_out, v_out, n_out, slot_src,
+    cask_oracle_compact(K, V, T, d, kind, seed_of, weight, s, eps, mass_in, k_out, v_out, n_out, slot_src,
                         slot_kind, slot_mass, assign);
     *status = plan[PL_FLAGS] | fl;
+    if (rho) cask_oracle_diagnostics(s, T, B, kind, slot_mass, *n_out, rho, rho + 1);
 }
 
 /*
@@ -334,10 +367,10 @@ void cask_oracle_event(const float* K, const float* V, const float* Q, int T, in
 void cask_oracle_event_batch(int n_units, const float* K, const float* V, const float* Q,
                              const int64_t* tok_off, const int* P, const int* B, const int* reserve,
                              int d, int g, int W, int causal, double gamma, double tau, double eps,
-                             int Bmax, double* s, int* plan, uint8_t* kind, int* seed_of, double* weight,
+                             const double* mass_in /* nullable [sum T] */, int Bmax, double* s, int* plan, uint8_t* kind, int* seed_of, double* weight,
                              double* sim, double* sim2, double* k_out, double* v_out, int* n_out,
                              int* slot_src, uint8_t* slot_kind, double* slot_mass, int* assign,
-                             int* status, double* lost_mass) {
+                             int* status, double* lost_mass, double* rho /* nullable [n_units, 2] */) {
 #ifdef _OPENMP
 #pragma omp parallel for schedule(dynamic, 1)
 #endif
@@ -346,10 +379,10 @@ void cask_oracle_event_batch(int n_units, const float* K, const float* V, const 
         int T = (int)(tok_off[u + 1] - tok_off[u]);
         size_t so = (size_t)u * (size_t)Bmax;
         cask_oracle_event(K + a * d, V + a * d, Q + (size_t)u * g * W * d, T, P[u], B[u], reserve[u], d, g,
-                          W, causal, gamma, tau, eps, NULL, s + a, plan + (size_t)u * 8, kind + a,
+                          W, causal, gamma, tau, eps, NULL, mass_in ? mass_in + a : NULL, s + a, plan + (size_t)u * 8, kind + a,
                           seed_of + a, weight + a, sim ? sim + a : NULL, sim2 ? sim2 + a : NULL,
                           k_out + so * d, v_out + so * d, n_out + u, slot_src + so, slot_kind + so,
-                          slot_mass + so, assign + a, status + u, lost_mass + u);
+                          slot_mass + so, assign + a, status + u, lost_mass + u, rho ? rho + 2 * (size_t)u : NULL);
     }
 }
 

@@ -85,7 +85,7 @@ def select_core(s, T: int, P: int, pl: np.ndarray, kind: np.ndarray) -> None:
     lib().cask_oracle_select_core(_p(s, C.c_double), int(T), int(P), _p(pl, C.c_int), _p(kind, C.c_uint8))
 
 
-def consolidate(K, s, P: int, pl: np.ndarray, kind: np.ndarray, tau: float = 0.9, eps: float = 1e-9):
+def consolidate(K, s, P: int, pl: np.ndarray, kind: np.ndarray, tau: float = 0.9, eps: float = 1e-9, mass_in=None):
     """Updates ``kind`` in place; returns dict(seed_of, weight, sim, sim2, flags, lost_mass)."""
     K = _f32(K)
     T, d = K.shape
@@ -94,16 +94,17 @@ def consolidate(K, s, P: int, pl: np.ndarray, kind: np.ndarray, tau: float = 0.9
     weight = np.zeros(T, dtype=np.float64)
     sim = np.zeros(T, dtype=np.float64)
     sim2 = np.zeros(T, dtype=np.float64)
+    mass_in = None if mass_in is None else np.ascontiguousarray(mass_in, dtype=np.float64)
     lost = C.c_double(0.0)
     fn = lib().cask_oracle_consolidate
     fn.restype = C.c_int
     fl = fn(_p(K, C.c_float), _p(s, C.c_double), T, int(P), d, _p(pl, C.c_int), C.c_double(tau),
-            C.c_double(eps), _p(kind, C.c_uint8), _p(seed_of, C.c_int), _p(weight, C.c_double),
-            _p(sim, C.c_double), _p(sim2, C.c_double), C.byref(lost))
+            C.c_double(eps), _p(mass_in, C.c_double), _p(kind, C.c_uint8), _p(seed_of, C.c_int),
+            _p(weight, C.c_double), _p(sim, C.c_double), _p(sim2, C.c_double), C.byref(lost))
     return dict(seed_of=seed_of, weight=weight, sim=sim, sim2=sim2, flags=int(fl), lost_mass=lost.value)
 
 
-def compact(K, V, kind, seed_of, weight, s, eps: float = 1e-9):
+def compact(K, V, kind, seed_of, weight, s, eps: float = 1e-9, mass_in=None):
     """Returns dict(k_out, v_out [n_out,d] float64, n_out, slot_src, slot_kind, slot_mass, assign, weight)."""
     K, V = _f32(K), _f32(V)
     T, d = K.shape
@@ -118,10 +119,11 @@ def compact(K, V, kind, seed_of, weight, s, eps: float = 1e-9):
     slot_kind = np.zeros(max(cap, 1), dtype=np.uint8)
     slot_mass = np.zeros(max(cap, 1), dtype=np.float64)
     assign = np.zeros(T, dtype=np.int32)
+    mass_in = None if mass_in is None else np.ascontiguousarray(mass_in, dtype=np.float64)
     n_out = C.c_int(0)
     lib().cask_oracle_compact(_p(K, C.c_float), _p(V, C.c_float), T, d, _p(kind, C.c_uint8),
                               _p(seed_of, C.c_int), _p(weight, C.c_double), _p(s, C.c_double),
-                              C.c_double(eps), _p(k_out, C.c_double), _p(v_out, C.c_double),
+                              C.c_double(eps), _p(mass_in, C.c_double), _p(k_out, C.c_double), _p(v_out, C.c_double),
                               C.byref(n_out), _p(slot_src, C.c_int), _p(slot_kind, C.c_uint8),
                               _p(slot_mass, C.c_double), _p(assign, C.c_int))
     n = n_out.value
@@ -130,7 +132,7 @@ def compact(K, V, kind, seed_of, weight, s, eps: float = 1e-9):
 
 
 def event_batch(K, V, Q, tok_off, P, B, reserve, causal: int = 1, gamma: float = 0.5, tau: float = 0.9,
-                eps: float = 1e-9) -> Dict[str, np.ndarray]:
+                eps: float = 1e-9, mass_in=None) -> Dict[str, np.ndarray]:
     """Whole event for many contiguous units.  K, V [sum T, d]; Q [n, g, W, d] (float32 values)."""
     K, V, Q = _f32(K), _f32(V), _f32(Q)
     n, g, W, d = Q.shape
@@ -147,17 +149,19 @@ def event_batch(K, V, Q, tok_off, P, B, reserve, causal: int = 1, gamma: float =
         v_out=np.zeros((n, Bmax, d), np.float64), n_out=np.zeros(n, np.int32),
         slot_src=np.zeros((n, Bmax), np.int32), slot_kind=np.zeros((n, Bmax), np.uint8),
         slot_mass=np.zeros((n, Bmax), np.float64), assign=np.zeros(Tt, np.int32),
-        status=np.zeros(n, np.int32), lost_mass=np.zeros(n, np.float64))
+        status=np.zeros(n, np.int32), lost_mass=np.zeros(n, np.float64), rho=np.zeros((n, 2), np.float64))
+    mass_in = None if mass_in is None else np.ascontiguousarray(mass_in, dtype=np.float64)
     lib().cask_oracle_event_batch(
         n, _p(K, C.c_float), _p(V, C.c_float), _p(Q, C.c_float), _p(tok_off, C.c_int64), _p(P, C.c_int),
         _p(B, C.c_int), _p(reserve, C.c_int), d, g, W, int(causal), C.c_double(gamma), C.c_double(tau),
-        C.c_double(eps), Bmax, _p(o["s"], C.c_double), _p(o["plan"], C.c_int), _p(o["kind"], C.c_uint8),
+        C.c_double(eps), _p(mass_in, C.c_double), Bmax, _p(o["s"], C.c_double), _p(o["plan"], C.c_int), _p(o["kind"], C.c_uint8),
         _p(o["seed_of"], C.c_int), _p(o["weight"], C.c_double), _p(o["sim"], C.c_double),
         _p(o["sim2"], C.c_double), _p(o["k_out"], C.c_double), _p(o["v_out"], C.c_double),
         _p(o["n_out"], C.c_int), _p(o["slot_src"], C.c_int), _p(o["slot_kind"], C.c_uint8),
         _p(o["slot_mass"], C.c_double), _p(o["assign"], C.c_int), _p(o["status"], C.c_int),
-        _p(o["lost_mass"], C.c_double))
+        _p(o["lost_mass"], C.c_double), _p(o["rho"], C.c_double))
     o["Bmax"] = Bmax
+    o["rho_core"], o["rho_rep"] = o["rho"][:, 0].copy(), o["rho"][:, 1].copy()
     return o
 
 
@@ -174,6 +178,7 @@ def event(K, V, Q, P: int, B: int, reserve: int, **kw) -> Dict[str, np.ndarray]:
     out["n_out"] = n
     out["status"] = int(o["status"][0])
     out["lost_mass"] = float(o["lost_mass"][0])
+    out["rho_core"], out["rho_rep"] = float(o["rho_core"][0]), float(o["rho_rep"][0])
     return out
 
 

@@ -44,11 +44,11 @@ def cosine(a: List[float], b: List[float]) -> float:
 
 
 def event(K, V, Q, P: int, B: int, reserve: int, gamma: float = 0.5, tau: float = 0.9,
-          eps: float = 1e-9, causal: bool = True) -> Dict:
+          eps: float = 1e-9, causal: bool = True, mass_in=None) -> Dict:
     T, d = len(K), len(K[0])
     W = len(Q[0])
     s = scores(K, Q, causal)
-    a = [x + eps for x in s]
+    a = [x + eps + (mass_in[i] if mass_in is not None else 0.0) for i, x in enumerate(s)]
     Nd = T - P
     prefix, decode = list(range(P)), list(range(P, T))
     flags = 0
@@ -125,5 +125,8 @@ def event(K, V, Q, P: int, B: int, reserve: int, gamma: float = 0.5, tau: float 
         for x in mem:
             if x != u:
                 kind[x] = 5
-    return dict(s=s, kind=kind, slots=slots, weight=weight, assign=assign, k_out=k_out, v_out=v_out,
+    top_mass = math.fsum(sorted(s, reverse=True)[:B])
+    rho_core = math.fsum(s[i] for i in range(T) if kind[i] in (2, 3)) / top_mass
+    rho_rep = math.fsum(mass) / top_mass
+    return dict(rho_core=rho_core, rho_rep=rho_rep, s=s, kind=kind, slots=slots, weight=weight, assign=assign, k_out=k_out, v_out=v_out,
                 mass=mass, flags=flags, lost=lost, n_out=len(slots))

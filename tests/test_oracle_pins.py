@@ -301,9 +301,11 @@ def test_planted_clusters_are_recovered_with_full_purity():
 
 # ---- whole event vs the separately written brute force -----------------------
 
-def _cmp_with_bruteforce(K, V, Q, P, B, res, tau):
-    o = orc.event(K, V, Q, P, B, res, tau=tau)
-    b = bf.event(K.tolist(), V.tolist(), Q.tolist(), P, B, res, tau=tau)
+def _cmp_with_bruteforce(K, V, Q, P, B, res, tau, mass_in=None):
+    o = orc.event(K, V, Q, P, B, res, tau=tau, mass_in=mass_in)
+    b = bf.event(K.tolist(), V.tolist(), Q.tolist(), P, B, res, tau=tau,
+                 mass_in=None if mass_in is None else list(mass_in))
+    assert abs(o["rho_core"] - b["rho_core"]) < 1e-12 and abs(o["rho_rep"] - b["rho_rep"]) < 1e-12
     assert np.allclose(o["s"], b["s"], rtol=1e-12, atol=1e-300)
     assert o["kind"].tolist() == b["kind"]
     assert o["slot_src"].tolist() == b["slots"]
@@ -333,6 +335,40 @@ def test_whole_event_against_bruteforce_all_small_shapes():
                     _cmp_with_bruteforce(K, V, Q, P, B, res, tau=0.9 if (P + B) % 2 else -1.0)
                     n += 1
     assert n > 1500
+
+
+def test_carried_mass_and_diagnostics_against_bruteforce_and_closed_forms():
+    """Rows that already carry group mass (representatives of an earlier event) fold with a_i = s_i + eps +
+    carried mass (Sec. 2.4: the fold preserves group mass); rho_core / rho_rep of Sec. 2.6."""
+    rng = np.random.default_rng(12)
+    T, d, W = 14, 4, 2
+    centres = rng.standard_normal((3, d))
+    K = (centres[rng.integers(0, 3, T)] + 0.05 * rng.standard_normal((T, d))).astype(np.float32)
+    V = rng.standard_normal((T, d)).astype(np.float32)
+    Q = rng.standard_normal((2, W, d)).astype(np.float32)
+    mass = np.where(rng.random(T) < 0.4, rng.random(T) * 0.5, 0.0)
+    for P, B, res in [(0, 6, 6), (3, 8, 5), (4, 9, 6), (0, 5, 5), (2, 7, 4)]:
+        for tau in (-1.0, 0.9):
+            _cmp_with_bruteforce(K, V, Q, P, B, res, tau, mass_in=mass)
+    # zero carried mass is the plain event
+    a = orc.event(K, V, Q, 3, 8, 5, tau=-1.0)
+    b = orc.event(K, V, Q, 3, 8, 5, tau=-1.0, mass_in=np.zeros(T))
+    for k in ("kind", "weight", "slot_mass", "k_out", "rho_rep"):
+        assert np.array_equal(a[k], b[k])
+    # tau = -1 loses nothing: the slots hold the a_i of every kept or merged row; selections ignore the mass
+    c = orc.event(K, V, Q, 0, 6, 6, tau=-1.0, mass_in=mass)
+    a0 = orc.event(K, V, Q, 0, 6, 6, tau=-1.0)
+    assert np.array_equal(c["kind"], a0["kind"]) and c["lost_mass"] == 0.0
+    assert np.isclose(c["slot_mass"].sum(), (c["s"] + 1e-9 + mass).sum(), rtol=1e-12)
+    # a heavy member pulls the representative towards itself: weights are a_i / m_G
+    grp = np.flatnonzero(c["assign"] == c["assign"][np.flatnonzero(c["kind"] == 5)[0]])
+    aw = c["s"][grp] + 1e-9 + mass[grp]
+    assert np.allclose(c["weight"][grp], aw / aw.sum(), rtol=1e-12)
+    # diagnostics: C is part of R, so rho_core <= rho_rep; with nothing lost and no prefix R carries all the
+    # mass, which is at least the mass of the best B rows; a cache under budget keeps everything
+    assert c["rho_core"] <= c["rho_rep"] and a0["rho_rep"] >= 1.0 - 1e-12
+    u = orc.event(K, V, Q, 2, T + 1, 3)
+    assert abs(u["rho_rep"] - (1.0 + T * 1e-9)) < 1e-12 and u["rho_core"] <= 1.0
 
 
 def test_whole_event_against_bruteforce_exhausted_boundary():
