@@ -116,6 +116,10 @@ typedef struct {
     const int32_t* block_table; /* DEVICE physical page id of every logical page, unit after unit */
     const int64_t* bt_off;   /* HOST [n_units+1] first entry of each unit; bt_off[u+1]-bt_off[u] >= ceil(T[u]/page_size) */
     int64_t n_pages;         /* pages in the k and v pools                      */
+    /* optional: mass already carried by a row (a representative of an earlier event brings the
+       slot_mass it was given then, every other row 0).  Merge weights become
+       a_i = s_i + eps + mass_in[i] (Sec. 2.4: the fold preserves group mass); NULL = all zero. */
+    const float* mass_in;    /* DEVICE [sumT] or NULL                           */
 } cask_batch;
 
 /*
@@ -149,6 +153,10 @@ typedef struct {
     float* s;              /* optional [sumT] scores                                          */
     float* lse;            /* optional [n_units, g, W] natural-log normalisers used           */
     float* sim;            /* optional [sumT] best cosine similarity of non-seed scratch rows, -2 elsewhere */
+    /* optional mass diagnostics of Sec. 2.6, [n_units] each: share of the mass of the B best rows of the
+       cache that the protected core (recent + core rows) holds, and that the output slots carry */
+    float* rho_core;
+    float* rho_rep;
 } cask_outputs;
 
 /* ---- context ------------------------------------------------------------ */
@@ -244,8 +252,8 @@ int cask_consolidate_scratch(cask_ctx* ctx, const cask_batch* batch, const cask_
  * accumulation, rounded once to the cache dtype; a group of one is a byte
  * copy); every other slot is a byte copy of its row.  `weight` is read for
  * kinds 4/5 and finalised (1 for kinds 1..3, 0 for kind 0).  Uses out->k_out,
- * v_out, Bmax, n_out, slot_src, slot_kind, slot_mass, assign; other fields of
- * `out` are ignored.
+ * v_out, Bmax, n_out, slot_src, slot_kind, slot_mass, assign and, when given,
+ * rho_core / rho_rep; other fields of `out` are ignored.
  */
 int cask_compact(cask_ctx* ctx, const cask_batch* batch, const cask_params* params,
                  const float* s, const uint8_t* kind, const int32_t* seed_of, float* weight,

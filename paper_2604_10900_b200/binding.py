@@ -45,6 +45,7 @@ class CaskBatch(C.Structure):
         ("T", C.c_void_p), ("P", C.c_void_p), ("B", C.c_void_p), ("reserve", C.c_void_p),
         ("tok_off", C.c_void_p),
         ("block_table", C.c_void_p), ("bt_off", C.c_void_p), ("n_pages", C.c_int64),
+        ("mass_in", C.c_void_p),
     ]
 
 
@@ -60,6 +61,7 @@ class CaskOutputs(C.Structure):
         ("assign", C.c_void_p), ("weight", C.c_void_p), ("kind", C.c_void_p), ("seed_of", C.c_void_p),
         ("plan", C.c_void_p), ("unit_status", C.c_void_p), ("lost_mass", C.c_void_p),
         ("s", C.c_void_p), ("lse", C.c_void_p), ("sim", C.c_void_p),
+        ("rho_core", C.c_void_p), ("rho_rep", C.c_void_p),
     ]
 
 
@@ -149,7 +151,7 @@ class HostArrays:
 
 def make_batch(k, v, q, T, P, B, reserve, tok_off, head_dim: int, group: int, window: int, dtype: int,
                k_off=None, v_off=None, row_stride: Optional[int] = None, lse_in=None, page_size: int = 0,
-               block_table=None, bt_off=None, n_pages: int = 0):
+               block_table=None, bt_off=None, n_pages: int = 0, mass_in=None):
     """Fills a cask_batch.  k, v, q, lse_in: tensors/arrays/addresses (device for the device calls,
     host for cask_compress_event_host).  Paged cache: page_size > 0, k and v the page pools,
     block_table a device int32 tensor, bt_off the host offsets of the units in it.
@@ -172,7 +174,8 @@ def make_batch(k, v, q, T, P, B, reserve, tok_off, head_dim: int, group: int, wi
     b.block_table = _ptr(block_table)
     b.bt_off = None if bt_host is None else bt_host.ctypes.data
     b.n_pages = n_pages
-    return b, (h, k, v, q, lse_in, block_table, bt_host)
+    b.mass_in = _ptr(mass_in)
+    return b, (h, k, v, q, lse_in, block_table, bt_host, mass_in)
 
 
 def make_outputs(d: Dict, Bmax: int) -> CaskOutputs:
@@ -360,7 +363,8 @@ def alloc_outputs(n_units: int, sum_T: int, Bmax: int, d: int, rows: int, dtype:
         unit_status=z((n_units,), torch.int32), lost_mass=z((n_units,), torch.float32))
     if optional:
         o.update(s=z((sum_T,), torch.float32), lse=z((n_units, rows), torch.float32),
-                 sim=z((sum_T,), torch.float32))
+                 sim=z((sum_T,), torch.float32), rho_core=z((n_units,), torch.float32),
+                 rho_rep=z((n_units,), torch.float32))
     return o
 
 

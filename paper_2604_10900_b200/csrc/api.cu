@@ -113,6 +113,7 @@ int check_batch(const cask_batch* b, const cask_params* p) {
     if (((uintptr_t)b->k | (uintptr_t)b->v | (uintptr_t)b->q) % 16 || (b->row_stride * e) % 16)
         return CASK_ERR_ALIGN;
     if (b->lse_in && (uintptr_t)b->lse_in % 4) return CASK_ERR_ALIGN;
+    if (b->mass_in && (uintptr_t)b->mass_in % 4) return CASK_ERR_ALIGN;
     for (int u = 0; u < b->n_units; ++u) {
         const int T = b->T[u], P = b->P[u], B = b->B[u], R = b->reserve[u];
         if (T < 1 || b->window > T || P < 0 || P > T || B < 1 || R < 0 || R > B) return CASK_ERR_SHAPE;
@@ -260,6 +261,7 @@ int prepare(cask_ctx* ctx, const cask_batch* b, const cask_params* p, void* ws, 
     L.sh.rows = b->group * b->window; L.sh.dtype = b->dtype; L.sh.row_stride = b->row_stride;
     L.sh.causal = p->causal;
     L.sh.page_size = b->page_size; L.sh.n_pages = b->n_pages; L.sh.bt = b->block_table; L.sh.err = W.err;
+    L.sh.mass_in = b->mass_in;
     L.desc = W.desc; L.hdesc = ctx->pinned;
     L.k = b->k; L.v = b->v; L.q = b->q;
     L.max_T = z.max_T; L.max_m = z.max_m; L.max_chunks = z.max_chunks; L.total_chunks = z.total_chunks;
@@ -369,7 +371,7 @@ int cask_kernel_count(void) { return KID_COUNT; }
 const char* cask_kernel_name(int id) {
     static const char* names[KID_COUNT] = {"score_norm", "row_combine", "score_mass", "prefix_evict",
                                            "select_core", "seeds", "seed_gather", "assign", "weights",
-                                           "slot_scan", "gather_merge"};
+                                           "slot_scan", "gather_merge", "diagnostics"};
     return (id >= 0 && id < KID_COUNT) ? names[id] : "";
 }
 
@@ -493,6 +495,7 @@ int cask_compact(cask_ctx* ctx, const cask_batch* b, const cask_params* p, const
     rc = prepare(ctx, b, p, ws, ws_bytes, L, W);
     if (rc != CASK_OK || b->n_units == 0) return rc;
     cudaError_t e = launch_compact(L, *p, s, kind, seed_of, weight, *out, W);
+    if (e == cudaSuccess) e = launch_diagnostics(L, s, kind, *out);
     return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
 }
 
@@ -515,6 +518,7 @@ int cask_compress_event(cask_ctx* ctx, const cask_batch* b, const cask_params* p
         e = launch_consolidate(L, *p, s, out->plan, out->kind, out->seed_of, out->weight, out->sim,
                                out->unit_status, out->lost_mass, W);
     if (e == cudaSuccess) e = launch_compact(L, *p, s, out->kind, out->seed_of, out->weight, *out, W);
+    if (e == cudaSuccess) e = launch_diagnostics(L, s, out->kind, *out);
     return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
 }
 
@@ -522,7 +526,7 @@ int cask_compress_event(cask_ctx* ctx, const cask_batch* b, const cask_params* p
 
 namespace {
 struct HostStage {
-    char *k, *v, *q, *lse_in;
+    char *k, *v, *q, *lse_in, *mass_in;
     cask_outputs o;
     char* ws;
     size_t ws_bytes, bytes;
@@ -546,6 +550,7 @@ HostStage stage_layout(char* base, const cask_batch* b, const cask_params* p, in
     h.v = take(h.kv_bytes);
     h.q = take(h.q_bytes);
     h.lse_in = take(h.lse_bytes);
+    h.mass_in = take(sumT * 4);
     h.o.Bmax = Bmax;
     h.o.k_out = take(n * Bmax * d * e);
     h.o.v_out = take(n * Bmax * d * e);
@@ -563,6 +568,8 @@ HostStage stage_layout(char* base, const cask_batch* b, const cask_params* p, in
     h.o.s = (float*)take(sumT * 4);
     h.o.lse = (float*)take(n * rows * 4);
     h.o.sim = (float*)take(sumT * 4);
+    h.o.rho_core = (float*)take(n * 4);
+    h.o.rho_rep = (float*)take(n * 4);
     h.ws_bytes = carve(nullptr, b, batch_sizes(b, p)).bytes;
     h.ws = take(h.ws_bytes);
     h.bytes = off;
@@ -603,8 +610,11 @@ int cask_compress_event_host(cask_ctx* ctx, const cask_batch* hb, const cask_par
     if (e == cudaSuccess) e = cudaMemcpyAsync(h.q, hb->q, h.q_bytes, cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess && hb->lse_in)
         e = cudaMemcpyAsync(h.lse_in, hb->lse_in, h.lse_bytes, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && hb->mass_in)
+        e = cudaMemcpyAsync(h.mass_in, hb->mass_in, (size_t)hb->tok_off[hb->n_units] * 4, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return fail_cuda(ctx, e);
     cask_batch db = *hb;
+    db.mass_in = hb->mass_in ? (const float*)h.mass_in : nullptr;
     db.k = h.k; db.v = h.v; db.q = h.q;
     db.lse_in = hb->lse_in ? (const float*)h.lse_in : nullptr;
     rc = cask_compress_event(ctx, &db, p, &h.o, h.ws, h.ws_bytes);
@@ -622,6 +632,7 @@ int cask_compress_event_host(cask_ctx* ctx, const cask_batch* hb, const cask_par
         {ho->plan, h.o.plan, n * 32}, {ho->unit_status, h.o.unit_status, n * 4},
         {ho->lost_mass, h.o.lost_mass, n * 4}, {ho->s, h.o.s, sumT * 4},
         {ho->lse, h.o.lse, n * rows * 4}, {ho->sim, h.o.sim, sumT * 4},
+        {ho->rho_core, h.o.rho_core, n * 4}, {ho->rho_rep, h.o.rho_rep, n * 4},
     };
     for (const Cp& c : cps) {
         if (!c.dst) continue;

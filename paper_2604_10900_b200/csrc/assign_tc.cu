@@ -299,7 +299,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 const int i = a0 + (tile0 + t) * kTileRows + my_row;
                 const bool in_range = i >= P && i < hi;
                 const uint8_t kd = in_range ? kind[tok_off + i] : (uint8_t)CASK_KIND_RECENT;
-                const float sc = in_range ? s[tok_off + i] : 0.f;
+                const float sc = in_range ? row_mass(sh, s, eps, tok_off + i) : 0.f;     // a_i
                 // squared norm of this thread's row, read from the staged tile (any order of the
                 // sixteen 16-byte pieces of the row gives the same set of elements)
                 ok = mbar_wait(&bar.k_full[st], (kit / kStages) & 1u, abort_flag);
@@ -357,7 +357,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     if (sim) sim[tok_off + i] = sm_;
                 }
                 const bool joined = cand && sm_ >= tau;
-                const unsigned long long fx = cand ? mass_to_fx(sc + eps) : 0ull;
+                const unsigned long long fx = cand ? mass_to_fx(sc) : 0ull;
                 if (joined) {
                     kind[tok_off + i] = CASK_KIND_MERGED;
                     seed_of[tok_off + i] = seed_rows[seed_base + best_u];

@@ -38,12 +38,13 @@ struct Shape {
     int64_t n_pages;
     const int32_t* bt;   // device
     int32_t* err;        // device flag word (CASK_ST_TIMEOUT, CASK_ST_BOUNDS)
+    const float* mass_in;   // device, optional [sumT]: group mass a row already carries
 };
 
 // Kernel ids for the optional per-kernel event timing.
 enum KernelId {
     KID_SCORE_NORM = 0, KID_ROW_COMBINE, KID_SCORE_MASS, KID_PREFIX_EVICT, KID_SELECT_CORE, KID_SEEDS,
-    KID_SEED_GATHER, KID_ASSIGN, KID_WEIGHTS, KID_SLOT_SCAN, KID_GATHER_MERGE, KID_COUNT
+    KID_SEED_GATHER, KID_ASSIGN, KID_WEIGHTS, KID_SLOT_SCAN, KID_GATHER_MERGE, KID_DIAGNOSTICS, KID_COUNT
 };
 
 // Records a CUDA event pair around every launch while switched on (defined in api.cu).
@@ -123,6 +124,8 @@ cudaError_t launch_consolidate(const Launch& L, const cask_params& prm, const fl
                                float* sim, int32_t* unit_status, float* lost_mass, Workspace& ws);
 cudaError_t launch_compact(const Launch& L, const cask_params& prm, const float* s, const uint8_t* kind,
                            const int32_t* seed_of, float* weight, const cask_outputs& out, Workspace& ws);
+// rho_core / rho_rep of Sec. 2.6 per unit (either pointer may be NULL).
+cudaError_t launch_diagnostics(const Launch& L, const float* s, const uint8_t* kind, const cask_outputs& out);
 
 // Tensor-core assignment of scratch rows to seeds (cosine Gram + argmax), same outputs as the SIMT kernel.
 bool assign_tc_supported(const Launch& L);
@@ -147,6 +150,11 @@ __device__ __forceinline__ int64_t paged_row(const Shape& sh, const UnitDesc& ud
         pg = 0;
     }
     return (int64_t)pg * sh.page_size + i % sh.page_size;
+}
+// Merge weight a_i of the row at per-row index idx (Sec. 2.4): score + eps, plus the mass it already carries.
+__device__ __forceinline__ float row_mass(const Shape& sh, const float* __restrict__ s, float eps, int64_t idx) {
+    const float a = s[idx] + eps;
+    return sh.mass_in ? a + sh.mass_in[idx] : a;
 }
 // Element offset of logical row i of a unit in the K (unit_off = k_off) or V (v_off) array.
 __device__ __forceinline__ int64_t row_elem_off(const Shape& sh, const UnitDesc& ud, int64_t unit_off, int i) {

@@ -116,7 +116,7 @@ __global__ void __launch_bounds__(256) slot_copy_kernel(
         const uint4 val = reinterpret_cast<const uint4*>(isv ? vsrc : ksrc)[c];
         reinterpret_cast<uint4*>(isv ? vo : ko)[c] = val;
     }
-    if (lane == 0) slot_mass[(size_t)u * Bmax + t] = s[ud.tok_off + src] + eps;
+    if (lane == 0) slot_mass[(size_t)u * Bmax + t] = row_mass(sh, s, eps, ud.tok_off + src);
 }
 
 // ---- 3. one warp per representative with joiners: ordered weighted merge over its copy -----
@@ -153,7 +153,7 @@ __global__ void __launch_bounds__(256) slot_merge_kernel(
             bal &= bal - 1;
             const int i = __shfl_sync(0xffffffffu, row, l);
             const float wi = weight[o + i];
-            msum += s[o + i] + eps;
+            msum += row_mass(sh, s, eps, o + i);
             ++count;
             const T* kr = K + row_elem_off(sh, ud, ud.k_off, i);
             const T* vr = V + row_elem_off(sh, ud, ud.v_off, i);

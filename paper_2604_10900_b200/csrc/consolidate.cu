@@ -76,7 +76,7 @@ __global__ void seed_gather_kernel(const UnitDesc* __restrict__ desc, Shape sh, 
     for (int off = 16; off >= 1; off >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, off);
     if (threadIdx.x == 0) {
         seed_norm[ud.seed_base + j] = sqrtf(n2);
-        atomicAdd(&mass_fx[(size_t)u * (max_m + 1) + j], mass_to_fx(s[ud.tok_off + row] + eps));
+        atomicAdd(&mass_fx[(size_t)u * (max_m + 1) + j], mass_to_fx(row_mass(sh, s, eps, ud.tok_off + row)));
     }
 }
 
@@ -186,7 +186,7 @@ __global__ void __launch_bounds__(kThreads) assign_simt_kernel(
         int i = lo + rr;
         if (tx == 0 && rr < nrows && kind[ud.tok_off + i] == CASK_KIND_DROPPED) {
             if (sim) sim[ud.tok_off + i] = best[a];
-            unsigned long long fx = mass_to_fx(s[ud.tok_off + i] + eps);
+            unsigned long long fx = mass_to_fx(row_mass(sh, s, eps, ud.tok_off + i));
             if (best_u[a] >= 0 && best[a] >= tau) {
                 kind[ud.tok_off + i] = CASK_KIND_MERGED;
                 seed_of[ud.tok_off + i] = seed_rows[ud.seed_base + best_u[a]];
@@ -201,7 +201,7 @@ __global__ void __launch_bounds__(kThreads) assign_simt_kernel(
 }
 
 // ---- 4. merge weights w_i = a_i / m_G, lost mass, status ---------------------------------
-__global__ void weights_kernel(const UnitDesc* __restrict__ desc, const float* __restrict__ s,
+__global__ void weights_kernel(const UnitDesc* __restrict__ desc, Shape sh, const float* __restrict__ s,
                                const int32_t* __restrict__ plan, const int32_t* __restrict__ grp,
                                const unsigned long long* __restrict__ mass_fx,
                                const int32_t* __restrict__ njoin, float* __restrict__ weight,
@@ -213,7 +213,7 @@ __global__ void weights_kernel(const UnitDesc* __restrict__ desc, const float* _
     const unsigned long long* mf = mass_fx + (size_t)u * (max_m + 1);
     if (i < ud.T) {
         int gidx = grp[ud.tok_off + i];
-        if (gidx >= 0 && gidx < max_m) weight[ud.tok_off + i] = (s[ud.tok_off + i] + eps) / fx_to_mass(mf[gidx]);
+        if (gidx >= 0 && gidx < max_m) weight[ud.tok_off + i] = row_mass(sh, s, eps, ud.tok_off + i) / fx_to_mass(mf[gidx]);
     }
     if (i == 0) {
         int fl = plan[u * 8 + CASK_PLAN_FLAGS];
@@ -259,7 +259,7 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const i
     {
         Timed t(L, KID_WEIGHTS);
         weights_kernel<<<dim3((L.max_T + 255) / 256, sh.n_units), 256, 0, L.stream>>>(
-            L.desc, s, plan, ws.grp, ws.mass_fx, ws.njoin, weight, unit_status, lost_mass, max_m, prm.eps, ws.err);
+            L.desc, sh, s, plan, ws.grp, ws.mass_fx, ws.njoin, weight, unit_status, lost_mass, max_m, prm.eps, ws.err);
     }
     return cudaGetLastError();
 }

@@ -60,6 +60,43 @@ def test_many_seeds_share_accumulator_buffers():
     assert st["cascaded"] <= 1 and st["merged_elems"] > 0
 
 
+def test_carried_mass_second_event_on_a_compacted_cache():
+    """Steady state: the cache left by one event, grown by 128 new decode rows, is compressed again; its
+    representatives bring the group mass they were given (a_i = s_i + eps + carried mass)."""
+    import gpu_harness as gh
+    w = _small("reasoning8k_b384", layers=1, kv_heads=3, decode=2048)
+    hb, run, g, o, st = _run(w)
+    rng = np.random.default_rng(77)
+    n_new, d, B = 128, w.head_dim, w.budget
+    ko, vo = run.out["k_out"].view(run.torch.uint16).cpu().numpy(), run.out["v_out"].view(run.torch.uint16).cpu().numpy()
+    k2, v2, mass, T2, P2 = [], [], [], [], []
+    for u in range(hb.n_units):
+        n = int(g["n_out"][u])
+        fresh_k = wl.to_cache_dtype(rng.standard_normal((n_new, d)).astype(np.float32) * wl.channel_scale(w, 0, 0), w.dtype)
+        # half of the new rows repeat kept rows with a little noise, so that the second event merges again
+        src = rng.integers(int(g["plan"][u][1]), n, n_new // 2)
+        noisy = wl.bf16_bits_to_f32(ko[u][src]) + 0.05 * rng.standard_normal((n_new // 2, d)).astype(np.float32)
+        fresh_k[: n_new // 2] = wl.to_cache_dtype(noisy, w.dtype)
+        k2.append(np.concatenate([ko[u][:n], fresh_k]))
+        v2.append(np.concatenate([vo[u][:n], wl.to_cache_dtype(rng.standard_normal((n_new, d)).astype(np.float32), w.dtype)]))
+        mass.append(np.concatenate([np.where(g["slot_kind"][u][:n] == 4, g["slot_mass"][u][:n], 0.0), np.zeros(n_new)]))
+        T2.append(n + n_new)
+        P2.append(int(g["plan"][u][1]))
+    T2 = np.array(T2, np.int32)
+    hb2 = wl.Batch(wl=w, k=np.concatenate(k2), v=np.concatenate(v2), q=hb.q, T=T2, P=np.array(P2, np.int32), B=hb.B,
+                   reserve=hb.reserve, tok_off=np.concatenate([[0], np.cumsum(T2)]).astype(np.int64), unit_ids=hb.unit_ids)
+    mass = np.concatenate(mass).astype(np.float32)
+    assert (mass > 0).any()
+    run2 = gh.GpuRun(hb2, mass_in=mass)
+    g2 = run2.event()
+    o2 = gh.run_oracle(hb2, mass_in=mass.astype(np.float64))
+    st2 = gh.compare_event(hb2, g2, o2)
+    assert (g2["n_out"] == B).all() and st2["merged_elems"] > 0 and st2["cascaded"] <= 1
+    # the carried mass changes the fold: without it the merged rows come out differently
+    g3 = gh.GpuRun(hb2).event()
+    assert np.array_equal(g3["kind"], g2["kind"]) and not np.array_equal(g3["weight"], g2["weight"])
+
+
 def test_prompt_heavy_two_stage():
     """Config-4 shape: prefix eviction fires before decode consolidation."""
     w = _small("prompt_heavy", layers=1, kv_heads=2, prefix=3072, decode=1024, budget=1024, reserve=256)
