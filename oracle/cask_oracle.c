@@ -200,13 +200,18 @@ void cask_oracle_select_core(const double* s, int T, int P, const int* plan, uin
  * 0) if that similarity is >= tau, else it is dropped and its a_j counts as
  * lost mass (the |Delta m_G| term of Sec. 2.6).  Merge weights (Sec. 2.4):
  *     a_i = s_i + eps (+ carried mass, see orc_a),  m_G = sum_{i in G} a_i,  w_i = a_i / m_G.
+ * chan_w (nullable, [d], >= 0) weighs the channels of the similarity (Sec. 2.5: differences in frequency
+ * bands with more future relevance count more; reading: the inner-product form
+ *     sim_w(j,u) = sum_c w_c k_jc k_uc / (|k_j|_w |k_u|_w),  |k|_w^2 = sum_c w_c k_c^2,
+ * with w_c = |kappa(omega_f)| on the channels of band f supplied by the caller; NULL = plain cosine).
  * Outputs: kind (adds 4 seed, 5 merged), seed_of (row of the group's seed, -1),
  * weight (w_i for group members, untouched elsewhere), sim / sim2 (best and
  * second-best similarity of each non-seed scratch row; -2 where undefined).
  * Returns flags to OR into the unit's status (MERGE_INACTIVE if nobody joins).
  */
 int cask_oracle_consolidate(const float* K, const double* s, int T, int P, int d, const int* plan,
-                            double tau, double eps, const double* mass_in, uint8_t* kind, int* seed_of,
+                            double tau, double eps, const double* mass_in, const float* chan_w, uint8_t* kind,
+                            int* seed_of,
                             double* weight, double* sim, double* sim2, double* lost_mass) {
     int r = plan[PL_R], m = plan[PL_M];
     for (int i = 0; i < T; ++i) { seed_of[i] = -1; if (sim) sim[i] = -2.0; if (sim2) sim2[i] = -2.0; }
@@ -220,7 +225,8 @@ int cask_oracle_consolidate(const float* K, const double* s, int T, int P, int d
         if (kind[i] == 4) {
             seeds[ns] = i;
             double n2 = 0.0;
-            for (int c = 0; c < d; ++c) n2 += (double)K[(size_t)i * d + c] * (double)K[(size_t)i * d + c];
+            for (int c = 0; c < d; ++c)
+                n2 += (chan_w ? (double)chan_w[c] : 1.0) * (double)K[(size_t)i * d + c] * (double)K[(size_t)i * d + c];
             snorm[ns] = sqrt(n2);
             seed_of[i] = i;
             ++ns;
@@ -230,14 +236,14 @@ int cask_oracle_consolidate(const float* K, const double* s, int T, int P, int d
         if (kind[j] != 0) continue;
         const float* kj = K + (size_t)j * d;
         double n2 = 0.0;
-        for (int c = 0; c < d; ++c) n2 += (double)kj[c] * (double)kj[c];
+        for (int c = 0; c < d; ++c) n2 += (chan_w ? (double)chan_w[c] : 1.0) * (double)kj[c] * (double)kj[c];
         double nj = sqrt(n2);
         double best = -INFINITY, second = -INFINITY;
         int best_u = -1;
         for (int u = 0; u < ns; ++u) {           /* seeds[] ascends, so '>' keeps the smallest row on ties */
             const float* ku = K + (size_t)seeds[u] * d;
             double dot = 0.0;
-            for (int c = 0; c < d; ++c) dot += (double)kj[c] * (double)ku[c];
+            for (int c = 0; c < d; ++c) dot += (chan_w ? (double)chan_w[c] : 1.0) * (double)kj[c] * (double)ku[c];
             double sm = (nj > 0.0 && snorm[u] > 0.0) ? dot / (nj * snorm[u]) : 0.0;
             if (sm > best) { second = best; best = sm; best_u = u; }
             else if (sm > second) second = sm;
@@ -340,7 +346,8 @@ void cask_oracle_diagnostics(const double* s, int T, int B, const uint8_t* kind,
 /* The whole event for one unit, the steps above in order.  plan[8] is written. */
 void cask_oracle_event(const float* K, const float* V, const float* Q, int T, int P, int B, int reserve,
                        int d, int g, int W, int causal, double gamma, double tau, double eps,
-                       const double* lse_in, const double* mass_in, double* s, int* plan, uint8_t* kind,
+                       const double* lse_in, const double* mass_in, const float* chan_w, double* s, int* plan,
+                       uint8_t* kind,
                        int* seed_of, double* weight, double* sim, double* sim2, double* k_out, double* v_out,
                        int* n_out, int* slot_src, uint8_t* slot_kind, double* slot_mass, int* assign,
                        int* status, double* lost_mass, double* rho /* nullable [2]: core, rep */) {
@@ -349,7 +356,7 @@ void cask_oracle_event(const float* K, const float* V, const float* Q, int T, in
     for (int i = 0; i < T; ++i) weight[i] = 0.0;
     cask_oracle_prefix_evict(s, P, plan, kind);
     cask_oracle_select_core(s, T, P, plan, kind);
-    int fl = cask_oracle_consolidate(K, s, T, P, d, plan, tau, eps, mass_in, kind, seed_of, weight, sim, sim2,
+    int fl = cask_oracle_consolidate(K, s, T, P, d, plan, tau, eps, mass_in, chan_w, kind, seed_of, weight, sim, sim2,
                                      lost_mass);
     if (!(plan[PL_FLAGS] & ORC_DECODE_CONSOLIDATED)) fl = 0;
     cask_oracle_compact(K, V, T, d, kind, seed_of, weight, s, eps, mass_in, k_out, v_out, n_out, slot_src,
@@ -367,7 +374,8 @@ void cask_oracle_event(const float* K, const float* V, const float* Q, int T, in
 void cask_oracle_event_batch(int n_units, const float* K, const float* V, const float* Q,
                              const int64_t* tok_off, const int* P, const int* B, const int* reserve,
                              int d, int g, int W, int causal, double gamma, double tau, double eps,
-                             const double* mass_in /* nullable [sum T] */, int Bmax, double* s, int* plan, uint8_t* kind, int* seed_of, double* weight,
+                             const double* mass_in /* nullable [sum T] */, const float* chan_w /* nullable [d] */,
+                             int Bmax, double* s, int* plan, uint8_t* kind, int* seed_of, double* weight,
                              double* sim, double* sim2, double* k_out, double* v_out, int* n_out,
                              int* slot_src, uint8_t* slot_kind, double* slot_mass, int* assign,
                              int* status, double* lost_mass, double* rho /* nullable [n_units, 2] */) {
@@ -379,7 +387,7 @@ void cask_oracle_event_batch(int n_units, const float* K, const float* V, const 
         int T = (int)(tok_off[u + 1] - tok_off[u]);
         size_t so = (size_t)u * (size_t)Bmax;
         cask_oracle_event(K + a * d, V + a * d, Q + (size_t)u * g * W * d, T, P[u], B[u], reserve[u], d, g,
-                          W, causal, gamma, tau, eps, NULL, mass_in ? mass_in + a : NULL, s + a, plan + (size_t)u * 8, kind + a,
+                          W, causal, gamma, tau, eps, NULL, mass_in ? mass_in + a : NULL, chan_w, s + a, plan + (size_t)u * 8, kind + a,
                           seed_of + a, weight + a, sim ? sim + a : NULL, sim2 ? sim2 + a : NULL,
                           k_out + so * d, v_out + so * d, n_out + u, slot_src + so, slot_kind + so,
                           slot_mass + so, assign + a, status + u, lost_mass + u, rho ? rho + 2 * (size_t)u : NULL);

@@ -35,16 +35,17 @@ def top(rows: List[int], s: List[float], k: int) -> List[int]:
     return sorted(rows, key=lambda i: (-s[i], i))[:max(k, 0)]
 
 
-def cosine(a: List[float], b: List[float]) -> float:
-    na = math.sqrt(math.fsum(x * x for x in a))
-    nb = math.sqrt(math.fsum(x * x for x in b))
+def cosine(a: List[float], b: List[float], w=None) -> float:
+    w = [1.0] * len(a) if w is None else w
+    na = math.sqrt(math.fsum(c * x * x for c, x in zip(w, a)))
+    nb = math.sqrt(math.fsum(c * x * x for c, x in zip(w, b)))
     if na == 0.0 or nb == 0.0:
         return 0.0
-    return math.fsum(x * y for x, y in zip(a, b)) / (na * nb)
+    return math.fsum(c * x * y for c, x, y in zip(w, a, b)) / (na * nb)
 
 
 def event(K, V, Q, P: int, B: int, reserve: int, gamma: float = 0.5, tau: float = 0.9,
-          eps: float = 1e-9, causal: bool = True, mass_in=None) -> Dict:
+          eps: float = 1e-9, causal: bool = True, mass_in=None, chan_w=None) -> Dict:
     T, d = len(K), len(K[0])
     W = len(Q[0])
     s = scores(K, Q, causal)
@@ -93,7 +94,7 @@ def event(K, V, Q, P: int, B: int, reserve: int, gamma: float = 0.5, tau: float 
             for j in scratch:
                 if j in groups:
                     continue
-                sims = [(cosine(K[j], K[u]), -u) for u in seeds]
+                sims = [(cosine(K[j], K[u], chan_w), -u) for u in seeds]
                 best, negu = max(sims)
                 if best >= tau:
                     groups[-negu].append(j)

@@ -301,10 +301,11 @@ def test_planted_clusters_are_recovered_with_full_purity():
 
 # ---- whole event vs the separately written brute force -----------------------
 
-def _cmp_with_bruteforce(K, V, Q, P, B, res, tau, mass_in=None):
-    o = orc.event(K, V, Q, P, B, res, tau=tau, mass_in=mass_in)
+def _cmp_with_bruteforce(K, V, Q, P, B, res, tau, mass_in=None, chan_w=None):
+    o = orc.event(K, V, Q, P, B, res, tau=tau, mass_in=mass_in, chan_w=chan_w)
     b = bf.event(K.tolist(), V.tolist(), Q.tolist(), P, B, res, tau=tau,
-                 mass_in=None if mass_in is None else list(mass_in))
+                 mass_in=None if mass_in is None else list(mass_in),
+                 chan_w=None if chan_w is None else [float(x) for x in chan_w])
     assert abs(o["rho_core"] - b["rho_core"]) < 1e-12 and abs(o["rho_rep"] - b["rho_rep"]) < 1e-12
     assert np.allclose(o["s"], b["s"], rtol=1e-12, atol=1e-300)
     assert o["kind"].tolist() == b["kind"]
@@ -369,6 +370,36 @@ def test_carried_mass_and_diagnostics_against_bruteforce_and_closed_forms():
     assert c["rho_core"] <= c["rho_rep"] and a0["rho_rep"] >= 1.0 - 1e-12
     u = orc.event(K, V, Q, 2, T + 1, 3)
     assert abs(u["rho_rep"] - (1.0 + T * 1e-9)) < 1e-12 and u["rho_core"] <= 1.0
+
+
+def test_channel_weighted_similarity():
+    """Sec. 2.5: channels (frequency bands) weigh differently in the merge geometry.  Unit weights are the plain
+    cosine; 0/1 weights are the cosine of the selected channels (numpy); a common factor changes nothing."""
+    rng = np.random.default_rng(13)
+    T, d, W, P, B, res = 40, 8, 2, 0, 12, 12
+    centres = rng.standard_normal((4, d))
+    K = (centres[rng.integers(0, 4, T)] + 0.2 * rng.standard_normal((T, d))).astype(np.float32)
+    V = rng.standard_normal((T, d)).astype(np.float32)
+    Q = rng.standard_normal((2, W, d)).astype(np.float32)
+    plain = orc.event(K, V, Q, P, B, res, tau=0.8)
+    ones = orc.event(K, V, Q, P, B, res, tau=0.8, chan_w=np.ones(d))
+    assert np.array_equal(plain["kind"], ones["kind"]) and np.array_equal(plain["sim"], ones["sim"])
+    w = rng.random(d).astype(np.float32) + 0.1
+    a = orc.event(K, V, Q, P, B, res, tau=0.8, chan_w=w)
+    b = orc.event(K, V, Q, P, B, res, tau=0.8, chan_w=4.0 * w)
+    assert np.array_equal(a["kind"], b["kind"]) and np.allclose(a["sim"], b["sim"], rtol=1e-12)
+    assert not np.array_equal(a["sim"], plain["sim"])
+    mask = np.array([1, 1, 0, 0, 1, 0, 1, 1], np.float32)
+    m = orc.event(K, V, Q, P, B, res, tau=0.8, chan_w=mask)
+    seeds = np.flatnonzero(m["kind"] == 4)
+    Ks = K[:, mask > 0].astype(np.float64)
+    for j in np.flatnonzero(m["sim"] > -1.5):
+        cs = Ks[seeds] @ Ks[j] / (np.linalg.norm(Ks[seeds], axis=1) * np.linalg.norm(Ks[j]))
+        assert abs(cs.max() - m["sim"][j]) < 1e-12
+        if m["kind"][j] == 5:
+            assert m["seed_of"][j] == seeds[int(np.argmax(cs))]
+    for tau in (-1.0, 0.8):
+        _cmp_with_bruteforce(K[:14], V[:14], Q, 2, 7, 4, tau, chan_w=w)
 
 
 def test_whole_event_against_bruteforce_exhausted_boundary():
