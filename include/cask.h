@@ -120,6 +120,10 @@ typedef struct {
        slot_mass it was given then, every other row 0).  Merge weights become
        a_i = s_i + eps + mass_in[i] (Sec. 2.4: the fold preserves group mass); NULL = all zero. */
     const float* mass_in;    /* DEVICE [sumT] or NULL                           */
+    /* optional: non-negative channel weights of the merge similarity (Sec. 2.5: frequency bands of
+       more future relevance count more; w_c = |kappa(omega_f)| on the channels of band f):
+       sim(j,u) = sum_c w_c k_jc k_uc / (|k_j|_w |k_u|_w), |k|_w^2 = sum_c w_c k_c^2.  NULL = cosine. */
+    const float* chan_w;     /* DEVICE [head_dim] or NULL                       */
 } cask_batch;
 
 /*

@@ -45,7 +45,7 @@ class CaskBatch(C.Structure):
         ("T", C.c_void_p), ("P", C.c_void_p), ("B", C.c_void_p), ("reserve", C.c_void_p),
         ("tok_off", C.c_void_p),
         ("block_table", C.c_void_p), ("bt_off", C.c_void_p), ("n_pages", C.c_int64),
-        ("mass_in", C.c_void_p),
+        ("mass_in", C.c_void_p), ("chan_w", C.c_void_p),
     ]
 
 
@@ -151,7 +151,7 @@ class HostArrays:
 
 def make_batch(k, v, q, T, P, B, reserve, tok_off, head_dim: int, group: int, window: int, dtype: int,
                k_off=None, v_off=None, row_stride: Optional[int] = None, lse_in=None, page_size: int = 0,
-               block_table=None, bt_off=None, n_pages: int = 0, mass_in=None):
+               block_table=None, bt_off=None, n_pages: int = 0, mass_in=None, chan_w=None):
     """Fills a cask_batch.  k, v, q, lse_in: tensors/arrays/addresses (device for the device calls,
     host for cask_compress_event_host).  Paged cache: page_size > 0, k and v the page pools,
     block_table a device int32 tensor, bt_off the host offsets of the units in it.
@@ -175,7 +175,8 @@ def make_batch(k, v, q, T, P, B, reserve, tok_off, head_dim: int, group: int, wi
     b.bt_off = None if bt_host is None else bt_host.ctypes.data
     b.n_pages = n_pages
     b.mass_in = _ptr(mass_in)
-    return b, (h, k, v, q, lse_in, block_table, bt_host, mass_in)
+    b.chan_w = _ptr(chan_w)
+    return b, (h, k, v, q, lse_in, block_table, bt_host, mass_in, chan_w)
 
 
 def make_outputs(d: Dict, Bmax: int) -> CaskOutputs:

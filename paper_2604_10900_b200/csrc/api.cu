@@ -114,6 +114,7 @@ int check_batch(const cask_batch* b, const cask_params* p) {
         return CASK_ERR_ALIGN;
     if (b->lse_in && (uintptr_t)b->lse_in % 4) return CASK_ERR_ALIGN;
     if (b->mass_in && (uintptr_t)b->mass_in % 4) return CASK_ERR_ALIGN;
+    if (b->chan_w && (uintptr_t)b->chan_w % 4) return CASK_ERR_ALIGN;
     for (int u = 0; u < b->n_units; ++u) {
         const int T = b->T[u], P = b->P[u], B = b->B[u], R = b->reserve[u];
         if (T < 1 || b->window > T || P < 0 || P > T || B < 1 || R < 0 || R > B) return CASK_ERR_SHAPE;
@@ -172,7 +173,7 @@ Workspace carve(char* base, const cask_batch* b, const Sizes& z) {
     w.part_l = (float*)take(parts * rows * 4);
     w.seed_rows = (int32_t*)take((size_t)z.sum_m * 4);
     w.seed_norm = (float*)take((size_t)z.sum_m * 4);
-    w.seed_k = take(((size_t)z.sum_m + 256) * b->head_dim * elem_size(b->dtype));
+    w.seed_k = take((2 * (size_t)z.sum_m + 256) * b->head_dim * elem_size(b->dtype));   // room for hi/lo rows
     w.grp = (int32_t*)take(sumT * 4);
     w.mass_fx = (unsigned long long*)take(n * ((size_t)z.max_m + 1) * 8);
     w.njoin = (int32_t*)take(n * 4);
@@ -261,7 +262,7 @@ int prepare(cask_ctx* ctx, const cask_batch* b, const cask_params* p, void* ws, 
     L.sh.rows = b->group * b->window; L.sh.dtype = b->dtype; L.sh.row_stride = b->row_stride;
     L.sh.causal = p->causal;
     L.sh.page_size = b->page_size; L.sh.n_pages = b->n_pages; L.sh.bt = b->block_table; L.sh.err = W.err;
-    L.sh.mass_in = b->mass_in;
+    L.sh.mass_in = b->mass_in; L.sh.chan_w = b->chan_w;
     L.desc = W.desc; L.hdesc = ctx->pinned;
     L.k = b->k; L.v = b->v; L.q = b->q;
     L.max_T = z.max_T; L.max_m = z.max_m; L.max_chunks = z.max_chunks; L.total_chunks = z.total_chunks;
@@ -526,7 +527,7 @@ int cask_compress_event(cask_ctx* ctx, const cask_batch* b, const cask_params* p
 
 namespace {
 struct HostStage {
-    char *k, *v, *q, *lse_in, *mass_in;
+    char *k, *v, *q, *lse_in, *mass_in, *chan_w;
     cask_outputs o;
     char* ws;
     size_t ws_bytes, bytes;
@@ -551,6 +552,7 @@ HostStage stage_layout(char* base, const cask_batch* b, const cask_params* p, in
     h.q = take(h.q_bytes);
     h.lse_in = take(h.lse_bytes);
     h.mass_in = take(sumT * 4);
+    h.chan_w = take(d * 4);
     h.o.Bmax = Bmax;
     h.o.k_out = take(n * Bmax * d * e);
     h.o.v_out = take(n * Bmax * d * e);
@@ -615,6 +617,11 @@ int cask_compress_event_host(cask_ctx* ctx, const cask_batch* hb, const cask_par
     if (e != cudaSuccess) return fail_cuda(ctx, e);
     cask_batch db = *hb;
     db.mass_in = hb->mass_in ? (const float*)h.mass_in : nullptr;
+    if (hb->chan_w) {
+        e = cudaMemcpyAsync(h.chan_w, hb->chan_w, (size_t)hb->head_dim * 4, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+    }
+    db.chan_w = hb->chan_w ? (const float*)h.chan_w : nullptr;
     db.k = h.k; db.v = h.v; db.q = h.q;
     db.lse_in = hb->lse_in ? (const float*)h.lse_in : nullptr;
     rc = cask_compress_event(ctx, &db, p, &h.o, h.ws, h.ws_bytes);

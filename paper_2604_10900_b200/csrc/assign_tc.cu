@@ -44,6 +44,7 @@ struct ASmemTail {
     uint32_t tmem_base;
     int abort;
     float inv_nu[2][256];     // 1/|k_seed| (0 for a zero seed), double-buffered by unit
+    alignas(16) float w[128]; // channel weights of the similarity (1 when none are given)
     float x_val[2][2][128];   // shared buffers: best dot product / seed norm and its seed,
     int x_idx[2][2][128];     //   per buffer, per use parity, per tile row
 };
@@ -81,41 +82,39 @@ struct TileWalk {
 };
 
 // Best seed among the accumulator columns [c_lo, c_hi) of this thread's row: the greatest dot * 1/|k_seed|, the
-// first column among equals.  A block of 32 columns costs a multiply and a maximum per column; the position of
+// first seed among equals.  PAIR = 1: a seed owns two adjacent columns (the hi and lo parts of its weighted key)
+// whose sum is its dot product.  A block of 32 columns costs a multiply and a maximum per seed; the position of
 // the maximum is looked for only in a block that beats everything before it.
+template <int PAIR>
 __device__ __forceinline__ void best_seed(uint32_t taddr, const float* inv, int c_lo, int c_hi, float& best, int& best_u) {
+    constexpr int kPer = PAIR ? 16 : 32;          // seeds per block of 32 columns
     for (int cc = c_lo; cc < c_hi; cc += 32) {
         float v[32];
         tc_ld32(taddr + cc, v);
         tc_wait_ld_regs(v);
+        const int u0 = PAIR ? cc >> 1 : cc, u_hi = PAIR ? c_hi >> 1 : c_hi;
         float bm = -INFINITY;
-        if (cc + 32 <= c_hi) {
+        const bool whole = cc + 32 <= c_hi;
 #pragma unroll
-            for (int x = 0; x < 32; ++x) {
-                v[x] *= inv[cc + x];
-                bm = fmaxf(bm, v[x]);
-            }
-        } else {
-#pragma unroll
-            for (int x = 0; x < 32; ++x) {
-                v[x] = (cc + x < c_hi) ? v[x] * inv[cc + x] : -INFINITY;
-                bm = fmaxf(bm, v[x]);
-            }
+        for (int x = 0; x < kPer; ++x) {
+            const float dot = PAIR ? v[2 * x] + v[2 * x + 1] : v[x];
+            v[x] = (whole || u0 + x < u_hi) ? dot * inv[u0 + x] : -INFINITY;
+            bm = fmaxf(bm, v[x]);
         }
         if (bm > best) {
             best = bm;
-            int at = 31;
+            int at = kPer - 1;
 #pragma unroll
-            for (int x = 30; x >= 0; --x)
+            for (int x = kPer - 2; x >= 0; --x)
                 if (v[x] == bm) at = x;
-            best_u = cc + at;
+            best_u = u0 + at;
         }
     }
 }
 
 __global__ void __launch_bounds__(kThreadsA, 1)
 assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmSeed,
-                 const UnitDesc* __restrict__ desc, Shape sh, int total_tiles, int n_bufs, int sub_rows,
+                 const UnitDesc* __restrict__ desc, Shape sh, int total_tiles, int n_bufs, int sub_rows, int wpair,
                  const float* __restrict__ s, const int32_t* __restrict__ plan,
                  const int32_t* __restrict__ seed_rows, const float* __restrict__ seed_norm,
                  uint8_t* __restrict__ kind, int32_t* __restrict__ seed_of, float* __restrict__ sim,
@@ -143,6 +142,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         tail->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (threadIdx.x < 128) tail->w[threadIdx.x] = sh.chan_w ? sh.chan_w[threadIdx.x] : 1.f;
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tail->tmem_base)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -165,8 +165,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 ok = mbar_wait(&bar.b_empty, (ucount & 1u) ^ 1u, abort_flag);
                 if (!ok) break;
                 mbar_expect_tx(&bar.b_full, kSeedBytes);
-                tma_load_2d(b_smem, &tmSeed, &bar.b_full, 0, ud.seed_base);
-                tma_load_2d(b_smem + kSeedRegionBytes, &tmSeed, &bar.b_full, 64, ud.seed_base);
+                tma_load_2d(b_smem, &tmSeed, &bar.b_full, 0, ud.seed_base << wpair);
+                tma_load_2d(b_smem + kSeedRegionBytes, &tmSeed, &bar.b_full, 64, ud.seed_base << wpair);
                 ++ucount;
                 // first cache row of the unit's tile sequence (a page-piece boundary in a paged cache)
                 const int a0 = ud.P - (sh.page_size ? ud.P % sub_rows : 0);
@@ -209,7 +209,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             while (wk.valid() && ok) {
                 const UnitDesc& ud = desc[wk.u];
                 const int m = max(0, min(plan[wk.u * 8 + CASK_PLAN_M], ud.plan[CASK_PLAN_M]));
-                const uint32_t idesc = umma_idesc(max(16, (m + 15) & ~15));
+                const uint32_t idesc = umma_idesc(max(16, ((m << wpair) + 15) & ~15));
                 ok = mbar_wait(&bar.b_full, ucount & 1u, abort_flag);
                 if (!ok) break;
                 ++ucount;
@@ -260,7 +260,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const int hi = T - r;
             const int a0 = P - (sh.page_size ? P % sub_rows : 0);
             // shared buffers: the finishing group also computes the row norm, so it takes fewer seed columns
-            const int c_split = split == 2 ? min(m, 32 * max(1, (((m + 31) >> 5) - 2) / 2)) : m;
+            const int mc = m << wpair;               // accumulator columns in use
+            const int c_split = split == 2 ? min(mc, 32 * max(1, (((mc + 31) >> 5) - 2) / 2)) : mc;
             unsigned long long* mass_u = mass_fx + (size_t)u * (max_m + 1);
             float* inv = tail->inv_nu[ucount & 1u];
             if (etid < 256) {
@@ -284,7 +285,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     tc_fence_after();
                     float best = -INFINITY;
                     int best_u = -1;
-                    best_seed(taddr, inv, c_split, m, best, best_u);
+                    if (wpair) best_seed<1>(taddr, inv, c_split, mc, best, best_u);
+                    else best_seed<0>(taddr, inv, c_split, mc, best, best_u);
                     tc_fence_before();
                     tail->x_val[eg][use & 1u][my_row] = best;
                     tail->x_idx[eg][use & 1u][my_row] = best_u;
@@ -317,7 +319,14 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll
                             for (int x = 0; x < 4; ++x) {
                                 const uint64_t f2 = pack2(__uint_as_float(wv[x] << 16), __uint_as_float(wv[x] & 0xFFFF0000u));
-                                n2p = fma2(f2, f2, n2p);
+                                if (sh.chan_w) {
+                                    // the 128-byte swizzle stores logical 16-byte piece p of row r at position p ^ (r & 7)
+                                    const float2 w2 = *reinterpret_cast<const float2*>(
+                                        &tail->w[kb * 64 + ((((c + lane) & 7) ^ (my_row & 7)) << 3) + 2 * x]);
+                                    n2p = fma2(fma2(f2, pack2(w2.x, w2.y), 0ull), f2, n2p);
+                                } else {
+                                    n2p = fma2(f2, f2, n2p);
+                                }
                             }
                         }
                 }
@@ -331,7 +340,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 tc_fence_after();
                 float best = -INFINITY;
                 int best_u = -1;
-                best_seed(taddr, inv, 0, c_split, best, best_u);
+                if (wpair) best_seed<1>(taddr, inv, 0, c_split, best, best_u);
+                else best_seed<0>(taddr, inv, 0, c_split, best, best_u);
                 tc_fence_before();
                 if (split == 2) {
                     // The other group's candidate has the larger seed indices, so it wins only when strictly
@@ -400,7 +410,8 @@ int assign_tc_box_rows(const Shape& sh) {
 
 bool assign_tc_supported(const Launch& L) {
     const Shape& sh = L.sh;
-    if (sh.dtype != CASK_DTYPE_BF16 || sh.d != 128 || L.max_m > 256 || L.max_m < 1 || L.total_atiles < 1)
+    const int cols = L.max_m << (sh.chan_w ? 1 : 0);      // a weighted seed takes two accumulator columns
+    if (sh.dtype != CASK_DTYPE_BF16 || sh.d != 128 || cols > 256 || L.max_m < 1 || L.total_atiles < 1)
         return false;
     if (sh.page_size) return assign_tc_box_rows(sh) != 0 && sh.n_pages * sh.page_size < ((int64_t)1 << 31);
     int64_t max_row = 0;
@@ -425,7 +436,8 @@ cudaError_t launch_assign_tc(const Launch& L, const cask_params& prm, const floa
     if (!encode_rows_bf16(tmap_encode_fn, &tmK, L.k, (uint64_t)k_rows, (uint64_t)sh.row_stride * 2, sub_rows))
         return cudaErrorInvalidValue;
     // the seed table has 256 spare rows behind the last seed, so a full box never leaves the allocation
-    if (!encode_rows_bf16(tmap_encode_fn, &tmSeed, ws.seed_k, (uint64_t)sum_m + 256, 256, 256))
+    const int wpair = sh.chan_w ? 1 : 0;
+    if (!encode_rows_bf16(tmap_encode_fn, &tmSeed, ws.seed_k, ((uint64_t)sum_m << wpair) + 256, 256, 256))
         return cudaErrorInvalidValue;
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -438,7 +450,7 @@ cudaError_t launch_assign_tc(const Launch& L, const cask_params& prm, const floa
     {
         Timed t(L, KID_ASSIGN);
         assign_tc_kernel<<<grid, kThreadsA, kSmemBytesA, L.stream>>>(
-            tmK, tmSeed, L.desc, sh, L.total_atiles, L.max_m <= 128 ? 4 : 2, sub_rows, s, plan, ws.seed_rows, ws.seed_norm, kind, seed_of, sim, ws.grp,
+            tmK, tmSeed, L.desc, sh, L.total_atiles, (L.max_m << wpair) <= 128 ? 4 : 2, sub_rows, wpair, s, plan, ws.seed_rows, ws.seed_norm, kind, seed_of, sim, ws.grp,
             ws.mass_fx, ws.njoin, L.max_m, prm.tau, prm.eps, ws.err);
     }
     return cudaGetLastError();

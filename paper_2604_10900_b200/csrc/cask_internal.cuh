@@ -39,6 +39,7 @@ struct Shape {
     const int32_t* bt;   // device
     int32_t* err;        // device flag word (CASK_ST_TIMEOUT, CASK_ST_BOUNDS)
     const float* mass_in;   // device, optional [sumT]: group mass a row already carries
+    const float* chan_w;    // device, optional [d]: channel weights of the merge similarity
 };
 
 // Kernel ids for the optional per-kernel event timing.

@@ -57,20 +57,29 @@ __global__ void seed_gather_kernel(const UnitDesc* __restrict__ desc, Shape sh, 
                                    const float* __restrict__ s, const int32_t* __restrict__ plan,
                                    const int32_t* __restrict__ seed_rows, T* __restrict__ seed_k,
                                    float* __restrict__ seed_norm, unsigned long long* __restrict__ mass_fx,
-                                   int max_m, float eps) {
+                                   int max_m, float eps, int split_rows) {
     const int u = blockIdx.y, j = blockIdx.x;
     const UnitDesc& ud = desc[u];
     const int m = max(0, min(plan[u * 8 + CASK_PLAN_M], ud.plan[CASK_PLAN_M]));
     if (j >= m) return;
     const int row = seed_rows[ud.seed_base + j];
     const T* src = K + row_elem_off(sh, ud, ud.k_off, row);
-    T* dst = seed_k + (size_t)(ud.seed_base + j) * sh.d;
+    // Plain copy, or (channel-weighted similarity on the tensor cores) the weighted key w*k as two rows
+    // hi + lo of the cache dtype, so that the bf16 contraction sees w*k to about 2^-17.
+    T* dst = seed_k + (size_t)(ud.seed_base + j) * (split_rows ? 2 : 1) * sh.d;
     float n2 = 0.f;
     for (int c = threadIdx.x; c < sh.d; c += 32) {
         T x = src[c];
-        dst[c] = x;
         float f = Elem<T>::ld(&x);
-        n2 = fmaf(f, f, n2);
+        const float wc = sh.chan_w ? sh.chan_w[c] : 1.f;
+        if (split_rows) {
+            const float wf = wc * f;
+            Elem<T>::st(dst + c, wf);
+            Elem<T>::st(dst + sh.d + c, wf - Elem<T>::ld(dst + c));
+        } else {
+            dst[c] = x;
+        }
+        n2 = fmaf(wc * f, f, n2);
     }
 #pragma unroll
     for (int off = 16; off >= 1; off >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, off);
@@ -119,7 +128,7 @@ __global__ void __launch_bounds__(kThreads) assign_simt_kernel(
         // 4 threads per row, fixed combination order
         int rr = threadIdx.x / 4, part = threadIdx.x % 4;
         float n2 = 0.f;
-        for (int c = part; c < d; c += 4) n2 = fmaf(St[rr * pitch + c], St[rr * pitch + c], n2);
+        for (int c = part; c < d; c += 4) n2 = fmaf((sh.chan_w ? sh.chan_w[c] : 1.f) * St[rr * pitch + c], St[rr * pitch + c], n2);
         n2 += __shfl_xor_sync(0xffffffffu, n2, 1);
         n2 += __shfl_xor_sync(0xffffffffu, n2, 2);
         if (part == 0) rnorm[rr] = sqrtf(n2);
@@ -138,7 +147,9 @@ __global__ void __launch_bounds__(kThreads) assign_simt_kernel(
 #pragma unroll
             for (int t = 0; t < 8; ++t)
                 Rt[rr * pitch + c8 + t] =
-                    (rr < nseed) ? Elem<T>::ld(seed_k + (size_t)(ud.seed_base + u0 + rr) * d + c8 + t) : 0.f;
+                    (rr < nseed) ? (sh.chan_w ? sh.chan_w[c8 + t] : 1.f) *
+                                       Elem<T>::ld(seed_k + (size_t)(ud.seed_base + u0 + rr) * d + c8 + t)
+                                 : 0.f;
         }
         __syncthreads();
         float acc[4][4];
@@ -234,14 +245,15 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const i
         seeds_kernel<<<sh.n_units, kSelThreads, 0, L.stream>>>(L.desc, s, plan, kind, seed_of, weight, sim,
                                                                ws.grp, ws.seed_rows, ws.mass_fx, ws.njoin, max_m);
     }
+    const bool use_tc = !L.force_simt && L.tmap_encode && assign_tc_supported(L);
     if (max_m > 0) {
         {
             Timed t(L, KID_SEED_GATHER);
             seed_gather_kernel<T><<<dim3(max_m, sh.n_units), 32, 0, L.stream>>>(
                 L.desc, sh, (const T*)L.k, s, plan, ws.seed_rows, (T*)ws.seed_k, ws.seed_norm, ws.mass_fx, max_m,
-                prm.eps);
+                prm.eps, (use_tc && sh.chan_w) ? 1 : 0);
         }
-        if (!L.force_simt && L.tmap_encode && assign_tc_supported(L)) {
+        if (use_tc) {
             cudaError_t e = launch_assign_tc(L, prm, s, plan, kind, seed_of, sim, ws, L.tmap_encode);
             if (e != cudaSuccess) return e;
         } else {

@@ -26,7 +26,7 @@ WEIGHT_RTOL = 2e-5
 
 
 def run_oracle(hb: wl.Batch, **kw) -> Dict:
-    """kw: tau, gamma, causal, eps, mass_in (per-row carried masses)."""
+    """kw: tau, gamma, causal, eps, mass_in (per-row carried masses), chan_w (similarity channel weights)."""
     w = hb.wl
     return orc.event_batch(wl.as_float32(hb.k, w.dtype), wl.as_float32(hb.v, w.dtype),
                            wl.as_float32(hb.q, w.dtype), hb.tok_off, hb.P, hb.B, hb.reserve, **kw)
@@ -36,7 +36,7 @@ class GpuRun:
     """Device copies of a host batch plus everything needed to call the library on it."""
 
     def __init__(self, hb: wl.Batch, device="cuda:0", row_stride=None, lse_in=None, page_size=0, bad_page=None,
-                 mass_in=None, **prm_kw):
+                 mass_in=None, chan_w=None, **prm_kw):
         import torch
         from paper_2604_10900_b200 import binding as cb
         self.cb, self.torch, self.hb = cb, torch, hb
@@ -78,10 +78,11 @@ class GpuRun:
             paged = dict(page_size=ps, block_table=self.block_table, bt_off=bt_off, n_pages=n_pages)
             k_off = None
         self.mass_in = None if mass_in is None else torch.from_numpy(np.ascontiguousarray(mass_in, np.float32)).to(device)
+        self.chan_w = None if chan_w is None else torch.from_numpy(np.ascontiguousarray(chan_w, np.float32)).to(device)
         self.lse_in = None if lse_in is None else torch.from_numpy(np.ascontiguousarray(lse_in, np.float32)).to(device)
         self.batch, self._keep = cb.make_batch(
             self.dev["k"], self.dev["v"], self.dev["q"], hb.T, hb.P, hb.B, hb.reserve, hb.tok_off, d, w.group,
-            w.window, w.dtype, k_off=k_off, row_stride=row_stride, lse_in=self.lse_in, mass_in=self.mass_in, **paged)
+            w.window, w.dtype, k_off=k_off, row_stride=row_stride, lse_in=self.lse_in, mass_in=self.mass_in, chan_w=self.chan_w, **paged)
         self.prm = cb.params(**prm_kw)
         self.ctx = cb.Context(torch.device(device).index or 0, torch.cuda.current_stream(device).cuda_stream)
         self.ws, self.ws_bytes = cb.alloc_workspace(self.batch, self.prm, device)

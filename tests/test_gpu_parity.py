@@ -97,6 +97,27 @@ def test_carried_mass_second_event_on_a_compacted_cache():
     assert np.array_equal(g3["kind"], g2["kind"]) and not np.array_equal(g3["weight"], g2["weight"])
 
 
+@pytest.mark.parametrize("name,kw,tensor_assign", [
+    ("reasoning32k_b512", dict(layers=1, kv_heads=2, decode=4096 + 77), True),      # m = 64: hi/lo seed columns
+    ("reasoning32k_b1024", dict(layers=1, kv_heads=2, decode=4096 + 77), False),    # m = 192: SIMT assignment
+    ("tiny", dict(), False)])
+def test_channel_weighted_similarity(name, kw, tensor_assign):
+    """Sec. 2.5: per-channel (frequency band) weights in the merge similarity."""
+    import gpu_harness as gh
+    w = _small(name, **kw)
+    hb = wl.make_batch(w)
+    rng = np.random.default_rng(5)
+    cw = (rng.random(w.head_dim) ** 2 + 0.02).astype(np.float32)
+    cw[rng.random(w.head_dim) < 0.1] = 0.0                      # bands of no future relevance
+    run = gh.GpuRun(hb, chan_w=cw)
+    g = run.event()
+    o = gh.run_oracle(hb, chan_w=cw)
+    st = gh.compare_event(hb, g, o)
+    assert st["cascaded"] <= 1 and st["merged_elems"] > 0
+    plain = gh.run_oracle(hb)
+    assert not np.array_equal(plain["sim"], o["sim"])
+
+
 def test_prompt_heavy_two_stage():
     """Config-4 shape: prefix eviction fires before decode consolidation."""
     w = _small("prompt_heavy", layers=1, kv_heads=2, prefix=3072, decode=1024, budget=1024, reserve=256)
