@@ -269,6 +269,18 @@ int cask_compress_event(cask_ctx* ctx, const cask_batch* batch, const cask_param
                         const cask_outputs* out, void* ws, size_t ws_bytes);
 
 /*
+ * Paged cache only: writes the compacted rows back into each unit's own pages (Sec. 2.3: the
+ * cache is replaced by its representative set R), slot t of `out` at logical row t, i.e. into
+ * the unit's first ceil(n_out/page_size) pages; the other pages of the unit are left as they
+ * are and can be returned to the pool by the caller, the block table is not changed.  Call it
+ * after the event on the same context (it is ordered on the context's stream); k_pool / v_pool
+ * are the pools batch->k / batch->v point to, passed again as writable DEVICE pointers.  Uses
+ * out->k_out, v_out, n_out, Bmax.  A contiguous batch is refused with CASK_ERR_SHAPE.
+ */
+int cask_writeback_paged(cask_ctx* ctx, const cask_batch* batch, const cask_params* params,
+                         const cask_outputs* out, void* k_pool, void* v_pool, void* ws, size_t ws_bytes);
+
+/*
  * The same event for callers whose cache lives in HOST memory (ideally
  * page-locked): batch->k, v, q, lse_in and every pointer in `out` are HOST
  * pointers here.  dev_buf is a DEVICE buffer of at least

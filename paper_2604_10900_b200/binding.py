@@ -31,7 +31,7 @@ EXPORTS = (
     "cask_launch_count", "cask_last_score_path_tensor", "cask_last_device_flags", "cask_profile_enable", "cask_profile_read",
     "cask_kernel_count", "cask_kernel_name", "cask_workspace_bytes", "cask_plan_host",
     "cask_score", "cask_prefix_evict", "cask_select_core", "cask_consolidate_scratch", "cask_compact",
-    "cask_compress_event", "cask_host_event_device_bytes", "cask_compress_event_host", "cask_score_noalloc",
+    "cask_compress_event", "cask_writeback_paged", "cask_host_event_device_bytes", "cask_compress_event_host", "cask_score_noalloc",
 )
 
 
@@ -103,6 +103,7 @@ def lib():
         L.cask_consolidate_scratch.argtypes = [vp, PB, PP, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz]
         L.cask_compact.argtypes = [vp, PB, PP, vp, vp, vp, vp, PO, vp, sz]
         L.cask_compress_event.argtypes = [vp, PB, PP, PO, vp, sz]
+        L.cask_writeback_paged.argtypes = [vp, PB, PP, PO, vp, vp, vp, sz]
         L.cask_host_event_device_bytes.argtypes = [PB, PP, C.c_int32]
         L.cask_host_event_device_bytes.restype = sz
         L.cask_compress_event_host.argtypes = [vp, PB, PP, PO, vp, sz]
@@ -302,6 +303,14 @@ def cask_compact(ctx, batch, prm, s, kind, seed_of, weight, out: CaskOutputs, ws
 
 def cask_compress_event(ctx, batch, prm, out: CaskOutputs, ws, ws_bytes: int, check: bool = True) -> int:
     rc = lib().cask_compress_event(ctx.handle, C.byref(batch), C.byref(prm), C.byref(out), _ptr(ws), ws_bytes)
+    if check:
+        _check(rc, ctx)
+    return rc
+
+
+def cask_writeback_paged(ctx, batch, prm, out: CaskOutputs, k_pool, v_pool, ws, ws_bytes: int, check: bool = True) -> int:
+    rc = lib().cask_writeback_paged(ctx.handle, C.byref(batch), C.byref(prm), C.byref(out), _ptr(k_pool), _ptr(v_pool),
+                                    _ptr(ws), ws_bytes)
     if check:
         _check(rc, ctx)
     return rc

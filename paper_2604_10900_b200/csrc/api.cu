@@ -523,6 +523,21 @@ int cask_compress_event(cask_ctx* ctx, const cask_batch* b, const cask_params* p
     return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
 }
 
+int cask_writeback_paged(cask_ctx* ctx, const cask_batch* b, const cask_params* p, const cask_outputs* out,
+                         void* k_pool, void* v_pool, void* ws, size_t ws_bytes) {
+    if (!out || !k_pool || !v_pool) return CASK_ERR_NULL;
+    if (!out->k_out || !out->v_out || !out->n_out) return CASK_ERR_NULL;
+    if (b && b->page_size <= 0) return CASK_ERR_SHAPE;
+    if (((uintptr_t)k_pool | (uintptr_t)v_pool | (uintptr_t)out->k_out | (uintptr_t)out->v_out) % 16) return CASK_ERR_ALIGN;
+    if (out->Bmax < max_budget(b)) return CASK_ERR_SHAPE;
+    Launch L{};
+    Workspace W{};
+    int rc = prepare(ctx, b, p, ws, ws_bytes, L, W);
+    if (rc != CASK_OK || b->n_units == 0) return rc;
+    cudaError_t e = launch_writeback(L, *out, k_pool, v_pool);
+    return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
+}
+
 // ---- host-resident caches ------------------------------------------------------------------
 
 namespace {

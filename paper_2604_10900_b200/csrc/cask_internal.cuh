@@ -125,6 +125,8 @@ cudaError_t launch_consolidate(const Launch& L, const cask_params& prm, const fl
                                float* sim, int32_t* unit_status, float* lost_mass, Workspace& ws);
 cudaError_t launch_compact(const Launch& L, const cask_params& prm, const float* s, const uint8_t* kind,
                            const int32_t* seed_of, float* weight, const cask_outputs& out, Workspace& ws);
+// Paged cache: copies the compacted rows into the unit's own pages (slot t -> logical row t).
+cudaError_t launch_writeback(const Launch& L, const cask_outputs& out, void* k_pool, void* v_pool);
 // rho_core / rho_rep of Sec. 2.6 per unit (either pointer may be NULL).
 cudaError_t launch_diagnostics(const Launch& L, const float* s, const uint8_t* kind, const cask_outputs& out);
 

@@ -182,6 +182,28 @@ __global__ void __launch_bounds__(256) slot_merge_kernel(
     }
 }
 
+// ---- 4. paged cache: the compacted rows go back into the unit's own pages, slot t at logical row t ----
+template <typename T>
+__global__ void __launch_bounds__(256) writeback_kernel(const UnitDesc* __restrict__ desc, Shape sh, int Bmax,
+                                                        const int32_t* __restrict__ n_out, const T* __restrict__ k_out,
+                                                        const T* __restrict__ v_out, T* __restrict__ k_pool,
+                                                        T* __restrict__ v_pool) {
+    const int u = blockIdx.y;
+    const UnitDesc& ud = desc[u];
+    const int lane = threadIdx.x & 31;
+    const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (t >= n_out[u] || t >= ud.T) return;
+    const int d = sh.d, nvec = d * (int)sizeof(T) / 16;
+    const int64_t dst = paged_row(sh, ud, t) * sh.row_stride;
+    const T* ks = k_out + ((size_t)u * Bmax + t) * d;
+    const T* vs = v_out + ((size_t)u * Bmax + t) * d;
+    for (int x = lane; x < 2 * nvec; x += 32) {
+        const bool isv = x >= nvec;
+        const int c = isv ? x - nvec : x;
+        reinterpret_cast<uint4*>((isv ? v_pool : k_pool) + dst)[c] = reinterpret_cast<const uint4*>(isv ? vs : ks)[c];
+    }
+}
+
 template <typename T>
 cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const uint8_t* kind,
                 const int32_t* seed_of, float* weight, const cask_outputs& out, Workspace& ws) {
@@ -210,6 +232,21 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const u
 }
 
 }  // namespace
+
+cudaError_t launch_writeback(const Launch& L, const cask_outputs& out, void* k_pool, void* v_pool) {
+    const Shape& sh = L.sh;
+    const int slots = min(out.Bmax, max(L.max_B, 1));
+    const dim3 grid((slots + 7) / 8, sh.n_units);
+    Timed t(L, KID_GATHER_MERGE);
+    if (sh.dtype == CASK_DTYPE_BF16)
+        writeback_kernel<__nv_bfloat16><<<grid, 256, 0, L.stream>>>(L.desc, sh, out.Bmax, out.n_out,
+                                                                   (const __nv_bfloat16*)out.k_out, (const __nv_bfloat16*)out.v_out,
+                                                                   (__nv_bfloat16*)k_pool, (__nv_bfloat16*)v_pool);
+    else
+        writeback_kernel<float><<<grid, 256, 0, L.stream>>>(L.desc, sh, out.Bmax, out.n_out, (const float*)out.k_out,
+                                                            (const float*)out.v_out, (float*)k_pool, (float*)v_pool);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_compact(const Launch& L, const cask_params& prm, const float* s, const uint8_t* kind,
                            const int32_t* seed_of, float* weight, const cask_outputs& out, Workspace& ws) {

@@ -58,3 +58,39 @@ def test_page_id_outside_the_pool_is_flagged_not_followed(page_size):
     assert run.ctx.device_flags() & ST_BOUNDS
     assert (g["unit_status"] & ST_BOUNDS).all()
     assert (g["n_out"] == 512).all()
+
+
+@pytest.mark.parametrize("page_size", [16, 48])
+def test_writeback_puts_the_compacted_rows_into_the_units_own_pages(page_size):
+    """After cask_writeback_paged, logical row t of a unit (read through its block table) is slot t of the
+    compacted cache, bit for bit; rows beyond n_out and the pool's spare pages are untouched."""
+    import torch
+    w = wl.WORKLOADS["reasoning32k_b512"].with_(layers=1, kv_heads=2, prefix=500, decode=1024 + 5)
+    hb = wl.make_batch(w)
+    run, g = _event(hb, page_size=page_size)
+    cb = run.cb
+    before = {n: run.dev[n].clone() for n in ("k", "v")}
+    cb.cask_writeback_paged(run.ctx, run.batch, run.prm, run.out_struct, run.dev["k"], run.dev["v"], run.ws, run.ws_bytes)
+    torch.cuda.synchronize()
+    assert run.ctx.device_flags() == 0
+    table = run.block_table.cpu().numpy().astype(np.int64)
+    ps = page_size
+    touched = np.zeros(run.dev["k"].shape[0], bool)
+    off = 0
+    for u in range(hb.n_units):
+        n = int(g["n_out"][u])
+        t = np.arange(n)
+        rows = table[off + t // ps] * ps + t % ps
+        touched[rows] = True
+        for name in ("k", "v"):
+            got = run.dev[name][torch.from_numpy(rows).to(run.device)].view(torch.uint16).cpu().numpy()
+            want = run.out[name + "_out"][u, :n].view(torch.uint16).cpu().numpy()
+            assert np.array_equal(got, want), (u, name)
+        off += (int(hb.T[u]) + ps - 1) // ps
+    keep = torch.from_numpy(~touched).to(run.device)
+    for name in ("k", "v"):
+        assert torch.equal(run.dev[name][keep].view(torch.uint16), before[name][keep].view(torch.uint16))
+    # a contiguous batch is refused
+    run_c, _ = _event(hb)
+    assert cb.cask_writeback_paged(run_c.ctx, run_c.batch, run_c.prm, run_c.out_struct, run_c.dev["k"], run_c.dev["v"],
+                                   run_c.ws, run_c.ws_bytes, check=False) == cb.ERR_SHAPE
