@@ -85,6 +85,34 @@ struct TileWalk {
 // first seed among equals.  PAIR = 1: a seed owns two adjacent columns (the hi and lo parts of its weighted key)
 // whose sum is its dot product.  A block of 32 columns costs a multiply and a maximum per seed; the position of
 // the maximum is looked for only in a block that beats everything before it.
+// Squared (channel-weighted) norm of one staged key row as a packed pair of partial sums.  The row's sixteen
+// 16-byte pieces are read in a lane-dependent order (no bank conflicts); a bf16 is the upper half of an fp32, so
+// two integer operations unpack a pair.  The 128-byte swizzle stores logical piece p of row r at position
+// p ^ (r & 7), which matters only for finding the piece's channel weights.
+template <bool WEIGHTED>
+__device__ __forceinline__ uint64_t row_norm2(const uint8_t* base, int lane, int row, const float* w) {
+    uint64_t n2p = 0ull;
+#pragma unroll
+    for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const int pos = (c + lane) & 7;
+            const uint4 raw = *reinterpret_cast<const uint4*>(base + kb * kKRegionBytes + (pos << 4));
+            const uint32_t wv[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                const uint64_t f2 = pack2(__uint_as_float(wv[x] << 16), __uint_as_float(wv[x] & 0xFFFF0000u));
+                if (WEIGHTED) {
+                    const float2 w2 = *reinterpret_cast<const float2*>(&w[kb * 64 + ((pos ^ (row & 7)) << 3) + 2 * x]);
+                    n2p = fma2(fma2(f2, pack2(w2.x, w2.y), 0ull), f2, n2p);
+                } else {
+                    n2p = fma2(f2, f2, n2p);
+                }
+            }
+        }
+    return n2p;
+}
+
 template <int PAIR>
 __device__ __forceinline__ void best_seed(uint32_t taddr, const float* inv, int c_lo, int c_hi, float& best, int& best_u) {
     constexpr int kPer = PAIR ? 16 : 32;          // seeds per block of 32 columns
@@ -94,12 +122,19 @@ __device__ __forceinline__ void best_seed(uint32_t taddr, const float* inv, int 
         tc_wait_ld_regs(v);
         const int u0 = PAIR ? cc >> 1 : cc, u_hi = PAIR ? c_hi >> 1 : c_hi;
         float bm = -INFINITY;
-        const bool whole = cc + 32 <= c_hi;
+        if (cc + 32 <= c_hi) {
 #pragma unroll
-        for (int x = 0; x < kPer; ++x) {
-            const float dot = PAIR ? v[2 * x] + v[2 * x + 1] : v[x];
-            v[x] = (whole || u0 + x < u_hi) ? dot * inv[u0 + x] : -INFINITY;
-            bm = fmaxf(bm, v[x]);
+            for (int x = 0; x < kPer; ++x) {
+                v[x] = (PAIR ? v[2 * x] + v[2 * x + 1] : v[x]) * inv[u0 + x];
+                bm = fmaxf(bm, v[x]);
+            }
+        } else {
+#pragma unroll
+            for (int x = 0; x < kPer; ++x) {
+                const float dot = PAIR ? v[2 * x] + v[2 * x + 1] : v[x];
+                v[x] = (u0 + x < u_hi) ? dot * inv[u0 + x] : -INFINITY;
+                bm = fmaxf(bm, v[x]);
+            }
         }
         if (bm > best) {
             best = bm;
@@ -309,26 +344,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 uint64_t n2p = 0ull;
                 {
                     const uint8_t* base = k_smem + st * kKStageBytes + my_row * 128;
-#pragma unroll
-                    for (int kb = 0; kb < 2; ++kb)
-#pragma unroll
-                        for (int c = 0; c < 8; ++c) {
-                            const uint4 raw = *reinterpret_cast<const uint4*>(base + kb * kKRegionBytes + (((c + lane) & 7) << 4));
-                            // a bf16 is the upper half of an fp32: two integer operations unpack a pair
-                            const uint32_t wv[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-                            for (int x = 0; x < 4; ++x) {
-                                const uint64_t f2 = pack2(__uint_as_float(wv[x] << 16), __uint_as_float(wv[x] & 0xFFFF0000u));
-                                if (sh.chan_w) {
-                                    // the 128-byte swizzle stores logical 16-byte piece p of row r at position p ^ (r & 7)
-                                    const float2 w2 = *reinterpret_cast<const float2*>(
-                                        &tail->w[kb * 64 + ((((c + lane) & 7) ^ (my_row & 7)) << 3) + 2 * x]);
-                                    n2p = fma2(fma2(f2, pack2(w2.x, w2.y), 0ull), f2, n2p);
-                                } else {
-                                    n2p = fma2(f2, f2, n2p);
-                                }
-                            }
-                        }
+                    if (!sh.chan_w) n2p = row_norm2<false>(base, lane, my_row, tail->w);
+                    else n2p = row_norm2<true>(base, lane, my_row, tail->w);
                 }
                 float n2, n2b;
                 unpack2(n2p, n2, n2b);
