@@ -8,6 +8,7 @@ namespace cask {
 namespace {
 
 constexpr int kScanThreads = 1024;
+constexpr int kScanMaxIters = 63;      // rows per unit below 64,512: the one-scan path of slot_scan_kernel
 
 // ---- 1. per-unit ordered scan: slots, index map, member list -------------------------------
 __global__ void __launch_bounds__(kScanThreads) slot_scan_kernel(
@@ -17,6 +18,7 @@ __global__ void __launch_bounds__(kScanThreads) slot_scan_kernel(
     int32_t* __restrict__ mem_row, int32_t* __restrict__ mem_slot, int32_t* __restrict__ n_mem,
     int32_t* __restrict__ seed_slot, int32_t* __restrict__ n_seed, int max_B) {
     __shared__ unsigned wk[kScanThreads / 32], wm[kScanThreads / 32];
+    __shared__ unsigned cell[kScanMaxIters * (kScanThreads / 32)];
     __shared__ int seeds_listed;
     if (threadIdx.x == 0) seeds_listed = 0;
     const int u = blockIdx.x;
@@ -25,40 +27,113 @@ __global__ void __launch_bounds__(kScanThreads) slot_scan_kernel(
     const int64_t o = ud.tok_off;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
     unsigned base_k = 0, base_m = 0;
-    for (int i0 = 0; i0 < T; i0 += blockDim.x) {
-        const int i = i0 + threadIdx.x;
-        const uint8_t kd = (i < T) ? kind[o + i] : (uint8_t)0;
-        const bool keep = kd >= CASK_KIND_PREFIX && kd <= CASK_KIND_SEED;
-        const bool mem = kd == CASK_KIND_SEED || kd == CASK_KIND_MERGED;
-        const unsigned bk = __ballot_sync(0xffffffffu, keep), bm = __ballot_sync(0xffffffffu, mem);
-        __syncthreads();
-        if (lane == 0) { wk[w] = __popc(bk); wm[w] = __popc(bm); }
-        __syncthreads();
-        unsigned pk = 0, pm = 0, ak = 0, am = 0;
-        for (int x = 0; x < nw; ++x) {
-            if (x < w) { pk += wk[x]; pm += wm[x]; }
-            ak += wk[x];
-            am += wm[x];
+    const int iters = (T + (int)blockDim.x - 1) / (int)blockDim.x;
+    if (iters <= kScanMaxIters) {
+        // Two coalesced sweeps around one scan: per (iteration, warp) cell the number of kept rows and of group
+        // members, an exclusive scan over the cells in row order, then every row finds its slot from its cell's
+        // base and the lower lanes of its warp.
+        const int cells = iters * nw;
+        for (int it = 0; it < iters; ++it) {
+            const int i = it * blockDim.x + threadIdx.x;
+            const uint8_t kd = (i < T) ? kind[o + i] : (uint8_t)0;
+            const bool keep = kd >= CASK_KIND_PREFIX && kd <= CASK_KIND_SEED;
+            const bool mem = kd == CASK_KIND_SEED || kd == CASK_KIND_MERGED;
+            const unsigned bk = __ballot_sync(0xffffffffu, keep), bm = __ballot_sync(0xffffffffu, mem);
+            if (lane == 0) cell[it * nw + w] = (unsigned)__popc(bk) | ((unsigned)__popc(bm) << 16);
         }
-        const unsigned below = (1u << lane) - 1u;
-        if (i < T) {
-            int slot = -1;
-            if (keep) {
-                slot = (int)(base_k + pk + __popc(bk & below));
-                if (slot < Bmax) {
-                    slot_src[(size_t)u * Bmax + slot] = i;
-                    slot_kind[(size_t)u * Bmax + slot] = kd;
-                } else {
-                    slot = -1;        // more kept rows than slots: cannot happen for a valid plan
-                }
+        __syncthreads();
+        // exclusive scan of the packed (kept, member) counts; a cell holds at most 32 of each and a unit fewer
+        // than 65,536 kept rows and members in this path, so the halves never carry into each other
+        {
+            const int per = (cells + (int)blockDim.x - 1) / (int)blockDim.x;
+            const int c0 = threadIdx.x * per, c1 = min(cells, c0 + per);
+            unsigned sum = 0;
+            for (int c = c0; c < c1; ++c) sum += cell[c];
+            // block exclusive scan of `sum`
+            unsigned incl = sum;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                unsigned v = __shfl_up_sync(0xffffffffu, incl, off);
+                if (lane >= off) incl += v;
             }
-            assign[o + i] = slot;
-            if (mem) mem_row[o + base_m + pm + __popc(bm & below)] = i;
-            if (kd >= CASK_KIND_PREFIX && kd <= CASK_KIND_CORE) weight[o + i] = 1.f;
-            if (kd == CASK_KIND_DROPPED) weight[o + i] = 0.f;
+            if (lane == 31) wk[w] = incl;
+            __syncthreads();
+            unsigned wbase = 0;
+            for (int x = 0; x < w; ++x) wbase += wk[x];
+            unsigned run = wbase + incl - sum;
+            unsigned total = 0;
+            for (int x = 0; x < nw; ++x) total += wk[x];
+            __syncthreads();
+            for (int c = c0; c < c1; ++c) {
+                const unsigned v = cell[c];
+                cell[c] = run;
+                run += v;
+            }
+            base_k = total & 0xFFFFu;
+            base_m = total >> 16;
         }
-        base_k += ak;
-        base_m += am;
+        __syncthreads();
+        for (int it = 0; it < iters; ++it) {
+            const int i = it * blockDim.x + threadIdx.x;
+            const uint8_t kd = (i < T) ? kind[o + i] : (uint8_t)0;
+            const bool keep = kd >= CASK_KIND_PREFIX && kd <= CASK_KIND_SEED;
+            const bool mem = kd == CASK_KIND_SEED || kd == CASK_KIND_MERGED;
+            const unsigned bk = __ballot_sync(0xffffffffu, keep), bm = __ballot_sync(0xffffffffu, mem);
+            const unsigned cb = cell[it * nw + w];
+            const unsigned below = (1u << lane) - 1u;
+            if (i < T) {
+                int slot = -1;
+                if (keep) {
+                    slot = (int)((cb & 0xFFFFu) + __popc(bk & below));
+                    if (slot < Bmax) {
+                        slot_src[(size_t)u * Bmax + slot] = i;
+                        slot_kind[(size_t)u * Bmax + slot] = kd;
+                    } else {
+                        slot = -1;        // more kept rows than slots: cannot happen for a valid plan
+                    }
+                }
+                assign[o + i] = slot;
+                if (mem) mem_row[o + (cb >> 16) + __popc(bm & below)] = i;
+                if (kd >= CASK_KIND_PREFIX && kd <= CASK_KIND_CORE) weight[o + i] = 1.f;
+                if (kd == CASK_KIND_DROPPED) weight[o + i] = 0.f;
+            }
+        }
+    } else {
+    for (int i0 = 0; i0 < T; i0 += blockDim.x) {
+            const int i = i0 + threadIdx.x;
+            const uint8_t kd = (i < T) ? kind[o + i] : (uint8_t)0;
+            const bool keep = kd >= CASK_KIND_PREFIX && kd <= CASK_KIND_SEED;
+            const bool mem = kd == CASK_KIND_SEED || kd == CASK_KIND_MERGED;
+            const unsigned bk = __ballot_sync(0xffffffffu, keep), bm = __ballot_sync(0xffffffffu, mem);
+            __syncthreads();
+            if (lane == 0) { wk[w] = __popc(bk); wm[w] = __popc(bm); }
+            __syncthreads();
+            unsigned pk = 0, pm = 0, ak = 0, am = 0;
+            for (int x = 0; x < nw; ++x) {
+                if (x < w) { pk += wk[x]; pm += wm[x]; }
+                ak += wk[x];
+                am += wm[x];
+            }
+            const unsigned below = (1u << lane) - 1u;
+            if (i < T) {
+                int slot = -1;
+                if (keep) {
+                    slot = (int)(base_k + pk + __popc(bk & below));
+                    if (slot < Bmax) {
+                        slot_src[(size_t)u * Bmax + slot] = i;
+                        slot_kind[(size_t)u * Bmax + slot] = kd;
+                    } else {
+                        slot = -1;        // more kept rows than slots: cannot happen for a valid plan
+                    }
+                }
+                assign[o + i] = slot;
+                if (mem) mem_row[o + base_m + pm + __popc(bm & below)] = i;
+                if (kd >= CASK_KIND_PREFIX && kd <= CASK_KIND_CORE) weight[o + i] = 1.f;
+                if (kd == CASK_KIND_DROPPED) weight[o + i] = 0.f;
+            }
+            base_k += ak;
+            base_m += am;
+        }
     }
     const int nk = min((int)base_k, Bmax), nm = (int)base_m;
     if (threadIdx.x == 0) { n_out[u] = nk; n_mem[u] = nm; }
