@@ -118,6 +118,18 @@ def test_channel_weighted_similarity(name, kw, tensor_assign):
     assert not np.array_equal(plain["sim"], o["sim"])
 
 
+@pytest.mark.parametrize("group,window", [(1, 32), (3, 32), (1, 128), (2, 128), (3, 128), (5, 96)])
+def test_query_row_counts_that_fill_one_to_four_accumulator_slots(group, window):
+    """32 to 480 window-query rows: one, two, three and four 128-column slots, a ragged last slot, idle epilogue
+    groups and warps (tensor-core scoring throughout)."""
+    w = _small("reasoning32k_b512", layers=1, kv_heads=2, group=group, window=window, decode=2048 + 61, prefix=300,
+               budget=512, reserve=256)
+    hb, run, g, o, st = _run(w)
+    assert run.ctx.used_tensor_path and run.ctx.device_flags() == 0
+    assert st["max_score_rel"] < 1e-5 and st["cascaded"] <= 1
+    assert (g["n_out"] == 512).all()
+
+
 def test_prompt_heavy_two_stage():
     """Config-4 shape: prefix eviction fires before decode consolidation."""
     w = _small("prompt_heavy", layers=1, kv_heads=2, prefix=3072, decode=1024, budget=1024, reserve=256)
