@@ -259,8 +259,10 @@ def run_ours(args):
               plan=np.zeros((hb.n_units, 8), np.int32), unit_status=np.zeros(hb.n_units, np.int32),
               lost_mass=np.zeros(hb.n_units, np.float32))
     ho_struct = cb.make_outputs(ho, Bmax)
-    h2d = hb.k.nbytes + hb.v.nbytes + hb.q.nbytes
-    d2h = sum(a.nbytes for a in ho.values())
+    # The host entry point sends the keys and queries whole but only the value rows that are kept or merged
+    # (counted from the row kinds of the device run); the row kinds come back once more in mid-call.
+    h2d = hb.k.nbytes + hb.q.nbytes + int(np.count_nonzero(kind)) * d * (2 if w.dtype == wl.DTYPE_BF16 else 4)
+    d2h = sum(a.nbytes for a in ho.values()) + sum_T
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
     cb.cask_compress_event_host(ctx, hbatch, prm, ho_struct, dev_buf, dev_bytes)   # warm-up
     barrier()

@@ -285,8 +285,11 @@ int cask_writeback_paged(cask_ctx* ctx, const cask_batch* batch, const cask_para
  * page-locked): batch->k, v, q, lse_in and every pointer in `out` are HOST
  * pointers here.  dev_buf is a DEVICE buffer of at least
  * cask_host_event_device_bytes() that holds the staged inputs, outputs and the
- * workspace.  Copies in, runs cask_compress_event, copies out and synchronises
- * the stream before returning.  Rows of a unit must be dense (row_stride ==
+ * workspace.  Copies the keys and queries in, decides every row's fate, copies
+ * in only the value rows that are kept or merged (gathered through a pinned
+ * staging buffer the context owns and grows as needed), compacts, copies out
+ * and synchronises the stream before returning; the results equal those of
+ * cask_compress_event.  Rows of a unit must be dense (row_stride ==
  * head_dim) and units laid out at k_off[u] == v_off[u] == tok_off[u]*head_dim;
  * a paged batch is refused with CASK_ERR_UNSUPPORTED.
  */

@@ -5,6 +5,7 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <thread>
 #include <vector>
 
 #include "cask_internal.cuh"
@@ -47,6 +48,9 @@ struct cask_ctx {
     cudaError_t last_err = cudaSuccess;
     int last_tc = 0;
     const int32_t* flags_dev = nullptr;   // flag word of the last call's workspace
+    // host-buffer entry point: pinned staging for the row kinds coming back and the packed value rows going in
+    char* hstage = nullptr;
+    size_t hstage_bytes = 0;
     void* tmap_encode = nullptr;     // cuTensorMapEncodeTiled, resolved at creation
     Profiler prof;
     ProfImpl prof_impl;
@@ -326,6 +330,7 @@ int cask_destroy(cask_ctx* ctx) {
     cudaSetDevice(ctx->device);
     if (ctx->staged_pending) cudaEventSynchronize(ctx->staged);
     if (ctx->pinned) cudaFreeHost(ctx->pinned);
+    if (ctx->hstage) cudaFreeHost(ctx->hstage);
     if (ctx->staged) cudaEventDestroy(ctx->staged);
     for (ProfRecord& r : ctx->prof_impl.live) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     for (cudaEvent_t e : ctx->prof_impl.pool) cudaEventDestroy(e);
@@ -500,6 +505,29 @@ int cask_compact(cask_ctx* ctx, const cask_batch* b, const cask_params* p, const
     return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
 }
 
+// The event up to the point where every row's fate is known (score, selections, group assignment, weights);
+// only keys are read.
+static int event_decide(cask_ctx* ctx, Launch& L, Workspace& W, const cask_batch* b, const cask_params* p,
+                        const cask_outputs* out) {
+    float* s = out->s ? out->s : W.s;
+    int rc = run_score(ctx, L, b, p, s, out->lse, W);
+    if (rc != CASK_OK) return rc;
+    cudaError_t e = launch_prefix_evict(L, s, out->kind, out->plan);
+    if (e == cudaSuccess) e = launch_select_core(L, s, out->plan, out->kind);
+    if (e == cudaSuccess)
+        e = launch_consolidate(L, *p, s, out->plan, out->kind, out->seed_of, out->weight, out->sim,
+                               out->unit_status, out->lost_mass, W);
+    return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
+}
+
+// The rest: compaction (the only step that reads values) and the optional diagnostics.
+static int event_compact(cask_ctx* ctx, Launch& L, Workspace& W, const cask_params* p, const cask_outputs* out) {
+    float* s = out->s ? out->s : W.s;
+    cudaError_t e = launch_compact(L, *p, s, out->kind, out->seed_of, out->weight, *out, W);
+    if (e == cudaSuccess) e = launch_diagnostics(L, s, out->kind, *out);
+    return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
+}
+
 int cask_compress_event(cask_ctx* ctx, const cask_batch* b, const cask_params* p, const cask_outputs* out,
                         void* ws, size_t ws_bytes) {
     int rc = check_compact_out(out, max_budget(b));
@@ -510,17 +538,9 @@ int cask_compress_event(cask_ctx* ctx, const cask_batch* b, const cask_params* p
     Workspace W{};
     rc = prepare(ctx, b, p, ws, ws_bytes, L, W);
     if (rc != CASK_OK || b->n_units == 0) return rc;
-    float* s = out->s ? out->s : W.s;
-    rc = run_score(ctx, L, b, p, s, out->lse, W);
+    rc = event_decide(ctx, L, W, b, p, out);
     if (rc != CASK_OK) return rc;
-    cudaError_t e = launch_prefix_evict(L, s, out->kind, out->plan);
-    if (e == cudaSuccess) e = launch_select_core(L, s, out->plan, out->kind);
-    if (e == cudaSuccess)
-        e = launch_consolidate(L, *p, s, out->plan, out->kind, out->seed_of, out->weight, out->sim,
-                               out->unit_status, out->lost_mass, W);
-    if (e == cudaSuccess) e = launch_compact(L, *p, s, out->kind, out->seed_of, out->weight, *out, W);
-    if (e == cudaSuccess) e = launch_diagnostics(L, s, out->kind, *out);
-    return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
+    return event_compact(ctx, L, W, p, out);
 }
 
 int cask_writeback_paged(cask_ctx* ctx, const cask_batch* b, const cask_params* p, const cask_outputs* out,
@@ -547,6 +567,8 @@ struct HostStage {
     char* ws;
     size_t ws_bytes, bytes;
     size_t kv_bytes, q_bytes, lse_bytes;
+    int32_t *v_pos, *n_need;
+    int64_t* v_base;
 };
 
 HostStage stage_layout(char* base, const cask_batch* b, const cask_params* p, int32_t Bmax) {
@@ -568,6 +590,9 @@ HostStage stage_layout(char* base, const cask_batch* b, const cask_params* p, in
     h.lse_in = take(h.lse_bytes);
     h.mass_in = take(sumT * 4);
     h.chan_w = take(d * 4);
+    h.v_pos = (int32_t*)take(sumT * 4);
+    h.n_need = (int32_t*)take(n * 4);
+    h.v_base = (int64_t*)take(n * 8);
     h.o.Bmax = Bmax;
     h.o.k_out = take(n * Bmax * d * e);
     h.o.v_out = take(n * Bmax * d * e);
@@ -622,8 +647,9 @@ int cask_compress_event_host(cask_ctx* ctx, const cask_batch* hb, const cask_par
     cudaError_t e = cudaSetDevice(ctx->device);
     if (e != cudaSuccess) return fail_cuda(ctx, e);
     cudaStream_t st = ctx->stream;
+    // Keys and queries go up whole.  Values do not: only the compaction reads them, and only the rows that are
+    // kept or merged, so they follow later, packed, once the rows' fates are known.
     e = cudaMemcpyAsync(h.k, hb->k, h.kv_bytes, cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(h.v, hb->v, h.kv_bytes, cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess) e = cudaMemcpyAsync(h.q, hb->q, h.q_bytes, cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess && hb->lse_in)
         e = cudaMemcpyAsync(h.lse_in, hb->lse_in, h.lse_bytes, cudaMemcpyHostToDevice, st);
@@ -639,11 +665,80 @@ int cask_compress_event_host(cask_ctx* ctx, const cask_batch* hb, const cask_par
     db.chan_w = hb->chan_w ? (const float*)h.chan_w : nullptr;
     db.k = h.k; db.v = h.v; db.q = h.q;
     db.lse_in = hb->lse_in ? (const float*)h.lse_in : nullptr;
-    rc = cask_compress_event(ctx, &db, p, &h.o, h.ws, h.ws_bytes);
-    if (rc != CASK_OK) return rc;
     const size_t es = elem_size(hb->dtype), n = (size_t)hb->n_units, d = (size_t)hb->head_dim;
     const size_t sumT = (size_t)hb->tok_off[hb->n_units], rows = (size_t)hb->group * hb->window;
     const size_t Bm = (size_t)ho->Bmax;
+    {
+        Launch L{};
+        Workspace W{};
+        rc = prepare(ctx, &db, p, h.ws, h.ws_bytes, L, W);
+        if (rc != CASK_OK) return rc;
+        rc = event_decide(ctx, L, W, &db, p, &h.o);
+        if (rc != CASK_OK) return rc;
+        e = launch_value_ranks(L, h.o.kind, h.v_pos, h.n_need, h.v_base);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+        // the row kinds come back; the rows with a kind other than 0 are the ones whose values are read
+        const size_t row_bytes = d * es;
+        if (ctx->hstage_bytes < sumT) {
+            if (ctx->hstage) cudaFreeHost(ctx->hstage);
+            ctx->hstage = nullptr;
+            ctx->hstage_bytes = 0;
+            e = cudaMallocHost((void**)&ctx->hstage, sumT + (sumT / 8 + 4096) * row_bytes);
+            if (e != cudaSuccess) return fail_cuda(ctx, e);
+            ctx->hstage_bytes = sumT + (sumT / 8 + 4096) * row_bytes;
+        }
+        uint8_t* hkind = (uint8_t*)ctx->hstage;
+        e = cudaMemcpyAsync(hkind, h.o.kind, sumT, cudaMemcpyDeviceToHost, st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+        std::vector<int64_t> vbase(n + 1, 0);
+        const unsigned nthr = std::max(1u, std::min(16u, std::thread::hardware_concurrency()));
+        auto over_units = [&](auto fn) {
+            std::vector<std::thread> th;
+            for (unsigned t = 0; t < nthr; ++t)
+                th.emplace_back([&, t] {
+                    for (size_t u = t; u < n; u += nthr) fn(u);
+                });
+            for (auto& x : th) x.join();
+        };
+        over_units([&](size_t u) {
+            const uint8_t* kd = hkind + hb->tok_off[u];
+            int64_t c = 0;
+            for (int i = 0; i < hb->T[u]; ++i) c += kd[i] != CASK_KIND_DROPPED;
+            vbase[u + 1] = c;
+        });
+        for (size_t u = 0; u < n; ++u) vbase[u + 1] += vbase[u];
+        const size_t need_rows = (size_t)vbase[n];
+        if (ctx->hstage_bytes < sumT + need_rows * row_bytes) {      // grow, keeping the kinds
+            char* bigger = nullptr;
+            const size_t nb = sumT + (need_rows + need_rows / 4 + 4096) * row_bytes;
+            e = cudaMallocHost((void**)&bigger, nb);
+            if (e != cudaSuccess) return fail_cuda(ctx, e);
+            memcpy(bigger, ctx->hstage, sumT);
+            cudaFreeHost(ctx->hstage);
+            ctx->hstage = bigger;
+            ctx->hstage_bytes = nb;
+            hkind = (uint8_t*)ctx->hstage;
+        }
+        char* hv = ctx->hstage + sumT;
+        over_units([&](size_t u) {
+            const uint8_t* kd = hkind + hb->tok_off[u];
+            const char* src = (const char*)hb->v + (size_t)hb->v_off[u] * es;
+            char* dst = hv + (size_t)vbase[u] * row_bytes;
+            for (int i = 0; i < hb->T[u]; ++i)
+                if (kd[i] != CASK_KIND_DROPPED) {
+                    memcpy(dst, src + (size_t)i * row_bytes, row_bytes);
+                    dst += row_bytes;
+                }
+        });
+        e = cudaMemcpyAsync(h.v, hv, need_rows * row_bytes, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+        L.v = h.v;
+        L.sh.v_pos = h.v_pos;
+        L.sh.v_base = h.v_base;
+        rc = event_compact(ctx, L, W, p, &h.o);
+        if (rc != CASK_OK) return rc;
+    }
     struct Cp { void* dst; const void* src; size_t bytes; };
     const Cp cps[] = {
         {ho->k_out, h.o.k_out, n * Bm * d * es}, {ho->v_out, h.o.v_out, n * Bm * d * es},

@@ -40,6 +40,11 @@ struct Shape {
     int32_t* err;        // device flag word (CASK_ST_TIMEOUT, CASK_ST_BOUNDS)
     const float* mass_in;   // device, optional [sumT]: group mass a row already carries
     const float* chan_w;    // device, optional [d]: channel weights of the merge similarity
+    // host-resident caches: only the value rows the compaction reads are on the device, packed unit after unit
+    // in ascending row order; v_pos[tok_off + i] is the position of row i inside its unit's run, v_base[u] the
+    // first packed row of unit u (both NULL when V is the full cache)
+    const int32_t* v_pos;
+    const int64_t* v_base;
 };
 
 // Kernel ids for the optional per-kernel event timing.
@@ -125,6 +130,9 @@ cudaError_t launch_consolidate(const Launch& L, const cask_params& prm, const fl
                                float* sim, int32_t* unit_status, float* lost_mass, Workspace& ws);
 cudaError_t launch_compact(const Launch& L, const cask_params& prm, const float* s, const uint8_t* kind,
                            const int32_t* seed_of, float* weight, const cask_outputs& out, Workspace& ws);
+// Host-resident caches: rank of every row among the rows of its unit whose values the compaction reads
+// (kind != 0), the number of such rows per unit and the exclusive prefix of those numbers.
+cudaError_t launch_value_ranks(const Launch& L, const uint8_t* kind, int32_t* v_pos, int32_t* n_need, int64_t* v_base);
 // Paged cache: copies the compacted rows into the unit's own pages (slot t -> logical row t).
 cudaError_t launch_writeback(const Launch& L, const cask_outputs& out, void* k_pool, void* v_pool);
 // rho_core / rho_rep of Sec. 2.6 per unit (either pointer may be NULL).
@@ -163,6 +171,11 @@ __device__ __forceinline__ float row_mass(const Shape& sh, const float* __restri
 __device__ __forceinline__ int64_t row_elem_off(const Shape& sh, const UnitDesc& ud, int64_t unit_off, int i) {
     if (sh.page_size == 0) return unit_off + (int64_t)i * sh.row_stride;
     return paged_row(sh, ud, i) * sh.row_stride;
+}
+// Element offset of the value row i of unit u.
+__device__ __forceinline__ int64_t v_elem_off(const Shape& sh, const UnitDesc& ud, int u, int i) {
+    if (sh.v_pos) return (sh.v_base[u] + sh.v_pos[ud.tok_off + i]) * (int64_t)sh.d;
+    return row_elem_off(sh, ud, ud.v_off, i);
 }
 
 template <typename T> struct Elem;

@@ -183,7 +183,7 @@ __global__ void __launch_bounds__(256) slot_copy_kernel(
     T* ko = k_out + ((size_t)u * Bmax + t) * d;
     T* vo = v_out + ((size_t)u * Bmax + t) * d;
     const T* ksrc = K + row_elem_off(sh, ud, ud.k_off, src);
-    const T* vsrc = V + row_elem_off(sh, ud, ud.v_off, src);
+    const T* vsrc = V + v_elem_off(sh, ud, u, src);
     const int nvec = d * (int)sizeof(T) / 16;
     for (int x = lane; x < 2 * nvec; x += 32) {
         const bool isv = x >= nvec;
@@ -231,7 +231,7 @@ __global__ void __launch_bounds__(256) slot_merge_kernel(
             msum += row_mass(sh, s, eps, o + i);
             ++count;
             const T* kr = K + row_elem_off(sh, ud, ud.k_off, i);
-            const T* vr = V + row_elem_off(sh, ud, ud.v_off, i);
+            const T* vr = V + v_elem_off(sh, ud, u, i);
 #pragma unroll
             for (int x = 0; x < kMaxPerLane; ++x) {
                 const int c = lane + 32 * x;
@@ -254,6 +254,53 @@ __global__ void __launch_bounds__(256) slot_merge_kernel(
             }
         }
         if (lane == 0) slot_mass[(size_t)u * Bmax + t] = msum;
+    }
+}
+
+// ---- host-resident caches: which value rows the compaction will read, and where they sit once packed ----
+__global__ void __launch_bounds__(kScanThreads) value_rank_kernel(const UnitDesc* __restrict__ desc,
+                                                                  const uint8_t* __restrict__ kind,
+                                                                  int32_t* __restrict__ v_pos,
+                                                                  int32_t* __restrict__ n_need) {
+    __shared__ unsigned wsum[kScanThreads / 32];
+    const int u = blockIdx.x;
+    const UnitDesc& ud = desc[u];
+    const int T = ud.T;
+    const int64_t o = ud.tok_off;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    const int chunk = (T + (int)blockDim.x - 1) / (int)blockDim.x;
+    const int b = threadIdx.x * chunk, e = min(T, b + chunk);
+    unsigned cnt = 0;
+    for (int i = b; i < e; ++i) cnt += (kind[o + i] != CASK_KIND_DROPPED);
+    unsigned incl = cnt;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        unsigned v = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += v;
+    }
+    if (lane == 31) wsum[w] = incl;
+    __syncthreads();
+    unsigned base = 0, total = 0;
+    for (int x = 0; x < nw; ++x) {
+        if (x < w) base += wsum[x];
+        total += wsum[x];
+    }
+    unsigned rank = base + incl - cnt;
+    for (int i = b; i < e; ++i) {
+        const bool need = kind[o + i] != CASK_KIND_DROPPED;
+        v_pos[o + i] = need ? (int)rank : -1;
+        rank += need;
+    }
+    if (threadIdx.x == 0) n_need[u] = (int)total;
+}
+
+__global__ void value_base_kernel(int n_units, const int32_t* __restrict__ n_need, int64_t* __restrict__ v_base) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        int64_t run = 0;
+        for (int u = 0; u < n_units; ++u) {
+            v_base[u] = run;
+            run += n_need[u];
+        }
     }
 }
 
@@ -307,6 +354,14 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const u
 }
 
 }  // namespace
+
+cudaError_t launch_value_ranks(const Launch& L, const uint8_t* kind, int32_t* v_pos, int32_t* n_need, int64_t* v_base) {
+    Timed t(L, KID_SLOT_SCAN);
+    value_rank_kernel<<<L.sh.n_units, kScanThreads, 0, L.stream>>>(L.desc, kind, v_pos, n_need);
+    value_base_kernel<<<1, 32, 0, L.stream>>>(L.sh.n_units, n_need, v_base);
+    ++*L.launches;
+    return cudaGetLastError();
+}
 
 cudaError_t launch_writeback(const Launch& L, const cask_outputs& out, void* k_pool, void* v_pool) {
     const Shape& sh = L.sh;
