@@ -19,7 +19,6 @@ def _properties(hb, g):
     w = hb.wl
     kf = hb.k.view(np.uint16) if w.dtype == wl.DTYPE_BF16 else hb.k
     vf = hb.v.view(np.uint16) if w.dtype == wl.DTYPE_BF16 else hb.v
-    from paper_2604_10900_b200 import workloads as W
     for u in range(hb.n_units):
         a, T, P, B = int(hb.tok_off[u]), int(hb.T[u]), int(hb.P[u]), int(hb.B[u])
         sl = slice(a, a + T)
@@ -77,11 +76,11 @@ def _slice_units(g, hb, idx, hb_s):
     return out
 
 
-def _full(name, sample):
+def _full(name, sample, units=None):
     import torch
     import gpu_harness as gh
     w = wl.WORKLOADS[name]
-    hb = wl.make_batch(w, threads=16)
+    hb = wl.make_batch(w, units, threads=16)
     run = gh.GpuRun(hb)
     g = run.event()
     assert run.ctx.used_tensor_path and run.ctx.device_flags() == 0
@@ -114,4 +113,16 @@ def test_reasoning8k_b384_full_size():
 def test_prompt_heavy_full_size():
     """Prefix eviction to 1536 rows before decode consolidation, budget 2048, m = 224 seeds."""
     st = _full("prompt_heavy", [3, 60, 108])
+    assert st["max_score_rel"] < 1e-5
+
+
+def test_batched_serving_ragged_slice():
+    """Config 5: 64 sequences with decode lengths between 4,096 and 32,768 in one launch (one layer, two KV heads
+    each: 128 ragged units); the shortest, the longest and a middle unit go through the oracle."""
+    w = wl.WORKLOADS["batched_serving"]
+    units = wl.unit_list(w, layers=range(1), heads=range(2))
+    T = np.array([w.prefix + wl.decode_len(w, s) for (s, _, _) in units])
+    assert T.min() < 8192 and T.max() > 30000
+    sample = sorted({int(np.argmin(T)), int(np.argmax(T)), int(np.argsort(T)[len(T) // 2])})
+    st = _full("batched_serving", sample, units)
     assert st["max_score_rel"] < 1e-5
