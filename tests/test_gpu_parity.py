@@ -372,17 +372,23 @@ def test_bad_arguments_are_refused_on_the_host_before_any_launch():
     run.event()
 
 
-def test_host_buffer_entry_point_matches_device_entry_point():
-    """cask_compress_event_host (host K/V/Q and host outputs) gives the bytes of the device call."""
+@pytest.mark.parametrize("extras", [False, True])
+def test_host_buffer_entry_point_matches_device_entry_point(extras):
+    """cask_compress_event_host (host K/V/Q and host outputs; only the value rows that are read go up) gives the
+    bytes of the device call, also with carried masses and channel weights passed as host arrays."""
     import gpu_harness as gh
     import torch
     w = _small("reasoning8k_b384", layers=1, kv_heads=2, decode=1000)
     hb = wl.make_batch(w)
-    run = gh.GpuRun(hb)
+    rng = np.random.default_rng(3)
+    mass = (np.where(rng.random(int(hb.tok_off[-1])) < 0.3, rng.random(int(hb.tok_off[-1])) * 1e-3, 0.0)
+            .astype(np.float32)) if extras else None
+    cw = (rng.random(w.head_dim) + 0.05).astype(np.float32) if extras else None
+    run = gh.GpuRun(hb, mass_in=mass, chan_w=cw)
     g = run.event()
     cb = run.cb
     hbatch, keep = cb.make_batch(hb.k, hb.v, hb.q, hb.T, hb.P, hb.B, hb.reserve, hb.tok_off, w.head_dim, w.group,
-                                 w.window, w.dtype)
+                                 w.window, w.dtype, mass_in=mass, chan_w=cw)
     nbytes = cb.cask_host_event_device_bytes(hbatch, run.prm, run.Bmax)
     assert nbytes > 0
     dev = torch.empty(nbytes, dtype=torch.uint8, device="cuda:0")
