@@ -147,7 +147,7 @@ def run_ours(args):
     w = wl.WORKLOADS[args.workload]
     # A batch of many sequences does not fit one GPU with all its layers (64 sequences x 36 layers x 8 heads of
     # the serving sweep hold 179 GB of K/V): it runs on a slice of the layers, every sequence present.
-    n_layers = w.layers if w.n_seqs == 1 else min(w.layers, args.layer_slice or 6)
+    n_layers = min(w.layers, args.layer_slice or w.layers_per_pass or w.layers)
     units = wl.unit_list(w, seqs=range(rank, rank + 1)) if w.n_seqs == 1 else \
         wl.shard_units(wl.unit_list(w, layers=range(n_layers)), rank, world)
     if args.max_units:
@@ -165,8 +165,9 @@ def run_ours(args):
     d, rows = w.head_dim, w.group * w.window
 
     dev = cb.to_device(hb, device)
+    mass_dev = None if hb.mass_in is None else torch.from_numpy(hb.mass_in).to(device)
     batch, keep = cb.make_batch(dev["k"], dev["v"], dev["q"], hb.T, hb.P, hb.B, hb.reserve, hb.tok_off, d, w.group,
-                                w.window, w.dtype)
+                                w.window, w.dtype, mass_in=mass_dev)
     prm = cb.params(score_path=args.score_path)
     stream = torch.cuda.current_stream(device)
     ctx = cb.Context(local, stream.cuda_stream)
@@ -218,7 +219,7 @@ def run_ours(args):
     # The same event when the caller hands over the window queries' softmax normalisers (a decode attention
     # kernel has them): the normaliser pass is skipped.  Reported beside the headline, never instead of it.
     batch_l, keep_l = cb.make_batch(dev["k"], dev["v"], dev["q"], hb.T, hb.P, hb.B, hb.reserve, hb.tok_off, d, w.group,
-                                    w.window, w.dtype, lse_in=out["lse"].clone())
+                                    w.window, w.dtype, lse_in=out["lse"].clone(), mass_in=mass_dev)
     cb.cask_compress_event(ctx, batch_l, prm, out_struct, ws, ws_bytes)
     barrier()
     ev0.record(stream)
@@ -244,7 +245,7 @@ def run_ours(args):
 
     # ---- end to end through the host-buffer entry point ---------------------------------------
     hbatch, hkeep = cb.make_batch(hb.k, hb.v, hb.q, hb.T, hb.P, hb.B, hb.reserve, hb.tok_off, d, w.group, w.window,
-                                  w.dtype)
+                                  w.dtype, mass_in=hb.mass_in)
     dev_bytes = cb.cask_host_event_device_bytes(hbatch, prm, Bmax)
     del dev, out, out_struct, ws
     torch.cuda.empty_cache()
@@ -261,7 +262,8 @@ def run_ours(args):
     ho_struct = cb.make_outputs(ho, Bmax)
     # The host entry point sends the keys and queries whole but only the value rows that are kept or merged
     # (counted from the row kinds of the device run); the row kinds come back once more in mid-call.
-    h2d = hb.k.nbytes + hb.q.nbytes + int(np.count_nonzero(kind)) * d * (2 if w.dtype == wl.DTYPE_BF16 else 4)
+    h2d = hb.k.nbytes + hb.q.nbytes + int(np.count_nonzero(kind)) * d * (2 if w.dtype == wl.DTYPE_BF16 else 4) \
+        + (0 if hb.mass_in is None else hb.mass_in.nbytes)
     d2h = sum(a.nbytes for a in ho.values()) + sum_T
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
     cb.cask_compress_event_host(ctx, hbatch, prm, ho_struct, dev_buf, dev_bytes)   # warm-up
@@ -332,7 +334,8 @@ def run_ours(args):
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == wl.DTYPE_BF16 else "f32",
+        "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak" if w.n_seqs == 1 else "strong", "vs_baseline": None, "dtype": "bf16" if w.dtype == wl.DTYPE_BF16 else "f32",
         "data": "synthetic",
         "config": {"workload": w.name, "units_per_gpu": hb.n_units, "rows_per_unit": int(hb.T.max()), "head_dim": d,
                    "query_rows": rows, "budget": int(hb.B.max()), "tokens_per_step": total_tokens,
@@ -343,6 +346,7 @@ def run_ours(args):
                        "events_per_s": w.n_seqs * n_layers / w.layers / (ms_step * 1e-3),
                        "events_per_s_note": "one event = all layers of one sequence; this pass held layers_per_pass of them"}
                       if w.n_seqs > 1 else {}),
+                   **({"carried_mass_rows": w.carried_rows} if w.carried_rows else {}),
                    "status_bits_seen": int(np.bitwise_or.reduce(status))},
         "with_supplied_normalisers": {"ms_per_step": ms_lse, "value": total_tokens / (ms_lse * 1e-3), "unit": UNIT,
                                       "note": "lse_in given by the caller: one scoring pass instead of two (this rank)"},
@@ -361,12 +365,13 @@ def run_ours(args):
 def cpu_baseline(w: wl.Workload, n_units: int):
     """The oracle, as it stands, on a bounded sample: the first `n_units` units of the workload."""
     from oracle import cask_oracle as orc
+    n_units = n_units or max(1, min(w.n_units, (32 * 33280) // (w.prefix + w.decode)))
     units = wl.unit_list(w)[:n_units]
     hb = wl.make_batch(w, units)
     kf, vf, qf = (wl.as_float32(x, w.dtype) for x in (hb.k, hb.v, hb.q))
     orc.lib()
     t = time.time()
-    orc.event_batch(kf, vf, qf, hb.tok_off, hb.P, hb.B, hb.reserve)
+    orc.event_batch(kf, vf, qf, hb.tok_off, hb.P, hb.B, hb.reserve, mass_in=hb.mass_in)
     dt = time.time() - t
     return {"value": float(hb.T.sum()) / dt, "unit": UNIT, "cores": orc.threads(), "kind": "oracle",
             "sample": f"{len(units)} of {w.n_units} units of {w.name} (whole event, fp64), {dt:.1f} s",
@@ -380,14 +385,14 @@ def run_reference(args):
         return
     from oracle import cask_oracle as orc
     w = wl.WORKLOADS[args.workload]
-    n_units = min(args.cpu_units, 16)
+    n_units = min(args.cpu_units, 16) if args.cpu_units else max(1, min(w.n_units, (16 * 33280) // (w.prefix + w.decode)))
     units = wl.unit_list(w)[:n_units]
     hb = wl.make_batch(w, units)
     kf, vf, qf = (wl.as_float32(x, w.dtype) for x in (hb.k, hb.v, hb.q))
     orc.lib()
 
     def step():
-        orc.event_batch(kf, vf, qf, hb.tok_off, hb.P, hb.B, hb.reserve)
+        orc.event_batch(kf, vf, qf, hb.tok_off, hb.P, hb.B, hb.reserve, mass_in=hb.mass_in)
 
     for _ in range(args.warmup):
         step()
@@ -418,7 +423,8 @@ def main():
     ap.add_argument("--workload", default="reasoning32k_b512", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--score-path", type=int, default=0, help="0: tensor-core scoring when the shape allows, 1: SIMT")
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--cpu-units", type=int, default=32, help="units in the oracle's bounded sample")
+    ap.add_argument("--cpu-units", type=int, default=0,
+                    help="units in the oracle's bounded sample (default: about a million cache rows)")
     ap.add_argument("--max-units", type=int, default=0, help="debug: cut the workload to this many units")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layer-slice", type=int, default=0,

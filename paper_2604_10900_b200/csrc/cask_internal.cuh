@@ -127,7 +127,11 @@ cudaError_t launch_prefix_evict(const Launch& L, const float* s, uint8_t* kind, 
 cudaError_t launch_select_core(const Launch& L, const float* s, const int32_t* plan, uint8_t* kind);
 cudaError_t launch_consolidate(const Launch& L, const cask_params& prm, const float* s,
                                const int32_t* plan, uint8_t* kind, int32_t* seed_of, float* weight,
-                               float* sim, int32_t* unit_status, float* lost_mass, Workspace& ws);
+                               float* sim, int32_t* unit_status, float* lost_mass, Workspace& ws,
+                               bool fused_small = false);
+// fused_small: every unit has at most kSmallUnitRows rows and `plan`, `kind` are still unwritten; one kernel then
+// does the prefix eviction, the core and seed selection and the seed gather (the event path only).
+constexpr int kSmallUnitRows = 1024;
 cudaError_t launch_compact(const Launch& L, const cask_params& prm, const float* s, const uint8_t* kind,
                            const int32_t* seed_of, float* weight, const cask_outputs& out, Workspace& ws);
 // Host-resident caches: rank of every row among the rows of its unit whose values the compaction reads

@@ -166,32 +166,63 @@ __global__ void __launch_bounds__(kScanThreads) slot_scan_kernel(
     }
 }
 
-// ---- 2. one warp per slot: byte copy of the slot's anchor row ------------------------------
+// ---- 2. byte copy of every slot's anchor row: one thread per 16-byte vector of K and of V ----
+// Flat over (unit, slot, vector) with four vectors in flight per thread, so that units of a few hundred
+// rows load the memory system as well as long ones.  The slot -> row lookups of the next round are issued
+// together with the row loads of the current one, so the two dependent levels overlap.
 template <typename T>
 __global__ void __launch_bounds__(256) slot_copy_kernel(
     const UnitDesc* __restrict__ desc, Shape sh, const T* __restrict__ K, const T* __restrict__ V,
-    const float* __restrict__ s, float eps, int Bmax, const int32_t* __restrict__ n_out,
+    const float* __restrict__ s, float eps, int Bmax, int slots, const int32_t* __restrict__ n_out,
     const int32_t* __restrict__ slot_src, T* __restrict__ k_out, T* __restrict__ v_out,
     float* __restrict__ slot_mass) {
-    const int u = blockIdx.y;
-    const UnitDesc& ud = desc[u];
-    const int lane = threadIdx.x & 31;
-    const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (t >= n_out[u]) return;
-    const int d = sh.d;
-    const int src = slot_src[(size_t)u * Bmax + t];
-    T* ko = k_out + ((size_t)u * Bmax + t) * d;
-    T* vo = v_out + ((size_t)u * Bmax + t) * d;
-    const T* ksrc = K + row_elem_off(sh, ud, ud.k_off, src);
-    const T* vsrc = V + v_elem_off(sh, ud, u, src);
-    const int nvec = d * (int)sizeof(T) / 16;
-    for (int x = lane; x < 2 * nvec; x += 32) {
-        const bool isv = x >= nvec;
-        const int c = isv ? x - nvec : x;
-        const uint4 val = reinterpret_cast<const uint4*>(isv ? vsrc : ksrc)[c];
-        reinterpret_cast<uint4*>(isv ? vo : ko)[c] = val;
+    const int nvec = sh.d * (int)sizeof(T) / 16;              // 8, 16 or 32
+    const int nvec_log2 = 31 - __clz(nvec);
+    const int64_t total = (int64_t)sh.n_units * slots * nvec;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    constexpr int kFly = 4;
+    // (unit, slot, row) of the kFly vectors of one round; row < 0: nothing to copy
+    struct Item { int u, t, src; };
+    auto lookup = [&](int64_t g) {
+        Item it{0, 0, -1};
+        if (g < total) {
+            // nvec is a power of two; units x slots stays far below 2^32 (the outputs alone would not fit the device)
+            const unsigned sg = (unsigned)(g >> nvec_log2);
+            it.u = (int)(sg / (unsigned)slots);
+            it.t = (int)(sg - (unsigned)it.u * (unsigned)slots);
+            if (it.t < n_out[it.u]) it.src = slot_src[(size_t)it.u * Bmax + it.t];
+        }
+        return it;
+    };
+    int64_t g0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    Item cur[kFly];
+#pragma unroll
+    for (int q = 0; q < kFly; ++q) cur[q] = lookup(g0 + q * stride);
+    for (; g0 < total; g0 += kFly * stride) {
+        uint4 kv[kFly], vv[kFly];
+        const int c = (int)(g0 & (nvec - 1));                 // the same for the whole round: stride is a multiple of nvec
+#pragma unroll
+        for (int q = 0; q < kFly; ++q) {
+            if (cur[q].src < 0) continue;
+            const UnitDesc& ud = desc[cur[q].u];
+            kv[q] = reinterpret_cast<const uint4*>(K + row_elem_off(sh, ud, ud.k_off, cur[q].src))[c];
+            vv[q] = reinterpret_cast<const uint4*>(V + v_elem_off(sh, ud, cur[q].u, cur[q].src))[c];
+            if (c == 0)
+                slot_mass[(size_t)cur[q].u * Bmax + cur[q].t] = row_mass(sh, s, eps, ud.tok_off + cur[q].src);
+        }
+        Item nxt[kFly];
+#pragma unroll
+        for (int q = 0; q < kFly; ++q) nxt[q] = lookup(g0 + (kFly + q) * stride);
+#pragma unroll
+        for (int q = 0; q < kFly; ++q) {
+            if (cur[q].src >= 0) {
+                const int64_t dst = ((int64_t)cur[q].u * Bmax + cur[q].t) * nvec + c;
+                reinterpret_cast<uint4*>(k_out)[dst] = kv[q];
+                reinterpret_cast<uint4*>(v_out)[dst] = vv[q];
+            }
+            cur[q] = nxt[q];
+        }
     }
-    if (lane == 0) slot_mass[(size_t)u * Bmax + t] = row_mass(sh, s, eps, ud.tok_off + src);
 }
 
 // ---- 3. one warp per representative with joiners: ordered weighted merge over its copy -----
@@ -254,6 +285,98 @@ __global__ void __launch_bounds__(256) slot_merge_kernel(
             }
         }
         if (lane == 0) slot_mass[(size_t)u * Bmax + t] = msum;
+    }
+}
+
+// ---- 3b. units of at most kMergeStageRows rows: one CTA per unit, member list staged in shared memory ----
+// Same arithmetic as slot_merge_kernel (members in ascending row order, one fp32 accumulator per channel),
+// but a warp first lists the members of its representative from shared memory and then reads their rows four
+// at a time, instead of walking the unit's whole member list in global memory with one row in flight.
+constexpr int kMergeStageRows = 2048;
+
+template <typename T, int CH>       // CH = d / 32 contiguous channels per lane
+__global__ void __launch_bounds__(256) slot_merge_small_kernel(
+    const UnitDesc* __restrict__ desc, Shape sh, const T* __restrict__ K, const T* __restrict__ V,
+    const float* __restrict__ s, const float* __restrict__ weight, float eps, int Bmax,
+    const int32_t* __restrict__ seed_slot, const int32_t* __restrict__ n_seed, int max_B,
+    const int32_t* __restrict__ mem_row, const int32_t* __restrict__ mem_slot,
+    const int32_t* __restrict__ n_mem, T* __restrict__ k_out, T* __restrict__ v_out,
+    float* __restrict__ slot_mass) {
+    __shared__ int32_t m_row[kMergeStageRows], m_slot[kMergeStageRows];
+    __shared__ float m_w[kMergeStageRows], m_a[kMergeStageRows];
+    __shared__ int32_t b_e[8][32];
+    const int u = blockIdx.x;
+    const UnitDesc& ud = desc[u];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    const int64_t o = ud.tok_off;
+    const int nm = min(n_mem[u], kMergeStageRows);
+    const int ns = n_seed[u];
+    for (int e = threadIdx.x; e < nm; e += blockDim.x) {
+        const int row = mem_row[o + e];
+        m_row[e] = row;
+        m_slot[e] = mem_slot[o + e];
+        m_w[e] = weight[o + row];
+        m_a[e] = row_mass(sh, s, eps, o + row);
+    }
+    __syncthreads();
+    struct alignas(CH * sizeof(T)) Vec { T x[CH]; };
+    for (int j = w; j < ns; j += nw) {
+        const int t = seed_slot[(size_t)u * max_B + j];
+        float ak[CH], av[CH];
+#pragma unroll
+        for (int x = 0; x < CH; ++x) { ak[x] = 0.f; av[x] = 0.f; }
+        int count = 0, held = 0;
+        float msum = 0.f;
+        auto flush = [&]() {
+            __syncwarp();
+            for (int h0 = 0; h0 < held; h0 += 4) {
+                Vec kr[4], vr[4];
+                float wi[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int e = b_e[w][min(h0 + q, held - 1)];
+                    const int i = m_row[e];
+                    wi[q] = m_w[e];
+                    kr[q] = reinterpret_cast<const Vec*>(K + row_elem_off(sh, ud, ud.k_off, i))[lane];
+                    vr[q] = reinterpret_cast<const Vec*>(V + v_elem_off(sh, ud, u, i))[lane];
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    if (h0 + q >= held) break;
+                    msum += m_a[b_e[w][h0 + q]];
+#pragma unroll
+                    for (int x = 0; x < CH; ++x) {
+                        ak[x] = fmaf(wi[q], Elem<T>::ld(&kr[q].x[x]), ak[x]);
+                        av[x] = fmaf(wi[q], Elem<T>::ld(&vr[q].x[x]), av[x]);
+                    }
+                }
+            }
+            count += held;
+            held = 0;
+            __syncwarp();
+        };
+        for (int e0 = 0; e0 < nm; e0 += 32) {
+            const int e = e0 + lane;
+            const bool hit = (e < nm) && m_slot[e] == t;
+            const unsigned bal = __ballot_sync(0xffffffffu, hit);
+            const int n = __popc(bal);
+            if (n == 0) continue;
+            if (held + n > 32) flush();
+            if (hit) b_e[w][held + __popc(bal & ((1u << lane) - 1u))] = e;
+            held += n;
+        }
+        flush();
+        if (count > 1) {       // a lone seed keeps its byte copy
+            Vec ko, vo;
+#pragma unroll
+            for (int x = 0; x < CH; ++x) {
+                Elem<T>::st(&ko.x[x], ak[x]);
+                Elem<T>::st(&vo.x[x], av[x]);
+            }
+            reinterpret_cast<Vec*>(k_out + ((size_t)u * Bmax + t) * sh.d)[lane] = ko;
+            reinterpret_cast<Vec*>(v_out + ((size_t)u * Bmax + t) * sh.d)[lane] = vo;
+            if (lane == 0) slot_mass[(size_t)u * Bmax + t] = msum;
+        }
     }
 }
 
@@ -332,7 +455,7 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const u
     const Shape& sh = L.sh;
     {
         Timed t(L, KID_SLOT_SCAN);
-        slot_scan_kernel<<<sh.n_units, kScanThreads, 0, L.stream>>>(L.desc, kind, seed_of, weight, out.Bmax,
+        slot_scan_kernel<<<sh.n_units, L.max_T <= 2048 ? 256 : kScanThreads, 0, L.stream>>>(L.desc, kind, seed_of, weight, out.Bmax,
                                                                     out.n_out, out.slot_src, out.slot_kind,
                                                                     out.slot_mass, out.assign, ws.mem_row,
                                                                     ws.mem_slot, ws.n_mem, ws.seed_slot, ws.n_seed,
@@ -342,12 +465,22 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const u
     {
         // the merge kernel overwrites slots the copy kernel wrote: same stream, in order
         Timed t(L, KID_GATHER_MERGE);
-        slot_copy_kernel<T><<<dim3((slots + 7) / 8, sh.n_units), 256, 0, L.stream>>>(
-            L.desc, sh, (const T*)L.k, (const T*)L.v, s, prm.eps, out.Bmax, out.n_out, out.slot_src, (T*)out.k_out,
-            (T*)out.v_out, out.slot_mass);
-        slot_merge_kernel<T><<<dim3((std::min(slots, ws.max_B) + 7) / 8, sh.n_units), 256, 0, L.stream>>>(
-            L.desc, sh, (const T*)L.k, (const T*)L.v, s, weight, prm.eps, out.Bmax, ws.seed_slot, ws.n_seed, ws.max_B,
-            ws.mem_row, ws.mem_slot, ws.n_mem, (T*)out.k_out, (T*)out.v_out, out.slot_mass);
+        const int nvec = sh.d * (int)sizeof(T) / 16;
+        const int64_t vecs = (int64_t)sh.n_units * slots * nvec;
+        const int copy_grid = (int)std::min<int64_t>((vecs + 256 * 4 - 1) / (256 * 4), 148 * 64);
+        slot_copy_kernel<T><<<std::max(copy_grid, 1), 256, 0, L.stream>>>(
+            L.desc, sh, (const T*)L.k, (const T*)L.v, s, prm.eps, out.Bmax, slots, out.n_out, out.slot_src,
+            (T*)out.k_out, (T*)out.v_out, out.slot_mass);
+        if (L.max_T <= kMergeStageRows && (sh.d == 64 || sh.d == 128)) {
+            auto kern = sh.d == 128 ? slot_merge_small_kernel<T, 4> : slot_merge_small_kernel<T, 2>;
+            kern<<<sh.n_units, 256, 0, L.stream>>>(
+                L.desc, sh, (const T*)L.k, (const T*)L.v, s, weight, prm.eps, out.Bmax, ws.seed_slot, ws.n_seed,
+                ws.max_B, ws.mem_row, ws.mem_slot, ws.n_mem, (T*)out.k_out, (T*)out.v_out, out.slot_mass);
+        } else {
+            slot_merge_kernel<T><<<dim3((std::min(slots, ws.max_B) + 7) / 8, sh.n_units), 256, 0, L.stream>>>(
+                L.desc, sh, (const T*)L.k, (const T*)L.v, s, weight, prm.eps, out.Bmax, ws.seed_slot, ws.n_seed,
+                ws.max_B, ws.mem_row, ws.mem_slot, ws.n_mem, (T*)out.k_out, (T*)out.v_out, out.slot_mass);
+        }
         ++*L.launches;
     }
     return cudaGetLastError();

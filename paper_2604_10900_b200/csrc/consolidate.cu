@@ -58,7 +58,9 @@ __global__ void seed_gather_kernel(const UnitDesc* __restrict__ desc, Shape sh, 
                                    const int32_t* __restrict__ seed_rows, T* __restrict__ seed_k,
                                    float* __restrict__ seed_norm, unsigned long long* __restrict__ mass_fx,
                                    int max_m, float eps, int split_rows) {
-    const int u = blockIdx.y, j = blockIdx.x;
+    // one warp per seed, eight seeds per CTA
+    const int u = blockIdx.y, j = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
     const UnitDesc& ud = desc[u];
     const int m = max(0, min(plan[u * 8 + CASK_PLAN_M], ud.plan[CASK_PLAN_M]));
     if (j >= m) return;
@@ -68,7 +70,7 @@ __global__ void seed_gather_kernel(const UnitDesc* __restrict__ desc, Shape sh, 
     // hi + lo of the cache dtype, so that the bf16 contraction sees w*k to about 2^-17.
     T* dst = seed_k + (size_t)(ud.seed_base + j) * (split_rows ? 2 : 1) * sh.d;
     float n2 = 0.f;
-    for (int c = threadIdx.x; c < sh.d; c += 32) {
+    for (int c = lane; c < sh.d; c += 32) {
         T x = src[c];
         float f = Elem<T>::ld(&x);
         const float wc = sh.chan_w ? sh.chan_w[c] : 1.f;
@@ -83,9 +85,124 @@ __global__ void seed_gather_kernel(const UnitDesc* __restrict__ desc, Shape sh, 
     }
 #pragma unroll
     for (int off = 16; off >= 1; off >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, off);
-    if (threadIdx.x == 0) {
+    if (lane == 0) {
         seed_norm[ud.seed_base + j] = sqrtf(n2);
         atomicAdd(&mass_fx[(size_t)u * (max_m + 1) + j], mass_to_fx(row_mass(sh, s, eps, ud.tok_off + row)));
+    }
+}
+
+// ---- 1+2 for units of at most kSmallSpan rows: prefix eviction, core selection, seed selection and the seed
+// gather in one CTA per unit (the event path; the staged calls keep their own kernels and give the same
+// result).  Keys and kinds live in shared memory; every row of a range counts the rows ahead of it in the total
+// order (score descending, row ascending), so the c greatest rows of the scratch range are the core and the next
+// m the seeds, which is what taking the top c and then the top m of the rest gives.
+template <typename T>
+__global__ void __launch_bounds__(256) decide_small_kernel(
+    const UnitDesc* __restrict__ desc, Shape sh, const T* __restrict__ K, const float* __restrict__ s,
+    int32_t* __restrict__ plan, uint8_t* __restrict__ kind, int32_t* __restrict__ seed_of,
+    float* __restrict__ weight, float* __restrict__ sim, int32_t* __restrict__ grp,
+    int32_t* __restrict__ seed_rows, T* __restrict__ seed_k, float* __restrict__ seed_norm,
+    unsigned long long* __restrict__ mass_fx, int32_t* __restrict__ njoin, int max_m, float eps, int split_rows) {
+    __shared__ unsigned keys[kSmallSpan];
+    __shared__ int32_t seed_list[kSmallSpan];
+    __shared__ uint8_t kd[kSmallSpan];
+    __shared__ unsigned wsum[8];
+    const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    const UnitDesc& ud = desc[u];
+    const int T_ = ud.T, P = ud.P;
+    const int64_t o = ud.tok_off;
+    const int pkeep = ud.plan[CASK_PLAN_PKEEP], c = max(0, ud.plan[CASK_PLAN_C]), m = max(0, ud.plan[CASK_PLAN_M]);
+    const int r = max(0, min(ud.plan[CASK_PLAN_R], T_ - P));
+    if (tid < 8) plan[u * 8 + tid] = ud.plan[tid];
+    const uint8_t pre = (P <= pkeep) ? CASK_KIND_PREFIX : CASK_KIND_DROPPED;
+    for (int i = tid; i < T_; i += blockDim.x) {
+        keys[i] = order_key(s[o + i]);
+        kd[i] = (i < P) ? pre : (i >= T_ - r ? CASK_KIND_RECENT : CASK_KIND_DROPPED);
+    }
+    __syncthreads();
+    // rows of [lo, hi) ahead of row i: greater keys, and equal keys at lower rows
+    auto ahead_of = [&](int lo, int hi, int i) {
+        const unsigned ki = keys[i];
+        int a = 0;
+        for (int j = lo; j < i; ++j) a += keys[j] >= ki;
+        for (int j = i + 1; j < hi; ++j) a += keys[j] > ki;
+        return a;
+    };
+    if (P > pkeep && pkeep > 0)
+        for (int i = tid; i < P; i += blockDim.x)
+            if (ahead_of(0, P, i) < pkeep) kd[i] = CASK_KIND_PREFIX;
+    const int lo = P, hi = T_ - r;
+    if (c + m > 0)
+        for (int i = lo + tid; i < hi; i += blockDim.x) {
+            const int a = ahead_of(lo, hi, i);
+            if (a < c) kd[i] = CASK_KIND_CORE;
+            else if (a < c + m) kd[i] = CASK_KIND_SEED;
+        }
+    __syncthreads();
+    for (int i = tid; i < T_; i += blockDim.x) {
+        kind[o + i] = kd[i];
+        seed_of[o + i] = -1;
+        weight[o + i] = 0.f;
+        grp[o + i] = -1;
+        if (sim) sim[o + i] = -2.f;
+    }
+    for (int j = tid; j <= max_m; j += blockDim.x) mass_fx[(size_t)u * (max_m + 1) + j] = 0ull;
+    if (tid == 0) njoin[u] = 0;
+    // ordered list of the seed rows: one contiguous chunk of the scratch range per thread, one block scan
+    const int span = max(hi - lo, 0);
+    const int chunk = (span + (int)blockDim.x - 1) / (int)blockDim.x;
+    const int b = lo + tid * chunk, e = min(hi, b + chunk);
+    unsigned cnt = 0;
+    for (int i = b; i < e; ++i) cnt += kd[i] == CASK_KIND_SEED;
+    unsigned incl = cnt;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const unsigned v = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += v;
+    }
+    if (lane == 31) wsum[w] = incl;
+    __syncthreads();       // also orders the per-row initialisation above before the seed rows' own entries
+    unsigned rank = incl - cnt;
+    for (int x = 0; x < w; ++x) rank += wsum[x];
+    for (int i = b; i < e; ++i)
+        if (kd[i] == CASK_KIND_SEED) {
+            if (rank < (unsigned)m) {
+                seed_list[rank] = i;
+                seed_rows[ud.seed_base + rank] = i;
+                seed_of[o + i] = i;
+                grp[o + i] = (int)rank;
+            }
+            ++rank;
+        }
+    __syncthreads();
+    unsigned n_seeds = 0;
+    for (int x = 0; x < (int)(blockDim.x >> 5); ++x) n_seeds += wsum[x];
+    const int ms = min((int)n_seeds, m);
+    // gather the seed keys, their norms and their own mass: one warp per seed
+    for (int j = w; j < ms; j += (int)(blockDim.x >> 5)) {
+        const int row = seed_list[j];
+        const T* src = K + row_elem_off(sh, ud, ud.k_off, row);
+        T* dst = seed_k + (size_t)(ud.seed_base + j) * (split_rows ? 2 : 1) * sh.d;
+        float n2 = 0.f;
+        for (int ch = lane; ch < sh.d; ch += 32) {
+            T x = src[ch];
+            float f = Elem<T>::ld(&x);
+            const float wc = sh.chan_w ? sh.chan_w[ch] : 1.f;
+            if (split_rows) {
+                const float wf = wc * f;
+                Elem<T>::st(dst + ch, wf);
+                Elem<T>::st(dst + sh.d + ch, wf - Elem<T>::ld(dst + ch));
+            } else {
+                dst[ch] = x;
+            }
+            n2 = fmaf(wc * f, f, n2);
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, off);
+        if (lane == 0) {
+            seed_norm[ud.seed_base + j] = sqrtf(n2);
+            mass_fx[(size_t)u * (max_m + 1) + j] = mass_to_fx(row_mass(sh, s, eps, o + row));
+        }
     }
 }
 
@@ -237,19 +354,24 @@ __global__ void weights_kernel(const UnitDesc* __restrict__ desc, Shape sh, cons
 template <typename T>
 cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const int32_t* plan, uint8_t* kind,
                 int32_t* seed_of, float* weight, float* sim, int32_t* unit_status, float* lost_mass,
-                Workspace& ws) {
+                Workspace& ws, bool fused_small) {
     const Shape& sh = L.sh;
     const int max_m = L.max_m;
-    {
+    const bool use_tc = !L.force_simt && L.tmap_encode && assign_tc_supported(L);
+    if (fused_small) {
         Timed t(L, KID_SEEDS);
-        seeds_kernel<<<sh.n_units, kSelThreads, 0, L.stream>>>(L.desc, s, plan, kind, seed_of, weight, sim,
+        decide_small_kernel<T><<<sh.n_units, 256, 0, L.stream>>>(
+            L.desc, sh, (const T*)L.k, s, const_cast<int32_t*>(plan), kind, seed_of, weight, sim, ws.grp, ws.seed_rows,
+            (T*)ws.seed_k, ws.seed_norm, ws.mass_fx, ws.njoin, max_m, prm.eps, (use_tc && sh.chan_w) ? 1 : 0);
+    } else {
+        Timed t(L, KID_SEEDS);
+        seeds_kernel<<<sh.n_units, select_threads(L.max_T), 0, L.stream>>>(L.desc, s, plan, kind, seed_of, weight, sim,
                                                                ws.grp, ws.seed_rows, ws.mass_fx, ws.njoin, max_m);
     }
-    const bool use_tc = !L.force_simt && L.tmap_encode && assign_tc_supported(L);
     if (max_m > 0) {
-        {
+        if (!fused_small) {
             Timed t(L, KID_SEED_GATHER);
-            seed_gather_kernel<T><<<dim3(max_m, sh.n_units), 32, 0, L.stream>>>(
+            seed_gather_kernel<T><<<dim3((max_m + 7) / 8, sh.n_units), 256, 0, L.stream>>>(
                 L.desc, sh, (const T*)L.k, s, plan, ws.seed_rows, (T*)ws.seed_k, ws.seed_norm, ws.mass_fx, max_m,
                 prm.eps, (use_tc && sh.chan_w) ? 1 : 0);
         }
@@ -280,10 +402,10 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const i
 
 cudaError_t launch_consolidate(const Launch& L, const cask_params& prm, const float* s, const int32_t* plan,
                                uint8_t* kind, int32_t* seed_of, float* weight, float* sim,
-                               int32_t* unit_status, float* lost_mass, Workspace& ws) {
+                               int32_t* unit_status, float* lost_mass, Workspace& ws, bool fused_small) {
     if (L.sh.dtype == CASK_DTYPE_BF16)
-        return run<__nv_bfloat16>(L, prm, s, plan, kind, seed_of, weight, sim, unit_status, lost_mass, ws);
-    return run<float>(L, prm, s, plan, kind, seed_of, weight, sim, unit_status, lost_mass, ws);
+        return run<__nv_bfloat16>(L, prm, s, plan, kind, seed_of, weight, sim, unit_status, lost_mass, ws, fused_small);
+    return run<float>(L, prm, s, plan, kind, seed_of, weight, sim, unit_status, lost_mass, ws, fused_small);
 }
 
 }  // namespace cask

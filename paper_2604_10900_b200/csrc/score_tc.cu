@@ -45,6 +45,7 @@ constexpr int kEpiWarps = 4 * kSlots;
 constexpr int kThreadsTc = (kEpiWarp0 + kEpiWarps) * 32;
 constexpr uint32_t kQRegionBytes = 256 * 128;          // 256 rows x 64 bf16
 constexpr uint32_t kQBytes = 4 * kQRegionBytes;        // 2 row halves x 2 K blocks
+constexpr uint32_t kQBlockBytes = 128 * 128;           // one 128-row query block inside a region
 constexpr uint32_t kKRegionBytes = 128 * 128;          // 128 keys x 64 bf16
 constexpr uint32_t kKStageBytes = 2 * kKRegionBytes;
 constexpr int kMaxSms = 1024;                          // upper bound used when sizing the partial tables
@@ -57,7 +58,7 @@ constexpr uint32_t kPolyPairs16N = 0x88u;
 constexpr uint32_t kPolyPairs16S = 0x80u;
 
 struct __align__(8) Barriers {
-    uint64_t q_full, q_empty;
+    uint64_t q_full[kSlots], q_empty[kSlots];   // one pair per 128-row block of the window queries
     uint64_t k_full[kStages], k_empty[kStages];
     uint64_t d_full[kSlots], d_empty[kSlots];
     uint64_t rw_ready;      // pass S: the row table of the segment is written
@@ -68,7 +69,7 @@ struct TcSmemTail {
     Barriers bar;
     uint32_t tmem_base;
     int abort;
-    alignas(16) float rc[2][512];  // pass S: log2(roww) - rowm per query row, double-buffered by segment
+    alignas(16) float rc[3][512];  // pass S: log2(roww) - rowm per query row, one buffer per segment in turn
     float red[8][4][128];         // pass S: partial key sums per (group, column half), eight tiles deep
 };
 
@@ -129,11 +130,18 @@ __device__ __forceinline__ void mass_block(const float (&v)[32], const float* nc
         }
     } else {
         float a = 0.f;
+        if (!causal || (W & 31) == 0) {
+            // the 32 rows of the block lie inside one head (r0 is a multiple of 32): one threshold for the block
+            const int thr = causal ? jmin - r0 % W : 0;
 #pragma unroll
-        for (int x = 0; x < 32; ++x) {
-            const int r = r0 + x;
-            const bool vis = !causal || (r % W) >= jmin;
-            if (vis) a += ex2(fmaf(v[x], scale2, nc[r]));
+            for (int x = 0; x < 32; ++x)
+                if (x >= thr) a += ex2(fmaf(v[x], scale2, nc[r0 + x]));
+        } else {
+#pragma unroll
+            for (int x = 0; x < 32; ++x) {
+                const int r = r0 + x;
+                if ((r % W) >= jmin) a += ex2(fmaf(v[x], scale2, nc[r]));
+            }
         }
         a01 = add2(a01, pack2(a, 0.f));
     }
@@ -238,13 +246,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rows = sh.rows;
     const int n_slots = (rows + 127) >> 7;           // 128-row query blocks in use
-    const int n_halves = (rows + 255) >> 8;          // 256-row Q regions in use
     const int n_issuers = min(2, n_slots);
     const int n_groups = n_issuers;                  // epilogue groups of eight warps
 
     if (threadIdx.x == 0) {
-        mbar_init(&bar.q_full, 1);
-        mbar_init(&bar.q_empty, n_issuers);
+        for (int i = 0; i < kSlots; ++i) { mbar_init(&bar.q_full[i], 1); mbar_init(&bar.q_empty[i], 1); }
         for (int i = 0; i < kStages; ++i) { mbar_init(&bar.k_full[i], 1); mbar_init(&bar.k_empty[i], n_issuers); }
         for (int i = 0; i < kSlots; ++i) { mbar_init(&bar.d_full[i], 1); mbar_init(&bar.d_empty[i], 8); }
         mbar_init(&bar.rw_ready, 256 * n_groups);
@@ -271,12 +277,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             bool ok = true;
             for (; wk.valid() && ok; wk.next_segment(), ++seg) {
                 const UnitDesc& ud = desc[wk.u];
-                ok = mbar_wait(&bar.q_empty, (seg & 1u) ^ 1u, abort_flag);
-                if (!ok) break;
-                mbar_expect_tx(&bar.q_full, n_halves * 2 * kQRegionBytes);
-                for (int nh = 0; nh < n_halves; ++nh)
-                    for (int kb = 0; kb < 2; ++kb)
-                        tma_load_3d(q_smem + (nh * 2 + kb) * kQRegionBytes, &tmQ, &bar.q_full, kb * 64, nh * 256, wk.u);
                 const int krow0 = sh.page_size ? 0 : (int)(ud.k_off / sh.row_stride);
                 const int key_begin = wk.key_begin();
                 const int nt = wk.seg_tiles();
@@ -301,12 +301,28 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                             tma_load_2d(dst + kKRegionBytes + sb * sub_rows * 128, &tmK, &bar.k_full[st], 64, prow);
                         }
                     }
+                    if (t == 0) {
+                        // The segment's query blocks, each as soon as the previous segment's last contraction
+                        // with that block has completed: block 0 is back in shared memory while the tensor pipe
+                        // still works on the later blocks of the previous unit.  (The first key tile of the
+                        // segment went out before, so it does not wait behind them.)
+                        for (int j = 0; j < n_slots && ok; ++j) {
+                            ok = mbar_wait(&bar.q_empty[j], (seg & 1u) ^ 1u, abort_flag);
+                            if (!ok) break;
+                            mbar_expect_tx(&bar.q_full[j], 2 * kQBlockBytes);
+                            uint8_t* qd_ = q_smem + (j >> 1) * 2 * kQRegionBytes + (j & 1) * kQBlockBytes;
+                            for (int kb = 0; kb < 2; ++kb)
+                                tma_load_3d(qd_ + kb * kQRegionBytes, &tmQ, &bar.q_full[j], kb * 64, j * 128, wk.u);
+                        }
+                    }
                 }
             }
             if (!ok) {
                 // copies already issued may still be landing: give each armed stage a bounded wait
                 for (uint32_t j = (kit >= (uint32_t)kStages ? kit - kStages : 0); j < kit; ++j)
                     for (uint32_t it = 0; it < 4096 && !mbar_try(&bar.k_full[j % kStages], (j / kStages) & 1u); ++it) {}
+                for (int j = 0; j < n_slots; ++j)
+                    for (uint32_t it = 0; it < 4096 && !mbar_try(&bar.q_full[j], seg & 1u); ++it) {}
             }
         }
     } else if (warp <= n_issuers) {
@@ -319,8 +335,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             // adding a compile-time constant (the address field counts 16-byte units and cannot carry).
             const uint32_t q_lo = umma_desc_lo(smem_u32(q_smem)), k_lo = umma_desc_lo(smem_u32(k_smem));
             for (; wk.valid() && ok; wk.next_segment(), ++seg) {
-                ok = mbar_wait(&bar.q_full, seg & 1u, abort_flag);
-                if (!ok) break;
                 const int nt = wk.seg_tiles();
                 for (int t = 0; t < nt && ok; ++t, ++kit) {
                     const int st = kit % kStages;
@@ -333,6 +347,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         if (j >= n_slots || !ok) break;
                         ok = mbar_wait(&bar.d_empty[j], (kit & 1u) ^ 1u, abort_flag);
                         if (!ok) break;
+                        if (t == 0) {                       // the segment's query block j has landed
+                            ok = mbar_wait(&bar.q_full[j], seg & 1u, abort_flag);
+                            if (!ok) break;
+                        }
                         tc_fence_after();
                         const uint32_t qblk_lo = q_lo + (((j >> 1) * 2 * kQRegionBytes + (j & 1) * (128 * 128)) >> 4);
                         const uint32_t idesc = umma_idesc(PASS == 1 ? min(128, rows - 128 * j) : 128);
@@ -347,10 +365,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                             else tc_mma_lo<true>(tmem_base + 128 * j, dq, dk, idesc);
                         }
                         tc_commit(&bar.d_full[j]);
+                        if (t == nt - 1) tc_commit(&bar.q_empty[j]);      // last use of query block j in this segment
                     }
                     tc_commit(&bar.k_empty[st]);
                 }
-                if (ok) tc_commit(&bar.q_empty);
             }
         }
     } else if (warp >= kEpiWarp0 && ((warp - kEpiWarp0) >> 3) < n_groups) {
@@ -369,20 +387,32 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         // pass N: running reference / sum of the two query rows this thread works on
         float mm[2] = {kNegBig, kNegBig}, l_run[2] = {0.f, 0.f};
 
+        if (PASS == 1 && wk.valid()) {
+            // roww * 2^(y - rowm) = 2^(y + (log2 roww - rowm)): one constant per query row
+            tail->rc[0][etid] = (etid < rows) ? log2f(roww[(size_t)wk.u * rows + etid]) - rowm[(size_t)wk.u * rows + etid]
+                                              : -1.0e30f;
+            mbar_arrive(&bar.rw_ready);
+        }
         for (; wk.valid() && ok; wk.next_segment(), ++seg) {
             const int T = wk.T;
             const int64_t tok_off = desc[wk.u].tok_off;
             const int last_all = sh.causal ? T - sh.W : T - 1;     // last key every query sees
-            const float* rc = tail->rc[seg & 1u];
+            const float* rc = tail->rc[seg % 3u];
+            float rc_next = -1.0e30f;
+            bool has_next = false;
             if (PASS == 1) {
-                // Every thread has passed the rw_ready phase of the previous segment, so nobody still
-                // reads the buffer used two segments ago.  roww * 2^(y - rowm) = 2^(y + (log2 roww - rowm)).
-                float* dst = tail->rc[seg & 1u];
-                dst[etid] = (etid < rows) ? log2f(roww[(size_t)wk.u * rows + etid]) - rowm[(size_t)wk.u * rows + etid]
-                                          : -1.0e30f;
-                mbar_arrive(&bar.rw_ready);
+                // The table of this segment was written during the previous one (before the loop for the first).
                 ok = mbar_wait(&bar.rw_ready, seg & 1u, abort_flag);
                 if (!ok) break;
+                // Fetch the next segment's entry now; it goes into the third buffer after this segment's first
+                // tile, when the loads have long landed.  Whoever passed the wait above knows that every thread
+                // is past the first tile of the previous segment, so nobody still reads the buffer of the segment
+                // before that one, which is the one written next.
+                TileWalk nx = wk;
+                nx.next_segment();
+                has_next = nx.valid();
+                if (has_next && etid < rows)
+                    rc_next = log2f(roww[(size_t)nx.u * rows + etid]) - rowm[(size_t)nx.u * rows + etid];
             } else {
                 mm[0] = mm[1] = kNegBig;
                 l_run[0] = l_run[1] = 0.f;
@@ -522,6 +552,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&bar.d_empty[j]);
                     }
+                }
+                if (PASS == 1 && t == 0 && has_next && ok) {       // before this tile's global stores
+                    tail->rc[(seg + 1) % 3u][etid] = rc_next;
+                    mbar_arrive(&bar.rw_ready);
                 }
                 if (PASS == 1 && ok) {
                     float a0, a1, a2, a3;
@@ -673,7 +707,7 @@ cudaError_t launch_score_tc(const Launch& L, const float* lse_in, float* s, floa
     {
         cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)sh.rows, (cuuint64_t)sh.n_units};
         cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)sh.rows * kD * 2};
-        cuuint32_t box[3] = {64, 256, 1};
+        cuuint32_t box[3] = {64, 128, 1};
         cuuint32_t estr[3] = {1, 1, 1};
         if (encode(&tmQ, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(L.q), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,

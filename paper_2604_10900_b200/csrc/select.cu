@@ -44,13 +44,13 @@ __global__ void __launch_bounds__(kSelThreads) select_core_kernel(const UnitDesc
 
 cudaError_t launch_prefix_evict(const Launch& L, const float* s, uint8_t* kind, int32_t* plan) {
     Timed t(L, KID_PREFIX_EVICT);
-    prefix_evict_kernel<<<L.sh.n_units, kSelThreads, 0, L.stream>>>(L.desc, s, kind, plan);
+    prefix_evict_kernel<<<L.sh.n_units, select_threads(L.max_T), 0, L.stream>>>(L.desc, s, kind, plan);
     return cudaGetLastError();
 }
 
 cudaError_t launch_select_core(const Launch& L, const float* s, const int32_t* plan, uint8_t* kind) {
     Timed t(L, KID_SELECT_CORE);
-    select_core_kernel<<<L.sh.n_units, kSelThreads, 0, L.stream>>>(L.desc, s, plan, kind);
+    select_core_kernel<<<L.sh.n_units, select_threads(L.max_T), 0, L.stream>>>(L.desc, s, plan, kind);
     return cudaGetLastError();
 }
 

@@ -5,6 +5,9 @@
 // Three histogram sweeps narrow the key of the k-th greatest row digit by digit (12 + 12 + 8
 // bits), a last sweep marks everything above it and the rows equal to it.  The sweeps read the
 // unit's scores from global memory; after the first one they are L1/L2 hits.
+// Ranges of at most kSmallSpan rows skip the sweeps: their keys sit in shared memory and every
+// eligible row counts the rows ahead of it in the total order (same result, a few microseconds
+// instead of a dozen block-wide barriers).
 #pragma once
 #include "cask_internal.cuh"
 
@@ -12,6 +15,11 @@ namespace cask {
 
 constexpr int kSelThreads = 1024;
 constexpr int kSelBins = 4096;
+constexpr int kSmallSpan = 1024;       // rows; keys and eligibility flags fit SelectSmem::hist
+
+// Threads per selection CTA: small units take the counting path, which needs no 4096-bin histogram
+// (find_digit wants nbins <= 4 * blockDim.x) and leaves room for several CTAs per SM.
+inline int select_threads(int max_rows_per_unit) { return max_rows_per_unit <= kSmallSpan ? 256 : kSelThreads; }
 
 struct SelectSmem {
     unsigned hist[kSelBins];
@@ -95,6 +103,40 @@ __device__ inline void block_topk_mark(const float* __restrict__ s, uint8_t* kin
     const int tid = threadIdx.x, lane = tid & 31, nthr = blockDim.x;
     const int span = hi - lo;
     const int iters = (span + nthr - 1) / nthr;
+
+    if (span <= kSmallSpan) {
+        // ---- counting path: rank of every eligible row under (key descending, row ascending) ----
+        unsigned* keys = sm.hist;                         // [span] rounded up to a multiple of 4
+        unsigned* elig = sm.hist + kSmallSpan;            // one bit per row
+        const int span4 = (span + 3) & ~3;
+        for (int b = tid; b < (kSmallSpan >> 5); b += nthr) elig[b] = 0u;
+        __syncthreads();
+        for (int x = tid; x < span4; x += nthr) {
+            const bool el = x < span && kind[lo + x] == 0;
+            keys[x] = el ? order_key(s[lo + x]) : 0u;
+            if (el) atomicOr(&elig[x >> 5], 1u << (x & 31));
+        }
+        __syncthreads();
+        for (int x = tid; x < span; x += nthr) {
+            if (!((elig[x >> 5] >> (x & 31)) & 1u)) continue;
+            const unsigned ki = keys[x];
+            unsigned ahead = 0;
+            for (int j = 0; j < span4; j += 4) {
+                const uint4 kj = *reinterpret_cast<const uint4*>(keys + j);
+                ahead += (kj.x > ki) + (kj.y > ki) + (kj.z > ki) + (kj.w > ki);
+                if (kj.x == ki || kj.y == ki || kj.z == ki || kj.w == ki) {
+                    // equal keys ahead of this row: lower rows that are eligible themselves
+                    const unsigned kk[4] = {kj.x, kj.y, kj.z, kj.w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        ahead += (kk[q] == ki && j + q < x && ((elig[(j + q) >> 5] >> ((j + q) & 31)) & 1u));
+                }
+            }
+            if (ahead < (unsigned)k) kind[lo + x] = mark;
+        }
+        __syncthreads();
+        return;
+    }
 
     // ---- sweep 1: top 12 bits ----
     for (int b = tid; b < kSelBins; b += nthr) sm.hist[b] = 0;

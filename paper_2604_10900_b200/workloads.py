@@ -59,6 +59,8 @@ class Workload:
     noise: float = 0.05
     n_seqs: int = 1
     decode_min: int = 0   # >0: N_d ~ U{decode_min..decode} per sequence
+    carried_rows: int = 0     # >0: the first carried_rows rows are an earlier event's output and carry its masses
+    layers_per_pass: int = 0  # >0: the benchmark holds this many layers of every sequence on the device at once
 
     @property
     def n_units(self) -> int:
@@ -93,7 +95,12 @@ WORKLOADS: Dict[str, Workload] = {
                                 reserve=256),
     "batched_serving": _w("batched_serving", 5, layers=36, kv_heads=8, group=4, head_dim=128,
                           dtype=DTYPE_BF16, prefix=512, decode=32768, window=128, budget=512, reserve=256,
-                          n_seqs=64, decode_min=4096),
+                          n_seqs=64, decode_min=4096, layers_per_pass=6),
+    # The serving sweep in its steady state: every cache was compacted to B = 512 rows by an earlier event
+    # (256 prefix + 256 decode slots, carrying their group masses) and 128 decode steps have appended 128 rows.
+    "serving_steady_b512": _w("serving_steady_b512", 6, layers=36, kv_heads=8, group=4, head_dim=128,
+                              dtype=DTYPE_BF16, prefix=256, decode=384, window=128, budget=512, reserve=256,
+                              n_seqs=64, carried_rows=512),
 }
 
 
@@ -190,6 +197,20 @@ def make_unit(wl: Workload, seq: int, layer: int, head: int,
     return to_cache_dtype(k, wl.dtype), to_cache_dtype(v, wl.dtype), to_cache_dtype(q, wl.dtype)
 
 
+def make_mass(wl: Workload, seq: int, layer: int, head: int, T: int) -> np.ndarray:
+    """Carried masses of one unit: rows [0, carried_rows) hold the mass an earlier event left on them (a quarter
+    of the decode slots stand for groups of 2 + Geometric(p) rows), the appended rows hold none."""
+    rng = _rng(wl.cfg_id, seq, layer, head, 0xA5)
+    n = min(wl.carried_rows, T)
+    mass = np.zeros(T, dtype=np.float32)
+    base = rng.uniform(0.5, 1.5, size=n) / max(n, 1)
+    size = np.ones(n)
+    rep = (np.arange(n) >= wl.prefix) & (rng.random(n) < 0.25)
+    size[rep] = 2 + rng.geometric(wl.geometric_p, size=int(rep.sum()))
+    mass[:n] = (base * size).astype(np.float32)
+    return mass
+
+
 @dataclasses.dataclass
 class Batch:
     """A ragged batch of independent units, contiguous rows, host-resident."""
@@ -204,6 +225,7 @@ class Batch:
     reserve: np.ndarray      # int32 [n_units]
     tok_off: np.ndarray      # int64 [n_units+1]
     unit_ids: List[Tuple[int, int, int]]
+    mass_in: Optional[np.ndarray] = None   # float32 [sum T] carried masses, when the workload has them
 
     @property
     def n_units(self) -> int:
@@ -239,6 +261,7 @@ def make_batch(wl: Workload, units: Optional[List[Tuple[int, int, int]]] = None,
     k = alloc((int(tok_off[-1]), wl.head_dim), st)
     v = alloc((int(tok_off[-1]), wl.head_dim), st)
     q = np.empty((n, wl.group, wl.window, wl.head_dim), dtype=st)
+    mass = np.zeros(int(tok_off[-1]), dtype=np.float32) if wl.carried_rows > 0 else None
 
     def work(u: int) -> None:
         s, l, h = units[u]
@@ -247,6 +270,8 @@ def make_batch(wl: Workload, units: Optional[List[Tuple[int, int, int]]] = None,
         k[a:b] = ku
         v[a:b] = vu
         q[u] = qu
+        if mass is not None:
+            mass[a:b] = make_mass(wl, s, l, h, b - a)
 
     if threads > 1 and n > 1:
         with ThreadPoolExecutor(max_workers=threads) as ex:
@@ -258,7 +283,7 @@ def make_batch(wl: Workload, units: Optional[List[Tuple[int, int, int]]] = None,
                  P=np.full(n, wl.prefix, dtype=np.int32),
                  B=np.full(n, wl.budget, dtype=np.int32),
                  reserve=np.full(n, wl.reserve, dtype=np.int32),
-                 tok_off=tok_off, unit_ids=list(units))
+                 tok_off=tok_off, unit_ids=list(units), mass_in=mass)
 
 
 def shard_units(units: List[Tuple[int, int, int]], rank: int, world: int) -> List[Tuple[int, int, int]]:

@@ -28,6 +28,8 @@ WEIGHT_RTOL = 2e-5
 def run_oracle(hb: wl.Batch, **kw) -> Dict:
     """kw: tau, gamma, causal, eps, mass_in (per-row carried masses), chan_w (similarity channel weights)."""
     w = hb.wl
+    if hb.mass_in is not None:
+        kw.setdefault("mass_in", hb.mass_in)
     return orc.event_batch(wl.as_float32(hb.k, w.dtype), wl.as_float32(hb.v, w.dtype),
                            wl.as_float32(hb.q, w.dtype), hb.tok_off, hb.P, hb.B, hb.reserve, **kw)
 
@@ -41,6 +43,8 @@ class GpuRun:
         from paper_2604_10900_b200 import binding as cb
         self.cb, self.torch, self.hb = cb, torch, hb
         w = hb.wl
+        if mass_in is None:
+            mass_in = hb.mass_in
         self.device = device
         self.dev = cb.to_device(hb, device)
         d = w.head_dim

@@ -126,3 +126,12 @@ def test_batched_serving_ragged_slice():
     sample = sorted({int(np.argmin(T)), int(np.argmax(T)), int(np.argsort(T)[len(T) // 2])})
     st = _full("batched_serving", sample, units)
     assert st["max_score_rel"] < 1e-5
+
+
+def test_serving_steady_state_slice():
+    """The serving sweep's steady state: 64 sequences x 4 layers x 8 KV heads = 2,048 caches of 640 rows (512
+    compacted rows carrying their masses + 128 appended ones) in one launch; three of them through the oracle."""
+    w = wl.WORKLOADS["serving_steady_b512"]
+    units = wl.unit_list(w, layers=range(4))
+    st = _full("serving_steady_b512", [0, 1023, 2047], units)
+    assert st["max_score_rel"] < 1e-5
