@@ -1,7 +1,7 @@
 // Compaction to the budget (Sec. 2.3: |R| <= B) with the weighted K/V merge of Sec. 2.4:
 //   slot order = ascending anchor row; kinds 1..3 and lone seeds are byte copies;
 //   a seed with joiners holds sum_i w_i k_i, sum_i w_i v_i (members in ascending row order).
-#include "cask_internal.cuh"
+#include "tc_common.cuh"
 
 namespace cask {
 
@@ -166,62 +166,87 @@ __global__ void __launch_bounds__(kScanThreads) slot_scan_kernel(
     }
 }
 
-// ---- 2. byte copy of every slot's anchor row: one thread per 16-byte vector of K and of V ----
-// Flat over (unit, slot, vector) with four vectors in flight per thread, so that units of a few hundred
-// rows load the memory system as well as long ones.  The slot -> row lookups of the next round are issued
-// together with the row loads of the current one, so the two dependent levels overlap.
+// ---- 2. byte copy of every slot's anchor row by bulk async copies through shared memory ----
+// A warp owns batches of up to 32 consecutive slots of one unit.  Every lane starts the bulk copy of its slot's K
+// and V row (row bytes each, any source row) into the warp's staging buffer; when the batch has landed (mbarrier,
+// byte count) one lane writes it out with two bulk stores, because consecutive slots are contiguous in k_out and
+// v_out.  Two staging buffers per warp, so the loads of a batch run under the stores of the one before.  No
+// registers hold data, which leaves enough copies in flight to load HBM with units of a few hundred rows.
+constexpr int kCopyWarps = 6;
+constexpr int kCopyStageBytes = 16384;       // per warp and stage: K half + V half
+
+struct CopyCtl {
+    uint64_t bar[kCopyWarps][2];
+    int abort;
+};
+
 template <typename T>
-__global__ void __launch_bounds__(256) slot_copy_kernel(
+__global__ void __launch_bounds__(kCopyWarps * 32) slot_copy_kernel(
     const UnitDesc* __restrict__ desc, Shape sh, const T* __restrict__ K, const T* __restrict__ V,
     const float* __restrict__ s, float eps, int Bmax, int slots, const int32_t* __restrict__ n_out,
     const int32_t* __restrict__ slot_src, T* __restrict__ k_out, T* __restrict__ v_out,
     float* __restrict__ slot_mass) {
-    const int nvec = sh.d * (int)sizeof(T) / 16;              // 8, 16 or 32
-    const int nvec_log2 = 31 - __clz(nvec);
-    const int64_t total = (int64_t)sh.n_units * slots * nvec;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    constexpr int kFly = 4;
-    // (unit, slot, row) of the kFly vectors of one round; row < 0: nothing to copy
-    struct Item { int u, t, src; };
-    auto lookup = [&](int64_t g) {
-        Item it{0, 0, -1};
-        if (g < total) {
-            // nvec is a power of two; units x slots stays far below 2^32 (the outputs alone would not fit the device)
-            const unsigned sg = (unsigned)(g >> nvec_log2);
-            it.u = (int)(sg / (unsigned)slots);
-            it.t = (int)(sg - (unsigned)it.u * (unsigned)slots);
-            if (it.t < n_out[it.u]) it.src = slot_src[(size_t)it.u * Bmax + it.t];
+    using namespace tc;
+    extern __shared__ __align__(128) uint8_t copy_smem[];
+    __shared__ CopyCtl ctl;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const uint32_t row_bytes = (uint32_t)(sh.d * sizeof(T));
+    const int sb = min(32, (int)(kCopyStageBytes / 2 / row_bytes));     // slots per batch
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kCopyWarps; ++i) { mbar_init(&ctl.bar[i][0], 1); mbar_init(&ctl.bar[i][1], 1); }
+        ctl.abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    volatile int* abort_flag = &ctl.abort;
+    uint8_t* my = copy_smem + (size_t)w * 2 * kCopyStageBytes;
+    const int bpu = (slots + sb - 1) / sb;                               // batches per unit
+    const int64_t total = (int64_t)sh.n_units * bpu;
+    uint32_t it = 0;
+    bool ok = true;
+    for (int64_t bi = (int64_t)blockIdx.x * kCopyWarps + w; bi < total && ok; bi += (int64_t)gridDim.x * kCopyWarps) {
+        const int u = (int)(bi / bpu), t0 = (int)(bi - (int64_t)u * bpu) * sb;
+        const int nv = min(sb, n_out[u] - t0);
+        if (nv <= 0) continue;
+        const UnitDesc& ud = desc[u];
+        const uint32_t st = it & 1u;
+        uint8_t* kbuf = my + st * kCopyStageBytes;
+        uint8_t* vbuf = kbuf + kCopyStageBytes / 2;
+        // the stores that read this buffer two batches ago must have read it
+        if (lane == 0) {
+            asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+            mbar_expect_tx(&ctl.bar[w][st], (uint32_t)nv * 2u * row_bytes);
         }
-        return it;
-    };
-    int64_t g0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    Item cur[kFly];
-#pragma unroll
-    for (int q = 0; q < kFly; ++q) cur[q] = lookup(g0 + q * stride);
-    for (; g0 < total; g0 += kFly * stride) {
-        uint4 kv[kFly], vv[kFly];
-        const int c = (int)(g0 & (nvec - 1));                 // the same for the whole round: stride is a multiple of nvec
-#pragma unroll
-        for (int q = 0; q < kFly; ++q) {
-            if (cur[q].src < 0) continue;
-            const UnitDesc& ud = desc[cur[q].u];
-            kv[q] = reinterpret_cast<const uint4*>(K + row_elem_off(sh, ud, ud.k_off, cur[q].src))[c];
-            vv[q] = reinterpret_cast<const uint4*>(V + v_elem_off(sh, ud, cur[q].u, cur[q].src))[c];
-            if (c == 0)
-                slot_mass[(size_t)cur[q].u * Bmax + cur[q].t] = row_mass(sh, s, eps, ud.tok_off + cur[q].src);
+        __syncwarp();
+        if (lane < nv) {
+            const int src = slot_src[(size_t)u * Bmax + t0 + lane];
+            const T* kr = K + row_elem_off(sh, ud, ud.k_off, src);
+            const T* vr = V + v_elem_off(sh, ud, u, src);
+            const uint32_t bar = smem_u32(&ctl.bar[w][st]);
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(smem_u32(kbuf + lane * row_bytes)), "l"(kr), "r"(row_bytes), "r"(bar) : "memory");
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(smem_u32(vbuf + lane * row_bytes)), "l"(vr), "r"(row_bytes), "r"(bar) : "memory");
+            slot_mass[(size_t)u * Bmax + t0 + lane] = row_mass(sh, s, eps, ud.tok_off + src);
         }
-        Item nxt[kFly];
-#pragma unroll
-        for (int q = 0; q < kFly; ++q) nxt[q] = lookup(g0 + (kFly + q) * stride);
-#pragma unroll
-        for (int q = 0; q < kFly; ++q) {
-            if (cur[q].src >= 0) {
-                const int64_t dst = ((int64_t)cur[q].u * Bmax + cur[q].t) * nvec + c;
-                reinterpret_cast<uint4*>(k_out)[dst] = kv[q];
-                reinterpret_cast<uint4*>(v_out)[dst] = vv[q];
-            }
-            cur[q] = nxt[q];
+        ok = mbar_wait(&ctl.bar[w][st], (it >> 1) & 1u, abort_flag);
+        if (!ok) break;
+        if (lane == 0) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            const size_t dst = ((size_t)u * Bmax + t0) * sh.d;
+            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                         ::"l"(k_out + dst), "r"(smem_u32(kbuf)), "r"((uint32_t)nv * row_bytes) : "memory");
+            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                         ::"l"(v_out + dst), "r"(smem_u32(vbuf)), "r"((uint32_t)nv * row_bytes) : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         }
+        ++it;
+    }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (!ok && lane == 0) {
+        // a copy that was started may still be landing: give the two barriers a bounded chance to complete
+        for (uint32_t k = 0; k < 4096 && !mbar_try(&ctl.bar[w][it & 1u], (it >> 1) & 1u); ++k) {}
+        atomicOr(sh.err, CASK_ST_TIMEOUT);
     }
 }
 
@@ -292,10 +317,10 @@ __global__ void __launch_bounds__(256) slot_merge_kernel(
 // Same arithmetic as slot_merge_kernel (members in ascending row order, one fp32 accumulator per channel),
 // but a warp first lists the members of its representative from shared memory and then reads their rows four
 // at a time, instead of walking the unit's whole member list in global memory with one row in flight.
-constexpr int kMergeStageRows = 2048;
+constexpr int kMergeStageRows = 1024;
 
 template <typename T, int CH>       // CH = d / 32 contiguous channels per lane
-__global__ void __launch_bounds__(256) slot_merge_small_kernel(
+__global__ void __launch_bounds__(256, 4) slot_merge_small_kernel(
     const UnitDesc* __restrict__ desc, Shape sh, const T* __restrict__ K, const T* __restrict__ V,
     const float* __restrict__ s, const float* __restrict__ weight, float eps, int Bmax,
     const int32_t* __restrict__ seed_slot, const int32_t* __restrict__ n_seed, int max_B,
@@ -304,13 +329,15 @@ __global__ void __launch_bounds__(256) slot_merge_small_kernel(
     float* __restrict__ slot_mass) {
     __shared__ int32_t m_row[kMergeStageRows], m_slot[kMergeStageRows];
     __shared__ float m_w[kMergeStageRows], m_a[kMergeStageRows];
+    __shared__ int32_t s_slot[kMergeStageRows];      // slot of every representative of the unit
     __shared__ int32_t b_e[8][32];
     const int u = blockIdx.x;
     const UnitDesc& ud = desc[u];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
     const int64_t o = ud.tok_off;
     const int nm = min(n_mem[u], kMergeStageRows);
-    const int ns = n_seed[u];
+    const int ns = min(n_seed[u], kMergeStageRows);
+    for (int j = threadIdx.x; j < ns; j += blockDim.x) s_slot[j] = seed_slot[(size_t)u * max_B + j];
     for (int e = threadIdx.x; e < nm; e += blockDim.x) {
         const int row = mem_row[o + e];
         m_row[e] = row;
@@ -321,7 +348,7 @@ __global__ void __launch_bounds__(256) slot_merge_small_kernel(
     __syncthreads();
     struct alignas(CH * sizeof(T)) Vec { T x[CH]; };
     for (int j = w; j < ns; j += nw) {
-        const int t = seed_slot[(size_t)u * max_B + j];
+        const int t = s_slot[j];
         float ak[CH], av[CH];
 #pragma unroll
         for (int x = 0; x < CH; ++x) { ak[x] = 0.f; av[x] = 0.f; }
@@ -465,10 +492,14 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const u
     {
         // the merge kernel overwrites slots the copy kernel wrote: same stream, in order
         Timed t(L, KID_GATHER_MERGE);
-        const int nvec = sh.d * (int)sizeof(T) / 16;
-        const int64_t vecs = (int64_t)sh.n_units * slots * nvec;
-        const int copy_grid = (int)std::min<int64_t>((vecs + 256 * 4 - 1) / (256 * 4), 148 * 64);
-        slot_copy_kernel<T><<<std::max(copy_grid, 1), 256, 0, L.stream>>>(
+        const int sb = std::min(32, (int)(kCopyStageBytes / 2 / (sh.d * sizeof(T))));
+        const int64_t batches = (int64_t)sh.n_units * ((slots + sb - 1) / sb);
+        const int copy_smem_bytes = kCopyWarps * 2 * kCopyStageBytes;
+        cudaError_t ce = cudaFuncSetAttribute(slot_copy_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              copy_smem_bytes);
+        if (ce != cudaSuccess) return ce;
+        const int copy_grid = (int)std::min<int64_t>((batches + kCopyWarps - 1) / kCopyWarps, 148);   // one CTA per SM
+        slot_copy_kernel<T><<<std::max(copy_grid, 1), kCopyWarps * 32, copy_smem_bytes, L.stream>>>(
             L.desc, sh, (const T*)L.k, (const T*)L.v, s, prm.eps, out.Bmax, slots, out.n_out, out.slot_src,
             (T*)out.k_out, (T*)out.v_out, out.slot_mass);
         if (L.max_T <= kMergeStageRows && (sh.d == 64 || sh.d == 128)) {
