@@ -512,7 +512,7 @@ static int event_decide(cask_ctx* ctx, Launch& L, Workspace& W, const cask_batch
     float* s = out->s ? out->s : W.s;
     int rc = run_score(ctx, L, b, p, s, out->lse, W);
     if (rc != CASK_OK) return rc;
-    const bool small = L.max_T <= kSmallUnitRows;      // one fused selection kernel per unit
+    const bool small = L.max_T <= kSmallUnitRows && L.sh.d <= 128;      // one fused selection kernel per unit
     cudaError_t e = cudaSuccess;
     if (!small) {
         e = launch_prefix_evict(L, s, out->kind, out->plan);

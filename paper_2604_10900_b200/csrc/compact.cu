@@ -313,10 +313,11 @@ __global__ void __launch_bounds__(256) slot_merge_kernel(
     }
 }
 
-// ---- 3b. units of at most kMergeStageRows rows: one CTA per unit, member list staged in shared memory ----
-// Same arithmetic as slot_merge_kernel (members in ascending row order, one fp32 accumulator per channel),
-// but a warp first lists the members of its representative from shared memory and then reads their rows four
-// at a time, instead of walking the unit's whole member list in global memory with one row in flight.
+// ---- 3b. units of at most kMergeStageRows rows: one CTA per unit, members sorted by representative in shared memory ----
+// Same arithmetic as slot_merge_kernel (members in ascending row order, one fp32 accumulator per channel).  The
+// unit's member list is staged once and sorted by representative with a stable counting sort (one warp places
+// 32 members per step: __match_any_sync gives every member its rank among the members of the same group in the
+// step), so a warp finds the members of its representative side by side and reads their rows four at a time.
 constexpr int kMergeStageRows = 1024;
 
 template <typename T, int CH>       // CH = d / 32 contiguous channels per lane
@@ -327,83 +328,113 @@ __global__ void __launch_bounds__(256, 4) slot_merge_small_kernel(
     const int32_t* __restrict__ mem_row, const int32_t* __restrict__ mem_slot,
     const int32_t* __restrict__ n_mem, T* __restrict__ k_out, T* __restrict__ v_out,
     float* __restrict__ slot_mass) {
-    __shared__ int32_t m_row[kMergeStageRows], m_slot[kMergeStageRows];
-    __shared__ float m_w[kMergeStageRows], m_a[kMergeStageRows];
-    __shared__ int32_t s_slot[kMergeStageRows];      // slot of every representative of the unit
-    __shared__ int32_t b_e[8][32];
+    constexpr int R = kMergeStageRows;
+    __shared__ int32_t m_row[R], list[R], s_slot[R], start[R + 1], fill[R];
+    __shared__ int16_t m_j[R], inv[R];
+    __shared__ float m_w[R], m_a[R];
+    __shared__ int32_t wsum[8];
     const int u = blockIdx.x;
     const UnitDesc& ud = desc[u];
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5, nw = blockDim.x >> 5;
     const int64_t o = ud.tok_off;
-    const int nm = min(n_mem[u], kMergeStageRows);
-    const int ns = min(n_seed[u], kMergeStageRows);
-    for (int j = threadIdx.x; j < ns; j += blockDim.x) s_slot[j] = seed_slot[(size_t)u * max_B + j];
-    for (int e = threadIdx.x; e < nm; e += blockDim.x) {
-        const int row = mem_row[o + e];
+    const int nm = min(n_mem[u], R);
+    const int ns = min(n_seed[u], R);
+    for (int t = tid; t < R; t += blockDim.x) { inv[t] = -1; fill[t] = 0; }
+    __syncthreads();
+    for (int j = tid; j < ns; j += blockDim.x) {
+        const int t = seed_slot[(size_t)u * max_B + j];
+        s_slot[j] = t;
+        if (t >= 0 && t < R) inv[t] = (int16_t)j;
+    }
+    __syncthreads();
+    for (int e = tid; e < nm; e += blockDim.x) {
+        const int row = mem_row[o + e], t = mem_slot[o + e];
+        const int j = (t >= 0 && t < R) ? inv[t] : -1;
         m_row[e] = row;
-        m_slot[e] = mem_slot[o + e];
+        m_j[e] = (int16_t)j;
         m_w[e] = weight[o + row];
         m_a[e] = row_mass(sh, s, eps, o + row);
+        if (j >= 0) atomicAdd(&fill[j], 1);
+    }
+    __syncthreads();
+    {   // start[j] = members of the representatives before j (exclusive scan of the counts)
+        const int per = (ns + (int)blockDim.x - 1) / (int)blockDim.x;
+        const int j0 = tid * per, j1 = min(ns, j0 + per);
+        int sum = 0;
+        for (int j = j0; j < j1; ++j) sum += fill[j];
+        int incl = sum;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += v;
+        }
+        if (lane == 31) wsum[w] = incl;
+        __syncthreads();
+        int run = incl - sum;
+        for (int x = 0; x < w; ++x) run += wsum[x];
+        for (int j = j0; j < j1; ++j) {
+            start[j] = run;
+            run += fill[j];
+            fill[j] = 0;
+        }
+        if (tid == (int)blockDim.x - 1) start[ns] = run;      // the last thread ends on the total
+    }
+    __syncthreads();
+    if (w == 0) {
+        // stable placement, 32 members per step in ascending row order
+        for (int e0 = 0; e0 < nm; e0 += 32) {
+            const int e = e0 + lane;
+            const int j = (e < nm) ? (int)m_j[e] : -1;
+            const unsigned peers = __match_any_sync(0xffffffffu, j);
+            const unsigned below = peers & ((1u << lane) - 1u);
+            if (j >= 0) list[start[j] + fill[j] + __popc(below)] = e;
+            __syncwarp();
+            if (j >= 0 && below == 0u) fill[j] += __popc(peers);
+            __syncwarp();
+        }
     }
     __syncthreads();
     struct alignas(CH * sizeof(T)) Vec { T x[CH]; };
     for (int j = w; j < ns; j += nw) {
+        const int first = start[j], count = start[j + 1] - first;
+        if (count <= 1) continue;       // a lone seed keeps its byte copy
         const int t = s_slot[j];
         float ak[CH], av[CH];
 #pragma unroll
         for (int x = 0; x < CH; ++x) { ak[x] = 0.f; av[x] = 0.f; }
-        int count = 0, held = 0;
         float msum = 0.f;
-        auto flush = [&]() {
-            __syncwarp();
-            for (int h0 = 0; h0 < held; h0 += 4) {
-                Vec kr[4], vr[4];
-                float wi[4];
+        for (int h0 = 0; h0 < count; h0 += 4) {
+            Vec kr[4], vr[4];
+            float wi[4], ai[4];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const int e = b_e[w][min(h0 + q, held - 1)];
-                    const int i = m_row[e];
-                    wi[q] = m_w[e];
-                    kr[q] = reinterpret_cast<const Vec*>(K + row_elem_off(sh, ud, ud.k_off, i))[lane];
-                    vr[q] = reinterpret_cast<const Vec*>(V + v_elem_off(sh, ud, u, i))[lane];
-                }
+            for (int q = 0; q < 4; ++q) {
+                const int e = list[first + min(h0 + q, count - 1)];
+                const int i = m_row[e];
+                wi[q] = m_w[e];
+                ai[q] = m_a[e];
+                kr[q] = reinterpret_cast<const Vec*>(K + row_elem_off(sh, ud, ud.k_off, i))[lane];
+                vr[q] = reinterpret_cast<const Vec*>(V + v_elem_off(sh, ud, u, i))[lane];
+            }
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    if (h0 + q >= held) break;
-                    msum += m_a[b_e[w][h0 + q]];
+            for (int q = 0; q < 4; ++q) {
+                if (h0 + q >= count) break;
+                msum += ai[q];
 #pragma unroll
-                    for (int x = 0; x < CH; ++x) {
-                        ak[x] = fmaf(wi[q], Elem<T>::ld(&kr[q].x[x]), ak[x]);
-                        av[x] = fmaf(wi[q], Elem<T>::ld(&vr[q].x[x]), av[x]);
-                    }
+                for (int x = 0; x < CH; ++x) {
+                    ak[x] = fmaf(wi[q], Elem<T>::ld(&kr[q].x[x]), ak[x]);
+                    av[x] = fmaf(wi[q], Elem<T>::ld(&vr[q].x[x]), av[x]);
                 }
             }
-            count += held;
-            held = 0;
-            __syncwarp();
-        };
-        for (int e0 = 0; e0 < nm; e0 += 32) {
-            const int e = e0 + lane;
-            const bool hit = (e < nm) && m_slot[e] == t;
-            const unsigned bal = __ballot_sync(0xffffffffu, hit);
-            const int n = __popc(bal);
-            if (n == 0) continue;
-            if (held + n > 32) flush();
-            if (hit) b_e[w][held + __popc(bal & ((1u << lane) - 1u))] = e;
-            held += n;
         }
-        flush();
-        if (count > 1) {       // a lone seed keeps its byte copy
-            Vec ko, vo;
+        Vec ko, vo;
 #pragma unroll
-            for (int x = 0; x < CH; ++x) {
-                Elem<T>::st(&ko.x[x], ak[x]);
-                Elem<T>::st(&vo.x[x], av[x]);
-            }
-            reinterpret_cast<Vec*>(k_out + ((size_t)u * Bmax + t) * sh.d)[lane] = ko;
-            reinterpret_cast<Vec*>(v_out + ((size_t)u * Bmax + t) * sh.d)[lane] = vo;
-            if (lane == 0) slot_mass[(size_t)u * Bmax + t] = msum;
+        for (int x = 0; x < CH; ++x) {
+            Elem<T>::st(&ko.x[x], ak[x]);
+            Elem<T>::st(&vo.x[x], av[x]);
         }
+        reinterpret_cast<Vec*>(k_out + ((size_t)u * Bmax + t) * sh.d)[lane] = ko;
+        reinterpret_cast<Vec*>(v_out + ((size_t)u * Bmax + t) * sh.d)[lane] = vo;
+        if (lane == 0) slot_mass[(size_t)u * Bmax + t] = msum;
     }
 }
 

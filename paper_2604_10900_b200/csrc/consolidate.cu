@@ -1,5 +1,7 @@
 // Scratch consolidation (Sec. 2.1, 2.4, 2.5): seed selection, cosine assignment of the
 // remaining scratch rows to seeds, group masses and merge weights.
+#include <type_traits>
+
 #include "select.cuh"
 
 namespace cask {
@@ -97,13 +99,13 @@ __global__ void seed_gather_kernel(const UnitDesc* __restrict__ desc, Shape sh, 
 // order (score descending, row ascending), so the c greatest rows of the scratch range are the core and the next
 // m the seeds, which is what taking the top c and then the top m of the rest gives.
 template <typename T>
-__global__ void __launch_bounds__(256) decide_small_kernel(
+__global__ void __launch_bounds__(256, 6) decide_small_kernel(
     const UnitDesc* __restrict__ desc, Shape sh, const T* __restrict__ K, const float* __restrict__ s,
     int32_t* __restrict__ plan, uint8_t* __restrict__ kind, int32_t* __restrict__ seed_of,
     float* __restrict__ weight, float* __restrict__ sim, int32_t* __restrict__ grp,
     int32_t* __restrict__ seed_rows, T* __restrict__ seed_k, float* __restrict__ seed_norm,
     unsigned long long* __restrict__ mass_fx, int32_t* __restrict__ njoin, int max_m, float eps, int split_rows) {
-    __shared__ unsigned keys[kSmallSpan];
+    __shared__ __align__(16) unsigned keys[kSmallSpan];
     __shared__ int32_t seed_list[kSmallSpan];
     __shared__ uint8_t kd[kSmallSpan];
     __shared__ unsigned wsum[8];
@@ -120,13 +122,23 @@ __global__ void __launch_bounds__(256) decide_small_kernel(
         kd[i] = (i < P) ? pre : (i >= T_ - r ? CASK_KIND_RECENT : CASK_KIND_DROPPED);
     }
     __syncthreads();
-    // rows of [lo, hi) ahead of row i: greater keys, and equal keys at lower rows
+    // rows of [lo, hi) ahead of row i: greater keys, and equal keys at lower rows.  Four keys per shared-memory
+    // load wherever the index is a multiple of four (the key array is 16-byte aligned).
+    auto count = [&](int a, int b, unsigned ki, auto ge) {       // #{j in [a,b): keys[j] >= ki (ge) or > ki}
+        constexpr bool GE = decltype(ge)::value;
+        int n = 0, j = a;
+        for (; j < b && (j & 3); ++j) n += GE ? keys[j] >= ki : keys[j] > ki;
+        for (; j + 4 <= b; j += 4) {
+            const uint4 k4 = *reinterpret_cast<const uint4*>(&keys[j]);
+            if (GE) n += (k4.x >= ki) + (k4.y >= ki) + (k4.z >= ki) + (k4.w >= ki);
+            else n += (k4.x > ki) + (k4.y > ki) + (k4.z > ki) + (k4.w > ki);
+        }
+        for (; j < b; ++j) n += GE ? keys[j] >= ki : keys[j] > ki;
+        return n;
+    };
     auto ahead_of = [&](int lo, int hi, int i) {
         const unsigned ki = keys[i];
-        int a = 0;
-        for (int j = lo; j < i; ++j) a += keys[j] >= ki;
-        for (int j = i + 1; j < hi; ++j) a += keys[j] > ki;
-        return a;
+        return count(lo, i, ki, std::true_type{}) + count(i + 1, hi, ki, std::false_type{});
     };
     if (P > pkeep && pkeep > 0)
         for (int i = tid; i < P; i += blockDim.x)
@@ -178,30 +190,48 @@ __global__ void __launch_bounds__(256) decide_small_kernel(
     unsigned n_seeds = 0;
     for (int x = 0; x < (int)(blockDim.x >> 5); ++x) n_seeds += wsum[x];
     const int ms = min((int)n_seeds, m);
-    // gather the seed keys, their norms and their own mass: one warp per seed
-    for (int j = w; j < ms; j += (int)(blockDim.x >> 5)) {
-        const int row = seed_list[j];
-        const T* src = K + row_elem_off(sh, ud, ud.k_off, row);
-        T* dst = seed_k + (size_t)(ud.seed_base + j) * (split_rows ? 2 : 1) * sh.d;
-        float n2 = 0.f;
-        for (int ch = lane; ch < sh.d; ch += 32) {
-            T x = src[ch];
-            float f = Elem<T>::ld(&x);
-            const float wc = sh.chan_w ? sh.chan_w[ch] : 1.f;
-            if (split_rows) {
-                const float wf = wc * f;
-                Elem<T>::st(dst + ch, wf);
-                Elem<T>::st(dst + sh.d + ch, wf - Elem<T>::ld(dst + ch));
-            } else {
-                dst[ch] = x;
-            }
-            n2 = fmaf(wc * f, f, n2);
+    // gather the seed keys, their norms and their own mass: one warp per seed, two seeds' rows in flight
+    const int nwarps = (int)(blockDim.x >> 5);
+    constexpr int kPerLane = 4;                       // head_dim <= 128: at most four channels per lane
+    for (int j0 = w; j0 < ms; j0 += 2 * nwarps) {
+        T x[2][kPerLane];
+        int row[2];
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const int j = j0 + q * nwarps;
+            row[q] = seed_list[min(j, ms - 1)];
+            const T* src = K + row_elem_off(sh, ud, ud.k_off, row[q]);
+#pragma unroll
+            for (int k = 0; k < kPerLane; ++k)
+                if (lane + 32 * k < sh.d) x[q][k] = src[lane + 32 * k];
         }
 #pragma unroll
-        for (int off = 16; off >= 1; off >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, off);
-        if (lane == 0) {
-            seed_norm[ud.seed_base + j] = sqrtf(n2);
-            mass_fx[(size_t)u * (max_m + 1) + j] = mass_to_fx(row_mass(sh, s, eps, o + row));
+        for (int q = 0; q < 2; ++q) {
+            const int j = j0 + q * nwarps;
+            if (j >= ms) break;
+            T* dst = seed_k + (size_t)(ud.seed_base + j) * (split_rows ? 2 : 1) * sh.d;
+            float n2 = 0.f;
+#pragma unroll
+            for (int k = 0; k < kPerLane; ++k) {
+                const int ch = lane + 32 * k;
+                if (ch >= sh.d) break;
+                const float f = Elem<T>::ld(&x[q][k]);
+                const float wc = sh.chan_w ? sh.chan_w[ch] : 1.f;
+                if (split_rows) {
+                    const float wf = wc * f;
+                    Elem<T>::st(dst + ch, wf);
+                    Elem<T>::st(dst + sh.d + ch, wf - Elem<T>::ld(dst + ch));
+                } else {
+                    dst[ch] = x[q][k];
+                }
+                n2 = fmaf(wc * f, f, n2);
+            }
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, off);
+            if (lane == 0) {
+                seed_norm[ud.seed_base + j] = sqrtf(n2);
+                mass_fx[(size_t)u * (max_m + 1) + j] = mass_to_fx(row_mass(sh, s, eps, o + row[q]));
+            }
         }
     }
 }

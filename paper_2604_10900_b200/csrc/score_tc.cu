@@ -198,13 +198,16 @@ __device__ __forceinline__ void norm_block(const float (&v)[32], bool fast, int 
     }
 }
 
-// Walks this CTA's contiguous range of key tiles, segment by segment.
+// Walks this CTA's contiguous range of key tiles, segment by segment.  The next unit's descriptor fields are
+// fetched a segment ahead, so a change of segment costs no memory round trip.
 struct TileWalk {
     const UnitDesc* desc;
-    int t, t_end, u;
+    int t, t_end, u, n_units;
     int tile0, n_tiles, T;
-    __device__ void init(const UnitDesc* d, int n_units, int total_tiles) {
+    int nx_tile0, nx_T;
+    __device__ void init(const UnitDesc* d, int units, int total_tiles) {
         desc = d;
+        n_units = units;
         t = (int)(((long long)total_tiles * blockIdx.x) / gridDim.x);
         t_end = (int)(((long long)total_tiles * (blockIdx.x + 1)) / gridDim.x);
         int lo = 0, hi = n_units - 1;
@@ -213,19 +216,29 @@ struct TileWalk {
             if (d[mid].tile0 <= t) lo = mid; else hi = mid - 1;
         }
         u = lo;
-        load();
-    }
-    __device__ void load() {
         tile0 = desc[u].tile0;
         T = desc[u].T;
         n_tiles = (T + kTileKeys - 1) / kTileKeys;
+        prefetch();
+    }
+    __device__ void prefetch() {
+        const int v = min(u + 1, n_units - 1);
+        nx_tile0 = desc[v].tile0;
+        nx_T = desc[v].T;
     }
     __device__ bool valid() const { return t < t_end; }
     __device__ int key_begin() const { return (t - tile0) * kTileKeys; }
     __device__ int seg_tiles() const { return min(t_end, tile0 + n_tiles) - t; }
+    __device__ bool has_next() const { return t + seg_tiles() < t_end; }
     __device__ void next_segment() {
         t += seg_tiles();
-        if (t < t_end) { ++u; load(); }
+        if (t < t_end) {
+            ++u;
+            tile0 = nx_tile0;
+            T = nx_T;
+            n_tiles = (T + kTileKeys - 1) / kTileKeys;
+            prefetch();
+        }
     }
 };
 
@@ -408,11 +421,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 // tile, when the loads have long landed.  Whoever passed the wait above knows that every thread
                 // is past the first tile of the previous segment, so nobody still reads the buffer of the segment
                 // before that one, which is the one written next.
-                TileWalk nx = wk;
-                nx.next_segment();
-                has_next = nx.valid();
+                has_next = wk.has_next();
                 if (has_next && etid < rows)
-                    rc_next = log2f(roww[(size_t)nx.u * rows + etid]) - rowm[(size_t)nx.u * rows + etid];
+                    rc_next = log2f(roww[(size_t)(wk.u + 1) * rows + etid]) - rowm[(size_t)(wk.u + 1) * rows + etid];
             } else {
                 mm[0] = mm[1] = kNegBig;
                 l_run[0] = l_run[1] = 0.f;
