@@ -32,10 +32,10 @@ constexpr uint32_t kKRegionBytes = 128 * 128;
 constexpr uint32_t kKStageBytes = 2 * kKRegionBytes;
 
 struct __align__(8) ABarriers {
-    uint64_t b_full, b_empty;
+    uint64_t b_full[2], b_empty[2];   // seed matrix buffers (two when every unit has at most 128 columns)
     uint64_t k_full[kStages], k_empty[kStages];
     uint64_t d_full[kMaxGroups], d_empty[kMaxGroups];
-    uint64_t nu_ready;
+    uint64_t inv_ready[kMaxGroups];   // a group's table of inverse seed norms is written
     uint64_t x_full[2];      // shared buffers: the second group's best seed of a tile is in shared memory
 };
 
@@ -43,7 +43,8 @@ struct ASmemTail {
     ABarriers bar;
     uint32_t tmem_base;
     int abort;
-    float inv_nu[2][256];     // 1/|k_seed| (0 for a zero seed), double-buffered by unit
+    float inv_nu[kMaxGroups][2][256];   // 1/|k_seed| (0 for a zero seed): every epilogue group keeps its own
+                                        // copy, double-buffered over the units it has tiles in
     alignas(16) float w[128]; // channel weights of the similarity (1 when none are given)
     float x_val[2][2][128];   // shared buffers: best dot product / seed norm and its seed,
     int x_idx[2][2][128];     //   per buffer, per use parity, per tile row
@@ -165,13 +166,16 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int buf_cols = 512 / n_bufs;                   // TMEM columns per accumulator buffer
     const int split = kMaxGroups / n_bufs;               // groups sharing one buffer (1 or 2)
+    // At most 128 accumulator columns in every unit: the seed matrix is loaded as 128 rows and the shared-memory
+    // area holds two of them, so the next unit's seeds arrive while the tensor pipe still works on this unit's.
+    const bool dual = n_bufs == kMaxGroups;
+    const uint32_t seed_region = dual ? 128u * 128u : kSeedRegionBytes;      // one 64-channel half of a seed buffer
 
     if (threadIdx.x == 0) {
-        mbar_init(&bar.b_full, 1);
-        mbar_init(&bar.b_empty, 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(&bar.b_full[i], 1); mbar_init(&bar.b_empty[i], 1); }
         for (int i = 0; i < kStages; ++i) { mbar_init(&bar.k_full[i], 1); mbar_init(&bar.k_empty[i], 1 + 4); }
         for (int i = 0; i < kMaxGroups; ++i) { mbar_init(&bar.d_full[i], 1); mbar_init(&bar.d_empty[i], 4 * split); }
-        mbar_init(&bar.nu_ready, 128 * kMaxGroups);
+        for (int i = 0; i < kMaxGroups; ++i) mbar_init(&bar.inv_ready[i], 128);
         mbar_init(&bar.x_full[0], 4);
         mbar_init(&bar.x_full[1], 4);
         tail->abort = 0;
@@ -197,11 +201,13 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             bool ok = true;
             while (wk.valid() && ok) {
                 const UnitDesc& ud = desc[wk.u];
-                ok = mbar_wait(&bar.b_empty, (ucount & 1u) ^ 1u, abort_flag);
+                const uint32_t sb = dual ? (ucount & 1u) : 0u, suse = dual ? (ucount >> 1) : ucount;
+                ok = mbar_wait(&bar.b_empty[sb], (suse & 1u) ^ 1u, abort_flag);
                 if (!ok) break;
-                mbar_expect_tx(&bar.b_full, kSeedBytes);
-                tma_load_2d(b_smem, &tmSeed, &bar.b_full, 0, ud.seed_base << wpair);
-                tma_load_2d(b_smem + kSeedRegionBytes, &tmSeed, &bar.b_full, 64, ud.seed_base << wpair);
+                mbar_expect_tx(&bar.b_full[sb], 2 * seed_region);
+                uint8_t* bdst = b_smem + sb * 2 * seed_region;
+                tma_load_2d(bdst, &tmSeed, &bar.b_full[sb], 0, ud.seed_base << wpair);
+                tma_load_2d(bdst + seed_region, &tmSeed, &bar.b_full[sb], 64, ud.seed_base << wpair);
                 ++ucount;
                 // first cache row of the unit's tile sequence (a page-piece boundary in a paged cache)
                 const int a0 = ud.P - (sh.page_size ? ud.P % sub_rows : 0);
@@ -245,9 +251,11 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 const UnitDesc& ud = desc[wk.u];
                 const int m = max(0, min(plan[wk.u * 8 + CASK_PLAN_M], ud.plan[CASK_PLAN_M]));
                 const uint32_t idesc = umma_idesc(max(16, ((m << wpair) + 15) & ~15));
-                ok = mbar_wait(&bar.b_full, ucount & 1u, abort_flag);
+                const uint32_t sb = dual ? (ucount & 1u) : 0u, suse = dual ? (ucount >> 1) : ucount;
+                ok = mbar_wait(&bar.b_full[sb], suse & 1u, abort_flag);
                 if (!ok) break;
                 ++ucount;
+                const uint32_t bu_lo = b_lo + ((sb * 2 * seed_region) >> 4), half_lo = seed_region >> 4;
                 const int nt = wk.run();
                 for (int t = 0; t < nt && ok; ++t, ++kit) {
                     const int st = kit % kStages;
@@ -259,18 +267,18 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     tc_fence_after();
                     const uint32_t kst_lo = k_lo + st * (kKStageBytes >> 4);
                     const uint32_t d_addr = tmem_base + buf * buf_cols;
-                    tc_mma_lo<false>(d_addr, kst_lo, b_lo, idesc);
+                    tc_mma_lo<false>(d_addr, kst_lo, bu_lo, idesc);
 #pragma unroll
                     for (int kk = 1; kk < 8; ++kk) {
                         const int kb = kk >> 2, ks = kk & 3;
                         tc_mma_lo<true>(d_addr, kst_lo + ((kb * kKRegionBytes + ks * 32) >> 4),
-                                        b_lo + ((kb * kSeedRegionBytes + ks * 32) >> 4), idesc);
+                                        bu_lo + kb * half_lo + ((ks * 32) >> 4), idesc);
                     }
                     tc_commit(&bar.d_full[buf]);
                     tc_commit(&bar.k_empty[st]);
                 }
                 wk.advance(nt);
-                if (ok) tc_commit(&bar.b_empty);
+                if (ok) tc_commit(&bar.b_empty[sb]);
             }
         }
     } else if (warp >= kEpiWarp0) {
@@ -279,7 +287,6 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         const int qd = ew & 3;                               // TMEM lane quadrant (== warp % 4)
         const uint32_t eg = (uint32_t)(ew >> 2) % (uint32_t)n_bufs;   // buffer: tiles eg, eg + n_bufs, ...
         const int half = (ew >> 2) / n_bufs;                 // 0: finishes the row; 1: the later seed columns only
-        const int etid = ew * 32 + lane;
         const uint32_t taddr = tmem_base + ((uint32_t)(32 * qd) << 16) + eg * buf_cols;
         const int my_row = 32 * qd + lane;                   // row of the tile this thread owns
         uint32_t kit = 0, ucount = 0;
@@ -298,17 +305,31 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const int mc = m << wpair;               // accumulator columns in use
             const int c_split = split == 2 ? min(mc, 32 * max(1, (((mc + 31) >> 5) - 2) / 2)) : mc;
             unsigned long long* mass_u = mass_fx + (size_t)u * (max_m + 1);
-            float* inv = tail->inv_nu[ucount & 1u];
-            if (etid < 256) {
-                const float nu = (etid < m) ? seed_norm[seed_base + etid] : 0.f;
-                inv[etid] = nu > 0.f ? 1.f / nu : 0.f;
-            }
-            mbar_arrive(&bar.nu_ready);
-            ok = mbar_wait(&bar.nu_ready, ucount & 1u, abort_flag);
-            if (!ok) break;
-            ++ucount;
             const int tile0 = wk.tile_in_unit();
             const int nt = wk.run();
+            // Does this group take a tile of the unit?  Only then it needs the table of inverse seed norms; it
+            // builds its own copy (two values per thread) and meets on its own barrier, so the groups never
+            // wait for one another between units.
+            const int first = (int)((eg + (uint32_t)n_bufs - kit % (uint32_t)n_bufs) % (uint32_t)n_bufs);
+            if (first >= nt) {
+                kit += nt;
+                wk.advance(nt);
+                continue;
+            }
+            float* inv = tail->inv_nu[ew >> 2][ucount & 1u];
+            {
+                const int gt = (ew & 3) * 32 + lane;           // thread of the group
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int c = gt + 128 * h;
+                    const float nu = (c < m) ? seed_norm[seed_base + c] : 0.f;
+                    inv[c] = nu > 0.f ? 1.f / nu : 0.f;
+                }
+                mbar_arrive(&bar.inv_ready[ew >> 2]);
+                ok = mbar_wait(&bar.inv_ready[ew >> 2], ucount & 1u, abort_flag);
+                if (!ok) break;
+            }
+            ++ucount;
             for (int t = 0; t < nt && ok; ++t, ++kit) {
                 if (kit % (uint32_t)n_bufs != eg) continue;
                 const int st = kit % kStages;
@@ -454,7 +475,8 @@ cudaError_t launch_assign_tc(const Launch& L, const cask_params& prm, const floa
         return cudaErrorInvalidValue;
     // the seed table has 256 spare rows behind the last seed, so a full box never leaves the allocation
     const int wpair = sh.chan_w ? 1 : 0;
-    if (!encode_rows_bf16(tmap_encode_fn, &tmSeed, ws.seed_k, ((uint64_t)sum_m << wpair) + 256, 256, 256))
+    const int n_bufs = (L.max_m << wpair) <= 128 ? 4 : 2;      // accumulator buffers; four: seed boxes of 128 rows
+    if (!encode_rows_bf16(tmap_encode_fn, &tmSeed, ws.seed_k, ((uint64_t)sum_m << wpair) + 256, 256, n_bufs == 4 ? 128 : 256))
         return cudaErrorInvalidValue;
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -467,7 +489,7 @@ cudaError_t launch_assign_tc(const Launch& L, const cask_params& prm, const floa
     {
         Timed t(L, KID_ASSIGN);
         assign_tc_kernel<<<grid, kThreadsA, kSmemBytesA, L.stream>>>(
-            tmK, tmSeed, L.desc, sh, L.total_atiles, (L.max_m << wpair) <= 128 ? 4 : 2, sub_rows, wpair, s, plan, ws.seed_rows, ws.seed_norm, kind, seed_of, sim, ws.grp,
+            tmK, tmSeed, L.desc, sh, L.total_atiles, n_bufs, sub_rows, wpair, s, plan, ws.seed_rows, ws.seed_norm, kind, seed_of, sim, ws.grp,
             ws.mass_fx, ws.njoin, L.max_m, prm.tau, prm.eps, ws.err);
     }
     return cudaGetLastError();

@@ -475,13 +475,28 @@ __global__ void __launch_bounds__(kScanThreads) value_rank_kernel(const UnitDesc
     if (threadIdx.x == 0) n_need[u] = (int)total;
 }
 
-__global__ void value_base_kernel(int n_units, const int32_t* __restrict__ n_need, int64_t* __restrict__ v_base) {
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        int64_t run = 0;
-        for (int u = 0; u < n_units; ++u) {
-            v_base[u] = run;
-            run += n_need[u];
-        }
+// v_base[u] = value rows needed by the units before u: one CTA, every thread a contiguous run of units.
+__global__ void __launch_bounds__(1024) value_base_kernel(int n_units, const int32_t* __restrict__ n_need,
+                                                          int64_t* __restrict__ v_base) {
+    __shared__ int64_t wsum[32];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int per = (n_units + (int)blockDim.x - 1) / (int)blockDim.x;
+    const int u0 = min(n_units, (int)threadIdx.x * per), u1 = min(n_units, u0 + per);
+    int64_t sum = 0;
+    for (int u = u0; u < u1; ++u) sum += n_need[u];
+    int64_t incl = sum;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int64_t v = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += v;
+    }
+    if (lane == 31) wsum[w] = incl;
+    __syncthreads();
+    int64_t run = incl - sum;
+    for (int x = 0; x < w; ++x) run += wsum[x];
+    for (int u = u0; u < u1; ++u) {
+        v_base[u] = run;
+        run += n_need[u];
     }
 }
 
@@ -553,7 +568,7 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const u
 cudaError_t launch_value_ranks(const Launch& L, const uint8_t* kind, int32_t* v_pos, int32_t* n_need, int64_t* v_base) {
     Timed t(L, KID_SLOT_SCAN);
     value_rank_kernel<<<L.sh.n_units, kScanThreads, 0, L.stream>>>(L.desc, kind, v_pos, n_need);
-    value_base_kernel<<<1, 32, 0, L.stream>>>(L.sh.n_units, n_need, v_base);
+    value_base_kernel<<<1, 1024, 0, L.stream>>>(L.sh.n_units, n_need, v_base);
     ++*L.launches;
     return cudaGetLastError();
 }
