@@ -133,9 +133,23 @@ __device__ __forceinline__ void mass_block(const float (&v)[32], const float* nc
         if (!causal || (W & 31) == 0) {
             // the 32 rows of the block lie inside one head (r0 is a multiple of 32): one threshold for the block
             const int thr = causal ? jmin - r0 % W : 0;
+            // arguments in packed pairs from 16-byte reads of the row table; only the exponentials of the visible
+            // columns are issued (the ex2 pipe is the bottleneck), into four independent sums
+            const float4* nc4 = reinterpret_cast<const float4*>(&nc[r0]);
+            const uint64_t s2 = pack2(scale2, scale2);
+            float b1 = 0.f, b2 = 0.f, b3 = 0.f;
 #pragma unroll
-            for (int x = 0; x < 32; ++x)
-                if (x >= thr) a += ex2(fmaf(v[x], scale2, nc[r0 + x]));
+            for (int x = 0; x < 8; ++x) {
+                const float4 c4 = nc4[x];
+                float t0, t1, t2, t3;
+                unpack2(fma2(pack2(v[4 * x], v[4 * x + 1]), s2, pack2(c4.x, c4.y)), t0, t1);
+                unpack2(fma2(pack2(v[4 * x + 2], v[4 * x + 3]), s2, pack2(c4.z, c4.w)), t2, t3);
+                if (4 * x >= thr) a += ex2(t0);
+                if (4 * x + 1 >= thr) b1 += ex2(t1);
+                if (4 * x + 2 >= thr) b2 += ex2(t2);
+                if (4 * x + 3 >= thr) b3 += ex2(t3);
+            }
+            a = (a + b1) + (b2 + b3);
         } else {
 #pragma unroll
             for (int x = 0; x < 32; ++x) {
