@@ -236,11 +236,17 @@ def test_supplied_normalisers():
     assert run.ctx.launches - n0 < run2.ctx.launches       # one pass fewer
 
 
-def test_deterministic_and_staged_equals_fused():
+@pytest.mark.parametrize("name,kw", [
+    ("reasoning8k_b384", dict(decode=1500)),
+    # units of at most 1,024 rows: the event takes its fused selection kernel, the staged calls their own kernels
+    ("reasoning8k_b384", dict(decode=600)),
+    ("prompt_heavy", dict(prefix=700, decode=200, budget=512, reserve=160)),     # with prefix eviction
+])
+def test_deterministic_and_staged_equals_fused(name, kw):
     """Same inputs twice -> same bytes; the five staged calls give the event's bytes."""
     import gpu_harness as gh
     import torch
-    w = _small("reasoning8k_b384", layers=1, kv_heads=2, decode=1500)
+    w = _small(name, layers=1, kv_heads=2, **kw)
     hb = wl.make_batch(w)
     run = gh.GpuRun(hb)
     g1 = run.event()
