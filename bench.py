@@ -365,7 +365,7 @@ def run_ours(args):
 def cpu_baseline(w: wl.Workload, n_units: int):
     """The oracle, as it stands, on a bounded sample: the first `n_units` units of the workload."""
     from oracle import cask_oracle as orc
-    n_units = n_units or max(1, min(w.n_units, (32 * 33280) // (w.prefix + w.decode)))
+    n_units = n_units or max(1, min(w.n_units, (96 * 33280) // (w.prefix + w.decode)))
     units = wl.unit_list(w)[:n_units]
     hb = wl.make_batch(w, units)
     kf, vf, qf = (wl.as_float32(x, w.dtype) for x in (hb.k, hb.v, hb.q))
@@ -424,7 +424,7 @@ def main():
     ap.add_argument("--score-path", type=int, default=0, help="0: tensor-core scoring when the shape allows, 1: SIMT")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-units", type=int, default=0,
-                    help="units in the oracle's bounded sample (default: about a million cache rows)")
+                    help="units in the oracle's bounded sample (default: about three million cache rows, 10 s of CPU work)")
     ap.add_argument("--max-units", type=int, default=0, help="debug: cut the workload to this many units")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layer-slice", type=int, default=0,
