@@ -192,6 +192,40 @@ void cask_oracle_select_core(const double* s, int T, int P, const int* plan, uin
 }
 
 /*
+ * Kappa-weighted merge geometry in its own form (Sec. 2.5):
+ *     d_kappa(k_i, k_j) = sum_f w_f * || k_{i,f} - k_{j,f} ||_2 ,   w_f = |kappa(omega_f)| >= 0 (caller-supplied),
+ * where band f is a pair of channels of the rotary embedding: (f, f + d/2) for layout 0 (the halves of the head
+ * are rotated against each other), (2f, 2f + 1) for layout 1 (adjacent channels).  The paper gives the distance
+ * and no rule for turning it into a merge decision; reading: the scale-free similarity
+ *     sim_kappa(j,u) = 1 - d_kappa(k_j,k_u) / (D_j + D_u),   D_x = sum_f w_f ||k_{x,f}||_2 ,
+ * which lies in [0,1] by the triangle inequality (1 for equal keys, 0 for opposite ones), takes the place of the
+ * cosine: argmax over the seeds, threshold tau, the same tie rule; a row or seed with D = 0 has similarity 0.
+ */
+static void orc_band(int f, int d, int layout, int* c0, int* c1) {
+    if (layout == 0) { *c0 = f; *c1 = f + d / 2; }
+    else { *c0 = 2 * f; *c1 = 2 * f + 1; }
+}
+static double orc_band_len(const float* k, int d, const float* bw, int layout) {
+    double D = 0.0;
+    for (int f = 0; f < d / 2; ++f) {
+        int c0, c1;
+        orc_band(f, d, layout, &c0, &c1);
+        D += (double)bw[f] * sqrt((double)k[c0] * (double)k[c0] + (double)k[c1] * (double)k[c1]);
+    }
+    return D;
+}
+static double orc_band_dist(const float* a, const float* b, int d, const float* bw, int layout) {
+    double dist = 0.0;
+    for (int f = 0; f < d / 2; ++f) {
+        int c0, c1;
+        orc_band(f, d, layout, &c0, &c1);
+        double x = (double)a[c0] - (double)b[c0], y = (double)a[c1] - (double)b[c1];
+        dist += (double)bw[f] * sqrt(x * x + y * y);
+    }
+    return dist;
+}
+
+/*
  * Scratch consolidation (Sec. 2.1 "representative construction only on this
  * part"; Sec. 2.4 m-folding; Sec. 2.5 cosine as the base merge geometry).
  * Scratch S = rows of [P, T-r) with kind 0.  Reading: the m greatest rows of S
@@ -204,14 +238,15 @@ void cask_oracle_select_core(const double* s, int T, int P, const int* plan, uin
  * bands with more future relevance count more; reading: the inner-product form
  *     sim_w(j,u) = sum_c w_c k_jc k_uc / (|k_j|_w |k_u|_w),  |k|_w^2 = sum_c w_c k_c^2,
  * with w_c = |kappa(omega_f)| on the channels of band f supplied by the caller; NULL = plain cosine).
+ * band_w (nullable, [d/2], >= 0; not together with chan_w) selects the un-squared per-band form sim_kappa above.
  * Outputs: kind (adds 4 seed, 5 merged), seed_of (row of the group's seed, -1),
  * weight (w_i for group members, untouched elsewhere), sim / sim2 (best and
  * second-best similarity of each non-seed scratch row; -2 where undefined).
  * Returns flags to OR into the unit's status (MERGE_INACTIVE if nobody joins).
  */
 int cask_oracle_consolidate(const float* K, const double* s, int T, int P, int d, const int* plan,
-                            double tau, double eps, const double* mass_in, const float* chan_w, uint8_t* kind,
-                            int* seed_of,
+                            double tau, double eps, const double* mass_in, const float* chan_w,
+                            const float* band_w, int band_layout, uint8_t* kind, int* seed_of,
                             double* weight, double* sim, double* sim2, double* lost_mass) {
     int r = plan[PL_R], m = plan[PL_M];
     for (int i = 0; i < T; ++i) { seed_of[i] = -1; if (sim) sim[i] = -2.0; if (sim2) sim2[i] = -2.0; }
@@ -227,7 +262,7 @@ int cask_oracle_consolidate(const float* K, const double* s, int T, int P, int d
             double n2 = 0.0;
             for (int c = 0; c < d; ++c)
                 n2 += (chan_w ? (double)chan_w[c] : 1.0) * (double)K[(size_t)i * d + c] * (double)K[(size_t)i * d + c];
-            snorm[ns] = sqrt(n2);
+            snorm[ns] = band_w ? orc_band_len(K + (size_t)i * d, d, band_w, band_layout) : sqrt(n2);
             seed_of[i] = i;
             ++ns;
         }
@@ -237,7 +272,7 @@ int cask_oracle_consolidate(const float* K, const double* s, int T, int P, int d
         const float* kj = K + (size_t)j * d;
         double n2 = 0.0;
         for (int c = 0; c < d; ++c) n2 += (chan_w ? (double)chan_w[c] : 1.0) * (double)kj[c] * (double)kj[c];
-        double nj = sqrt(n2);
+        double nj = band_w ? orc_band_len(kj, d, band_w, band_layout) : sqrt(n2);
         double best = -INFINITY, second = -INFINITY;
         int best_u = -1;
         for (int u = 0; u < ns; ++u) {           /* seeds[] ascends, so '>' keeps the smallest row on ties */
@@ -245,6 +280,9 @@ int cask_oracle_consolidate(const float* K, const double* s, int T, int P, int d
             double dot = 0.0;
             for (int c = 0; c < d; ++c) dot += (chan_w ? (double)chan_w[c] : 1.0) * (double)kj[c] * (double)ku[c];
             double sm = (nj > 0.0 && snorm[u] > 0.0) ? dot / (nj * snorm[u]) : 0.0;
+            if (band_w)
+                sm = (nj > 0.0 && snorm[u] > 0.0) ? 1.0 - orc_band_dist(kj, ku, d, band_w, band_layout) / (nj + snorm[u])
+                                                  : 0.0;
             if (sm > best) { second = best; best = sm; best_u = u; }
             else if (sm > second) second = sm;
         }
@@ -346,8 +384,8 @@ void cask_oracle_diagnostics(const double* s, int T, int B, const uint8_t* kind,
 /* The whole event for one unit, the steps above in order.  plan[8] is written. */
 void cask_oracle_event(const float* K, const float* V, const float* Q, int T, int P, int B, int reserve,
                        int d, int g, int W, int causal, double gamma, double tau, double eps,
-                       const double* lse_in, const double* mass_in, const float* chan_w, double* s, int* plan,
-                       uint8_t* kind,
+                       const double* lse_in, const double* mass_in, const float* chan_w, const float* band_w,
+                       int band_layout, double* s, int* plan, uint8_t* kind,
                        int* seed_of, double* weight, double* sim, double* sim2, double* k_out, double* v_out,
                        int* n_out, int* slot_src, uint8_t* slot_kind, double* slot_mass, int* assign,
                        int* status, double* lost_mass, double* rho /* nullable [2]: core, rep */) {
@@ -356,8 +394,8 @@ void cask_oracle_event(const float* K, const float* V, const float* Q, int T, in
     for (int i = 0; i < T; ++i) weight[i] = 0.0;
     cask_oracle_prefix_evict(s, P, plan, kind);
     cask_oracle_select_core(s, T, P, plan, kind);
-    int fl = cask_oracle_consolidate(K, s, T, P, d, plan, tau, eps, mass_in, chan_w, kind, seed_of, weight, sim, sim2,
-                                     lost_mass);
+    int fl = cask_oracle_consolidate(K, s, T, P, d, plan, tau, eps, mass_in, chan_w, band_w, band_layout, kind, seed_of,
+                                     weight, sim, sim2, lost_mass);
     if (!(plan[PL_FLAGS] & ORC_DECODE_CONSOLIDATED)) fl = 0;
     cask_oracle_compact(K, V, T, d, kind, seed_of, weight, s, eps, mass_in, k_out, v_out, n_out, slot_src,
                         slot_kind, slot_mass, assign);
@@ -375,7 +413,7 @@ void cask_oracle_event_batch(int n_units, const float* K, const float* V, const 
                              const int64_t* tok_off, const int* P, const int* B, const int* reserve,
                              int d, int g, int W, int causal, double gamma, double tau, double eps,
                              const double* mass_in /* nullable [sum T] */, const float* chan_w /* nullable [d] */,
-                             int Bmax, double* s, int* plan, uint8_t* kind, int* seed_of, double* weight,
+                             const float* band_w /* nullable [d/2] */, int band_layout, int Bmax, double* s, int* plan, uint8_t* kind, int* seed_of, double* weight,
                              double* sim, double* sim2, double* k_out, double* v_out, int* n_out,
                              int* slot_src, uint8_t* slot_kind, double* slot_mass, int* assign,
                              int* status, double* lost_mass, double* rho /* nullable [n_units, 2] */) {
@@ -387,7 +425,7 @@ void cask_oracle_event_batch(int n_units, const float* K, const float* V, const 
         int T = (int)(tok_off[u + 1] - tok_off[u]);
         size_t so = (size_t)u * (size_t)Bmax;
         cask_oracle_event(K + a * d, V + a * d, Q + (size_t)u * g * W * d, T, P[u], B[u], reserve[u], d, g,
-                          W, causal, gamma, tau, eps, NULL, mass_in ? mass_in + a : NULL, chan_w, s + a, plan + (size_t)u * 8, kind + a,
+                          W, causal, gamma, tau, eps, NULL, mass_in ? mass_in + a : NULL, chan_w, band_w, band_layout, s + a, plan + (size_t)u * 8, kind + a,
                           seed_of + a, weight + a, sim ? sim + a : NULL, sim2 ? sim2 + a : NULL,
                           k_out + so * d, v_out + so * d, n_out + u, slot_src + so, slot_kind + so,
                           slot_mass + so, assign + a, status + u, lost_mass + u, rho ? rho + 2 * (size_t)u : NULL);

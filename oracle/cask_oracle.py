@@ -86,7 +86,7 @@ def select_core(s, T: int, P: int, pl: np.ndarray, kind: np.ndarray) -> None:
 
 
 def consolidate(K, s, P: int, pl: np.ndarray, kind: np.ndarray, tau: float = 0.9, eps: float = 1e-9, mass_in=None,
-                chan_w=None):
+                chan_w=None, band_w=None, band_layout: int = 0):
     """Updates ``kind`` in place; returns dict(seed_of, weight, sim, sim2, flags, lost_mass)."""
     K = _f32(K)
     T, d = K.shape
@@ -97,11 +97,14 @@ def consolidate(K, s, P: int, pl: np.ndarray, kind: np.ndarray, tau: float = 0.9
     sim2 = np.zeros(T, dtype=np.float64)
     mass_in = None if mass_in is None else np.ascontiguousarray(mass_in, dtype=np.float64)
     chan_w = None if chan_w is None else np.ascontiguousarray(chan_w, dtype=np.float32)
+    band_w = None if band_w is None else np.ascontiguousarray(band_w, dtype=np.float32)
+    assert band_w is None or (chan_w is None and band_w.shape == (d // 2,))
     lost = C.c_double(0.0)
     fn = lib().cask_oracle_consolidate
     fn.restype = C.c_int
     fl = fn(_p(K, C.c_float), _p(s, C.c_double), T, int(P), d, _p(pl, C.c_int), C.c_double(tau),
-            C.c_double(eps), _p(mass_in, C.c_double), _p(chan_w, C.c_float), _p(kind, C.c_uint8), _p(seed_of, C.c_int),
+            C.c_double(eps), _p(mass_in, C.c_double), _p(chan_w, C.c_float), _p(band_w, C.c_float), int(band_layout),
+            _p(kind, C.c_uint8), _p(seed_of, C.c_int),
             _p(weight, C.c_double), _p(sim, C.c_double), _p(sim2, C.c_double), C.byref(lost))
     return dict(seed_of=seed_of, weight=weight, sim=sim, sim2=sim2, flags=int(fl), lost_mass=lost.value)
 
@@ -134,7 +137,7 @@ def compact(K, V, kind, seed_of, weight, s, eps: float = 1e-9, mass_in=None):
 
 
 def event_batch(K, V, Q, tok_off, P, B, reserve, causal: int = 1, gamma: float = 0.5, tau: float = 0.9,
-                eps: float = 1e-9, mass_in=None, chan_w=None) -> Dict[str, np.ndarray]:
+                eps: float = 1e-9, mass_in=None, chan_w=None, band_w=None, band_layout: int = 0) -> Dict[str, np.ndarray]:
     """Whole event for many contiguous units.  K, V [sum T, d]; Q [n, g, W, d] (float32 values)."""
     K, V, Q = _f32(K), _f32(V), _f32(Q)
     n, g, W, d = Q.shape
@@ -154,10 +157,13 @@ def event_batch(K, V, Q, tok_off, P, B, reserve, causal: int = 1, gamma: float =
         status=np.zeros(n, np.int32), lost_mass=np.zeros(n, np.float64), rho=np.zeros((n, 2), np.float64))
     mass_in = None if mass_in is None else np.ascontiguousarray(mass_in, dtype=np.float64)
     chan_w = None if chan_w is None else np.ascontiguousarray(chan_w, dtype=np.float32)
+    band_w = None if band_w is None else np.ascontiguousarray(band_w, dtype=np.float32)
+    assert band_w is None or (chan_w is None and band_w.shape == (d // 2,))
     lib().cask_oracle_event_batch(
         n, _p(K, C.c_float), _p(V, C.c_float), _p(Q, C.c_float), _p(tok_off, C.c_int64), _p(P, C.c_int),
         _p(B, C.c_int), _p(reserve, C.c_int), d, g, W, int(causal), C.c_double(gamma), C.c_double(tau),
-        C.c_double(eps), _p(mass_in, C.c_double), _p(chan_w, C.c_float), Bmax, _p(o["s"], C.c_double), _p(o["plan"], C.c_int), _p(o["kind"], C.c_uint8),
+        C.c_double(eps), _p(mass_in, C.c_double), _p(chan_w, C.c_float), _p(band_w, C.c_float), int(band_layout), Bmax,
+        _p(o["s"], C.c_double), _p(o["plan"], C.c_int), _p(o["kind"], C.c_uint8),
         _p(o["seed_of"], C.c_int), _p(o["weight"], C.c_double), _p(o["sim"], C.c_double),
         _p(o["sim2"], C.c_double), _p(o["k_out"], C.c_double), _p(o["v_out"], C.c_double),
         _p(o["n_out"], C.c_int), _p(o["slot_src"], C.c_int), _p(o["slot_kind"], C.c_uint8),

@@ -44,8 +44,20 @@ def cosine(a: List[float], b: List[float], w=None) -> float:
     return math.fsum(c * x * y for c, x, y in zip(w, a, b)) / (na * nb)
 
 
+def band_similarity(a: List[float], b: List[float], bw: List[float], layout: int) -> float:
+    """1 - d_kappa(a,b) / (D_a + D_b) with d_kappa = sum_f w_f ||a_f - b_f||, D_x = sum_f w_f ||x_f|| (Sec. 2.5)."""
+    d = len(a)
+    pairs = [(f, f + d // 2) if layout == 0 else (2 * f, 2 * f + 1) for f in range(d // 2)]
+    Da = math.fsum(w * math.hypot(a[i], a[j]) for w, (i, j) in zip(bw, pairs))
+    Db = math.fsum(w * math.hypot(b[i], b[j]) for w, (i, j) in zip(bw, pairs))
+    if Da == 0.0 or Db == 0.0:
+        return 0.0
+    dist = math.fsum(w * math.hypot(a[i] - b[i], a[j] - b[j]) for w, (i, j) in zip(bw, pairs))
+    return 1.0 - dist / (Da + Db)
+
+
 def event(K, V, Q, P: int, B: int, reserve: int, gamma: float = 0.5, tau: float = 0.9,
-          eps: float = 1e-9, causal: bool = True, mass_in=None, chan_w=None) -> Dict:
+          eps: float = 1e-9, causal: bool = True, mass_in=None, chan_w=None, band_w=None, band_layout: int = 0) -> Dict:
     T, d = len(K), len(K[0])
     W = len(Q[0])
     s = scores(K, Q, causal)
@@ -94,7 +106,10 @@ def event(K, V, Q, P: int, B: int, reserve: int, gamma: float = 0.5, tau: float 
             for j in scratch:
                 if j in groups:
                     continue
-                sims = [(cosine(K[j], K[u], chan_w), -u) for u in seeds]
+                if band_w is not None:
+                    sims = [(band_similarity(K[j], K[u], band_w, band_layout), -u) for u in seeds]
+                else:
+                    sims = [(cosine(K[j], K[u], chan_w), -u) for u in seeds]
                 best, negu = max(sims)
                 if best >= tau:
                     groups[-negu].append(j)

@@ -301,11 +301,12 @@ def test_planted_clusters_are_recovered_with_full_purity():
 
 # ---- whole event vs the separately written brute force -----------------------
 
-def _cmp_with_bruteforce(K, V, Q, P, B, res, tau, mass_in=None, chan_w=None):
-    o = orc.event(K, V, Q, P, B, res, tau=tau, mass_in=mass_in, chan_w=chan_w)
+def _cmp_with_bruteforce(K, V, Q, P, B, res, tau, mass_in=None, chan_w=None, band_w=None, band_layout=0):
+    o = orc.event(K, V, Q, P, B, res, tau=tau, mass_in=mass_in, chan_w=chan_w, band_w=band_w, band_layout=band_layout)
     b = bf.event(K.tolist(), V.tolist(), Q.tolist(), P, B, res, tau=tau,
                  mass_in=None if mass_in is None else list(mass_in),
-                 chan_w=None if chan_w is None else [float(x) for x in chan_w])
+                 chan_w=None if chan_w is None else [float(x) for x in chan_w],
+                 band_w=None if band_w is None else [float(x) for x in band_w], band_layout=band_layout)
     assert abs(o["rho_core"] - b["rho_core"]) < 1e-12 and abs(o["rho_rep"] - b["rho_rep"]) < 1e-12
     assert np.allclose(o["s"], b["s"], rtol=1e-12, atol=1e-300)
     assert o["kind"].tolist() == b["kind"]
@@ -400,6 +401,68 @@ def test_channel_weighted_similarity():
             assert m["seed_of"][j] == seeds[int(np.argmax(cs))]
     for tau in (-1.0, 0.8):
         _cmp_with_bruteforce(K[:14], V[:14], Q, 2, 7, 4, tau, chan_w=w)
+
+
+def test_band_distance_geometry():
+    """Sec. 2.5, d_kappa = sum_f w_f ||k_if - k_jf||_2 over rotary bands f, read as the similarity
+    1 - d_kappa / (D_i + D_j).  Closed forms: equal keys 1, opposite keys 0, orthogonal equal-norm bands
+    1 - sqrt(2)/2; one band of weight one is numpy's Euclidean distance on that band's two channels; a common
+    factor on the weights or on all keys changes nothing; the two band layouts pair different channels."""
+    rng = np.random.default_rng(17)
+    d, W = 8, 2
+    # two-row closed forms through the whole event: one seed (row 1 scores higher), one candidate (row 0)
+    def sim_of(k0, k1, bw, layout):
+        K = np.array([k0, k1, k1, k1], np.float32)          # rows 2,3: the recent window (W = 2)
+        K[2:] += 100.0                                       # keep them away from the seed choice
+        V = np.zeros_like(K)
+        Q = np.zeros((1, W, d), np.float32)
+        pl = np.array([0, 0, 2, 0, 0, 1, 0, 0], np.int32)    # r = 0, c = 0, m = 1 over rows [0, 2)
+        kind = np.zeros(4, np.uint8)
+        s = np.array([0.1, 0.9, 0.0, 0.0])
+        o = orc.consolidate(K[:2], s[:2], 0, pl, kind[:2], tau=2.0, band_w=bw, band_layout=layout)
+        return o["sim"][0]
+    k = rng.standard_normal(d).astype(np.float32)
+    ones = np.ones(d // 2, np.float32)
+    for layout in (0, 1):
+        assert abs(sim_of(k, k, ones, layout) - 1.0) < 1e-15
+        assert abs(sim_of(k, -k, ones, layout)) < 1e-15
+        assert abs(sim_of(k, 4.0 * k, ones, layout) - 0.4) < 1e-12        # 1 - |1-4| / (1+4) in every band
+    e = np.zeros(d, np.float32); e[0] = 2.0                                # band 0, first channel
+    f0 = np.zeros(d, np.float32); f0[d // 2] = 2.0                         # layout 0: band 0, second channel
+    f1 = np.zeros(d, np.float32); f1[1] = 2.0                              # layout 1: band 0, second channel
+    assert abs(sim_of(e, f0, ones, 0) - (1.0 - math.sqrt(2.0) / 2.0)) < 1e-12
+    assert abs(sim_of(e, f1, ones, 1) - (1.0 - math.sqrt(2.0) / 2.0)) < 1e-12
+    assert abs(sim_of(e, f1, ones, 0)) < 1e-12      # layout 0 puts channels 0 and 1 in different bands: d = D_i + D_j
+    # whole events: weights, scale invariance, one-band weights against numpy, brute force
+    T, P, B, res = 40, 0, 12, 12
+    centres = rng.standard_normal((4, d))
+    K = (centres[rng.integers(0, 4, T)] + 0.2 * rng.standard_normal((T, d))).astype(np.float32)
+    V = rng.standard_normal((T, d)).astype(np.float32)
+    Q = rng.standard_normal((2, W, d)).astype(np.float32)
+    bw = (rng.random(d // 2) + 0.1).astype(np.float32)
+    plain = orc.event(K, V, Q, P, B, res, tau=0.6)
+    a = orc.event(K, V, Q, P, B, res, tau=0.6, band_w=bw)
+    b = orc.event(K, V, Q, P, B, res, tau=0.6, band_w=4.0 * bw)
+    c = orc.event(2.0 * K, V, 0.5 * Q, P, B, res, tau=0.6, band_w=bw)      # same scores (q.k unchanged), keys doubled
+    assert np.array_equal(a["kind"], b["kind"]) and np.allclose(a["sim"], b["sim"], rtol=1e-12)
+    assert np.array_equal(a["kind"], c["kind"]) and np.allclose(a["sim"], c["sim"], rtol=1e-6, atol=1e-7)
+    assert (a["kind"] == 5).any() and not np.array_equal(a["sim"], plain["sim"])
+    cand = a["sim"] > -1.5
+    assert (a["sim"][cand] >= 0.0).all() and (a["sim"][cand] <= 1.0).all()
+    for layout, (c0, c1) in ((0, (1, 1 + d // 2)), (1, (2, 3))):
+        one = np.zeros(d // 2, np.float32); one[1] = 1.0
+        m = orc.event(K, V, Q, P, B, res, tau=0.6, band_w=one, band_layout=layout)
+        seeds = np.flatnonzero(m["kind"] == 4)
+        Kb = K[:, [c0, c1]].astype(np.float64)
+        for j in np.flatnonzero(m["sim"] > -1.5):
+            dist = np.linalg.norm(Kb[seeds] - Kb[j], axis=1)
+            sm = 1.0 - dist / (np.linalg.norm(Kb[seeds], axis=1) + np.linalg.norm(Kb[j]))
+            assert abs(sm.max() - m["sim"][j]) < 1e-12
+            if m["kind"][j] == 5:
+                assert m["seed_of"][j] == seeds[int(np.argmax(sm))]
+    for layout in (0, 1):
+        for tau in (-1.0, 0.6):
+            _cmp_with_bruteforce(K[:14], V[:14], Q, 2, 7, 4, tau, band_w=bw, band_layout=layout)
 
 
 def test_whole_event_against_bruteforce_exhausted_boundary():
