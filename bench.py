@@ -166,8 +166,13 @@ def run_ours(args):
 
     dev = cb.to_device(hb, device)
     mass_dev = None if hb.mass_in is None else torch.from_numpy(hb.mass_in).to(device)
+    # merge similarity (Sec. 2.5): plain cosine, or synthetic weights |kappa| that fall off with the band index
+    chan_host, band_host = similarity_weights(args.similarity, d)
+    sim_dev = dict(chan_w=None if chan_host is None else torch.from_numpy(chan_host).to(device),
+                   band_w=None if band_host is None else torch.from_numpy(band_host).to(device))
+    sim_host = dict(chan_w=chan_host, band_w=band_host)
     batch, keep = cb.make_batch(dev["k"], dev["v"], dev["q"], hb.T, hb.P, hb.B, hb.reserve, hb.tok_off, d, w.group,
-                                w.window, w.dtype, mass_in=mass_dev)
+                                w.window, w.dtype, mass_in=mass_dev, **sim_dev)
     prm = cb.params(score_path=args.score_path)
     stream = torch.cuda.current_stream(device)
     ctx = cb.Context(local, stream.cuda_stream)
@@ -219,7 +224,7 @@ def run_ours(args):
     # The same event when the caller hands over the window queries' softmax normalisers (a decode attention
     # kernel has them): the normaliser pass is skipped.  Reported beside the headline, never instead of it.
     batch_l, keep_l = cb.make_batch(dev["k"], dev["v"], dev["q"], hb.T, hb.P, hb.B, hb.reserve, hb.tok_off, d, w.group,
-                                    w.window, w.dtype, lse_in=out["lse"].clone(), mass_in=mass_dev)
+                                    w.window, w.dtype, lse_in=out["lse"].clone(), mass_in=mass_dev, **sim_dev)
     cb.cask_compress_event(ctx, batch_l, prm, out_struct, ws, ws_bytes)
     barrier()
     ev0.record(stream)
@@ -245,7 +250,7 @@ def run_ours(args):
 
     # ---- end to end through the host-buffer entry point ---------------------------------------
     hbatch, hkeep = cb.make_batch(hb.k, hb.v, hb.q, hb.T, hb.P, hb.B, hb.reserve, hb.tok_off, d, w.group, w.window,
-                                  w.dtype, mass_in=hb.mass_in)
+                                  w.dtype, mass_in=hb.mass_in, **sim_host)
     dev_bytes = cb.cask_host_event_device_bytes(hbatch, prm, Bmax)
     del dev, out, out_struct, ws
     torch.cuda.empty_cache()
@@ -330,7 +335,7 @@ def run_ours(args):
     # ---- the oracle on this machine's host cores, bounded sample ------------------------------------
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        cpu = cpu_baseline(w, args.cpu_units)
+        cpu = cpu_baseline(w, args.cpu_units, args.similarity)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
@@ -347,6 +352,7 @@ def run_ours(args):
                        "events_per_s_note": "one event = all layers of one sequence; this pass held layers_per_pass of them"}
                       if w.n_seqs > 1 else {}),
                    **({"carried_mass_rows": w.carried_rows} if w.carried_rows else {}),
+                   "similarity": args.similarity,
                    "status_bits_seen": int(np.bitwise_or.reduce(status))},
         "with_supplied_normalisers": {"ms_per_step": ms_lse, "value": total_tokens / (ms_lse * 1e-3), "unit": UNIT,
                                       "note": "lse_in given by the caller: one scoring pass instead of two (this rank)"},
@@ -362,7 +368,18 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def cpu_baseline(w: wl.Workload, n_units: int):
+def similarity_weights(kind: str, d: int):
+    """(chan_w [d], band_w [d/2]) for --similarity: None for the cosine; |kappa|-like weights 1 / (1 + f/8) on band
+    f = channels (f, f + d/2) otherwise, per channel (inner-product form) or per band (distance form)."""
+    if kind == "cosine":
+        return None, None
+    bw = (1.0 / (1.0 + np.arange(d // 2) / 8.0)).astype(np.float32)
+    if kind == "channel":
+        return np.concatenate([bw, bw]).astype(np.float32), None
+    return None, bw
+
+
+def cpu_baseline(w: wl.Workload, n_units: int, similarity: str = "cosine"):
     """The oracle, as it stands, on a bounded sample: the first `n_units` units of the workload."""
     from oracle import cask_oracle as orc
     n_units = n_units or max(1, min(w.n_units, (96 * 33280) // (w.prefix + w.decode)))
@@ -371,7 +388,8 @@ def cpu_baseline(w: wl.Workload, n_units: int):
     kf, vf, qf = (wl.as_float32(x, w.dtype) for x in (hb.k, hb.v, hb.q))
     orc.lib()
     t = time.time()
-    orc.event_batch(kf, vf, qf, hb.tok_off, hb.P, hb.B, hb.reserve, mass_in=hb.mass_in)
+    cw, bw = similarity_weights(similarity, w.head_dim)
+    orc.event_batch(kf, vf, qf, hb.tok_off, hb.P, hb.B, hb.reserve, mass_in=hb.mass_in, chan_w=cw, band_w=bw)
     dt = time.time() - t
     return {"value": float(hb.T.sum()) / dt, "unit": UNIT, "cores": orc.threads(), "kind": "oracle",
             "sample": f"{len(units)} of {w.n_units} units of {w.name} (whole event, fp64), {dt:.1f} s",
@@ -392,8 +410,9 @@ def run_reference(args):
     orc.lib()
 
     def step():
-        orc.event_batch(kf, vf, qf, hb.tok_off, hb.P, hb.B, hb.reserve, mass_in=hb.mass_in)
+        orc.event_batch(kf, vf, qf, hb.tok_off, hb.P, hb.B, hb.reserve, mass_in=hb.mass_in, chan_w=cw, band_w=bw)
 
+    cw, bw = similarity_weights(args.similarity, w.head_dim)
     for _ in range(args.warmup):
         step()
     t = time.time()
@@ -423,6 +442,8 @@ def main():
     ap.add_argument("--workload", default="reasoning32k_b512", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--score-path", type=int, default=0, help="0: tensor-core scoring when the shape allows, 1: SIMT")
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--similarity", default="cosine", choices=["cosine", "channel", "band"],
+                    help="merge similarity: cosine, channel-weighted inner product, or per-band distance (Sec. 2.5)")
     ap.add_argument("--cpu-units", type=int, default=0,
                     help="units in the oracle's bounded sample (default: about three million cache rows, 10 s of CPU work)")
     ap.add_argument("--max-units", type=int, default=0, help="debug: cut the workload to this many units")

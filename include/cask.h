@@ -124,6 +124,15 @@ typedef struct {
        more future relevance count more; w_c = |kappa(omega_f)| on the channels of band f):
        sim(j,u) = sum_c w_c k_jc k_uc / (|k_j|_w |k_u|_w), |k|_w^2 = sum_c w_c k_c^2.  NULL = cosine. */
     const float* chan_w;     /* DEVICE [head_dim] or NULL                       */
+    /* optional, instead of chan_w: the merge distance of Sec. 2.5 in its own, un-squared form,
+       d_kappa(k_i,k_j) = sum_f w_f ||k_if - k_jf||_2 over the rotary bands f (pairs of channels), w_f =
+       |kappa(omega_f)| >= 0 from the caller.  The paper gives no decision rule for it; the library uses the
+       scale-free similarity 1 - d_kappa(k_j,k_u) / (D_j + D_u), D_x = sum_f w_f ||k_xf||_2 (in [0,1]; a row with
+       D = 0 has similarity 0) exactly where it uses the cosine: argmax over the seeds, threshold tau.
+       band_layout 0: band f = channels (f, f + head_dim/2); 1: channels (2f, 2f + 1).  head_dim must be even.
+       This form runs on the SIMT path (one square root per row, seed and band).  NULL = not used. */
+    const float* band_w;     /* DEVICE [head_dim/2] or NULL                     */
+    int32_t band_layout;     /* 0 | 1; ignored when band_w is NULL              */
 } cask_batch;
 
 /*

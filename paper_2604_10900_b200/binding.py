@@ -46,6 +46,7 @@ class CaskBatch(C.Structure):
         ("tok_off", C.c_void_p),
         ("block_table", C.c_void_p), ("bt_off", C.c_void_p), ("n_pages", C.c_int64),
         ("mass_in", C.c_void_p), ("chan_w", C.c_void_p),
+        ("band_w", C.c_void_p), ("band_layout", C.c_int32),
     ]
 
 
@@ -152,7 +153,8 @@ class HostArrays:
 
 def make_batch(k, v, q, T, P, B, reserve, tok_off, head_dim: int, group: int, window: int, dtype: int,
                k_off=None, v_off=None, row_stride: Optional[int] = None, lse_in=None, page_size: int = 0,
-               block_table=None, bt_off=None, n_pages: int = 0, mass_in=None, chan_w=None):
+               block_table=None, bt_off=None, n_pages: int = 0, mass_in=None, chan_w=None, band_w=None,
+               band_layout: int = 0):
     """Fills a cask_batch.  k, v, q, lse_in: tensors/arrays/addresses (device for the device calls,
     host for cask_compress_event_host).  Paged cache: page_size > 0, k and v the page pools,
     block_table a device int32 tensor, bt_off the host offsets of the units in it.
@@ -177,7 +179,9 @@ def make_batch(k, v, q, T, P, B, reserve, tok_off, head_dim: int, group: int, wi
     b.n_pages = n_pages
     b.mass_in = _ptr(mass_in)
     b.chan_w = _ptr(chan_w)
-    return b, (h, k, v, q, lse_in, block_table, bt_host, mass_in, chan_w)
+    b.band_w = _ptr(band_w)
+    b.band_layout = int(band_layout)
+    return b, (h, k, v, q, lse_in, block_table, bt_host, mass_in, chan_w, band_w)
 
 
 def make_outputs(d: Dict, Bmax: int) -> CaskOutputs:

@@ -119,6 +119,10 @@ int check_batch(const cask_batch* b, const cask_params* p) {
     if (b->lse_in && (uintptr_t)b->lse_in % 4) return CASK_ERR_ALIGN;
     if (b->mass_in && (uintptr_t)b->mass_in % 4) return CASK_ERR_ALIGN;
     if (b->chan_w && (uintptr_t)b->chan_w % 4) return CASK_ERR_ALIGN;
+    if (b->band_w) {
+        if ((uintptr_t)b->band_w % 4) return CASK_ERR_ALIGN;
+        if (b->chan_w || (b->head_dim & 1) || (b->band_layout != 0 && b->band_layout != 1)) return CASK_ERR_SHAPE;
+    }
     for (int u = 0; u < b->n_units; ++u) {
         const int T = b->T[u], P = b->P[u], B = b->B[u], R = b->reserve[u];
         if (T < 1 || b->window > T || P < 0 || P > T || B < 1 || R < 0 || R > B) return CASK_ERR_SHAPE;
@@ -267,6 +271,7 @@ int prepare(cask_ctx* ctx, const cask_batch* b, const cask_params* p, void* ws, 
     L.sh.causal = p->causal;
     L.sh.page_size = b->page_size; L.sh.n_pages = b->n_pages; L.sh.bt = b->block_table; L.sh.err = W.err;
     L.sh.mass_in = b->mass_in; L.sh.chan_w = b->chan_w;
+    L.sh.band_w = b->band_w; L.sh.band_layout = b->band_layout;
     L.desc = W.desc; L.hdesc = ctx->pinned;
     L.k = b->k; L.v = b->v; L.q = b->q;
     L.max_T = z.max_T; L.max_m = z.max_m; L.max_chunks = z.max_chunks; L.total_chunks = z.total_chunks;
@@ -566,7 +571,7 @@ int cask_writeback_paged(cask_ctx* ctx, const cask_batch* b, const cask_params* 
 
 namespace {
 struct HostStage {
-    char *k, *v, *q, *lse_in, *mass_in, *chan_w;
+    char *k, *v, *q, *lse_in, *mass_in, *chan_w, *band_w;
     cask_outputs o;
     char* ws;
     size_t ws_bytes, bytes;
@@ -594,6 +599,7 @@ HostStage stage_layout(char* base, const cask_batch* b, const cask_params* p, in
     h.lse_in = take(h.lse_bytes);
     h.mass_in = take(sumT * 4);
     h.chan_w = take(d * 4);
+    h.band_w = take(d * 2);
     h.v_pos = (int32_t*)take(sumT * 4);
     h.n_need = (int32_t*)take(n * 4);
     h.v_base = (int64_t*)take(n * 8);
@@ -667,6 +673,11 @@ int cask_compress_event_host(cask_ctx* ctx, const cask_batch* hb, const cask_par
         if (e != cudaSuccess) return fail_cuda(ctx, e);
     }
     db.chan_w = hb->chan_w ? (const float*)h.chan_w : nullptr;
+    if (hb->band_w) {
+        e = cudaMemcpyAsync(h.band_w, hb->band_w, (size_t)(hb->head_dim / 2) * 4, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+    }
+    db.band_w = hb->band_w ? (const float*)h.band_w : nullptr;
     db.k = h.k; db.v = h.v; db.q = h.q;
     db.lse_in = hb->lse_in ? (const float*)h.lse_in : nullptr;
     const size_t es = elem_size(hb->dtype), n = (size_t)hb->n_units, d = (size_t)hb->head_dim;

@@ -40,6 +40,8 @@ struct Shape {
     int32_t* err;        // device flag word (CASK_ST_TIMEOUT, CASK_ST_BOUNDS)
     const float* mass_in;   // device, optional [sumT]: group mass a row already carries
     const float* chan_w;    // device, optional [d]: channel weights of the merge similarity
+    const float* band_w;    // device, optional [d/2]: band weights of the un-squared per-band distance (Sec. 2.5)
+    int band_layout;        // 0: band f = channels (f, f + d/2); 1: channels (2f, 2f + 1)
     // host-resident caches: only the value rows the compaction reads are on the device, packed unit after unit
     // in ascending row order; v_pos[tok_off + i] is the position of row i inside its unit's run, v_base[u] the
     // first packed row of unit u (both NULL when V is the full cache)

@@ -358,6 +358,152 @@ __global__ void __launch_bounds__(kThreads) assign_simt_kernel(
     }
 }
 
+// ---- 3b. assignment under the un-squared per-band distance of Sec. 2.5 -----------------------------------------
+// d_kappa(k_j, k_u) = sum_f w_f ||k_jf - k_uf||_2 over the rotary bands (pairs of channels), used as the similarity
+// 1 - d_kappa / (D_j + D_u), D_x = sum_f w_f ||k_xf||_2.  One square root per (row, seed, band), so the special-
+// function pipe bounds it; same tiling as assign_simt_kernel (64 rows x 64 seeds per step, 4 x 4 per thread).
+__device__ __forceinline__ float sqrt_fast(float x) {
+    float y;
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads) assign_band_kernel(
+    const UnitDesc* __restrict__ desc, Shape sh, const T* __restrict__ K, const float* __restrict__ s,
+    const int32_t* __restrict__ plan, const int32_t* __restrict__ seed_rows, const T* __restrict__ seed_k,
+    uint8_t* __restrict__ kind, int32_t* __restrict__ seed_of, float* __restrict__ sim, int32_t* __restrict__ grp,
+    unsigned long long* __restrict__ mass_fx, int32_t* __restrict__ njoin, int max_m, float tau, float eps) {
+    extern __shared__ float2 smem2[];
+    const int u = blockIdx.y;
+    const UnitDesc& ud = desc[u];
+    const int T_ = ud.T, P = ud.P;
+    const int r = max(0, min(plan[u * 8 + CASK_PLAN_R], T_ - P));
+    const int m = max(0, min(plan[u * 8 + CASK_PLAN_M], ud.plan[CASK_PLAN_M]));
+    const int lo = P + blockIdx.x * kTile, hi = T_ - r;
+    if (m <= 0 || lo >= hi) return;
+    const int d = sh.d, nb = d / 2, pitch = nb + 1;      // a row is nb bands of (x, y); odd pitch: no bank conflicts
+    float2* St = smem2;                                   // [64][pitch] stationary rows
+    float2* Rt = St + kTile * pitch;                      // [64][pitch] seeds of the current step
+    float* rlen = reinterpret_cast<float*>(Rt + kTile * pitch);   // [64] D of the stationary rows
+    float* slen = rlen + kTile;                           // [64] D of the seeds of the current step
+    float* bw = slen + kTile;                             // [d/2] band weights
+    const int ty = threadIdx.x / 16, tx = threadIdx.x % 16;
+    const int nrows = min(kTile, hi - lo);
+    const int second = sh.band_layout == 0 ? nb : 1, step = sh.band_layout == 0 ? 1 : 2;   // band f: channels (f*step, f*step + second)
+    for (int f = threadIdx.x; f < nb; f += kThreads) bw[f] = sh.band_w[f];
+    // rows of a tile into band order
+    auto stage = [&](float2* dst, const T* base, int64_t row_off, bool valid, int rr, int f) {
+        float2 v = make_float2(0.f, 0.f);
+        if (valid) {
+            v.x = Elem<T>::ld(base + row_off + f * step);
+            v.y = Elem<T>::ld(base + row_off + f * step + second);
+        }
+        dst[rr * pitch + f] = v;
+    };
+    for (int idx = threadIdx.x; idx < kTile * nb; idx += kThreads) {
+        const int rr = idx / nb, f = idx % nb;
+        stage(St, K, rr < nrows ? row_elem_off(sh, ud, ud.k_off, lo + rr) : 0, rr < nrows, rr, f);
+    }
+    __syncthreads();
+    // D of a row: four threads per row, a quarter of the bands each, fixed combination order
+    auto band_len = [&](const float2* row, int part) {
+        float D = 0.f;
+        for (int f = part; f < nb; f += 4) {
+            const float2 v = row[f];
+            D = fmaf(bw[f], sqrt_fast(fmaf(v.x, v.x, v.y * v.y)), D);
+        }
+        D += __shfl_xor_sync(0xffffffffu, D, 1);
+        D += __shfl_xor_sync(0xffffffffu, D, 2);
+        return D;
+    };
+    {
+        const int rr = threadIdx.x / 4, part = threadIdx.x % 4;
+        const float D = band_len(St + rr * pitch, part);
+        if (part == 0) rlen[rr] = D;
+    }
+    float best[4];
+    int best_u[4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a) { best[a] = -INFINITY; best_u[a] = -1; }
+
+    for (int u0 = 0; u0 < m; u0 += kTile) {
+        __syncthreads();
+        const int nseed = min(kTile, m - u0);
+        for (int idx = threadIdx.x; idx < kTile * nb; idx += kThreads) {
+            const int rr = idx / nb, f = idx % nb;
+            stage(Rt, seed_k, (int64_t)(ud.seed_base + u0 + rr) * d, rr < nseed, rr, f);
+        }
+        __syncthreads();
+        {
+            const int rr = threadIdx.x / 4, part = threadIdx.x % 4;
+            const float D = band_len(Rt + rr * pitch, part);
+            if (part == 0) slen[rr] = D;
+        }
+        float acc[4][4];
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+#pragma unroll 2
+        for (int f = 0; f < nb; ++f) {
+            const float w = bw[f];
+            float2 sv[4], rv[4];
+#pragma unroll
+            for (int a = 0; a < 4; ++a) sv[a] = St[(ty + 16 * a) * pitch + f];
+#pragma unroll
+            for (int b = 0; b < 4; ++b) rv[b] = Rt[(tx + 16 * b) * pitch + f];
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    const float dx = sv[a].x - rv[b].x, dy = sv[a].y - rv[b].y;
+                    acc[a][b] = fmaf(w, sqrt_fast(fmaf(dx, dx, dy * dy)), acc[a][b]);
+                }
+        }
+        __syncthreads();        // slen is complete
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            int su = u0 + tx + 16 * b;
+            if (su >= m) continue;
+            const float Du = slen[tx + 16 * b];
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+                const float Dj = rlen[ty + 16 * a];
+                float sm_ = (Dj > 0.f && Du > 0.f) ? 1.f - acc[a][b] / (Dj + Du) : 0.f;
+                if (sm_ > best[a]) { best[a] = sm_; best_u[a] = su; }
+            }
+        }
+    }
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+#pragma unroll
+        for (int off = 8; off >= 1; off >>= 1) {
+            float ob = __shfl_xor_sync(0xffffffffu, best[a], off);
+            int ou = __shfl_xor_sync(0xffffffffu, best_u[a], off);
+            if (ou >= 0 && (ob > best[a] || (ob == best[a] && ou < best_u[a]) || best_u[a] < 0)) {
+                best[a] = ob;
+                best_u[a] = ou;
+            }
+        }
+        int rr = ty + 16 * a;
+        int i = lo + rr;
+        if (tx == 0 && rr < nrows && kind[ud.tok_off + i] == CASK_KIND_DROPPED) {
+            if (sim) sim[ud.tok_off + i] = best[a];
+            unsigned long long fx = mass_to_fx(row_mass(sh, s, eps, ud.tok_off + i));
+            if (best_u[a] >= 0 && best[a] >= tau) {
+                kind[ud.tok_off + i] = CASK_KIND_MERGED;
+                seed_of[ud.tok_off + i] = seed_rows[ud.seed_base + best_u[a]];
+                grp[ud.tok_off + i] = best_u[a];
+                atomicAdd(&mass_fx[(size_t)u * (max_m + 1) + best_u[a]], fx);
+                atomicAdd(&njoin[u], 1);
+            } else {
+                atomicAdd(&mass_fx[(size_t)u * (max_m + 1) + max_m], fx);
+            }
+        }
+    }
+}
+
 // ---- 4. merge weights w_i = a_i / m_G, lost mass, status ---------------------------------
 __global__ void weights_kernel(const UnitDesc* __restrict__ desc, Shape sh, const float* __restrict__ s,
                                const int32_t* __restrict__ plan, const int32_t* __restrict__ grp,
@@ -387,7 +533,7 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const i
                 Workspace& ws, bool fused_small) {
     const Shape& sh = L.sh;
     const int max_m = L.max_m;
-    const bool use_tc = !L.force_simt && L.tmap_encode && assign_tc_supported(L);
+    const bool use_tc = !L.force_simt && L.tmap_encode && assign_tc_supported(L) && !sh.band_w;
     if (fused_small) {
         Timed t(L, KID_SEEDS);
         decide_small_kernel<T><<<sh.n_units, 256, 0, L.stream>>>(
@@ -408,6 +554,15 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const i
         if (use_tc) {
             cudaError_t e = launch_assign_tc(L, prm, s, plan, kind, seed_of, sim, ws, L.tmap_encode);
             if (e != cudaSuccess) return e;
+        } else if (sh.band_w) {
+            const size_t smem = (size_t)2 * kTile * (sh.d / 2 + 1) * sizeof(float2) + ((size_t)2 * kTile + sh.d / 2) * sizeof(float);
+            cudaError_t e = cudaFuncSetAttribute(assign_band_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 (int)smem);
+            if (e != cudaSuccess) return e;
+            Timed t(L, KID_ASSIGN);
+            assign_band_kernel<T><<<dim3((L.max_T + kTile - 1) / kTile, sh.n_units), kThreads, smem, L.stream>>>(
+                L.desc, sh, (const T*)L.k, s, plan, ws.seed_rows, (const T*)ws.seed_k, kind, seed_of, sim, ws.grp,
+                ws.mass_fx, ws.njoin, max_m, prm.tau, prm.eps);
         } else {
         const size_t smem = ((size_t)2 * kTile * (sh.d + 1) + kTile) * sizeof(float);
         cudaError_t e = cudaFuncSetAttribute(assign_simt_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,

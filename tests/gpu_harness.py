@@ -26,7 +26,7 @@ WEIGHT_RTOL = 2e-5
 
 
 def run_oracle(hb: wl.Batch, **kw) -> Dict:
-    """kw: tau, gamma, causal, eps, mass_in (per-row carried masses), chan_w (similarity channel weights)."""
+    """kw: tau, gamma, causal, eps, mass_in (per-row carried masses), chan_w (similarity channel weights), band_w / band_layout (per-band distance)."""
     w = hb.wl
     if hb.mass_in is not None:
         kw.setdefault("mass_in", hb.mass_in)
@@ -38,7 +38,7 @@ class GpuRun:
     """Device copies of a host batch plus everything needed to call the library on it."""
 
     def __init__(self, hb: wl.Batch, device="cuda:0", row_stride=None, lse_in=None, page_size=0, bad_page=None,
-                 mass_in=None, chan_w=None, **prm_kw):
+                 mass_in=None, chan_w=None, band_w=None, band_layout=0, **prm_kw):
         import torch
         from paper_2604_10900_b200 import binding as cb
         self.cb, self.torch, self.hb = cb, torch, hb
@@ -83,10 +83,12 @@ class GpuRun:
             k_off = None
         self.mass_in = None if mass_in is None else torch.from_numpy(np.ascontiguousarray(mass_in, np.float32)).to(device)
         self.chan_w = None if chan_w is None else torch.from_numpy(np.ascontiguousarray(chan_w, np.float32)).to(device)
+        self.band_w = None if band_w is None else torch.from_numpy(np.ascontiguousarray(band_w, np.float32)).to(device)
         self.lse_in = None if lse_in is None else torch.from_numpy(np.ascontiguousarray(lse_in, np.float32)).to(device)
         self.batch, self._keep = cb.make_batch(
             self.dev["k"], self.dev["v"], self.dev["q"], hb.T, hb.P, hb.B, hb.reserve, hb.tok_off, d, w.group,
-            w.window, w.dtype, k_off=k_off, row_stride=row_stride, lse_in=self.lse_in, mass_in=self.mass_in, chan_w=self.chan_w, **paged)
+            w.window, w.dtype, k_off=k_off, row_stride=row_stride, lse_in=self.lse_in, mass_in=self.mass_in, chan_w=self.chan_w,
+            band_w=self.band_w, band_layout=band_layout, **paged)
         self.prm = cb.params(**prm_kw)
         self.ctx = cb.Context(torch.device(device).index or 0, torch.cuda.current_stream(device).cuda_stream)
         self.ws, self.ws_bytes = cb.alloc_workspace(self.batch, self.prm, device)

@@ -118,6 +118,34 @@ def test_channel_weighted_similarity(name, kw, tensor_assign):
     assert not np.array_equal(plain["sim"], o["sim"])
 
 
+@pytest.mark.parametrize("name,kw,layout", [
+    ("reasoning32k_b512", dict(layers=1, kv_heads=2, decode=2048 + 77), 0),
+    ("reasoning32k_b1024", dict(layers=1, kv_heads=2, decode=2048 + 77), 1),       # m = 192: three seed steps
+    ("serving_steady_b512", dict(layers=1, kv_heads=2, n_seqs=2), 0),              # short units, carried masses
+    ("tiny", dict(), 1)])
+def test_band_distance_similarity(name, kw, layout):
+    """Sec. 2.5 in its own form: d_kappa = sum_f w_f ||k_if - k_jf|| over rotary bands, as the similarity
+    1 - d_kappa / (D_i + D_j), in place of the cosine."""
+    import gpu_harness as gh
+    w = _small(name, **kw)
+    hb = wl.make_batch(w)
+    rng = np.random.default_rng(7)
+    bw = (rng.random(w.head_dim // 2) ** 2 + 0.02).astype(np.float32)
+    bw[rng.random(w.head_dim // 2) < 0.1] = 0.0                 # bands of no future relevance
+    run = gh.GpuRun(hb, band_w=bw, band_layout=layout, tau=0.8)
+    g = run.event()
+    assert run.ctx.device_flags() == 0
+    o = gh.run_oracle(hb, band_w=bw, band_layout=layout, tau=0.8)
+    st = gh.compare_event(hb, g, o)
+    assert st["cascaded"] <= 1 and st["merged_elems"] > 0
+    other = gh.run_oracle(hb, band_w=bw, band_layout=1 - layout, tau=0.8)
+    assert not np.array_equal(other["sim"], o["sim"])
+    # both kinds of weights at once are refused before any launch
+    cb = run.cb
+    bad = gh.GpuRun(hb, band_w=bw, chan_w=np.ones(w.head_dim, np.float32))
+    assert cb.cask_compress_event(bad.ctx, bad.batch, bad.prm, bad.out_struct, bad.ws, bad.ws_bytes, check=False) == cb.ERR_SHAPE
+
+
 @pytest.mark.parametrize("group,window", [(1, 32), (3, 32), (1, 128), (2, 128), (3, 128), (5, 96)])
 def test_query_row_counts_that_fill_one_to_four_accumulator_slots(group, window):
     """32 to 480 window-query rows: one, two, three and four 128-column slots, a ragged last slot, idle epilogue
@@ -378,10 +406,11 @@ def test_bad_arguments_are_refused_on_the_host_before_any_launch():
     run.event()
 
 
-@pytest.mark.parametrize("extras", [False, True])
+@pytest.mark.parametrize("extras", [0, 1, 2])
 def test_host_buffer_entry_point_matches_device_entry_point(extras):
     """cask_compress_event_host (host K/V/Q and host outputs; only the value rows that are read go up) gives the
-    bytes of the device call, also with carried masses and channel weights passed as host arrays."""
+    bytes of the device call, also with carried masses and channel weights (1) or band weights (2) passed as host
+    arrays."""
     import gpu_harness as gh
     import torch
     w = _small("reasoning8k_b384", layers=1, kv_heads=2, decode=1000)
@@ -389,12 +418,13 @@ def test_host_buffer_entry_point_matches_device_entry_point(extras):
     rng = np.random.default_rng(3)
     mass = (np.where(rng.random(int(hb.tok_off[-1])) < 0.3, rng.random(int(hb.tok_off[-1])) * 1e-3, 0.0)
             .astype(np.float32)) if extras else None
-    cw = (rng.random(w.head_dim) + 0.05).astype(np.float32) if extras else None
-    run = gh.GpuRun(hb, mass_in=mass, chan_w=cw)
+    cw = (rng.random(w.head_dim) + 0.05).astype(np.float32) if extras == 1 else None
+    bw = (rng.random(w.head_dim // 2) + 0.05).astype(np.float32) if extras == 2 else None
+    run = gh.GpuRun(hb, mass_in=mass, chan_w=cw, band_w=bw, band_layout=1)
     g = run.event()
     cb = run.cb
     hbatch, keep = cb.make_batch(hb.k, hb.v, hb.q, hb.T, hb.P, hb.B, hb.reserve, hb.tok_off, w.head_dim, w.group,
-                                 w.window, w.dtype, mass_in=mass, chan_w=cw)
+                                 w.window, w.dtype, mass_in=mass, chan_w=cw, band_w=bw, band_layout=1)
     nbytes = cb.cask_host_event_device_bytes(hbatch, run.prm, run.Bmax)
     assert nbytes > 0
     dev = torch.empty(nbytes, dtype=torch.uint8, device="cuda:0")
