@@ -381,6 +381,41 @@ void cask_oracle_diagnostics(const double* s, int T, int B, const uint8_t* kind,
     free(it);
 }
 
+/*
+ * Within-group dispersion, the first term of the perturbation bound of Sec. 2.6:
+ *     sum over groups G of  sum_{i in G} a_i || k_i - k~_G ||_kappa ,
+ * a_i the merge weights' numerators (orc_a), k~_G the representative as the cache holds it: k_rep[slot] is passed in,
+ * rounded to the cache's number format by the caller (a lone seed is its own copy and adds nothing).  The norm is the
+ * one of the merge geometry in use: Euclidean; sqrt(sum_c w_c x_c^2) with channel weights; sum_f w_f ||x_f||_2 with
+ * band weights (reading: the paper names the norm ||.||_kappa and gives it no formula beyond d_kappa of Sec. 2.5).
+ */
+double cask_oracle_dispersion(const float* K, const double* s, int T, int d, double eps, const double* mass_in,
+                              const uint8_t* kind, const int* assign, const float* k_rep, const float* chan_w,
+                              const float* band_w, int band_layout) {
+    double total = 0.0;
+    double* dd = (double*)malloc(sizeof(double) * (size_t)d);
+    for (int i = 0; i < T; ++i) {
+        if (kind[i] != 4 && kind[i] != 5) continue;
+        int slot = assign[i];
+        if (slot < 0) continue;
+        for (int c = 0; c < d; ++c) dd[c] = (double)K[(size_t)i * d + c] - (double)k_rep[(size_t)slot * d + c];
+        double norm = 0.0;
+        if (band_w) {
+            for (int f = 0; f < d / 2; ++f) {
+                int c0, c1;
+                orc_band(f, d, band_layout, &c0, &c1);
+                norm += (double)band_w[f] * sqrt(dd[c0] * dd[c0] + dd[c1] * dd[c1]);
+            }
+        } else {
+            for (int c = 0; c < d; ++c) norm += (chan_w ? (double)chan_w[c] : 1.0) * dd[c] * dd[c];
+            norm = sqrt(norm);
+        }
+        total += orc_a(s, mass_in, eps, i) * norm;
+    }
+    free(dd);
+    return total;
+}
+
 /* The whole event for one unit, the steps above in order.  plan[8] is written. */
 void cask_oracle_event(const float* K, const float* V, const float* Q, int T, int P, int B, int reserve,
                        int d, int g, int W, int causal, double gamma, double tau, double eps,

@@ -136,6 +136,26 @@ def compact(K, V, kind, seed_of, weight, s, eps: float = 1e-9, mass_in=None):
                 slot_mass=slot_mass[:n], assign=assign, weight=weight)
 
 
+def dispersion(K, s, kind, assign, k_rep, eps: float = 1e-9, mass_in=None, chan_w=None, band_w=None,
+               band_layout: int = 0) -> float:
+    """Within-group dispersion of one unit (Sec. 2.6): sum_i a_i ||k_i - k_rep[assign[i]]|| over the rows of kind 4/5.
+    ``k_rep`` [n_out, d] holds the representatives as stored (rounded to the cache dtype by the caller)."""
+    K = _f32(K)
+    T, d = K.shape
+    s = np.ascontiguousarray(s, dtype=np.float64)
+    kind = np.ascontiguousarray(kind, dtype=np.uint8)
+    assign = np.ascontiguousarray(assign, dtype=np.int32)
+    k_rep = _f32(k_rep)
+    mass_in = None if mass_in is None else np.ascontiguousarray(mass_in, dtype=np.float64)
+    chan_w = None if chan_w is None else np.ascontiguousarray(chan_w, dtype=np.float32)
+    band_w = None if band_w is None else np.ascontiguousarray(band_w, dtype=np.float32)
+    fn = lib().cask_oracle_dispersion
+    fn.restype = C.c_double
+    return float(fn(_p(K, C.c_float), _p(s, C.c_double), T, d, C.c_double(eps), _p(mass_in, C.c_double),
+                    _p(kind, C.c_uint8), _p(assign, C.c_int), _p(k_rep, C.c_float), _p(chan_w, C.c_float),
+                    _p(band_w, C.c_float), int(band_layout)))
+
+
 def event_batch(K, V, Q, tok_off, P, B, reserve, causal: int = 1, gamma: float = 0.5, tau: float = 0.9,
                 eps: float = 1e-9, mass_in=None, chan_w=None, band_w=None, band_layout: int = 0) -> Dict[str, np.ndarray]:
     """Whole event for many contiguous units.  K, V [sum T, d]; Q [n, g, W, d] (float32 values)."""

@@ -465,6 +465,45 @@ def test_band_distance_geometry():
             _cmp_with_bruteforce(K[:14], V[:14], Q, 2, 7, 4, tau, band_w=bw, band_layout=layout)
 
 
+def test_within_group_dispersion():
+    """Sec. 2.6, first term of the bound: sum_i a_i ||k_i - k~_G|| over group members.  Hand-worked values for
+    the three norms; exact duplicates have none; a two-member group with equal weights and the exact representative
+    has a_1 |delta|/2 + a_2 |delta|/2; brute force over a whole event."""
+    K = np.array([[1, 0, 0, 0], [3, 4, 0, 0], [0, 0, 0, 0]], np.float32)
+    s = np.array([0.2, 0.3, 0.5])
+    kind = np.array([4, 5, 0], np.uint8)
+    asg = np.array([0, 0, -1], np.int32)
+    rep = np.array([[1, 0, 0, 0]], np.float32)
+    assert abs(orc.dispersion(K, s, kind, asg, rep, eps=0.0) - 0.3 * math.sqrt(20.0)) < 1e-15
+    assert abs(orc.dispersion(K, s, kind, asg, rep, eps=0.0, chan_w=[4, 0.25, 1, 1]) - 0.3 * math.sqrt(16 + 4)) < 1e-15
+    assert abs(orc.dispersion(K, s, kind, asg, rep, eps=0.0, band_w=[1, 2], band_layout=1) - 0.3 * math.sqrt(20.0)) < 1e-15
+    assert abs(orc.dispersion(K, s, kind, asg, rep, eps=0.0, band_w=[1, 2], band_layout=0) - 0.3 * (2 + 2 * 4)) < 1e-15
+    assert abs(orc.dispersion(K, s, kind, asg, rep, eps=0.0, mass_in=[0, 0.7, 0]) - 1.0 * math.sqrt(20.0)) < 1e-15
+    # a whole event on exact duplicates: every representative equals its members
+    rng = np.random.default_rng(23)
+    T, d, W = 30, 8, 2
+    centres = rng.standard_normal((3, d)).astype(np.float32)
+    K = centres[rng.integers(0, 3, T)]
+    V = rng.standard_normal((T, d)).astype(np.float32)
+    Q = rng.standard_normal((2, W, d)).astype(np.float32)
+    o = orc.event(K, V, Q, 0, 10, 10, tau=0.99)
+    assert (o["kind"] == 5).any()
+    assert orc.dispersion(K, o["s"], o["kind"], o["assign"], o["k_out"]) < 1e-12
+    # noisy clusters: the definition written out with numpy on the oracle's own groups and representatives
+    K = (centres[rng.integers(0, 3, T)] + 0.1 * rng.standard_normal((T, d))).astype(np.float32)
+    o = orc.event(K, V, Q, 0, 10, 10, tau=0.8)
+    mem = np.flatnonzero(np.isin(o["kind"], (4, 5)))
+    a = o["s"][mem] + 1e-9
+    want = float(np.sum(a * np.linalg.norm(K[mem].astype(np.float64) - o["k_out"][o["assign"][mem]], axis=1)))
+    got = orc.dispersion(K, o["s"], o["kind"], o["assign"], o["k_out"].astype(np.float32))
+    assert want > 0 and abs(got - want) < 1e-6 * want
+    # two members, equal weights: each lies |delta|/2 from the mean
+    K2 = np.array([[1, 1, 0, 0], [3, 1, 0, 0]], np.float32)
+    d2 = orc.dispersion(K2, np.array([0.5, 0.5]), np.array([4, 5], np.uint8), np.array([0, 0], np.int32),
+                        np.array([[2, 1, 0, 0]], np.float32), eps=0.0)
+    assert abs(d2 - 1.0) < 1e-15
+
+
 def test_whole_event_against_bruteforce_exhausted_boundary():
     rng = np.random.default_rng(11)
     T, P, W, d = 16, 10, 3, 4
