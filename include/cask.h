@@ -170,6 +170,11 @@ typedef struct {
        cache that the protected core (recent + core rows) holds, and that the output slots carry */
     float* rho_core;
     float* rho_rep;
+    /* optional, [n_units]: within-group dispersion, the first term of the perturbation bound of Sec. 2.6:
+       sum over the rows of kind 4/5 of a_i * ||k_i - k~_G||, k~_G the representative as written to k_out, in the
+       norm of the merge geometry in use (Euclidean; sqrt(sum_c w_c x_c^2) with chan_w; sum_f w_f ||x_f||_2 with
+       band_w).  The second term of that bound is lost_mass. */
+    float* dispersion;
 } cask_outputs;
 
 /* ---- context ------------------------------------------------------------ */
@@ -266,7 +271,7 @@ int cask_consolidate_scratch(cask_ctx* ctx, const cask_batch* batch, const cask_
  * copy); every other slot is a byte copy of its row.  `weight` is read for
  * kinds 4/5 and finalised (1 for kinds 1..3, 0 for kind 0).  Uses out->k_out,
  * v_out, Bmax, n_out, slot_src, slot_kind, slot_mass, assign and, when given,
- * rho_core / rho_rep; other fields of `out` are ignored.
+ * rho_core / rho_rep / dispersion; other fields of `out` are ignored.
  */
 int cask_compact(cask_ctx* ctx, const cask_batch* batch, const cask_params* params,
                  const float* s, const uint8_t* kind, const int32_t* seed_of, float* weight,

@@ -62,7 +62,7 @@ class CaskOutputs(C.Structure):
         ("assign", C.c_void_p), ("weight", C.c_void_p), ("kind", C.c_void_p), ("seed_of", C.c_void_p),
         ("plan", C.c_void_p), ("unit_status", C.c_void_p), ("lost_mass", C.c_void_p),
         ("s", C.c_void_p), ("lse", C.c_void_p), ("sim", C.c_void_p),
-        ("rho_core", C.c_void_p), ("rho_rep", C.c_void_p),
+        ("rho_core", C.c_void_p), ("rho_rep", C.c_void_p), ("dispersion", C.c_void_p),
     ]
 
 
@@ -378,7 +378,7 @@ def alloc_outputs(n_units: int, sum_T: int, Bmax: int, d: int, rows: int, dtype:
     if optional:
         o.update(s=z((sum_T,), torch.float32), lse=z((n_units, rows), torch.float32),
                  sim=z((sum_T,), torch.float32), rho_core=z((n_units,), torch.float32),
-                 rho_rep=z((n_units,), torch.float32))
+                 rho_rep=z((n_units,), torch.float32), dispersion=z((n_units,), torch.float32))
     return o
 
 

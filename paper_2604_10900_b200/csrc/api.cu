@@ -506,7 +506,7 @@ int cask_compact(cask_ctx* ctx, const cask_batch* b, const cask_params* p, const
     rc = prepare(ctx, b, p, ws, ws_bytes, L, W);
     if (rc != CASK_OK || b->n_units == 0) return rc;
     cudaError_t e = launch_compact(L, *p, s, kind, seed_of, weight, *out, W);
-    if (e == cudaSuccess) e = launch_diagnostics(L, s, kind, *out);
+    if (e == cudaSuccess) e = launch_diagnostics(L, *p, s, kind, *out);
     return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
 }
 
@@ -533,7 +533,7 @@ static int event_decide(cask_ctx* ctx, Launch& L, Workspace& W, const cask_batch
 static int event_compact(cask_ctx* ctx, Launch& L, Workspace& W, const cask_params* p, const cask_outputs* out) {
     float* s = out->s ? out->s : W.s;
     cudaError_t e = launch_compact(L, *p, s, out->kind, out->seed_of, out->weight, *out, W);
-    if (e == cudaSuccess) e = launch_diagnostics(L, s, out->kind, *out);
+    if (e == cudaSuccess) e = launch_diagnostics(L, *p, s, out->kind, *out);
     return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
 }
 
@@ -622,6 +622,7 @@ HostStage stage_layout(char* base, const cask_batch* b, const cask_params* p, in
     h.o.sim = (float*)take(sumT * 4);
     h.o.rho_core = (float*)take(n * 4);
     h.o.rho_rep = (float*)take(n * 4);
+    h.o.dispersion = (float*)take(n * 4);
     h.ws_bytes = carve(nullptr, b, batch_sizes(b, p)).bytes;
     h.ws = take(h.ws_bytes);
     h.bytes = off;
@@ -765,6 +766,7 @@ int cask_compress_event_host(cask_ctx* ctx, const cask_batch* hb, const cask_par
         {ho->lost_mass, h.o.lost_mass, n * 4}, {ho->s, h.o.s, sumT * 4},
         {ho->lse, h.o.lse, n * rows * 4}, {ho->sim, h.o.sim, sumT * 4},
         {ho->rho_core, h.o.rho_core, n * 4}, {ho->rho_rep, h.o.rho_rep, n * 4},
+        {ho->dispersion, h.o.dispersion, n * 4},
     };
     for (const Cp& c : cps) {
         if (!c.dst) continue;

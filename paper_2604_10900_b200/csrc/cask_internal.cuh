@@ -141,8 +141,9 @@ cudaError_t launch_compact(const Launch& L, const cask_params& prm, const float*
 cudaError_t launch_value_ranks(const Launch& L, const uint8_t* kind, int32_t* v_pos, int32_t* n_need, int64_t* v_base);
 // Paged cache: copies the compacted rows into the unit's own pages (slot t -> logical row t).
 cudaError_t launch_writeback(const Launch& L, const cask_outputs& out, void* k_pool, void* v_pool);
-// rho_core / rho_rep of Sec. 2.6 per unit (either pointer may be NULL).
-cudaError_t launch_diagnostics(const Launch& L, const float* s, const uint8_t* kind, const cask_outputs& out);
+// rho_core / rho_rep and the within-group dispersion of Sec. 2.6 per unit (any of the pointers may be NULL).
+cudaError_t launch_diagnostics(const Launch& L, const cask_params& prm, const float* s, const uint8_t* kind,
+                               const cask_outputs& out);
 
 // Tensor-core assignment of scratch rows to seeds (cosine Gram + argmax), same outputs as the SIMT kernel.
 bool assign_tc_supported(const Launch& L);

@@ -82,13 +82,70 @@ __global__ void __launch_bounds__(kSelThreads) diagnostics_kernel(
     }
 }
 
+// Within-group dispersion (Sec. 2.6, first term of the bound): sum_i a_i ||k_i - k~_G|| over the rows of kind 4/5, k~_G
+// read back from k_out.  One CTA per unit, one warp per member row in turn; a lane takes the bands lane, lane + 32, ...
+// (both channels of a band, so the per-band norm needs no exchange); fixed-order double-precision sums.
+template <typename T>
+__global__ void __launch_bounds__(256) dispersion_kernel(
+    const UnitDesc* __restrict__ desc, Shape sh, const T* __restrict__ K, const float* __restrict__ s, float eps,
+    const uint8_t* __restrict__ kind, const int32_t* __restrict__ assign, const T* __restrict__ k_out, int Bmax,
+    float* __restrict__ dispersion) {
+    __shared__ double red[8];
+    const int u = blockIdx.x;
+    const UnitDesc& ud = desc[u];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    const int nb = sh.d / 2;
+    const int second = (sh.band_w && sh.band_layout == 1) ? 1 : nb, step = (sh.band_w && sh.band_layout == 1) ? 2 : 1;
+    double acc = 0.0;
+    for (int i = w; i < ud.T; i += nw) {
+        const uint8_t kd = kind[ud.tok_off + i];
+        if (kd != CASK_KIND_SEED && kd != CASK_KIND_MERGED) continue;      // the same for the whole warp
+        const int slot = assign[ud.tok_off + i];
+        if (slot < 0 || slot >= Bmax) continue;
+        const T* kr = K + row_elem_off(sh, ud, ud.k_off, i);
+        const T* rep = k_out + ((size_t)u * Bmax + slot) * sh.d;
+        float part = 0.f;
+        for (int f = lane; f < nb; f += 32) {
+            const int c0 = f * step, c1 = c0 + second;
+            const float dx = Elem<T>::ld(kr + c0) - Elem<T>::ld(rep + c0), dy = Elem<T>::ld(kr + c1) - Elem<T>::ld(rep + c1);
+            if (sh.band_w) part = fmaf(sh.band_w[f], sqrtf(fmaf(dx, dx, dy * dy)), part);
+            else if (sh.chan_w) part = fmaf(sh.chan_w[c0] * dx, dx, fmaf(sh.chan_w[c1] * dy, dy, part));
+            else part = fmaf(dx, dx, fmaf(dy, dy, part));
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+        const float norm = sh.band_w ? part : sqrtf(part);
+        acc += (double)row_mass(sh, s, eps, ud.tok_off + i) * (double)norm;
+    }
+    if (lane == 0) red[w] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int x = 0; x < nw; ++x) t += red[x];
+        dispersion[u] = (float)t;
+    }
+}
+
 }  // namespace
 
-cudaError_t launch_diagnostics(const Launch& L, const float* s, const uint8_t* kind, const cask_outputs& out) {
-    if (!out.rho_core && !out.rho_rep) return cudaSuccess;
-    Timed t(L, KID_DIAGNOSTICS);
-    diagnostics_kernel<<<L.sh.n_units, kSelThreads, 0, L.stream>>>(L.desc, s, kind, out.slot_mass, out.n_out, out.Bmax,
-                                                                  out.rho_core, out.rho_rep);
+cudaError_t launch_diagnostics(const Launch& L, const cask_params& prm, const float* s, const uint8_t* kind,
+                               const cask_outputs& out) {
+    if (out.rho_core || out.rho_rep) {
+        Timed t(L, KID_DIAGNOSTICS);
+        diagnostics_kernel<<<L.sh.n_units, kSelThreads, 0, L.stream>>>(L.desc, s, kind, out.slot_mass, out.n_out,
+                                                                      out.Bmax, out.rho_core, out.rho_rep);
+    }
+    if (out.dispersion) {
+        Timed t(L, KID_DIAGNOSTICS);
+        if (L.sh.dtype == CASK_DTYPE_BF16)
+            dispersion_kernel<__nv_bfloat16><<<L.sh.n_units, 256, 0, L.stream>>>(
+                L.desc, L.sh, (const __nv_bfloat16*)L.k, s, prm.eps, kind, out.assign, (const __nv_bfloat16*)out.k_out,
+                out.Bmax, out.dispersion);
+        else
+            dispersion_kernel<float><<<L.sh.n_units, 256, 0, L.stream>>>(L.desc, L.sh, (const float*)L.k, s, prm.eps, kind,
+                                                                        out.assign, (const float*)out.k_out, out.Bmax,
+                                                                        out.dispersion);
+    }
     return cudaGetLastError();
 }
 

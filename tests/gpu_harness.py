@@ -156,9 +156,13 @@ def exempt_rows(o: Dict, u: int, a: int, T: int, P: int, tau: float) -> np.ndarr
 
 
 def compare_event(hb: wl.Batch, g: Dict, o: Dict, tau: float = 0.9, eps: float = 1e-9,
-                  check_scores: bool = True) -> Dict:
-    """Asserts parity of a GPU event `g` with the oracle event `o`; returns statistics."""
+                  check_scores: bool = True, geom: Dict = None) -> Dict:
+    """Asserts parity of a GPU event `g` with the oracle event `o`; returns statistics.  `geom`: what the event was
+    run with beyond the defaults (mass_in, chan_w, band_w, band_layout, eps), for the dispersion diagnostic."""
     w = hb.wl
+    disp_kw = dict(geom or {})
+    if hb.mass_in is not None:
+        disp_kw.setdefault("mass_in", hb.mass_in)
     d = w.head_dim
     kf, vf = wl.as_float32(hb.k, w.dtype), wl.as_float32(hb.v, w.dtype)
     st = dict(units=hb.n_units, exempt_rows=0, flipped_rows=0, cascaded=0, merged_elems=0, strict_ok=0,
@@ -216,6 +220,16 @@ def compare_event(hb: wl.Batch, g: Dict, o: Dict, tau: float = 0.9, eps: float =
         if "rho_core" in g and "rho_core" in o:      # Sec. 2.6 diagnostics
             assert np.isclose(g["rho_core"][u], o["rho_core"][u], rtol=2e-5, atol=1e-7), (u, g["rho_core"][u], o["rho_core"][u])
             assert np.isclose(g["rho_rep"][u], o["rho_rep"][u], rtol=2e-5, atol=1e-7), (u, g["rho_rep"][u], o["rho_rep"][u])
+        if "dispersion" in g:                        # Sec. 2.6: within-group dispersion against the stored representatives
+            krep = o["k_out"][u][:n_out]
+            krep = orc.round_bf16(krep) if w.dtype == wl.DTYPE_BF16 else krep.astype(np.float32)
+            want = orc.dispersion(kf[sl], o["s"][sl], o["kind"][sl], o["assign"][sl], krep, eps=disp_kw.get("eps", 1e-9),
+                                  mass_in=None if disp_kw.get("mass_in") is None else np.asarray(disp_kw["mass_in"])[sl],
+                                  chan_w=disp_kw.get("chan_w"), band_w=disp_kw.get("band_w"),
+                                  band_layout=disp_kw.get("band_layout", 0))
+            # a representative may differ from the oracle's by one unit in the last place of the cache dtype
+            assert np.isclose(g["dispersion"][u], want, rtol=2e-3, atol=1e-9), (u, g["dispersion"][u], want)
+            st["dispersion_checked"] = st.get("dispersion_checked", 0) + 1
         # per-slot weight sums (Sec. 2.4: a convex combination)
         sums = np.bincount(g["assign"][sl][g["assign"][sl] >= 0], weights=wg[g["assign"][sl] >= 0], minlength=n_out)
         assert np.allclose(sums, 1.0, atol=1e-5)

@@ -90,7 +90,8 @@ def test_carried_mass_second_event_on_a_compacted_cache():
     run2 = gh.GpuRun(hb2, mass_in=mass)
     g2 = run2.event()
     o2 = gh.run_oracle(hb2, mass_in=mass.astype(np.float64))
-    st2 = gh.compare_event(hb2, g2, o2)
+    st2 = gh.compare_event(hb2, g2, o2, geom=dict(mass_in=mass))
+    assert st2["dispersion_checked"] > 0
     assert (g2["n_out"] == B).all() and st2["merged_elems"] > 0 and st2["cascaded"] <= 1
     # the carried mass changes the fold: without it the merged rows come out differently
     g3 = gh.GpuRun(hb2).event()
@@ -112,7 +113,7 @@ def test_channel_weighted_similarity(name, kw, tensor_assign):
     run = gh.GpuRun(hb, chan_w=cw)
     g = run.event()
     o = gh.run_oracle(hb, chan_w=cw)
-    st = gh.compare_event(hb, g, o)
+    st = gh.compare_event(hb, g, o, geom=dict(chan_w=cw))
     assert st["cascaded"] <= 1 and st["merged_elems"] > 0
     plain = gh.run_oracle(hb)
     assert not np.array_equal(plain["sim"], o["sim"])
@@ -136,7 +137,8 @@ def test_band_distance_similarity(name, kw, layout):
     g = run.event()
     assert run.ctx.device_flags() == 0
     o = gh.run_oracle(hb, band_w=bw, band_layout=layout, tau=0.8)
-    st = gh.compare_event(hb, g, o)
+    st = gh.compare_event(hb, g, o, tau=0.8, geom=dict(band_w=bw, band_layout=layout))
+    assert st["dispersion_checked"] > 0
     assert st["cascaded"] <= 1 and st["merged_elems"] > 0
     other = gh.run_oracle(hb, band_w=bw, band_layout=1 - layout, tau=0.8)
     assert not np.array_equal(other["sim"], o["sim"])
