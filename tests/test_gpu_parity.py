@@ -60,42 +60,72 @@ def test_many_seeds_share_accumulator_buffers():
     assert st["cascaded"] <= 1 and st["merged_elems"] > 0
 
 
-def test_carried_mass_second_event_on_a_compacted_cache():
-    """Steady state: the cache left by one event, grown by 128 new decode rows, is compressed again; its
-    representatives bring the group mass they were given (a_i = s_i + eps + carried mass)."""
+def _next_cache(w, hb, o, rng, n_new=128):
+    """The cache a serving loop holds after an event and n_new more decode steps, built from the ORACLE's result of
+    that event (rounded to the cache dtype): its compacted rows, then n_new appended rows of which half repeat kept
+    rows with a little noise; representatives carry the group mass they were given."""
+    from oracle import cask_oracle as orc
+    d = w.head_dim
+    k2, v2, mass, T2, P2 = [], [], [], [], []
+    for u in range(hb.n_units):
+        n = int(o["n_out"][u])
+        ko = wl.to_cache_dtype(orc.round_bf16(o["k_out"][u][:n]), w.dtype)
+        vo = wl.to_cache_dtype(orc.round_bf16(o["v_out"][u][:n]), w.dtype)
+        pkeep = int(o["plan"][u][1])
+        fresh_k = wl.to_cache_dtype(rng.standard_normal((n_new, d)).astype(np.float32) * wl.channel_scale(w, 0, 0), w.dtype)
+        src = rng.integers(pkeep, n, n_new // 2)
+        noisy = wl.as_float32(ko[src], w.dtype) + 0.05 * rng.standard_normal((n_new // 2, d)).astype(np.float32)
+        fresh_k[: n_new // 2] = wl.to_cache_dtype(noisy, w.dtype)
+        k2.append(np.concatenate([ko, fresh_k]))
+        v2.append(np.concatenate([vo, wl.to_cache_dtype(rng.standard_normal((n_new, d)).astype(np.float32), w.dtype)]))
+        mass.append(np.concatenate([np.where(o["slot_kind"][u][:n] == 4, o["slot_mass"][u][:n], 0.0), np.zeros(n_new)]))
+        T2.append(n + n_new)
+        P2.append(pkeep)
+    T2 = np.array(T2, np.int32)
+    hb2 = wl.Batch(wl=w, k=np.concatenate(k2), v=np.concatenate(v2), q=hb.q, T=T2, P=np.array(P2, np.int32), B=hb.B,
+                   reserve=hb.reserve, tok_off=np.concatenate([[0], np.cumsum(T2)]).astype(np.int64),
+                   unit_ids=hb.unit_ids, mass_in=np.concatenate(mass).astype(np.float32))
+    return hb2
+
+
+def test_carried_mass_trigger_loop_on_compacted_caches():
+    """Steady state of a serving loop: the cache left by one event, grown by 128 new decode rows, is compressed
+    again, three times over; representatives bring the group mass they were given (a_i = s_i + eps + carried mass).
+    Every event's inputs are built from the oracle's previous result, identical bytes for both sides; the second
+    event runs on a paged cache and is written back into its pages."""
     import gpu_harness as gh
+    import torch
     w = _small("reasoning8k_b384", layers=1, kv_heads=3, decode=2048)
     hb, run, g, o, st = _run(w)
     rng = np.random.default_rng(77)
-    n_new, d, B = 128, w.head_dim, w.budget
-    ko, vo = run.out["k_out"].view(run.torch.uint16).cpu().numpy(), run.out["v_out"].view(run.torch.uint16).cpu().numpy()
-    k2, v2, mass, T2, P2 = [], [], [], [], []
-    for u in range(hb.n_units):
-        n = int(g["n_out"][u])
-        fresh_k = wl.to_cache_dtype(rng.standard_normal((n_new, d)).astype(np.float32) * wl.channel_scale(w, 0, 0), w.dtype)
-        # half of the new rows repeat kept rows with a little noise, so that the second event merges again
-        src = rng.integers(int(g["plan"][u][1]), n, n_new // 2)
-        noisy = wl.bf16_bits_to_f32(ko[u][src]) + 0.05 * rng.standard_normal((n_new // 2, d)).astype(np.float32)
-        fresh_k[: n_new // 2] = wl.to_cache_dtype(noisy, w.dtype)
-        k2.append(np.concatenate([ko[u][:n], fresh_k]))
-        v2.append(np.concatenate([vo[u][:n], wl.to_cache_dtype(rng.standard_normal((n_new, d)).astype(np.float32), w.dtype)]))
-        mass.append(np.concatenate([np.where(g["slot_kind"][u][:n] == 4, g["slot_mass"][u][:n], 0.0), np.zeros(n_new)]))
-        T2.append(n + n_new)
-        P2.append(int(g["plan"][u][1]))
-    T2 = np.array(T2, np.int32)
-    hb2 = wl.Batch(wl=w, k=np.concatenate(k2), v=np.concatenate(v2), q=hb.q, T=T2, P=np.array(P2, np.int32), B=hb.B,
-                   reserve=hb.reserve, tok_off=np.concatenate([[0], np.cumsum(T2)]).astype(np.int64), unit_ids=hb.unit_ids)
-    mass = np.concatenate(mass).astype(np.float32)
-    assert (mass > 0).any()
-    run2 = gh.GpuRun(hb2, mass_in=mass)
-    g2 = run2.event()
-    o2 = gh.run_oracle(hb2, mass_in=mass.astype(np.float64))
-    st2 = gh.compare_event(hb2, g2, o2, geom=dict(mass_in=mass))
-    assert st2["dispersion_checked"] > 0
-    assert (g2["n_out"] == B).all() and st2["merged_elems"] > 0 and st2["cascaded"] <= 1
+    B = w.budget
+    for step in range(3):
+        hb = _next_cache(w, hb, o, rng)
+        assert (hb.mass_in > 0).any() and int(hb.T.max()) <= 1024          # the small-unit kernels serve it
+        run = gh.GpuRun(hb, page_size=64 if step == 1 else 0)
+        g = run.event()
+        assert run.ctx.device_flags() == 0
+        o = gh.run_oracle(hb)
+        st = gh.compare_event(hb, g, o)
+        assert st["dispersion_checked"] > 0
+        assert (g["n_out"] == B).all() and st["merged_elems"] > 0 and st["cascaded"] <= 1
+        if step == 1:
+            cb = run.cb
+            cb.cask_writeback_paged(run.ctx, run.batch, run.prm, run.out_struct, run.dev["k"], run.dev["v"], run.ws,
+                                    run.ws_bytes)
+            torch.cuda.synchronize()
+            table = run.block_table.cpu().numpy().astype(np.int64)
+            off = 0
+            for u in range(hb.n_units):
+                t = np.arange(int(g["n_out"][u]))
+                rows = torch.from_numpy(table[off + t // 64] * 64 + t % 64).to(run.device)
+                assert torch.equal(run.dev["k"][rows].view(torch.uint16), run.out["k_out"][u, :len(t)].view(torch.uint16))
+                off += (int(hb.T[u]) + 63) // 64
     # the carried mass changes the fold: without it the merged rows come out differently
-    g3 = gh.GpuRun(hb2).event()
-    assert np.array_equal(g3["kind"], g2["kind"]) and not np.array_equal(g3["weight"], g2["weight"])
+    plain = wl.Batch(wl=w, k=hb.k, v=hb.v, q=hb.q, T=hb.T, P=hb.P, B=hb.B, reserve=hb.reserve, tok_off=hb.tok_off,
+                     unit_ids=hb.unit_ids)
+    g3 = gh.GpuRun(plain).event()
+    assert np.array_equal(g3["kind"], g["kind"]) and not np.array_equal(g3["weight"], g["weight"])
 
 
 @pytest.mark.parametrize("name,kw,tensor_assign", [
