@@ -248,6 +248,40 @@ def test_ragged_batch_mixed_outcomes():
         assert np.array_equal(g1["v_out"][0][:n], g["v_out"][u][:n])
 
 
+@pytest.mark.parametrize("seed,max_rows", [(1, 1024), (2, 1024), (3, 2600)])
+def test_random_ragged_batches(seed, max_rows):
+    """48 units of random length, prefix, budget and reserve in one call (all at most 1,024 rows: the short-unit
+    kernels; or up to 2,600: the general ones), every one against the oracle.  Prefix-only units, units under budget,
+    exhausted decode budgets and single-slot budgets all occur."""
+    import gpu_harness as gh
+    rng = np.random.default_rng(seed)
+    base = wl.WORKLOADS["tiny"].with_(dtype=wl.DTYPE_BF16, head_dim=128, group=2, window=16, cluster_frac=0.6,
+                                      n_centres=0)
+    ks, vs, qs, T, P, B, R = [], [], [], [], [], [], []
+    for i in range(48):
+        t = int(rng.integers(16, max_rows + 1))
+        p = int(rng.integers(0, t - 15)) if rng.random() < 0.8 else t       # a fifth are prefix-only caches
+        b = int(rng.integers(1, min(t + 40, 700)))
+        r = int(rng.integers(0, b + 1))
+        w = base.with_(prefix=p, decode=t - p, budget=b, reserve=r)
+        k, v, q = wl.make_unit(w, i, seed, 0)
+        ks.append(k); vs.append(v); qs.append(q[None])
+        T.append(t); P.append(p); B.append(b); R.append(r)
+    hb = wl.Batch(wl=base, k=np.concatenate(ks), v=np.concatenate(vs), q=np.concatenate(qs),
+                  T=np.array(T, np.int32), P=np.array(P, np.int32), B=np.array(B, np.int32),
+                  reserve=np.array(R, np.int32), tok_off=np.concatenate([[0], np.cumsum(T)]).astype(np.int64),
+                  unit_ids=[(i, 0, 0) for i in range(len(T))])
+    run = gh.GpuRun(hb)
+    g = run.event()
+    assert run.ctx.device_flags() == 0
+    o = gh.run_oracle(hb)
+    st = gh.compare_event(hb, g, o)
+    from oracle import cask_oracle as orc
+    seen = np.bitwise_or.reduce(g["unit_status"])
+    assert seen & orc.NOOP_UNDER_BUDGET and seen & orc.PREFIX_EVICTED and seen & orc.DECODE_CONSOLIDATED
+    assert st["cascaded"] <= 4
+
+
 @pytest.mark.parametrize("tau", [-1.0, 1.5])
 def test_tau_extremes(tau):
     """tau = -1 merges every scratch row (no lost mass); tau > 1 is plain top-k eviction."""
