@@ -37,8 +37,8 @@ UNIT = "tokens/s"
 # DRAM bytes per cache row (dram__bytes_read.sum + dram__bytes_write.sum of one launch / rows streamed) from the
 # ncu captures summarised under profiles/; traffic grows in proportion to the rows a launch streams.
 NCU_TRAFFIC = {
-    "score_norm": (268.6, "profiles/score_tc_reasoning32k_16units.txt"),
-    "score_mass": (276.8, "profiles/score_tc_reasoning32k_16units.txt"),
+    "score_norm": (268.0, "profiles/score_tc_reasoning32k_16units.txt"),
+    "score_mass": (274.2, "profiles/score_tc_reasoning32k_16units.txt"),
     "assign": (266.2, "profiles/assign_tc_reasoning32k_16units.txt"),
 }
 # ex2 units: 16 results per clock per SM (special-function pipe), 148 SMs, 1.965 GHz maximum SM clock.
