@@ -467,6 +467,52 @@ void cask_oracle_event_batch(int n_units, const float* K, const float* V, const 
     }
 }
 
+/*
+ * Query-statistics scorer of the Phase-1 archive (App. B): the horizon kernel
+ *     kappa_{pi_h}(omega) = E_{delta ~ pi_h}[ e^{i omega delta} ] = sum_n pi_h[n] e^{i omega delta_n}
+ * for a discrete horizon distribution pi_h on the offsets delta_n, and the horizon-averaged mean score
+ *     S_h(k, Delta) = Re sum_f mu_{h,f} conj(k_f) kappa_{pi_h}(omega_f) e^{i omega_f Delta} ,
+ * with band f of a vector read as the complex number x[c0] + i x[c1] (channel pairs as in orc_band).  Reading: the
+ * score of cache row i is the mean of S_h over the g query heads of the KV head, at Delta_i = delta[i] when the
+ * caller gives offsets, else T - 1 - i (distance to the newest row).  The score is real and may be negative.
+ * mu [g, d/2, 2] (re, im), pi [g, n_delta], delta_grid [n_delta], omega [d/2].
+ */
+void cask_oracle_score_stats(const float* K, int T, int d, int g, const float* mu, const double* pi,
+                             const double* delta_grid, int n_delta, const double* omega, int band_layout,
+                             const double* delta, double* s) {
+    int nb = d / 2;
+    double* kr = (double*)malloc(sizeof(double) * (size_t)g * nb);      /* kappa_{h,f}: re */
+    double* ki = (double*)malloc(sizeof(double) * (size_t)g * nb);      /*              im */
+    for (int h = 0; h < g; ++h)
+        for (int f = 0; f < nb; ++f) {
+            double re = 0.0, im = 0.0;
+            for (int n = 0; n < n_delta; ++n) {
+                re += pi[(size_t)h * n_delta + n] * cos(omega[f] * delta_grid[n]);
+                im += pi[(size_t)h * n_delta + n] * sin(omega[f] * delta_grid[n]);
+            }
+            kr[h * nb + f] = re;
+            ki[h * nb + f] = im;
+        }
+    for (int i = 0; i < T; ++i) {
+        double D = delta ? delta[i] : (double)(T - 1 - i);
+        double tot = 0.0;
+        for (int h = 0; h < g; ++h)
+            for (int f = 0; f < nb; ++f) {
+                int c0, c1;
+                orc_band(f, d, band_layout, &c0, &c1);
+                double mr = mu[((size_t)h * nb + f) * 2], mi = mu[((size_t)h * nb + f) * 2 + 1];
+                double xr = K[(size_t)i * d + c0], xi = -(double)K[(size_t)i * d + c1];      /* conj(k_f) */
+                double ar = mr * xr - mi * xi, ai = mr * xi + mi * xr;                        /* mu conj(k) */
+                double br = ar * kr[h * nb + f] - ai * ki[h * nb + f];                       /* ... kappa  */
+                double bi = ar * ki[h * nb + f] + ai * kr[h * nb + f];
+                tot += br * cos(omega[f] * D) - bi * sin(omega[f] * D);                      /* Re(... e^{i omega D}) */
+            }
+        s[i] = tot / g;
+    }
+    free(kr);
+    free(ki);
+}
+
 /* Scores only, many units (used where only the dominant step is timed or compared). */
 void cask_oracle_score_batch(int n_units, const float* K, const float* Q, const int64_t* tok_off, int d,
                              int g, int W, int causal, double* s, double* lse_out) {

@@ -211,6 +211,25 @@ def event(K, V, Q, P: int, B: int, reserve: int, **kw) -> Dict[str, np.ndarray]:
     return out
 
 
+def score_stats(K, mu, pi, delta_grid, omega, band_layout: int = 0, delta=None) -> np.ndarray:
+    """Horizon-averaged mean score of one unit (App. B): K [T,d]; mu [g, d/2, 2]; pi [g, n_delta]; delta_grid
+    [n_delta]; omega [d/2]; optional per-row offsets delta [T] (default T-1-i).  Returns s [T] float64."""
+    K = _f32(K)
+    T, d = K.shape
+    mu = np.ascontiguousarray(mu, dtype=np.float32)
+    g = mu.shape[0]
+    pi = np.ascontiguousarray(pi, dtype=np.float64)
+    delta_grid = np.ascontiguousarray(delta_grid, dtype=np.float64)
+    omega = np.ascontiguousarray(omega, dtype=np.float64)
+    assert mu.shape == (g, d // 2, 2) and pi.shape == (g, delta_grid.size) and omega.shape == (d // 2,)
+    delta = None if delta is None else np.ascontiguousarray(delta, dtype=np.float64)
+    s = np.zeros(T, np.float64)
+    lib().cask_oracle_score_stats(_p(K, C.c_float), T, d, g, _p(mu, C.c_float), _p(pi, C.c_double),
+                                  _p(delta_grid, C.c_double), int(delta_grid.size), _p(omega, C.c_double),
+                                  int(band_layout), _p(delta, C.c_double), _p(s, C.c_double))
+    return s
+
+
 def score_batch(K, Q, tok_off, causal: int = 1):
     K, Q = _f32(K), _f32(Q)
     n, g, W, d = Q.shape

@@ -504,6 +504,57 @@ def test_within_group_dispersion():
     assert abs(d2 - 1.0) < 1e-15
 
 
+def test_query_statistics_scorer():
+    """App. B: horizon kernel kappa = E_{delta~pi}[e^{i omega delta}] and mean score
+    S = Re sum_f mu_f conj(k_f) kappa(omega_f) e^{i omega_f Delta}.  Closed forms: one band, mu = kappa = 1 gives
+    k_x cos(omega Delta) + k_y sin(omega Delta); a point-mass horizon at delta_0 shifts Delta by delta_0; a uniform
+    symmetric horizon gives the real Dirichlet kernel; the score is linear in mu; numpy complex arithmetic."""
+    rng = np.random.default_rng(29)
+    T, d, g = 9, 8, 3
+    nb = d // 2
+    K = rng.standard_normal((T, d)).astype(np.float32)
+    om = 1.0 / (50.0 ** (np.arange(nb) / nb))
+    # one band active, mu = 1, horizon = point mass at 0
+    for layout, (c0, c1) in ((0, (2, 2 + nb)), (1, (4, 5))):
+        mu = np.zeros((1, nb, 2), np.float32); mu[0, 2, 0] = 1.0
+        s = orc.score_stats(K, mu, [[1.0]], [0.0], om, layout)
+        D = T - 1 - np.arange(T)
+        want = K[:, c0] * np.cos(om[2] * D) + K[:, c1] * np.sin(om[2] * D)
+        assert np.abs(s - want).max() < 1e-12
+        # point mass at delta_0 = 3: the same score three steps later
+        s3 = orc.score_stats(K, mu, [[1.0]], [3.0], om, layout)
+        want3 = K[:, c0] * np.cos(om[2] * (D + 3)) + K[:, c1] * np.sin(om[2] * (D + 3))
+        assert np.abs(s3 - want3).max() < 1e-12
+        # explicit offsets replace T-1-i
+        sd = orc.score_stats(K, mu, [[1.0]], [0.0], om, layout, delta=np.full(T, 2.5))
+        assert np.abs(sd - (K[:, c0] * np.cos(om[2] * 2.5) + K[:, c1] * np.sin(om[2] * 2.5))).max() < 1e-12
+    # uniform horizon on {-a..a}: kappa is the Dirichlet kernel, real
+    a = 4
+    grid = np.arange(-a, a + 1, dtype=np.float64)
+    mu = np.zeros((1, nb, 2), np.float32); mu[0, 1, 0] = 1.0
+    s = orc.score_stats(K, mu, [np.full(2 * a + 1, 1.0 / (2 * a + 1))], grid, om, 0)
+    dirichlet = np.sin((2 * a + 1) * om[1] / 2) / ((2 * a + 1) * np.sin(om[1] / 2))
+    D = T - 1 - np.arange(T)
+    assert np.abs(s - dirichlet * (K[:, 1] * np.cos(om[1] * D) + K[:, 1 + nb] * np.sin(om[1] * D))).max() < 1e-12
+    # general case against numpy, linearity in mu, mean over heads
+    mu = rng.standard_normal((g, nb, 2)).astype(np.float32)
+    grid = np.array([0.0, 1.0, 2.0, 7.0])
+    pi = rng.random((g, 4)); pi /= pi.sum(1, keepdims=True)
+    for layout in (0, 1):
+        c0 = np.arange(nb) if layout == 0 else 2 * np.arange(nb)
+        c1 = c0 + (nb if layout == 0 else 1)
+        kc = K[:, c0].astype(np.float64) + 1j * K[:, c1]
+        muc = mu[..., 0].astype(np.float64) + 1j * mu[..., 1]
+        kap = (pi[:, :, None] * np.exp(1j * om[None, None, :] * grid[None, :, None])).sum(1)
+        want = np.real(np.einsum("hf,if,hf,if->i", muc, np.conj(kc), kap, np.exp(1j * om[None, :] * D[:, None]))) / g
+        got = orc.score_stats(K, mu, pi, grid, om, layout)
+        assert np.abs(got - want).max() < 1e-12
+        heads = [orc.score_stats(K, mu[h:h + 1], pi[h:h + 1], grid, om, layout) for h in range(g)]
+        assert np.abs(got - np.mean(heads, axis=0)).max() < 1e-12
+        assert np.abs(orc.score_stats(K, 2.0 * mu, pi, grid, om, layout) - 2.0 * got).max() < 1e-12
+    assert (got < 0).any() and (got > 0).any()
+
+
 def test_whole_event_against_bruteforce_exhausted_boundary():
     rng = np.random.default_rng(11)
     T, P, W, d = 16, 10, 3, 4
