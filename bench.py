@@ -433,6 +433,63 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_stats_scorer(args):
+    """Times the query-statistics scorer (App. B) alone: one pass over the keys, reported against HBM bandwidth."""
+    import torch
+    from paper_2604_10900_b200 import binding as cb
+    world, rank, local = _dist()
+    if rank != 0:
+        return
+    torch.cuda.set_device(local)
+    device = f"cuda:{local}"
+    w = wl.WORKLOADS[args.workload]
+    n_layers = min(w.layers, args.layer_slice or w.layers_per_pass or w.layers)
+    units = wl.unit_list(w, layers=range(n_layers))
+    if args.max_units:
+        units = units[:args.max_units]
+    hb = wl.make_batch(w, units, threads=min(16, os.cpu_count() or 8))
+    d, nb, sum_T = w.head_dim, w.head_dim // 2, int(hb.tok_off[-1])
+    dev = cb.to_device(hb, device)
+    batch, keep = cb.make_batch(dev["k"], dev["v"], dev["q"], hb.T, hb.P, hb.B, hb.reserve, hb.tok_off, d, w.group,
+                                w.window, w.dtype)
+    prm = cb.params()
+    stream = torch.cuda.current_stream(device)
+    ctx = cb.Context(local, stream.cuda_stream)
+    ws, ws_bytes = cb.alloc_workspace(batch, prm, device)
+    rng = np.random.default_rng(2604)
+    n_delta = 64
+    mu = torch.from_numpy(rng.standard_normal((hb.n_units, w.group, nb, 2)).astype(np.float32)).to(device)
+    pi = rng.random((hb.n_units, w.group, n_delta)).astype(np.float32)
+    pi = torch.from_numpy(pi / pi.sum(-1, keepdims=True)).to(device)
+    grid = torch.arange(n_delta, dtype=torch.float32, device=device) * 16.0
+    omega = torch.from_numpy((1.0 / (10000.0 ** (np.arange(nb) / nb))).astype(np.float32)).to(device)
+    qs, keep2 = cb.make_query_stats(mu, pi, grid, omega, 0)
+    s = torch.empty(sum_T, dtype=torch.float32, device=device)
+    for _ in range(max(args.warmup, 3)):
+        cb.cask_score_stats(ctx, batch, prm, qs, s, ws, ws_bytes)
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for _ in range(args.steps):
+        cb.cask_score_stats(ctx, batch, prm, qs, s, ws, ws_bytes)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / args.steps
+    peaks = _peaks()
+    byts = hb.k.nbytes + 4 * sum_T
+    gbs = byts / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": "kv_tokens_scored_per_s", "value": sum_T / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+        "dtype": "bf16" if w.dtype == wl.DTYPE_BF16 else "f32", "data": "synthetic",
+        "config": {"workload": w.name, "scorer": "query statistics (horizon kernel, mean score)", "units": hb.n_units,
+                   "rows_per_unit": int(hb.T.max()), "n_delta": n_delta,
+                   "l2": "inputs larger than L2: %.2f GB of K read per step" % (hb.k.nbytes / 1e9)},
+        "roofline": {"kernel": "score_stats_kernel", "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]},
+        "gpu_launches": 2 * args.steps}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -442,6 +499,9 @@ def main():
     ap.add_argument("--workload", default="reasoning32k_b512", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--score-path", type=int, default=0, help="0: tensor-core scoring when the shape allows, 1: SIMT")
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--scorer", default="attention", choices=["attention", "stats"],
+                    help="attention: the whole event with the windowed attention-mass score (default); "
+                         "stats: time the query-statistics scorer of App. B alone")
     ap.add_argument("--similarity", default="cosine", choices=["cosine", "channel", "band"],
                     help="merge similarity: cosine, channel-weighted inner product, or per-band distance (Sec. 2.5)")
     ap.add_argument("--cpu-units", type=int, default=0,
@@ -453,6 +513,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.scorer == "stats":
+        run_stats_scorer(args)
     else:
         run_ours(args)
 

@@ -235,6 +235,32 @@ int cask_score(cask_ctx* ctx, const cask_batch* batch, const cask_params* params
                float* s, float* lse_out, void* ws, size_t ws_bytes);
 
 /*
+ * A second scorer, from the query-statistics family of the paper's Phase-1 archive (App. B): the horizon kernel
+ *     kappa_{pi_h}(omega) = E_{delta ~ pi_h}[e^{i omega delta}] = sum_n pi_h[n] e^{i omega delta_n}
+ * of a discrete horizon distribution pi_h over the offsets delta_n, and the horizon-averaged mean score
+ *     S_h(k, Delta) = Re sum_f mu_{h,f} conj(k_f) kappa_{pi_h}(omega_f) e^{i omega_f Delta},
+ * band f of a vector read as the complex number x[c0] + i x[c1] (channel pairs as for band_w: band_layout 0 =
+ * (f, f + head_dim/2), 1 = (2f, 2f + 1)).  The paper gives the two formulas and none of mu, pi, omega, Delta; all
+ * come from the caller.  s_i = mean over the g query heads of S_h(k_i, Delta_i), Delta_i = delta[i] or, without
+ * `delta`, T - 1 - i (distance to the newest cached row).  No window queries are read and no exponentials taken:
+ * one pass over the keys, bound by HBM.  The score is real and can be negative; the merge weights of Sec. 2.4 need
+ * a_i > 0, so a caller that feeds these scores to the later stages must shift or clamp them first.
+ */
+typedef struct {
+    const float* mu;          /* DEVICE [n_units, group, head_dim/2, 2] (re, im): mean query per head and band */
+    const float* pi;          /* DEVICE [n_units, group, n_delta]: horizon distribution of each head           */
+    const float* delta_grid;  /* DEVICE [n_delta]: the offsets pi is defined on                                */
+    int32_t n_delta;          /* 1 .. 4096                                                                      */
+    const float* omega;       /* DEVICE [head_dim/2]: band frequencies                                          */
+    int32_t band_layout;      /* 0 | 1                                                                          */
+    const float* delta;       /* DEVICE [sumT] per-row offsets Delta_i, or NULL                                 */
+} cask_query_stats;
+
+/* s [sumT] fp32 out.  Uses batch->k, the row layout (contiguous or paged), T, tok_off, group and head_dim (even). */
+int cask_score_stats(cask_ctx* ctx, const cask_batch* batch, const cask_params* params,
+                     const cask_query_stats* stats, float* s, void* ws, size_t ws_bytes);
+
+/*
  * Stage 1, prefix eviction (Sec. 2.2): writes plan[n_units,8] and kind for the
  * prefix rows [0,P): the P_keep rows greatest under (score descending, row
  * ascending) get CASK_KIND_PREFIX, the others 0; all P rows if P <= B_p.

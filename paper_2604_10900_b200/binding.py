@@ -30,7 +30,7 @@ EXPORTS = (
     "cask_create", "cask_destroy", "cask_set_stream", "cask_strerror", "cask_last_cuda_error",
     "cask_launch_count", "cask_last_score_path_tensor", "cask_last_device_flags", "cask_profile_enable", "cask_profile_read",
     "cask_kernel_count", "cask_kernel_name", "cask_workspace_bytes", "cask_plan_host",
-    "cask_score", "cask_prefix_evict", "cask_select_core", "cask_consolidate_scratch", "cask_compact",
+    "cask_score", "cask_score_stats", "cask_prefix_evict", "cask_select_core", "cask_consolidate_scratch", "cask_compact",
     "cask_compress_event", "cask_writeback_paged", "cask_host_event_device_bytes", "cask_compress_event_host", "cask_score_noalloc",
 )
 
@@ -47,6 +47,13 @@ class CaskBatch(C.Structure):
         ("block_table", C.c_void_p), ("bt_off", C.c_void_p), ("n_pages", C.c_int64),
         ("mass_in", C.c_void_p), ("chan_w", C.c_void_p),
         ("band_w", C.c_void_p), ("band_layout", C.c_int32),
+    ]
+
+
+class CaskQueryStats(C.Structure):
+    _fields_ = [
+        ("mu", C.c_void_p), ("pi", C.c_void_p), ("delta_grid", C.c_void_p), ("n_delta", C.c_int32),
+        ("omega", C.c_void_p), ("band_layout", C.c_int32), ("delta", C.c_void_p),
     ]
 
 
@@ -99,6 +106,7 @@ def lib():
         L.cask_workspace_bytes.restype = sz
         L.cask_plan_host.argtypes = [PB, PP, vp]
         L.cask_score.argtypes = [vp, PB, PP, vp, vp, vp, sz]
+        L.cask_score_stats.argtypes = [vp, PB, PP, C.POINTER(CaskQueryStats), vp, vp, sz]
         L.cask_prefix_evict.argtypes = [vp, PB, PP, vp, vp, vp, vp, sz]
         L.cask_select_core.argtypes = [vp, PB, PP, vp, vp, vp, vp, sz]
         L.cask_consolidate_scratch.argtypes = [vp, PB, PP, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz]
@@ -265,6 +273,22 @@ def cask_plan_host(batch: CaskBatch, prm: CaskParams) -> np.ndarray:
 
 def cask_score(ctx: Context, batch, prm, s, lse_out, ws, ws_bytes: int, check: bool = True) -> int:
     rc = lib().cask_score(ctx.handle, C.byref(batch), C.byref(prm), _ptr(s), _ptr(lse_out), _ptr(ws), ws_bytes)
+    if check:
+        _check(rc, ctx)
+    return rc
+
+
+def make_query_stats(mu, pi, delta_grid, omega, band_layout: int = 0, delta=None):
+    """(struct, keep-alive) for cask_score_stats; every array is a device tensor (float32)."""
+    q = CaskQueryStats()
+    q.mu, q.pi, q.delta_grid, q.omega, q.delta = _ptr(mu), _ptr(pi), _ptr(delta_grid), _ptr(omega), _ptr(delta)
+    q.n_delta = int(delta_grid.shape[0])
+    q.band_layout = int(band_layout)
+    return q, (mu, pi, delta_grid, omega, delta)
+
+
+def cask_score_stats(ctx: Context, batch, prm, stats: CaskQueryStats, s, ws, ws_bytes: int, check: bool = True) -> int:
+    rc = lib().cask_score_stats(ctx.handle, C.byref(batch), C.byref(prm), C.byref(stats), _ptr(s), _ptr(ws), ws_bytes)
     if check:
         _check(rc, ctx)
     return rc

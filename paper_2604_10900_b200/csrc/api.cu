@@ -192,6 +192,7 @@ Workspace carve(char* base, const cask_batch* b, const Sizes& z) {
     w.n_seed = (int32_t*)take(n * 4);
     w.max_B = std::max(z.max_B, 1);
     w.err = (int32_t*)take(16);
+    w.stats_a = (float*)take((n + 4) * (size_t)b->head_dim * 4);      // per-unit coefficients + one table of band constants
     w.bytes = off;
     return w;
 }
@@ -444,6 +445,22 @@ int cask_score(cask_ctx* ctx, const cask_batch* b, const cask_params* p, float* 
     int rc = prepare(ctx, b, p, ws, ws_bytes, L, W);
     if (rc != CASK_OK || b->n_units == 0) return rc;
     return run_score(ctx, L, b, p, s, lse_out, W);
+}
+
+int cask_score_stats(cask_ctx* ctx, const cask_batch* b, const cask_params* p, const cask_query_stats* qs, float* s,
+                     void* ws, size_t ws_bytes) {
+    if (!s || !qs || !qs->mu || !qs->pi || !qs->delta_grid || !qs->omega) return CASK_ERR_NULL;
+    if (qs->n_delta < 1 || qs->n_delta > 4096 || (qs->band_layout != 0 && qs->band_layout != 1)) return CASK_ERR_SHAPE;
+    if (((uintptr_t)qs->mu | (uintptr_t)qs->pi | (uintptr_t)qs->delta_grid | (uintptr_t)qs->omega |
+         (uintptr_t)qs->delta) % 4)
+        return CASK_ERR_ALIGN;
+    Launch L{};
+    Workspace W{};
+    int rc = prepare(ctx, b, p, ws, ws_bytes, L, W);
+    if (rc != CASK_OK || b->n_units == 0) return rc;
+    if (b->head_dim & 1) return CASK_ERR_SHAPE;
+    cudaError_t e = launch_score_stats(L, *qs, s, W);
+    return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
 }
 
 int cask_prefix_evict(cask_ctx* ctx, const cask_batch* b, const cask_params* p, const float* s, uint8_t* kind,

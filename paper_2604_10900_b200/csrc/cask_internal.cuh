@@ -118,6 +118,7 @@ struct Workspace {
     int32_t* n_seed;     // [units]
     int32_t max_B;
     int32_t* err;        // [1]
+    float* stats_a;      // [units, d] query-statistics scorer: head-pooled mu * kappa per band (re, im)
     size_t bytes;
 };
 
@@ -150,6 +151,9 @@ bool assign_tc_supported(const Launch& L);
 int assign_tc_box_rows(const Shape& sh);   // rows per TMA box of the key stream, 0 if the page size does not fit
 cudaError_t launch_assign_tc(const Launch& L, const cask_params& prm, const float* s, const int32_t* plan,
                              uint8_t* kind, int32_t* seed_of, float* sim, Workspace& ws, void* tmap_encode_fn);
+
+// Query-statistics scorer (App. B): horizon kernel and horizon-averaged mean score, one pass over the keys.
+cudaError_t launch_score_stats(const Launch& L, const cask_query_stats& qs, float* s, Workspace& ws);
 
 // Tensor-core scoring (tcgen05 + TMA); returns cudaErrorNotSupported when the shape does not fit.
 bool score_tc_supported(const Launch& L);

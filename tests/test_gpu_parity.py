@@ -282,6 +282,64 @@ def test_random_ragged_batches(seed, max_rows):
     assert st["cascaded"] <= 4
 
 
+def _query_stats(w, n_units, rng, n_delta=9):
+    nb = w.head_dim // 2
+    mu = rng.standard_normal((n_units, w.group, nb, 2)).astype(np.float32)
+    pi = rng.random((n_units, w.group, n_delta)).astype(np.float32)
+    pi /= pi.sum(-1, keepdims=True)
+    grid = np.concatenate([[0.0], np.sort(rng.integers(1, 4096, n_delta - 1))]).astype(np.float32)
+    omega = (1.0 / (10000.0 ** (np.arange(nb) / nb))).astype(np.float32)       # rotary-embedding frequencies
+    return mu, pi, grid, omega
+
+
+@pytest.mark.parametrize("name,kw,layout,paged", [
+    ("reasoning32k_b512", dict(layers=1, kv_heads=2, decode=8192 + 77), 0, 0),
+    ("reasoning8k_b384", dict(layers=1, kv_heads=2, decode=3000), 1, 64),
+    ("tiny", dict(), 0, 0)])
+def test_query_statistics_scorer(name, kw, layout, paged):
+    """App. B: horizon kernel + horizon-averaged mean score, one pass over the keys, against the oracle.  The sum
+    has d/2 terms of size |A_f||k_f|; single-precision sine, cosine and accumulation leave an error of a few 1e-7
+    of sum_f |A_f||k_f| per row, so the bound is 2e-6 of that sum (about ten times what is seen)."""
+    import gpu_harness as gh
+    import torch
+    from oracle import cask_oracle as orc
+    w = _small(name, **kw)
+    hb = wl.make_batch(w)
+    rng = np.random.default_rng(41)
+    mu, pi, grid, omega = _query_stats(w, hb.n_units, rng)
+    run = gh.GpuRun(hb, page_size=paged)
+    cb = run.cb
+    dev = [torch.from_numpy(x).to(run.device) for x in (mu, pi, grid, omega)]
+    for use_delta in (False, True):
+        delta = rng.uniform(0.0, 40000.0, int(hb.tok_off[-1])).astype(np.float32) if use_delta else None
+        ddev = None if delta is None else torch.from_numpy(delta).to(run.device)
+        qs, keep = cb.make_query_stats(dev[0], dev[1], dev[2], dev[3], layout, ddev)
+        s = torch.full((int(hb.tok_off[-1]),), float("nan"), dtype=torch.float32, device=run.device)
+        cb.cask_score_stats(run.ctx, run.batch, run.prm, qs, s, run.ws, run.ws_bytes)
+        torch.cuda.synchronize()
+        assert run.ctx.device_flags() == 0
+        got = s.cpu().numpy().astype(np.float64)
+        kf = wl.as_float32(hb.k, w.dtype)
+        nb = w.head_dim // 2
+        c0 = np.arange(nb) if layout == 0 else 2 * np.arange(nb)
+        c1 = c0 + (nb if layout == 0 else 1)
+        worst = 0.0
+        for u in range(hb.n_units):
+            a, b = int(hb.tok_off[u]), int(hb.tok_off[u + 1])
+            want = orc.score_stats(kf[a:b], mu[u], pi[u].astype(np.float64), grid.astype(np.float64),
+                                   omega.astype(np.float64), layout, None if delta is None else delta[a:b].astype(np.float64))
+            kap = (pi[u].astype(np.float64)[:, :, None] * np.exp(1j * omega[None, None, :].astype(np.float64) * grid[None, :, None])).sum(1)
+            A = np.abs(((mu[u][..., 0] + 1j * mu[u][..., 1]) * kap).mean(0))
+            scale = (np.hypot(kf[a:b][:, c0], kf[a:b][:, c1]) * A[None, :]).sum(1)
+            err = np.abs(got[a:b] - want) / scale
+            worst = max(worst, float(err.max()))
+        assert worst < 2e-6, worst
+        assert (got < 0).any() and (got > 0).any()
+    # arguments are checked on the host
+    bad, _ = cb.make_query_stats(dev[0], dev[1], dev[2], dev[3], 2)
+    assert cb.cask_score_stats(run.ctx, run.batch, run.prm, bad, s, run.ws, run.ws_bytes, check=False) == cb.ERR_SHAPE
+
+
 @pytest.mark.parametrize("tau", [-1.0, 1.5])
 def test_tau_extremes(tau):
     """tau = -1 merges every scratch row (no lost mass); tau > 1 is plain top-k eviction."""
