@@ -97,7 +97,7 @@ template <> struct Quad<float> {
     }
 };
 
-template <typename T, bool STEP>      // STEP: no caller-supplied offsets, Delta falls by one per row
+template <typename T, bool STEP, int LAYOUT>      // STEP: no caller-supplied offsets, Delta falls by one per row
 __global__ void __launch_bounds__(256) score_stats_kernel(const UnitDesc* __restrict__ desc, Shape sh, const T* __restrict__ K,
                                                              cask_query_stats qs, const float* __restrict__ A, BandTable tab,
                                                              int n_stages, float* __restrict__ s) {
@@ -116,11 +116,19 @@ __global__ void __launch_bounds__(256) score_stats_kernel(const UnitDesc* __rest
         if (k < n_tiles) {
             const int row0 = first_row + k * kRowsPerCta, nrows = min(kRowsPerCta, ud.T - row0);
             T* dst = stages + (size_t)(k % n_stages) * stage_elems;
-            for (int v = threadIdx.x; v < nrows * vec_per_row; v += blockDim.x) {
-                const int rr = v / vec_per_row, c = (v - rr * vec_per_row) * kPer;
-                const T* src = K + row_elem_off(sh, ud, ud.k_off, row0 + rr) + c;
-                const unsigned sa = (unsigned)__cvta_generic_to_shared(dst + (size_t)rr * d + c);
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(src) : "memory");
+            if (sh.page_size == 0 && sh.row_stride == d) {
+                // rows back to back in the cache: the tile is one contiguous run of 16-byte vectors
+                const T* src = K + ud.k_off + (int64_t)row0 * d;
+                const unsigned sa0 = (unsigned)__cvta_generic_to_shared(dst);
+                for (int v = threadIdx.x; v < nrows * vec_per_row; v += blockDim.x)
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa0 + 16u * v), "l"(src + (size_t)v * kPer) : "memory");
+            } else {
+                for (int v = threadIdx.x; v < nrows * vec_per_row; v += blockDim.x) {
+                    const int rr = v / vec_per_row, c = (v - rr * vec_per_row) * kPer;
+                    const T* src = K + row_elem_off(sh, ud, ud.k_off, row0 + rr) + c;
+                    const unsigned sa = (unsigned)__cvta_generic_to_shared(dst + (size_t)rr * d + c);
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(src) : "memory");
+                }
             }
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
@@ -179,7 +187,9 @@ __global__ void __launch_bounds__(256) score_stats_kernel(const UnitDesc* __rest
             Dm[j] = (unsigned)abs(Di);
             Dsg[j] = Di < 0 ? -2.3283064365386963e-10f : 2.3283064365386963e-10f;      // +-2^-32
         }
-        const bool rotate = STEP && r_first + 3 < nrows;          // all four rows exist: Delta falls by exactly one per row
+        // Without caller offsets Delta falls by exactly one per row: rows 1..3 turn the phase of row 0.  (Rows past
+        // the end of the unit get a phase that means nothing; they are not stored.)
+        constexpr bool rotate = STEP;
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         for (int qq = q; qq < nq; qq += 16) {
             QuadConst c = c0;
@@ -189,7 +199,7 @@ __global__ void __launch_bounds__(256) score_stats_kernel(const UnitDesc* __rest
             for (int j = 0; j < 4; ++j) {
                 const T* row = tile + (size_t)rloc[j] * d;
                 float kx[4], ky[4];
-                if (qs.band_layout == 0) {
+                if (LAYOUT == 0) {
                     Quad<T>::ld(row + 4 * qq, kx);
                     Quad<T>::ld(row + nb + 4 * qq, ky);
                 } else {
@@ -246,17 +256,24 @@ cudaError_t launch_score_stats(const Launch& L, const cask_query_stats& qs, floa
     const int rows_per_cta = kTilesPerCta * kRowsPerCta;
     const dim3 grid((L.max_T + rows_per_cta - 1) / rows_per_cta, sh.n_units);
     Timed t(L, KID_SCORE_MASS);
+    auto launch = [&](auto kern, const auto* kptr) -> cudaError_t {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        kern<<<grid, 256, smem, L.stream>>>(L.desc, sh, kptr, qs, ws.stats_a, tab, n_stages, s);
+        return cudaSuccess;
+    };
+    const bool step = qs.delta == nullptr;
+    cudaError_t e;
     if (sh.dtype == CASK_DTYPE_BF16) {
-        auto kern = qs.delta ? score_stats_kernel<__nv_bfloat16, false> : score_stats_kernel<__nv_bfloat16, true>;
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        kern<<<grid, 256, smem, L.stream>>>(L.desc, sh, (const __nv_bfloat16*)L.k, qs, ws.stats_a, tab, n_stages, s);
+        const __nv_bfloat16* kp = (const __nv_bfloat16*)L.k;
+        if (qs.band_layout == 0) e = step ? launch(score_stats_kernel<__nv_bfloat16, true, 0>, kp) : launch(score_stats_kernel<__nv_bfloat16, false, 0>, kp);
+        else e = step ? launch(score_stats_kernel<__nv_bfloat16, true, 1>, kp) : launch(score_stats_kernel<__nv_bfloat16, false, 1>, kp);
     } else {
-        auto kern = qs.delta ? score_stats_kernel<float, false> : score_stats_kernel<float, true>;
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        kern<<<grid, 256, smem, L.stream>>>(L.desc, sh, (const float*)L.k, qs, ws.stats_a, tab, n_stages, s);
+        const float* kp = (const float*)L.k;
+        if (qs.band_layout == 0) e = step ? launch(score_stats_kernel<float, true, 0>, kp) : launch(score_stats_kernel<float, false, 0>, kp);
+        else e = step ? launch(score_stats_kernel<float, true, 1>, kp) : launch(score_stats_kernel<float, false, 1>, kp);
     }
+    if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
 
