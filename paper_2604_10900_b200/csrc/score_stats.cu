@@ -105,20 +105,24 @@ __global__ void __launch_bounds__(256) score_stats_kernel(const UnitDesc* __rest
     const int u = blockIdx.y;
     const UnitDesc& ud = desc[u];
     const int first_row = blockIdx.x * kTilesPerCta * kRowsPerCta;
-    if (first_row >= ud.T) return;
+    // descriptor fields in registers: the asynchronous copies below are memory barriers to the compiler, which
+    // would otherwise read them again after every one
+    const int T_u = ud.T;
+    const int64_t tok_u = ud.tok_off, koff_u = ud.k_off;
+    if (first_row >= T_u) return;
     const int d = sh.d, nb = d / 2, nq = nb / 4;
-    const int n_tiles = min(kTilesPerCta, (ud.T - first_row + kRowsPerCta - 1) / kRowsPerCta);
+    const int n_tiles = min(kTilesPerCta, (T_u - first_row + kRowsPerCta - 1) / kRowsPerCta);
     constexpr int kPer = 16 / (int)sizeof(T);                 // elements per 16-byte vector
     const int vec_per_row = d / kPer;
     const size_t stage_elems = (size_t)kRowsPerCta * d;
     T* stages = reinterpret_cast<T*>(ring);
     auto issue = [&](int k) {                                  // tile k of this CTA into stage k % n_stages
         if (k < n_tiles) {
-            const int row0 = first_row + k * kRowsPerCta, nrows = min(kRowsPerCta, ud.T - row0);
+            const int row0 = first_row + k * kRowsPerCta, nrows = min(kRowsPerCta, T_u - row0);
             T* dst = stages + (size_t)(k % n_stages) * stage_elems;
             if (sh.page_size == 0 && sh.row_stride == d) {
                 // rows back to back in the cache: the tile is one contiguous run of 16-byte vectors
-                const T* src = K + ud.k_off + (int64_t)row0 * d;
+                const T* src = K + koff_u + (int64_t)row0 * d;
                 const unsigned sa0 = (unsigned)__cvta_generic_to_shared(dst);
                 for (int v = threadIdx.x; v < nrows * vec_per_row; v += blockDim.x)
                     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa0 + 16u * v), "l"(src + (size_t)v * kPer) : "memory");
@@ -167,7 +171,7 @@ __global__ void __launch_bounds__(256) score_stats_kernel(const UnitDesc* __rest
         else if (n_stages == 2) asm volatile("cp.async.wait_group 1;" ::: "memory");
         else asm volatile("cp.async.wait_group 0;" ::: "memory");
         __syncthreads();
-        const int row0 = first_row + k * kRowsPerCta, nrows = min(kRowsPerCta, ud.T - row0);
+        const int row0 = first_row + k * kRowsPerCta, nrows = min(kRowsPerCta, T_u - row0);
         const T* tile = stages + (size_t)(k % n_stages) * stage_elems;
         // offsets of this thread's rows: magnitude of the integer part, its sign, the fractional part
         unsigned Dm[4];
@@ -177,10 +181,10 @@ __global__ void __launch_bounds__(256) score_stats_kernel(const UnitDesc* __rest
         for (int j = 0; j < 4; ++j) {
             rloc[j] = min(r_first + j, nrows - 1);                // rows past the end repeat the last one; not stored
             const int i = row0 + rloc[j];
-            int Di = ud.T - 1 - i;
+            int Di = T_u - 1 - i;
             Df[j] = 0.f;
             if (!STEP) {
-                const float dv = qs.delta[ud.tok_off + i], fl = floorf(dv);
+                const float dv = qs.delta[tok_u + i], fl = floorf(dv);
                 Di = (int)fl;
                 Df[j] = dv - fl;
             }
@@ -232,7 +236,7 @@ __global__ void __launch_bounds__(256) score_stats_kernel(const UnitDesc* __rest
         for (int j = 0; j < 4; ++j) {
 #pragma unroll
             for (int off = 1; off < 16; off <<= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], off);
-            if (q == 0 && r_first + j < nrows) s[ud.tok_off + row0 + r_first + j] = acc[j];
+            if (q == 0 && r_first + j < nrows) s[tok_u + row0 + r_first + j] = acc[j];
         }
         __syncthreads();            // the stage is free for the tile issued at the top of the next round
     }
