@@ -534,15 +534,9 @@ static int event_decide(cask_ctx* ctx, Launch& L, Workspace& W, const cask_batch
     float* s = out->s ? out->s : W.s;
     int rc = run_score(ctx, L, b, p, s, out->lse, W);
     if (rc != CASK_OK) return rc;
-    const bool small = L.max_T <= kSmallUnitRows && L.sh.d <= 128;      // one fused selection kernel per unit
-    cudaError_t e = cudaSuccess;
-    if (!small) {
-        e = launch_prefix_evict(L, s, out->kind, out->plan);
-        if (e == cudaSuccess) e = launch_select_core(L, s, out->plan, out->kind);
-    }
-    if (e == cudaSuccess)
-        e = launch_consolidate(L, *p, s, out->plan, out->kind, out->seed_of, out->weight, out->sim,
-                               out->unit_status, out->lost_mass, W, small);
+    // the event leaves prefix eviction and core selection to the fused selection kernel of the consolidation step
+    cudaError_t e = launch_consolidate(L, *p, s, out->plan, out->kind, out->seed_of, out->weight, out->sim,
+                                       out->unit_status, out->lost_mass, W, true);
     return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
 }
 

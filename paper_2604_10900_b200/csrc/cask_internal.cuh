@@ -131,9 +131,9 @@ cudaError_t launch_select_core(const Launch& L, const float* s, const int32_t* p
 cudaError_t launch_consolidate(const Launch& L, const cask_params& prm, const float* s,
                                const int32_t* plan, uint8_t* kind, int32_t* seed_of, float* weight,
                                float* sim, int32_t* unit_status, float* lost_mass, Workspace& ws,
-                               bool fused_small = false);
-// fused_small: every unit has at most kSmallUnitRows rows and `plan`, `kind` are still unwritten; one kernel then
-// does the prefix eviction, the core and seed selection and the seed gather (the event path only).
+                               bool fused = false);
+// fused (the event path only): `plan` and `kind` are still unwritten; one kernel per unit then does the prefix eviction
+// and the core and seed selection, and for units of at most kSmallUnitRows rows the seed gather as well.
 constexpr int kSmallUnitRows = 1024;
 cudaError_t launch_compact(const Launch& L, const cask_params& prm, const float* s, const uint8_t* kind,
                            const int32_t* seed_of, float* weight, const cask_outputs& out, Workspace& ws);

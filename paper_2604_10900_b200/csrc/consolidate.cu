@@ -53,6 +53,45 @@ __global__ void __launch_bounds__(kSelThreads) seeds_kernel(const UnitDesc* __re
     });
 }
 
+// ---- 1 for longer units on the event path: prefix eviction, core and seed selection in one CTA per unit ----
+// The same result as prefix_evict_kernel, select_core_kernel and seeds_kernel in turn; the core and the seeds come out of
+// one pair of thresholds (block_topk2_mark) and the per-row arrays are initialised once.
+__global__ void __launch_bounds__(kSelThreads) decide_long_kernel(
+    const UnitDesc* __restrict__ desc, const float* __restrict__ s, int32_t* __restrict__ plan,
+    uint8_t* __restrict__ kind, int32_t* __restrict__ seed_of, float* __restrict__ weight, float* __restrict__ sim,
+    int32_t* __restrict__ grp, int32_t* __restrict__ seed_rows, unsigned long long* __restrict__ mass_fx,
+    int32_t* __restrict__ njoin, int max_m) {
+    __shared__ SelectSmem sm, sm2;
+    const int u = blockIdx.x;
+    const UnitDesc& ud = desc[u];
+    const int T = ud.T, P = ud.P;
+    const int64_t o = ud.tok_off;
+    const int pkeep = ud.plan[CASK_PLAN_PKEEP], c = ud.plan[CASK_PLAN_C], m = max(0, ud.plan[CASK_PLAN_M]);
+    const int r = max(0, min(ud.plan[CASK_PLAN_R], T - P));
+    if (threadIdx.x < 8) plan[u * 8 + threadIdx.x] = ud.plan[threadIdx.x];
+    const uint8_t pre = (P <= pkeep) ? CASK_KIND_PREFIX : CASK_KIND_DROPPED;
+    for (int i = threadIdx.x; i < T; i += blockDim.x) {
+        kind[o + i] = (i < P) ? pre : (i >= T - r ? CASK_KIND_RECENT : CASK_KIND_DROPPED);
+        seed_of[o + i] = -1;
+        weight[o + i] = 0.f;
+        grp[o + i] = -1;
+        if (sim) sim[o + i] = -2.f;
+    }
+    for (int j = threadIdx.x; j <= max_m; j += blockDim.x) mass_fx[(size_t)u * (max_m + 1) + j] = 0ull;
+    if (threadIdx.x == 0) njoin[u] = 0;
+    __syncthreads();
+    if (P > pkeep) block_topk_mark(s + o, kind + o, 0, P, pkeep, CASK_KIND_PREFIX, sm);
+    block_topk2_mark(s + o, kind + o, P, T - r, c, CASK_KIND_CORE, m, CASK_KIND_SEED, sm, sm2);
+    if (m <= 0) return;
+    block_ordered_rows(kind + o, P, T - r, CASK_KIND_SEED, sm, [&](unsigned idx, int i) {
+        if (idx < (unsigned)m) {
+            seed_rows[ud.seed_base + idx] = i;
+            seed_of[o + i] = i;
+            grp[o + i] = (int)idx;
+        }
+    });
+}
+
 // ---- 2. gather seed keys, their norms and their own mass ---------------------------------
 template <typename T>
 __global__ void seed_gather_kernel(const UnitDesc* __restrict__ desc, Shape sh, const T* __restrict__ K,
@@ -530,11 +569,17 @@ __global__ void weights_kernel(const UnitDesc* __restrict__ desc, Shape sh, cons
 template <typename T>
 cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const int32_t* plan, uint8_t* kind,
                 int32_t* seed_of, float* weight, float* sim, int32_t* unit_status, float* lost_mass,
-                Workspace& ws, bool fused_small) {
+                Workspace& ws, bool fused) {
     const Shape& sh = L.sh;
     const int max_m = L.max_m;
     const bool use_tc = !L.force_simt && L.tmap_encode && assign_tc_supported(L) && !sh.band_w;
-    if (fused_small) {
+    const bool small_units = L.max_T <= kSmallUnitRows && sh.d <= 128;
+    if (fused && !small_units) {
+        Timed t(L, KID_SEEDS);
+        decide_long_kernel<<<sh.n_units, kSelThreads, 0, L.stream>>>(L.desc, s, const_cast<int32_t*>(plan), kind, seed_of,
+                                                                     weight, sim, ws.grp, ws.seed_rows, ws.mass_fx, ws.njoin,
+                                                                     max_m);
+    } else if (fused) {
         Timed t(L, KID_SEEDS);
         decide_small_kernel<T><<<sh.n_units, 256, 0, L.stream>>>(
             L.desc, sh, (const T*)L.k, s, const_cast<int32_t*>(plan), kind, seed_of, weight, sim, ws.grp, ws.seed_rows,
@@ -545,7 +590,7 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const i
                                                                ws.grp, ws.seed_rows, ws.mass_fx, ws.njoin, max_m);
     }
     if (max_m > 0) {
-        if (!fused_small) {
+        if (!(fused && small_units)) {
             Timed t(L, KID_SEED_GATHER);
             seed_gather_kernel<T><<<dim3((max_m + 7) / 8, sh.n_units), 256, 0, L.stream>>>(
                 L.desc, sh, (const T*)L.k, s, plan, ws.seed_rows, (T*)ws.seed_k, ws.seed_norm, ws.mass_fx, max_m,
@@ -587,10 +632,10 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const i
 
 cudaError_t launch_consolidate(const Launch& L, const cask_params& prm, const float* s, const int32_t* plan,
                                uint8_t* kind, int32_t* seed_of, float* weight, float* sim,
-                               int32_t* unit_status, float* lost_mass, Workspace& ws, bool fused_small) {
+                               int32_t* unit_status, float* lost_mass, Workspace& ws, bool fused) {
     if (L.sh.dtype == CASK_DTYPE_BF16)
-        return run<__nv_bfloat16>(L, prm, s, plan, kind, seed_of, weight, sim, unit_status, lost_mass, ws, fused_small);
-    return run<float>(L, prm, s, plan, kind, seed_of, weight, sim, unit_status, lost_mass, ws, fused_small);
+        return run<__nv_bfloat16>(L, prm, s, plan, kind, seed_of, weight, sim, unit_status, lost_mass, ws, fused);
+    return run<float>(L, prm, s, plan, kind, seed_of, weight, sim, unit_status, lost_mass, ws, fused);
 }
 
 }  // namespace cask

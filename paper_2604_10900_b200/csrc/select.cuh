@@ -238,6 +238,86 @@ __device__ inline void block_topk_mark(const float* __restrict__ s, uint8_t* kin
     __syncthreads();
 }
 
+// Two selections in one: among rows [lo,hi) with kind == 0 the k1 greatest get mark1 and the next k2 get mark2, which
+// is what block_topk_mark(k1, mark1) followed by block_topk_mark(k2, mark2) gives.  The three histogram sweeps narrow
+// both thresholds (rank k1 and rank k1 + k2) at once, with a second histogram where their digit prefixes part; one
+// marking sweep follows.  A tie at either threshold, or a selection that takes every row, goes the plain way.
+__device__ inline void block_topk2_mark(const float* __restrict__ s, uint8_t* kind, int lo, int hi, int k1, uint8_t mark1,
+                                        int k2, uint8_t mark2, SelectSmem& sm, SelectSmem& sm2) {
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int span = hi - lo;
+    auto plain = [&]() {
+        block_topk_mark(s, kind, lo, hi, k1, mark1, sm);
+        block_topk_mark(s, kind, lo, hi, k2, mark2, sm);
+    };
+    if (k1 <= 0 || k2 <= 0 || span <= kSmallSpan) { plain(); return; }
+    const int iters = (span + nthr - 1) / nthr;
+    // ---- sweep 1: top 12 bits, shared by both thresholds ----
+    for (int b = tid; b < kSelBins; b += nthr) sm.hist[b] = 0;
+    __syncthreads();
+    unsigned mine = 0;
+    for (int it = 0; it < iters; ++it) {
+        const int i = lo + it * nthr + tid;
+        if (i < hi && kind[i] == 0) { atomicAdd(&sm.hist[order_key(s[i]) >> 20], 1u); ++mine; }
+    }
+    const unsigned n_elig = block_sum(mine, sm);
+    if ((unsigned)(k1 + k2) >= n_elig) { __syncthreads(); plain(); return; }
+    find_digit(sm, kSelBins, (unsigned)k1);
+    const unsigned a1 = sm.digit;
+    unsigned ka = sm.krem;
+    __syncthreads();
+    find_digit(sm, kSelBins, (unsigned)(k1 + k2));
+    const unsigned b1 = sm.digit;
+    unsigned kb = sm.krem;
+    __syncthreads();
+    // ---- sweeps 2 and 3: next 12 and last 8 bits; one histogram while the prefixes agree, else one each ----
+    unsigned pa = a1, pb = b1;           // prefixes so far
+    unsigned neq_a = 0, neq_b = 0;
+    for (int pass = 1; pass < 3; ++pass) {
+        const int bits = pass == 1 ? 12 : 8, shift = pass == 1 ? 8 : 0, nbins = 1 << bits;
+        const bool same = pa == pb;
+        for (int b = tid; b < nbins; b += nthr) { sm.hist[b] = 0; sm2.hist[b] = 0; }
+        __syncthreads();
+        for (int it = 0; it < iters; ++it) {
+            const int i = lo + it * nthr + tid;
+            if (i < hi && kind[i] == 0) {
+                const unsigned key = order_key(s[i]), pre = key >> (shift + bits), dg = (key >> shift) & (unsigned)(nbins - 1);
+                if (pre == pa) atomicAdd(&sm.hist[dg], 1u);
+                else if (pre == pb) atomicAdd(&sm2.hist[dg], 1u);
+            }
+        }
+        __syncthreads();
+        find_digit(sm, nbins, ka);
+        const unsigned da = sm.digit;
+        const unsigned ka2 = sm.krem;
+        neq_a = sm.neq;
+        __syncthreads();
+        unsigned db, kb2;
+        if (same) {
+            find_digit(sm, nbins, kb);
+            db = sm.digit; kb2 = sm.krem; neq_b = sm.neq;
+        } else {
+            find_digit(sm2, nbins, kb);
+            db = sm2.digit; kb2 = sm2.krem; neq_b = sm2.neq;
+        }
+        __syncthreads();
+        pa = (pa << bits) | da;
+        pb = (pb << bits) | db;
+        ka = ka2;
+        kb = kb2;
+    }
+    // pa, pb: keys of the rows of rank k1 and k1 + k2; ka of the neq_a rows equal to pa fall inside the first
+    // selection, kb of the neq_b rows equal to pb inside the two together
+    if (ka != neq_a || kb != neq_b) { plain(); return; }      // rows tie across a boundary: index order decides
+    for (int i = lo + tid; i < hi; i += nthr)
+        if (kind[i] == 0) {
+            const unsigned key = order_key(s[i]);
+            if (key >= pa) kind[i] = mark1;
+            else if (key >= pb) kind[i] = mark2;
+        }
+    __syncthreads();
+}
+
 // Rows of [lo,hi) with kind == want, in ascending order: calls emit(rank, row) for each.  Every
 // thread walks one contiguous chunk, so one block scan orders the whole range.
 template <typename Emit>
