@@ -666,6 +666,10 @@ int cask_compress_event_host(cask_ctx* ctx, const cask_batch* hb, const cask_par
     HostStage h = stage_layout(nullptr, hb, p, ho->Bmax);
     if (!dev_buf || dev_bytes < h.bytes || (uintptr_t)dev_buf % 256) return CASK_ERR_WORKSPACE;
     h = stage_layout((char*)dev_buf, hb, p, ho->Bmax);
+    // optional diagnostics are computed only when the caller has a place for them
+    if (!ho->rho_core) h.o.rho_core = nullptr;
+    if (!ho->rho_rep) h.o.rho_rep = nullptr;
+    if (!ho->dispersion) h.o.dispersion = nullptr;
     cudaError_t e = cudaSetDevice(ctx->device);
     if (e != cudaSuccess) return fail_cuda(ctx, e);
     cudaStream_t st = ctx->stream;
