@@ -340,6 +340,27 @@ def test_query_statistics_scorer(name, kw, layout, paged):
     assert cb.cask_score_stats(run.ctx, run.batch, run.prm, bad, s, run.ws, run.ws_bytes, check=False) == cb.ERR_SHAPE
 
 
+@pytest.mark.parametrize("decode", [600, 3000])
+def test_exact_duplicates_tie_at_the_selection_thresholds(decode):
+    """Decode rows that are exact copies of a few centres have exactly equal scores, so the core and seed thresholds
+    fall inside runs of equal keys and the row index decides (short-unit ranking and two-threshold radix select,
+    both through their tie paths); merged rows equal their centre."""
+    import gpu_harness as gh
+    w = _small("reasoning8k_b384", layers=1, kv_heads=2, decode=decode, noise=0.0, cluster_frac=1.0, n_centres=37)
+    hb = wl.make_batch(w)
+    run = gh.GpuRun(hb)
+    g = run.event()
+    o = gh.run_oracle(hb)
+    # the duplicates really tie: far fewer distinct scores than rows in the decode region
+    a, T, P = 0, int(hb.T[0]), int(hb.P[0])
+    assert len(np.unique(o["s"][a + P:a + T - w.window])) < (T - P) // 4
+    # Equal keys in differently masked tiles can come out one unit in the last place apart in fp32 (the masked and the
+    # plain block forms add in a different order), so a unit may resolve a run of ties differently from the oracle;
+    # compare_event accepts that only inside the tolerance band around a threshold.
+    st = gh.compare_event(hb, g, o)
+    assert st["exempt_rows"] > 0 and st["cascaded"] <= hb.n_units
+
+
 @pytest.mark.parametrize("tau", [-1.0, 1.5])
 def test_tau_extremes(tau):
     """tau = -1 merges every scratch row (no lost mass); tau > 1 is plain top-k eviction."""
@@ -393,6 +414,9 @@ def test_supplied_normalisers():
     # units of at most 1,024 rows: the event takes its fused selection kernel, the staged calls their own kernels
     ("reasoning8k_b384", dict(decode=600)),
     ("prompt_heavy", dict(prefix=700, decode=200, budget=512, reserve=160)),     # with prefix eviction
+    # exact duplicates: runs of equal scores across the thresholds, the fused selections take their tie paths
+    ("reasoning8k_b384", dict(decode=3000, noise=0.0, cluster_frac=1.0, n_centres=37)),
+    ("reasoning8k_b384", dict(decode=600, noise=0.0, cluster_frac=1.0, n_centres=37)),
 ])
 def test_deterministic_and_staged_equals_fused(name, kw):
     """Same inputs twice -> same bytes; the five staged calls give the event's bytes."""
