@@ -425,7 +425,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             const int64_t tok_off = desc[wk.u].tok_off;
             const int last_all = sh.causal ? T - sh.W : T - 1;     // last key every query sees
             const float* rc = tail->rc[seg % 3u];
-            float rc_next = -1.0e30f;
+            float nx_w = 0.f, nx_m = 0.f;      // next segment's row weight and offset: loaded now, used after the first tile
             bool has_next = false;
             if (PASS == 1) {
                 // The table of this segment was written during the previous one (before the loop for the first).
@@ -437,7 +437,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 // before that one, which is the one written next.
                 has_next = wk.has_next();
                 if (has_next && etid < rows)
-                    rc_next = log2f(roww[(size_t)(wk.u + 1) * rows + etid]) - rowm[(size_t)(wk.u + 1) * rows + etid];
+                    { nx_w = roww[(size_t)(wk.u + 1) * rows + etid]; nx_m = rowm[(size_t)(wk.u + 1) * rows + etid]; }
             } else {
                 mm[0] = mm[1] = kNegBig;
                 l_run[0] = l_run[1] = 0.f;
@@ -579,7 +579,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     }
                 }
                 if (PASS == 1 && t == 0 && has_next && ok) {       // before this tile's global stores
-                    tail->rc[(seg + 1) % 3u][etid] = rc_next;
+                    tail->rc[(seg + 1) % 3u][etid] = (etid < rows) ? log2f(nx_w) - nx_m : -1.0e30f;
                     mbar_arrive(&bar.rw_ready);
                 }
                 if (PASS == 1 && ok) {
