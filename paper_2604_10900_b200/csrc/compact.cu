@@ -315,9 +315,9 @@ __global__ void __launch_bounds__(256) slot_merge_kernel(
 
 // ---- 3b. units of at most kMergeStageRows rows: one CTA per unit, members sorted by representative in shared memory ----
 // Same arithmetic as slot_merge_kernel (members in ascending row order, one fp32 accumulator per channel).  The
-// unit's member list is staged once and sorted by representative with a stable counting sort (one warp places
-// 32 members per step: __match_any_sync gives every member its rank among the members of the same group in the
-// step), so a warp finds the members of its representative side by side and reads their rows four at a time.
+// unit's member list is staged once and sorted by representative with a stable counting sort (every member counts
+// the earlier members of its group in shared memory), so a warp finds the members of its representative side by side
+// and reads their rows four at a time.
 constexpr int kMergeStageRows = 1024;
 
 template <typename T, int CH>       // CH = d / 32 contiguous channels per lane
@@ -380,18 +380,13 @@ __global__ void __launch_bounds__(256, 4) slot_merge_small_kernel(
         if (tid == (int)blockDim.x - 1) start[ns] = run;      // the last thread ends on the total
     }
     __syncthreads();
-    if (w == 0) {
-        // stable placement, 32 members per step in ascending row order
-        for (int e0 = 0; e0 < nm; e0 += 32) {
-            const int e = e0 + lane;
-            const int j = (e < nm) ? (int)m_j[e] : -1;
-            const unsigned peers = __match_any_sync(0xffffffffu, j);
-            const unsigned below = peers & ((1u << lane) - 1u);
-            if (j >= 0) list[start[j] + fill[j] + __popc(below)] = e;
-            __syncwarp();
-            if (j >= 0 && below == 0u) fill[j] += __popc(peers);
-            __syncwarp();
-        }
+    // stable placement: a member's position inside its group is the number of earlier members of the same group
+    for (int e = tid; e < nm; e += blockDim.x) {
+        const int j = m_j[e];
+        if (j < 0) continue;
+        int before = 0;
+        for (int x = 0; x < e; ++x) before += m_j[x] == j;
+        list[start[j] + before] = e;
     }
     __syncthreads();
     struct alignas(CH * sizeof(T)) Vec { T x[CH]; };
