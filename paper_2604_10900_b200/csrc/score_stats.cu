@@ -44,32 +44,52 @@ __global__ void __launch_bounds__(256) stats_fold_kernel(int g, int nb, cask_que
         }
     for (int f0 = 0; f0 < nb; f0 += 64) {
         const int f = f0 + (threadIdx.x >> 2);
-        const double om = f < nb ? (double)qs.omega[f] : 0.0;
-        double ar = 0.0, ai = 0.0;
-        for (int h = 0; h < g; ++h) {
-            const float* pi = qs.pi + ((size_t)u * g + h) * qs.n_delta;
-            float kr = 0.f, ki = 0.f;
+        // omega_f / 2 pi in turns (float) and as a 0.64 fixed-point fraction: the phase of an offset is formed from its
+        // integer part by two 32-bit multiplies (whole turns wrap away) and from its fractional part in single precision,
+        // so the loop below needs no double-precision arithmetic
+        const double tr = f < nb ? (double)qs.omega[f] * (1.0 / kTwoPi) : 0.0;
+        const double frt = tr - floor(tr);
+        const float ot = (float)tr;
+        const unsigned long long ofx = (unsigned long long)(frt * 18446744073709551616.0);
+        const unsigned fx_hi = (unsigned)(ofx >> 32), fx_lo = (unsigned)ofx;
+        float ar = 0.f, ai = 0.f;
+        // e^{i omega_f delta_n} does not depend on the head: one sine and cosine per offset serve eight heads at a time
+        for (int h0 = 0; h0 < g; h0 += 8) {
+            float kr[8], ki[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) { kr[k] = 0.f; ki[k] = 0.f; }
             for (int n = part; n < qs.n_delta; n += 4) {
                 float sn, cs;
-                double th = om * (double)qs.delta_grid[n];
-                th -= kTwoPi * rint(th * (1.0 / kTwoPi));
-                sincosf((float)th, &sn, &cs);
-                kr = fmaf(pi[n], cs, kr);
-                ki = fmaf(pi[n], sn, ki);
+                const float dv = qs.delta_grid[n], fl = floorf(dv);
+                const int di = (int)fl;
+                const unsigned dm = (unsigned)abs(di);
+                const int hi = (int)(fx_hi * dm + __umulhi(fx_lo, dm));
+                const float turns = fmaf((float)hi, di < 0 ? -2.3283064365386963e-10f : 2.3283064365386963e-10f, ot * (dv - fl));
+                sincosf(6.2831853071795865f * turns, &sn, &cs);
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    if (h0 + k < g) {
+                        const float pv = qs.pi[((size_t)u * g + h0 + k) * qs.n_delta + n];
+                        kr[k] = fmaf(pv, cs, kr[k]);
+                        ki[k] = fmaf(pv, sn, ki[k]);
+                    }
             }
-            kr += __shfl_xor_sync(0xffffffffu, kr, 1);
-            ki += __shfl_xor_sync(0xffffffffu, ki, 1);
-            kr += __shfl_xor_sync(0xffffffffu, kr, 2);
-            ki += __shfl_xor_sync(0xffffffffu, ki, 2);
-            if (f < nb) {
-                const float* mu = qs.mu + (((size_t)u * g + h) * nb + f) * 2;
-                ar += (double)mu[0] * kr - (double)mu[1] * ki;
-                ai += (double)mu[0] * ki + (double)mu[1] * kr;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                kr[k] += __shfl_xor_sync(0xffffffffu, kr[k], 1);
+                ki[k] += __shfl_xor_sync(0xffffffffu, ki[k], 1);
+                kr[k] += __shfl_xor_sync(0xffffffffu, kr[k], 2);
+                ki[k] += __shfl_xor_sync(0xffffffffu, ki[k], 2);
+                if (f < nb && h0 + k < g) {
+                    const float* mu = qs.mu + (((size_t)u * g + h0 + k) * nb + f) * 2;
+                    ar += fmaf(mu[0], kr[k], -mu[1] * ki[k]);
+                    ai += fmaf(mu[0], ki[k], mu[1] * kr[k]);
+                }
             }
         }
         if (part == 0 && f < nb) {
-            A[((size_t)u * nb + f) * 2] = (float)(ar / g);
-            A[((size_t)u * nb + f) * 2 + 1] = (float)(ai / g);
+            A[((size_t)u * nb + f) * 2] = ar / (float)g;
+            A[((size_t)u * nb + f) * 2 + 1] = ai / (float)g;
         }
     }
 }

@@ -311,7 +311,7 @@ def test_query_statistics_scorer(name, kw, layout, paged):
     cb = run.cb
     dev = [torch.from_numpy(x).to(run.device) for x in (mu, pi, grid, omega)]
     for use_delta in (False, True):
-        delta = rng.uniform(0.0, 40000.0, int(hb.tok_off[-1])).astype(np.float32) if use_delta else None
+        delta = rng.uniform(-5000.0, 40000.0, int(hb.tok_off[-1])).astype(np.float32) if use_delta else None
         ddev = None if delta is None else torch.from_numpy(delta).to(run.device)
         qs, keep = cb.make_query_stats(dev[0], dev[1], dev[2], dev[3], layout, ddev)
         s = torch.full((int(hb.tok_off[-1]),), float("nan"), dtype=torch.float32, device=run.device)
