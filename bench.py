@@ -154,7 +154,8 @@ def run_ours(args):
         units = units[:args.max_units]
 
     def pinned(shape, dt):
-        t = torch.empty(tuple(shape), dtype={np.dtype(np.uint16): torch.uint16, np.dtype(np.float32): torch.float32}[np.dtype(dt)],
+        t = torch.empty(tuple(shape), dtype={np.dtype(np.uint16): torch.uint16, np.dtype(np.float32): torch.float32,
+                                             np.dtype(np.int32): torch.int32, np.dtype(np.uint8): torch.uint8}[np.dtype(dt)],
                         pin_memory=True)
         return t.numpy()
 
@@ -257,13 +258,16 @@ def run_ours(args):
     dev_buf = torch.empty(dev_bytes, dtype=torch.uint8, device=device)
     e = 2 if w.dtype == wl.DTYPE_BF16 else 4
     st = np.uint16 if w.dtype == wl.DTYPE_BF16 else np.float32
+    # every result lands in pinned memory: a copy into pageable memory would hold the host until it is done
     ho = dict(k_out=pinned((hb.n_units, Bmax, d), st), v_out=pinned((hb.n_units, Bmax, d), st),
-              n_out=np.zeros(hb.n_units, np.int32), slot_src=np.zeros((hb.n_units, Bmax), np.int32),
-              slot_kind=np.zeros((hb.n_units, Bmax), np.uint8), slot_mass=np.zeros((hb.n_units, Bmax), np.float32),
-              assign=pinned((sum_T,), np.float32).view(np.int32), weight=pinned((sum_T,), np.float32),
-              kind=np.zeros(sum_T, np.uint8), seed_of=pinned((sum_T,), np.float32).view(np.int32),
-              plan=np.zeros((hb.n_units, 8), np.int32), unit_status=np.zeros(hb.n_units, np.int32),
-              lost_mass=np.zeros(hb.n_units, np.float32))
+              n_out=pinned((hb.n_units,), np.int32), slot_src=pinned((hb.n_units, Bmax), np.int32),
+              slot_kind=pinned((hb.n_units, Bmax), np.uint8), slot_mass=pinned((hb.n_units, Bmax), np.float32),
+              assign=pinned((sum_T,), np.int32), weight=pinned((sum_T,), np.float32),
+              kind=pinned((sum_T,), np.uint8), seed_of=pinned((sum_T,), np.int32),
+              plan=pinned((hb.n_units, 8), np.int32), unit_status=pinned((hb.n_units,), np.int32),
+              lost_mass=pinned((hb.n_units,), np.float32))
+    for a in ho.values():
+        a[...] = 0
     ho_struct = cb.make_outputs(ho, Bmax)
     # The host entry point sends the keys and queries whole but only the value rows that are kept or merged
     # (counted from the row kinds of the device run); the row kinds come back once more in mid-call.

@@ -321,17 +321,32 @@ int cask_writeback_paged(cask_ctx* ctx, const cask_batch* batch, const cask_para
                          const cask_outputs* out, void* k_pool, void* v_pool, void* ws, size_t ws_bytes);
 
 /*
- * The same event for callers whose cache lives in HOST memory (ideally
- * page-locked): batch->k, v, q, lse_in and every pointer in `out` are HOST
+ * The same event for callers whose cache lives in HOST memory: batch->k, v,
+ * q, lse_in, mass_in, chan_w, band_w and every pointer in `out` are HOST
  * pointers here.  dev_buf is a DEVICE buffer of at least
  * cask_host_event_device_bytes() that holds the staged inputs, outputs and the
  * workspace.  Copies the keys and queries in, decides every row's fate, copies
  * in only the value rows that are kept or merged (gathered through a pinned
  * staging buffer the context owns and grows as needed), compacts, copies out
- * and synchronises the stream before returning; the results equal those of
- * cask_compress_event.  Rows of a unit must be dense (row_stride ==
- * head_dim) and units laid out at k_off[u] == v_off[u] == tok_off[u]*head_dim;
- * a paged batch is refused with CASK_ERR_UNSUPPORTED.
+ * and returns when everything has arrived.
+ *
+ * A batch with more than 16 MB of keys is cut into up to about ten slices of
+ * consecutive units, each a batch of its own inside dev_buf; they take turns
+ * on streams the context owns (ordered after the work already queued on the
+ * context's stream), so that one slice's upload runs while the slice before it
+ * is decided, packed, compacted and read back.  For that overlap every HOST
+ * array, inputs and outputs, has to be page-locked: a copy to or from pageable
+ * memory holds the calling thread until the copy is done.  Units are
+ * independent, so the results are those of cask_compress_event on the same
+ * units; against one call on the whole batch the last bits of the scores can
+ * differ, because the scoring kernel divides a unit's tiles between its CTAs
+ * according to what else is in the batch (a batch of one slice gives the same
+ * bytes).  cask_last_device_flags() afterwards gives the flags of all slices.
+ *
+ * Rows of a unit must be dense (row_stride == head_dim) and units laid out at
+ * k_off[u] == v_off[u] == tok_off[u]*head_dim; a paged batch is refused with
+ * CASK_ERR_UNSUPPORTED, a dev_buf that is too small or not 256-byte aligned
+ * with CASK_ERR_WORKSPACE.
  */
 size_t cask_host_event_device_bytes(const cask_batch* batch, const cask_params* params, int32_t Bmax);
 int cask_compress_event_host(cask_ctx* ctx, const cask_batch* host_batch, const cask_params* params,

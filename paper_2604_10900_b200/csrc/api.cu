@@ -51,6 +51,12 @@ struct cask_ctx {
     // host-buffer entry point: pinned staging for the row kinds coming back and the packed value rows going in
     char* hstage = nullptr;
     size_t hstage_bytes = 0;
+    // streams and events the slices of a large host batch take turns on; one flag word per slice
+    cudaStream_t hs[4] = {nullptr, nullptr, nullptr, nullptr};
+    cudaEvent_t hs_start = nullptr;
+    std::vector<cudaEvent_t> hs_kinds;
+    int32_t* hs_flags = nullptr;     // pinned, kMaxSlices words
+    int32_t flags_last = 0;          // flags of a call that has already read them back
     void* tmap_encode = nullptr;     // cuTensorMapEncodeTiled, resolved at creation
     Profiler prof;
     ProfImpl prof_impl;
@@ -265,6 +271,7 @@ int prepare(cask_ctx* ctx, const cask_batch* b, const cask_params* p, void* ws, 
     e = cudaMemsetAsync(W.err, 0, 16, ctx->stream);      // device-side flags of this call
     if (e != cudaSuccess) return fail_cuda(ctx, e);
     ctx->flags_dev = W.err;
+    ctx->flags_last = 0;
 
     L.stream = ctx->stream;
     L.sh.n_units = b->n_units; L.sh.d = b->head_dim; L.sh.g = b->group; L.sh.W = b->window;
@@ -338,6 +345,11 @@ int cask_destroy(cask_ctx* ctx) {
     if (ctx->pinned) cudaFreeHost(ctx->pinned);
     if (ctx->hstage) cudaFreeHost(ctx->hstage);
     if (ctx->staged) cudaEventDestroy(ctx->staged);
+    for (cudaStream_t st : ctx->hs)
+        if (st) cudaStreamDestroy(st);
+    if (ctx->hs_start) cudaEventDestroy(ctx->hs_start);
+    if (ctx->hs_flags) cudaFreeHost(ctx->hs_flags);
+    for (cudaEvent_t ev : ctx->hs_kinds) cudaEventDestroy(ev);
     for (ProfRecord& r : ctx->prof_impl.live) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     for (cudaEvent_t e : ctx->prof_impl.pool) cudaEventDestroy(e);
     delete ctx;
@@ -410,7 +422,7 @@ int cask_last_score_path_tensor(const cask_ctx* ctx) { return ctx ? ctx->last_tc
 
 int cask_last_device_flags(cask_ctx* ctx, int32_t* flags_host) {
     if (!ctx || !flags_host) return CASK_ERR_NULL;
-    *flags_host = 0;
+    *flags_host = ctx->flags_last;
     if (!ctx->flags_dev) return CASK_OK;
     cudaError_t e = cudaSetDevice(ctx->device);
     if (e == cudaSuccess)
@@ -578,6 +590,8 @@ int cask_writeback_paged(cask_ctx* ctx, const cask_batch* b, const cask_params* 
     return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
 }
 
+}  // extern "C"
+
 // ---- host-resident caches ------------------------------------------------------------------
 
 namespace {
@@ -646,11 +660,141 @@ int check_host_layout(const cask_batch* b) {
         if (b->k_off[u] != b->tok_off[u] * b->head_dim || b->v_off[u] != b->k_off[u]) return CASK_ERR_SHAPE;
     return CASK_OK;
 }
+
+// A large batch goes through the device in slices of consecutive units, so that one slice's upload runs while
+// the one before it is being decided, packed and read back.  A slice is a batch of its own: offsets rebased to
+// zero, host pointers moved to its first unit, its own staging area and workspace on the device.
+constexpr size_t kSliceMinBytes = (size_t)16 << 20;   // of keys; below this the copies are too short to hide anything
+constexpr int kSliceTarget = 10;                      // slices a large batch is cut into
+constexpr int kSliceStreams = 4;
+constexpr size_t kMaxSlices = 64;
+
+struct HostSlice {
+    int u0 = 0, u1 = 0;
+    int64_t r0 = 0;                      // first row (caller's tok_off) of the slice
+    std::vector<int64_t> tok, off;       // rebased offsets
+    cask_batch hb;                       // host pointers of the slice
+    cask_outputs ho;
+    HostStage h;                         // device staging
+    Launch L;
+    Workspace W;
+    size_t v_row0 = 0, need_rows = 0;    // place of the packed value rows in the pinned staging
+    std::vector<int64_t> vbase;
+};
+
+std::vector<int> slice_bounds(const cask_batch* b) {
+    const size_t row_bytes = (size_t)b->head_dim * elem_size(b->dtype);
+    const size_t total = (size_t)b->tok_off[b->n_units] * row_bytes;
+    const size_t target = std::max(kSliceMinBytes, total / kSliceTarget);
+    std::vector<int> bounds{0};
+    size_t acc = 0;
+    for (int u = 0; u < b->n_units; ++u) {
+        acc += (size_t)(b->tok_off[u + 1] - b->tok_off[u]) * row_bytes;
+        const size_t left = (size_t)(b->tok_off[b->n_units] - b->tok_off[u + 1]) * row_bytes;
+        if (acc >= target && left >= target / 2) {
+            bounds.push_back(u + 1);
+            acc = 0;
+        }
+    }
+    if (bounds.back() != b->n_units) bounds.push_back(b->n_units);
+    return bounds;
+}
+
+template <typename T>
+T* moved(T* p, size_t n) { return p ? p + n : nullptr; }
+inline void* moved_bytes(const void* p, size_t n) { return p ? (char*)p + n : nullptr; }
+
+void make_slice(HostSlice& s, const cask_batch* hb, const cask_outputs* ho, int u0, int u1) {
+    const size_t es = elem_size(hb->dtype), d = (size_t)hb->head_dim, rows = (size_t)hb->group * hb->window;
+    s.u0 = u0; s.u1 = u1; s.r0 = hb->tok_off[u0];
+    const size_t n = (size_t)(u1 - u0), r0 = (size_t)s.r0;
+    s.tok.resize(n + 1);
+    s.off.resize(n);
+    for (size_t u = 0; u <= n; ++u) s.tok[u] = hb->tok_off[u0 + u] - s.r0;
+    for (size_t u = 0; u < n; ++u) s.off[u] = s.tok[u] * (int64_t)d;
+    s.hb = *hb;
+    s.hb.n_units = (int32_t)n;
+    s.hb.T = hb->T + u0; s.hb.P = hb->P + u0; s.hb.B = hb->B + u0; s.hb.reserve = hb->reserve + u0;
+    s.hb.tok_off = s.tok.data();
+    s.hb.k_off = s.off.data();
+    s.hb.v_off = s.off.data();
+    s.hb.k = moved_bytes(hb->k, r0 * d * es);
+    s.hb.v = moved_bytes(hb->v, r0 * d * es);
+    s.hb.q = moved_bytes(hb->q, (size_t)u0 * rows * d * es);
+    s.hb.lse_in = moved(hb->lse_in, (size_t)u0 * rows);
+    s.hb.mass_in = moved(hb->mass_in, r0);
+    if (!ho) return;
+    const size_t Bm = (size_t)ho->Bmax;
+    s.ho = *ho;
+    s.ho.k_out = moved_bytes(ho->k_out, (size_t)u0 * Bm * d * es);
+    s.ho.v_out = moved_bytes(ho->v_out, (size_t)u0 * Bm * d * es);
+    s.ho.n_out = moved(ho->n_out, (size_t)u0);
+    s.ho.slot_src = moved(ho->slot_src, (size_t)u0 * Bm);
+    s.ho.slot_kind = moved(ho->slot_kind, (size_t)u0 * Bm);
+    s.ho.slot_mass = moved(ho->slot_mass, (size_t)u0 * Bm);
+    s.ho.assign = moved(ho->assign, r0);
+    s.ho.weight = moved(ho->weight, r0);
+    s.ho.kind = moved(ho->kind, r0);
+    s.ho.seed_of = moved(ho->seed_of, r0);
+    s.ho.plan = moved(ho->plan, (size_t)u0 * 8);
+    s.ho.unit_status = moved(ho->unit_status, (size_t)u0);
+    s.ho.lost_mass = moved(ho->lost_mass, (size_t)u0);
+    s.ho.s = moved(ho->s, r0);
+    s.ho.lse = moved(ho->lse, (size_t)u0 * rows);
+    s.ho.sim = moved(ho->sim, r0);
+    s.ho.rho_core = moved(ho->rho_core, (size_t)u0);
+    s.ho.rho_rep = moved(ho->rho_rep, (size_t)u0);
+    s.ho.dispersion = moved(ho->dispersion, (size_t)u0);
+}
+
+// Runs fn(u) for u in [0, n) on up to 16 host threads.
+template <typename F>
+void over_units(size_t n, F fn) {
+    const unsigned nthr = (unsigned)std::min<size_t>(n, std::max(1u, std::min(16u, std::thread::hardware_concurrency())));
+    if (nthr <= 1) {
+        for (size_t u = 0; u < n; ++u) fn(u);
+        return;
+    }
+    std::vector<std::thread> th;
+    for (unsigned t = 0; t < nthr; ++t)
+        th.emplace_back([&, t] {
+            for (size_t u = t; u < n; u += nthr) fn(u);
+        });
+    for (auto& x : th) x.join();
+}
+
+// Upload of a slice's keys, queries and per-row inputs.  Values do not go up here: only the compaction reads
+// them, and only the rows that are kept or merged, so they follow later, packed, once the rows' fates are known.
+cudaError_t slice_upload(HostSlice& s, cudaStream_t st) {
+    const cask_batch& hb = s.hb;
+    HostStage& h = s.h;
+    // the small arrays first: one of them in pageable memory then holds the host only until the stream's earlier
+    // work is done, not until the keys queued here have arrived
+    cudaError_t e = cudaMemcpyAsync(h.q, hb.q, h.q_bytes, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && hb.lse_in) e = cudaMemcpyAsync(h.lse_in, hb.lse_in, h.lse_bytes, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && hb.mass_in)
+        e = cudaMemcpyAsync(h.mass_in, hb.mass_in, (size_t)hb.tok_off[hb.n_units] * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && hb.chan_w)
+        e = cudaMemcpyAsync(h.chan_w, hb.chan_w, (size_t)hb.head_dim * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && hb.band_w)
+        e = cudaMemcpyAsync(h.band_w, hb.band_w, (size_t)(hb.head_dim / 2) * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h.k, hb.k, h.kv_bytes, cudaMemcpyHostToDevice, st);
+    return e;
+}
 }  // namespace
+
+extern "C" {
 
 size_t cask_host_event_device_bytes(const cask_batch* b, const cask_params* p, int32_t Bmax) {
     if (check_batch(b, p) != CASK_OK || b->n_units == 0 || Bmax < 1) return 0;
-    return stage_layout(nullptr, b, p, Bmax).bytes;
+    const std::vector<int> bounds = slice_bounds(b);
+    size_t bytes = 0;
+    for (size_t i = 0; i + 1 < bounds.size(); ++i) {
+        HostSlice s;
+        make_slice(s, b, nullptr, bounds[i], bounds[i + 1]);
+        bytes += stage_layout(nullptr, &s.hb, p, Bmax).bytes;
+    }
+    return bytes;
 }
 
 int cask_compress_event_host(cask_ctx* ctx, const cask_batch* hb, const cask_params* p,
@@ -663,133 +807,221 @@ int cask_compress_event_host(cask_ctx* ctx, const cask_batch* hb, const cask_par
     rc = check_host_layout(hb);
     if (rc != CASK_OK) return rc;
     if (ho->Bmax < 1) return CASK_ERR_SHAPE;
-    HostStage h = stage_layout(nullptr, hb, p, ho->Bmax);
-    if (!dev_buf || dev_bytes < h.bytes || (uintptr_t)dev_buf % 256) return CASK_ERR_WORKSPACE;
-    h = stage_layout((char*)dev_buf, hb, p, ho->Bmax);
-    // optional diagnostics are computed only when the caller has a place for them
-    if (!ho->rho_core) h.o.rho_core = nullptr;
-    if (!ho->rho_rep) h.o.rho_rep = nullptr;
-    if (!ho->dispersion) h.o.dispersion = nullptr;
+    if (!dev_buf || (uintptr_t)dev_buf % 256) return CASK_ERR_WORKSPACE;
+
+    const std::vector<int> bounds = slice_bounds(hb);
+    const size_t C = bounds.size() - 1;
+    if (C > kMaxSlices) return CASK_ERR_SHAPE;      // cannot happen: a slice holds a tenth of the batch or more
+    std::vector<HostSlice> sl(C);
+    size_t used = 0;
+    for (size_t i = 0; i < C; ++i) {
+        make_slice(sl[i], hb, ho, bounds[i], bounds[i + 1]);
+        const size_t need = stage_layout(nullptr, &sl[i].hb, p, ho->Bmax).bytes;
+        if (used + need > dev_bytes) return CASK_ERR_WORKSPACE;
+        sl[i].h = stage_layout((char*)dev_buf + used, &sl[i].hb, p, ho->Bmax);
+        used += need;
+        // optional diagnostics are computed only when the caller has a place for them
+        if (!ho->rho_core) sl[i].h.o.rho_core = nullptr;
+        if (!ho->rho_rep) sl[i].h.o.rho_rep = nullptr;
+        if (!ho->dispersion) sl[i].h.o.dispersion = nullptr;
+    }
     cudaError_t e = cudaSetDevice(ctx->device);
     if (e != cudaSuccess) return fail_cuda(ctx, e);
-    cudaStream_t st = ctx->stream;
-    // Keys and queries go up whole.  Values do not: only the compaction reads them, and only the rows that are
-    // kept or merged, so they follow later, packed, once the rows' fates are known.
-    e = cudaMemcpyAsync(h.k, hb->k, h.kv_bytes, cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(h.q, hb->q, h.q_bytes, cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess && hb->lse_in)
-        e = cudaMemcpyAsync(h.lse_in, hb->lse_in, h.lse_bytes, cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess && hb->mass_in)
-        e = cudaMemcpyAsync(h.mass_in, hb->mass_in, (size_t)hb->tok_off[hb->n_units] * 4, cudaMemcpyHostToDevice, st);
-    if (e != cudaSuccess) return fail_cuda(ctx, e);
-    cask_batch db = *hb;
-    db.mass_in = hb->mass_in ? (const float*)h.mass_in : nullptr;
-    if (hb->chan_w) {
-        e = cudaMemcpyAsync(h.chan_w, hb->chan_w, (size_t)hb->head_dim * 4, cudaMemcpyHostToDevice, st);
+
+    // One slice runs on the caller's stream.  Several take turns on streams of the context, which start after
+    // the work already queued on the caller's stream and are drained before the call returns.
+    cudaStream_t const user = ctx->stream;
+    const bool sliced = C > 1;
+    if (sliced) {
+        for (int j = 0; j < kSliceStreams && e == cudaSuccess; ++j)
+            if (!ctx->hs[j]) e = cudaStreamCreateWithFlags(&ctx->hs[j], cudaStreamNonBlocking);
+        if (e == cudaSuccess && !ctx->hs_start) e = cudaEventCreateWithFlags(&ctx->hs_start, cudaEventDisableTiming);
+        while (e == cudaSuccess && ctx->hs_kinds.size() < C) {
+            cudaEvent_t ev = nullptr;
+            e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+            if (e == cudaSuccess) ctx->hs_kinds.push_back(ev);
+        }
+        if (e == cudaSuccess) e = cudaEventRecord(ctx->hs_start, user);
+        for (int j = 0; j < kSliceStreams && e == cudaSuccess; ++j) e = cudaStreamWaitEvent(ctx->hs[j], ctx->hs_start, 0);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
     }
-    db.chan_w = hb->chan_w ? (const float*)h.chan_w : nullptr;
-    if (hb->band_w) {
-        e = cudaMemcpyAsync(h.band_w, hb->band_w, (size_t)(hb->head_dim / 2) * 4, cudaMemcpyHostToDevice, st);
-        if (e != cudaSuccess) return fail_cuda(ctx, e);
-    }
-    db.band_w = hb->band_w ? (const float*)h.band_w : nullptr;
-    db.k = h.k; db.v = h.v; db.q = h.q;
-    db.lse_in = hb->lse_in ? (const float*)h.lse_in : nullptr;
-    const size_t es = elem_size(hb->dtype), n = (size_t)hb->n_units, d = (size_t)hb->head_dim;
+    auto stream_of = [&](size_t i) { return sliced ? ctx->hs[i % kSliceStreams] : user; };
+    auto drain = [&]() {
+        cudaError_t first = cudaSuccess;
+        if (sliced)
+            for (int j = 0; j < kSliceStreams; ++j) {
+                const cudaError_t x = cudaStreamSynchronize(ctx->hs[j]);
+                if (first == cudaSuccess) first = x;
+            }
+        else
+            first = cudaStreamSynchronize(user);
+        return first;
+    };
+    // leaves with the context's stream restored and nothing of this call still in flight
+    auto leave = [&](int code, cudaError_t ce) {
+        ctx->stream = user;
+        const cudaError_t de = drain();
+        if (code == CASK_OK && ce == cudaSuccess && de != cudaSuccess) ce = de;
+        if (ce != cudaSuccess) return fail_cuda(ctx, ce);
+        return code;
+    };
+
+    const size_t es = elem_size(hb->dtype), d = (size_t)hb->head_dim, row_bytes = d * es;
     const size_t sumT = (size_t)hb->tok_off[hb->n_units], rows = (size_t)hb->group * hb->window;
     const size_t Bm = (size_t)ho->Bmax;
-    {
-        Launch L{};
-        Workspace W{};
-        rc = prepare(ctx, &db, p, h.ws, h.ws_bytes, L, W);
-        if (rc != CASK_OK) return rc;
-        rc = event_decide(ctx, L, W, &db, p, &h.o);
-        if (rc != CASK_OK) return rc;
-        e = launch_value_ranks(L, h.o.kind, h.v_pos, h.n_need, h.v_base);
-        if (e != cudaSuccess) return fail_cuda(ctx, e);
-        // the row kinds come back; the rows with a kind other than 0 are the ones whose values are read
-        const size_t row_bytes = d * es;
-        if (ctx->hstage_bytes < sumT) {
-            if (ctx->hstage) cudaFreeHost(ctx->hstage);
-            ctx->hstage = nullptr;
-            ctx->hstage_bytes = 0;
-            e = cudaMallocHost((void**)&ctx->hstage, sumT + (sumT / 8 + 4096) * row_bytes);
-            if (e != cudaSuccess) return fail_cuda(ctx, e);
-            ctx->hstage_bytes = sumT + (sumT / 8 + 4096) * row_bytes;
-        }
-        uint8_t* hkind = (uint8_t*)ctx->hstage;
-        e = cudaMemcpyAsync(hkind, h.o.kind, sumT, cudaMemcpyDeviceToHost, st);
-        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-        if (e != cudaSuccess) return fail_cuda(ctx, e);
-        std::vector<int64_t> vbase(n + 1, 0);
-        const unsigned nthr = std::max(1u, std::min(16u, std::thread::hardware_concurrency()));
-        auto over_units = [&](auto fn) {
-            std::vector<std::thread> th;
-            for (unsigned t = 0; t < nthr; ++t)
-                th.emplace_back([&, t] {
-                    for (size_t u = t; u < n; u += nthr) fn(u);
-                });
-            for (auto& x : th) x.join();
-        };
-        over_units([&](size_t u) {
-            const uint8_t* kd = hkind + hb->tok_off[u];
+    if (ctx->hstage_bytes < sumT + 4096 * row_bytes) {
+        if (ctx->hstage) cudaFreeHost(ctx->hstage);
+        ctx->hstage = nullptr;
+        ctx->hstage_bytes = 0;
+        const size_t nb = sumT + (sumT / 8 + 4096) * row_bytes;
+        e = cudaMallocHost((void**)&ctx->hstage, nb);
+        if (e != cudaSuccess) return leave(CASK_OK, e);
+        ctx->hstage_bytes = nb;
+    }
+
+    // keys up, the rows' fates decided, the row kinds on their way back
+    auto decide = [&](size_t i) -> int {
+        HostSlice& s = sl[i];
+        cudaStream_t st = stream_of(i);
+        cask_batch db = s.hb;
+        db.k = s.h.k; db.v = s.h.v; db.q = s.h.q;
+        db.lse_in = s.hb.lse_in ? (const float*)s.h.lse_in : nullptr;
+        db.mass_in = s.hb.mass_in ? (const float*)s.h.mass_in : nullptr;
+        db.chan_w = s.hb.chan_w ? (const float*)s.h.chan_w : nullptr;
+        db.band_w = s.hb.band_w ? (const float*)s.h.band_w : nullptr;
+        ctx->stream = st;
+        int r = prepare(ctx, &db, p, s.h.ws, s.h.ws_bytes, s.L, s.W);
+        ctx->stream = user;
+        if (r != CASK_OK) return r;
+        r = event_decide(ctx, s.L, s.W, &db, p, &s.h.o);
+        if (r != CASK_OK) return r;
+        cudaError_t ce = launch_value_ranks(s.L, s.h.o.kind, s.h.v_pos, s.h.n_need, s.h.v_base);
+        // the rows with a kind other than 0 are the ones whose values are read
+        if (ce == cudaSuccess)
+            ce = cudaMemcpyAsync(ctx->hstage + s.r0, s.h.o.kind, (size_t)s.tok.back(), cudaMemcpyDeviceToHost, st);
+        if (ce == cudaSuccess && sliced) ce = cudaEventRecord(ctx->hs_kinds[i], st);
+        return ce == cudaSuccess ? CASK_OK : fail_cuda(ctx, ce);
+    };
+
+    size_t v_rows_used = 0;
+    // the needed value rows packed and sent up, the compaction
+    auto compact = [&](size_t i) -> int {
+        HostSlice& s = sl[i];
+        cudaStream_t st = stream_of(i);
+        cudaError_t ce = sliced ? cudaEventSynchronize(ctx->hs_kinds[i]) : cudaStreamSynchronize(st);
+        if (ce != cudaSuccess) return fail_cuda(ctx, ce);
+        const size_t n = (size_t)s.hb.n_units;
+        const uint8_t* hkind = (const uint8_t*)ctx->hstage + s.r0;
+        s.vbase.assign(n + 1, 0);
+        over_units(n, [&](size_t u) {
+            const uint8_t* kd = hkind + s.tok[u];
             int64_t c = 0;
-            for (int i = 0; i < hb->T[u]; ++i) c += kd[i] != CASK_KIND_DROPPED;
-            vbase[u + 1] = c;
+            for (int r = 0; r < s.hb.T[u]; ++r) c += kd[r] != CASK_KIND_DROPPED;
+            s.vbase[u + 1] = c;
         });
-        for (size_t u = 0; u < n; ++u) vbase[u + 1] += vbase[u];
-        const size_t need_rows = (size_t)vbase[n];
-        if (ctx->hstage_bytes < sumT + need_rows * row_bytes) {      // grow, keeping the kinds
+        for (size_t u = 0; u < n; ++u) s.vbase[u + 1] += s.vbase[u];
+        s.need_rows = (size_t)s.vbase[n];
+        s.v_row0 = v_rows_used;
+        if (ctx->hstage_bytes < sumT + (v_rows_used + s.need_rows) * row_bytes) {
+            // Grow, keeping the kinds.  Earlier slices may still be reading their packed rows: wait for them first.
+            ce = drain();
+            if (ce != cudaSuccess) return fail_cuda(ctx, ce);
             char* bigger = nullptr;
-            const size_t nb = sumT + (need_rows + need_rows / 4 + 4096) * row_bytes;
-            e = cudaMallocHost((void**)&bigger, nb);
-            if (e != cudaSuccess) return fail_cuda(ctx, e);
+            const size_t want = v_rows_used + s.need_rows;
+            const size_t nb = sumT + (want + want / 4 + 4096) * row_bytes;
+            ce = cudaMallocHost((void**)&bigger, nb);
+            if (ce != cudaSuccess) return fail_cuda(ctx, ce);
             memcpy(bigger, ctx->hstage, sumT);
             cudaFreeHost(ctx->hstage);
             ctx->hstage = bigger;
             ctx->hstage_bytes = nb;
-            hkind = (uint8_t*)ctx->hstage;
+            hkind = (const uint8_t*)ctx->hstage + s.r0;
         }
-        char* hv = ctx->hstage + sumT;
-        over_units([&](size_t u) {
-            const uint8_t* kd = hkind + hb->tok_off[u];
-            const char* src = (const char*)hb->v + (size_t)hb->v_off[u] * es;
-            char* dst = hv + (size_t)vbase[u] * row_bytes;
-            for (int i = 0; i < hb->T[u]; ++i)
-                if (kd[i] != CASK_KIND_DROPPED) {
-                    memcpy(dst, src + (size_t)i * row_bytes, row_bytes);
+        v_rows_used += s.need_rows;
+        char* hv = ctx->hstage + sumT + s.v_row0 * row_bytes;
+        over_units(n, [&](size_t u) {
+            const uint8_t* kd = hkind + s.tok[u];
+            const char* src = (const char*)s.hb.v + (size_t)s.off[u] * es;
+            char* dst = hv + (size_t)s.vbase[u] * row_bytes;
+            for (int r = 0; r < s.hb.T[u]; ++r)
+                if (kd[r] != CASK_KIND_DROPPED) {
+                    memcpy(dst, src + (size_t)r * row_bytes, row_bytes);
                     dst += row_bytes;
                 }
         });
-        e = cudaMemcpyAsync(h.v, hv, need_rows * row_bytes, cudaMemcpyHostToDevice, st);
-        if (e != cudaSuccess) return fail_cuda(ctx, e);
-        L.v = h.v;
-        L.sh.v_pos = h.v_pos;
-        L.sh.v_base = h.v_base;
-        rc = event_compact(ctx, L, W, p, &h.o);
-        if (rc != CASK_OK) return rc;
-    }
-    struct Cp { void* dst; const void* src; size_t bytes; };
-    const Cp cps[] = {
-        {ho->k_out, h.o.k_out, n * Bm * d * es}, {ho->v_out, h.o.v_out, n * Bm * d * es},
-        {ho->n_out, h.o.n_out, n * 4}, {ho->slot_src, h.o.slot_src, n * Bm * 4},
-        {ho->slot_kind, h.o.slot_kind, n * Bm}, {ho->slot_mass, h.o.slot_mass, n * Bm * 4},
-        {ho->assign, h.o.assign, sumT * 4}, {ho->weight, h.o.weight, sumT * 4},
-        {ho->kind, h.o.kind, sumT}, {ho->seed_of, h.o.seed_of, sumT * 4},
-        {ho->plan, h.o.plan, n * 32}, {ho->unit_status, h.o.unit_status, n * 4},
-        {ho->lost_mass, h.o.lost_mass, n * 4}, {ho->s, h.o.s, sumT * 4},
-        {ho->lse, h.o.lse, n * rows * 4}, {ho->sim, h.o.sim, sumT * 4},
-        {ho->rho_core, h.o.rho_core, n * 4}, {ho->rho_rep, h.o.rho_rep, n * 4},
-        {ho->dispersion, h.o.dispersion, n * 4},
+        ce = cudaMemcpyAsync(s.h.v, hv, s.need_rows * row_bytes, cudaMemcpyHostToDevice, st);
+        if (ce != cudaSuccess) return fail_cuda(ctx, ce);
+        s.L.v = s.h.v;
+        s.L.sh.v_pos = s.h.v_pos;
+        s.L.sh.v_base = s.h.v_base;
+        return event_compact(ctx, s.L, s.W, p, &s.h.o);
     };
-    for (const Cp& c : cps) {
-        if (!c.dst) continue;
-        e = cudaMemcpyAsync(c.dst, c.src, c.bytes, cudaMemcpyDeviceToHost, st);
-        if (e != cudaSuccess) return fail_cuda(ctx, e);
+    auto results = [&](size_t i) -> int {
+        HostSlice& s = sl[i];
+        cudaStream_t st = stream_of(i);
+        cudaError_t ce = cudaSuccess;
+        const size_t n = (size_t)s.hb.n_units, sT = (size_t)s.tok.back();
+        struct Cp { void* dst; const void* src; size_t bytes; };
+        const cask_outputs &o = s.ho, &g = s.h.o;
+        const Cp cps[] = {
+            {o.k_out, g.k_out, n * Bm * d * es}, {o.v_out, g.v_out, n * Bm * d * es},
+            {o.n_out, g.n_out, n * 4}, {o.slot_src, g.slot_src, n * Bm * 4},
+            {o.slot_kind, g.slot_kind, n * Bm}, {o.slot_mass, g.slot_mass, n * Bm * 4},
+            {o.assign, g.assign, sT * 4}, {o.weight, g.weight, sT * 4},
+            {o.kind, g.kind, sT}, {o.seed_of, g.seed_of, sT * 4},
+            {o.plan, g.plan, n * 32}, {o.unit_status, g.unit_status, n * 4},
+            {o.lost_mass, g.lost_mass, n * 4}, {o.s, g.s, sT * 4},
+            {o.lse, g.lse, n * rows * 4}, {o.sim, g.sim, sT * 4},
+            {o.rho_core, g.rho_core, n * 4}, {o.rho_rep, g.rho_rep, n * 4},
+            {o.dispersion, g.dispersion, n * 4},
+        };
+        for (const Cp& c : cps) {
+            if (!c.dst) continue;
+            ce = cudaMemcpyAsync(c.dst, c.src, c.bytes, cudaMemcpyDeviceToHost, st);
+            if (ce != cudaSuccess) return fail_cuda(ctx, ce);
+        }
+        // the slice's flag word joins the call's
+        ce = cudaMemcpyAsync(&ctx->hs_flags[i], s.W.err, sizeof(int32_t), cudaMemcpyDeviceToHost, st);
+        return ce == cudaSuccess ? CASK_OK : fail_cuda(ctx, ce);
+    };
+
+    // Order of the host's work for slice i: pack and compact it, decide slice i+1, queue slice i+2's upload, then
+    // queue slice i's results.  The descriptor staging of the context serves one slice at a time, so slice i+1 is
+    // decided only after slice i's compaction has been queued; the results come last because a copy into pageable
+    // memory holds the host until the slice is done, and by then the next upload and decision are already queued.
+    if (!ctx->hs_flags) {
+        e = cudaMallocHost((void**)&ctx->hs_flags, kMaxSlices * sizeof(int32_t));
+        if (e != cudaSuccess) return leave(CASK_OK, e);
     }
-    e = cudaStreamSynchronize(st);
-    return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
+    e = slice_upload(sl[0], stream_of(0));
+    if (e != cudaSuccess) return leave(CASK_OK, e);
+    rc = decide(0);
+    if (rc != CASK_OK) return leave(rc, cudaSuccess);
+    if (C > 1) {
+        e = slice_upload(sl[1], stream_of(1));
+        if (e != cudaSuccess) return leave(CASK_OK, e);
+    }
+    for (size_t i = 0; i < C; ++i) {
+        rc = compact(i);
+        if (rc != CASK_OK) return leave(rc, cudaSuccess);
+        if (i + 1 < C) {
+            rc = decide(i + 1);
+            if (rc != CASK_OK) return leave(rc, cudaSuccess);
+        }
+        if (i + 2 < C) {
+            e = slice_upload(sl[i + 2], stream_of(i + 2));
+            if (e != cudaSuccess) return leave(CASK_OK, e);
+        }
+        rc = results(i);
+        if (rc != CASK_OK) return leave(rc, cudaSuccess);
+    }
+    rc = leave(CASK_OK, cudaSuccess);
+    if (rc != CASK_OK) return rc;
+    int32_t flags = 0;
+    for (size_t i = 0; i < C; ++i) flags |= ctx->hs_flags[i];
+    ctx->flags_dev = nullptr;
+    ctx->flags_last = flags;
+    return CASK_OK;
 }
 
 }  // extern "C"

@@ -248,7 +248,7 @@ def make_batch(wl: Workload, units: Optional[List[Tuple[int, int, int]]] = None,
                threads: int = 8, pinned_alloc=None) -> Batch:
     """Generate the listed units (default: all) into one contiguous host batch.
 
-    ``pinned_alloc(shape, np_dtype) -> np.ndarray`` lets a caller place K/V in
+    ``pinned_alloc(shape, np_dtype) -> np.ndarray`` lets a caller place the arrays in
     page-locked memory; the default is ordinary numpy memory.
     """
     units = unit_list(wl) if units is None else units
@@ -260,8 +260,10 @@ def make_batch(wl: Workload, units: Optional[List[Tuple[int, int, int]]] = None,
     alloc = pinned_alloc if pinned_alloc is not None else (lambda shape, dt: np.empty(shape, dtype=dt))
     k = alloc((int(tok_off[-1]), wl.head_dim), st)
     v = alloc((int(tok_off[-1]), wl.head_dim), st)
-    q = np.empty((n, wl.group, wl.window, wl.head_dim), dtype=st)
-    mass = np.zeros(int(tok_off[-1]), dtype=np.float32) if wl.carried_rows > 0 else None
+    q = alloc((n, wl.group, wl.window, wl.head_dim), st)
+    mass = alloc((int(tok_off[-1]),), np.float32) if wl.carried_rows > 0 else None
+    if mass is not None:
+        mass[...] = 0.0
 
     def work(u: int) -> None:
         s, l, h = units[u]

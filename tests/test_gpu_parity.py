@@ -582,3 +582,53 @@ def test_host_buffer_entry_point_matches_device_entry_point(extras):
     for k in g:
         got = wl.bf16_bits_to_f32(ho[k]) if ho[k].dtype == np.uint16 else ho[k]
         assert np.array_equal(got, g[k]), k
+
+
+def test_host_buffer_entry_point_in_slices():
+    """A host batch of 60 MB of keys goes through the device in several slices of units (each with its own staging
+    and workspace, uploads overlapping the slice before); 44 ragged units with odd lengths, carried masses and
+    channel weights, every one against the oracle.  Against the device entry point on the whole batch only the
+    last bits of the scores may differ (a unit's tiles are shared out between the CTAs differently)."""
+    import gpu_harness as gh
+    import torch
+    rng = np.random.default_rng(11)
+    base = wl.WORKLOADS["tiny"].with_(dtype=wl.DTYPE_BF16, head_dim=128, group=2, window=16, cluster_frac=0.6,
+                                      n_centres=0)
+    ks, vs, qs, T, P, B, R = [], [], [], [], [], [], []
+    for i in range(44):
+        t = int(rng.integers(4000, 7001))
+        p = int(rng.integers(0, 600))
+        b = int(rng.integers(64, 385))
+        r = int(rng.integers(0, b + 1))
+        w = base.with_(prefix=p, decode=t - p, budget=b, reserve=r)
+        k, v, q = wl.make_unit(w, i, 5, 0)
+        ks.append(k); vs.append(v); qs.append(q[None])
+        T.append(t); P.append(p); B.append(b); R.append(r)
+    hb = wl.Batch(wl=base, k=np.concatenate(ks), v=np.concatenate(vs), q=np.concatenate(qs),
+                  T=np.array(T, np.int32), P=np.array(P, np.int32), B=np.array(B, np.int32),
+                  reserve=np.array(R, np.int32), tok_off=np.concatenate([[0], np.cumsum(T)]).astype(np.int64),
+                  unit_ids=[(i, 0, 0) for i in range(len(T))])
+    sumT = int(hb.tok_off[-1])
+    assert sumT * 256 > 3 * (16 << 20)           # enough keys for three slices or more
+    mass = np.where(rng.random(sumT) < 0.3, rng.random(sumT) * 1e-3, 0.0).astype(np.float32)
+    cw = (rng.random(128) + 0.05).astype(np.float32)
+    run = gh.GpuRun(hb, mass_in=mass, chan_w=cw)
+    whole = run.event()
+    cb = run.cb
+    hbatch, keep = cb.make_batch(hb.k, hb.v, hb.q, hb.T, hb.P, hb.B, hb.reserve, hb.tok_off, 128, 2, 16,
+                                 wl.DTYPE_BF16, mass_in=mass, chan_w=cw)
+    nbytes = cb.cask_host_event_device_bytes(hbatch, run.prm, run.Bmax)
+    assert nbytes > 0
+    dev = torch.empty(nbytes, dtype=torch.uint8, device="cuda:0")
+    ho = {k: (np.zeros(tuple(t.shape), np.uint16) if t.dtype == torch.bfloat16 else np.zeros(tuple(t.shape), t.cpu().numpy().dtype))
+          for k, t in run.out.items()}
+    assert cb.cask_compress_event_host(run.ctx, hbatch, run.prm, cb.make_outputs(ho, run.Bmax), dev, nbytes - 256,
+                                       check=False) == cb.ERR_WORKSPACE
+    cb.cask_compress_event_host(run.ctx, hbatch, run.prm, cb.make_outputs(ho, run.Bmax), dev, nbytes)
+    assert run.ctx.device_flags() == 0
+    g = {k: (wl.bf16_bits_to_f32(a) if a.dtype == np.uint16 else a) for k, a in ho.items()}
+    o = gh.run_oracle(hb, mass_in=mass, chan_w=cw)
+    st = gh.compare_event(hb, g, o, geom=dict(mass_in=mass, chan_w=cw))
+    assert st["units"] == 44
+    assert np.allclose(g["s"], whole["s"], rtol=1e-5, atol=1e-12)
+    assert np.array_equal(g["plan"], whole["plan"]) and np.array_equal(g["unit_status"], whole["unit_status"])
