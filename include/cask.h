@@ -331,10 +331,11 @@ int cask_writeback_paged(cask_ctx* ctx, const cask_batch* batch, const cask_para
  * and returns when everything has arrived.
  *
  * A batch with more than 16 MB of keys is cut into up to about ten slices of
- * consecutive units, each a batch of its own inside dev_buf; they take turns
- * on streams the context owns (ordered after the work already queued on the
- * context's stream), so that one slice's upload runs while the slice before it
- * is decided, packed, compacted and read back.  For that overlap every HOST
+ * consecutive units, each a batch of its own inside dev_buf, on streams the
+ * context owns (ordered after the work already queued on the context's
+ * stream: one for every copy to the device, four the slices take turns on),
+ * so that one slice's upload runs while the slice before it is decided,
+ * packed, compacted and read back.  For that overlap every HOST
  * array, inputs and outputs, has to be page-locked: a copy to or from pageable
  * memory holds the calling thread until the copy is done.  Units are
  * independent, so the results are those of cask_compress_event on the same
