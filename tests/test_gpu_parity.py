@@ -584,11 +584,14 @@ def test_host_buffer_entry_point_matches_device_entry_point(extras):
         assert np.array_equal(got, g[k]), k
 
 
-def test_host_buffer_entry_point_in_slices():
+@pytest.mark.parametrize("budgets", ["small", "near_full"])
+def test_host_buffer_entry_point_in_slices(budgets):
     """A host batch of 60 MB of keys goes through the device in several slices of units (each with its own staging
     and workspace, uploads overlapping the slice before); 44 ragged units with odd lengths, carried masses and
     channel weights, every one against the oracle.  Against the device entry point on the whole batch only the
-    last bits of the scores may differ (a unit's tiles are shared out between the CTAs differently)."""
+    last bits of the scores may differ (a unit's tiles are shared out between the CTAs differently).
+    "near_full": budgets a few hundred rows short of the cache, so nearly every value row is needed and the pinned
+    staging of the context has to grow while earlier slices are in flight."""
     import gpu_harness as gh
     import torch
     rng = np.random.default_rng(11)
@@ -598,8 +601,8 @@ def test_host_buffer_entry_point_in_slices():
     for i in range(44):
         t = int(rng.integers(4000, 7001))
         p = int(rng.integers(0, 600))
-        b = int(rng.integers(64, 385))
-        r = int(rng.integers(0, b + 1))
+        b = int(rng.integers(64, 385)) if budgets == "small" else t - int(rng.integers(50, 400))
+        r = int(rng.integers(0, b + 1)) if budgets == "small" else b // 2
         w = base.with_(prefix=p, decode=t - p, budget=b, reserve=r)
         k, v, q = wl.make_unit(w, i, 5, 0)
         ks.append(k); vs.append(v); qs.append(q[None])
