@@ -7,21 +7,27 @@
 // as a 0.64 fraction times the integer part of Delta wraps around by itself, so a distance of tens of thousands of
 // rows costs no accuracy and no double-precision arithmetic in the inner loop; the fractional part of Delta is added
 // in single precision.
-#include "cask_internal.cuh"
+#include "tc_common.cuh"
 
 namespace cask {
 
 namespace {
 
+using tc::pack2;
+using tc::unpack2;
+using tc::fma2;
+
 constexpr double kTwoPi = 6.283185307179586476925286766559;
 constexpr int kRowsPerCta = 64;
 
 // Per-band constants shared by all units (global memory, read through the L1): omega / 2 pi in turns and in 0.64 fixed
-// point, and e^{i omega} for the row-to-row phase step.
+// point, e^{i omega} for the row-to-row phase step and e^{i 64 omega} for the step from a tile to the next.
 struct BandTable {
     float* om_t;
     float* rot_c;
     float* rot_s;
+    float* r64_c;
+    float* r64_s;
     unsigned long long* om_fx;
 };
 
@@ -41,6 +47,10 @@ __global__ void __launch_bounds__(256) stats_fold_kernel(int g, int nb, cask_que
             sincosf((float)(kTwoPi * (fr > 0.5 ? fr - 1.0 : fr)), &sn, &cs);
             tab.rot_c[f] = cs;
             tab.rot_s[f] = sn;
+            const double t64 = fr * (double)kRowsPerCta, f64 = t64 - floor(t64);
+            sincosf((float)(kTwoPi * (f64 > 0.5 ? f64 - 1.0 : f64)), &sn, &cs);
+            tab.r64_c[f] = cs;
+            tab.r64_s[f] = sn;
         }
     for (int f0 = 0; f0 < nb; f0 += 64) {
         const int f = f0 + (threadIdx.x >> 2);
@@ -117,6 +127,51 @@ template <> struct Quad<float> {
     }
 };
 
+// The real parts (kx) and imaginary parts (ky) of a quad of bands as two packed pairs each, straight from shared
+// memory: a bf16 pair becomes a packed fp32 pair by one shift and one mask into the two halves of a 64-bit register.
+__device__ __forceinline__ uint64_t widen_pair(unsigned w) {            // (lo, hi) halves of w as two floats
+    uint64_t r;
+    asm("{\n\t.reg .b32 lo, hi;\n\tshl.b32 lo, %1, 16;\n\tand.b32 hi, %1, 0xffff0000;\n\tmov.b64 %0, {lo, hi};\n\t}" : "=l"(r) : "r"(w));
+    return r;
+}
+__device__ __forceinline__ uint64_t widen_lows(unsigned w0, unsigned w1) {      // low halves of w0 and w1
+    uint64_t r;
+    asm("{\n\t.reg .b32 a, b;\n\tshl.b32 a, %1, 16;\n\tshl.b32 b, %2, 16;\n\tmov.b64 %0, {a, b};\n\t}" : "=l"(r) : "r"(w0), "r"(w1));
+    return r;
+}
+__device__ __forceinline__ uint64_t widen_highs(unsigned w0, unsigned w1) {     // high halves of w0 and w1
+    uint64_t r;
+    asm("{\n\t.reg .b32 a, b;\n\tand.b32 a, %1, 0xffff0000;\n\tand.b32 b, %2, 0xffff0000;\n\tmov.b64 %0, {a, b};\n\t}" : "=l"(r) : "r"(w0), "r"(w1));
+    return r;
+}
+template <typename T, int LAYOUT> struct QuadPairs;
+template <int LAYOUT> struct QuadPairs<__nv_bfloat16, LAYOUT> {
+    static __device__ __forceinline__ void ld(const __nv_bfloat16* row, int nb, int q, uint64_t (&kx)[2], uint64_t (&ky)[2]) {
+        if (LAYOUT == 0) {
+            const uint2 x = *reinterpret_cast<const uint2*>(row + 4 * q), y = *reinterpret_cast<const uint2*>(row + nb + 4 * q);
+            kx[0] = widen_pair(x.x); kx[1] = widen_pair(x.y);
+            ky[0] = widen_pair(y.x); ky[1] = widen_pair(y.y);
+        } else {
+            const uint4 v = *reinterpret_cast<const uint4*>(row + 8 * q);      // (x0 y0)(x1 y1)(x2 y2)(x3 y3)
+            kx[0] = widen_lows(v.x, v.y); kx[1] = widen_lows(v.z, v.w);
+            ky[0] = widen_highs(v.x, v.y); ky[1] = widen_highs(v.z, v.w);
+        }
+    }
+};
+template <int LAYOUT> struct QuadPairs<float, LAYOUT> {
+    static __device__ __forceinline__ void ld(const float* row, int nb, int q, uint64_t (&kx)[2], uint64_t (&ky)[2]) {
+        if (LAYOUT == 0) {
+            const float4 x = *reinterpret_cast<const float4*>(row + 4 * q), y = *reinterpret_cast<const float4*>(row + nb + 4 * q);
+            kx[0] = pack2(x.x, x.y); kx[1] = pack2(x.z, x.w);
+            ky[0] = pack2(y.x, y.y); ky[1] = pack2(y.z, y.w);
+        } else {
+            const float4 a = *reinterpret_cast<const float4*>(row + 8 * q), b = *reinterpret_cast<const float4*>(row + 8 * q + 4);
+            kx[0] = pack2(a.x, a.z); kx[1] = pack2(b.x, b.z);
+            ky[0] = pack2(a.y, a.w); ky[1] = pack2(b.y, b.w);
+        }
+    }
+};
+
 template <typename T, bool STEP, int LAYOUT>      // STEP: no caller-supplied offsets, Delta falls by one per row
 __global__ void __launch_bounds__(256) score_stats_kernel(const UnitDesc* __restrict__ desc, Shape sh, const T* __restrict__ K,
                                                              cask_query_stats qs, const float* __restrict__ A, BandTable tab,
@@ -184,6 +239,103 @@ __global__ void __launch_bounds__(256) score_stats_kernel(const UnitDesc* __rest
     const bool one_quad = nq <= 16;          // head_dim <= 128: a thread has at most one quad, its constants load once
     QuadConst c0 = {};
     if (one_quad && q < nq) load_const(q, c0);
+    if constexpr (STEP) {
+        if (one_quad) {
+            // Delta falls by one per row and by 64 per tile, so the whole factor G = A e^{i omega Delta} of each of the
+            // thread's sixteen (row, band) pairs lives in registers: formed once per CTA (one sine and cosine per
+            // band for the first row, the other rows by turning it by e^{-i omega}), turned by e^{-i 64 omega} from
+            // tile to tile, and a row's score is sum_f Gr kx + Gi ky.  Two bands per instruction (packed fp32).
+            const bool active = q < nq;
+            uint64_t Gr[4][2], Gi[4][2], Rc[2], Rs[2], Rn[2];
+            {
+                float gr[4][4], gi[4][4];
+#pragma unroll
+                for (int b4 = 0; b4 < 4; ++b4) {
+                    const int Di = T_u - 1 - (first_row + r_first);       // negative only for rows past the end, never stored
+                    const unsigned dm = (unsigned)abs(Di);
+                    const int hi = (int)(c0.fx_hi[b4] * dm + __umulhi(c0.fx_lo[b4], dm));
+                    float sn, cs;
+                    __sincosf(6.2831853071795865f * ((float)hi * (Di < 0 ? -2.3283064365386963e-10f : 2.3283064365386963e-10f)), &sn, &cs);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (j > 0) {
+                            const float c2 = fmaf(cs, c0.rc[b4], sn * c0.rs[b4]);      // (c + i s) e^{-i omega}
+                            sn = fmaf(sn, c0.rc[b4], -cs * c0.rs[b4]);
+                            cs = c2;
+                        }
+                        gr[j][b4] = fmaf(c0.ar[b4], cs, -c0.ai[b4] * sn);              // A e^{i theta}
+                        gi[j][b4] = fmaf(c0.ar[b4], sn, c0.ai[b4] * cs);
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+#pragma unroll
+                    for (int pp = 0; pp < 2; ++pp) {
+                        Gr[j][pp] = pack2(gr[j][2 * pp], gr[j][2 * pp + 1]);
+                        Gi[j][pp] = pack2(gi[j][2 * pp], gi[j][2 * pp + 1]);
+                    }
+                float4 c64 = make_float4(1.f, 1.f, 1.f, 1.f), s64 = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (active) {
+                    c64 = *reinterpret_cast<const float4*>(tab.r64_c + 4 * q);
+                    s64 = *reinterpret_cast<const float4*>(tab.r64_s + 4 * q);
+                }
+                Rc[0] = pack2(c64.x, c64.y); Rc[1] = pack2(c64.z, c64.w);
+                Rs[0] = pack2(s64.x, s64.y); Rs[1] = pack2(s64.z, s64.w);
+                Rn[0] = pack2(-s64.x, -s64.y); Rn[1] = pack2(-s64.z, -s64.w);
+            }
+            const uint64_t zero2 = pack2(0.f, 0.f);
+            for (int k = 0; k < n_tiles; ++k) {
+                issue(k + n_stages - 1);
+                if (n_stages == 3) asm volatile("cp.async.wait_group 2;" ::: "memory");
+                else if (n_stages == 2) asm volatile("cp.async.wait_group 1;" ::: "memory");
+                else asm volatile("cp.async.wait_group 0;" ::: "memory");
+                __syncthreads();
+                const int row0 = first_row + k * kRowsPerCta, nrows = min(kRowsPerCta, T_u - row0);
+                const T* tile = stages + (size_t)(k % n_stages) * stage_elems;
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                if (active) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        // rows past the end of the unit repeat the last one (their sums are not stored)
+                        const T* row = tile + (size_t)(nrows == kRowsPerCta ? r_first + j : min(r_first + j, nrows - 1)) * d;
+                        uint64_t kx[2], ky[2];
+                        QuadPairs<T, LAYOUT>::ld(row, nb, q, kx, ky);
+                        uint64_t a2 = zero2;
+#pragma unroll
+                        for (int pp = 0; pp < 2; ++pp) {
+                            a2 = fma2(Gr[j][pp], kx[pp], a2);
+                            a2 = fma2(Gi[j][pp], ky[pp], a2);
+                            // on to the next tile: G e^{-i 64 omega} = (Gr c + Gi s) + i (Gi c - Gr s)
+                            const uint64_t nr = fma2(Gr[j][pp], Rc[pp], fma2(Gi[j][pp], Rs[pp], zero2));
+                            Gi[j][pp] = fma2(Gi[j][pp], Rc[pp], fma2(Gr[j][pp], Rn[pp], zero2));
+                            Gr[j][pp] = nr;
+                        }
+                        float lo, hi2;
+                        unpack2(a2, lo, hi2);
+                        acc[j] = lo + hi2;
+                    }
+                }
+                // The four row sums meet over the sixteen lanes of a row group: the first two exchanges halve what a
+                // lane carries (a lane keeps the rows whose index bit matches its own), the last two add the rest;
+                // lane l of the group ends with the whole sum of row r_first + (l & 3) in its bit-reversed order.
+                {
+                    const bool up1 = (q & 1) != 0;
+                    const float give0 = up1 ? acc[0] : acc[1], give1 = up1 ? acc[2] : acc[3];
+                    const float keep0 = up1 ? acc[1] : acc[0], keep1 = up1 ? acc[3] : acc[2];
+                    const float h0 = keep0 + __shfl_xor_sync(0xffffffffu, give0, 1);       // rows (0|1), (2|3) by bit 0
+                    const float h1 = keep1 + __shfl_xor_sync(0xffffffffu, give1, 1);
+                    const bool up2 = (q & 2) != 0;
+                    float t = (up2 ? h1 : h0) + __shfl_xor_sync(0xffffffffu, up2 ? h0 : h1, 2);
+                    t += __shfl_xor_sync(0xffffffffu, t, 4);
+                    t += __shfl_xor_sync(0xffffffffu, t, 8);
+                    const int jr = (q & 1) + 2 * ((q >> 1) & 1);                          // the row this lane holds
+                    if (q < 4 && r_first + jr < nrows) s[tok_u + row0 + r_first + jr] = t;
+                }
+                __syncthreads();        // the stage is free for the tile issued at the top of the next round
+            }
+            return;
+        }
+    }
     for (int k = 0; k < n_tiles; ++k) {
         issue(k + n_stages - 1);
         // all but the newest n_stages - 1 groups have landed: tile k is in shared memory
@@ -269,7 +421,8 @@ cudaError_t launch_score_stats(const Launch& L, const cask_query_stats& qs, floa
     const int nb = sh.d / 2;
     // the table of per-band constants sits behind the per-unit coefficients in the same workspace array
     float* tbase = ws.stats_a + (size_t)sh.n_units * sh.d;
-    BandTable tab{tbase, tbase + nb, tbase + 2 * nb, reinterpret_cast<unsigned long long*>(tbase + 4 * nb)};
+    BandTable tab{tbase, tbase + nb, tbase + 2 * nb, tbase + 3 * nb, tbase + 6 * nb,
+                  reinterpret_cast<unsigned long long*>(tbase + 4 * nb)};
     {
         Timed t(L, KID_ROW_COMBINE);
         stats_fold_kernel<<<sh.n_units, 256, 0, L.stream>>>(sh.g, nb, qs, ws.stats_a, tab);
