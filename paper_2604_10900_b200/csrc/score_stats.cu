@@ -212,8 +212,6 @@ __global__ void __launch_bounds__(256) score_stats_kernel(const UnitDesc* __rest
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    for (int k = 0; k < n_stages - 1; ++k) issue(k);
-
     const int q = threadIdx.x & 15, rg = threadIdx.x >> 4;       // band quad (and its multiples of 16), row group
     const int r_first = 4 * rg;
     // constants of a quad: coefficient A, omega in turns (float and the two halves of the 0.64 fixed-point value),
@@ -284,12 +282,52 @@ __global__ void __launch_bounds__(256) score_stats_kernel(const UnitDesc* __rest
                 Rn[0] = pack2(-s64.x, -s64.y); Rn[1] = pack2(-s64.z, -s64.w);
             }
             const uint64_t zero2 = pack2(0.f, 0.f);
-            for (int k = 0; k < n_tiles; ++k) {
-                issue(k + n_stages - 1);
-                if (n_stages == 3) asm volatile("cp.async.wait_group 2;" ::: "memory");
-                else if (n_stages == 2) asm volatile("cp.async.wait_group 1;" ::: "memory");
-                else asm volatile("cp.async.wait_group 0;" ::: "memory");
+            // Rows back to back in the cache: a tile is one run of bytes, fetched by one bulk copy that one thread
+            // issues and a barrier of the stage reports (no per-thread copy instructions, one CTA-wide barrier less
+            // per tile).  Any other layout goes through the per-thread 16-byte copies.
+            __shared__ uint64_t full_bar[3];
+            __shared__ int gave_up;
+            const bool bulk = sh.page_size == 0 && sh.row_stride == d;
+            if (bulk) {
+                if (threadIdx.x == 0) {
+                    for (int i = 0; i < 3; ++i) tc::mbar_init(&full_bar[i], 1);
+                    gave_up = 0;
+                    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+                }
                 __syncthreads();
+            }
+            auto fetch = [&](int k) {
+                if (!bulk) { issue(k); return; }
+                if (threadIdx.x == 0 && k < n_tiles) {
+                    const int row0 = first_row + k * kRowsPerCta, nrows = min(kRowsPerCta, T_u - row0);
+                    const uint32_t bytes = (uint32_t)nrows * (uint32_t)d * (uint32_t)sizeof(T);
+                    uint64_t* bar = &full_bar[k % n_stages];
+                    tc::mbar_expect_tx(bar, bytes);
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                 ::"r"(tc::smem_u32(stages + (size_t)(k % n_stages) * stage_elems)),
+                                   "l"(K + koff_u + (int64_t)row0 * d), "r"(bytes), "r"(tc::smem_u32(bar)) : "memory");
+                }
+            };
+            for (int k = 0; k < n_stages - 1; ++k) fetch(k);
+            for (int k = 0; k < n_tiles; ++k) {
+                fetch(k + n_stages - 1);
+                if (bulk) {
+                    if (!tc::mbar_wait(&full_bar[k % n_stages], (uint32_t)(k / n_stages) & 1u, &gave_up)) {
+                        // The wait ran out (about a second).  Copies already started may still land in this CTA's
+                        // shared memory: the issuing thread gives their barriers a bounded chance before it leaves.
+                        if (threadIdx.x == 0) {
+                            for (int kk = k; kk < min(n_tiles, k + n_stages); ++kk)
+                                for (uint32_t it = 0; it < 4096 && !tc::mbar_try(&full_bar[kk % n_stages], (uint32_t)(kk / n_stages) & 1u); ++it) {}
+                            atomicOr(sh.err, CASK_ST_TIMEOUT);
+                        }
+                        return;
+                    }
+                } else {
+                    if (n_stages == 3) asm volatile("cp.async.wait_group 2;" ::: "memory");
+                    else if (n_stages == 2) asm volatile("cp.async.wait_group 1;" ::: "memory");
+                    else asm volatile("cp.async.wait_group 0;" ::: "memory");
+                    __syncthreads();
+                }
                 const int row0 = first_row + k * kRowsPerCta, nrows = min(kRowsPerCta, T_u - row0);
                 const T* tile = stages + (size_t)(k % n_stages) * stage_elems;
                 float acc[4] = {0.f, 0.f, 0.f, 0.f};
@@ -336,6 +374,7 @@ __global__ void __launch_bounds__(256) score_stats_kernel(const UnitDesc* __rest
             return;
         }
     }
+    for (int k = 0; k < n_stages - 1; ++k) issue(k);
     for (int k = 0; k < n_tiles; ++k) {
         issue(k + n_stages - 1);
         // all but the newest n_stages - 1 groups have landed: tile k is in shared memory
