@@ -105,12 +105,14 @@ __global__ void __launch_bounds__(256) stats_fold_kernel(int g, int nb, cask_que
 }
 
 // One pass over the keys.  A CTA takes a run of up to kTilesPerCta tiles of 64 rows of one unit and streams them
-// through a ring of shared-memory stages with 16-byte asynchronous copies (cp.async), so several tiles are in flight
-// per CTA while it computes; the data stays in the cache dtype in shared memory.  A thread owns four consecutive rows
-// of a tile and a quad of four bands; sixteen threads cover a row.  The quad's constants sit in registers; the row
-// sums meet by shuffles.  Without caller-supplied offsets Delta falls by one from a row to the next, so after the
-// first of its rows a thread turns the phase by e^{-i omega} (four multiply-adds) instead of forming it anew.
-constexpr int kTilesPerCta = 8;
+// through a ring of shared-memory stages, so several tiles are in flight per CTA while it computes; the data stays in
+// the cache dtype in shared memory.  A thread owns four consecutive rows of a tile and a quad of four bands; sixteen
+// threads cover a row and the row sums meet by shuffles.
+// With caller-supplied offsets every (row, band) pair gets its own sine and cosine.  Without them Delta falls by one
+// from a row to the next and by 64 from a tile to the next, and the thread keeps the whole factor A e^{i omega Delta} of
+// its sixteen pairs in registers, turned by e^{-i 64 omega} once per tile (head_dim <= 128; larger heads form the
+// first row's phase per tile and turn it by e^{-i omega} from row to row).
+constexpr int kTilesPerCta = 16;
 
 template <typename T> struct Quad;       // four consecutive elements of a row as floats
 template <> struct Quad<__nv_bfloat16> {
