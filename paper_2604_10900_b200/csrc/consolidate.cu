@@ -56,7 +56,7 @@ __global__ void __launch_bounds__(kSelThreads) seeds_kernel(const UnitDesc* __re
 // ---- 1 for longer units on the event path: prefix eviction, core and seed selection in one CTA per unit ----
 // The same result as prefix_evict_kernel, select_core_kernel and seeds_kernel in turn; the core and the seeds come out of
 // one pair of thresholds (block_topk2_mark) and the per-row arrays are initialised once.
-__global__ void __launch_bounds__(kSelThreads) decide_long_kernel(
+__global__ void __launch_bounds__(kSelThreads, 2) decide_long_kernel(
     const UnitDesc* __restrict__ desc, const float* __restrict__ s, int32_t* __restrict__ plan,
     uint8_t* __restrict__ kind, int32_t* __restrict__ seed_of, float* __restrict__ weight, float* __restrict__ sim,
     int32_t* __restrict__ grp, int32_t* __restrict__ seed_rows, unsigned long long* __restrict__ mass_fx,
