@@ -467,7 +467,10 @@ def run_stats_scorer(args):
     pi = torch.from_numpy(pi / pi.sum(-1, keepdims=True)).to(device)
     grid = torch.arange(n_delta, dtype=torch.float32, device=device) * 16.0
     omega = torch.from_numpy((1.0 / (10000.0 ** (np.arange(nb) / nb))).astype(np.float32)).to(device)
-    qs, keep2 = cb.make_query_stats(mu, pi, grid, omega, 0)
+    # "stats_offsets": every row brings its own (fractional, signed) offset instead of Delta_i = T - 1 - i
+    offsets = args.scorer == "stats_offsets"
+    delta = (torch.rand(sum_T, dtype=torch.float32, device=device) * 45000.0 - 5000.0) if offsets else None
+    qs, keep2 = cb.make_query_stats(mu, pi, grid, omega, 0, delta)
     s = torch.empty(sum_T, dtype=torch.float32, device=device)
     for _ in range(max(args.warmup, 3)):
         cb.cask_score_stats(ctx, batch, prm, qs, s, ws, ws_bytes)
@@ -480,17 +483,21 @@ def run_stats_scorer(args):
     torch.cuda.synchronize()
     ms = ev0.elapsed_time(ev1) / args.steps
     peaks = _peaks()
-    byts = hb.k.nbytes + 4 * sum_T
+    byts = hb.k.nbytes + 4 * sum_T * (2 if offsets else 1)
     gbs = byts / (ms * 1e-3) / 1e9
     print(json.dumps({
         "metric": "kv_tokens_scored_per_s", "value": sum_T / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
         "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
         "dtype": "bf16" if w.dtype == wl.DTYPE_BF16 else "f32", "data": "synthetic",
-        "config": {"workload": w.name, "scorer": "query statistics (horizon kernel, mean score)", "units": hb.n_units,
+        "config": {"workload": w.name, "scorer": "query statistics (horizon kernel, mean score)" + (", caller offsets" if offsets else ""), "units": hb.n_units,
                    "rows_per_unit": int(hb.T.max()), "n_delta": n_delta,
                    "l2": "inputs larger than L2: %.2f GB of K read per step" % (hb.k.nbytes / 1e9)},
         "roofline": {"kernel": "score_stats_kernel", "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"],
-                     "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]},
+                     "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                     # bytes per cache row from the ncu capture of this kernel on a 16-unit slice x the rows of this
+                     # launch; the kernel for caller offsets has no capture
+                     "traffic": None if offsets else 263.6 * sum_T, "peak_source": peaks["source"],
+                     "traffic_source": None if offsets else "profiles/score_stats_reasoning32k_16units.txt"},
         "gpu_launches": 2 * args.steps}))
 
 
@@ -503,7 +510,7 @@ def main():
     ap.add_argument("--workload", default="reasoning32k_b512", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--score-path", type=int, default=0, help="0: tensor-core scoring when the shape allows, 1: SIMT")
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--scorer", default="attention", choices=["attention", "stats"],
+    ap.add_argument("--scorer", default="attention", choices=["attention", "stats", "stats_offsets"],
                     help="attention: the whole event with the windowed attention-mass score (default); "
                          "stats: time the query-statistics scorer of App. B alone")
     ap.add_argument("--similarity", default="cosine", choices=["cosine", "channel", "band"],
@@ -517,7 +524,7 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
-    elif args.scorer == "stats":
+    elif args.scorer in ("stats", "stats_offsets"):
         run_stats_scorer(args)
     else:
         run_ours(args)

@@ -239,6 +239,70 @@ __global__ void __launch_bounds__(256) score_stats_kernel(const UnitDesc* __rest
     const bool one_quad = nq <= 16;          // head_dim <= 128: a thread has at most one quad, its constants load once
     QuadConst c0 = {};
     if (one_quad && q < nq) load_const(q, c0);
+    // Rows back to back in the cache: a tile is one run of bytes, fetched by one bulk copy that one thread
+    // issues and a barrier of the stage reports (no per-thread copy instructions, one CTA-wide barrier less
+    // per tile).  Any other layout goes through the per-thread 16-byte copies.
+    __shared__ uint64_t full_bar[3];
+    __shared__ int gave_up;
+    const bool bulk = sh.page_size == 0 && sh.row_stride == d;
+    if (bulk) {
+        if (threadIdx.x == 0) {
+            for (int i = 0; i < 3; ++i) tc::mbar_init(&full_bar[i], 1);
+            gave_up = 0;
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        __syncthreads();
+    }
+    auto fetch = [&](int k) {
+        if (!bulk) { issue(k); return; }
+        if (threadIdx.x == 0 && k < n_tiles) {
+            const int row0 = first_row + k * kRowsPerCta, nrows = min(kRowsPerCta, T_u - row0);
+            const uint32_t bytes = (uint32_t)nrows * (uint32_t)d * (uint32_t)sizeof(T);
+            uint64_t* bar = &full_bar[k % n_stages];
+            tc::mbar_expect_tx(bar, bytes);
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(tc::smem_u32(stages + (size_t)(k % n_stages) * stage_elems)),
+                           "l"(K + koff_u + (int64_t)row0 * d), "r"(bytes), "r"(tc::smem_u32(bar)) : "memory");
+        }
+    };
+    // Tile k is in shared memory for every thread of the CTA; false when the bounded wait ran out.
+    auto landed = [&](int k) -> bool {
+        if (bulk) {
+            if (!tc::mbar_wait(&full_bar[k % n_stages], (uint32_t)(k / n_stages) & 1u, &gave_up)) {
+                // The wait ran out (about a second).  Copies already started may still land in this CTA's shared
+                // memory: the issuing thread gives their barriers a bounded chance before it leaves.
+                if (threadIdx.x == 0) {
+                    for (int kk = k; kk < min(n_tiles, k + n_stages); ++kk)
+                        for (uint32_t it = 0; it < 4096 && !tc::mbar_try(&full_bar[kk % n_stages], (uint32_t)(kk / n_stages) & 1u); ++it) {}
+                    atomicOr(sh.err, CASK_ST_TIMEOUT);
+                }
+                return false;
+            }
+        } else {
+            // all but the newest n_stages - 1 groups have landed
+            if (n_stages == 3) asm volatile("cp.async.wait_group 2;" ::: "memory");
+            else if (n_stages == 2) asm volatile("cp.async.wait_group 1;" ::: "memory");
+            else asm volatile("cp.async.wait_group 0;" ::: "memory");
+            __syncthreads();
+        }
+        return true;
+    };
+    // The four row sums meet over the sixteen lanes of a row group: the first two exchanges halve what a
+    // lane carries (a lane keeps the rows whose index bit matches its own), the last two add the rest;
+    // lane l of the group ends with the whole sum of row r_first + (l & 3) in its bit-reversed order.
+    auto reduce_store = [&](const float (&acc)[4], int row0, int nrows) {
+        const bool up1 = (q & 1) != 0;
+        const float give0 = up1 ? acc[0] : acc[1], give1 = up1 ? acc[2] : acc[3];
+        const float keep0 = up1 ? acc[1] : acc[0], keep1 = up1 ? acc[3] : acc[2];
+        const float h0 = keep0 + __shfl_xor_sync(0xffffffffu, give0, 1);       // rows (0|1), (2|3) by bit 0
+        const float h1 = keep1 + __shfl_xor_sync(0xffffffffu, give1, 1);
+        const bool up2 = (q & 2) != 0;
+        float t = (up2 ? h1 : h0) + __shfl_xor_sync(0xffffffffu, up2 ? h0 : h1, 2);
+        t += __shfl_xor_sync(0xffffffffu, t, 4);
+        t += __shfl_xor_sync(0xffffffffu, t, 8);
+        const int jr = (q & 1) + 2 * ((q >> 1) & 1);                          // the row this lane holds
+        if (q < 4 && r_first + jr < nrows) s[tok_u + row0 + r_first + jr] = t;
+    };
     if constexpr (STEP) {
         if (one_quad) {
             // Delta falls by one per row and by 64 per tile, so the whole factor G = A e^{i omega Delta} of each of the
@@ -284,52 +348,10 @@ __global__ void __launch_bounds__(256) score_stats_kernel(const UnitDesc* __rest
                 Rn[0] = pack2(-s64.x, -s64.y); Rn[1] = pack2(-s64.z, -s64.w);
             }
             const uint64_t zero2 = pack2(0.f, 0.f);
-            // Rows back to back in the cache: a tile is one run of bytes, fetched by one bulk copy that one thread
-            // issues and a barrier of the stage reports (no per-thread copy instructions, one CTA-wide barrier less
-            // per tile).  Any other layout goes through the per-thread 16-byte copies.
-            __shared__ uint64_t full_bar[3];
-            __shared__ int gave_up;
-            const bool bulk = sh.page_size == 0 && sh.row_stride == d;
-            if (bulk) {
-                if (threadIdx.x == 0) {
-                    for (int i = 0; i < 3; ++i) tc::mbar_init(&full_bar[i], 1);
-                    gave_up = 0;
-                    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-                }
-                __syncthreads();
-            }
-            auto fetch = [&](int k) {
-                if (!bulk) { issue(k); return; }
-                if (threadIdx.x == 0 && k < n_tiles) {
-                    const int row0 = first_row + k * kRowsPerCta, nrows = min(kRowsPerCta, T_u - row0);
-                    const uint32_t bytes = (uint32_t)nrows * (uint32_t)d * (uint32_t)sizeof(T);
-                    uint64_t* bar = &full_bar[k % n_stages];
-                    tc::mbar_expect_tx(bar, bytes);
-                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                                 ::"r"(tc::smem_u32(stages + (size_t)(k % n_stages) * stage_elems)),
-                                   "l"(K + koff_u + (int64_t)row0 * d), "r"(bytes), "r"(tc::smem_u32(bar)) : "memory");
-                }
-            };
             for (int k = 0; k < n_stages - 1; ++k) fetch(k);
             for (int k = 0; k < n_tiles; ++k) {
                 fetch(k + n_stages - 1);
-                if (bulk) {
-                    if (!tc::mbar_wait(&full_bar[k % n_stages], (uint32_t)(k / n_stages) & 1u, &gave_up)) {
-                        // The wait ran out (about a second).  Copies already started may still land in this CTA's
-                        // shared memory: the issuing thread gives their barriers a bounded chance before it leaves.
-                        if (threadIdx.x == 0) {
-                            for (int kk = k; kk < min(n_tiles, k + n_stages); ++kk)
-                                for (uint32_t it = 0; it < 4096 && !tc::mbar_try(&full_bar[kk % n_stages], (uint32_t)(kk / n_stages) & 1u); ++it) {}
-                            atomicOr(sh.err, CASK_ST_TIMEOUT);
-                        }
-                        return;
-                    }
-                } else {
-                    if (n_stages == 3) asm volatile("cp.async.wait_group 2;" ::: "memory");
-                    else if (n_stages == 2) asm volatile("cp.async.wait_group 1;" ::: "memory");
-                    else asm volatile("cp.async.wait_group 0;" ::: "memory");
-                    __syncthreads();
-                }
+                if (!landed(k)) return;
                 const int row0 = first_row + k * kRowsPerCta, nrows = min(kRowsPerCta, T_u - row0);
                 const T* tile = stages + (size_t)(k % n_stages) * stage_elems;
                 float acc[4] = {0.f, 0.f, 0.f, 0.f};
@@ -355,35 +377,16 @@ __global__ void __launch_bounds__(256) score_stats_kernel(const UnitDesc* __rest
                         acc[j] = lo + hi2;
                     }
                 }
-                // The four row sums meet over the sixteen lanes of a row group: the first two exchanges halve what a
-                // lane carries (a lane keeps the rows whose index bit matches its own), the last two add the rest;
-                // lane l of the group ends with the whole sum of row r_first + (l & 3) in its bit-reversed order.
-                {
-                    const bool up1 = (q & 1) != 0;
-                    const float give0 = up1 ? acc[0] : acc[1], give1 = up1 ? acc[2] : acc[3];
-                    const float keep0 = up1 ? acc[1] : acc[0], keep1 = up1 ? acc[3] : acc[2];
-                    const float h0 = keep0 + __shfl_xor_sync(0xffffffffu, give0, 1);       // rows (0|1), (2|3) by bit 0
-                    const float h1 = keep1 + __shfl_xor_sync(0xffffffffu, give1, 1);
-                    const bool up2 = (q & 2) != 0;
-                    float t = (up2 ? h1 : h0) + __shfl_xor_sync(0xffffffffu, up2 ? h0 : h1, 2);
-                    t += __shfl_xor_sync(0xffffffffu, t, 4);
-                    t += __shfl_xor_sync(0xffffffffu, t, 8);
-                    const int jr = (q & 1) + 2 * ((q >> 1) & 1);                          // the row this lane holds
-                    if (q < 4 && r_first + jr < nrows) s[tok_u + row0 + r_first + jr] = t;
-                }
+                reduce_store(acc, row0, nrows);
                 __syncthreads();        // the stage is free for the tile issued at the top of the next round
             }
             return;
         }
     }
-    for (int k = 0; k < n_stages - 1; ++k) issue(k);
+    for (int k = 0; k < n_stages - 1; ++k) fetch(k);
     for (int k = 0; k < n_tiles; ++k) {
-        issue(k + n_stages - 1);
-        // all but the newest n_stages - 1 groups have landed: tile k is in shared memory
-        if (n_stages == 3) asm volatile("cp.async.wait_group 2;" ::: "memory");
-        else if (n_stages == 2) asm volatile("cp.async.wait_group 1;" ::: "memory");
-        else asm volatile("cp.async.wait_group 0;" ::: "memory");
-        __syncthreads();
+        fetch(k + n_stages - 1);
+        if (!landed(k)) return;
         const int row0 = first_row + k * kRowsPerCta, nrows = min(kRowsPerCta, T_u - row0);
         const T* tile = stages + (size_t)(k % n_stages) * stage_elems;
         // offsets of this thread's rows: magnitude of the integer part, its sign, the fractional part
@@ -445,12 +448,7 @@ __global__ void __launch_bounds__(256) score_stats_kernel(const UnitDesc* __rest
                 }
             }
         }
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-#pragma unroll
-            for (int off = 1; off < 16; off <<= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], off);
-            if (q == 0 && r_first + j < nrows) s[tok_u + row0 + r_first + j] = acc[j];
-        }
+        reduce_store(acc, row0, nrows);
         __syncthreads();            // the stage is free for the tile issued at the top of the next round
     }
 }
