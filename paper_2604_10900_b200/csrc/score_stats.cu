@@ -193,10 +193,13 @@ __global__ void __launch_bounds__(256) score_stats_kernel(const UnitDesc* __rest
     const int vec_per_row = d / kPer;
     const size_t stage_elems = (size_t)kRowsPerCta * d;
     T* stages = reinterpret_cast<T*>(ring);
-    auto issue = [&](int k) {                                  // tile k of this CTA into stage k % n_stages
+    // Stages are used in turn; the positions are counted along (a remainder by the run-time number of stages in every
+    // round costs a division sequence per thread).
+    int f_stage = 0;                                           // stage of the next tile to be requested
+    auto issue = [&](int k) {                                  // tile k of this CTA into the next stage
         if (k < n_tiles) {
             const int row0 = first_row + k * kRowsPerCta, nrows = min(kRowsPerCta, T_u - row0);
-            T* dst = stages + (size_t)(k % n_stages) * stage_elems;
+            T* dst = stages + (size_t)f_stage * stage_elems;
             if (sh.page_size == 0 && sh.row_stride == d) {
                 // rows back to back in the cache: the tile is one contiguous run of 16-byte vectors
                 const T* src = K + koff_u + (int64_t)row0 * d;
@@ -254,21 +257,24 @@ __global__ void __launch_bounds__(256) score_stats_kernel(const UnitDesc* __rest
         __syncthreads();
     }
     auto fetch = [&](int k) {
-        if (!bulk) { issue(k); return; }
-        if (threadIdx.x == 0 && k < n_tiles) {
+        if (!bulk) issue(k);
+        else if (threadIdx.x == 0 && k < n_tiles) {
             const int row0 = first_row + k * kRowsPerCta, nrows = min(kRowsPerCta, T_u - row0);
             const uint32_t bytes = (uint32_t)nrows * (uint32_t)d * (uint32_t)sizeof(T);
-            uint64_t* bar = &full_bar[k % n_stages];
+            uint64_t* bar = &full_bar[f_stage];
             tc::mbar_expect_tx(bar, bytes);
             asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                         ::"r"(tc::smem_u32(stages + (size_t)(k % n_stages) * stage_elems)),
+                         ::"r"(tc::smem_u32(stages + (size_t)f_stage * stage_elems)),
                            "l"(K + koff_u + (int64_t)row0 * d), "r"(bytes), "r"(tc::smem_u32(bar)) : "memory");
         }
+        if (++f_stage == n_stages) f_stage = 0;
     };
     // Tile k is in shared memory for every thread of the CTA; false when the bounded wait ran out.
+    int c_stage = 0;                      // stage of the tile being consumed and the parity of its barrier phase
+    uint32_t c_phase = 0;
     auto landed = [&](int k) -> bool {
         if (bulk) {
-            if (!tc::mbar_wait(&full_bar[k % n_stages], (uint32_t)(k / n_stages) & 1u, &gave_up)) {
+            if (!tc::mbar_wait(&full_bar[c_stage], c_phase, &gave_up)) {
                 // The wait ran out (about a second).  Copies already started may still land in this CTA's shared
                 // memory: the issuing thread gives their barriers a bounded chance before it leaves.
                 if (threadIdx.x == 0) {
@@ -353,7 +359,8 @@ __global__ void __launch_bounds__(256) score_stats_kernel(const UnitDesc* __rest
                 fetch(k + n_stages - 1);
                 if (!landed(k)) return;
                 const int row0 = first_row + k * kRowsPerCta, nrows = min(kRowsPerCta, T_u - row0);
-                const T* tile = stages + (size_t)(k % n_stages) * stage_elems;
+                const T* tile = stages + (size_t)c_stage * stage_elems;
+                if (++c_stage == n_stages) { c_stage = 0; c_phase ^= 1u; }
                 float acc[4] = {0.f, 0.f, 0.f, 0.f};
                 if (active) {
 #pragma unroll
@@ -388,7 +395,8 @@ __global__ void __launch_bounds__(256) score_stats_kernel(const UnitDesc* __rest
         fetch(k + n_stages - 1);
         if (!landed(k)) return;
         const int row0 = first_row + k * kRowsPerCta, nrows = min(kRowsPerCta, T_u - row0);
-        const T* tile = stages + (size_t)(k % n_stages) * stage_elems;
+        const T* tile = stages + (size_t)c_stage * stage_elems;
+        if (++c_stage == n_stages) { c_stage = 0; c_phase ^= 1u; }
         // offsets of this thread's rows: magnitude of the integer part, its sign, the fractional part
         unsigned Dm[4];
         float Dsg[4], Df[4];
