@@ -169,6 +169,9 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     // At most 128 accumulator columns in every unit: the seed matrix is loaded as 128 rows and the shared-memory
     // area holds two of them, so the next unit's seeds arrive while the tensor pipe still works on this unit's.
     const bool dual = n_bufs == kMaxGroups;
+    // n_bufs is 2 or 4: positions among the buffers by mask and shift (a remainder by a run-time value is a division
+    // sequence, and the epilogue warps take one per tile, their own or not)
+    const uint32_t buf_mask = (uint32_t)n_bufs - 1u, buf_shift = n_bufs == 4 ? 2u : 1u;
     const uint32_t seed_region = dual ? 128u * 128u : kSeedRegionBytes;      // one 64-channel half of a seed buffer
 
     if (threadIdx.x == 0) {
@@ -259,7 +262,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 const int nt = wk.run();
                 for (int t = 0; t < nt && ok; ++t, ++kit) {
                     const int st = kit % kStages;
-                    const uint32_t buf = kit % (uint32_t)n_bufs, use = kit / (uint32_t)n_bufs;
+                    const uint32_t buf = kit & buf_mask, use = kit >> buf_shift;
                     ok = mbar_wait(&bar.k_full[st], (kit / kStages) & 1u, abort_flag);
                     if (!ok) break;
                     ok = mbar_wait(&bar.d_empty[buf], (use & 1u) ^ 1u, abort_flag);
@@ -285,8 +288,8 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         // ================= epilogue =================
         const int ew = warp - kEpiWarp0;
         const int qd = ew & 3;                               // TMEM lane quadrant (== warp % 4)
-        const uint32_t eg = (uint32_t)(ew >> 2) % (uint32_t)n_bufs;   // buffer: tiles eg, eg + n_bufs, ...
-        const int half = (ew >> 2) / n_bufs;                 // 0: finishes the row; 1: the later seed columns only
+        const uint32_t eg = (uint32_t)(ew >> 2) & buf_mask;   // buffer: tiles eg, eg + n_bufs, ...
+        const int half = (ew >> 2) >> buf_shift;                 // 0: finishes the row; 1: the later seed columns only
         const uint32_t taddr = tmem_base + ((uint32_t)(32 * qd) << 16) + eg * buf_cols;
         const int my_row = 32 * qd + lane;                   // row of the tile this thread owns
         uint32_t kit = 0, ucount = 0;
@@ -310,7 +313,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             // Does this group take a tile of the unit?  Only then it needs the table of inverse seed norms; it
             // builds its own copy (two values per thread) and meets on its own barrier, so the groups never
             // wait for one another between units.
-            const int first = (int)((eg + (uint32_t)n_bufs - kit % (uint32_t)n_bufs) % (uint32_t)n_bufs);
+            const int first = (int)((eg + (uint32_t)n_bufs - (kit & buf_mask)) & buf_mask);
             if (first >= nt) {
                 kit += nt;
                 wk.advance(nt);
@@ -331,9 +334,9 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             }
             ++ucount;
             for (int t = 0; t < nt && ok; ++t, ++kit) {
-                if (kit % (uint32_t)n_bufs != eg) continue;
+                if ((kit & buf_mask) != eg) continue;
                 const int st = kit % kStages;
-                const uint32_t use = kit / (uint32_t)n_bufs;
+                const uint32_t use = kit >> buf_shift;
                 if (half == 1) {
                     // second group of a shared buffer: best seed among the columns [c_split, m)
                     ok = mbar_wait(&bar.d_full[eg], use & 1u, abort_flag);
