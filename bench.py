@@ -39,7 +39,7 @@ UNIT = "tokens/s"
 NCU_TRAFFIC = {
     "score_norm": (268.0, "profiles/score_tc_reasoning32k_16units.txt"),
     "score_mass": (274.2, "profiles/score_tc_reasoning32k_16units.txt"),
-    "assign": (266.2, "profiles/assign_tc_reasoning32k_16units.txt"),
+    "assign": (264.9, "profiles/assign_tc_reasoning32k_16units.txt"),
 }
 # ex2 units: 16 results per clock per SM (special-function pipe), 148 SMs, 1.965 GHz maximum SM clock.
 EX2_PEAK_T_PER_S = 148 * 16 * 1.965e9 / 1e12
