@@ -496,7 +496,7 @@ def run_stats_scorer(args):
                      "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
                      # bytes per cache row from the ncu capture of this kernel on a 16-unit slice x the rows of this
                      # launch; the kernel for caller offsets has no capture
-                     "traffic": None if offsets else 263.6 * sum_T, "peak_source": peaks["source"],
+                     "traffic": None if offsets else 268.5 * sum_T, "peak_source": peaks["source"],
                      "traffic_source": None if offsets else "profiles/score_stats_reasoning32k_16units.txt"},
         "gpu_launches": 2 * args.steps}))
 
