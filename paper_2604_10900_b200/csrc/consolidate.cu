@@ -81,7 +81,8 @@ __global__ void __launch_bounds__(kSelThreads, 2) decide_long_kernel(
     if (threadIdx.x == 0) njoin[u] = 0;
     __syncthreads();
     if (P > pkeep) block_topk_mark(s + o, kind + o, 0, P, pkeep, CASK_KIND_PREFIX, sm);
-    block_topk2_mark(s + o, kind + o, P, T - r, c, CASK_KIND_CORE, m, CASK_KIND_SEED, sm, sm2);
+    // the rows of [P, T - r) were all set to kind 0 above and the prefix eviction touches [0, P) only
+    block_topk2_mark<true>(s + o, kind + o, P, T - r, c, CASK_KIND_CORE, m, CASK_KIND_SEED, sm, sm2);
     if (m <= 0) return;
     block_ordered_rows(kind + o, P, T - r, CASK_KIND_SEED, sm, [&](unsigned idx, int i) {
         if (idx < (unsigned)m) {

@@ -242,6 +242,8 @@ __device__ inline void block_topk_mark(const float* __restrict__ s, uint8_t* kin
 // is what block_topk_mark(k1, mark1) followed by block_topk_mark(k2, mark2) gives.  The three histogram sweeps narrow
 // both thresholds (rank k1 and rank k1 + k2) at once, with a second histogram where their digit prefixes part; one
 // marking sweep follows.  A tie at either threshold, or a selection that takes every row, goes the plain way.
+// ALL_OPEN: the caller knows that every row of [lo, hi) is still unmarked (kind 0), so the sweeps need not read the kinds.
+template <bool ALL_OPEN = false>
 __device__ inline void block_topk2_mark(const float* __restrict__ s, uint8_t* kind, int lo, int hi, int k1, uint8_t mark1,
                                         int k2, uint8_t mark2, SelectSmem& sm, SelectSmem& sm2) {
     const int tid = threadIdx.x, nthr = blockDim.x;
@@ -258,7 +260,7 @@ __device__ inline void block_topk2_mark(const float* __restrict__ s, uint8_t* ki
     unsigned mine = 0;
     for (int it = 0; it < iters; ++it) {
         const int i = lo + it * nthr + tid;
-        if (i < hi && kind[i] == 0) { atomicAdd(&sm.hist[order_key(s[i]) >> 20], 1u); ++mine; }
+        if (i < hi && (ALL_OPEN || kind[i] == 0)) { atomicAdd(&sm.hist[order_key(s[i]) >> 20], 1u); ++mine; }
     }
     const unsigned n_elig = block_sum(mine, sm);
     if ((unsigned)(k1 + k2) >= n_elig) { __syncthreads(); plain(); return; }
@@ -280,7 +282,7 @@ __device__ inline void block_topk2_mark(const float* __restrict__ s, uint8_t* ki
         __syncthreads();
         for (int it = 0; it < iters; ++it) {
             const int i = lo + it * nthr + tid;
-            if (i < hi && kind[i] == 0) {
+            if (i < hi && (ALL_OPEN || kind[i] == 0)) {
                 const unsigned key = order_key(s[i]), pre = key >> (shift + bits), dg = (key >> shift) & (unsigned)(nbins - 1);
                 if (pre == pa) atomicAdd(&sm.hist[dg], 1u);
                 else if (pre == pb) atomicAdd(&sm2.hist[dg], 1u);
@@ -310,7 +312,7 @@ __device__ inline void block_topk2_mark(const float* __restrict__ s, uint8_t* ki
     // selection, kb of the neq_b rows equal to pb inside the two together
     if (ka != neq_a || kb != neq_b) { plain(); return; }      // rows tie across a boundary: index order decides
     for (int i = lo + tid; i < hi; i += nthr)
-        if (kind[i] == 0) {
+        if (ALL_OPEN || kind[i] == 0) {
             const unsigned key = order_key(s[i]);
             if (key >= pa) kind[i] = mark1;
             else if (key >= pb) kind[i] = mark2;
