@@ -545,6 +545,7 @@ __global__ void __launch_bounds__(kThreads) assign_band_kernel(
 }
 
 // ---- 4. merge weights w_i = a_i / m_G, lost mass, status ---------------------------------
+constexpr int kWeightRows = 4;     // rows per thread
 __global__ void weights_kernel(const UnitDesc* __restrict__ desc, Shape sh, const float* __restrict__ s,
                                const int32_t* __restrict__ plan, const int32_t* __restrict__ grp,
                                const unsigned long long* __restrict__ mass_fx,
@@ -553,13 +554,24 @@ __global__ void weights_kernel(const UnitDesc* __restrict__ desc, Shape sh, cons
                                float eps, const int32_t* __restrict__ err) {
     const int u = blockIdx.y;
     const UnitDesc& ud = desc[u];
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
     const unsigned long long* mf = mass_fx + (size_t)u * (max_m + 1);
-    if (i < ud.T) {
-        int gidx = grp[ud.tok_off + i];
-        if (gidx >= 0 && gidx < max_m) weight[ud.tok_off + i] = row_mass(sh, s, eps, ud.tok_off + i) / fx_to_mass(mf[gidx]);
+    const int T = ud.T;
+    const int64_t o = ud.tok_off;
+    // four rows per thread, a block apart (most rows belong to no group and only read their group index; a CTA
+    // per 256 rows spent its time being launched)
+    const int i0 = blockIdx.x * (kWeightRows * (int)blockDim.x) + threadIdx.x;
+    int gidx[kWeightRows];
+#pragma unroll
+    for (int j = 0; j < kWeightRows; ++j) {
+        const int i = i0 + j * (int)blockDim.x;
+        gidx[j] = i < T ? grp[o + i] : -1;
     }
-    if (i == 0) {
+#pragma unroll
+    for (int j = 0; j < kWeightRows; ++j) {
+        const int i = i0 + j * (int)blockDim.x;
+        if (gidx[j] >= 0 && gidx[j] < max_m) weight[o + i] = row_mass(sh, s, eps, o + i) / fx_to_mass(mf[gidx[j]]);
+    }
+    if (i0 == 0) {
         int fl = plan[u * 8 + CASK_PLAN_FLAGS];
         if ((fl & CASK_ST_DECODE_CONSOLIDATED) && njoin[u] == 0) fl |= CASK_ST_MERGE_INACTIVE;
         unit_status[u] = fl | *err;     // device-side flags of this call (bounded wait gave up, bad page id)
@@ -623,7 +635,7 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const i
     }
     {
         Timed t(L, KID_WEIGHTS);
-        weights_kernel<<<dim3((L.max_T + 255) / 256, sh.n_units), 256, 0, L.stream>>>(
+        weights_kernel<<<dim3((L.max_T + 256 * kWeightRows - 1) / (256 * kWeightRows), sh.n_units), 256, 0, L.stream>>>(
             L.desc, sh, s, plan, ws.grp, ws.mass_fx, ws.njoin, weight, unit_status, lost_mass, max_m, prm.eps, ws.err);
     }
     return cudaGetLastError();
