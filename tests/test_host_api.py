@@ -78,3 +78,26 @@ def test_null_context_is_refused():
     b, keep = _batch([1000], [100], [128], [64])
     rc = cb.lib().cask_score(None, C.byref(b), C.byref(cb.params()), 0x100, None, 0x100, 1 << 30)
     assert rc == cb.ERR_NULL
+
+
+def test_host_event_device_bytes_of_one_slice_and_of_many():
+    """The host-buffer entry point cuts a batch with more than 16 MB of keys into slices of units, each with its own
+    staging area and workspace inside the caller's buffer: the size it asks for holds the keys and values of every
+    unit once, grows with the batch, and is the plain single-batch size below the cut."""
+    prm = cb.params()
+    d, W, g, Bmax = 128, 16, 2, 256
+    kv = lambda T: 2 * int(np.sum(T)) * d * 4          # fp32 keys + values (the dtype _batch builds)
+    small_T = [3000] * 4                                # 6 MB of keys: one slice
+    b1, keep1 = _batch(small_T, [100] * 4, [Bmax] * 4, [64] * 4, W=W, d=d, g=g)
+    n1 = cb.cask_host_event_device_bytes(b1, prm, Bmax)
+    assert n1 % 256 == 0 and n1 > kv(small_T) + cb.cask_workspace_bytes(b1, prm)
+    big_T = [9000 + 37 * (i % 5) for i in range(60)]    # 277 MB of keys: about ten slices of ragged units
+    b2, keep2 = _batch(big_T, [100] * 60, [Bmax] * 60, [64] * 60, W=W, d=d, g=g)
+    n2 = cb.cask_host_event_device_bytes(b2, prm, Bmax)
+    assert n2 % 256 == 0 and n2 > kv(big_T)
+    # per-slice workspaces together stay close to the workspace of the whole batch (a fixed part per slice)
+    whole = kv(big_T) + cb.cask_workspace_bytes(b2, prm)
+    assert whole < n2 < 1.6 * whole
+    assert cb.cask_host_event_device_bytes(b2, prm, 0) == 0          # no output rows
+    bad, keep3 = _batch(big_T, [100] * 60, [Bmax] * 60, [300] * 60, W=W, d=d, g=g)   # reserve > B
+    assert cb.cask_host_event_device_bytes(bad, prm, Bmax) == 0
