@@ -37,7 +37,8 @@ extern "C" {
 #define CASK_ERR_ALIGN         -3   /* a base pointer, offset or row stride breaks the 16-byte rule */
 #define CASK_ERR_WORKSPACE     -4   /* workspace NULL or smaller than cask_workspace_bytes */
 #define CASK_ERR_UNSUPPORTED   -5   /* a documented but unbuilt combination (paged cache through
-                                       the host-buffer or the no-allocation entry point) */
+                                       the host-buffer or the no-allocation entry point, the
+                                       no-allocation entry point on a stream that is being captured) */
 #define CASK_ERR_CUDA          -6   /* a CUDA runtime call failed (see cask_last_cuda_error) */
 #define CASK_ERR_PARAM         -7   /* gamma/tau/eps/causal out of range              */
 #define CASK_ERR_TOO_LARGE     -8   /* batch exceeds a fixed capacity (cask_score_noalloc) */
@@ -202,9 +203,35 @@ const char* cask_kernel_name(int id);
 /* 1 if the last cask_score / cask_compress_event used the tensor-core kernels. */
 int cask_last_score_path_tensor(const cask_ctx* ctx);
 /* Device-side flags (CASK_ST_TIMEOUT, CASK_ST_BOUNDS) raised by the kernels of the last call of this
- * context; waits for the context's stream.  cask_consolidate_scratch and cask_compress_event also OR
- * them into unit_status. */
+ * context; waits for the context's stream.  cask_consolidate_scratch ORs the flags raised up to the
+ * end of that call into unit_status; cask_compress_event and cask_compress_event_host do so once more
+ * as the last step of the event, so there unit_status also carries flags raised by the compaction.
+ * The staged cask_compact and cask_writeback_paged write no unit_status: their flags are read here. */
 int cask_last_device_flags(cask_ctx* ctx, int32_t* flags_host);
+
+/*
+ * Self-test of the bounded device waits (no counterpart in the paper).  Every wait of the kernels on a
+ * hardware barrier gives up after a wall-time limit and makes the kernel end with CASK_ST_TIMEOUT
+ * instead of hanging; in a healthy run that path never executes.  This call runs it once: one small
+ * CTA waits for `limit_ns` (1,000 .. 100,000,000) on a barrier nobody arrives at, gives up, raises
+ * the flag and returns.  Nothing faults and the context stays usable.  ws: DEVICE, at least 64 bytes,
+ * 16-byte aligned.  Waits for the stream.  flags_host receives the device flags of the call (also
+ * readable through cask_last_device_flags until the next call); waited_ns_host, optional, two words:
+ * the time the waiting warp spent before it gave up, and the time a second warp of the CTA, waiting
+ * with the default limit, spent before it saw the first one give up and followed it.
+ */
+int cask_selftest_wait_timeout(cask_ctx* ctx, uint64_t limit_ns, void* ws, size_t ws_bytes,
+                               int32_t* flags_host, uint64_t* waited_ns_host);
+
+/*
+ * Measures what the special-function unit of this GPU sustains (no counterpart in the paper): one CTA of
+ * 16 warps per SM runs `iters` (16 .. 2^20) rounds of eight independent chains of the scoring epilogue's
+ * per-element mix (FFMA, ex2.approx, FADD, FMUL) and times itself with the SM clock; rate_host receives
+ * the median over the SMs of exponentials per clock per SM.  The scoring passes evaluate one exponential
+ * per (query row, key), so this rate x SMs x clock is the roof the benchmark holds them against.
+ * ws: DEVICE, at least 16 + 8 x SMs bytes, 16-byte aligned.  Waits for the stream.
+ */
+int cask_selftest_exp_rate(cask_ctx* ctx, int32_t iters, void* ws, size_t ws_bytes, double* rate_host);
 
 /* Bytes of workspace that any call below needs for this batch (host-only arithmetic). */
 size_t cask_workspace_bytes(const cask_batch* batch, const cask_params* params);
@@ -373,7 +400,10 @@ int cask_compress_event_host(cask_ctx* ctx, const cask_batch* host_batch, const 
  *   + the descriptor table  <=  CASK_NOALLOC_SCRATCH_BYTES;
  * beyond either, CASK_ERR_TOO_LARGE is returned before anything is launched.
  * The first call on a device looks the array's device address up (cudaGetSymbolAddress, once per
- * device); make that first call before any stream capture begins.  All calls on a device share
+ * device); make that first call before any stream capture begins.  A call whose stream is being
+ * captured is refused with CASK_ERR_UNSUPPORTED before anything is launched or copied (the unit
+ * descriptors go up from a host array that lives only for the duration of the call).  The calling
+ * thread's current device is the same after the call as before it.  All calls on a device share
  * the one array: two calls whose kernels may overlap on the GPU (different streams, or different
  * host threads without ordering) race on it and must be serialised by the caller.  Nothing in the
  * array needs clearing between calls: each call writes every word it later reads.

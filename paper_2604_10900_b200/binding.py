@@ -32,6 +32,7 @@ EXPORTS = (
     "cask_kernel_count", "cask_kernel_name", "cask_workspace_bytes", "cask_plan_host",
     "cask_score", "cask_score_stats", "cask_prefix_evict", "cask_select_core", "cask_consolidate_scratch", "cask_compact",
     "cask_compress_event", "cask_writeback_paged", "cask_host_event_device_bytes", "cask_compress_event_host", "cask_score_noalloc",
+    "cask_selftest_wait_timeout", "cask_selftest_exp_rate",
 )
 
 
@@ -117,6 +118,8 @@ def lib():
         L.cask_host_event_device_bytes.restype = sz
         L.cask_compress_event_host.argtypes = [vp, PB, PP, PO, vp, sz]
         L.cask_score_noalloc.argtypes = [i32, vp, PB, PP, vp, vp]
+        L.cask_selftest_wait_timeout.argtypes = [vp, C.c_uint64, vp, sz, vp, vp]
+        L.cask_selftest_exp_rate.argtypes = [vp, C.c_int32, vp, sz, vp]
         _lib = L
     return _lib
 
@@ -364,6 +367,24 @@ def cask_score_noalloc(device: int, stream, batch, prm, s, lse_out=None, check: 
     if check:
         _check(rc)
     return rc
+
+
+def cask_selftest_wait_timeout(ctx: Context, limit_ns: int, ws, ws_bytes: int, check: bool = True):
+    """Makes one bounded device wait run out (see ``cask_selftest_wait_timeout`` in ``include/cask.h``).
+    Returns (return code, device flags, ns the waiting warp spent, ns the following warp spent)."""
+    flags = C.c_int32(0)
+    waited = (C.c_uint64 * 2)(0, 0)
+    rc = lib().cask_selftest_wait_timeout(ctx.handle, limit_ns, _ptr(ws), ws_bytes, C.addressof(flags), C.addressof(waited))
+    if check:
+        _check(rc, ctx)
+    return rc, int(flags.value), int(waited[0]), int(waited[1])
+
+
+def cask_selftest_exp_rate(ctx: Context, iters: int, ws, ws_bytes: int) -> float:
+    """Exponentials per clock per SM the special-function unit sustains in the scoring epilogue's instruction mix."""
+    rate = C.c_double(0.0)
+    _check(lib().cask_selftest_exp_rate(ctx.handle, iters, _ptr(ws), ws_bytes, C.addressof(rate)), ctx)
+    return float(rate.value)
 
 
 # ---- device-memory plumbing (torch): allocation of inputs, outputs and workspace -------------

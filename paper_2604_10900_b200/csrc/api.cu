@@ -62,6 +62,7 @@ struct cask_ctx {
     int32_t* hs_flags = nullptr;     // pinned, kMaxSlices words
     int32_t flags_last = 0;          // flags of a call that has already read them back
     void* tmap_encode = nullptr;     // cuTensorMapEncodeTiled, resolved at creation
+    int sms = 0;                     // multiprocessors of the device
     Profiler prof;
     ProfImpl prof_impl;
 };
@@ -292,6 +293,7 @@ int prepare(cask_ctx* ctx, const cask_batch* b, const cask_params* p, void* ws, 
     L.total_tiles = tile0;
     L.tmap_encode = ctx->tmap_encode;
     L.force_simt = p->score_path;
+    L.sms = ctx->sms;
     L.launches = &ctx->launches;
     L.prof = &ctx->prof;
     return CASK_OK;
@@ -315,6 +317,16 @@ int run_score(cask_ctx* ctx, const Launch& L, const cask_batch* b, const cask_pa
 namespace cask {
 // The host-side argument check, for entry points that live in other files.
 int check_batch_host(const cask_batch* b, const cask_params* p) { return check_batch(b, p); }
+// The self-tests: their flag word (if any) becomes the one cask_last_device_flags reads, their launches are counted.
+int selftest_set_flags_source(cask_ctx* ctx, const int32_t* flags_dev, int n_launches, cudaStream_t* stream, int* device) {
+    if (!ctx) return CASK_ERR_NULL;
+    ctx->flags_dev = flags_dev;
+    ctx->flags_last = 0;
+    ctx->launches += n_launches;
+    *stream = ctx->stream;
+    *device = ctx->device;
+    return CASK_OK;
+}
 }  // namespace cask
 
 extern "C" {
@@ -331,6 +343,7 @@ int cask_create(cask_ctx** out, int device, void* cuda_stream) {
     c->prof.impl = &c->prof_impl;
     e = cudaEventCreateWithFlags(&c->staged, cudaEventDisableTiming);
     if (e != cudaSuccess) { delete c; return CASK_ERR_CUDA; }
+    if (cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) c->sms = 0;
     cudaDriverEntryPointQueryResult qres;
     void* fn = nullptr;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
@@ -374,7 +387,7 @@ const char* cask_strerror(int code) {
         case CASK_ERR_SHAPE: return "shape out of range (head_dim, group, window, T, P, B, reserve, offsets)";
         case CASK_ERR_ALIGN: return "pointer, offset or row stride is not a multiple of 16 bytes";
         case CASK_ERR_WORKSPACE: return "workspace missing, misaligned (256 B) or too small";
-        case CASK_ERR_UNSUPPORTED: return "mode not built (paged cache through the host-buffer entry point)";
+        case CASK_ERR_UNSUPPORTED: return "mode not built (paged cache through the host-buffer or no-allocation entry point, or a capturing stream there)";
         case CASK_ERR_CUDA: return "CUDA runtime error";
         case CASK_ERR_PARAM: return "policy parameter out of range";
         case CASK_ERR_TOO_LARGE: return "batch exceeds the fixed capacity of the no-allocation entry point";
@@ -562,6 +575,7 @@ static int event_compact(cask_ctx* ctx, Launch& L, Workspace& W, const cask_para
     float* s = out->s ? out->s : W.s;
     cudaError_t e = launch_compact(L, *p, s, out->kind, out->seed_of, out->weight, *out, W);
     if (e == cudaSuccess) e = launch_diagnostics(L, *p, s, out->kind, *out);
+    if (e == cudaSuccess) e = launch_status_flags(L, W.err, out->unit_status);
     return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
 }
 

@@ -78,6 +78,7 @@ struct Launch {
     Profiler* prof;
     void* tmap_encode;        // cuTensorMapEncodeTiled or nullptr
     int force_simt;
+    int sms;                  // multiprocessors of the context's device (0: not known)
 };
 
 // Scope guard around one kernel launch: counts it and, in profiling mode, times it.
@@ -145,6 +146,10 @@ cudaError_t launch_writeback(const Launch& L, const cask_outputs& out, void* k_p
 // rho_core / rho_rep and the within-group dispersion of Sec. 2.6 per unit (any of the pointers may be NULL).
 cudaError_t launch_diagnostics(const Launch& L, const cask_params& prm, const float* s, const uint8_t* kind,
                                const cask_outputs& out);
+
+// Last kernel of an event: the device flags of the call (ws.err) are ORed into every unit's status word once more,
+// so that flags raised by the compaction kernels are not missed by a caller that reads unit_status alone.
+cudaError_t launch_status_flags(const Launch& L, const int32_t* err, int32_t* unit_status);
 
 // Tensor-core assignment of scratch rows to seeds (cosine Gram + argmax), same outputs as the SIMT kernel.
 bool assign_tc_supported(const Launch& L);

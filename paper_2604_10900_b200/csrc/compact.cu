@@ -539,7 +539,7 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const u
         cudaError_t ce = cudaFuncSetAttribute(slot_copy_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               copy_smem_bytes);
         if (ce != cudaSuccess) return ce;
-        const int copy_grid = (int)std::min<int64_t>((batches + kCopyWarps - 1) / kCopyWarps, 148);   // one CTA per SM
+        const int copy_grid = (int)std::min<int64_t>((batches + kCopyWarps - 1) / kCopyWarps, L.sms > 0 ? L.sms : 128);   // one CTA per SM
         slot_copy_kernel<T><<<std::max(copy_grid, 1), kCopyWarps * 32, copy_smem_bytes, L.stream>>>(
             L.desc, sh, (const T*)L.k, (const T*)L.v, s, prm.eps, out.Bmax, slots, out.n_out, out.slot_src,
             (T*)out.k_out, (T*)out.v_out, out.slot_mass);

@@ -34,6 +34,19 @@ void* g_scratch_addr[kMaxDevices] = {};
 
 inline size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 
+// Makes `device` current for the duration of a call and puts the caller's device back on every way out.
+struct DeviceGuard {
+    int prev = -1;
+    bool enter(int device) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { prev = -1; return false; }
+        if (prev == device) { prev = -1; return true; }
+        return cudaSetDevice(device) == cudaSuccess;
+    }
+    ~DeviceGuard() {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
 }  // namespace
 
 extern "C" int cask_score_noalloc(int device, void* cuda_stream, const cask_batch* b, const cask_params* p,
@@ -64,8 +77,16 @@ extern "C" int cask_score_noalloc(int device, void* cuda_stream, const cask_batc
     const size_t need = off_pl + up256(total_chunks * rows * 4);
     if (need > (size_t)CASK_NOALLOC_SCRATCH_BYTES) return CASK_ERR_TOO_LARGE;
 
-    cudaError_t e = cudaSetDevice(device);
+    // The calling thread keeps the current device it came with.
+    DeviceGuard guard;
+    if (!guard.enter(device)) return CASK_ERR_CUDA;
+    // A stream that is being captured is refused: the descriptor upload below reads a host array that is gone
+    // when this call returns, so a recorded copy of it could never be replayed.
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    cudaError_t e = cudaStreamIsCapturing(st, &cap);
     if (e != cudaSuccess) return CASK_ERR_CUDA;
+    if (cap != cudaStreamCaptureStatusNone) return CASK_ERR_UNSUPPORTED;
     unsigned char* base = nullptr;
     {
         // first call on this device: resolve the array's device address (once per device, with that
@@ -95,7 +116,6 @@ extern "C" int cask_score_noalloc(int device, void* cuda_stream, const cask_batc
         d.n_chunks = (d.T + kChunkKeys - 1) / kChunkKeys;
         chunk0 += d.n_chunks;
     }
-    cudaStream_t st = (cudaStream_t)cuda_stream;
     // pageable source: the runtime has taken its copy of hd[] when this returns
     e = cudaMemcpyAsync(base + off_desc, hd, sizeof(UnitDesc) * n, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return CASK_ERR_CUDA;

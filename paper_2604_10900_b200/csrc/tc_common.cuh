@@ -41,9 +41,10 @@ __device__ __forceinline__ uint64_t global_ns() {
     return t;
 }
 // Bounded wait: false when the time limit ran out or another role already gave up.  The limit is
-// wall time (kWaitLimitNs), so a wait that cannot end costs about a second, whatever the hardware's
-// own suspend interval is.
-__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag) {
+// wall time (one second unless the caller gives another), so a wait that cannot end costs about that
+// long, whatever the hardware's own suspend interval is.
+__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag,
+                                          uint64_t limit_ns = kWaitLimitNs) {
     uint64_t t0 = 0;
     for (uint32_t it = 0; it < kSpinLimit; ++it) {
         if (mbar_try(b, parity)) return true;
@@ -51,7 +52,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile
         if ((it & 63u) == 63u) {
             const uint64_t now = global_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) break;
+            else if (now - t0 > limit_ns) break;
         }
     }
     *abort_flag = 1;

@@ -554,6 +554,40 @@ def test_bad_arguments_are_refused_on_the_host_before_any_launch():
     run.event()
 
 
+def test_a_bounded_device_wait_that_runs_out_reports_timeout_and_leaves_the_context_usable():
+    """Every barrier wait of the kernels gives up after a wall-time limit and ends the kernel with CASK_ST_TIMEOUT
+    instead of hanging.  The self-test entry point makes one such wait run out (a barrier nobody arrives at, a limit
+    of two milliseconds): the kernel must return by itself, the flag must show, a second warp waiting with the
+    default one-second limit must follow the first out at once, and the context must still give a correct event."""
+    import gpu_harness as gh
+    import torch
+    hb = wl.make_batch(wl.WORKLOADS["tiny"])
+    run = gh.GpuRun(hb)
+    cb = run.cb
+    before = run.event()
+    assert run.ctx.device_flags() == 0
+    limit = 2_000_000
+    rc, flags, waited, followed = cb.cask_selftest_wait_timeout(run.ctx, limit, run.ws, run.ws_bytes)
+    assert rc == cb.OK and flags == cb.ST_TIMEOUT
+    assert run.ctx.device_flags() == cb.ST_TIMEOUT
+    assert limit <= waited < 50 * limit              # gave up after the limit, not after the default second
+    assert 0 < followed < 50 * limit                 # the follower left on the abort flag
+    # out-of-range limits and a missing workspace are refused on the host
+    n0 = run.ctx.launches
+    assert cb.cask_selftest_wait_timeout(run.ctx, 10, run.ws, run.ws_bytes, check=False)[0] == cb.ERR_PARAM
+    assert cb.cask_selftest_wait_timeout(run.ctx, 10**10, run.ws, run.ws_bytes, check=False)[0] == cb.ERR_PARAM
+    assert cb.cask_selftest_wait_timeout(run.ctx, limit, None, 0, check=False)[0] == cb.ERR_WORKSPACE
+    assert run.ctx.launches == n0
+    # the context and the device carry on: the same event, the same bytes, no flag
+    after = run.event()
+    assert run.ctx.device_flags() == 0
+    for k in before:
+        assert np.array_equal(before[k], after[k], equal_nan=True), k
+    o = gh.run_oracle(hb)
+    gh.compare_event(hb, after, o)
+    torch.cuda.synchronize()
+
+
 @pytest.mark.parametrize("extras", [0, 1, 2])
 def test_host_buffer_entry_point_matches_device_entry_point(extras):
     """cask_compress_event_host (host K/V/Q and host outputs; only the value rows that are read go up) gives the
