@@ -41,8 +41,6 @@ NCU_TRAFFIC = {
     "score_mass": (274.2, "profiles/score_tc_reasoning32k_16units.txt"),
     "assign": (264.9, "profiles/assign_tc_reasoning32k_16units.txt"),
 }
-# ex2 units: 16 results per clock per SM (special-function pipe), 148 SMs, 1.965 GHz maximum SM clock.
-EX2_PEAK_T_PER_S = 148 * 16 * 1.965e9 / 1e12
 
 
 def _peaks():
@@ -131,6 +129,162 @@ def algorithmic_bytes(hb: wl.Batch, n_out: np.ndarray, kind: np.ndarray) -> int:
             + 2 * int(n_out.sum()) * d * e + 8 * sum_T + 12 * int(hb.B.sum()))
 
 
+def sm_count(device) -> int:
+    import torch
+    return int(torch.cuda.get_device_properties(device).multi_processor_count)
+
+
+def ex2_peak(sms: int, clocks: dict) -> tuple:
+    """Roof of the exponential pipe in T exp/s: 16 results per clock per SM (special-function unit) x SMs x the
+    maximum SM clock nvidia-smi reports (1.965 GHz when it could not be read)."""
+    mhz = clocks.get("sm_max_mhz") or 1965.0
+    return sms * 16 * mhz * 1e6 / 1e12, "%d SMs x 16 ex2/clk x %.3f GHz" % (sms, mhz / 1e3)
+
+
+class Event:
+    """One workload resident on the device with everything a compression event needs."""
+
+    def __init__(self, w, units, args, device, local, similarity="cosine", shared=None, pinned=None):
+        import torch
+        from paper_2604_10900_b200 import binding as cb
+        self.cb, self.torch, self.w, self.device = cb, torch, w, device
+        t_gen = time.time()
+        if shared is not None:       # same rows as an earlier workload, other budget
+            hb0 = shared.hb
+            n = hb0.n_units
+            self.hb = hb = wl.Batch(wl=w, k=hb0.k, v=hb0.v, q=hb0.q, T=hb0.T, P=hb0.P, B=np.full(n, w.budget, np.int32),
+                                    reserve=np.full(n, w.reserve, np.int32), tok_off=hb0.tok_off, unit_ids=hb0.unit_ids,
+                                    mass_in=hb0.mass_in)
+            self.dev = shared.dev
+        else:
+            self.hb = hb = wl.make_batch(w, units, threads=min(16, os.cpu_count() or 8), pinned_alloc=pinned)
+            self.dev = cb.to_device(hb, device)
+        self.t_gen = time.time() - t_gen
+        self.sum_T = int(hb.tok_off[-1])
+        d, rows = w.head_dim, w.group * w.window
+        self.d, self.rows = d, rows
+        self.mass_dev = None if hb.mass_in is None else torch.from_numpy(hb.mass_in).to(device)
+        chan_host, band_host = similarity_weights(similarity, d)
+        self.sim_host = dict(chan_w=chan_host, band_w=band_host)
+        self.sim_dev = dict(chan_w=None if chan_host is None else torch.from_numpy(chan_host).to(device),
+                            band_w=None if band_host is None else torch.from_numpy(band_host).to(device))
+        self.batch, self._keep = cb.make_batch(self.dev["k"], self.dev["v"], self.dev["q"], hb.T, hb.P, hb.B, hb.reserve,
+                                               hb.tok_off, d, w.group, w.window, w.dtype, mass_in=self.mass_dev,
+                                               **self.sim_dev)
+        self.prm = cb.params(score_path=args.score_path)
+        self.stream = torch.cuda.current_stream(device)
+        self.ctx = cb.Context(local, self.stream.cuda_stream)
+        self.ws, self.ws_bytes = cb.alloc_workspace(self.batch, self.prm, device)
+        self.Bmax = int(hb.B.max())
+        self.out = cb.alloc_outputs(hb.n_units, self.sum_T, self.Bmax, d, rows, w.dtype, device, optional=False)
+        self.out["lse"] = torch.zeros((hb.n_units, rows), dtype=torch.float32, device=device)   # normalisers used
+        self.out_struct = cb.make_outputs(self.out, self.Bmax)
+
+    def step(self, batch=None):
+        self.cb.cask_compress_event(self.ctx, batch if batch is not None else self.batch, self.prm, self.out_struct,
+                                    self.ws, self.ws_bytes)
+
+    def time_steps(self, steps, barrier, batch=None):
+        """Times `steps` events back to back on the stream.  Returns (total ms over all steps, per-step ms list):
+        one CUDA event before the first step and one after every step, all on the launching stream, so the total
+        is the bracketed time of exactly `steps` steps and the list gives the median and the best."""
+        torch = self.torch
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        barrier()
+        evs[0].record(self.stream)
+        for i in range(steps):
+            self.step(batch)
+            evs[i + 1].record(self.stream)
+        barrier()
+        return evs[0].elapsed_time(evs[-1]), [evs[i].elapsed_time(evs[i + 1]) for i in range(steps)]
+
+    def kernel_split(self, steps):
+        """Per-kernel times from a loop of its own, with an event pair around every launch."""
+        self.ctx.profile_enable(True)
+        self.ctx.profile_read()
+        for _ in range(steps):
+            self.step()
+        self.torch.cuda.synchronize()
+        prof = self.ctx.profile_read()
+        self.ctx.profile_enable(False)
+        tot = max(sum(x["ms"] for x in prof.values()), 1e-9)
+        return {k: dict(ms_per_launch=v["ms"] / v["launches"], launches_per_step=v["launches"] / steps,
+                        share=v["ms"] / tot) for k, v in prof.items()}
+
+    def results(self):
+        return (self.out["n_out"].cpu().numpy(), self.out["kind"].cpu().numpy(), self.out["unit_status"].cpu().numpy())
+
+
+def event_roofline(hb, n_out, kind, ms_step, peaks, n_pass=2):
+    """The whole event against the HBM roof (algorithmic bytes of the event over its time) and against the composite
+    floor max(bytes / bandwidth, scoring flops / tensor peak)."""
+    w = hb.wl
+    rows, d, sum_T = w.group * w.window, w.head_dim, float(hb.T.sum())
+    ev_bytes = algorithmic_bytes(hb, n_out, kind)
+    flops_pass = 2.0 * rows * sum_T * d
+    t_hbm = ev_bytes / (peaks["hbm_gbs"] * 1e9)
+    t_tensor = n_pass * flops_pass / (peaks["bf16_tflops_sustained"] * 1e12)
+    gbs = ev_bytes / (ms_step * 1e-3) / 1e9
+    return dict(algorithmic_bytes=ev_bytes, gbs=gbs, hbm_frac_measured_peak=gbs / peaks["hbm_gbs"],
+                hbm_frac_nominal_8tbs=gbs / 8000.0, composite_floor_ms=max(t_hbm, t_tensor) * 1e3,
+                composite_frac=max(t_hbm, t_tensor) * 1e3 / ms_step)
+
+
+# The other configurations of the benchmark family, timed after the headline on one GPU: the 8k reasoning shape at
+# both budgets, the 32k shape at the other two budgets (same rows as the headline), the prompt-heavy two-stage shape
+# and its variant at the exhaustion boundary, one layer of the 64-sequence serving sweep, and the sweep's steady state.
+OTHER_WORKLOADS = ("reasoning32k_b384", "reasoning32k_b1024", "reasoning8k_b384", "reasoning8k_b512", "prompt_heavy",
+                   "prompt_heavy_boundary", "batched_serving", "serving_steady_b512")
+
+
+def other_workloads(args, device, local, peaks, headline: "Event"):
+    import torch
+    out = {}
+    steps = max(20, args.steps)
+
+    def barrier():
+        torch.cuda.synchronize()
+
+    for name in OTHER_WORKLOADS:
+        w = wl.WORKLOADS[name]
+        n_layers = w.layers
+        if name == "batched_serving":
+            n_layers = 1                      # one layer of every sequence: 512 ragged units
+        elif name == "serving_steady_b512":
+            n_layers = 12                     # a third of the layers of every sequence: 6,144 caches of 640 rows
+        units = wl.unit_list(w, layers=range(n_layers)) if w.n_seqs > 1 else None
+        shared = headline if (w.cfg_id == headline.w.cfg_id and w.n_seqs == 1 and w.prefix == headline.w.prefix
+                              and w.decode == headline.w.decode and not args.max_units) else None
+        ev = Event(w, units, args, device, local, shared=shared)
+        for _ in range(3):
+            ev.step()
+        barrier()
+        total, per = ev.time_steps(steps, barrier)
+        n_out, kind, status = ev.results()
+        kern = ev.kernel_split(5)
+        top = max(kern, key=lambda k: kern[k]["ms_per_launch"] * kern[k]["launches_per_step"])
+        med, best = float(np.median(per)), float(min(per))
+        hb = ev.hb
+        tokens = float(ev.sum_T)
+        rec = dict(units=hb.n_units, rows_per_unit=[int(hb.T.min()), int(hb.T.max())], budget=int(hb.B.max()),
+                   steps=steps, ms_per_step=total / steps, ms_per_step_median=med, ms_per_step_best=best,
+                   value=tokens / (total / steps * 1e-3), unit=UNIT, tokens_per_step=tokens,
+                   event_roofline=event_roofline(hb, n_out, kind, med, peaks), dominant_kernel=top,
+                   dominant_kernel_ms=kern[top]["ms_per_launch"] * kern[top]["launches_per_step"],
+                   kernels={k: round(v["ms_per_launch"] * v["launches_per_step"], 5) for k, v in kern.items()},
+                   score_path="tcgen05" if ev.ctx.used_tensor_path else "simt",
+                   status_bits_seen=int(np.bitwise_or.reduce(status)),
+                   l2="inputs larger than L2: %.2f GB of K/V read per step" % ((hb.k.nbytes + hb.v.nbytes) / 1e9))
+        if w.n_seqs > 1:
+            rec.update(sequences=w.n_seqs, layers_in_this_pass=n_layers, layers=w.layers,
+                       events_per_s=w.n_seqs * n_layers / w.layers / (med * 1e-3),
+                       events_per_s_note="one event = all layers of one sequence; this pass held layers_in_this_pass of them")
+        out[name] = rec
+        del ev
+        torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args):
     import torch
     from paper_2604_10900_b200 import binding as cb
@@ -159,32 +313,10 @@ def run_ours(args):
                         pin_memory=True)
         return t.numpy()
 
-    t_gen = time.time()
-    hb = wl.make_batch(w, units, threads=min(16, os.cpu_count() or 8), pinned_alloc=pinned)
-    t_gen = time.time() - t_gen
-    sum_T = int(hb.tok_off[-1])
-    d, rows = w.head_dim, w.group * w.window
-
-    dev = cb.to_device(hb, device)
-    mass_dev = None if hb.mass_in is None else torch.from_numpy(hb.mass_in).to(device)
-    # merge similarity (Sec. 2.5): plain cosine, or synthetic weights |kappa| that fall off with the band index
-    chan_host, band_host = similarity_weights(args.similarity, d)
-    sim_dev = dict(chan_w=None if chan_host is None else torch.from_numpy(chan_host).to(device),
-                   band_w=None if band_host is None else torch.from_numpy(band_host).to(device))
-    sim_host = dict(chan_w=chan_host, band_w=band_host)
-    batch, keep = cb.make_batch(dev["k"], dev["v"], dev["q"], hb.T, hb.P, hb.B, hb.reserve, hb.tok_off, d, w.group,
-                                w.window, w.dtype, mass_in=mass_dev, **sim_dev)
-    prm = cb.params(score_path=args.score_path)
-    stream = torch.cuda.current_stream(device)
-    ctx = cb.Context(local, stream.cuda_stream)
-    ws, ws_bytes = cb.alloc_workspace(batch, prm, device)
-    Bmax = int(hb.B.max())
-    out = cb.alloc_outputs(hb.n_units, sum_T, Bmax, d, rows, w.dtype, device, optional=False)
-    out["lse"] = torch.zeros((hb.n_units, rows), dtype=torch.float32, device=device)   # normalisers used
-    out_struct = cb.make_outputs(out, Bmax)
-
-    def step():
-        cb.cask_compress_event(ctx, batch, prm, out_struct, ws, ws_bytes)
+    ev = Event(w, units, args, device, local, similarity=args.similarity, pinned=pinned)
+    hb, ctx, stream = ev.hb, ev.ctx, ev.stream
+    sum_T, d, rows, Bmax = ev.sum_T, ev.d, ev.rows, ev.Bmax
+    t_gen = ev.t_gen
 
     def barrier():
         torch.cuda.synchronize()
@@ -193,48 +325,35 @@ def run_ours(args):
             dist.barrier()
             torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
-        step()
+    warm = max(args.warmup, 3)
+    for _ in range(warm):
+        ev.step()
     barrier()
-    n_out = out["n_out"].cpu().numpy()
-    kind = out["kind"].cpu().numpy()
-    status = out["unit_status"].cpu().numpy()
+    n_out, kind, status = ev.results()
     assert (n_out == np.minimum(hb.B, hb.T)).all() or (n_out <= hb.B).all()
 
+    # ---- the timed region: exactly `steps` events, no per-kernel events inside ----------------------------------
     sampler = ClockSampler(local)
     sampler.start()
     time.sleep(0.3)
-    ctx.profile_enable(True)
-    ctx.profile_read()
     l0 = ctx.launches
-    barrier()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0 = time.time()
-    ev0.record(stream)
-    for _ in range(args.steps):
-        step()
-    ev1.record(stream)
-    barrier()
+    ms_total, per_step = ev.time_steps(args.steps, barrier)
     t1 = time.time()
-    ms_total = ev0.elapsed_time(ev1)
     launches = ctx.launches - l0
-    prof = ctx.profile_read()
-    ctx.profile_enable(False)
     clocks = sampler.stop(t0, t1)
+    # per-kernel split: a second loop with an event pair around every launch
+    per_kernel = ev.kernel_split(min(args.steps, 10))
 
     # The same event when the caller hands over the window queries' softmax normalisers (a decode attention
     # kernel has them): the normaliser pass is skipped.  Reported beside the headline, never instead of it.
-    batch_l, keep_l = cb.make_batch(dev["k"], dev["v"], dev["q"], hb.T, hb.P, hb.B, hb.reserve, hb.tok_off, d, w.group,
-                                    w.window, w.dtype, lse_in=out["lse"].clone(), mass_in=mass_dev, **sim_dev)
-    cb.cask_compress_event(ctx, batch_l, prm, out_struct, ws, ws_bytes)
-    barrier()
-    ev0.record(stream)
-    for _ in range(args.steps):
-        cb.cask_compress_event(ctx, batch_l, prm, out_struct, ws, ws_bytes)
-    ev1.record(stream)
-    barrier()
-    ms_lse = ev0.elapsed_time(ev1) / args.steps
-    assert (out["n_out"].cpu().numpy() == n_out).all()
+    batch_l, keep_l = cb.make_batch(ev.dev["k"], ev.dev["v"], ev.dev["q"], hb.T, hb.P, hb.B, hb.reserve, hb.tok_off, d,
+                                    w.group, w.window, w.dtype, lse_in=ev.out["lse"].clone(), mass_in=ev.mass_dev,
+                                    **ev.sim_dev)
+    ev.step(batch_l)
+    ms_lse_total, _ = ev.time_steps(args.steps, barrier, batch_l)
+    ms_lse = ms_lse_total / args.steps
+    assert (ev.out["n_out"].cpu().numpy() == n_out).all()
 
     if world > 1:
         import torch.distributed as dist
@@ -249,14 +368,24 @@ def run_ours(args):
     ms_step = ms_total / args.steps
     value = total_tokens / (ms_step * 1e-3)
 
+    # what the special-function unit sustains on this GPU, measured by the library's own loop
+    ex2_rate = cb.cask_selftest_exp_rate(ctx, 4096, ev.ws, ev.ws_bytes) if ev.ws_bytes >= 16384 else None
+    peaks = _peaks()
+    others = None
+    if world == 1 and not args.no_other_workloads and args.workload == "reasoning32k_b512" and \
+            args.similarity == "cosine" and not args.max_units:
+        others = other_workloads(args, device, local, peaks, ev)
+
     # ---- end to end through the host-buffer entry point ---------------------------------------
+    prm = ev.prm
     hbatch, hkeep = cb.make_batch(hb.k, hb.v, hb.q, hb.T, hb.P, hb.B, hb.reserve, hb.tok_off, d, w.group, w.window,
-                                  w.dtype, mass_in=hb.mass_in, **sim_host)
+                                  w.dtype, mass_in=hb.mass_in, **ev.sim_host)
     dev_bytes = cb.cask_host_event_device_bytes(hbatch, prm, Bmax)
-    del dev, out, out_struct, ws
+    ctx_tensor_path = ctx.used_tensor_path
+    ev.dev = ev.out = ev.out_struct = ev.ws = ev.batch = None
+    del batch_l, keep_l
     torch.cuda.empty_cache()
     dev_buf = torch.empty(dev_bytes, dtype=torch.uint8, device=device)
-    e = 2 if w.dtype == wl.DTYPE_BF16 else 4
     st = np.uint16 if w.dtype == wl.DTYPE_BF16 else np.float32
     # every result lands in pinned memory: a copy into pageable memory would hold the host until it is done
     ho = dict(k_out=pinned((hb.n_units, Bmax, d), st), v_out=pinned((hb.n_units, Bmax, d), st),
@@ -274,9 +403,10 @@ def run_ours(args):
     h2d = hb.k.nbytes + hb.q.nbytes + int(np.count_nonzero(kind)) * d * (2 if w.dtype == wl.DTYPE_BF16 else 4) \
         + (0 if hb.mass_in is None else hb.mass_in.nbytes)
     d2h = sum(a.nbytes for a in ho.values()) + sum_T
-    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    e2e_steps = max(1, args.e2e_steps)
     cb.cask_compress_event_host(ctx, hbatch, prm, ho_struct, dev_buf, dev_bytes)   # warm-up
     barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record(stream)
     for _ in range(e2e_steps):
         cb.cask_compress_event_host(ctx, hbatch, prm, ho_struct, dev_buf, dev_bytes)
@@ -298,22 +428,20 @@ def run_ours(args):
         return
 
     # ---- roofline of the dominant kernel -------------------------------------------------------
-    ctx_tensor_path = ctx.used_tensor_path
-    peaks = _peaks()
-    per_kernel = {k: dict(ms_per_launch=v["ms"] / v["launches"], launches_per_step=v["launches"] / args.steps,
-                          share=v["ms"] / max(sum(x["ms"] for x in prof.values()), 1e-9)) for k, v in prof.items()}
-    top = max(prof, key=lambda k: prof[k]["ms"])
-    top_ms = prof[top]["ms"] / prof[top]["launches"]
+    top = max(per_kernel, key=lambda k: per_kernel[k]["ms_per_launch"] * per_kernel[k]["launches_per_step"])
+    top_ms = per_kernel[top]["ms_per_launch"]
     flops_pass = 2.0 * rows * float(sum_T) * d        # one Q_w K^T contraction over every unit
     tensor_roof = None
     if top in ("score_norm", "score_mass"):
         # One exponential per (query row, key): the pass is bound by the ex2 pipe, not by the contraction that
-        # feeds it (profiles/score_tc_*: ex2 pipe 65-72 % busy, tensor pipe 37-40 %, DRAM 17 %).
+        # feeds it (profiles/score_tc_*: ex2 pipe the busiest unit, tensor pipe about 40 %, DRAM under 20 %).
         exps = float(rows) * float(sum_T)
         achieved = exps / (top_ms * 1e-3) / 1e12
-        roof = dict(kernel=top, bound="alu", achieved=achieved, peak=EX2_PEAK_T_PER_S, unit="Texp/s",
-                    frac=achieved / EX2_PEAK_T_PER_S, traffic=None,
-                    peak_source="148 SMs x 16 ex2/clk x 1.965 GHz", ms_per_launch=top_ms, exps_per_launch=exps)
+        peak, peak_src = ex2_peak(sm_count(device), clocks)
+        roof = dict(kernel=top, bound="alu", achieved=achieved, peak=peak, unit="Texp/s", frac=achieved / peak,
+                    traffic=None, peak_source=peak_src, ms_per_launch=top_ms, exps_per_launch=exps,
+                    ex2_per_clk_per_sm_measured=ex2_rate,
+                    ex2_measured_note="cask_selftest_exp_rate: FFMA + ex2 + FADD + FMUL loop, 16 warps per SM, median over SMs")
         t_ach = flops_pass / (top_ms * 1e-3) / 1e12
         tensor_roof = dict(kernel=top, bound="tensor", achieved=t_ach, peak=peaks["bf16_tflops_sustained"],
                            unit="TFLOP/s", frac=t_ach / peaks["bf16_tflops_sustained"],
@@ -326,15 +454,7 @@ def run_ours(args):
     if top in NCU_TRAFFIC and ctx_tensor_path:
         roof["traffic"] = NCU_TRAFFIC[top][0] * float(sum_T)
         roof["traffic_source"] = NCU_TRAFFIC[top][1] + " (bytes per cache row x rows of this launch)"
-    ev_bytes = algorithmic_bytes(hb, n_out, kind)
-    t_hbm = ev_bytes / (peaks["hbm_gbs"] * 1e9)
-    n_pass = 2          # normaliser pass + score pass (no caller-supplied normalisers here)
-    t_tensor = n_pass * flops_pass / (peaks["bf16_tflops_sustained"] * 1e12)
-    event = dict(algorithmic_bytes=ev_bytes, gbs=ev_bytes / (ms_step * 1e-3) / 1e9,
-                 hbm_frac_measured_peak=ev_bytes / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                 hbm_frac_nominal_8tbs=ev_bytes / (ms_step * 1e-3) / 1e9 / 8000.0,
-                 composite_floor_ms=max(t_hbm, t_tensor) * 1e3,
-                 composite_frac=max(t_hbm, t_tensor) * 1e3 / ms_step)
+    event = event_roofline(hb, n_out, kind, ms_step, peaks)
 
     # ---- the oracle on this machine's host cores, bounded sample ------------------------------------
     cpu = None
@@ -342,15 +462,19 @@ def run_ours(args):
         cpu = cpu_baseline(w, args.cpu_units, args.similarity)
 
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-        "ms_per_step": ms_step, "higher_is_better": True,
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
+        "ms_per_step": ms_step, "ms_per_step_median": float(np.median(per_step)), "ms_per_step_best": float(min(per_step)),
+        "higher_is_better": True,
         "scaling": "weak" if w.n_seqs == 1 else "strong", "vs_baseline": None, "dtype": "bf16" if w.dtype == wl.DTYPE_BF16 else "f32",
         "data": "synthetic",
         "config": {"workload": w.name, "units_per_gpu": hb.n_units, "rows_per_unit": int(hb.T.max()), "head_dim": d,
                    "query_rows": rows, "budget": int(hb.B.max()), "tokens_per_step": total_tokens,
                    "l2": "inputs larger than L2: %.2f GB of K/V read per step" % ((hb.k.nbytes + hb.v.nbytes) / 1e9),
-                   "score_path": "tcgen05" if ctx.used_tensor_path else "simt", "gen_seconds": round(t_gen, 1),
+                   "score_path": "tcgen05" if ctx_tensor_path else "simt", "gen_seconds": round(t_gen, 1),
                    "reduced": bool(args.max_units),
+                   "timing": "CUDA events on the launching stream: one bracket around all steps (value, ms_per_step), "
+                             "one event after every step (median, best, this rank); per-kernel event pairs only in a "
+                             "separate loop (kernels)",
                    **({"sequences": w.n_seqs, "layers_per_pass": n_layers, "layers": w.layers,
                        "events_per_s": w.n_seqs * n_layers / w.layers / (ms_step * 1e-3),
                        "events_per_s_note": "one event = all layers of one sequence; this pass held layers_per_pass of them"}
@@ -361,6 +485,7 @@ def run_ours(args):
         "with_supplied_normalisers": {"ms_per_step": ms_lse, "value": total_tokens / (ms_lse * 1e-3), "unit": UNIT,
                                       "note": "lse_in given by the caller: one scoring pass instead of two (this rank)"},
         "roofline": roof, "tensor_roofline": tensor_roof, "event_roofline": event, "kernels": per_kernel,
+        "other_workloads": others,
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                 "ms_per_step": e2e_ms, "steps": e2e_steps},
@@ -504,12 +629,14 @@ def run_stats_scorer(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="reasoning32k_b512", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--score-path", type=int, default=0, help="0: tensor-core scoring when the shape allows, 1: SIMT")
-    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-other-workloads", action="store_true",
+                    help="skip the block of the other benchmark configurations timed after the headline (N = 1 only)")
     ap.add_argument("--scorer", default="attention", choices=["attention", "stats", "stats_offsets"],
                     help="attention: the whole event with the windowed attention-mass score (default); "
                          "stats: time the query-statistics scorer of App. B alone")
