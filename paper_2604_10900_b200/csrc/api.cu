@@ -573,9 +573,9 @@ static int event_decide(cask_ctx* ctx, Launch& L, Workspace& W, const cask_batch
 // The rest: compaction (the only step that reads values) and the optional diagnostics.
 static int event_compact(cask_ctx* ctx, Launch& L, Workspace& W, const cask_params* p, const cask_outputs* out) {
     float* s = out->s ? out->s : W.s;
-    cudaError_t e = launch_compact(L, *p, s, out->kind, out->seed_of, out->weight, *out, W);
+    const EventFusion ev{out->plan, out->unit_status, out->lost_mass};
+    cudaError_t e = launch_compact(L, *p, s, out->kind, out->seed_of, out->weight, *out, W, &ev);
     if (e == cudaSuccess) e = launch_diagnostics(L, *p, s, out->kind, *out);
-    if (e == cudaSuccess) e = launch_status_flags(L, W.err, out->unit_status);
     return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
 }
 

@@ -136,8 +136,17 @@ cudaError_t launch_consolidate(const Launch& L, const cask_params& prm, const fl
 // fused (the event path only): `plan` and `kind` are still unwritten; one kernel per unit then does the prefix eviction
 // and the core and seed selection, and for units of at most kSmallUnitRows rows the seed gather as well.
 constexpr int kSmallUnitRows = 1024;
+// ev != nullptr (the event path, after launch_consolidate(..., fused = true)): the ordered scan of the compaction also
+// writes the merge weights, the status words and the lost mass, which the fused consolidation left out, and the merge
+// kernel, the last of the event, ORs late device flags into the status words.
+struct EventFusion {
+    const int32_t* plan;
+    int32_t* unit_status;
+    float* lost_mass;
+};
 cudaError_t launch_compact(const Launch& L, const cask_params& prm, const float* s, const uint8_t* kind,
-                           const int32_t* seed_of, float* weight, const cask_outputs& out, Workspace& ws);
+                           const int32_t* seed_of, float* weight, const cask_outputs& out, Workspace& ws,
+                           const EventFusion* ev = nullptr);
 // Host-resident caches: rank of every row among the rows of its unit whose values the compaction reads
 // (kind != 0), the number of such rows per unit and the exclusive prefix of those numbers.
 cudaError_t launch_value_ranks(const Launch& L, const uint8_t* kind, int32_t* v_pos, int32_t* n_need, int64_t* v_base);
@@ -146,10 +155,6 @@ cudaError_t launch_writeback(const Launch& L, const cask_outputs& out, void* k_p
 // rho_core / rho_rep and the within-group dispersion of Sec. 2.6 per unit (any of the pointers may be NULL).
 cudaError_t launch_diagnostics(const Launch& L, const cask_params& prm, const float* s, const uint8_t* kind,
                                const cask_outputs& out);
-
-// Last kernel of an event: the device flags of the call (ws.err) are ORed into every unit's status word once more,
-// so that flags raised by the compaction kernels are not missed by a caller that reads unit_status alone.
-cudaError_t launch_status_flags(const Launch& L, const int32_t* err, int32_t* unit_status);
 
 // Tensor-core assignment of scratch rows to seeds (cosine Gram + argmax), same outputs as the SIMT kernel.
 bool assign_tc_supported(const Launch& L);

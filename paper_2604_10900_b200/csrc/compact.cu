@@ -7,6 +7,23 @@ namespace cask {
 
 namespace {
 
+// On the event path the scan also does what weights_kernel does in the staged consolidation call (merge weights
+// w_i = a_i / m_G of the rows of kind 4/5, the unit's status word and lost mass): same formulas, same bits, one
+// launch fewer.  s == nullptr: not fused, the weights are already there.
+struct FusedWeights {
+    const float* s;
+    const int32_t* grp;
+    const unsigned long long* mass_fx;
+    const int32_t* njoin;
+    const int32_t* plan;
+    int32_t* unit_status;
+    float* lost_mass;
+    const int32_t* err;
+    Shape sh;
+    int max_m;
+    float eps;
+};
+
 constexpr int kScanThreads = 1024;
 constexpr int kScanMaxIters = 63;      // rows per unit below 64,512: the one-scan path of slot_scan_kernel
 
@@ -16,7 +33,7 @@ __global__ void __launch_bounds__(kScanThreads) slot_scan_kernel(
     float* __restrict__ weight, int Bmax, int32_t* __restrict__ n_out, int32_t* __restrict__ slot_src,
     uint8_t* __restrict__ slot_kind, float* __restrict__ slot_mass, int32_t* __restrict__ assign,
     int32_t* __restrict__ mem_row, int32_t* __restrict__ mem_slot, int32_t* __restrict__ n_mem,
-    int32_t* __restrict__ seed_slot, int32_t* __restrict__ n_seed, int max_B) {
+    int32_t* __restrict__ seed_slot, int32_t* __restrict__ n_seed, int max_B, FusedWeights fw) {
     __shared__ unsigned wk[kScanThreads / 32], wm[kScanThreads / 32];
     __shared__ unsigned cell[kScanMaxIters * (kScanThreads / 32)];
     __shared__ int seeds_listed;
@@ -96,6 +113,12 @@ __global__ void __launch_bounds__(kScanThreads) slot_scan_kernel(
                 if (mem) mem_row[o + (cb >> 16) + __popc(bm & below)] = i;
                 if (kd >= CASK_KIND_PREFIX && kd <= CASK_KIND_CORE) weight[o + i] = 1.f;
                 if (kd == CASK_KIND_DROPPED) weight[o + i] = 0.f;
+                if (fw.s && mem) {
+                    const int gi = fw.grp[o + i];
+                    if (gi >= 0 && gi < fw.max_m)
+                        weight[o + i] = row_mass(fw.sh, fw.s, fw.eps, o + i) /
+                                        fx_to_mass(fw.mass_fx[(size_t)u * (fw.max_m + 1) + gi]);
+                }
             }
         }
     } else {
@@ -130,6 +153,12 @@ __global__ void __launch_bounds__(kScanThreads) slot_scan_kernel(
                 if (mem) mem_row[o + base_m + pm + __popc(bm & below)] = i;
                 if (kd >= CASK_KIND_PREFIX && kd <= CASK_KIND_CORE) weight[o + i] = 1.f;
                 if (kd == CASK_KIND_DROPPED) weight[o + i] = 0.f;
+                if (fw.s && mem) {
+                    const int gi = fw.grp[o + i];
+                    if (gi >= 0 && gi < fw.max_m)
+                        weight[o + i] = row_mass(fw.sh, fw.s, fw.eps, o + i) /
+                                        fx_to_mass(fw.mass_fx[(size_t)u * (fw.max_m + 1) + gi]);
+                }
             }
             base_k += ak;
             base_m += am;
@@ -137,6 +166,12 @@ __global__ void __launch_bounds__(kScanThreads) slot_scan_kernel(
     }
     const int nk = min((int)base_k, Bmax), nm = (int)base_m;
     if (threadIdx.x == 0) { n_out[u] = nk; n_mem[u] = nm; }
+    if (fw.s && threadIdx.x == 0) {
+        int fl = fw.plan[u * 8 + CASK_PLAN_FLAGS];
+        if ((fl & CASK_ST_DECODE_CONSOLIDATED) && fw.njoin[u] == 0) fl |= CASK_ST_MERGE_INACTIVE;
+        fw.unit_status[u] = fl | *fw.err;     // device-side flags of this call so far
+        fw.lost_mass[u] = fx_to_mass(fw.mass_fx[(size_t)u * (fw.max_m + 1) + fw.max_m]);
+    }
     for (int t = nk + threadIdx.x; t < Bmax; t += blockDim.x) {
         slot_src[(size_t)u * Bmax + t] = -1;
         slot_kind[(size_t)u * Bmax + t] = 0;
@@ -251,18 +286,23 @@ __global__ void __launch_bounds__(kCopyWarps * 32) slot_copy_kernel(
 }
 
 // ---- 3. one warp per representative with joiners: ordered weighted merge over its copy -----
-template <typename T>
+// CH > 0: head_dim == 32 * CH, every lane owns CH contiguous channels and reads them with one vector load per row;
+// CH == 0: any head_dim up to 256, channels lane, lane + 32, ...  The sums per channel are the same either way.
+template <typename T, int CH>
 __global__ void __launch_bounds__(256) slot_merge_kernel(
     const UnitDesc* __restrict__ desc, Shape sh, const T* __restrict__ K, const T* __restrict__ V,
     const float* __restrict__ s, const float* __restrict__ weight, float eps, int Bmax,
     const int32_t* __restrict__ seed_slot, const int32_t* __restrict__ n_seed, int max_B,
     const int32_t* __restrict__ mem_row, const int32_t* __restrict__ mem_slot,
     const int32_t* __restrict__ n_mem, T* __restrict__ k_out, T* __restrict__ v_out,
-    float* __restrict__ slot_mass) {
+    float* __restrict__ slot_mass, int32_t* __restrict__ unit_status) {
     const int u = blockIdx.y;
     const UnitDesc& ud = desc[u];
     const int lane = threadIdx.x & 31;
     const int j = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    // Last kernel of an event: flags raised on the device since the status words were written (a bulk copy of the
+    // compaction that gave up) join them.  A page id outside the pool was already met by the scoring pass.
+    if (unit_status && blockIdx.x == 0 && threadIdx.x == 0 && *sh.err) unit_status[u] |= *sh.err;
     if (j >= n_seed[u]) return;
     const int t = seed_slot[(size_t)u * max_B + j];
     const int d = sh.d;
@@ -274,37 +314,83 @@ __global__ void __launch_bounds__(256) slot_merge_kernel(
     int count = 0;
     float msum = 0.f;
     const int nm = n_mem[u];
-    for (int e0 = 0; e0 < nm; e0 += 32) {
-        const int e = e0 + lane;
-        const int row = (e < nm) ? mem_row[o + e] : -1;
-        const bool hit = (e < nm) && mem_slot[o + e] == t;
-        unsigned bal = __ballot_sync(0xffffffffu, hit);
-        while (bal) {
-            const int l = __ffs(bal) - 1;
-            bal &= bal - 1;
-            const int i = __shfl_sync(0xffffffffu, row, l);
-            const float wi = weight[o + i];
-            msum += row_mass(sh, s, eps, o + i);
-            ++count;
-            const T* kr = K + row_elem_off(sh, ud, ud.k_off, i);
-            const T* vr = V + v_elem_off(sh, ud, u, i);
+    // The member list of the unit is walked 128 entries at a time (the eight index loads of a round are independent)
+    // and the round's own members are listed in shared memory in ascending order; their rows are then read four at a
+    // time, so the latency of a row is paid once per four members and not once per member, and added in list order.
+    constexpr int kWalk = 4;
+    __shared__ int32_t hits[8][32 * kWalk];
+    int32_t* my_hits = hits[threadIdx.x >> 5];
+    const unsigned below = (1u << lane) - 1u;
+    for (int e0 = 0; e0 < nm; e0 += 32 * kWalk) {
+        int row[kWalk];
+        bool hit[kWalk];
 #pragma unroll
-            for (int x = 0; x < kMaxPerLane; ++x) {
-                const int c = lane + 32 * x;
-                if (c < d) {
-                    ak[x] = fmaf(wi, Elem<T>::ld(kr + c), ak[x]);
-                    av[x] = fmaf(wi, Elem<T>::ld(vr + c), av[x]);
+        for (int q = 0; q < kWalk; ++q) {
+            const int e = e0 + 32 * q + lane;
+            row[q] = (e < nm) ? mem_row[o + e] : -1;
+            hit[q] = (e < nm) && mem_slot[o + e] == t;
+        }
+        int n_hits = 0;
+#pragma unroll
+        for (int q = 0; q < kWalk; ++q) {
+            const unsigned bal = __ballot_sync(0xffffffffu, hit[q]);
+            if (hit[q]) my_hits[n_hits + __popc(bal & below)] = row[q];
+            n_hits += __popc(bal);
+        }
+        __syncwarp();
+        constexpr int kRows = 4;           // member rows in flight per warp
+        for (int h0 = 0; h0 < n_hits; h0 += kRows) {
+            if (CH > 0) {
+                struct alignas((CH > 0 ? CH : 1) * sizeof(T)) Vec { T x[CH > 0 ? CH : 1]; };
+                Vec kv[kRows], vv[kRows];
+                float wi[kRows], ai[kRows];
+#pragma unroll
+                for (int q = 0; q < kRows; ++q) {
+                    const int i = my_hits[min(h0 + q, n_hits - 1)];
+                    wi[q] = weight[o + i];
+                    ai[q] = row_mass(sh, s, eps, o + i);
+                    kv[q] = reinterpret_cast<const Vec*>(K + row_elem_off(sh, ud, ud.k_off, i))[lane];
+                    vv[q] = reinterpret_cast<const Vec*>(V + v_elem_off(sh, ud, u, i))[lane];
+                }
+#pragma unroll
+                for (int q = 0; q < kRows; ++q) {
+                    if (h0 + q >= n_hits) break;
+                    msum += ai[q];
+                    ++count;
+#pragma unroll
+                    for (int x = 0; x < CH; ++x) {
+                        ak[x] = fmaf(wi[q], Elem<T>::ld(&kv[q].x[x]), ak[x]);
+                        av[x] = fmaf(wi[q], Elem<T>::ld(&vv[q].x[x]), av[x]);
+                    }
+                }
+            } else {
+                for (int q = 0; q < kRows && h0 + q < n_hits; ++q) {
+                    const int i = my_hits[h0 + q];
+                    const float wq = weight[o + i];
+                    msum += row_mass(sh, s, eps, o + i);
+                    ++count;
+                    const T* kr = K + row_elem_off(sh, ud, ud.k_off, i);
+                    const T* vr = V + v_elem_off(sh, ud, u, i);
+#pragma unroll
+                    for (int x = 0; x < kMaxPerLane; ++x) {
+                        const int c = lane + 32 * x;
+                        if (c < d) {
+                            ak[x] = fmaf(wq, Elem<T>::ld(kr + c), ak[x]);
+                            av[x] = fmaf(wq, Elem<T>::ld(vr + c), av[x]);
+                        }
+                    }
                 }
             }
         }
+        __syncwarp();
     }
     if (count > 1) {       // a lone seed keeps its byte copy
         T* ko = k_out + ((size_t)u * Bmax + t) * d;
         T* vo = v_out + ((size_t)u * Bmax + t) * d;
 #pragma unroll
         for (int x = 0; x < kMaxPerLane; ++x) {
-            const int c = lane + 32 * x;
-            if (c < d) {
+            const int c = CH > 0 ? lane * CH + x : lane + 32 * x;
+            if ((CH > 0 && x < CH) || (CH == 0 && c < d)) {
                 Elem<T>::st(ko + c, ak[x]);
                 Elem<T>::st(vo + c, av[x]);
             }
@@ -327,7 +413,7 @@ __global__ void __launch_bounds__(256, 4) slot_merge_small_kernel(
     const int32_t* __restrict__ seed_slot, const int32_t* __restrict__ n_seed, int max_B,
     const int32_t* __restrict__ mem_row, const int32_t* __restrict__ mem_slot,
     const int32_t* __restrict__ n_mem, T* __restrict__ k_out, T* __restrict__ v_out,
-    float* __restrict__ slot_mass) {
+    float* __restrict__ slot_mass, int32_t* __restrict__ unit_status) {
     constexpr int R = kMergeStageRows;
     __shared__ int32_t m_row[R], list[R], s_slot[R], start[R + 1], fill[R];
     __shared__ int16_t m_j[R], inv[R];
@@ -339,6 +425,7 @@ __global__ void __launch_bounds__(256, 4) slot_merge_small_kernel(
     const int64_t o = ud.tok_off;
     const int nm = min(n_mem[u], R);
     const int ns = min(n_seed[u], R);
+    if (unit_status && tid == 0 && *sh.err) unit_status[u] |= *sh.err;      // see slot_merge_kernel
     for (int t = tid; t < R; t += blockDim.x) { inv[t] = -1; fill[t] = 0; }
     __syncthreads();
     for (int j = tid; j < ns; j += blockDim.x) {
@@ -519,15 +606,18 @@ __global__ void __launch_bounds__(256) writeback_kernel(const UnitDesc* __restri
 
 template <typename T>
 cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const uint8_t* kind,
-                const int32_t* seed_of, float* weight, const cask_outputs& out, Workspace& ws) {
+                const int32_t* seed_of, float* weight, const cask_outputs& out, Workspace& ws, const EventFusion* ev) {
     const Shape& sh = L.sh;
+    FusedWeights fw{};
+    if (ev) fw = FusedWeights{s, ws.grp, ws.mass_fx, ws.njoin, ev->plan, ev->unit_status, ev->lost_mass, ws.err, sh, L.max_m, prm.eps};
+    int32_t* const status = ev ? ev->unit_status : nullptr;
     {
         Timed t(L, KID_SLOT_SCAN);
         slot_scan_kernel<<<sh.n_units, L.max_T <= 2048 ? 256 : kScanThreads, 0, L.stream>>>(L.desc, kind, seed_of, weight, out.Bmax,
                                                                     out.n_out, out.slot_src, out.slot_kind,
                                                                     out.slot_mass, out.assign, ws.mem_row,
                                                                     ws.mem_slot, ws.n_mem, ws.seed_slot, ws.n_seed,
-                                                                    ws.max_B);
+                                                                    ws.max_B, fw);
     }
     const int slots = min(out.Bmax, max(L.max_B, 1));
     {
@@ -547,11 +637,15 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const u
             auto kern = sh.d == 128 ? slot_merge_small_kernel<T, 4> : slot_merge_small_kernel<T, 2>;
             kern<<<sh.n_units, 256, 0, L.stream>>>(
                 L.desc, sh, (const T*)L.k, (const T*)L.v, s, weight, prm.eps, out.Bmax, ws.seed_slot, ws.n_seed,
-                ws.max_B, ws.mem_row, ws.mem_slot, ws.n_mem, (T*)out.k_out, (T*)out.v_out, out.slot_mass);
+                ws.max_B, ws.mem_row, ws.mem_slot, ws.n_mem, (T*)out.k_out, (T*)out.v_out, out.slot_mass, status);
         } else {
-            slot_merge_kernel<T><<<dim3((std::min(slots, ws.max_B) + 7) / 8, sh.n_units), 256, 0, L.stream>>>(
+            auto mk = sh.d == 128 ? slot_merge_kernel<T, 4> : sh.d == 64 ? slot_merge_kernel<T, 2> : slot_merge_kernel<T, 0>;
+            // one warp per representative: on the event path no unit has more than max_m of them (the plan's count);
+            // a staged call may be handed any kinds, so there the slot count bounds them
+            const int reps = ev ? std::max(L.max_m, 1) : std::min(slots, ws.max_B);
+            mk<<<dim3((reps + 7) / 8, sh.n_units), 256, 0, L.stream>>>(
                 L.desc, sh, (const T*)L.k, (const T*)L.v, s, weight, prm.eps, out.Bmax, ws.seed_slot, ws.n_seed,
-                ws.max_B, ws.mem_row, ws.mem_slot, ws.n_mem, (T*)out.k_out, (T*)out.v_out, out.slot_mass);
+                ws.max_B, ws.mem_row, ws.mem_slot, ws.n_mem, (T*)out.k_out, (T*)out.v_out, out.slot_mass, status);
         }
         ++*L.launches;
     }
@@ -584,9 +678,10 @@ cudaError_t launch_writeback(const Launch& L, const cask_outputs& out, void* k_p
 }
 
 cudaError_t launch_compact(const Launch& L, const cask_params& prm, const float* s, const uint8_t* kind,
-                           const int32_t* seed_of, float* weight, const cask_outputs& out, Workspace& ws) {
-    if (L.sh.dtype == CASK_DTYPE_BF16) return run<__nv_bfloat16>(L, prm, s, kind, seed_of, weight, out, ws);
-    return run<float>(L, prm, s, kind, seed_of, weight, out, ws);
+                           const int32_t* seed_of, float* weight, const cask_outputs& out, Workspace& ws,
+                           const EventFusion* ev) {
+    if (L.sh.dtype == CASK_DTYPE_BF16) return run<__nv_bfloat16>(L, prm, s, kind, seed_of, weight, out, ws, ev);
+    return run<float>(L, prm, s, kind, seed_of, weight, out, ws, ev);
 }
 
 }  // namespace cask

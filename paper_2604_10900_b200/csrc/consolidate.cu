@@ -633,7 +633,7 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const i
             sim, ws.grp, ws.mass_fx, ws.njoin, max_m, prm.tau, prm.eps);
         }
     }
-    {
+    if (!fused) {      // the event path leaves the weights, the status words and the lost mass to the compaction's scan
         Timed t(L, KID_WEIGHTS);
         weights_kernel<<<dim3((L.max_T + 256 * kWeightRows - 1) / (256 * kWeightRows), sh.n_units), 256, 0, L.stream>>>(
             L.desc, sh, s, plan, ws.grp, ws.mass_fx, ws.njoin, weight, unit_status, lost_mass, max_m, prm.eps, ws.err);

@@ -126,21 +126,7 @@ __global__ void __launch_bounds__(256) dispersion_kernel(
     }
 }
 
-// Flags raised on the device after the merge weights were written (a bulk copy of the compaction that gave up, a
-// page id outside the pool met only there) join every unit's status word.
-__global__ void status_flags_kernel(int n_units, const int32_t* __restrict__ err, int32_t* __restrict__ unit_status) {
-    const int u = blockIdx.x * blockDim.x + threadIdx.x;
-    const int32_t f = *err;
-    if (u < n_units && f) unit_status[u] |= f;
-}
-
 }  // namespace
-
-cudaError_t launch_status_flags(const Launch& L, const int32_t* err, int32_t* unit_status) {
-    Timed t(L, KID_DIAGNOSTICS);
-    status_flags_kernel<<<(L.sh.n_units + 255) / 256, 256, 0, L.stream>>>(L.sh.n_units, err, unit_status);
-    return cudaGetLastError();
-}
 
 cudaError_t launch_diagnostics(const Launch& L, const cask_params& prm, const float* s, const uint8_t* kind,
                                const cask_outputs& out) {
