@@ -210,6 +210,16 @@ int cask_last_score_path_tensor(const cask_ctx* ctx);
 int cask_last_device_flags(cask_ctx* ctx, int32_t* flags_host);
 
 /*
+ * SM clock, in kHz, at which the two tensor-core scoring passes of the context's last cask_score /
+ * cask_compress_event ran (no counterpart in the paper): one CTA of each pass divides the SM cycles it
+ * spent by the wall time they took.  khz_host: HOST, two words (normaliser pass, score pass; 0 for a
+ * pass that did not run, both 0 after a call that used the SIMT kernels or the host-buffer entry point).
+ * A pass that keeps the exponential, FMA and tensor pipes busy together runs under the board's power
+ * limit, below the maximum clock; its rate per clock is judged against this figure.  Waits for the stream.
+ */
+int cask_last_score_clock_khz(cask_ctx* ctx, int32_t* khz_host);
+
+/*
  * Self-test of the bounded device waits (no counterpart in the paper).  Every wait of the kernels on a
  * hardware barrier gives up after a wall-time limit and makes the kernel end with CASK_ST_TIMEOUT
  * instead of hanging; in a healthy run that path never executes.  This call runs it once: one small

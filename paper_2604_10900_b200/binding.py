@@ -32,7 +32,7 @@ EXPORTS = (
     "cask_kernel_count", "cask_kernel_name", "cask_workspace_bytes", "cask_plan_host",
     "cask_score", "cask_score_stats", "cask_prefix_evict", "cask_select_core", "cask_consolidate_scratch", "cask_compact",
     "cask_compress_event", "cask_writeback_paged", "cask_host_event_device_bytes", "cask_compress_event_host", "cask_score_noalloc",
-    "cask_selftest_wait_timeout", "cask_selftest_exp_rate",
+    "cask_selftest_wait_timeout", "cask_selftest_exp_rate", "cask_last_score_clock_khz",
 )
 
 
@@ -120,6 +120,7 @@ def lib():
         L.cask_score_noalloc.argtypes = [i32, vp, PB, PP, vp, vp]
         L.cask_selftest_wait_timeout.argtypes = [vp, C.c_uint64, vp, sz, vp, vp]
         L.cask_selftest_exp_rate.argtypes = [vp, C.c_int32, vp, sz, vp]
+        L.cask_last_score_clock_khz.argtypes = [vp, vp]
         _lib = L
     return _lib
 
@@ -249,6 +250,14 @@ class Context:
     @property
     def used_tensor_path(self) -> bool:
         return bool(lib().cask_last_score_path_tensor(self.handle))
+
+    def score_clock_mhz(self):
+        """(normaliser pass, score pass) SM clock in MHz of the last tensor-core scoring call (0: did not run)."""
+        khz = (C.c_int32 * 2)(0, 0)
+        rc = lib().cask_last_score_clock_khz(self.handle, C.addressof(khz))
+        if rc != OK:
+            raise CaskError(rc, self.handle)
+        return khz[0] / 1e3, khz[1] / 1e3
 
     def device_flags(self) -> int:
         """CASK_ST_* bits raised on the device by the last call (waits for the stream)."""

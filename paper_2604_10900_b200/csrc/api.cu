@@ -322,6 +322,7 @@ int selftest_set_flags_source(cask_ctx* ctx, const int32_t* flags_dev, int n_lau
     if (!ctx) return CASK_ERR_NULL;
     ctx->flags_dev = flags_dev;
     ctx->flags_last = 0;
+    ctx->last_tc = 0;
     ctx->launches += n_launches;
     *stream = ctx->stream;
     *device = ctx->device;
@@ -437,6 +438,17 @@ int cask_profile_read(cask_ctx* ctx, float* ms, int64_t* launches) {
     return CASK_OK;
 }
 int cask_last_score_path_tensor(const cask_ctx* ctx) { return ctx ? ctx->last_tc : 0; }
+
+int cask_last_score_clock_khz(cask_ctx* ctx, int32_t* khz_host) {
+    if (!ctx || !khz_host) return CASK_ERR_NULL;
+    khz_host[0] = khz_host[1] = 0;
+    if (!ctx->flags_dev || !ctx->last_tc) return CASK_OK;
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(khz_host, ctx->flags_dev + 2, 2 * sizeof(int32_t), cudaMemcpyDeviceToHost, ctx->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+    return e == cudaSuccess ? CASK_OK : fail_cuda(ctx, e);
+}
 
 int cask_last_device_flags(cask_ctx* ctx, int32_t* flags_host) {
     if (!ctx || !flags_host) return CASK_ERR_NULL;

@@ -296,6 +296,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 
     TileWalk wk;
     wk.init(desc, sh.n_units, total_tiles);
+    // CTA 0 reports the SM clock it ran at (cycles over wall time), so that a pass can be held against the
+    // exponential roof at the clock the power limit left it, not only at the nominal one.
+    long long clk0 = 0;
+    uint64_t ns0 = 0;
+    if (blockIdx.x == 0 && threadIdx.x == 0) { clk0 = clock64(); ns0 = global_ns(); }
 
     if (warp == 0) {
         // ================= TMA producer =================
@@ -633,6 +638,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0 && tail->abort) atomicOr(err, CASK_ST_TIMEOUT);
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        const uint64_t ns = global_ns() - ns0;
+        const long long clk = clock64() - clk0;
+        err[2 + PASS] = ns > 0 ? (int32_t)((double)clk * 1.0e6 / (double)ns) : 0;      // kHz
+    }
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
