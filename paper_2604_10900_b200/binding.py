@@ -125,6 +125,16 @@ def lib():
     return _lib
 
 
+def use_library(path: Optional[str] = None) -> str:
+    """Loads another build of the library for every later call (contexts made before keep working only until then:
+    make new ones).  ``None`` goes back to libcask.so.  Meant for the self-checking build, libcask_bounds.so."""
+    global _lib, LIB_PATH
+    LIB_PATH = os.path.join(_HERE, "libcask.so") if path is None else path
+    _lib = None
+    lib()
+    return LIB_PATH
+
+
 class CaskError(RuntimeError):
     def __init__(self, code: int, ctx=None):
         msg = lib().cask_strerror(code).decode()
@@ -211,13 +221,14 @@ class Context:
 
     def __init__(self, device: int = 0, stream: Optional[int] = None):
         self.handle = C.c_void_p()
-        rc = lib().cask_create(C.byref(self.handle), device, stream)
+        self._lib = lib()          # a context belongs to the build of the library that made it
+        rc = self._lib.cask_create(C.byref(self.handle), device, stream)
         if rc != OK:
             raise CaskError(rc)
 
     def close(self):
         if self.handle:
-            lib().cask_destroy(self.handle)
+            self._lib.cask_destroy(self.handle)
             self.handle = C.c_void_p()
 
     def __del__(self):
@@ -227,34 +238,34 @@ class Context:
             pass
 
     def set_stream(self, stream: Optional[int]):
-        lib().cask_set_stream(self.handle, stream)
+        self._lib.cask_set_stream(self.handle, stream)
 
     @property
     def launches(self) -> int:
-        return int(lib().cask_launch_count(self.handle))
+        return int(self._lib.cask_launch_count(self.handle))
 
     def profile_enable(self, on: bool = True):
-        lib().cask_profile_enable(self.handle, int(on))
+        self._lib.cask_profile_enable(self.handle, int(on))
 
     def profile_read(self) -> Dict[str, Dict]:
         """{kernel name: {"ms": total, "launches": n}} since the last read."""
-        n = lib().cask_kernel_count()
+        n = self._lib.cask_kernel_count()
         ms = np.zeros(n, np.float32)
         cnt = np.zeros(n, np.int64)
-        rc = lib().cask_profile_read(self.handle, ms.ctypes.data, cnt.ctypes.data)
+        rc = self._lib.cask_profile_read(self.handle, ms.ctypes.data, cnt.ctypes.data)
         if rc != OK:
             raise CaskError(rc, self.handle)
-        return {lib().cask_kernel_name(i).decode(): dict(ms=float(ms[i]), launches=int(cnt[i]))
+        return {self._lib.cask_kernel_name(i).decode(): dict(ms=float(ms[i]), launches=int(cnt[i]))
                 for i in range(n) if cnt[i]}
 
     @property
     def used_tensor_path(self) -> bool:
-        return bool(lib().cask_last_score_path_tensor(self.handle))
+        return bool(self._lib.cask_last_score_path_tensor(self.handle))
 
     def score_clock_mhz(self):
         """(normaliser pass, score pass) SM clock in MHz of the last tensor-core scoring call (0: did not run)."""
         khz = (C.c_int32 * 2)(0, 0)
-        rc = lib().cask_last_score_clock_khz(self.handle, C.addressof(khz))
+        rc = self._lib.cask_last_score_clock_khz(self.handle, C.addressof(khz))
         if rc != OK:
             raise CaskError(rc, self.handle)
         return khz[0] / 1e3, khz[1] / 1e3
@@ -262,7 +273,7 @@ class Context:
     def device_flags(self) -> int:
         """CASK_ST_* bits raised on the device by the last call (waits for the stream)."""
         f = C.c_int32(0)
-        rc = lib().cask_last_device_flags(self.handle, C.byref(f))
+        rc = self._lib.cask_last_device_flags(self.handle, C.byref(f))
         if rc != OK:
             raise CaskError(rc, self.handle)
         return int(f.value)
@@ -284,7 +295,7 @@ def cask_plan_host(batch: CaskBatch, prm: CaskParams) -> np.ndarray:
 
 
 def cask_score(ctx: Context, batch, prm, s, lse_out, ws, ws_bytes: int, check: bool = True) -> int:
-    rc = lib().cask_score(ctx.handle, C.byref(batch), C.byref(prm), _ptr(s), _ptr(lse_out), _ptr(ws), ws_bytes)
+    rc = ctx._lib.cask_score(ctx.handle, C.byref(batch), C.byref(prm), _ptr(s), _ptr(lse_out), _ptr(ws), ws_bytes)
     if check:
         _check(rc, ctx)
     return rc
@@ -300,14 +311,14 @@ def make_query_stats(mu, pi, delta_grid, omega, band_layout: int = 0, delta=None
 
 
 def cask_score_stats(ctx: Context, batch, prm, stats: CaskQueryStats, s, ws, ws_bytes: int, check: bool = True) -> int:
-    rc = lib().cask_score_stats(ctx.handle, C.byref(batch), C.byref(prm), C.byref(stats), _ptr(s), _ptr(ws), ws_bytes)
+    rc = ctx._lib.cask_score_stats(ctx.handle, C.byref(batch), C.byref(prm), C.byref(stats), _ptr(s), _ptr(ws), ws_bytes)
     if check:
         _check(rc, ctx)
     return rc
 
 
 def cask_prefix_evict(ctx, batch, prm, s, kind, plan, ws, ws_bytes: int, check: bool = True) -> int:
-    rc = lib().cask_prefix_evict(ctx.handle, C.byref(batch), C.byref(prm), _ptr(s), _ptr(kind), _ptr(plan),
+    rc = ctx._lib.cask_prefix_evict(ctx.handle, C.byref(batch), C.byref(prm), _ptr(s), _ptr(kind), _ptr(plan),
                                  _ptr(ws), ws_bytes)
     if check:
         _check(rc, ctx)
@@ -315,7 +326,7 @@ def cask_prefix_evict(ctx, batch, prm, s, kind, plan, ws, ws_bytes: int, check: 
 
 
 def cask_select_core(ctx, batch, prm, s, plan, kind, ws, ws_bytes: int, check: bool = True) -> int:
-    rc = lib().cask_select_core(ctx.handle, C.byref(batch), C.byref(prm), _ptr(s), _ptr(plan), _ptr(kind),
+    rc = ctx._lib.cask_select_core(ctx.handle, C.byref(batch), C.byref(prm), _ptr(s), _ptr(plan), _ptr(kind),
                                 _ptr(ws), ws_bytes)
     if check:
         _check(rc, ctx)
@@ -324,7 +335,7 @@ def cask_select_core(ctx, batch, prm, s, plan, kind, ws, ws_bytes: int, check: b
 
 def cask_consolidate_scratch(ctx, batch, prm, s, plan, kind, seed_of, weight, sim, unit_status, lost_mass,
                              ws, ws_bytes: int, check: bool = True) -> int:
-    rc = lib().cask_consolidate_scratch(ctx.handle, C.byref(batch), C.byref(prm), _ptr(s), _ptr(plan),
+    rc = ctx._lib.cask_consolidate_scratch(ctx.handle, C.byref(batch), C.byref(prm), _ptr(s), _ptr(plan),
                                         _ptr(kind), _ptr(seed_of), _ptr(weight), _ptr(sim), _ptr(unit_status),
                                         _ptr(lost_mass), _ptr(ws), ws_bytes)
     if check:
@@ -334,7 +345,7 @@ def cask_consolidate_scratch(ctx, batch, prm, s, plan, kind, seed_of, weight, si
 
 def cask_compact(ctx, batch, prm, s, kind, seed_of, weight, out: CaskOutputs, ws, ws_bytes: int,
                  check: bool = True) -> int:
-    rc = lib().cask_compact(ctx.handle, C.byref(batch), C.byref(prm), _ptr(s), _ptr(kind), _ptr(seed_of),
+    rc = ctx._lib.cask_compact(ctx.handle, C.byref(batch), C.byref(prm), _ptr(s), _ptr(kind), _ptr(seed_of),
                             _ptr(weight), C.byref(out), _ptr(ws), ws_bytes)
     if check:
         _check(rc, ctx)
@@ -342,14 +353,14 @@ def cask_compact(ctx, batch, prm, s, kind, seed_of, weight, out: CaskOutputs, ws
 
 
 def cask_compress_event(ctx, batch, prm, out: CaskOutputs, ws, ws_bytes: int, check: bool = True) -> int:
-    rc = lib().cask_compress_event(ctx.handle, C.byref(batch), C.byref(prm), C.byref(out), _ptr(ws), ws_bytes)
+    rc = ctx._lib.cask_compress_event(ctx.handle, C.byref(batch), C.byref(prm), C.byref(out), _ptr(ws), ws_bytes)
     if check:
         _check(rc, ctx)
     return rc
 
 
 def cask_writeback_paged(ctx, batch, prm, out: CaskOutputs, k_pool, v_pool, ws, ws_bytes: int, check: bool = True) -> int:
-    rc = lib().cask_writeback_paged(ctx.handle, C.byref(batch), C.byref(prm), C.byref(out), _ptr(k_pool), _ptr(v_pool),
+    rc = ctx._lib.cask_writeback_paged(ctx.handle, C.byref(batch), C.byref(prm), C.byref(out), _ptr(k_pool), _ptr(v_pool),
                                     _ptr(ws), ws_bytes)
     if check:
         _check(rc, ctx)
@@ -362,7 +373,7 @@ def cask_host_event_device_bytes(batch, prm, Bmax: int) -> int:
 
 def cask_compress_event_host(ctx, host_batch, prm, host_out: CaskOutputs, dev_buf, dev_bytes: int,
                              check: bool = True) -> int:
-    rc = lib().cask_compress_event_host(ctx.handle, C.byref(host_batch), C.byref(prm), C.byref(host_out),
+    rc = ctx._lib.cask_compress_event_host(ctx.handle, C.byref(host_batch), C.byref(prm), C.byref(host_out),
                                         _ptr(dev_buf), dev_bytes)
     if check:
         _check(rc, ctx)
@@ -383,7 +394,7 @@ def cask_selftest_wait_timeout(ctx: Context, limit_ns: int, ws, ws_bytes: int, c
     Returns (return code, device flags, ns the waiting warp spent, ns the following warp spent)."""
     flags = C.c_int32(0)
     waited = (C.c_uint64 * 2)(0, 0)
-    rc = lib().cask_selftest_wait_timeout(ctx.handle, limit_ns, _ptr(ws), ws_bytes, C.addressof(flags), C.addressof(waited))
+    rc = ctx._lib.cask_selftest_wait_timeout(ctx.handle, limit_ns, _ptr(ws), ws_bytes, C.addressof(flags), C.addressof(waited))
     if check:
         _check(rc, ctx)
     return rc, int(flags.value), int(waited[0]), int(waited[1])
@@ -392,7 +403,7 @@ def cask_selftest_wait_timeout(ctx: Context, limit_ns: int, ws, ws_bytes: int, c
 def cask_selftest_exp_rate(ctx: Context, iters: int, ws, ws_bytes: int) -> float:
     """Exponentials per clock per SM the special-function unit sustains in the scoring epilogue's instruction mix."""
     rate = C.c_double(0.0)
-    _check(lib().cask_selftest_exp_rate(ctx.handle, iters, _ptr(ws), ws_bytes, C.addressof(rate)), ctx)
+    _check(ctx._lib.cask_selftest_exp_rate(ctx.handle, iters, _ptr(ws), ws_bytes, C.addressof(rate)), ctx)
     return float(rate.value)
 
 

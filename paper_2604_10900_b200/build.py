@@ -9,6 +9,9 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcask.so")
+# the self-checking build: the same sources with -DCASK_BOUNDS (index checks that raise CASK_ST_BOUNDS, see
+# csrc/cask_internal.cuh); a debugging aid and a test target, never loaded by default
+LIB_BOUNDS = os.path.join(HERE, "libcask_bounds.so")
 
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
@@ -20,20 +23,22 @@ def sources():
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
-def stale() -> bool:
-    if not os.path.exists(LIB):
+def stale(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + [os.path.join(HERE, "..", "include", "cask.h")]
     return any(os.path.getmtime(p) > t for p in deps)
 
 
-def build_lib(force: bool = False, verbose: bool = False) -> str:
-    if not force and not stale():
+def build_lib(force: bool = False, verbose: bool = False, bounds: bool = False) -> str:
+    LIB = LIB_BOUNDS if bounds else globals()["LIB"]
+    if not force and not stale(LIB):
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     objs = []
-    bdir = os.path.join(HERE, "_build")
+    bdir = os.path.join(HERE, "_build_bounds" if bounds else "_build")
+    NVCC_FLAGS = globals()["NVCC_FLAGS"] + (["-DCASK_BOUNDS"] if bounds else [])
     os.makedirs(bdir, exist_ok=True)
     procs = []
     for src in sources():
@@ -59,3 +64,5 @@ def build_lib(force: bool = False, verbose: bool = False) -> str:
 
 if __name__ == "__main__":
     print(build_lib(force="--force" in sys.argv, verbose=True))
+    if "--bounds" in sys.argv:
+        print(build_lib(force="--force" in sys.argv, verbose=True, bounds=True))

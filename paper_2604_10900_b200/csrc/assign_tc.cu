@@ -410,10 +410,11 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 const bool joined = cand && sm_ >= tau;
                 const unsigned long long fx = cand ? mass_to_fx(sc) : 0ull;
                 if (joined) {
+                    const int bu = CASK_IDX(best_u, m, err);
                     kind[tok_off + i] = CASK_KIND_MERGED;
-                    seed_of[tok_off + i] = seed_rows[seed_base + best_u];
-                    grp[tok_off + i] = best_u;
-                    atomicAdd(&mass_u[best_u], fx);
+                    seed_of[tok_off + i] = seed_rows[seed_base + bu];
+                    grp[tok_off + i] = bu;
+                    atomicAdd(&mass_u[bu], fx);
                 }
                 // Joiner count and lost mass go out once per warp: the fixed-point sums are exact, so
                 // the grouping of the additions does not show in the result.

@@ -199,6 +199,23 @@ __device__ __forceinline__ int64_t v_elem_off(const Shape& sh, const UnitDesc& u
     return row_elem_off(sh, ud, ud.v_off, i);
 }
 
+// Self-checking build (-DCASK_BOUNDS, libcask_bounds.so): every index the kernels take from an array that they or an
+// earlier kernel wrote (seed rows, member rows, slots, seed numbers) is checked against its range before it addresses
+// memory.  A bad one raises CASK_ST_BOUNDS in the call's flag word and is replaced by 0, so nothing is read or written
+// out of bounds and nothing traps.  The ordinary build compiles the checks out.
+#ifdef CASK_BOUNDS
+__device__ __forceinline__ int checked_index(int i, int n, int32_t* err) {
+    if ((unsigned)i >= (unsigned)n) {
+        atomicOr(err, CASK_ST_BOUNDS);
+        return 0;
+    }
+    return i;
+}
+#define CASK_IDX(i, n, err) ::cask::checked_index((i), (n), (err))
+#else
+#define CASK_IDX(i, n, err) (i)
+#endif
+
 template <typename T> struct Elem;
 template <> struct Elem<float> {
     static __device__ __forceinline__ float ld(const float* p) { return *p; }

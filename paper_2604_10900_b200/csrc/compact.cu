@@ -33,7 +33,8 @@ __global__ void __launch_bounds__(kScanThreads) slot_scan_kernel(
     float* __restrict__ weight, int Bmax, int32_t* __restrict__ n_out, int32_t* __restrict__ slot_src,
     uint8_t* __restrict__ slot_kind, float* __restrict__ slot_mass, int32_t* __restrict__ assign,
     int32_t* __restrict__ mem_row, int32_t* __restrict__ mem_slot, int32_t* __restrict__ n_mem,
-    int32_t* __restrict__ seed_slot, int32_t* __restrict__ n_seed, int max_B, FusedWeights fw) {
+    int32_t* __restrict__ seed_slot, int32_t* __restrict__ n_seed, int max_B, FusedWeights fw,
+    int32_t* __restrict__ err) {
     __shared__ unsigned wk[kScanThreads / 32], wm[kScanThreads / 32];
     __shared__ unsigned cell[kScanMaxIters * (kScanThreads / 32)];
     __shared__ int seeds_listed;
@@ -188,7 +189,7 @@ __global__ void __launch_bounds__(kScanThreads) slot_scan_kernel(
     if (threadIdx.x == 0) n_seed[u] = min(seeds_listed, max_B);
     // members point at their seed's slot
     for (int e = threadIdx.x; e < nm; e += blockDim.x) {
-        const int i = mem_row[o + e];
+        const int i = CASK_IDX(mem_row[o + e], T, err);
         int slot = -1;
         if (kind[o + i] == CASK_KIND_SEED) {
             slot = assign[o + i];
@@ -254,7 +255,7 @@ __global__ void __launch_bounds__(kCopyWarps * 32) slot_copy_kernel(
         }
         __syncwarp();
         if (lane < nv) {
-            const int src = slot_src[(size_t)u * Bmax + t0 + lane];
+            const int src = CASK_IDX(slot_src[(size_t)u * Bmax + t0 + lane], ud.T, sh.err);
             const T* kr = K + row_elem_off(sh, ud, ud.k_off, src);
             const T* vr = V + v_elem_off(sh, ud, u, src);
             const uint32_t bar = smem_u32(&ctl.bar[w][st]);
@@ -304,7 +305,7 @@ __global__ void __launch_bounds__(256) slot_merge_kernel(
     // compaction that gave up) join them.  A page id outside the pool was already met by the scoring pass.
     if (unit_status && blockIdx.x == 0 && threadIdx.x == 0 && *sh.err) unit_status[u] |= *sh.err;
     if (j >= n_seed[u]) return;
-    const int t = seed_slot[(size_t)u * max_B + j];
+    const int t = CASK_IDX(seed_slot[(size_t)u * max_B + j], Bmax, sh.err);
     const int d = sh.d;
     const int64_t o = ud.tok_off;
     constexpr int kMaxPerLane = 8;      // d <= 256
@@ -346,7 +347,7 @@ __global__ void __launch_bounds__(256) slot_merge_kernel(
                 float wi[kRows], ai[kRows];
 #pragma unroll
                 for (int q = 0; q < kRows; ++q) {
-                    const int i = my_hits[min(h0 + q, n_hits - 1)];
+                    const int i = CASK_IDX(my_hits[min(h0 + q, n_hits - 1)], ud.T, sh.err);
                     wi[q] = weight[o + i];
                     ai[q] = row_mass(sh, s, eps, o + i);
                     kv[q] = reinterpret_cast<const Vec*>(K + row_elem_off(sh, ud, ud.k_off, i))[lane];
@@ -365,7 +366,7 @@ __global__ void __launch_bounds__(256) slot_merge_kernel(
                 }
             } else {
                 for (int q = 0; q < kRows && h0 + q < n_hits; ++q) {
-                    const int i = my_hits[h0 + q];
+                    const int i = CASK_IDX(my_hits[h0 + q], ud.T, sh.err);
                     const float wq = weight[o + i];
                     msum += row_mass(sh, s, eps, o + i);
                     ++count;
@@ -435,7 +436,7 @@ __global__ void __launch_bounds__(256, 4) slot_merge_small_kernel(
     }
     __syncthreads();
     for (int e = tid; e < nm; e += blockDim.x) {
-        const int row = mem_row[o + e], t = mem_slot[o + e];
+        const int row = CASK_IDX(mem_row[o + e], ud.T, sh.err), t = mem_slot[o + e];
         const int j = (t >= 0 && t < R) ? inv[t] : -1;
         m_row[e] = row;
         m_j[e] = (int16_t)j;
@@ -617,7 +618,7 @@ cudaError_t run(const Launch& L, const cask_params& prm, const float* s, const u
                                                                     out.n_out, out.slot_src, out.slot_kind,
                                                                     out.slot_mass, out.assign, ws.mem_row,
                                                                     ws.mem_slot, ws.n_mem, ws.seed_slot, ws.n_seed,
-                                                                    ws.max_B, fw);
+                                                                    ws.max_B, fw, ws.err);
     }
     const int slots = min(out.Bmax, max(L.max_B, 1));
     {

@@ -106,7 +106,7 @@ __global__ void seed_gather_kernel(const UnitDesc* __restrict__ desc, Shape sh, 
     const UnitDesc& ud = desc[u];
     const int m = max(0, min(plan[u * 8 + CASK_PLAN_M], ud.plan[CASK_PLAN_M]));
     if (j >= m) return;
-    const int row = seed_rows[ud.seed_base + j];
+    const int row = CASK_IDX(seed_rows[ud.seed_base + j], ud.T, sh.err);
     const T* src = K + row_elem_off(sh, ud, ud.k_off, row);
     // Plain copy, or (channel-weighted similarity on the tensor cores) the weighted key w*k as two rows
     // hi + lo of the cache dtype, so that the bf16 contraction sees w*k to about 2^-17.
@@ -239,7 +239,7 @@ __global__ void __launch_bounds__(256, 6) decide_small_kernel(
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
             const int j = j0 + q * nwarps;
-            row[q] = seed_list[min(j, ms - 1)];
+            row[q] = CASK_IDX(seed_list[min(j, ms - 1)], T_, sh.err);
             const T* src = K + row_elem_off(sh, ud, ud.k_off, row[q]);
 #pragma unroll
             for (int k = 0; k < kPerLane; ++k)
@@ -387,7 +387,7 @@ __global__ void __launch_bounds__(kThreads) assign_simt_kernel(
             unsigned long long fx = mass_to_fx(row_mass(sh, s, eps, ud.tok_off + i));
             if (best_u[a] >= 0 && best[a] >= tau) {
                 kind[ud.tok_off + i] = CASK_KIND_MERGED;
-                seed_of[ud.tok_off + i] = seed_rows[ud.seed_base + best_u[a]];
+                seed_of[ud.tok_off + i] = seed_rows[ud.seed_base + CASK_IDX(best_u[a], m, sh.err)];
                 grp[ud.tok_off + i] = best_u[a];
                 atomicAdd(&mass_fx[(size_t)u * (max_m + 1) + best_u[a]], fx);
                 atomicAdd(&njoin[u], 1);
@@ -533,7 +533,7 @@ __global__ void __launch_bounds__(kThreads) assign_band_kernel(
             unsigned long long fx = mass_to_fx(row_mass(sh, s, eps, ud.tok_off + i));
             if (best_u[a] >= 0 && best[a] >= tau) {
                 kind[ud.tok_off + i] = CASK_KIND_MERGED;
-                seed_of[ud.tok_off + i] = seed_rows[ud.seed_base + best_u[a]];
+                seed_of[ud.tok_off + i] = seed_rows[ud.seed_base + CASK_IDX(best_u[a], m, sh.err)];
                 grp[ud.tok_off + i] = best_u[a];
                 atomicAdd(&mass_fx[(size_t)u * (max_m + 1) + best_u[a]], fx);
                 atomicAdd(&njoin[u], 1);
