@@ -54,7 +54,7 @@ constexpr int kMaxSms = 1024;                          // upper bound used when 
 constexpr uint32_t kPolyMaskN = 0x80808080u;
 constexpr uint32_t kPolyPairsS = 0x8080u;      // pairs of columns (of the 16 in a block of 32) on the FMA pipe
 // the same for the 8 pairs of a 16-column chunk of the streamed path (normaliser pass / score pass)
-constexpr uint32_t kPolyPairs16N = 0x88u;
+constexpr uint32_t kPolyPairs16N = 0x80u;
 constexpr uint32_t kPolyPairs16S = 0x80u;
 
 struct __align__(8) Barriers {
