@@ -43,8 +43,9 @@ struct ASmemTail {
     ABarriers bar;
     uint32_t tmem_base;
     int abort;
-    float inv_nu[kMaxGroups][2][256];   // 1/|k_seed| (0 for a zero seed): every epilogue group keeps its own
-                                        // copy, double-buffered over the units it has tiles in
+    alignas(16) float inv_nu[kMaxGroups][2][256];   // 1/|k_seed| (0 for a zero seed): every epilogue group keeps its
+                                        // own copy, double-buffered over the units it has tiles in
+    int seed_row[kMaxGroups][2][256];   // cache row of every seed of the unit, buffered the same way
     alignas(16) float w[128]; // channel weights of the similarity (1 when none are given)
     float x_val[2][2][128];   // shared buffers: best dot product / seed norm and its seed,
     int x_idx[2][2][128];     //   per buffer, per use parity, per tile row
@@ -89,29 +90,36 @@ struct TileWalk {
 // Squared (channel-weighted) norm of one staged key row as a packed pair of partial sums.  The row's sixteen
 // 16-byte pieces are read in a lane-dependent order (no bank conflicts); a bf16 is the upper half of an fp32, so
 // two integer operations unpack a pair.  The 128-byte swizzle stores logical piece p of row r at position
-// p ^ (r & 7), which matters only for finding the piece's channel weights.
+// p ^ (r & 7), which matters only for finding the piece's channel weights.  Four running sums, one per 32-bit
+// word of a piece, keep the dependent chain of packed multiply-adds at sixteen links instead of sixty-four.
+__device__ __forceinline__ uint4 lds128(uint32_t a) {
+    uint4 r;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(a));
+    return r;
+}
 template <bool WEIGHTED>
 __device__ __forceinline__ uint64_t row_norm2(const uint8_t* base, int lane, int row, const float* w) {
-    uint64_t n2p = 0ull;
+    uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
+    const uint32_t b32 = smem_u32(base);
 #pragma unroll
     for (int kb = 0; kb < 2; ++kb)
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
             const int pos = (c + lane) & 7;
-            const uint4 raw = *reinterpret_cast<const uint4*>(base + kb * kKRegionBytes + (pos << 4));
+            const uint4 raw = lds128(b32 + kb * kKRegionBytes + (pos << 4));
             const uint32_t wv[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
                 const uint64_t f2 = pack2(__uint_as_float(wv[x] << 16), __uint_as_float(wv[x] & 0xFFFF0000u));
                 if (WEIGHTED) {
                     const float2 w2 = *reinterpret_cast<const float2*>(&w[kb * 64 + ((pos ^ (row & 7)) << 3) + 2 * x]);
-                    n2p = fma2(fma2(f2, pack2(w2.x, w2.y), 0ull), f2, n2p);
+                    acc[x] = fma2(fma2(f2, pack2(w2.x, w2.y), 0ull), f2, acc[x]);
                 } else {
-                    n2p = fma2(f2, f2, n2p);
+                    acc[x] = fma2(f2, f2, acc[x]);
                 }
             }
         }
-    return n2p;
+    return add2(add2(acc[0], acc[1]), add2(acc[2], acc[3]));
 }
 
 template <int PAIR>
@@ -320,6 +328,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 continue;
             }
             float* inv = tail->inv_nu[ew >> 2][ucount & 1u];
+            int* srow = tail->seed_row[ew >> 2][ucount & 1u];
             {
                 const int gt = (ew & 3) * 32 + lane;           // thread of the group
 #pragma unroll
@@ -327,12 +336,16 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     const int c = gt + 128 * h;
                     const float nu = (c < m) ? seed_norm[seed_base + c] : 0.f;
                     inv[c] = nu > 0.f ? 1.f / nu : 0.f;
+                    srow[c] = (c < m) ? seed_rows[seed_base + c] : 0;
                 }
                 mbar_arrive(&bar.inv_ready[ew >> 2]);
                 ok = mbar_wait(&bar.inv_ready[ew >> 2], ucount & 1u, abort_flag);
                 if (!ok) break;
             }
             ++ucount;
+            uint8_t kd_n = (uint8_t)CASK_KIND_RECENT;
+            float s_n = 0.f, mi_n = 0.f;
+            bool pre = false;
             for (int t = 0; t < nt && ok; ++t, ++kit) {
                 if ((kit & buf_mask) != eg) continue;
                 const int st = kit % kStages;
@@ -356,11 +369,33 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     }
                     continue;
                 }
-                // the row's kind and score are fetched now and used after the contraction
+                // The row's kind and score are used after the contraction.  They were requested during this
+                // group's previous tile of the unit (a load issued here would still be waited for before the
+                // norm: the cache is saturated by the key stream and a miss costs well over a thousand cycles);
+                // only a group's first tile of a unit loads them directly.
                 const int i = a0 + (tile0 + t) * kTileRows + my_row;
                 const bool in_range = i >= P && i < hi;
-                const uint8_t kd = in_range ? kind[tok_off + i] : (uint8_t)CASK_KIND_RECENT;
-                const float sc = in_range ? row_mass(sh, s, eps, tok_off + i) : 0.f;     // a_i
+                uint8_t kd = (uint8_t)CASK_KIND_RECENT;
+                float s_c = 0.f, mi_c = 0.f;
+                if (pre) {
+                    kd = kd_n; s_c = s_n; mi_c = mi_n;
+                } else if (in_range) {
+                    kd = kind[tok_off + i];
+                    s_c = s[tok_off + i];
+                    if (sh.mass_in) mi_c = sh.mass_in[tok_off + i];
+                }
+                // the same fields of this group's next tile of the unit, in flight during this tile (a row's kind
+                // is read and written by the thread that owns the row only, so reading it early sees the same byte)
+                pre = t + n_bufs < nt;
+                kd_n = (uint8_t)CASK_KIND_RECENT; s_n = 0.f; mi_n = 0.f;
+                if (pre) {
+                    const int in_ = i + n_bufs * kTileRows;
+                    if (in_ >= P && in_ < hi) {
+                        kd_n = kind[tok_off + in_];
+                        s_n = s[tok_off + in_];
+                        if (sh.mass_in) mi_n = sh.mass_in[tok_off + in_];
+                    }
+                }
                 // squared norm of this thread's row, read from the staged tile (any order of the
                 // sixteen 16-byte pieces of the row gives the same set of elements)
                 ok = mbar_wait(&bar.k_full[st], (kit / kStages) & 1u, abort_flag);
@@ -408,11 +443,13 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     if (sim) sim[tok_off + i] = sm_;
                 }
                 const bool joined = cand && sm_ >= tau;
+                float sc = 0.f;                                   // a_i = score + eps (+ the mass it carries)
+                if (in_range) { const float a = s_c + eps; sc = sh.mass_in ? a + mi_c : a; }
                 const unsigned long long fx = cand ? mass_to_fx(sc) : 0ull;
                 if (joined) {
                     const int bu = CASK_IDX(best_u, m, err);
                     kind[tok_off + i] = CASK_KIND_MERGED;
-                    seed_of[tok_off + i] = seed_rows[seed_base + bu];
+                    seed_of[tok_off + i] = srow[bu];
                     grp[tok_off + i] = bu;
                     atomicAdd(&mass_u[bu], fx);
                 }
