@@ -315,6 +315,16 @@ __global__ void __launch_bounds__(256) slot_merge_kernel(
     int count = 0;
     float msum = 0.f;
     const int nm = n_mem[u];
+    // A representative nobody joined keeps the byte copy of its row: count the list entries of this slot first (the
+    // list is shared by the unit's warps and stays in cache) and leave before any row is requested.
+    {
+        int total = 0;
+        for (int e0 = 0; e0 < nm; e0 += 32) {
+            const int e = e0 + lane;
+            total += __popc(__ballot_sync(0xffffffffu, e < nm && mem_slot[o + e] == t));
+        }
+        if (total <= 1) return;
+    }
     // The member list of the unit is walked 128 entries at a time (the eight index loads of a round are independent)
     // and the round's own members are listed in shared memory in ascending order; their rows are then read four at a
     // time, so the latency of a row is paid once per four members and not once per member, and added in list order.
@@ -345,13 +355,41 @@ __global__ void __launch_bounds__(256) slot_merge_kernel(
                 struct alignas((CH > 0 ? CH : 1) * sizeof(T)) Vec { T x[CH > 0 ? CH : 1]; };
                 Vec kv[kRows], vv[kRows];
                 float wi[kRows], ai[kRows];
+                // Offsets first, loads after, uses last, with no branch in between: a branch inside the loop over the
+                // rows (paged or not, carried mass or not) makes every row wait for the one before it.
+                int64_t io[kRows], ko[kRows], vo[kRows];
+#pragma unroll
+                for (int q = 0; q < kRows; ++q)
+                    io[q] = o + CASK_IDX(my_hits[min(h0 + q, n_hits - 1)], ud.T, sh.err);
+                if (sh.page_size == 0 && !sh.v_pos) {
+#pragma unroll
+                    for (int q = 0; q < kRows; ++q) {
+                        ko[q] = ud.k_off + (io[q] - o) * sh.row_stride;
+                        vo[q] = ud.v_off + (io[q] - o) * sh.row_stride;
+                    }
+                } else {
+#pragma unroll
+                    for (int q = 0; q < kRows; ++q) {
+                        ko[q] = row_elem_off(sh, ud, ud.k_off, (int)(io[q] - o));
+                        vo[q] = v_elem_off(sh, ud, u, (int)(io[q] - o));
+                    }
+                }
 #pragma unroll
                 for (int q = 0; q < kRows; ++q) {
-                    const int i = CASK_IDX(my_hits[min(h0 + q, n_hits - 1)], ud.T, sh.err);
-                    wi[q] = weight[o + i];
-                    ai[q] = row_mass(sh, s, eps, o + i);
-                    kv[q] = reinterpret_cast<const Vec*>(K + row_elem_off(sh, ud, ud.k_off, i))[lane];
-                    vv[q] = reinterpret_cast<const Vec*>(V + v_elem_off(sh, ud, u, i))[lane];
+                    wi[q] = weight[io[q]];
+                    ai[q] = s[io[q]];
+                    kv[q] = reinterpret_cast<const Vec*>(K + ko[q])[lane];
+                    vv[q] = reinterpret_cast<const Vec*>(V + vo[q])[lane];
+                }
+                if (sh.mass_in) {
+                    float mi[kRows];
+#pragma unroll
+                    for (int q = 0; q < kRows; ++q) mi[q] = sh.mass_in[io[q]];
+#pragma unroll
+                    for (int q = 0; q < kRows; ++q) ai[q] = (ai[q] + eps) + mi[q];      // row_mass()
+                } else {
+#pragma unroll
+                    for (int q = 0; q < kRows; ++q) ai[q] += eps;
                 }
 #pragma unroll
                 for (int q = 0; q < kRows; ++q) {
@@ -489,14 +527,32 @@ __global__ void __launch_bounds__(256, 4) slot_merge_small_kernel(
         for (int h0 = 0; h0 < count; h0 += 4) {
             Vec kr[4], vr[4];
             float wi[4], ai[4];
+            int64_t ko4[4], vo4[4];       // offsets first, loads after (see slot_merge_kernel)
+            int i4[4];
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 const int e = list[first + min(h0 + q, count - 1)];
-                const int i = m_row[e];
+                i4[q] = m_row[e];
                 wi[q] = m_w[e];
                 ai[q] = m_a[e];
-                kr[q] = reinterpret_cast<const Vec*>(K + row_elem_off(sh, ud, ud.k_off, i))[lane];
-                vr[q] = reinterpret_cast<const Vec*>(V + v_elem_off(sh, ud, u, i))[lane];
+            }
+            if (sh.page_size == 0 && !sh.v_pos) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    ko4[q] = ud.k_off + (int64_t)i4[q] * sh.row_stride;
+                    vo4[q] = ud.v_off + (int64_t)i4[q] * sh.row_stride;
+                }
+            } else {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    ko4[q] = row_elem_off(sh, ud, ud.k_off, i4[q]);
+                    vo4[q] = v_elem_off(sh, ud, u, i4[q]);
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                kr[q] = reinterpret_cast<const Vec*>(K + ko4[q])[lane];
+                vr[q] = reinterpret_cast<const Vec*>(V + vo4[q])[lane];
             }
 #pragma unroll
             for (int q = 0; q < 4; ++q) {

@@ -650,12 +650,20 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 }
 
 // CTA that owns tile x when `total` tiles are split over `grid` CTAs as in TileWalk::init.
-__device__ __forceinline__ int owner_cta(long long x, long long total, long long grid) {
-    long long b = (x * grid) / total;
+template <typename I>
+__device__ __forceinline__ int owner_cta_as(I x, I total, I grid) {
+    I b = (x * grid) / total;
     while (b + 1 < grid && (total * (b + 1)) / grid <= x) ++b;
     while (b > 0 && (total * b) / grid > x) --b;
     return (int)b;
 }
+// 32-bit divisions when total * grid fits (a 64-bit division is a sequence of a hundred instructions)
+__device__ __forceinline__ int owner_cta(long long x, long long total, long long grid) {
+    if (total * grid < (1ll << 31)) return owner_cta_as<uint32_t>((uint32_t)x, (uint32_t)total, (uint32_t)grid);
+    return owner_cta_as<long long>(x, total, grid);
+}
+
+constexpr int kCombineThreads = 128;      // four rows per thread cover the 512 rows the scoring kernels accept
 
 // Folds the per-segment (reference, sum) pairs of every query row into the row offset and weight
 // used by the score pass: rowm = max reference, roww = 1/(rows * sum 2^(y - rowm)).  With
@@ -664,31 +672,74 @@ __global__ void score_tc_combine(const UnitDesc* __restrict__ desc, int rows, in
                                  const float* __restrict__ part_m, const float* __restrict__ part_l,
                                  const float* __restrict__ lse_in, float* __restrict__ rowm,
                                  float* __restrict__ roww, float* __restrict__ lse_out) {
+    // One block per unit, up to four query rows per thread (rows <= 512), every load of a round independent of the
+    // others: the kernel is a chain of cache latencies and nothing else, so it wants as many rows in flight per
+    // resident thread as it can have.  The range of CTAs that hold partials of the unit costs a few divisions: one
+    // thread finds it for the block.  The additions keep the order of the partials.
     const int u = blockIdx.x;
-    const UnitDesc& ud = desc[u];
+    __shared__ int b_range[2];
+    if (threadIdx.x == 0) {
+        const UnitDesc& ud = desc[u];
+        const int n_tiles = (ud.T + kTileKeys - 1) / kTileKeys;
+        b_range[0] = owner_cta(ud.tile0, total_tiles, grid);
+        b_range[1] = owner_cta((long long)ud.tile0 + n_tiles - 1, total_tiles, grid);
+    }
+    __syncthreads();
+    const int lo = 2 * b_range[0], hi = 2 * b_range[1] + 1;
     const float inv_rows = 1.f / (float)rows;
-    const int n_tiles = (ud.T + kTileKeys - 1) / kTileKeys;
-    const int b0 = owner_cta(ud.tile0, total_tiles, grid);
-    const int b1 = owner_cta((long long)ud.tile0 + n_tiles - 1, total_tiles, grid);
-    for (int r = threadIdx.x; r < rows; r += blockDim.x) {
-        const size_t o = (size_t)u * rows + r;
-        if (lse_in) {
-            const float lse = lse_in[o];
-            rowm[o] = lse * kLog2e;
-            roww[o] = inv_rows;
-            if (lse_out) lse_out[o] = lse;
-            continue;
+    constexpr int kR = 4;
+    const size_t ou = (size_t)u * rows;
+    if (lse_in) {
+#pragma unroll
+        for (int x = 0; x < kR; ++x) {
+            const int r = threadIdx.x + x * kCombineThreads;
+            if (r >= rows) break;
+            const float lse = lse_in[ou + r];
+            rowm[ou + r] = lse * kLog2e;
+            roww[ou + r] = inv_rows;
+            if (lse_out) lse_out[ou + r] = lse;
         }
-        float m = kNegBig;
-        for (int b = 2 * b0; b <= 2 * b1 + 1; ++b) m = fmaxf(m, part_m[((size_t)2 * u + b) * rows + r]);
-        float l = 0.f;
-        for (int b = 2 * b0; b <= 2 * b1 + 1; ++b) {
-            const size_t p = ((size_t)2 * u + b) * rows + r;
-            l += part_l[p] * exp2f(part_m[p] - m);
-        }
-        rowm[o] = m;
-        roww[o] = inv_rows / l;
-        if (lse_out) lse_out[o] = (m + log2f(l)) * kLn2;
+        return;
+    }
+    float m[kR], l[kR];
+#pragma unroll
+    for (int x = 0; x < kR; ++x) { m[x] = kNegBig; l[x] = 0.f; }
+    for (int b = lo; b <= hi; b += 2) {
+        float pm[kR][2];
+#pragma unroll
+        for (int x = 0; x < kR; ++x)
+#pragma unroll
+            for (int y = 0; y < 2; ++y) {
+                const int r = threadIdx.x + x * kCombineThreads;
+                pm[x][y] = (r < rows && b + y <= hi) ? part_m[((size_t)2 * u + b + y) * rows + r] : kNegBig;
+            }
+#pragma unroll
+        for (int x = 0; x < kR; ++x) m[x] = fmaxf(fmaxf(m[x], pm[x][0]), pm[x][1]);
+    }
+    for (int b = lo; b <= hi; b += 2) {
+        float pm[kR][2], pl[kR][2];
+#pragma unroll
+        for (int x = 0; x < kR; ++x)
+#pragma unroll
+            for (int y = 0; y < 2; ++y) {
+                const int r = min(threadIdx.x + x * kCombineThreads, rows - 1);
+                const size_t p = ((size_t)2 * u + min(b + y, hi)) * rows + r;
+                pm[x][y] = part_m[p];
+                pl[x][y] = part_l[p];
+            }
+#pragma unroll
+        for (int x = 0; x < kR; ++x)
+#pragma unroll
+            for (int y = 0; y < 2; ++y)
+                if (b + y <= hi) l[x] += pl[x][y] * exp2f(pm[x][y] - m[x]);
+    }
+#pragma unroll
+    for (int x = 0; x < kR; ++x) {
+        const int r = threadIdx.x + x * kCombineThreads;
+        if (r >= rows) break;
+        rowm[ou + r] = m[x];
+        roww[ou + r] = inv_rows / l[x];
+        if (lse_out) lse_out[ou + r] = (m[x] + log2f(l[x])) * kLn2;
     }
 }
 
@@ -766,8 +817,8 @@ cudaError_t launch_score_tc(const Launch& L, const float* lse_in, float* s, floa
     }
     {
         Timed t(L, KID_ROW_COMBINE);
-        score_tc_combine<<<sh.n_units, 128, 0, L.stream>>>(L.desc, sh.rows, L.total_tiles, grid, ws.part_m, ws.part_l,
-                                                           lse_in, ws.rowm, ws.roww, lse_out);
+        score_tc_combine<<<sh.n_units, kCombineThreads, 0, L.stream>>>(
+            L.desc, sh.rows, L.total_tiles, grid, ws.part_m, ws.part_l, lse_in, ws.rowm, ws.roww, lse_out);
     }
     {
         Timed t(L, KID_SCORE_MASS);
