@@ -227,8 +227,10 @@ int cask_last_score_clock_khz(cask_ctx* ctx, int32_t* khz_host);
  * the flag and returns.  Nothing faults and the context stays usable.  ws: DEVICE, at least 64 bytes,
  * 16-byte aligned.  Waits for the stream.  flags_host receives the device flags of the call (also
  * readable through cask_last_device_flags until the next call); waited_ns_host, optional, two words:
- * the time the waiting warp spent before it gave up, and the time a second warp of the CTA, waiting
- * with the default limit, spent before it saw the first one give up and followed it.
+ * the time the waiting warp spent before it gave up, and the time two more warps of the CTA, waiting
+ * with the default limit (one with each of the two forms of the wait the kernels use: the abort flag
+ * read after every probe, or only together with the clock), spent before they saw the first one give
+ * up and followed it: the later of the two, 0 if either did not follow.
  */
 int cask_selftest_wait_timeout(cask_ctx* ctx, uint64_t limit_ns, void* ws, size_t ws_bytes,
                                int32_t* flags_host, uint64_t* waited_ns_host);

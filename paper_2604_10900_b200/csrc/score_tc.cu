@@ -314,7 +314,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 const int nt = wk.seg_tiles();
                 for (int t = 0; t < nt && ok; ++t, ++kit) {
                     const int st = kit % kStages;
-                    ok = mbar_wait(&bar.k_empty[st], ((kit / kStages) & 1u) ^ 1u, abort_flag);
+                    ok = mbar_wait<true>(&bar.k_empty[st], ((kit / kStages) & 1u) ^ 1u, abort_flag);
                     if (!ok) break;
                     uint8_t* dst = k_smem + st * kKStageBytes;
                     const int key0 = key_begin + t * kTileKeys;
@@ -339,7 +339,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         // still works on the later blocks of the previous unit.  (The first key tile of the
                         // segment went out before, so it does not wait behind them.)
                         for (int j = 0; j < n_slots && ok; ++j) {
-                            ok = mbar_wait(&bar.q_empty[j], (seg & 1u) ^ 1u, abort_flag);
+                            ok = mbar_wait<true>(&bar.q_empty[j], (seg & 1u) ^ 1u, abort_flag);
                             if (!ok) break;
                             mbar_expect_tx(&bar.q_full[j], 2 * kQBlockBytes);
                             uint8_t* qd_ = q_smem + (j >> 1) * 2 * kQRegionBytes + (j & 1) * kQBlockBytes;
@@ -370,17 +370,17 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 const int nt = wk.seg_tiles();
                 for (int t = 0; t < nt && ok; ++t, ++kit) {
                     const int st = kit % kStages;
-                    ok = mbar_wait(&bar.k_full[st], (kit / kStages) & 1u, abort_flag);
+                    ok = mbar_wait<true>(&bar.k_full[st], (kit / kStages) & 1u, abort_flag);
                     if (!ok) break;
                     const uint32_t kst_lo = k_lo + st * (kKStageBytes >> 4);
 #pragma unroll
                     for (int jj = 0; jj < kSlots; jj += 2) {
                         const int j = jj + j0;
                         if (j >= n_slots || !ok) break;
-                        ok = mbar_wait(&bar.d_empty[j], (kit & 1u) ^ 1u, abort_flag);
+                        ok = mbar_wait<true>(&bar.d_empty[j], (kit & 1u) ^ 1u, abort_flag);
                         if (!ok) break;
                         if (t == 0) {                       // the segment's query block j has landed
-                            ok = mbar_wait(&bar.q_full[j], seg & 1u, abort_flag);
+                            ok = mbar_wait<true>(&bar.q_full[j], seg & 1u, abort_flag);
                             if (!ok) break;
                         }
                         tc_fence_after();
@@ -434,7 +434,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             bool has_next = false;
             if (PASS == 1) {
                 // The table of this segment was written during the previous one (before the loop for the first).
-                ok = mbar_wait(&bar.rw_ready, seg & 1u, abort_flag);
+                ok = mbar_wait<true>(&bar.rw_ready, seg & 1u, abort_flag);
                 if (!ok) break;
                 // Fetch the next segment's entry now; it goes into the third buffer after this segment's first
                 // tile, when the loads have long landed.  Whoever passed the wait above knows that every thread
@@ -471,7 +471,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     // behind them.
                     const uint64_t s2 = pack2(scale2, scale2);
                     float v[16];
-                    ok = mbar_wait(&bar.d_full[j0], kit & 1u, abort_flag);
+                    ok = mbar_wait<true>(&bar.d_full[j0], kit & 1u, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
                     tc_ld16(taddr + 128 * j0, v);
@@ -499,7 +499,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                             if (lane == 0) mbar_arrive(&bar.d_empty[j]);
                         }
                         if (c == 3) {
-                            ok = mbar_wait(&bar.d_full[j1], kit & 1u, abort_flag);
+                            ok = mbar_wait<true>(&bar.d_full[j1], kit & 1u, abort_flag);
                             if (!ok) break;
                             tc_fence_after();
                         }
@@ -567,7 +567,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     for (int p = 0; p < 2; ++p) {
                         const int j = p ? j1 : j0;
                         if (j >= n_slots || !ok) break;
-                        ok = mbar_wait(&bar.d_full[j], kit & 1u, abort_flag);
+                        ok = mbar_wait<true>(&bar.d_full[j], kit & 1u, abort_flag);
                         if (!ok) break;
                         tc_fence_after();
                         const int cend = p ? cend1 : cend0;
@@ -601,7 +601,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         const int64_t off = pend_off[kit & 1u];
                         if (kit >= 2) {
                             const uint32_t pk = kit - 2;
-                            ok = mbar_wait(&bar.red_full[pk & 7u], (pk >> 3) & 1u, abort_flag);
+                            ok = mbar_wait<true>(&bar.red_full[pk & 7u], (pk >> 3) & 1u, abort_flag);
                             if (!ok) break;
                             float acc = tail->red[pk & 7u][0][32 * qd + lane];
                             for (int k = 1; k < 2 * n_groups; ++k) acc += tail->red[pk & 7u][k][32 * qd + lane];
@@ -626,7 +626,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         if (PASS == 1 && ew < 4 && ok) {
             // the last two tiles of this CTA
             for (uint32_t pk = (kit >= 2 ? kit - 2 : 0); pk < kit; ++pk) {
-                if (!mbar_wait(&bar.red_full[pk & 7u], (pk >> 3) & 1u, abort_flag)) break;
+                if (!mbar_wait<true>(&bar.red_full[pk & 7u], (pk >> 3) & 1u, abort_flag)) break;
                 float acc = tail->red[pk & 7u][0][32 * qd + lane];
                 for (int k = 1; k < 2 * n_groups; ++k) acc += tail->red[pk & 7u][k][32 * qd + lane];
                 const int64_t off = pend_off[pk & 1u];

@@ -13,30 +13,36 @@ using namespace cask;
 
 namespace {
 
-__global__ void __launch_bounds__(64) wait_timeout_kernel(unsigned long long limit_ns, int32_t* __restrict__ err,
+__global__ void __launch_bounds__(96) wait_timeout_kernel(unsigned long long limit_ns, int32_t* __restrict__ err,
                                                           unsigned long long* __restrict__ waited_ns) {
     using namespace tc;
     __shared__ uint64_t bar;
     __shared__ int abort_flag;
+    __shared__ unsigned long long followed[2];
     if (threadIdx.x == 0) {
         mbar_init(&bar, 1);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    // warp 0 waits for a phase that never completes; warp 1 waits on the same barrier and leaves as soon as the
-    // first one has given up (the abort flag), the way the other roles of a kernel follow the one that timed out
+    // warp 0 waits for a phase that never completes; warps 1 and 2 wait on the same barrier with the default limit
+    // and leave as soon as the first one has given up (the abort flag), the way the other roles of a kernel follow
+    // the one that timed out: warp 1 with the form that reads the flag after every probe, warp 2 with the form that
+    // reads it with the clock only
     const unsigned long long t0 = global_ns();
     bool ok = true;
-    if ((threadIdx.x & 31) == 0)
-        ok = mbar_wait(&bar, 0u, &abort_flag, threadIdx.x == 0 ? limit_ns : kWaitLimitNs);
+    if (threadIdx.x == 0) ok = mbar_wait(&bar, 0u, &abort_flag, limit_ns);
+    if (threadIdx.x == 32) ok = mbar_wait<false>(&bar, 0u, &abort_flag);
+    if (threadIdx.x == 64) ok = mbar_wait<true>(&bar, 0u, &abort_flag);
     const unsigned long long t1 = global_ns();
+    if (threadIdx.x == 32 || threadIdx.x == 64) followed[threadIdx.x / 32 - 1] = ok ? 0ull : t1 - t0;
     __syncthreads();
     if (threadIdx.x == 0) {
         if (!ok && abort_flag) atomicOr(err, CASK_ST_TIMEOUT);
         waited_ns[0] = t1 - t0;
+        // 0 unless both followers left on the flag; else the later of the two
+        waited_ns[1] = (followed[0] && followed[1]) ? max(followed[0], followed[1]) : 0ull;
     }
-    if (threadIdx.x == 32) waited_ns[1] = ok ? 0ull : t1 - t0;
 }
 
 // Throughput of the special-function unit in the instruction mix of the scoring epilogue: per element one FFMA (the
@@ -114,7 +120,7 @@ extern "C" int cask_selftest_wait_timeout(cask_ctx* ctx, uint64_t limit_ns, void
     cudaError_t e = cudaSetDevice(device);
     if (e == cudaSuccess) e = cudaMemsetAsync(ws, 0, 64, st);
     if (e == cudaSuccess) {
-        wait_timeout_kernel<<<1, 64, 0, st>>>((unsigned long long)limit_ns, err, waited);
+        wait_timeout_kernel<<<1, 96, 0, st>>>((unsigned long long)limit_ns, err, waited);
         e = cudaGetLastError();
     }
     unsigned long long w2[2] = {0, 0};
