@@ -5,9 +5,10 @@
 // Three histogram sweeps narrow the key of the k-th greatest row digit by digit (12 + 12 + 8
 // bits), a last sweep marks everything above it and the rows equal to it.  The sweeps read the
 // unit's scores from global memory; after the first one they are L1/L2 hits.
-// Ranges of at most kSmallSpan rows skip the sweeps: their keys sit in shared memory and every
-// eligible row counts the rows ahead of it in the total order (same result, a few microseconds
-// instead of a dozen block-wide barriers).
+// Ranges of at most kSmallSpan rows skip the sweeps: their keys sit in shared memory and, up to
+// kCountSpan rows, every eligible row counts the rows ahead of it in the total order; above that
+// the (key, row) pairs are sorted by a bitonic network (same result, a few microseconds instead
+// of a dozen block-wide barriers over global memory).
 #pragma once
 #include "cask_internal.cuh"
 
@@ -21,7 +22,9 @@ constexpr int kSmallSpan = 1024;       // rows; keys and eligibility flags fit S
 // (find_digit wants nbins <= 4 * blockDim.x) and leaves room for several CTAs per SM.
 inline int select_threads(int max_rows_per_unit) { return max_rows_per_unit <= kSmallSpan ? 256 : kSelThreads; }
 
-struct SelectSmem {
+constexpr int kCountSpan = 256;        // rows; up to here every row counts the rows ahead of it, above it the rows are sorted
+
+struct alignas(16) SelectSmem {
     unsigned hist[kSelBins];
     unsigned warp_cnt[kSelThreads / 32];
     unsigned digit, krem, neq;
@@ -104,7 +107,36 @@ __device__ inline void block_topk_mark(const float* __restrict__ s, uint8_t* kin
     const int span = hi - lo;
     const int iters = (span + nthr - 1) / nthr;
 
-    if (span <= kSmallSpan) {
+    if (span > kCountSpan && span <= kSmallSpan) {
+        // ---- sorting path: (key, row) pairs in shared memory, in the total order (key descending, row ascending) by a
+        // bitonic network; counting costs span^2 comparisons, which at a thousand rows is ten times the network ----
+        unsigned long long* pk = reinterpret_cast<unsigned long long*>(sm.hist);      // [n2] <= 1024 pairs of 8 bytes
+        int n2 = 2 * kCountSpan;
+        while (n2 < span) n2 <<= 1;
+        for (int x = tid; x < n2; x += nthr) {
+            const bool el = x < span && kind[lo + x] == 0;
+            // a greater pair comes earlier: greater key, then lower row; 0 (below every eligible row) for the rest
+            pk[x] = el ? ((unsigned long long)order_key(s[lo + x]) << 32) | (unsigned)(0xFFFFFFFFu - (unsigned)x) : 0ull;
+        }
+        __syncthreads();
+        for (int k2 = 2; k2 <= n2; k2 <<= 1)
+            for (int j = k2 >> 1; j > 0; j >>= 1) {
+                for (int t = tid; t < (n2 >> 1); t += nthr) {
+                    const int i = 2 * t - (t & (j - 1)), l = i + j;
+                    const unsigned long long a = pk[i], b = pk[l];
+                    const bool desc = (i & k2) == 0;          // this run ends up descending
+                    if ((a < b) == desc) { pk[i] = b; pk[l] = a; }
+                }
+                __syncthreads();
+            }
+        for (int x = tid; x < min(k, n2); x += nthr) {
+            const unsigned long long v = pk[x];
+            if (v != 0ull) kind[lo + (int)(0xFFFFFFFFu - (unsigned)v)] = mark;
+        }
+        __syncthreads();
+        return;
+    }
+    if (span <= kCountSpan) {
         // ---- counting path: rank of every eligible row under (key descending, row ascending) ----
         unsigned* keys = sm.hist;                         // [span] rounded up to a multiple of 4
         unsigned* elig = sm.hist + kSmallSpan;            // one bit per row
@@ -257,10 +289,21 @@ __device__ inline void block_topk2_mark(const float* __restrict__ s, uint8_t* ki
     // ---- sweep 1: top 12 bits, shared by both thresholds ----
     for (int b = tid; b < kSelBins; b += nthr) sm.hist[b] = 0;
     __syncthreads();
+    // (the sweeps take four rows a round so that their loads are in flight together: a loop of one load and one
+    // shared-memory atomic per round runs at one cache latency per row)
     unsigned mine = 0;
-    for (int it = 0; it < iters; ++it) {
-        const int i = lo + it * nthr + tid;
-        if (i < hi && (ALL_OPEN || kind[i] == 0)) { atomicAdd(&sm.hist[order_key(s[i]) >> 20], 1u); ++mine; }
+    for (int it = 0; it < iters; it += 4) {
+        unsigned key[4];
+        bool el[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int i = lo + (it + q) * nthr + tid;
+            el[q] = (i < hi) && (ALL_OPEN || kind[i] == 0);
+            key[q] = el[q] ? order_key(s[i]) : 0u;
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            if (el[q]) { atomicAdd(&sm.hist[key[q] >> 20], 1u); ++mine; }
     }
     const unsigned n_elig = block_sum(mine, sm);
     if ((unsigned)(k1 + k2) >= n_elig) { __syncthreads(); plain(); return; }
@@ -280,13 +323,22 @@ __device__ inline void block_topk2_mark(const float* __restrict__ s, uint8_t* ki
         const bool same = pa == pb;
         for (int b = tid; b < nbins; b += nthr) { sm.hist[b] = 0; sm2.hist[b] = 0; }
         __syncthreads();
-        for (int it = 0; it < iters; ++it) {
-            const int i = lo + it * nthr + tid;
-            if (i < hi && (ALL_OPEN || kind[i] == 0)) {
-                const unsigned key = order_key(s[i]), pre = key >> (shift + bits), dg = (key >> shift) & (unsigned)(nbins - 1);
-                if (pre == pa) atomicAdd(&sm.hist[dg], 1u);
-                else if (pre == pb) atomicAdd(&sm2.hist[dg], 1u);
+        for (int it = 0; it < iters; it += 4) {
+            unsigned key[4];
+            bool el[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int i = lo + (it + q) * nthr + tid;
+                el[q] = (i < hi) && (ALL_OPEN || kind[i] == 0);
+                key[q] = el[q] ? order_key(s[i]) : 0u;
             }
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (el[q]) {
+                    const unsigned pre = key[q] >> (shift + bits), dg = (key[q] >> shift) & (unsigned)(nbins - 1);
+                    if (pre == pa) atomicAdd(&sm.hist[dg], 1u);
+                    else if (pre == pb) atomicAdd(&sm2.hist[dg], 1u);
+                }
         }
         __syncthreads();
         find_digit(sm, nbins, ka);
@@ -311,12 +363,23 @@ __device__ inline void block_topk2_mark(const float* __restrict__ s, uint8_t* ki
     // pa, pb: keys of the rows of rank k1 and k1 + k2; ka of the neq_a rows equal to pa fall inside the first
     // selection, kb of the neq_b rows equal to pb inside the two together
     if (ka != neq_a || kb != neq_b) { plain(); return; }      // rows tie across a boundary: index order decides
-    for (int i = lo + tid; i < hi; i += nthr)
-        if (ALL_OPEN || kind[i] == 0) {
-            const unsigned key = order_key(s[i]);
-            if (key >= pa) kind[i] = mark1;
-            else if (key >= pb) kind[i] = mark2;
+    for (int it = 0; it < iters; it += 4) {
+        unsigned key[4];
+        bool el[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int i = lo + (it + q) * nthr + tid;
+            el[q] = (i < hi) && (ALL_OPEN || kind[i] == 0);
+            key[q] = el[q] ? order_key(s[i]) : 0u;
         }
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            if (el[q]) {
+                const int i = lo + (it + q) * nthr + tid;
+                if (key[q] >= pa) kind[i] = mark1;
+                else if (key[q] >= pb) kind[i] = mark2;
+            }
+    }
     __syncthreads();
 }
 

@@ -361,6 +361,59 @@ def test_exact_duplicates_tie_at_the_selection_thresholds(decode):
     assert st["exempt_rows"] > 0 and st["cascaded"] <= hb.n_units
 
 
+@pytest.mark.parametrize("prefix,decode,budget,reserve", [
+    (200, 230, 128, 64),        # prefix eviction and scratch selection over at most 256 rows: ranking by counting
+    (700, 900, 256, 128),       # 257 .. 1,024 rows each: the sorted path
+    (1000, 1040, 384, 192),     # exactly 1,000 and 1,024 - 48 rows: the sorted path at its upper end, ragged
+    (1500, 3000, 384, 192),     # above 1,024 rows: radix select (one and two thresholds)
+])
+def test_every_selection_path_with_injected_tied_scores(prefix, decode, budget, reserve):
+    """Prefix eviction, core selection and seed selection on injected scores that take a dozen distinct values, so
+    every threshold falls inside a long run of equal keys and the row index decides: the kinds must equal the
+    oracle's on the same scores, through the staged calls, for ranges that take each of the three selection paths
+    (counting, sorting network, radix select)."""
+    import gpu_harness as gh
+    import torch
+    from oracle import cask_oracle as orc
+    w = _small("reasoning8k_b384", layers=1, kv_heads=3, group=2, window=16, prefix=prefix, decode=decode,
+               budget=budget, reserve=reserve)
+    hb = wl.make_batch(w)
+    run = gh.GpuRun(hb)
+    cb, o = run.cb, run.out
+    kf = wl.as_float32(hb.k, w.dtype)
+    rng = np.random.default_rng(prefix * 7 + decode)
+    n = int(hb.tok_off[-1])
+    s32 = (rng.integers(1, 13, n) / np.float32(16.0)).astype(np.float32)
+    s32[rng.random(n) < 0.02] += np.float32(1.0)           # a few rows clear of every tie
+    sd = s32.astype(np.float64)
+    s_dev = run.dev_f32(s32)
+    cb.cask_prefix_evict(run.ctx, run.batch, run.prm, s_dev, o["kind"], o["plan"], run.ws, run.ws_bytes)
+    cb.cask_select_core(run.ctx, run.batch, run.prm, s_dev, o["plan"], o["kind"], run.ws, run.ws_bytes)
+    torch.cuda.synchronize()
+    kind_g, plan_g = o["kind"].cpu().numpy(), o["plan"].cpu().numpy()
+    want = []
+    for u in range(hb.n_units):
+        a, T, P = int(hb.tok_off[u]), int(hb.T[u]), int(hb.P[u])
+        pl = orc.plan(T, P, int(hb.B[u]), int(hb.reserve[u]), w.window, 0.5)
+        assert np.array_equal(plan_g[u], pl)
+        kind = np.zeros(T, np.uint8)
+        orc.prefix_evict(sd[a:a + T], P, pl, kind)
+        orc.select_core(sd[a:a + T], T, P, pl, kind)
+        assert np.array_equal(kind_g[a:a + T], kind), f"unit {u}"
+        want.append(kind)
+    cb.cask_consolidate_scratch(run.ctx, run.batch, run.prm, s_dev, o["plan"], o["kind"], o["seed_of"], o["weight"],
+                                o["sim"], o["unit_status"], o["lost_mass"], run.ws, run.ws_bytes)
+    torch.cuda.synchronize()
+    kind_g2 = o["kind"].cpu().numpy()
+    for u in range(hb.n_units):
+        a, T, P = int(hb.tok_off[u]), int(hb.T[u]), int(hb.P[u])
+        kind = want[u].copy()
+        orc.consolidate(kf[a:a + T], sd[a:a + T], P, plan_g[u], kind, tau=0.9, eps=float(np.float32(1e-9)))
+        assert (kind == 4).any()
+        assert np.array_equal(kind == 4, kind_g2[a:a + T] == 4), f"unit {u}: seed rows"
+    assert run.ctx.device_flags() == 0
+
+
 @pytest.mark.parametrize("tau", [-1.0, 1.5])
 def test_tau_extremes(tau):
     """tau = -1 merges every scratch row (no lost mass); tau > 1 is plain top-k eviction."""
