@@ -98,6 +98,39 @@ __device__ __forceinline__ void find_digit(SelectSmem& sm, int nbins, unsigned k
     __syncthreads();
 }
 
+// Rows [lo,hi), at most kSmallSpan of them: among those with kind == 0 the k1 greatest get mark1 and the next k2 get
+// mark2 (k2 may be 0).  The (key, row) pairs are sorted in shared memory, in the total order (key descending, row
+// ascending), by a bitonic network: counting the rows ahead of every row costs span^2 comparisons, which at a thousand
+// rows is ten times the network.
+__device__ inline void block_sort_mark(const float* __restrict__ s, uint8_t* kind, int lo, int hi, int k1, uint8_t mark1,
+                                       int k2, uint8_t mark2, SelectSmem& sm) {
+    const int tid = threadIdx.x, nthr = blockDim.x, span = hi - lo;
+    unsigned long long* pk = reinterpret_cast<unsigned long long*>(sm.hist);      // [n2] <= 1024 pairs of 8 bytes
+    int n2 = 32;
+    while (n2 < span) n2 <<= 1;
+    for (int x = tid; x < n2; x += nthr) {
+        const bool el = x < span && kind[lo + x] == 0;
+        // a greater pair comes earlier: greater key, then lower row; 0 (below every eligible row) for the rest
+        pk[x] = el ? ((unsigned long long)order_key(s[lo + x]) << 32) | (unsigned)(0xFFFFFFFFu - (unsigned)x) : 0ull;
+    }
+    __syncthreads();
+    for (int k2b = 2; k2b <= n2; k2b <<= 1)
+        for (int j = k2b >> 1; j > 0; j >>= 1) {
+            for (int t = tid; t < (n2 >> 1); t += nthr) {
+                const int i = 2 * t - (t & (j - 1)), l = i + j;
+                const unsigned long long a = pk[i], b = pk[l];
+                const bool desc = (i & k2b) == 0;          // this run ends up descending
+                if ((a < b) == desc) { pk[i] = b; pk[l] = a; }
+            }
+            __syncthreads();
+        }
+    for (int x = tid; x < min(k1 + k2, n2); x += nthr) {
+        const unsigned long long v = pk[x];
+        if (v != 0ull) kind[lo + (int)(0xFFFFFFFFu - (unsigned)v)] = x < k1 ? mark1 : mark2;
+    }
+    __syncthreads();
+}
+
 // Among rows [lo,hi) with kind == 0, give `mark` to the k greatest.  All threads of the
 // block must call it with the same arguments.  s and kind are per-unit pointers.
 __device__ inline void block_topk_mark(const float* __restrict__ s, uint8_t* kind, int lo, int hi, int k,
@@ -107,35 +140,7 @@ __device__ inline void block_topk_mark(const float* __restrict__ s, uint8_t* kin
     const int span = hi - lo;
     const int iters = (span + nthr - 1) / nthr;
 
-    if (span > kCountSpan && span <= kSmallSpan) {
-        // ---- sorting path: (key, row) pairs in shared memory, in the total order (key descending, row ascending) by a
-        // bitonic network; counting costs span^2 comparisons, which at a thousand rows is ten times the network ----
-        unsigned long long* pk = reinterpret_cast<unsigned long long*>(sm.hist);      // [n2] <= 1024 pairs of 8 bytes
-        int n2 = 2 * kCountSpan;
-        while (n2 < span) n2 <<= 1;
-        for (int x = tid; x < n2; x += nthr) {
-            const bool el = x < span && kind[lo + x] == 0;
-            // a greater pair comes earlier: greater key, then lower row; 0 (below every eligible row) for the rest
-            pk[x] = el ? ((unsigned long long)order_key(s[lo + x]) << 32) | (unsigned)(0xFFFFFFFFu - (unsigned)x) : 0ull;
-        }
-        __syncthreads();
-        for (int k2 = 2; k2 <= n2; k2 <<= 1)
-            for (int j = k2 >> 1; j > 0; j >>= 1) {
-                for (int t = tid; t < (n2 >> 1); t += nthr) {
-                    const int i = 2 * t - (t & (j - 1)), l = i + j;
-                    const unsigned long long a = pk[i], b = pk[l];
-                    const bool desc = (i & k2) == 0;          // this run ends up descending
-                    if ((a < b) == desc) { pk[i] = b; pk[l] = a; }
-                }
-                __syncthreads();
-            }
-        for (int x = tid; x < min(k, n2); x += nthr) {
-            const unsigned long long v = pk[x];
-            if (v != 0ull) kind[lo + (int)(0xFFFFFFFFu - (unsigned)v)] = mark;
-        }
-        __syncthreads();
-        return;
-    }
+    if (span > kCountSpan && span <= kSmallSpan) { block_sort_mark(s, kind, lo, hi, k, mark, 0, mark, sm); return; }
     if (span <= kCountSpan) {
         // ---- counting path: rank of every eligible row under (key descending, row ascending) ----
         unsigned* keys = sm.hist;                         // [span] rounded up to a multiple of 4
@@ -284,6 +289,10 @@ __device__ inline void block_topk2_mark(const float* __restrict__ s, uint8_t* ki
         block_topk_mark(s, kind, lo, hi, k1, mark1, sm);
         block_topk_mark(s, kind, lo, hi, k2, mark2, sm);
     };
+    if (k1 > 0 && k2 > 0 && span > kCountSpan && span <= kSmallSpan) {      // one sort serves both selections
+        block_sort_mark(s, kind, lo, hi, k1, mark1, k2, mark2, sm);
+        return;
+    }
     if (k1 <= 0 || k2 <= 0 || span <= kSmallSpan) { plain(); return; }
     const int iters = (span + nthr - 1) / nthr;
     // ---- sweep 1: top 12 bits, shared by both thresholds ----
