@@ -107,17 +107,25 @@ __device__ __forceinline__ uint64_t ex2_poly2(uint64_t t2) {
                  __int_as_float(__float_as_int(p1) + (__float_as_int(n1) << 23)));
 }
 
+// 16 bytes of the row table by a shared-space load: through a generic pointer the same read goes the way of
+// global loads and comes back later (the score pass is 2.5 % faster this way).
+__device__ __forceinline__ float4 lds_f4(uint32_t a) {
+    float4 r;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "r"(a));
+    return r;
+}
+
 // Pass S, one block of 32 query columns (rows r0..r0+31 of the window) for the key this thread owns:
 // adds sum_r 2^(y_r*scale2 + nc[r]) over the visible rows to the two packed pairs of partial sums.
 // Pairs of columns go through packed fp32 instructions; the pairs named by kPolyPairsS take the polynomial.
 __device__ __forceinline__ void mass_block(const float (&v)[32], const float* nc, int r0, bool fast, int causal, int W,
                                            int jmin, float scale2, uint64_t& a01, uint64_t& a23) {
     if (fast) {
-        const float4* nc4 = reinterpret_cast<const float4*>(&nc[r0]);
+        const uint32_t nc32 = smem_u32(&nc[r0]);
         const uint64_t s2 = pack2(scale2, scale2);
 #pragma unroll
         for (int x = 0; x < 8; ++x) {
-            const float4 c4 = nc4[x];
+            const float4 c4 = lds_f4(nc32 + 16u * x);
             const uint64_t tA = fma2(pack2(v[4 * x], v[4 * x + 1]), s2, pack2(c4.x, c4.y));
             const uint64_t tB = fma2(pack2(v[4 * x + 2], v[4 * x + 3]), s2, pack2(c4.z, c4.w));
             float t0, t1, t2, t3;
@@ -135,12 +143,12 @@ __device__ __forceinline__ void mass_block(const float (&v)[32], const float* nc
             const int thr = causal ? jmin - r0 % W : 0;
             // arguments in packed pairs from 16-byte reads of the row table; only the exponentials of the visible
             // columns are issued (the ex2 pipe is the bottleneck), into four independent sums
-            const float4* nc4 = reinterpret_cast<const float4*>(&nc[r0]);
+            const uint32_t nc32 = smem_u32(&nc[r0]);
             const uint64_t s2 = pack2(scale2, scale2);
             float b1 = 0.f, b2 = 0.f, b3 = 0.f;
 #pragma unroll
             for (int x = 0; x < 8; ++x) {
-                const float4 c4 = nc4[x];
+                const float4 c4 = lds_f4(nc32 + 16u * x);
                 float t0, t1, t2, t3;
                 unpack2(fma2(pack2(v[4 * x], v[4 * x + 1]), s2, pack2(c4.x, c4.y)), t0, t1);
                 unpack2(fma2(pack2(v[4 * x + 2], v[4 * x + 3]), s2, pack2(c4.z, c4.w)), t2, t3);
@@ -481,10 +489,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         const int p = c >> 2, j = p ? j1 : j0, col = 16 * (c & 3);
                         uint64_t t2[8];
                         if (PASS == 1) {
-                            const float4* nc4 = reinterpret_cast<const float4*>(&rc[128 * j + 64 * ch + col]);
+                            const uint32_t nc32 = smem_u32(&rc[128 * j + 64 * ch + col]);
 #pragma unroll
                             for (int x = 0; x < 4; ++x) {
-                                const float4 c4 = nc4[x];
+                                const float4 c4 = lds_f4(nc32 + 16u * x);
                                 t2[2 * x] = fma2(pack2(v[4 * x], v[4 * x + 1]), s2, pack2(c4.x, c4.y));
                                 t2[2 * x + 1] = fma2(pack2(v[4 * x + 2], v[4 * x + 3]), s2, pack2(c4.z, c4.w));
                             }
