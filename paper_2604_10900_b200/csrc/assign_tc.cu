@@ -125,6 +125,7 @@ __device__ __forceinline__ uint64_t row_norm2(const uint8_t* base, int lane, int
 template <int PAIR>
 __device__ __forceinline__ void best_seed(uint32_t taddr, const float* inv, int c_lo, int c_hi, float& best, int& best_u) {
     constexpr int kPer = PAIR ? 16 : 32;          // seeds per block of 32 columns
+    const uint32_t inv32 = smem_u32(inv);        // full blocks read the inverse norms 16 bytes at a time, shared-space
     for (int cc = c_lo; cc < c_hi; cc += 32) {
         float v[32];
         tc_ld32(taddr + cc, v);
@@ -133,9 +134,14 @@ __device__ __forceinline__ void best_seed(uint32_t taddr, const float* inv, int 
         float bm = -INFINITY;
         if (cc + 32 <= c_hi) {
 #pragma unroll
-            for (int x = 0; x < kPer; ++x) {
-                v[x] = (PAIR ? v[2 * x] + v[2 * x + 1] : v[x]) * inv[u0 + x];
-                bm = fmaxf(bm, v[x]);
+            for (int x = 0; x < kPer; x += 4) {
+                const uint4 q = lds128(inv32 + (uint32_t)(u0 + x) * 4u);
+                const float nv[4] = {__uint_as_float(q.x), __uint_as_float(q.y), __uint_as_float(q.z), __uint_as_float(q.w)};
+#pragma unroll
+                for (int y = 0; y < 4; ++y) {
+                    v[x + y] = (PAIR ? v[2 * (x + y)] + v[2 * (x + y) + 1] : v[x + y]) * nv[y];
+                    bm = fmaxf(bm, v[x + y]);
+                }
             }
         } else {
 #pragma unroll

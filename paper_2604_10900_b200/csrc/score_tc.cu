@@ -115,6 +115,21 @@ __device__ __forceinline__ float4 lds_f4(uint32_t a) {
     return r;
 }
 
+// Sum of the n <= 4 partial key sums of one key (one per epilogue group and column half, 128 floats apart), added in
+// that order; the four reads are independent shared-space loads, so the fold costs one latency and not four.
+__device__ __forceinline__ float fold_partials(const float* p, int n) {
+    const uint32_t a = smem_u32(p);
+    float v[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v[k]) : "r"(a + 512u * (uint32_t)min(k, n - 1)));
+    float acc = v[0];
+#pragma unroll
+    for (int k = 1; k < 4; ++k)
+        if (k < n) acc += v[k];
+    return acc;
+}
+
 // Pass S, one block of 32 query columns (rows r0..r0+31 of the window) for the key this thread owns:
 // adds sum_r 2^(y_r*scale2 + nc[r]) over the visible rows to the two packed pairs of partial sums.
 // Pairs of columns go through packed fp32 instructions; the pairs named by kPolyPairsS take the polynomial.
@@ -611,8 +626,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                             const uint32_t pk = kit - 2;
                             ok = mbar_wait<true>(&bar.red_full[pk & 7u], (pk >> 3) & 1u, abort_flag);
                             if (!ok) break;
-                            float acc = tail->red[pk & 7u][0][32 * qd + lane];
-                            for (int k = 1; k < 2 * n_groups; ++k) acc += tail->red[pk & 7u][k][32 * qd + lane];
+                            const float acc = fold_partials(&tail->red[pk & 7u][0][32 * qd + lane], 2 * n_groups);
                             if (off >= 0) s[off] = acc;
                         }
                         pend_off[kit & 1u] = (my_key < T) ? tok_off + my_key : -1;
@@ -635,8 +649,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             // the last two tiles of this CTA
             for (uint32_t pk = (kit >= 2 ? kit - 2 : 0); pk < kit; ++pk) {
                 if (!mbar_wait<true>(&bar.red_full[pk & 7u], (pk >> 3) & 1u, abort_flag)) break;
-                float acc = tail->red[pk & 7u][0][32 * qd + lane];
-                for (int k = 1; k < 2 * n_groups; ++k) acc += tail->red[pk & 7u][k][32 * qd + lane];
+                const float acc = fold_partials(&tail->red[pk & 7u][0][32 * qd + lane], 2 * n_groups);
                 const int64_t off = pend_off[pk & 1u];
                 if (off >= 0) s[off] = acc;
             }
