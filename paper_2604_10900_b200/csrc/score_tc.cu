@@ -494,6 +494,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     // behind them.
                     const uint64_t s2 = pack2(scale2, scale2);
                     float v[16];
+                    float lbs[4] = {0.f, 0.f, 0.f, 0.f};      // pass N: the sums of a slot's four chunks
                     ok = mbar_wait<true>(&bar.d_full[j0], kit & 1u, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
@@ -550,33 +551,47 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                             }
                             float b0, b1;
                             unpack2(add2(b01, b23), b0, b1);
-                            float lb = b0 + b1;
-                            const bool redo = !(lb <= 65536.f);
-                            if (__any_sync(0xffffffffu, redo)) {
-                                // Some row of the warp has a column that exceeds its reference by more than 16
-                                // (or its reference is still unset).  The whole warp reads the chunk again (the
-                                // load is warp-wide; the slot is still held); the rows concerned move their
-                                // reference to the chunk maximum and redo the chunk.
-                                float w[16];
-                                tc_ld16(taddr + 128 * j + col, w);
-                                tc_wait_ld_regs(w);
-                                if (redo) {
-                                    float cm = w[0];
+                            lbs[c & 3] = b0 + b1;
+                            if (c == 3 || c == 7) {
+                                // The four chunk sums of the slot are checked together, once, before the slot is
+                                // released: a check per chunk drains the warp's exponentials eight times a tile.
+                                const bool redo = !(lbs[0] <= 65536.f) || !(lbs[1] <= 65536.f) || !(lbs[2] <= 65536.f) ||
+                                                  !(lbs[3] <= 65536.f);
+                                if (__any_sync(0xffffffffu, redo)) {
+                                    // Some row of the warp has a column that exceeds its reference by more than 16
+                                    // (or its reference is still unset).  The whole warp reads the slot's 64 columns
+                                    // again (the loads are warp-wide; the slot is still held); the rows concerned
+                                    // move their reference to the maximum of the 64 and redo the four sums.
+                                    float w[16];
+                                    float cm = kNegBig;
 #pragma unroll
-                                    for (int x = 1; x < 16; ++x) cm = fmaxf(cm, w[x]);
+                                    for (int k = 0; k < 4; ++k) {
+                                        tc_ld16(taddr + 128 * j + 16 * k, w);
+                                        tc_wait_ld_regs(w);
+#pragma unroll
+                                        for (int x = 0; x < 16; ++x) cm = fmaxf(cm, w[x]);
+                                    }
                                     cm *= scale2;
-                                    if (cm > mm[p]) {
+                                    if (redo && cm > mm[p]) {
                                         l_run[p] *= ex2(mm[p] - cm);
                                         mm[p] = cm;
                                     }
-                                    lb = 0.f;
 #pragma unroll
-                                    for (int x = 0; x < 16; ++x) lb += ex2(fmaf(w[x], scale2, -mm[p]));
+                                    for (int k = 0; k < 4; ++k) {
+                                        tc_ld16(taddr + 128 * j + 16 * k, w);
+                                        tc_wait_ld_regs(w);
+                                        if (redo) {
+                                            float lb = 0.f;
+#pragma unroll
+                                            for (int x = 0; x < 16; ++x) lb += ex2(fmaf(w[x], scale2, -mm[p]));
+                                            lbs[k] = lb;
+                                        }
+                                    }
+                                    __syncwarp();
                                 }
-                                __syncwarp();
-                            }
-                            l_run[p] += lb;
-                            if (c == 3 || c == 7) {           // the slot is no longer needed
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) l_run[p] += lbs[k];
+                                // the slot is no longer needed
                                 tc_fence_before();
                                 __syncwarp();
                                 if (lane == 0) mbar_arrive(&bar.d_empty[j]);
