@@ -39,7 +39,7 @@ UNIT = "tokens/s"
 NCU_TRAFFIC = {
     "score_norm": (268.7, "profiles/score_tc_reasoning32k_16units.txt"),
     "score_mass": (272.1, "profiles/score_tc_reasoning32k_16units.txt"),
-    "assign": (266.3, "profiles/assign_tc_reasoning32k_16units.txt"),
+    "assign": (264.7, "profiles/assign_tc_reasoning32k_16units.txt"),
 }
 
 
