@@ -11,8 +11,8 @@
 //               tiles are in flight and the global-memory round trips of a tile (row kind, score,
 //               the fixed-point mass atomics) overlap with the next tiles
 // With m <= 128 seeds in every unit the TMEM holds four buffers of 128 columns, one per group.  With more
-// seeds it holds two buffers of 256 columns and two groups share each: one takes the seed columns
-// the first columns and finishes the row, the other takes the rest and hands its best seed over through shared memory.
+// seeds it holds two buffers of 256 columns and two groups share each: one takes the first seed columns and
+// finishes the row, the other takes the rest and hands its best seed over through shared memory.
 #include "tc_common.cuh"
 
 namespace cask {
@@ -83,20 +83,18 @@ struct TileWalk {
     }
 };
 
-// Best seed among the accumulator columns [c_lo, c_hi) of this thread's row: the greatest dot * 1/|k_seed|, the
-// first seed among equals.  PAIR = 1: a seed owns two adjacent columns (the hi and lo parts of its weighted key)
-// whose sum is its dot product.  A block of 32 columns costs a multiply and a maximum per seed; the position of
-// the maximum is looked for only in a block that beats everything before it.
-// Squared (channel-weighted) norm of one staged key row as a packed pair of partial sums.  The row's sixteen
-// 16-byte pieces are read in a lane-dependent order (no bank conflicts); a bf16 is the upper half of an fp32, so
-// two integer operations unpack a pair.  The 128-byte swizzle stores logical piece p of row r at position
-// p ^ (r & 7), which matters only for finding the piece's channel weights.  Four running sums, one per 32-bit
-// word of a piece, keep the dependent chain of packed multiply-adds at sixteen links instead of sixty-four.
+// 16 bytes of shared memory by a shared-space load (through a generic pointer the read takes the path of global loads).
 __device__ __forceinline__ uint4 lds128(uint32_t a) {
     uint4 r;
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(a));
     return r;
 }
+
+// Squared (channel-weighted) norm of one staged key row as a packed pair of partial sums.  The row's sixteen
+// 16-byte pieces are read in a lane-dependent order (no bank conflicts); a bf16 is the upper half of an fp32, so
+// two integer operations unpack a pair.  The 128-byte swizzle stores logical piece p of row r at position
+// p ^ (r & 7), which matters only for finding the piece's channel weights.  Four running sums, one per 32-bit
+// word of a piece, keep the dependent chain of packed multiply-adds at sixteen links instead of sixty-four.
 template <bool WEIGHTED>
 __device__ __forceinline__ uint64_t row_norm2(const uint8_t* base, int lane, int row, const float* w) {
     uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
@@ -122,6 +120,10 @@ __device__ __forceinline__ uint64_t row_norm2(const uint8_t* base, int lane, int
     return add2(add2(acc[0], acc[1]), add2(acc[2], acc[3]));
 }
 
+// Best seed among the accumulator columns [c_lo, c_hi) of this thread's row: the greatest dot * 1/|k_seed|, the
+// first seed among equals.  PAIR = 1: a seed owns two adjacent columns (the hi and lo parts of its weighted key)
+// whose sum is its dot product.  A block of 32 columns costs a multiply and a maximum per seed; the position of
+// the maximum is looked for only in a block that beats everything before it.
 template <int PAIR>
 __device__ __forceinline__ void best_seed(uint32_t taddr, const float* inv, int c_lo, int c_hi, float& best, int& best_u) {
     constexpr int kPer = PAIR ? 16 : 32;          // seeds per block of 32 columns
