@@ -364,6 +364,7 @@ def test_exact_duplicates_tie_at_the_selection_thresholds(decode):
 @pytest.mark.parametrize("prefix,decode,budget,reserve", [
     (200, 230, 128, 64),        # prefix eviction and scratch selection over at most 256 rows: ranking by counting
     (700, 900, 256, 128),       # 257 .. 1,024 rows each: the sorted path
+    (300, 650, 256, 128),       # the same in units of at most 1,024 rows, whose selection CTAs have 256 threads
     (1000, 1040, 384, 192),     # exactly 1,000 and 1,024 - 48 rows: the sorted path at its upper end, ragged
     (1500, 3000, 384, 192),     # above 1,024 rows: radix select (one and two thresholds)
 ])
