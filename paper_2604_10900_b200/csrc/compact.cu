@@ -50,14 +50,24 @@ __global__ void __launch_bounds__(kScanThreads) slot_scan_kernel(
         // Two coalesced sweeps around one scan: per (iteration, warp) cell the number of kept rows and of group
         // members, an exclusive scan over the cells in row order, then every row finds its slot from its cell's
         // base and the lower lanes of its warp.
+        // (both sweeps read four rows' kinds a round, so that the loads are in flight together)
         const int cells = iters * nw;
-        for (int it = 0; it < iters; ++it) {
-            const int i = it * blockDim.x + threadIdx.x;
-            const uint8_t kd = (i < T) ? kind[o + i] : (uint8_t)0;
-            const bool keep = kd >= CASK_KIND_PREFIX && kd <= CASK_KIND_SEED;
-            const bool mem = kd == CASK_KIND_SEED || kd == CASK_KIND_MERGED;
-            const unsigned bk = __ballot_sync(0xffffffffu, keep), bm = __ballot_sync(0xffffffffu, mem);
-            if (lane == 0) cell[it * nw + w] = (unsigned)__popc(bk) | ((unsigned)__popc(bm) << 16);
+        for (int it0 = 0; it0 < iters; it0 += 4) {
+            uint8_t kd4[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int i = (it0 + q) * blockDim.x + threadIdx.x;
+                kd4[q] = (it0 + q < iters && i < T) ? kind[o + i] : (uint8_t)0;
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (it0 + q >= iters) break;          // uniform over the block
+                const uint8_t kd = kd4[q];
+                const bool keep = kd >= CASK_KIND_PREFIX && kd <= CASK_KIND_SEED;
+                const bool mem = kd == CASK_KIND_SEED || kd == CASK_KIND_MERGED;
+                const unsigned bk = __ballot_sync(0xffffffffu, keep), bm = __ballot_sync(0xffffffffu, mem);
+                if (lane == 0) cell[(it0 + q) * nw + w] = (unsigned)__popc(bk) | ((unsigned)__popc(bm) << 16);
+            }
         }
         __syncthreads();
         // exclusive scan of the packed (kept, member) counts; a cell holds at most 32 of each and a unit fewer
@@ -91,9 +101,19 @@ __global__ void __launch_bounds__(kScanThreads) slot_scan_kernel(
             base_m = total >> 16;
         }
         __syncthreads();
-        for (int it = 0; it < iters; ++it) {
+        for (int it0 = 0; it0 < iters; it0 += 4) {
+          uint8_t kd4[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+              const int i = (it0 + q) * blockDim.x + threadIdx.x;
+              kd4[q] = (it0 + q < iters && i < T) ? kind[o + i] : (uint8_t)0;
+          }
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int it = it0 + q;
+            if (it >= iters) break;                   // uniform over the block
             const int i = it * blockDim.x + threadIdx.x;
-            const uint8_t kd = (i < T) ? kind[o + i] : (uint8_t)0;
+            const uint8_t kd = kd4[q];
             const bool keep = kd >= CASK_KIND_PREFIX && kd <= CASK_KIND_SEED;
             const bool mem = kd == CASK_KIND_SEED || kd == CASK_KIND_MERGED;
             const unsigned bk = __ballot_sync(0xffffffffu, keep), bm = __ballot_sync(0xffffffffu, mem);
@@ -121,6 +141,7 @@ __global__ void __launch_bounds__(kScanThreads) slot_scan_kernel(
                                         fx_to_mass(fw.mass_fx[(size_t)u * (fw.max_m + 1) + gi]);
                 }
             }
+          }
         }
     } else {
     for (int i0 = 0; i0 < T; i0 += blockDim.x) {
