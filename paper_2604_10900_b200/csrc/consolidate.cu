@@ -230,23 +230,43 @@ __global__ void __launch_bounds__(256, 6) decide_small_kernel(
     unsigned n_seeds = 0;
     for (int x = 0; x < (int)(blockDim.x >> 5); ++x) n_seeds += wsum[x];
     const int ms = min((int)n_seeds, m);
-    // gather the seed keys, their norms and their own mass: one warp per seed, two seeds' rows in flight
+    // gather the seed keys, their norms and their own mass: one warp per seed, four seeds' rows in flight (offsets
+    // first, loads after, with no branch between the loads: a branch per row makes every row wait for the one before)
     const int nwarps = (int)(blockDim.x >> 5);
     constexpr int kPerLane = 4;                       // head_dim <= 128: at most four channels per lane
-    for (int j0 = w; j0 < ms; j0 += 2 * nwarps) {
-        T x[2][kPerLane];
-        int row[2];
+    constexpr int kSeedsInFlight = 4;
+    for (int j0 = w; j0 < ms; j0 += kSeedsInFlight * nwarps) {
+        T x[kSeedsInFlight][kPerLane];
+        int row[kSeedsInFlight];
+        int64_t off[kSeedsInFlight];
 #pragma unroll
-        for (int q = 0; q < 2; ++q) {
-            const int j = j0 + q * nwarps;
-            row[q] = CASK_IDX(seed_list[min(j, ms - 1)], T_, sh.err);
-            const T* src = K + row_elem_off(sh, ud, ud.k_off, row[q]);
+        for (int q = 0; q < kSeedsInFlight; ++q)
+            row[q] = CASK_IDX(seed_list[min(j0 + q * nwarps, ms - 1)], T_, sh.err);
+        if (sh.page_size == 0) {
+#pragma unroll
+            for (int q = 0; q < kSeedsInFlight; ++q) off[q] = ud.k_off + (int64_t)row[q] * sh.row_stride;
+        } else {
+#pragma unroll
+            for (int q = 0; q < kSeedsInFlight; ++q) off[q] = row_elem_off(sh, ud, ud.k_off, row[q]);
+        }
+        float am[kSeedsInFlight];
+#pragma unroll
+        for (int q = 0; q < kSeedsInFlight; ++q) {
+            const T* src = K + off[q];
 #pragma unroll
             for (int k = 0; k < kPerLane; ++k)
                 if (lane + 32 * k < sh.d) x[q][k] = src[lane + 32 * k];
+            am[q] = s[o + row[q]];
+        }
+        if (sh.mass_in) {
+#pragma unroll
+            for (int q = 0; q < kSeedsInFlight; ++q) am[q] = (am[q] + eps) + sh.mass_in[o + row[q]];     // row_mass()
+        } else {
+#pragma unroll
+            for (int q = 0; q < kSeedsInFlight; ++q) am[q] += eps;
         }
 #pragma unroll
-        for (int q = 0; q < 2; ++q) {
+        for (int q = 0; q < kSeedsInFlight; ++q) {
             const int j = j0 + q * nwarps;
             if (j >= ms) break;
             T* dst = seed_k + (size_t)(ud.seed_base + j) * (split_rows ? 2 : 1) * sh.d;
@@ -267,10 +287,10 @@ __global__ void __launch_bounds__(256, 6) decide_small_kernel(
                 n2 = fmaf(wc * f, f, n2);
             }
 #pragma unroll
-            for (int off = 16; off >= 1; off >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, off);
+            for (int off2 = 16; off2 >= 1; off2 >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, off2);
             if (lane == 0) {
                 seed_norm[ud.seed_base + j] = sqrtf(n2);
-                mass_fx[(size_t)u * (max_m + 1) + j] = mass_to_fx(row_mass(sh, s, eps, o + row[q]));
+                mass_fx[(size_t)u * (max_m + 1) + j] = mass_to_fx(am[q]);
             }
         }
     }
