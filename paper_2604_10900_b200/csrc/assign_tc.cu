@@ -26,6 +26,12 @@ constexpr int kStages = 4;
 constexpr int kEpiWarp0 = 4;
 constexpr int kMaxGroups = 4;
 constexpr int kThreadsA = (kEpiWarp0 + 4 * kMaxGroups) * 32;
+// A parity wait is only sound for a waiter that has seen the phase before the one it waits for complete: a phase
+// further behind has the same parity as the one awaited and the wait would pass at once.  Tile t uses key stage
+// t % kStages and belongs to epilogue group t % n_bufs (n_bufs = 4 or 2), so with kStages a multiple of n_bufs a group
+// meets every phase of the stages it reads, in order.  Any other ring depth lets a fast group reach a stage whose
+// previous tile (another group's) has not landed yet, pass the wait and release the stage early.
+static_assert(kStages % kMaxGroups == 0, "key ring depth must be a multiple of the epilogue group count");
 constexpr uint32_t kSeedRegionBytes = 256 * 128;       // 256 seeds x 64 bf16
 constexpr uint32_t kSeedBytes = 2 * kSeedRegionBytes;
 constexpr uint32_t kKRegionBytes = 128 * 128;
