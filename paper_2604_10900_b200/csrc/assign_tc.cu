@@ -43,6 +43,7 @@ struct __align__(8) ABarriers {
     uint64_t d_full[kMaxGroups], d_empty[kMaxGroups];
     uint64_t inv_ready[kMaxGroups];   // a group's table of inverse seed norms is written
     uint64_t x_full[2];      // shared buffers: the second group's best seed of a tile is in shared memory
+    uint64_t mma_drain;      // give-up path only: the contractions in flight have completed
 };
 
 struct ASmemTail {
@@ -203,6 +204,7 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         for (int i = 0; i < kMaxGroups; ++i) mbar_init(&bar.inv_ready[i], 128);
         mbar_init(&bar.x_full[0], 4);
         mbar_init(&bar.x_full[1], 4);
+        mbar_init(&bar.mma_drain, 1);
         tail->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -304,6 +306,12 @@ assign_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 }
                 wk.advance(nt);
                 if (ok) tc_commit(&bar.b_empty[sb]);
+            }
+            if (!ok) {
+                // contractions already issued may still be running: the TMEM they write is freed below, so give them
+                // a bounded wait (a commit completes when everything this thread issued before it has)
+                tc_commit(&bar.mma_drain);
+                for (uint32_t it = 0; it < 4096 && !mbar_try(&bar.mma_drain, 0u); ++it) {}
             }
         }
     } else if (warp >= kEpiWarp0) {

@@ -63,6 +63,7 @@ struct __align__(8) Barriers {
     uint64_t d_full[kSlots], d_empty[kSlots];
     uint64_t rw_ready;      // pass S: the row table of the segment is written
     uint64_t red_full[8];   // pass S: every warp's partial key sums of a tile are in shared memory
+    uint64_t mma_drain[2];  // give-up path only: an issuer's contractions in flight have completed
 };
 
 struct TcSmemTail {
@@ -305,6 +306,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         for (int i = 0; i < kSlots; ++i) { mbar_init(&bar.d_full[i], 1); mbar_init(&bar.d_empty[i], 8); }
         mbar_init(&bar.rw_ready, 256 * n_groups);
         for (int i = 0; i < 8; ++i) mbar_init(&bar.red_full[i], 8 * n_groups);
+        mbar_init(&bar.mma_drain[0], 1);
+        mbar_init(&bar.mma_drain[1], 1);
         tail->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -424,6 +427,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     }
                     tc_commit(&bar.k_empty[st]);
                 }
+            }
+            if (!ok) {
+                // contractions already issued may still be running: the TMEM they write is freed below, so give them
+                // a bounded wait (a commit completes when everything this thread issued before it has)
+                tc_commit(&bar.mma_drain[j0]);
+                for (uint32_t it = 0; it < 4096 && !mbar_try(&bar.mma_drain[j0], 0u); ++it) {}
             }
         }
     } else if (warp >= kEpiWarp0 && ((warp - kEpiWarp0) >> 3) < n_groups) {
