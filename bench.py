@@ -37,8 +37,8 @@ UNIT = "tokens/s"
 # DRAM bytes per cache row (dram__bytes_read.sum + dram__bytes_write.sum of one launch / rows streamed) from the
 # ncu captures summarised under profiles/; traffic grows in proportion to the rows a launch streams.
 NCU_TRAFFIC = {
-    "score_norm": (267.9, "profiles/score_tc_reasoning32k_16units.txt"),
-    "score_mass": (272.3, "profiles/score_tc_reasoning32k_16units.txt"),
+    "score_norm": (269.4, "profiles/score_tc_reasoning32k_16units.txt"),
+    "score_mass": (272.8, "profiles/score_tc_reasoning32k_16units.txt"),
     "assign": (264.4, "profiles/assign_tc_reasoning32k_16units.txt"),
 }
 

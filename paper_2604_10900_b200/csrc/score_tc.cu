@@ -489,6 +489,26 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             const int row0 = 128 * j0 + 32 * qd + lane, row1 = 128 * j1 + 32 * qd + lane;      // pass N
             const int lastvis0 = (row0 < rows) ? (sh.causal ? T - sh.W + (row0 % sh.W) : T - 1) : -1;
             const int lastvis1 = (row1 < rows) ? (sh.causal ? T - sh.W + (row1 % sh.W) : T - 1) : -1;
+            if (PASS == 0 && full_cols && nt > 0 && key_begin + kTileKeys - 1 <= last_all) {
+                // The rows have no reference at the start of a segment, and a streamed tile without one is redone
+                // whole.  Once per segment, before its first tile: wait for the tile's two slots (the waits inside
+                // the loop then pass at once), read the first chunk of each and take its maximum as the reference.
+                float w[16];
+#pragma unroll
+                for (int p = 0; p < 2; ++p) {
+                    const int j = p ? j1 : j0;
+                    ok = mbar_wait<true>(&bar.d_full[j], kit & 1u, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    tc_ld16(taddr + 128 * j, w);
+                    tc_wait_ld_regs(w);
+                    float cm = w[0];
+#pragma unroll
+                    for (int x = 1; x < 16; ++x) cm = fmaxf(cm, w[x]);
+                    mm[p] = cm * scale2;
+                }
+                if (!ok) break;
+            }
             for (int t = 0; t < nt && ok; ++t, ++kit) {
                 const int key0 = key_begin + t * kTileKeys;
                 const bool fast = key0 + kTileKeys - 1 <= last_all;
