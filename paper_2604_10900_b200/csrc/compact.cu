@@ -102,46 +102,46 @@ __global__ void __launch_bounds__(kScanThreads) slot_scan_kernel(
         }
         __syncthreads();
         for (int it0 = 0; it0 < iters; it0 += 4) {
-          uint8_t kd4[4];
+            uint8_t kd4[4];
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-              const int i = (it0 + q) * blockDim.x + threadIdx.x;
-              kd4[q] = (it0 + q < iters && i < T) ? kind[o + i] : (uint8_t)0;
-          }
+            for (int q = 0; q < 4; ++q) {
+                const int i = (it0 + q) * blockDim.x + threadIdx.x;
+                kd4[q] = (it0 + q < iters && i < T) ? kind[o + i] : (uint8_t)0;
+            }
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const int it = it0 + q;
-            if (it >= iters) break;                   // uniform over the block
-            const int i = it * blockDim.x + threadIdx.x;
-            const uint8_t kd = kd4[q];
-            const bool keep = kd >= CASK_KIND_PREFIX && kd <= CASK_KIND_SEED;
-            const bool mem = kd == CASK_KIND_SEED || kd == CASK_KIND_MERGED;
-            const unsigned bk = __ballot_sync(0xffffffffu, keep), bm = __ballot_sync(0xffffffffu, mem);
-            const unsigned cb = cell[it * nw + w];
-            const unsigned below = (1u << lane) - 1u;
-            if (i < T) {
-                int slot = -1;
-                if (keep) {
-                    slot = (int)((cb & 0xFFFFu) + __popc(bk & below));
-                    if (slot < Bmax) {
-                        slot_src[(size_t)u * Bmax + slot] = i;
-                        slot_kind[(size_t)u * Bmax + slot] = kd;
-                    } else {
-                        slot = -1;        // more kept rows than slots: cannot happen for a valid plan
+            for (int q = 0; q < 4; ++q) {
+                const int it = it0 + q;
+                if (it >= iters) break;                   // uniform over the block
+                const int i = it * blockDim.x + threadIdx.x;
+                const uint8_t kd = kd4[q];
+                const bool keep = kd >= CASK_KIND_PREFIX && kd <= CASK_KIND_SEED;
+                const bool mem = kd == CASK_KIND_SEED || kd == CASK_KIND_MERGED;
+                const unsigned bk = __ballot_sync(0xffffffffu, keep), bm = __ballot_sync(0xffffffffu, mem);
+                const unsigned cb = cell[it * nw + w];
+                const unsigned below = (1u << lane) - 1u;
+                if (i < T) {
+                    int slot = -1;
+                    if (keep) {
+                        slot = (int)((cb & 0xFFFFu) + __popc(bk & below));
+                        if (slot < Bmax) {
+                            slot_src[(size_t)u * Bmax + slot] = i;
+                            slot_kind[(size_t)u * Bmax + slot] = kd;
+                        } else {
+                            slot = -1;        // more kept rows than slots: cannot happen for a valid plan
+                        }
+                    }
+                    assign[o + i] = slot;
+                    if (mem) mem_row[o + (cb >> 16) + __popc(bm & below)] = i;
+                    if (kd >= CASK_KIND_PREFIX && kd <= CASK_KIND_CORE) weight[o + i] = 1.f;
+                    if (kd == CASK_KIND_DROPPED) weight[o + i] = 0.f;
+                    if (fw.s && mem) {
+                        const int gi = fw.grp[o + i];
+                        if (gi >= 0 && gi < fw.max_m)
+                            weight[o + i] = row_mass(fw.sh, fw.s, fw.eps, o + i) /
+                                            fx_to_mass(fw.mass_fx[(size_t)u * (fw.max_m + 1) + gi]);
                     }
                 }
-                assign[o + i] = slot;
-                if (mem) mem_row[o + (cb >> 16) + __popc(bm & below)] = i;
-                if (kd >= CASK_KIND_PREFIX && kd <= CASK_KIND_CORE) weight[o + i] = 1.f;
-                if (kd == CASK_KIND_DROPPED) weight[o + i] = 0.f;
-                if (fw.s && mem) {
-                    const int gi = fw.grp[o + i];
-                    if (gi >= 0 && gi < fw.max_m)
-                        weight[o + i] = row_mass(fw.sh, fw.s, fw.eps, o + i) /
-                                        fx_to_mass(fw.mass_fx[(size_t)u * (fw.max_m + 1) + gi]);
-                }
             }
-          }
         }
     } else {
     for (int i0 = 0; i0 < T; i0 += blockDim.x) {
